@@ -1,0 +1,133 @@
+/*
+ * ssconv: 2:4 semi-structured sparse convolution for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the inference path of "Inducing Semi-Structured Sparsity by Masking for
+ * Efficient Model Inference in Convolutional Networks": a convolution whose weight
+ * matrix carries a 2:4 mask (Sec. 3.1, Sec. 3.3), executed as an implicit GEMM on the
+ * sparse tensor cores.
+ *
+ * Conventions shared by every entry point
+ *  - All tensor pointers are DEVICE pointers owned by the caller; the library keeps
+ *    nothing between calls, allocates no device memory and never synchronises.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *    Work is enqueued on it and the call returns immediately.
+ *  - Every function returns an ssconv_status_t.  Errors the host can see (null
+ *    pointers, bad descriptor, unsupported shape, misalignment, wrong device) are
+ *    returned before anything is launched.
+ *  - Activations x, y: bf16, NHWC.  Weights: bf16 [C_out, KH, KW, C_in], read as the
+ *    row-major matrix W in R^{C_out x K}, K = KH*KW*C_in ordered (kh, kw, c_in)
+ *    (Eq. 5).  Bias: fp32 [C_out].
+ *  - Group g = ((c_out*KH + kh)*KW + kw)*(C_in/4) + q covers the 4 consecutive input
+ *    channels 4q..4q+3 of one filter tap: 4 contiguous entries of a row of W (Eq. 2,
+ *    Eq. 6).  `pattern[g]` in 0..5 names the kept pair of positions in lexicographic
+ *    order: {0,1},{0,2},{0,3},{1,2},{1,3},{2,3} (the columns of the pattern matrix D).
+ */
+#ifndef SSCONV_H_
+#define SSCONV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SSCONV_OK = 0,
+  SSCONV_ERR_NULL = 1,              /* a required pointer is NULL */
+  SSCONV_ERR_BAD_DESC = 2,          /* non-positive extent, stride or dilation; negative pad; empty output */
+  SSCONV_ERR_UNSUPPORTED_SHAPE = 3, /* shape outside what the kernels cover (see each call) */
+  SSCONV_ERR_ALIGNMENT = 4,         /* a tensor pointer is not 16-byte aligned */
+  SSCONV_ERR_WORKSPACE = 5,         /* workspace missing or too small */
+  SSCONV_ERR_ARCH = 6,              /* current device is not compute capability 10.x */
+  SSCONV_ERR_CUDA = 7,              /* a CUDA runtime/driver call or a launch failed */
+  SSCONV_ERR_TIMEOUT = 8            /* written to *dev_status by a kernel whose bounded wait ran out */
+} ssconv_status_t;
+
+typedef struct {
+  int32_t N, H, W, C_in;
+  int32_t C_out, KH, KW;
+  int32_t stride_h, stride_w;
+  int32_t pad_h, pad_w;
+  int32_t dil_h, dil_w;
+  uint32_t flags; /* SSCONV_FLAG_* */
+} ssconv_desc_t;
+
+enum { SSCONV_FLAG_BIAS = 1u, SSCONV_FLAG_RELU = 2u };
+
+enum {
+  SSCONV_MASK_LOGITS_F32 = 0,    /* scores: float [G,6], one score per pattern            */
+  SSCONV_MASK_MAGNITUDE_BF16 = 1 /* scores: bf16 weights [C_out,KH,KW,C_in] = [G,4]       */
+};
+
+/* Library version (major*10000 + minor*100 + patch). */
+int32_t ssconv_version(void);
+
+/* Static string for a status code. */
+const char* ssconv_status_string(int32_t status);
+
+/* Output extent, H_out = floor((H + 2*pad - dil*(KH-1) - 1)/stride) + 1 (same for W):
+ * the count of filter placements of Eq. 4 under zero padding (Sec. 3.3; with
+ * pad = floor(k/2), stride 1, this gives H_out*W_out = H*W as the paper states). */
+int32_t ssconv_out_shape(const ssconv_desc_t* desc, int32_t* H_out, int32_t* W_out);
+
+/* Sizes for a layer: number of groups G = C_out*K/4, bytes of the compressed value
+ * blob and of the metadata blob written by ssconv_compress, and workspace bytes the two
+ * forward calls need (may be 0).  Any output pointer may be NULL.  The blobs are padded
+ * to whole tiles, so they can be slightly larger than C_out*K and C_out*K/8 bytes. */
+int32_t ssconv_sizes(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes,
+                     size_t* meta_bytes, size_t* ws_bytes_sparse, size_t* ws_bytes_dense);
+
+/* Hard pattern choice per group (Eq. 1 of Sec. 3.1 without the one-hot: the index of the
+ * winning pattern).
+ *   mode LOGITS:    pattern[g] = argmax_i scores[g][i]; the caller has already added any
+ *                   Gumbel noise g_i to log pi_i.  Ties: lowest index.  Scores must be
+ *                   finite.
+ *   mode MAGNITUDE: pattern[g] keeps the two entries of largest |w| of the group (the
+ *                   magnitude heuristic of Sec. 2); equal magnitudes: lower position
+ *                   first; +0 and -0 are equal.
+ * scores: device, 8-byte aligned.  pattern: device uint8 [G].  G >= 0 (0 is a no-op). */
+int32_t ssconv_select_mask(int32_t mode, const void* scores, int64_t G, uint8_t* pattern,
+                           void* stream);
+
+/* Apply the mask (M .* W of Eq. 6) and pack the result in the structured form of Fig. 1:
+ * the two kept bf16 values of each group, in ascending position order, bit-exact, plus
+ * two 2-bit position indices per group, laid out in the tile order the sparse tensor-core
+ * instruction reads.  Needs C_in % 8 == 0 (else SSCONV_ERR_UNSUPPORTED_SHAPE: run such a
+ * layer through ssconv_forward_dense).  w_comp / meta: device, 16-byte aligned, of the
+ * sizes ssconv_sizes reports; every byte of both blobs is written. */
+int32_t ssconv_compress(const ssconv_desc_t* desc, const void* w_bf16, const uint8_t* pattern,
+                        void* w_comp, void* meta, void* stream);
+
+/* Inverse of ssconv_compress: w_masked [C_out,KH,KW,C_in] bf16 = M .* W with +0 in the
+ * dropped positions; pattern_out (nullable) [G] receives the pattern read back from the
+ * metadata. */
+int32_t ssconv_decompress(const ssconv_desc_t* desc, const void* w_comp, const void* meta,
+                          void* w_masked_bf16, uint8_t* pattern_out, void* stream);
+
+/* Masked convolution forward (Eq. 6 with the direct definition Eq. 4):
+ *   y[n,ho,wo,co] = act( bias[co] + sum_{kh,kw,ci} x[n, ho*s-p+kh*d, wo*s-p+kw*d, ci]
+ *                                                  * (M .* W)[co,kh,kw,ci] ),
+ * taps outside the image contribute 0, products are exact, accumulation is fp32, the
+ * result is rounded once to bf16 (nearest even).  act = ReLU if SSCONV_FLAG_RELU, bias is
+ * read only if SSCONV_FLAG_BIAS.
+ * x, y, w_comp, meta: device, 16-byte aligned.  Needs C_in % 8 == 0, C_out % 8 == 0,
+ * pad <= 127, dil*(K-1) <= 255, stride <= 8.  ws may be NULL when ssconv_sizes reports 0.
+ * dev_status (nullable): device int32; a kernel whose bounded wait expires stores
+ * SSCONV_ERR_TIMEOUT there and drains instead of hanging; it is never written on success,
+ * so the caller zeroes it once and reads it after its own synchronisation. */
+int32_t ssconv_forward(const ssconv_desc_t* desc, const void* x, const void* w_comp,
+                       const void* meta, const float* bias, void* y, void* ws, size_t ws_bytes,
+                       int32_t* dev_status, void* stream);
+
+/* Dense counterpart (Eq. 5, the unmasked reformulation): same formula with the dense
+ * weights w_bf16 [C_out,KH,KW,C_in], same tiling and pipeline, dense tensor-core
+ * instruction.  Needs C_in % 8 == 0 and C_out % 8 == 0. */
+int32_t ssconv_forward_dense(const ssconv_desc_t* desc, const void* x, const void* w_bf16,
+                             const float* bias, void* y, void* ws, size_t ws_bytes,
+                             int32_t* dev_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSCONV_H_ */

@@ -1,0 +1,160 @@
+// extern "C" boundary: argument validation and dispatch to the launchers.  Nothing here
+// touches device memory, synchronises or allocates.
+#include <cuda_runtime.h>
+
+#include "layout.cuh"
+#include "ssconv.h"
+
+namespace ssconv {
+cudaError_t launch_select(int mode, const void* scores, int64_t G, uint8_t* pattern, cudaStream_t st);
+cudaError_t launch_compress(const ssconv_desc_t& d, const void* w, const uint8_t* pattern, void* w_comp, void* meta,
+                            cudaStream_t st);
+cudaError_t launch_decompress(const ssconv_desc_t& d, const void* w_comp, const void* meta, void* w_out,
+                              uint8_t* pattern_out, cudaStream_t st);
+int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
+                              const float* bias, void* y, int32_t* dev_status, cudaStream_t stream);
+int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias, void* y,
+                             int32_t* dev_status, cudaStream_t stream);
+}  // namespace ssconv
+
+namespace {
+
+using ssconv::Geometry;
+using ssconv::make_geometry;
+
+int out_extent(int in, int k, int stride, int pad, int dil) {
+  long long span = (long long)in + 2LL * pad - (long long)dil * (k - 1) - 1;
+  return span < 0 ? 0 : (int)(span / stride + 1);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Checks every shape rule both forward kernels share; `sparse` adds the 2:4 ones.
+int32_t check_desc(const ssconv_desc_t* d, bool need_tma_shape) {
+  if (!d) return SSCONV_ERR_NULL;
+  if (d->N <= 0 || d->H <= 0 || d->W <= 0 || d->C_in <= 0 || d->C_out <= 0 || d->KH <= 0 || d->KW <= 0)
+    return SSCONV_ERR_BAD_DESC;
+  if (d->stride_h <= 0 || d->stride_w <= 0 || d->dil_h <= 0 || d->dil_w <= 0 || d->pad_h < 0 || d->pad_w < 0)
+    return SSCONV_ERR_BAD_DESC;
+  if (d->flags & ~(SSCONV_FLAG_BIAS | SSCONV_FLAG_RELU)) return SSCONV_ERR_BAD_DESC;
+  int Ho = out_extent(d->H, d->KH, d->stride_h, d->pad_h, d->dil_h);
+  int Wo = out_extent(d->W, d->KW, d->stride_w, d->pad_w, d->dil_w);
+  if (Ho <= 0 || Wo <= 0) return SSCONV_ERR_BAD_DESC;
+  if ((long long)d->N * Ho * Wo > 0x7FFFFF00LL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)d->C_out * d->KH * d->KW * d->C_in > 0x7FFFFFFFLL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if (need_tma_shape) {
+    if (d->C_in % 8 != 0 || d->C_out % 8 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+    if (d->pad_h > 127 || d->pad_w > 127) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+    if ((d->KH - 1) * d->dil_h > 255 || (d->KW - 1) * d->dil_w > 255) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+    // lower corner -pad and upper corner pad - (K-1)*dil of the filter-placement box are 8-bit fields
+    if (d->pad_h - (d->KH - 1) * d->dil_h < -128 || d->pad_w - (d->KW - 1) * d->dil_w < -128)
+      return SSCONV_ERR_UNSUPPORTED_SHAPE;
+    if (d->stride_h > 8 || d->stride_w > 8) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  }
+  return SSCONV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t ssconv_version(void) { return 100; }
+
+const char* ssconv_status_string(int32_t status) {
+  switch (status) {
+    case SSCONV_OK: return "ok";
+    case SSCONV_ERR_NULL: return "null pointer";
+    case SSCONV_ERR_BAD_DESC: return "bad descriptor";
+    case SSCONV_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case SSCONV_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+    case SSCONV_ERR_WORKSPACE: return "workspace missing or too small";
+    case SSCONV_ERR_ARCH: return "device is not sm_100";
+    case SSCONV_ERR_CUDA: return "CUDA call or launch failed";
+    case SSCONV_ERR_TIMEOUT: return "kernel wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int32_t ssconv_out_shape(const ssconv_desc_t* desc, int32_t* H_out, int32_t* W_out) {
+  if (!desc || !H_out || !W_out) return SSCONV_ERR_NULL;
+  int32_t rc = check_desc(desc, false);
+  if (rc != SSCONV_OK) return rc;
+  *H_out = out_extent(desc->H, desc->KH, desc->stride_h, desc->pad_h, desc->dil_h);
+  *W_out = out_extent(desc->W, desc->KW, desc->stride_w, desc->pad_w, desc->dil_w);
+  return SSCONV_OK;
+}
+
+int32_t ssconv_sizes(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes, size_t* meta_bytes,
+                     size_t* ws_bytes_sparse, size_t* ws_bytes_dense) {
+  int32_t rc = check_desc(desc, false);
+  if (rc != SSCONV_OK) return rc;
+  if (desc->C_in % 4 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  Geometry geo = make_geometry(*desc);
+  if (G) *G = (int64_t)desc->C_out * geo.taps * (desc->C_in / 4);
+  if (w_comp_bytes) *w_comp_bytes = (size_t)geo.Mp * geo.KC * 2;
+  if (meta_bytes) *meta_bytes = (size_t)geo.m_tiles * geo.stages * ssconv::kMetaImageBytes;
+  if (ws_bytes_sparse) *ws_bytes_sparse = 0;
+  if (ws_bytes_dense) *ws_bytes_dense = 0;
+  return SSCONV_OK;
+}
+
+int32_t ssconv_select_mask(int32_t mode, const void* scores, int64_t G, uint8_t* pattern, void* stream) {
+  if (mode != SSCONV_MASK_LOGITS_F32 && mode != SSCONV_MASK_MAGNITUDE_BF16) return SSCONV_ERR_BAD_DESC;
+  if (G < 0) return SSCONV_ERR_BAD_DESC;
+  if (G == 0) return SSCONV_OK;
+  if (!scores || !pattern) return SSCONV_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(scores) & 7u) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_select(mode, scores, G, pattern, (cudaStream_t)stream) == cudaSuccess ? SSCONV_OK
+                                                                                              : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_compress(const ssconv_desc_t* desc, const void* w_bf16, const uint8_t* pattern, void* w_comp,
+                        void* meta, void* stream) {
+  int32_t rc = check_desc(desc, false);
+  if (rc != SSCONV_OK) return rc;
+  if (desc->C_in % 8 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if (!w_bf16 || !pattern || !w_comp || !meta) return SSCONV_ERR_NULL;
+  if (!aligned16(w_bf16) || !aligned16(w_comp) || !aligned16(meta)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_compress(*desc, w_bf16, pattern, w_comp, meta, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_decompress(const ssconv_desc_t* desc, const void* w_comp, const void* meta, void* w_masked_bf16,
+                          uint8_t* pattern_out, void* stream) {
+  int32_t rc = check_desc(desc, false);
+  if (rc != SSCONV_OK) return rc;
+  if (desc->C_in % 8 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if (!w_comp || !meta || !w_masked_bf16) return SSCONV_ERR_NULL;
+  if (!aligned16(w_comp) || !aligned16(meta) || !aligned16(w_masked_bf16)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_decompress(*desc, w_comp, meta, w_masked_bf16, pattern_out, (cudaStream_t)stream) ==
+                 cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_forward(const ssconv_desc_t* desc, const void* x, const void* w_comp, const void* meta,
+                       const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
+  (void)ws;
+  (void)ws_bytes;
+  int32_t rc = check_desc(desc, true);
+  if (rc != SSCONV_OK) return rc;
+  if (!x || !w_comp || !meta || !y) return SSCONV_ERR_NULL;
+  if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
+  if (!aligned16(x) || !aligned16(w_comp) || !aligned16(meta) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_forward_sparse(*desc, x, w_comp, meta, bias, y, dev_status, (cudaStream_t)stream);
+}
+
+int32_t ssconv_forward_dense(const ssconv_desc_t* desc, const void* x, const void* w_bf16, const float* bias,
+                             void* y, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
+  (void)ws;
+  (void)ws_bytes;
+  int32_t rc = check_desc(desc, true);
+  if (rc != SSCONV_OK) return rc;
+  if (!x || !w_bf16 || !y) return SSCONV_ERR_NULL;
+  if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
+  if (!aligned16(x) || !aligned16(w_bf16) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_forward_dense(*desc, x, w_bf16, bias, y, dev_status, (cudaStream_t)stream);
+}
+
+}  // extern "C"

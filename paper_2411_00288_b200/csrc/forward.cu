@@ -1,0 +1,419 @@
+// Masked (2:4 sparse) and dense NHWC bf16 convolution forward as an implicit GEMM on the
+// sm_100a tensor cores (Eq. 5 / Eq. 6 of the paper; the unfold U(X) is never materialised).
+//
+//   D[C_out x P] = A[C_out x K] * B[K x P],   P = N*H_out*W_out pixels, K = KH*KW*C_in
+//
+// A = weights (the only operand tcgen05.mma.sp accepts in 2:4 form), B = activations.  A CTA
+// owns a 128 (output channels) x 128 (pixels) tile of D at a time and walks a static list of
+// tiles (persistent kernel).  Warp roles:
+//   warp 0      TMA producer: per stage one weight tile, one or two im2col activation tiles
+//               (64 channels x 128 pixels at one filter tap, zero-filled outside the image),
+//               and for the sparse kernel the 2 KB metadata image.
+//   warp 1      owns TMEM; one thread copies metadata smem->TMEM and issues the MMAs into one of
+//               two fp32 accumulators (128 lanes x 128 columns each).
+//   warps 2-5   epilogue: TMEM -> registers, + bias, ReLU, bf16, transpose through shared
+//               memory to pixel-major rows, one TMA store per tile (clipped at the tensor edge).
+// All mbarrier waits are bounded; when one runs out the CTA raises a flag, every role leaves
+// its loop, TMEM is freed and SSCONV_ERR_TIMEOUT is stored to *dev_status.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "layout.cuh"
+#include "sm100_ptx.cuh"
+#include "ssconv.h"
+
+namespace ssconv {
+
+constexpr int kBN = 128;                 // pixels per tile (N of the MMA)
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kMetaCol = 2 * kBN;   // first TMEM column of the metadata (2 slots x 4 columns)
+constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 1.9 GHz
+constexpr uint32_t kATileBytes = 128 * 128;          // 128 rows x 128 B
+constexpr uint32_t kBTileBytes = kBN * 128;          // 128 pixels x 64 channels bf16
+constexpr uint32_t kOutStageBytes = kBN * 256;       // 128 pixels x 128 channels bf16
+
+template <bool SPARSE>
+struct Cfg {
+  static constexpr int kBlocksPerStage = SPARSE ? 2 : 1;
+  static constexpr int kStages = SPARSE ? 3 : 5;
+  static constexpr uint32_t kMetaBytes = SPARSE ? (uint32_t)kMetaImageBytes : 0u;
+  static constexpr uint32_t kStageBytes = kATileBytes + kBlocksPerStage * kBTileBytes + kMetaBytes;
+  static constexpr uint32_t kBarrierBytes = 256;
+  static constexpr uint32_t kSmemBytes = kStages * kStageBytes + kOutStageBytes + kBarrierBytes + 1024;
+};
+
+struct FwdParams {
+  int C_in, C_out, P, HoWo, Wo;
+  int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
+  int cblocks, kblocks;
+  int m_tiles, num_tiles;
+  int iters;  // pipeline stages per tile
+  uint32_t flags;
+  const float* bias;
+  const uint8_t* meta;
+  int32_t* dev_status;
+};
+
+__device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+template <bool SPARSE>
+__global__ void __launch_bounds__(kThreads, 1)
+ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                  const __grid_constant__ CUtensorMap tm_y, const FwdParams p) {
+  using C = Cfg<SPARSE>;
+  constexpr int STAGES = C::kStages;
+  constexpr int KBS = C::kBlocksPerStage;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* out_stage = smem + STAGES * C::kStageBytes;
+  uint64_t* bar_full = reinterpret_cast<uint64_t*>(out_stage + kOutStageBytes);
+  uint64_t* bar_empty = bar_full + STAGES;
+  uint64_t* bar_acc_full = bar_empty + STAGES;
+  uint64_t* bar_acc_empty = bar_acc_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* epi_go = abort_flag + 1;  // two slots: the epilogue leader's go/stop verdict per tile
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&bar_full[s], 1);
+      mbar_init(&bar_empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&bar_acc_full[b], 1);
+      mbar_init(&bar_acc_empty[b], 4);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t g = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+        const int m = tile % p.m_tiles;
+        const int p0 = (tile / p.m_tiles) * kBN;
+        const int n0 = p0 / p.HoWo;
+        const int rem = p0 - n0 * p.HoWo;
+        const int ho0 = rem / p.Wo;
+        const int wo0 = rem - ho0 * p.Wo;
+        const int base_w = wo0 * p.stride_w - p.pad_w;
+        const int base_h = ho0 * p.stride_h - p.pad_h;
+        for (int it = 0; it < p.iters; ++it, ++g) {
+          const int s = g % STAGES;
+          const uint32_t ph = (g / STAGES) & 1u;
+          if (!mbar_wait_bounded(&bar_empty[s], ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+          uint8_t* st = smem + s * C::kStageBytes;
+          int nb = p.kblocks - KBS * it;
+          if (nb > KBS) nb = KBS;
+          mbar_expect_tx(&bar_full[s], kATileBytes + nb * kBTileBytes + C::kMetaBytes);
+          if (SPARSE) {
+            tma_load_2d(st, &tm_a, &bar_full[s], it * 64, m * kTileM);
+          } else {
+            tma_load_3d(st, &tm_a, &bar_full[s], (it % p.cblocks) * kBlockK, it / p.cblocks, m * kTileM);
+          }
+          for (int j = 0; j < nb; ++j) {
+            const int b = KBS * it + j;
+            const int tap = b / p.cblocks;
+            const int cc = b - tap * p.cblocks;
+            const int kh = tap / p.KW;
+            const int kw = tap - kh * p.KW;
+            tma_load_im2col_4d(st + kATileBytes + j * kBTileBytes, &tm_b, &bar_full[s], cc * kBlockK, base_w, base_h,
+                               n0, (uint16_t)(kw * p.dil_w), (uint16_t)(kh * p.dil_h));
+          }
+          if (SPARSE) {
+            bulk_load(st + kATileBytes + KBS * kBTileBytes, p.meta + ((size_t)m * p.iters + it) * kMetaImageBytes,
+                      kMetaImageBytes, &bar_full[s]);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(kTileM, kBN, SPARSE);
+      uint32_t g = 0;
+      uint32_t tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x, ++tcount) {
+        const uint32_t buf = tcount & 1u;
+        const uint32_t aph = (tcount >> 1) & 1u;
+        if (!mbar_wait_bounded(&bar_acc_empty[buf], aph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * kBN;
+        uint32_t accumulate = 0;
+        for (int it = 0; it < p.iters; ++it, ++g) {
+          const int s = g % STAGES;
+          const uint32_t ph = (g / STAGES) & 1u;
+          if (!mbar_wait_bounded(&bar_full[s], ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t st = smem_u32(smem + s * C::kStageBytes);
+          const uint64_t a_desc = smem_desc_sw128(st);
+          int nb = p.kblocks - KBS * it;
+          if (nb > KBS) nb = KBS;
+          if (SPARSE) {
+            // two metadata slots of 4 columns, alternating per stage
+            const uint32_t meta_tmem = tmem_base + kMetaCol + 4u * (g & 1u);
+            tc_cp_128x128b(meta_tmem, smem_desc_noswizzle(st + kATileBytes + KBS * kBTileBytes, 16, 128));
+            for (int j = 0; j < nb; ++j) {
+              const int b = KBS * it + j;
+              const int cc = b % p.cblocks;
+              int vc = p.C_in - cc * kBlockK;
+              if (vc > kBlockK) vc = kBlockK;
+              const int n_mma = (vc + 31) >> 5;  // 32 dense columns per sparse MMA
+              const uint64_t b_desc = smem_desc_sw128(st + kATileBytes + j * kBTileBytes);
+              for (int k2 = 0; k2 < n_mma; ++k2) {
+                const uint32_t kk = 2 * j + k2;  // MMA slot within the stage (= metadata column)
+                // A advances 16 kept values = 32 B, B advances 32 channels = 64 B (descriptor units of 16 B)
+                tc_mma_sparse(d_tmem, a_desc + 2 * kk, b_desc + 4 * k2, meta_tmem + (kk & ~1u), idesc | (kk & 1u),
+                              accumulate);
+                accumulate = 1;
+              }
+            }
+          } else {
+            const int cc = it % p.cblocks;
+            int vc = p.C_in - cc * kBlockK;
+            if (vc > kBlockK) vc = kBlockK;
+            const int n_mma = (vc + 15) >> 4;  // 16 columns per dense MMA
+            const uint64_t b_desc = smem_desc_sw128(st + kATileBytes);
+            for (int kk = 0; kk < n_mma; ++kk) {
+              tc_mma_dense(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, accumulate);
+              accumulate = 1;
+            }
+          }
+          tc_commit(&bar_empty[s]);
+        }
+        if (ok) tc_commit(&bar_acc_full[buf]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int q = warp & 3;  // TMEM lane quadrant this warp may read
+    const int row = q * 32 + lane;
+    const bool leader = (warp == 2 && lane == 0);
+    uint32_t tcount = 0;
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++tcount) {
+      const int m = tile % p.m_tiles;
+      const int p0 = (tile / p.m_tiles) * kBN;
+      const uint32_t buf = tcount & 1u;
+      const uint32_t aph = (tcount >> 1) & 1u;
+      const bool got = mbar_wait_bounded(&bar_acc_full[buf], aph, abort_flag, kWaitLimitCycles);
+      // All 128 epilogue threads must take the same branch (they meet at named barriers below):
+      // the leader publishes one verdict, everybody reads it after the barrier.
+      if (leader) {
+        epi_go[tcount & 1u] = (got && *abort_flag == 0) ? 1 : 0;
+        bulk_wait_group_read0();  // the previous tile's TMA store has finished reading the staging buffer
+      }
+      epilogue_bar_sync();
+      if (epi_go[tcount & 1u] == 0) break;
+      tc_fence_after();
+      const int co = m * kTileM + row;
+      const float bias_v = ((p.flags & SSCONV_FLAG_BIAS) && co < p.C_out) ? p.bias[co] : 0.0f;
+      const bool relu = (p.flags & SSCONV_FLAG_RELU) != 0;
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kBN;
+      uint16_t* stage_col = reinterpret_cast<uint16_t*>(out_stage) + row;
+#pragma unroll 1
+      for (int c0 = 0; c0 < kBN; c0 += 32) {
+        uint32_t r[32];
+        tc_ld_32x32(t_row + c0, r);
+        tc_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          float v = __uint_as_float(r[j]) + bias_v;
+          if (relu) v = fmaxf(v, 0.0f);
+          stage_col[(c0 + j) * 128] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
+      fence_proxy_async_smem();
+      epilogue_bar_sync();
+      if (leader) {
+        tma_store_2d(&tm_y, out_stage, m * kTileM, p0);
+        bulk_commit_group();
+      }
+    }
+    if (leader) bulk_wait_group0();
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag != 0) {
+    // give copies and MMAs still in flight time to land before shared memory and TMEM go away
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    if (threadIdx.x == 0 && p.dev_status != nullptr) atomicExch(p.dev_status, (int)SSCONV_ERR_TIMEOUT);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn g_encode_tiled = nullptr;
+static EncodeIm2colFn g_encode_im2col = nullptr;
+
+static bool load_driver_entry_points() {
+  if (g_encode_tiled && g_encode_im2col) return true;
+  void* f1 = nullptr;
+  void* f2 = nullptr;
+  cudaDriverEntryPointQueryResult q1, q2;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f1, cudaEnableDefault, &q1) != cudaSuccess) return false;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f2, cudaEnableDefault, &q2) != cudaSuccess) return false;
+  if (q1 != cudaDriverEntryPointSuccess || q2 != cudaDriverEntryPointSuccess || !f1 || !f2) return false;
+  g_encode_tiled = reinterpret_cast<EncodeTiledFn>(f1);
+  g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(f2);
+  return true;
+}
+
+static int out_extent(int in, int k, int stride, int pad, int dil) {
+  int span = in + 2 * pad - dil * (k - 1) - 1;
+  return span < 0 ? 0 : span / stride + 1;
+}
+
+static int g_sm_count[64] = {0};
+static bool g_attr_set[64][2] = {{false}};
+
+template <bool SPARSE>
+static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const void* weights, const void* meta,
+                                   const float* bias, void* y, int32_t* dev_status, cudaStream_t stream) {
+  if (!load_driver_entry_points()) return SSCONV_ERR_CUDA;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SSCONV_ERR_CUDA;
+  if (g_sm_count[dev] == 0) {
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SSCONV_ERR_CUDA;
+    if (major != 10) return SSCONV_ERR_ARCH;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+      return SSCONV_ERR_CUDA;
+    g_sm_count[dev] = sms;
+  }
+  using C = Cfg<SPARSE>;
+  if (!g_attr_set[dev][SPARSE ? 1 : 0]) {
+    if (cudaFuncSetAttribute(ssconv_fwd_kernel<SPARSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)C::kSmemBytes) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
+    g_attr_set[dev][SPARSE ? 1 : 0] = true;
+  }
+
+  const Geometry geo = make_geometry(d);
+  const int Ho = out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h);
+  const int Wo = out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
+  const long long P = (long long)d.N * Ho * Wo;
+
+  CUtensorMap tm_a, tm_b, tm_y;
+  // activations: NHWC seen as (c, w, h, n), im2col mode; base pixels range over the filter
+  // placements, elements outside the image read as zero (= the zero padding of Eq. 4)
+  {
+    cuuint64_t dims[4] = {(cuuint64_t)d.C_in, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
+    cuuint64_t strides[3] = {(cuuint64_t)d.C_in * 2, (cuuint64_t)d.W * d.C_in * 2,
+                             (cuuint64_t)d.H * d.W * d.C_in * 2};
+    int lower[2] = {-d.pad_w, -d.pad_h};
+    int upper[2] = {d.pad_w - (d.KW - 1) * d.dil_w, d.pad_h - (d.KH - 1) * d.dil_h};
+    cuuint32_t estr[4] = {1, (cuuint32_t)d.stride_w, (cuuint32_t)d.stride_h, 1};
+    CUresult r = g_encode_im2col(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), dims, strides,
+                                 lower, upper, (cuuint32_t)kBlockK, (cuuint32_t)kBN, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
+  }
+  if (SPARSE) {
+    cuuint64_t dims[2] = {(cuuint64_t)geo.KC, (cuuint64_t)geo.Mp};
+    cuuint64_t strides[1] = {(cuuint64_t)geo.KC * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kTileM};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode_tiled(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(weights), dims, strides,
+                                box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
+  } else {
+    cuuint64_t dims[3] = {(cuuint64_t)d.C_in, (cuuint64_t)geo.taps, (cuuint64_t)d.C_out};
+    cuuint64_t strides[2] = {(cuuint64_t)d.C_in * 2, (cuuint64_t)geo.taps * d.C_in * 2};
+    cuuint32_t box[3] = {(cuuint32_t)kBlockK, 1, (cuuint32_t)kTileM};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode_tiled(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(weights), dims, strides,
+                                box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
+  }
+  {
+    cuuint64_t dims[2] = {(cuuint64_t)d.C_out, (cuuint64_t)P};
+    cuuint64_t strides[1] = {(cuuint64_t)d.C_out * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kTileM, (cuuint32_t)kBN};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode_tiled(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
+  }
+
+  FwdParams p;
+  p.C_in = d.C_in;
+  p.C_out = d.C_out;
+  p.P = (int)P;
+  p.HoWo = Ho * Wo;
+  p.Wo = Wo;
+  p.stride_h = d.stride_h;
+  p.stride_w = d.stride_w;
+  p.pad_h = d.pad_h;
+  p.pad_w = d.pad_w;
+  p.dil_h = d.dil_h;
+  p.dil_w = d.dil_w;
+  p.KW = d.KW;
+  p.cblocks = geo.cblocks;
+  p.kblocks = geo.kblocks;
+  p.m_tiles = geo.m_tiles;
+  const long long p_tiles = (P + kBN - 1) / kBN;
+  p.num_tiles = (int)(p_tiles * geo.m_tiles);
+  p.iters = SPARSE ? geo.stages : geo.kblocks;
+  p.flags = d.flags;
+  p.bias = bias;
+  p.meta = static_cast<const uint8_t*>(meta);
+  p.dev_status = dev_status;
+
+  int grid = p.num_tiles < g_sm_count[dev] ? p.num_tiles : g_sm_count[dev];
+  ssconv_fwd_kernel<SPARSE><<<grid, kThreads, C::kSmemBytes, stream>>>(tm_a, tm_b, tm_y, p);
+  return cudaGetLastError() == cudaSuccess ? SSCONV_OK : SSCONV_ERR_CUDA;
+}
+
+int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
+                              const float* bias, void* y, int32_t* dev_status, cudaStream_t stream) {
+  return launch_forward_impl<true>(d, x, w_comp, meta, bias, y, dev_status, stream);
+}
+int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias, void* y,
+                             int32_t* dev_status, cudaStream_t stream) {
+  return launch_forward_impl<false>(d, x, w, nullptr, bias, y, dev_status, stream);
+}
+
+}  // namespace ssconv

@@ -1,0 +1,74 @@
+// Geometry of the compressed 2:4 operand as the forward kernel consumes it.
+//
+// The weight matrix W [C_out x K], K ordered (kh, kw, c_in), is cut along K into "k-blocks"
+// of 64 dense columns that never straddle a filter tap: each tap contributes
+// ceil(C_in/64) k-blocks, the last of which may be partly (or, after rounding the block
+// count up to even, wholly) padding.  Two consecutive k-blocks form one pipeline stage of
+// the sparse kernel (128 dense columns = 64 kept values per row).
+//
+// Value blob:    bf16 [Mp][KC], Mp = C_out rounded up to 128, KC = 32 * n_kblocks_padded.
+//                Column 32*b + 2*q + s holds kept value s (0 = lower position) of the q-th
+//                group of k-block b; padding is +0.
+// Metadata blob: [Mp/128][n_stages] images of 2048 bytes.  An image is what one
+//                tcgen05.cp 128x128b moves into 4 TMEM columns: 128 lanes x 4 words.
+//                Word j of lane L belongs to the j-th sparse MMA of the stage (32 dense
+//                columns each): its low half describes row (L%8) + 16*(L/16), its high half
+//                that row + 8, both for the 16 dense columns starting at 32*j + 16*((L/8)%2):
+//                four 4-bit codes, lowest group in the lowest nibble, code = pos0 | pos1<<2.
+//                Padding groups carry the legal code 0x4.
+#pragma once
+
+#include <stdint.h>
+
+#include "ssconv.h"
+
+namespace ssconv {
+
+constexpr int kTileM = 128;          // rows of W (output channels) per CTA tile
+constexpr int kBlockK = 64;          // dense columns per k-block
+constexpr int kMetaImageBytes = 2048;
+
+struct Geometry {
+  int taps;          // KH*KW
+  int cblocks;       // k-blocks per tap = ceil(C_in/64)
+  int kblocks;       // taps*cblocks
+  int kblocks_pad;   // rounded up to even
+  int stages;        // kblocks_pad/2 (sparse pipeline stages per tile)
+  int m_tiles;       // ceil(C_out/128)
+  int Mp;            // m_tiles*128
+  int KC;            // 32*kblocks_pad: kept values per padded row
+};
+
+__host__ __device__ inline Geometry make_geometry(const ssconv_desc_t& d) {
+  Geometry g;
+  g.taps = d.KH * d.KW;
+  g.cblocks = (d.C_in + kBlockK - 1) / kBlockK;
+  g.kblocks = g.taps * g.cblocks;
+  g.kblocks_pad = (g.kblocks + 1) & ~1;
+  g.stages = g.kblocks_pad / 2;
+  g.m_tiles = (d.C_out + kTileM - 1) / kTileM;
+  g.Mp = g.m_tiles * kTileM;
+  g.KC = 32 * g.kblocks_pad;
+  return g;
+}
+
+// 4-bit position code (pos0 | pos1 << 2) of the six patterns, lexicographic in the kept
+// positions: {0,1},{0,2},{0,3},{1,2},{1,3},{2,3}.
+__host__ __device__ inline uint32_t pattern_code(uint32_t p) {
+  const uint32_t codes = 0x4u | (0x8u << 4) | (0xCu << 8) | (0x9u << 12) | (0xDu << 16) | (0xEu << 20);
+  return (codes >> (4 * p)) & 0xFu;
+}
+// Inverse: 4-bit code -> pattern index, 0xFF for a code that is not two ascending positions.
+__host__ __device__ inline uint32_t code_pattern(uint32_t code) {
+  switch (code & 0xFu) {
+    case 0x4: return 0;
+    case 0x8: return 1;
+    case 0xC: return 2;
+    case 0x9: return 3;
+    case 0xD: return 4;
+    case 0xE: return 5;
+    default: return 0xFFu;
+  }
+}
+
+}  // namespace ssconv

@@ -1,0 +1,198 @@
+// Mask selection (Eq. 1), mask application + 2:4 packing (Eq. 6, Fig. 1) and its inverse.
+// All three are one-off, memory-bound, integer-only kernels: values are compared and moved,
+// never computed with.
+#include <cuda_runtime.h>
+
+#include "layout.cuh"
+#include "ssconv.h"
+
+namespace ssconv {
+
+// ---------------------------------------------------------------------------------------
+// select_mask
+// ---------------------------------------------------------------------------------------
+
+// Eq. 1 without the one-hot: first maximum of the six scores of each group.
+__global__ void select_logits_kernel(const float2* __restrict__ scores, int64_t G, uint8_t* __restrict__ pattern) {
+  int64_t g = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (g >= G) return;
+  float2 a = scores[3 * g], b = scores[3 * g + 1], c = scores[3 * g + 2];
+  float v[6] = {a.x, a.y, b.x, b.y, c.x, c.y};
+  int best = 0;
+  float bv = v[0];
+#pragma unroll
+  for (int i = 1; i < 6; ++i) {
+    if (v[i] > bv) {
+      bv = v[i];
+      best = i;
+    }
+  }
+  pattern[g] = (uint8_t)best;
+}
+
+// Magnitude heuristic: keep the two largest |w| of the group.  Magnitudes are compared as
+// the 15-bit integers below the sign bit (monotone in |w|, +0 == -0); a position beats
+// another when it is larger, or equal and earlier, so exactly two positions are beaten by
+// fewer than two others.
+__device__ __forceinline__ uint32_t magnitude_pattern(uint32_t lo, uint32_t hi) {
+  uint32_t a[4] = {lo & 0x7FFFu, (lo >> 16) & 0x7FFFu, hi & 0x7FFFu, (hi >> 16) & 0x7FFFu};
+  int first = -1, second = -1;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    int beaten = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (j == i) continue;
+      beaten += (a[j] > a[i]) || (a[j] == a[i] && j < i);
+    }
+    if (beaten < 2) {
+      if (first < 0) first = i; else second = i;
+    }
+  }
+  // lexicographic index of the pair (first < second):
+  // {0,1}->0 {0,2}->1 {0,3}->2 {1,2}->3 {1,3}->4 {2,3}->5
+  return (uint32_t)(first == 0 ? second - 1 : (first == 1 ? second + 1 : 5));
+}
+
+__global__ void select_magnitude_kernel(const uint2* __restrict__ w, int64_t G, uint8_t* __restrict__ pattern) {
+  int64_t g = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (g >= G) return;
+  uint2 v = w[g];
+  pattern[g] = (uint8_t)magnitude_pattern(v.x, v.y);
+}
+
+// ---------------------------------------------------------------------------------------
+// compress: values
+// ---------------------------------------------------------------------------------------
+// One thread per (row, k-block, group-in-block): writes the two kept values (one 32-bit
+// store), +0 for padding.
+__global__ void compress_values_kernel(ssconv_desc_t d, Geometry geo, const uint2* __restrict__ w,
+                                       const uint8_t* __restrict__ pattern, uint32_t* __restrict__ w_comp) {
+  int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  int64_t total = (int64_t)geo.Mp * geo.kblocks_pad * 16;
+  if (t >= total) return;
+  int q = (int)(t % 16);
+  int b = (int)((t / 16) % geo.kblocks_pad);
+  int co = (int)(t / (16 * (int64_t)geo.kblocks_pad));
+  uint32_t out = 0;
+  if (co < d.C_out && b < geo.kblocks) {
+    int tap = b / geo.cblocks;
+    int c = (b % geo.cblocks) * kBlockK + 4 * q;
+    if (c < d.C_in) {
+      int64_t g = ((int64_t)co * geo.taps + tap) * (d.C_in / 4) + c / 4;
+      uint2 v = w[g];
+      uint32_t vals[4] = {v.x & 0xFFFFu, v.x >> 16, v.y & 0xFFFFu, v.y >> 16};
+      uint32_t code = pattern_code(pattern[g]);
+      out = vals[code & 3u] | (vals[(code >> 2) & 3u] << 16);
+    }
+  }
+  // row-major [Mp][KC] bf16; this thread's pair sits at column 32*b + 2*q
+  w_comp[((int64_t)co * geo.KC + 32 * b + 2 * q) / 2] = out;
+}
+
+// ---------------------------------------------------------------------------------------
+// compress: metadata
+// ---------------------------------------------------------------------------------------
+// One thread per 32-bit metadata word (layout.cuh says what a word holds).
+__global__ void compress_meta_kernel(ssconv_desc_t d, Geometry geo, const uint8_t* __restrict__ pattern,
+                                     uint32_t* __restrict__ meta) {
+  int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  int64_t total = (int64_t)geo.m_tiles * geo.stages * 128 * 4;
+  if (t >= total) return;
+  int j = (int)(t % 4);
+  int L = (int)((t / 4) % 128);
+  int s = (int)((t / 512) % geo.stages);
+  int mt = (int)(t / (512 * (int64_t)geo.stages));
+  int b = 2 * s + (j >> 1);
+  int tap = b / geo.cblocks;
+  int cbase = (b % geo.cblocks) * kBlockK + (j & 1) * 32 + 16 * ((L >> 3) & 1);
+  uint32_t word = 0;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    int co = mt * kTileM + (L & 7) + 16 * (L >> 4) + 8 * h;
+#pragma unroll
+    for (int gi = 0; gi < 4; ++gi) {
+      int c = cbase + 4 * gi;
+      uint32_t code = 0x4u;
+      if (co < d.C_out && b < geo.kblocks && c < d.C_in) {
+        int64_t g = ((int64_t)co * geo.taps + tap) * (d.C_in / 4) + c / 4;
+        code = pattern_code(pattern[g]);
+      }
+      word |= code << (16 * h + 4 * gi);
+    }
+  }
+  meta[t] = word;
+}
+
+// ---------------------------------------------------------------------------------------
+// decompress
+// ---------------------------------------------------------------------------------------
+// One thread per group: reads its code and its two values back and scatters them.
+__global__ void decompress_kernel(ssconv_desc_t d, Geometry geo, const uint32_t* __restrict__ w_comp,
+                                  const uint32_t* __restrict__ meta, uint2* __restrict__ w_out,
+                                  uint8_t* __restrict__ pattern_out) {
+  int64_t g = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  int groups_per_tap = d.C_in / 4;
+  int64_t G = (int64_t)d.C_out * geo.taps * groups_per_tap;
+  if (g >= G) return;
+  int c = (int)(g % groups_per_tap) * 4;
+  int tap = (int)((g / groups_per_tap) % geo.taps);
+  int co = (int)(g / ((int64_t)groups_per_tap * geo.taps));
+  int b = tap * geo.cblocks + c / kBlockK;
+  int cl = c % kBlockK;
+  // metadata word and nibble of this group
+  int mt = co / kTileM, r = co % kTileM;
+  int h = (r >> 3) & 1;
+  int L = (r & 7) + 8 * ((cl % 32) / 16) + 16 * (r >> 4);
+  int s = b >> 1;
+  int j = (b & 1) * 2 + cl / 32;
+  int gi = (cl % 16) / 4;
+  uint32_t word = meta[(((int64_t)mt * geo.stages + s) * 128 + L) * 4 + j];
+  uint32_t code = (word >> (16 * h + 4 * gi)) & 0xFu;
+  uint32_t pair = w_comp[((int64_t)co * geo.KC + 32 * b + cl / 2) / 2];
+  uint32_t vals[4] = {0, 0, 0, 0};
+  vals[code & 3u] = pair & 0xFFFFu;
+  vals[(code >> 2) & 3u] = pair >> 16;
+  w_out[g] = make_uint2(vals[0] | (vals[1] << 16), vals[2] | (vals[3] << 16));
+  if (pattern_out) pattern_out[g] = (uint8_t)code_pattern(code);
+}
+
+// ---------------------------------------------------------------------------------------
+// host launchers (called from the C ABI)
+// ---------------------------------------------------------------------------------------
+static inline unsigned blocks_for(int64_t n, int threads) { return (unsigned)((n + threads - 1) / threads); }
+
+cudaError_t launch_select(int mode, const void* scores, int64_t G, uint8_t* pattern, cudaStream_t st) {
+  if (G == 0) return cudaSuccess;
+  const int T = 256;
+  if (mode == SSCONV_MASK_LOGITS_F32)
+    select_logits_kernel<<<blocks_for(G, T), T, 0, st>>>((const float2*)scores, G, pattern);
+  else
+    select_magnitude_kernel<<<blocks_for(G, T), T, 0, st>>>((const uint2*)scores, G, pattern);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_compress(const ssconv_desc_t& d, const void* w, const uint8_t* pattern, void* w_comp, void* meta,
+                            cudaStream_t st) {
+  Geometry geo = make_geometry(d);
+  const int T = 256;
+  int64_t nv = (int64_t)geo.Mp * geo.kblocks_pad * 16;
+  compress_values_kernel<<<blocks_for(nv, T), T, 0, st>>>(d, geo, (const uint2*)w, pattern, (uint32_t*)w_comp);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  int64_t nm = (int64_t)geo.m_tiles * geo.stages * 512;
+  compress_meta_kernel<<<blocks_for(nm, T), T, 0, st>>>(d, geo, pattern, (uint32_t*)meta);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decompress(const ssconv_desc_t& d, const void* w_comp, const void* meta, void* w_out,
+                              uint8_t* pattern_out, cudaStream_t st) {
+  Geometry geo = make_geometry(d);
+  const int T = 256;
+  int64_t G = (int64_t)d.C_out * geo.taps * (d.C_in / 4);
+  decompress_kernel<<<blocks_for(G, T), T, 0, st>>>(d, geo, (const uint32_t*)w_comp, (const uint32_t*)meta,
+                                                    (uint2*)w_out, pattern_out);
+  return cudaGetLastError();
+}
+
+}  // namespace ssconv
