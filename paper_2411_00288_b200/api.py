@@ -1,0 +1,203 @@
+"""ctypes binding of libssconv.so: the same entry points as include/ssconv.h.
+
+Only argument marshalling happens here; torch supplies device memory and the current
+stream.  There is no CPU path: if the library is missing or a call fails, an exception
+is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional, Tuple
+
+import torch
+
+FLAG_BIAS = 1
+FLAG_RELU = 2
+MASK_LOGITS_F32 = 0
+MASK_MAGNITUDE_BF16 = 1
+OK = 0
+ERR_TIMEOUT = 8
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.so")
+EXPORTS = ("ssconv_version", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes", "ssconv_select_mask",
+           "ssconv_compress", "ssconv_decompress", "ssconv_forward", "ssconv_forward_dense")
+
+
+class SsconvError(RuntimeError):
+    def __init__(self, fn: str, status: int, text: str):
+        super().__init__(f"{fn} failed: status {status} ({text})")
+        self.status = status
+
+
+class Desc(ctypes.Structure):
+    """Mirror of ssconv_desc_t."""
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "N", "H", "W", "C_in", "C_out", "KH", "KW", "stride_h", "stride_w", "pad_h", "pad_w", "dil_h", "dil_w")] + [
+        ("flags", ctypes.c_uint32)]
+
+
+def make_desc(N, H, W, C_in, C_out, KH, KW, stride=1, pad=0, dil=1, bias=True, relu=False) -> Desc:
+    def pair(v):
+        return (v, v) if isinstance(v, int) else tuple(v)
+    (sh, sw), (ph, pw), (dh, dw) = pair(stride), pair(pad), pair(dil)
+    flags = (FLAG_BIAS if bias else 0) | (FLAG_RELU if relu else 0)
+    return Desc(N, H, W, C_in, C_out, KH, KW, sh, sw, ph, pw, dh, dw, flags)
+
+
+def desc_from_spec(spec) -> Desc:
+    """Descriptor for a synth.LayerSpec."""
+    return make_desc(spec.N, spec.H, spec.W, spec.C_in, spec.C_out, spec.KH, spec.KW, spec.stride, spec.pad,
+                     spec.dil, bias=spec.has_bias, relu=spec.relu)
+
+
+_lib = None
+
+
+def lib():
+    """Load libssconv.so once; raise if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise FileNotFoundError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2411_00288_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        dp = ctypes.POINTER(Desc)
+        L.ssconv_version.restype = i32
+        L.ssconv_version.argtypes = []
+        L.ssconv_status_string.restype = ctypes.c_char_p
+        L.ssconv_status_string.argtypes = [i32]
+        L.ssconv_out_shape.restype = i32
+        L.ssconv_out_shape.argtypes = [dp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.ssconv_sizes.restype = i32
+        L.ssconv_sizes.argtypes = [dp, ctypes.POINTER(i64)] + [ctypes.POINTER(sz)] * 4
+        L.ssconv_select_mask.restype = i32
+        L.ssconv_select_mask.argtypes = [i32, vp, i64, vp, vp]
+        L.ssconv_compress.restype = i32
+        L.ssconv_compress.argtypes = [dp, vp, vp, vp, vp, vp]
+        L.ssconv_decompress.restype = i32
+        L.ssconv_decompress.argtypes = [dp, vp, vp, vp, vp, vp]
+        L.ssconv_forward.restype = i32
+        L.ssconv_forward.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.ssconv_forward_dense.restype = i32
+        L.ssconv_forward_dense.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().ssconv_status_string(status).decode()
+
+
+def _check(fn: str, status: int):
+    if status != OK:
+        raise SsconvError(fn, status, status_string(status))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _need_cuda(*tensors):
+    for t in tensors:
+        if t is not None and not (t.is_cuda and t.is_contiguous()):
+            raise ValueError("tensors must be contiguous CUDA tensors")
+
+
+def ssconv_version() -> int:
+    return int(lib().ssconv_version())
+
+
+def ssconv_out_shape(desc: Desc) -> Tuple[int, int]:
+    h, w = ctypes.c_int32(), ctypes.c_int32()
+    _check("ssconv_out_shape", lib().ssconv_out_shape(ctypes.byref(desc), ctypes.byref(h), ctypes.byref(w)))
+    return int(h.value), int(w.value)
+
+
+@dataclass(frozen=True)
+class Sizes:
+    G: int
+    w_comp_bytes: int
+    meta_bytes: int
+    ws_bytes_sparse: int
+    ws_bytes_dense: int
+
+
+def ssconv_sizes(desc: Desc) -> Sizes:
+    G = ctypes.c_int64()
+    a, b, c, d = (ctypes.c_size_t() for _ in range(4))
+    _check("ssconv_sizes", lib().ssconv_sizes(ctypes.byref(desc), ctypes.byref(G), ctypes.byref(a), ctypes.byref(b),
+                                              ctypes.byref(c), ctypes.byref(d)))
+    return Sizes(int(G.value), int(a.value), int(b.value), int(c.value), int(d.value))
+
+
+def ssconv_select_mask(mode: int, scores: torch.Tensor, G: int, pattern: Optional[torch.Tensor] = None,
+                       stream=None) -> torch.Tensor:
+    """pattern uint8 [G] from fp32 scores [G,6] (mode LOGITS) or bf16 weights (mode MAGNITUDE)."""
+    _need_cuda(scores, pattern)
+    if pattern is None:
+        pattern = torch.empty((G,), dtype=torch.uint8, device=scores.device)
+    _check("ssconv_select_mask", lib().ssconv_select_mask(mode, _ptr(scores), G, _ptr(pattern), _stream(stream)))
+    return pattern
+
+
+def ssconv_compress(desc: Desc, w: torch.Tensor, pattern: torch.Tensor, stream=None):
+    """(w_comp, meta) uint8 blobs from bf16 weights [C_out,KH,KW,C_in] and pattern [G]."""
+    _need_cuda(w, pattern)
+    sz = ssconv_sizes(desc)
+    w_comp = torch.empty((sz.w_comp_bytes,), dtype=torch.uint8, device=w.device)
+    meta = torch.empty((sz.meta_bytes,), dtype=torch.uint8, device=w.device)
+    _check("ssconv_compress", lib().ssconv_compress(ctypes.byref(desc), _ptr(w), _ptr(pattern), _ptr(w_comp),
+                                                    _ptr(meta), _stream(stream)))
+    return w_comp, meta
+
+
+def ssconv_decompress(desc: Desc, w_comp: torch.Tensor, meta: torch.Tensor, want_pattern: bool = True, stream=None):
+    """(w_masked bf16 [C_out,KH,KW,C_in], pattern uint8 [G] or None) read back from the blobs."""
+    _need_cuda(w_comp, meta)
+    sz = ssconv_sizes(desc)
+    w_out = torch.empty((desc.C_out, desc.KH, desc.KW, desc.C_in), dtype=torch.bfloat16, device=w_comp.device)
+    pat = torch.empty((sz.G,), dtype=torch.uint8, device=w_comp.device) if want_pattern else None
+    _check("ssconv_decompress", lib().ssconv_decompress(ctypes.byref(desc), _ptr(w_comp), _ptr(meta), _ptr(w_out),
+                                                        _ptr(pat), _stream(stream)))
+    return w_out, pat
+
+
+def _alloc_y(desc: Desc, x: torch.Tensor) -> torch.Tensor:
+    ho, wo = ssconv_out_shape(desc)
+    return torch.empty((desc.N, ho, wo, desc.C_out), dtype=torch.bfloat16, device=x.device)
+
+
+def ssconv_forward(desc: Desc, x: torch.Tensor, w_comp: torch.Tensor, meta: torch.Tensor,
+                   bias: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None,
+                   ws: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                   stream=None) -> torch.Tensor:
+    """2:4 masked convolution forward; returns y bf16 [N,H_out,W_out,C_out] (enqueued, not synchronised)."""
+    _need_cuda(x, w_comp, meta, bias, y, ws, dev_status)
+    if y is None:
+        y = _alloc_y(desc, x)
+    _check("ssconv_forward", lib().ssconv_forward(
+        ctypes.byref(desc), _ptr(x), _ptr(w_comp), _ptr(meta), _ptr(bias), _ptr(y), _ptr(ws),
+        0 if ws is None else ws.numel() * ws.element_size(), _ptr(dev_status), _stream(stream)))
+    return y
+
+
+def ssconv_forward_dense(desc: Desc, x: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor] = None,
+                         y: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None,
+                         dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Dense counterpart with bf16 weights [C_out,KH,KW,C_in]."""
+    _need_cuda(x, w, bias, y, ws, dev_status)
+    if y is None:
+        y = _alloc_y(desc, x)
+    _check("ssconv_forward_dense", lib().ssconv_forward_dense(
+        ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _ptr(ws),
+        0 if ws is None else ws.numel() * ws.element_size(), _ptr(dev_status), _stream(stream)))
+    return y

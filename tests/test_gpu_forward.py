@@ -1,0 +1,81 @@
+"""GPU parity of the sparse and dense forward kernels against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2411_00288_b200 import api, synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _assert_ok(rel, mx, what):
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"{what}: rel_fro={rel:.3e} max_abs={mx:.3e}"
+
+
+def test_config1_sparse_and_dense():
+    spec = synth.config_layers(1)[0]
+    _assert_ok(*parity.check_layer(spec, DEV, sparse=True), "config 1 sparse")
+    _assert_ok(*parity.check_layer(spec, DEV, sparse=False), "config 1 dense")
+
+
+SWEEP = [
+    # name                      N  H   W   Ci   Co  KH KW s  p  d
+    ("pw_64",                   2, 9,  7,  64,  64, 1, 1, 1, 0, 1),
+    ("pw_ragged_96to136",       3, 11, 5,  96, 136, 1, 1, 1, 0, 1),
+    ("pw_s2",                   2, 10, 10, 64, 128, 1, 1, 2, 0, 1),
+    ("c3_s1p1",                 2, 12, 9,  64, 128, 3, 3, 1, 1, 1),
+    ("c3_s2p1",                 2, 13, 12, 128, 64, 3, 3, 2, 1, 1),
+    ("c3_nopad",                1, 10, 10, 64,  64, 3, 3, 1, 0, 1),
+    ("c3_dil2",                 1, 12, 12, 64,  64, 3, 3, 1, 2, 2),
+    ("c5_p2",                   1, 9,  9,  32,  40, 5, 5, 1, 2, 1),
+    ("c3_small_channels",       2, 8,  8,  8,   8,  3, 3, 1, 1, 1),
+    ("c3_7x7_maps_wrap_images", 9, 7,  7,  128, 256, 3, 3, 1, 1, 1),
+    ("pw_deepK",                1, 6,  6,  1024, 64, 1, 1, 1, 0, 1),
+]
+
+
+@pytest.mark.parametrize("case", SWEEP, ids=[c[0] for c in SWEEP])
+@pytest.mark.parametrize("sparse", [True, False], ids=["sparse", "dense"])
+def test_shape_sweep(case, sparse):
+    name, N, H, W, Ci, Co, KH, KW, s, p, d = case
+    spec = synth.LayerSpec(name, N, H, W, Ci, Co, KH, KW, s, p, d, relu=(Co % 16 == 0), w_std="fan_in",
+                           mask_source="magnitude", config=9, index=SWEEP.index(case))
+    _assert_ok(*parity.check_layer(spec, DEV, sparse=sparse), name)
+
+
+def test_no_bias_no_relu_and_gumbel_logit_masks():
+    spec = synth.LayerSpec("nobias", 2, 14, 14, 128, 128, 3, 3, 1, 1, 1, relu=False, has_bias=False, w_std="he",
+                           mask_source="gumbel_logits", config=9, index=50)
+    _assert_ok(*parity.check_layer(spec, DEV, sparse=True), "no bias")
+
+
+def test_sparse_equals_dense_on_masked_weights():
+    """Eq. 6: the sparse kernel on (values, metadata) and the dense kernel on M .* W agree closely."""
+    spec = synth.LayerSpec("x", 2, 14, 14, 128, 128, 3, 3, 1, 1, 1, config=9, index=51)
+    inp = synth.make_inputs(spec)
+    desc = api.desc_from_spec(spec)
+    x, w, b = inp.x.to(DEV), inp.w.to(DEV), inp.bias.to(DEV)
+    pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
+    w_comp, meta = api.ssconv_compress(desc, w, pat)
+    w_masked, _ = api.ssconv_decompress(desc, w_comp, meta)
+    ys = api.ssconv_forward(desc, x, w_comp, meta, b)
+    yd = api.ssconv_forward_dense(desc, x, w_masked, b)
+    torch.cuda.synchronize()
+    assert (ys.float() - yd.float()).abs().max().item() <= 2 ** -6
+
+
+def test_all_ones_input_closed_form_borders():
+    """x == 1, w == 2^-3: y = bias + 2^-3 * (C_in/2) * #taps inside the image, exactly representable."""
+    N, H, W, C, Co, K = 1, 9, 10, 64, 64, 3
+    desc = api.make_desc(N, H, W, C, Co, K, K, 1, 1, 1, bias=False, relu=False)
+    x = torch.ones((N, H, W, C), dtype=torch.bfloat16, device=DEV)
+    w = torch.full((Co, K, K, C), 0.125, dtype=torch.bfloat16, device=DEV)
+    pat = torch.randint(0, 6, (Co * K * K * C // 4,), dtype=torch.uint8, device=DEV)
+    w_comp, meta = api.ssconv_compress(desc, w, pat)
+    y = api.ssconv_forward(desc, x, w_comp, meta).float().cpu().numpy()
+    for ho in range(H):
+        for wo in range(W):
+            taps = sum(1 for kh in range(K) for kw in range(K) if 0 <= ho - 1 + kh < H and 0 <= wo - 1 + kw < W)
+            assert (y[0, ho, wo, :] == 0.125 * (C // 2) * taps).all()
