@@ -39,6 +39,7 @@ class LayerSpec:
     mask_source: str = "magnitude"  # "magnitude" | "gumbel_logits" | "uniform_pattern"
     config: int = 0
     index: int = 0
+    extra: bool = False            # parity-only row, not part of the timed sweep
 
     @property
     def K(self) -> int:
@@ -96,7 +97,8 @@ def config_layers(config: int, batch: Optional[int] = None) -> List[LayerSpec]:
         for hw, c in ((56, 64), (28, 128), (14, 256)):
             L.append(LayerSpec(f"r18_3x3s2_{c}to{2 * c}_{hw}", n, hw, hw, c, 2 * c, 3, 3, 2, 1))
         for hw, c in ((56, 64), (28, 128), (14, 256)):
-            L.append(LayerSpec(f"r18_1x1s2_{c}to{2 * c}_{hw}", n, hw, hw, c, 2 * c, 1, 1, 2, 0, relu=False))
+            L.append(LayerSpec(f"r18_1x1s2_{c}to{2 * c}_{hw}", n, hw, hw, c, 2 * c, 1, 1, 2, 0, relu=False,
+                               extra=True))
         return _number(L, 2)
     if config == 3:
         n = batch or 64
