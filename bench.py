@@ -178,6 +178,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layer-iters", type=int, default=200)
+    ap.add_argument("--only-layer", type=int, default=None,
+                    help="profiling aid: launch just this layer of the sweep --layer-iters times and exit")
+    ap.add_argument("--dense", action="store_true", help="with --only-layer: use the dense kernel")
     args = ap.parse_args()
     if args.impl == "reference":
         reference_arm(args)
@@ -204,6 +207,8 @@ def main():
     warmup = max(3, args.warmup)
 
     layers = timed_layers()
+    if args.only_layer is not None:
+        layers = [layers[args.only_layer]]
     # ---- one-off preparation with the library's own kernels: select -> compress (S1, S2)
     prep = []
     set_bytes = sum(2 * (s.N * s.H * s.W * s.C_in + s.P * s.C_out) for s in layers)
@@ -227,6 +232,20 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     torch.cuda.synchronize()
     prep_seconds = time.perf_counter() - t_prep0
+
+    if args.only_layer is not None:
+        L = prep[0]
+        for i in range(args.layer_iters):
+            r = i % n_sets
+            if args.dense:
+                api.ssconv_forward_dense(L["desc"], L["xs"][r], L["w"], L["bias"], y=L["ys"][r], dev_status=status)
+            else:
+                api.ssconv_forward(L["desc"], L["xs"][r], L["w_comp"], L["meta"], L["bias"], y=L["ys"][r],
+                                   dev_status=status)
+        torch.cuda.synchronize()
+        print(json.dumps({"only_layer": L["spec"].name, "launches": args.layer_iters, "dense": args.dense,
+                          "dev_status": int(status.item())}))
+        return
 
     def step(r, sparse=True):
         for L in prep:

@@ -105,42 +105,56 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t g = 0;
+      // All index arithmetic below is incremental: this single thread's instruction stream
+      // is on the critical path of every stage, so there is no division inside the loops.
+      int s = 0;
+      uint32_t ph = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
-        const int m = tile % p.m_tiles;
-        const int p0 = (tile / p.m_tiles) * kBN;
+        const int pt = tile / p.m_tiles;
+        const int m = tile - pt * p.m_tiles;
+        const int p0 = pt * kBN;
         const int n0 = p0 / p.HoWo;
         const int rem = p0 - n0 * p.HoWo;
         const int ho0 = rem / p.Wo;
         const int wo0 = rem - ho0 * p.Wo;
         const int base_w = wo0 * p.stride_w - p.pad_w;
         const int base_h = ho0 * p.stride_h - p.pad_h;
-        for (int it = 0; it < p.iters; ++it, ++g) {
-          const int s = g % STAGES;
-          const uint32_t ph = (g / STAGES) & 1u;
+        const uint8_t* meta_src = p.meta + (size_t)m * p.iters * kMetaImageBytes;
+        int b = 0, cc = 0, tap = 0, off_w = 0, off_h = 0, kw = 0;
+        for (int it = 0; it < p.iters; ++it) {
           if (!mbar_wait_bounded(&bar_empty[s], ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
           uint8_t* st = smem + s * C::kStageBytes;
-          int nb = p.kblocks - KBS * it;
+          int nb = p.kblocks - b;
           if (nb > KBS) nb = KBS;
           mbar_expect_tx(&bar_full[s], kATileBytes + nb * kBTileBytes + C::kMetaBytes);
           if (SPARSE) {
             tma_load_2d(st, &tm_a, &bar_full[s], it * 64, m * kTileM);
           } else {
-            tma_load_3d(st, &tm_a, &bar_full[s], (it % p.cblocks) * kBlockK, it / p.cblocks, m * kTileM);
+            tma_load_3d(st, &tm_a, &bar_full[s], cc * kBlockK, tap, m * kTileM);
           }
           for (int j = 0; j < nb; ++j) {
-            const int b = KBS * it + j;
-            const int tap = b / p.cblocks;
-            const int cc = b - tap * p.cblocks;
-            const int kh = tap / p.KW;
-            const int kw = tap - kh * p.KW;
             tma_load_im2col_4d(st + kATileBytes + j * kBTileBytes, &tm_b, &bar_full[s], cc * kBlockK, base_w, base_h,
-                               n0, (uint16_t)(kw * p.dil_w), (uint16_t)(kh * p.dil_h));
+                               n0, (uint16_t)off_w, (uint16_t)off_h);
+            ++b;
+            if (++cc == p.cblocks) {  // next filter tap
+              cc = 0;
+              ++tap;
+              off_w += p.dil_w;
+              if (++kw == p.KW) {
+                kw = 0;
+                off_w = 0;
+                off_h += p.dil_h;
+              }
+            }
           }
           if (SPARSE) {
-            bulk_load(st + kATileBytes + KBS * kBTileBytes, p.meta + ((size_t)m * p.iters + it) * kMetaImageBytes,
-                      kMetaImageBytes, &bar_full[s]);
+            bulk_load(st + kATileBytes + KBS * kBTileBytes, meta_src, kMetaImageBytes, &bar_full[s]);
+            meta_src += kMetaImageBytes;
+          }
+          if (++s == STAGES) {
+            s = 0;
+            ph ^= 1u;
           }
         }
       }
@@ -149,8 +163,19 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_bf16(kTileM, kBN, SPARSE);
-      uint32_t g = 0;
+      constexpr uint32_t kStageDesc = C::kStageBytes >> 4;   // descriptor address units are 16 B
+      constexpr uint32_t kBTileDesc = kBTileBytes >> 4;
+      const uint64_t a_desc0 = smem_desc_sw128(smem_u32(smem));
+      const uint64_t b_desc0 = smem_desc_sw128(smem_u32(smem) + kATileBytes);
+      const uint64_t m_desc0 = smem_desc_noswizzle(smem_u32(smem) + kATileBytes + KBS * kBTileBytes, 16, 128);
+      // channels left in the last k-block of a tap decide how many MMAs it needs
+      const int tail_c = p.C_in - (p.cblocks - 1) * kBlockK;
+      const int mma_full = SPARSE ? 2 : 4;
+      const int mma_tail = SPARSE ? ((tail_c + 31) >> 5) : ((tail_c + 15) >> 4);
+      int s = 0;
+      uint32_t ph = 0;
       uint32_t tcount = 0;
+      uint32_t gpar = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x, ++tcount) {
         const uint32_t buf = tcount & 1u;
@@ -159,26 +184,22 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kBN;
         uint32_t accumulate = 0;
-        for (int it = 0; it < p.iters; ++it, ++g) {
-          const int s = g % STAGES;
-          const uint32_t ph = (g / STAGES) & 1u;
+        int b = 0, cc = 0;
+        for (int it = 0; it < p.iters; ++it) {
           if (!mbar_wait_bounded(&bar_full[s], ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t st = smem_u32(smem + s * C::kStageBytes);
-          const uint64_t a_desc = smem_desc_sw128(st);
-          int nb = p.kblocks - KBS * it;
+          const uint64_t a_desc = a_desc0 + (uint64_t)(s * kStageDesc);
+          const uint64_t b_desc_s = b_desc0 + (uint64_t)(s * kStageDesc);
+          int nb = p.kblocks - b;
           if (nb > KBS) nb = KBS;
           if (SPARSE) {
             // two metadata slots of 4 columns, alternating per stage
-            const uint32_t meta_tmem = tmem_base + kMetaCol + 4u * (g & 1u);
-            tc_cp_128x128b(meta_tmem, smem_desc_noswizzle(st + kATileBytes + KBS * kBTileBytes, 16, 128));
+            const uint32_t meta_tmem = tmem_base + kMetaCol + 4u * gpar;
+            gpar ^= 1u;
+            tc_cp_128x128b(meta_tmem, m_desc0 + (uint64_t)(s * kStageDesc));
             for (int j = 0; j < nb; ++j) {
-              const int b = KBS * it + j;
-              const int cc = b % p.cblocks;
-              int vc = p.C_in - cc * kBlockK;
-              if (vc > kBlockK) vc = kBlockK;
-              const int n_mma = (vc + 31) >> 5;  // 32 dense columns per sparse MMA
-              const uint64_t b_desc = smem_desc_sw128(st + kATileBytes + j * kBTileBytes);
+              const int n_mma = (cc == p.cblocks - 1) ? mma_tail : mma_full;  // 32 dense columns per sparse MMA
+              const uint64_t b_desc = b_desc_s + (uint64_t)(j * kBTileDesc);
               for (int k2 = 0; k2 < n_mma; ++k2) {
                 const uint32_t kk = 2 * j + k2;  // MMA slot within the stage (= metadata column)
                 // A advances 16 kept values = 32 B, B advances 32 channels = 64 B (descriptor units of 16 B)
@@ -186,19 +207,23 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                               accumulate);
                 accumulate = 1;
               }
+              ++b;
+              if (++cc == p.cblocks) cc = 0;
             }
           } else {
-            const int cc = it % p.cblocks;
-            int vc = p.C_in - cc * kBlockK;
-            if (vc > kBlockK) vc = kBlockK;
-            const int n_mma = (vc + 15) >> 4;  // 16 columns per dense MMA
-            const uint64_t b_desc = smem_desc_sw128(st + kATileBytes);
+            const int n_mma = (cc == p.cblocks - 1) ? mma_tail : mma_full;  // 16 columns per dense MMA
             for (int kk = 0; kk < n_mma; ++kk) {
-              tc_mma_dense(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, accumulate);
+              tc_mma_dense(d_tmem, a_desc + 2 * kk, b_desc_s + 2 * kk, idesc, accumulate);
               accumulate = 1;
             }
+            ++b;
+            if (++cc == p.cblocks) cc = 0;
           }
           tc_commit(&bar_empty[s]);
+          if (++s == STAGES) {
+            s = 0;
+            ph ^= 1u;
+          }
         }
         if (ok) tc_commit(&bar_acc_full[buf]);
       }
