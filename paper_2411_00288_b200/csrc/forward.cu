@@ -4,15 +4,19 @@
 //   D[C_out x P] = A[C_out x K] * B[K x P],   P = N*H_out*W_out pixels, K = KH*KW*C_in
 //
 // A = weights (the only operand tcgen05.mma.sp accepts in 2:4 form), B = activations.  A CTA
-// owns a 128 (output channels) x 128 (pixels) tile of D at a time and walks a static list of
-// tiles (persistent kernel).  Warp roles:
-//   warp 0      TMA producer: per stage one weight tile, one or two im2col activation tiles
-//               (64 channels x 128 pixels at one filter tap, zero-filled outside the image),
-//               and for the sparse kernel the 2 KB metadata image.
+// owns a 128 (output channels) x 240 (pixels) tile of D at a time and walks a static list of
+// tiles (persistent kernel).  The pixel extent is as wide as two fp32 accumulators plus the
+// metadata columns allow in the 512 TMEM columns: one thread issues every MMA, and the cost of
+// issuing one is what bounds narrow tiles.  Warp roles:
+//   warp 0      TMA producer.  Two rings: weight tiles (128 rows x 128 B, plus the 2 KB
+//               metadata image for the sparse kernel) and activation tiles (240 pixels x 64
+//               channels at one filter tap, im2col mode, zero-filled outside the image).  A
+//               sparse weight tile spans two activation tiles (128 dense columns).
 //   warp 1      owns TMEM; one thread copies metadata smem->TMEM and issues the MMAs into one of
-//               two fp32 accumulators (128 lanes x 128 columns each).
+//               two fp32 accumulators (128 lanes x 240 columns each).
 //   warps 2-5   epilogue: TMEM -> registers, + bias, ReLU, bf16, transpose through shared
-//               memory to pixel-major rows, one TMA store per tile (clipped at the tensor edge).
+//               memory to pixel-major rows, TMA stores of 80-pixel pieces (clipped at the
+//               tensor edge) from a double-buffered staging area.
 // All mbarrier waits are bounded; when one runs out the CTA raises a flag, every role leaves
 // its loop, TMEM is freed and SSCONV_ERR_TIMEOUT is stored to *dev_status.
 #include <cuda.h>
@@ -25,23 +29,27 @@
 
 namespace ssconv {
 
-constexpr int kBN = 128;                 // pixels per tile (N of the MMA)
+constexpr int kBN = 240;                 // pixels per tile (N of the MMA)
+constexpr int kPiece = 80;               // pixels per epilogue store
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kMetaCol = 2 * kBN;   // first TMEM column of the metadata (2 slots x 4 columns)
+constexpr uint32_t kAccCol1 = 256;       // second accumulator; the first starts at column 0
+constexpr uint32_t kMetaCol = kBN;       // metadata: 2 slots x 4 columns in [240, 248)
 constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 1.9 GHz
 constexpr uint32_t kATileBytes = 128 * 128;          // 128 rows x 128 B
-constexpr uint32_t kBTileBytes = kBN * 128;          // 128 pixels x 64 channels bf16
-constexpr uint32_t kOutStageBytes = kBN * 256;       // 128 pixels x 128 channels bf16
+constexpr uint32_t kBTileBytes = kBN * 128;          // 240 pixels x 64 channels bf16
+constexpr uint32_t kPieceBytes = kPiece * 256;       // 80 pixels x 128 channels bf16
+constexpr int kNA = 3;                               // weight ring depth
+constexpr int kNB = 4;                               // activation ring depth
 
 template <bool SPARSE>
 struct Cfg {
-  static constexpr int kBlocksPerStage = SPARSE ? 2 : 1;
-  static constexpr int kStages = SPARSE ? 3 : 5;
+  static constexpr int kBlocksPerA = SPARSE ? 2 : 1;  // k-blocks of 64 dense columns per weight tile
   static constexpr uint32_t kMetaBytes = SPARSE ? (uint32_t)kMetaImageBytes : 0u;
-  static constexpr uint32_t kStageBytes = kATileBytes + kBlocksPerStage * kBTileBytes + kMetaBytes;
+  static constexpr uint32_t kAEntryBytes = kATileBytes + kMetaBytes;
   static constexpr uint32_t kBarrierBytes = 256;
-  static constexpr uint32_t kSmemBytes = kStages * kStageBytes + kOutStageBytes + kBarrierBytes + 1024;
+  static constexpr uint32_t kSmemBytes =
+      kNA * kAEntryBytes + kNB * kBTileBytes + 2 * kPieceBytes + kBarrierBytes + 1024;
 };
 
 struct FwdParams {
@@ -49,7 +57,7 @@ struct FwdParams {
   int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
   int cblocks, kblocks;
   int m_tiles, num_tiles;
-  int iters;  // pipeline stages per tile
+  int a_tiles;  // weight tiles per output tile
   uint32_t flags;
   const float* bias;
   const uint8_t* meta;
@@ -63,15 +71,18 @@ __global__ void __launch_bounds__(kThreads, 1)
 ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                   const __grid_constant__ CUtensorMap tm_y, const FwdParams p) {
   using C = Cfg<SPARSE>;
-  constexpr int STAGES = C::kStages;
-  constexpr int KBS = C::kBlocksPerStage;
+  constexpr int APER = C::kBlocksPerA;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* out_stage = smem + STAGES * C::kStageBytes;
-  uint64_t* bar_full = reinterpret_cast<uint64_t*>(out_stage + kOutStageBytes);
-  uint64_t* bar_empty = bar_full + STAGES;
-  uint64_t* bar_acc_full = bar_empty + STAGES;
+  uint8_t* a_ring = smem;
+  uint8_t* b_ring = a_ring + kNA * C::kAEntryBytes;
+  uint8_t* out_stage = b_ring + kNB * kBTileBytes;
+  uint64_t* bar_a_full = reinterpret_cast<uint64_t*>(out_stage + 2 * kPieceBytes);
+  uint64_t* bar_a_empty = bar_a_full + kNA;
+  uint64_t* bar_b_full = bar_a_empty + kNA;
+  uint64_t* bar_b_empty = bar_b_full + kNB;
+  uint64_t* bar_acc_full = bar_b_empty + kNB;
   uint64_t* bar_acc_empty = bar_acc_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -81,9 +92,13 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      mbar_init(&bar_full[s], 1);
-      mbar_init(&bar_empty[s], 1);
+    for (int s = 0; s < kNA; ++s) {
+      mbar_init(&bar_a_full[s], 1);
+      mbar_init(&bar_a_empty[s], 1);
+    }
+    for (int s = 0; s < kNB; ++s) {
+      mbar_init(&bar_b_full[s], 1);
+      mbar_init(&bar_b_empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bar_acc_full[b], 1);
@@ -105,10 +120,10 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      // All index arithmetic below is incremental: this single thread's instruction stream
-      // is on the critical path of every stage, so there is no division inside the loops.
-      int s = 0;
-      uint32_t ph = 0;
+      // All index arithmetic in the k loop is incremental: this single thread's instruction
+      // stream is on the critical path of every stage.
+      int sa = 0, sb = 0;
+      uint32_t pha = 0, phb = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
         const int pt = tile / p.m_tiles;
@@ -120,41 +135,44 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         const int wo0 = rem - ho0 * p.Wo;
         const int base_w = wo0 * p.stride_w - p.pad_w;
         const int base_h = ho0 * p.stride_h - p.pad_h;
-        const uint8_t* meta_src = p.meta + (size_t)m * p.iters * kMetaImageBytes;
-        int b = 0, cc = 0, tap = 0, off_w = 0, off_h = 0, kw = 0;
-        for (int it = 0; it < p.iters; ++it) {
-          if (!mbar_wait_bounded(&bar_empty[s], ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-          uint8_t* st = smem + s * C::kStageBytes;
-          int nb = p.kblocks - b;
-          if (nb > KBS) nb = KBS;
-          mbar_expect_tx(&bar_full[s], kATileBytes + nb * kBTileBytes + C::kMetaBytes);
-          if (SPARSE) {
-            tma_load_2d(st, &tm_a, &bar_full[s], it * 64, m * kTileM);
-          } else {
-            tma_load_3d(st, &tm_a, &bar_full[s], cc * kBlockK, tap, m * kTileM);
-          }
-          for (int j = 0; j < nb; ++j) {
-            tma_load_im2col_4d(st + kATileBytes + j * kBTileBytes, &tm_b, &bar_full[s], cc * kBlockK, base_w, base_h,
-                               n0, (uint16_t)off_w, (uint16_t)off_h);
-            ++b;
-            if (++cc == p.cblocks) {  // next filter tap
-              cc = 0;
-              ++tap;
-              off_w += p.dil_w;
-              if (++kw == p.KW) {
-                kw = 0;
-                off_w = 0;
-                off_h += p.dil_h;
-              }
+        const uint8_t* meta_src = p.meta + (size_t)m * p.a_tiles * kMetaImageBytes;
+        int cc = 0, tap = 0, off_w = 0, off_h = 0, kw = 0, a_idx = 0, a_sub = 0;
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (a_sub == 0) {
+            if (!mbar_wait_bounded(&bar_a_empty[sa], pha ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+            uint8_t* st = a_ring + sa * C::kAEntryBytes;
+            mbar_expect_tx(&bar_a_full[sa], C::kAEntryBytes);
+            if (SPARSE) {
+              tma_load_2d(st, &tm_a, &bar_a_full[sa], a_idx * 64, m * kTileM);
+              bulk_load(st + kATileBytes, meta_src, kMetaImageBytes, &bar_a_full[sa]);
+              meta_src += kMetaImageBytes;
+            } else {
+              tma_load_3d(st, &tm_a, &bar_a_full[sa], cc * kBlockK, tap, m * kTileM);
+            }
+            ++a_idx;
+            if (++sa == kNA) {
+              sa = 0;
+              pha ^= 1u;
             }
           }
-          if (SPARSE) {
-            bulk_load(st + kATileBytes + KBS * kBTileBytes, meta_src, kMetaImageBytes, &bar_full[s]);
-            meta_src += kMetaImageBytes;
+          if (++a_sub == APER) a_sub = 0;
+          if (!mbar_wait_bounded(&bar_b_empty[sb], phb ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+          mbar_expect_tx(&bar_b_full[sb], kBTileBytes);
+          tma_load_im2col_4d(b_ring + sb * kBTileBytes, &tm_b, &bar_b_full[sb], cc * kBlockK, base_w, base_h, n0,
+                             (uint16_t)off_w, (uint16_t)off_h);
+          if (++sb == kNB) {
+            sb = 0;
+            phb ^= 1u;
           }
-          if (++s == STAGES) {
-            s = 0;
-            ph ^= 1u;
+          if (++cc == p.cblocks) {  // next filter tap
+            cc = 0;
+            ++tap;
+            off_w += p.dil_w;
+            if (++kw == p.KW) {
+              kw = 0;
+              off_w = 0;
+              off_h += p.dil_h;
+            }
           }
         }
       }
@@ -163,66 +181,71 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_bf16(kTileM, kBN, SPARSE);
-      constexpr uint32_t kStageDesc = C::kStageBytes >> 4;   // descriptor address units are 16 B
+      constexpr uint32_t kAEntryDesc = C::kAEntryBytes >> 4;  // descriptor address units are 16 B
       constexpr uint32_t kBTileDesc = kBTileBytes >> 4;
-      const uint64_t a_desc0 = smem_desc_sw128(smem_u32(smem));
-      const uint64_t b_desc0 = smem_desc_sw128(smem_u32(smem) + kATileBytes);
-      const uint64_t m_desc0 = smem_desc_noswizzle(smem_u32(smem) + kATileBytes + KBS * kBTileBytes, 16, 128);
+      const uint64_t a_desc0 = smem_desc_sw128(smem_u32(a_ring));
+      const uint64_t b_desc0 = smem_desc_sw128(smem_u32(b_ring));
+      const uint64_t m_desc0 = smem_desc_noswizzle(smem_u32(a_ring) + kATileBytes, 16, 128);
       // channels left in the last k-block of a tap decide how many MMAs it needs
       const int tail_c = p.C_in - (p.cblocks - 1) * kBlockK;
       const int mma_full = SPARSE ? 2 : 4;
       const int mma_tail = SPARSE ? ((tail_c + 31) >> 5) : ((tail_c + 15) >> 4);
-      int s = 0;
-      uint32_t ph = 0;
+      int sa = 0, sb = 0;
+      uint32_t pha = 0, phb = 0;
       uint32_t tcount = 0;
-      uint32_t gpar = 0;
+      uint32_t mslot = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x, ++tcount) {
         const uint32_t buf = tcount & 1u;
         const uint32_t aph = (tcount >> 1) & 1u;
         if (!mbar_wait_bounded(&bar_acc_empty[buf], aph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * kBN;
+        const uint32_t d_tmem = tmem_base + buf * kAccCol1;
         uint32_t accumulate = 0;
-        int b = 0, cc = 0;
-        for (int it = 0; it < p.iters; ++it) {
-          if (!mbar_wait_bounded(&bar_full[s], ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-          tc_fence_after();
-          const uint64_t a_desc = a_desc0 + (uint64_t)(s * kStageDesc);
-          const uint64_t b_desc_s = b_desc0 + (uint64_t)(s * kStageDesc);
-          int nb = p.kblocks - b;
-          if (nb > KBS) nb = KBS;
-          if (SPARSE) {
-            // two metadata slots of 4 columns, alternating per stage
-            const uint32_t meta_tmem = tmem_base + kMetaCol + 4u * gpar;
-            gpar ^= 1u;
-            tc_cp_128x128b(meta_tmem, m_desc0 + (uint64_t)(s * kStageDesc));
-            for (int j = 0; j < nb; ++j) {
-              const int n_mma = (cc == p.cblocks - 1) ? mma_tail : mma_full;  // 32 dense columns per sparse MMA
-              const uint64_t b_desc = b_desc_s + (uint64_t)(j * kBTileDesc);
-              for (int k2 = 0; k2 < n_mma; ++k2) {
-                const uint32_t kk = 2 * j + k2;  // MMA slot within the stage (= metadata column)
-                // A advances 16 kept values = 32 B, B advances 32 channels = 64 B (descriptor units of 16 B)
-                tc_mma_sparse(d_tmem, a_desc + 2 * kk, b_desc + 4 * k2, meta_tmem + (kk & ~1u), idesc | (kk & 1u),
-                              accumulate);
-                accumulate = 1;
-              }
-              ++b;
-              if (++cc == p.cblocks) cc = 0;
+        int cc = 0, a_sub = 0;
+        uint64_t a_desc = 0;
+        uint32_t meta_tmem = 0;
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (a_sub == 0) {
+            if (!mbar_wait_bounded(&bar_a_full[sa], pha, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+            tc_fence_after();
+            a_desc = a_desc0 + (uint64_t)(sa * kAEntryDesc);
+            if (SPARSE) {
+              // two metadata slots of 4 TMEM columns, alternating per weight tile
+              meta_tmem = tmem_base + kMetaCol + 4u * mslot;
+              mslot ^= 1u;
+              tc_cp_128x128b(meta_tmem, m_desc0 + (uint64_t)(sa * kAEntryDesc));
             }
-          } else {
-            const int n_mma = (cc == p.cblocks - 1) ? mma_tail : mma_full;  // 16 columns per dense MMA
-            for (int kk = 0; kk < n_mma; ++kk) {
-              tc_mma_dense(d_tmem, a_desc + 2 * kk, b_desc_s + 2 * kk, idesc, accumulate);
-              accumulate = 1;
-            }
-            ++b;
-            if (++cc == p.cblocks) cc = 0;
           }
-          tc_commit(&bar_empty[s]);
-          if (++s == STAGES) {
-            s = 0;
-            ph ^= 1u;
+          if (!mbar_wait_bounded(&bar_b_full[sb], phb, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t b_desc = b_desc0 + (uint64_t)(sb * kBTileDesc);
+          const int n_mma = (cc == p.cblocks - 1) ? mma_tail : mma_full;
+          if (SPARSE) {
+            // k-block a_sub of the weight tile: kept values start 64 B in, metadata 2 columns in;
+            // per MMA A advances 16 kept values = 32 B, B 32 channels = 64 B (descriptor units of 16 B)
+            const uint64_t a_kb = a_desc + 4 * a_sub;
+            const uint32_t meta_kb = meta_tmem + 2 * a_sub;
+            tc_mma_sparse(d_tmem, a_kb, b_desc, meta_kb, idesc, accumulate);
+            if (n_mma > 1) tc_mma_sparse(d_tmem, a_kb + 2, b_desc + 4, meta_kb, idesc | 1u, 1);
+          } else {
+            tc_mma_dense(d_tmem, a_desc, b_desc, idesc, accumulate);
+            for (int kk = 1; kk < n_mma; ++kk) tc_mma_dense(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, 1);
+          }
+          accumulate = 1;
+          tc_commit(&bar_b_empty[sb]);
+          if (++sb == kNB) {
+            sb = 0;
+            phb ^= 1u;
+          }
+          if (++cc == p.cblocks) cc = 0;
+          if (++a_sub == APER || kb == p.kblocks - 1) {
+            a_sub = 0;
+            tc_commit(&bar_a_empty[sa]);
+            if (++sa == kNA) {
+              sa = 0;
+              pha ^= 1u;
+            }
           }
         }
         if (ok) tc_commit(&bar_acc_full[buf]);
@@ -233,47 +256,56 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     const int q = warp & 3;  // TMEM lane quadrant this warp may read
     const int row = q * 32 + lane;
     const bool leader = (warp == 2 && lane == 0);
+    const bool relu = (p.flags & SSCONV_FLAG_RELU) != 0;
     uint32_t tcount = 0;
+    uint32_t piece_count = 0;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++tcount) {
-      const int m = tile % p.m_tiles;
-      const int p0 = (tile / p.m_tiles) * kBN;
+      const int pt = tile / p.m_tiles;
+      const int m = tile - pt * p.m_tiles;
+      const int p0 = pt * kBN;
       const uint32_t buf = tcount & 1u;
       const uint32_t aph = (tcount >> 1) & 1u;
       const bool got = mbar_wait_bounded(&bar_acc_full[buf], aph, abort_flag, kWaitLimitCycles);
       // All 128 epilogue threads must take the same branch (they meet at named barriers below):
       // the leader publishes one verdict, everybody reads it after the barrier.
-      if (leader) {
-        epi_go[tcount & 1u] = (got && *abort_flag == 0) ? 1 : 0;
-        bulk_wait_group_read0();  // the previous tile's TMA store has finished reading the staging buffer
-      }
+      if (leader) epi_go[tcount & 1u] = (got && *abort_flag == 0) ? 1 : 0;
       epilogue_bar_sync();
       if (epi_go[tcount & 1u] == 0) break;
       tc_fence_after();
       const int co = m * kTileM + row;
       const float bias_v = ((p.flags & SSCONV_FLAG_BIAS) && co < p.C_out) ? p.bias[co] : 0.0f;
-      const bool relu = (p.flags & SSCONV_FLAG_RELU) != 0;
-      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kBN;
-      uint16_t* stage_col = reinterpret_cast<uint16_t*>(out_stage) + row;
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCol1;
 #pragma unroll 1
-      for (int c0 = 0; c0 < kBN; c0 += 32) {
-        uint32_t r[32];
-        tc_ld_32x32(t_row + c0, r);
-        tc_wait_ld();
+      for (int piece = 0; piece < kBN / kPiece; ++piece, ++piece_count) {
+        uint8_t* stage = out_stage + (piece_count & 1u) * kPieceBytes;
+        // the store issued two pieces ago has finished reading this staging buffer
+        if (leader) bulk_wait_group_read1();
+        epilogue_bar_sync();
+        uint16_t* stage_col = reinterpret_cast<uint16_t*>(stage) + row;
+#pragma unroll 1
+        for (int c0 = 0; c0 < kPiece; c0 += 16) {
+          uint32_t r[16];
+          tc_ld_32x16(t_row + piece * kPiece + c0, r);
+          tc_wait_ld();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          float v = __uint_as_float(r[j]) + bias_v;
-          if (relu) v = fmaxf(v, 0.0f);
-          stage_col[(c0 + j) * 128] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+          for (int j = 0; j < 16; ++j) {
+            float v = __uint_as_float(r[j]) + bias_v;
+            if (relu) v = fmaxf(v, 0.0f);
+            stage_col[(c0 + j) * 128] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+          }
         }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
-      fence_proxy_async_smem();
-      epilogue_bar_sync();
-      if (leader) {
-        tma_store_2d(&tm_y, out_stage, m * kTileM, p0);
-        bulk_commit_group();
+        if (piece == kBN / kPiece - 1) {
+          // accumulator fully read: hand it back to the MMA thread
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
+        }
+        fence_proxy_async_smem();
+        epilogue_bar_sync();
+        if (leader) {
+          tma_store_2d(&tm_y, stage, m * kTileM, p0 + piece * kPiece);
+          bulk_commit_group();
+        }
       }
     }
     if (leader) bulk_wait_group0();
@@ -395,7 +427,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   {
     cuuint64_t dims[2] = {(cuuint64_t)d.C_out, (cuuint64_t)P};
     cuuint64_t strides[1] = {(cuuint64_t)d.C_out * 2};
-    cuuint32_t box[2] = {(cuuint32_t)kTileM, (cuuint32_t)kBN};
+    cuuint32_t box[2] = {(cuuint32_t)kTileM, (cuuint32_t)kPiece};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode_tiled(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, dims, strides, box, estr,
                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
@@ -421,7 +453,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.m_tiles = geo.m_tiles;
   const long long p_tiles = (P + kBN - 1) / kBN;
   p.num_tiles = (int)(p_tiles * geo.m_tiles);
-  p.iters = SPARSE ? geo.stages : geo.kblocks;
+  p.a_tiles = SPARSE ? geo.stages : geo.kblocks;
   p.flags = d.flags;
   p.bias = bias;
   p.meta = static_cast<const uint8_t*>(meta);
