@@ -73,8 +73,9 @@ int32_t ssconv_out_shape(const ssconv_desc_t* desc, int32_t* H_out, int32_t* W_o
 
 /* Sizes for a layer: number of groups G = C_out*K/4, bytes of the compressed value
  * blob and of the metadata blob written by ssconv_compress, and workspace bytes the two
- * forward calls need (may be 0).  Any output pointer may be NULL.  The blobs are padded
- * to whole tiles, so they can be slightly larger than C_out*K and C_out*K/8 bytes. */
+ * forward calls may need.  Any output pointer may be NULL.  The blobs are padded to whole
+ * tiles, so they can be slightly larger than C_out*K and C_out*K/8 bytes.  The workspace
+ * size is the same for every layer (about 36 MB), so one buffer serves a whole network. */
 int32_t ssconv_sizes(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes,
                      size_t* meta_bytes, size_t* ws_bytes_sparse, size_t* ws_bytes_dense);
 
@@ -112,7 +113,16 @@ int32_t ssconv_decompress(const ssconv_desc_t* desc, const void* w_comp, const v
  * result is rounded once to bf16 (nearest even).  act = ReLU if SSCONV_FLAG_RELU, bias is
  * read only if SSCONV_FLAG_BIAS.
  * x, y, w_comp, meta: device, 16-byte aligned.  Needs C_in % 8 == 0, C_out % 8 == 0,
- * pad <= 127, dil*(K-1) <= 255, stride <= 8.  ws may be NULL when ssconv_sizes reports 0.
+ * pad <= 127, dil*(K-1) <= 255, stride <= 8.
+ * ws: device scratch of at least the size ssconv_sizes reports, 16-byte aligned.  It is used
+ * only by layers with too few output tiles to fill the GPU, whose K range is then split over
+ * several thread blocks that park fp32 partial results there and sum them in a fixed order,
+ * so results are reproducible.  Contract: the caller zero-fills ws once (only the counters at
+ * its end must be zero, the rest is overwritten before it is read); every call that completes
+ * leaves the counters zero, so ws can be reused by later calls on the same stream.  Calls
+ * that may overlap on the GPU need separate workspaces.  After SSCONV_ERR_TIMEOUT zero-fill
+ * it again.  If ws is NULL or too small and
+ * the layer needs it, SSCONV_ERR_WORKSPACE is returned and nothing is launched.
  * dev_status (nullable): device int32; a kernel whose bounded wait expires stores
  * SSCONV_ERR_TIMEOUT there and drains instead of hanging; it is never written on success,
  * so the caller zeroes it once and reads it after its own synchronisation. */

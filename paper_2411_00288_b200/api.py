@@ -171,6 +171,21 @@ def ssconv_decompress(desc: Desc, w_comp: torch.Tensor, meta: torch.Tensor, want
     return w_out, pat
 
 
+_workspaces = {}
+
+
+def default_workspace(device) -> torch.Tensor:
+    """One zero-filled scratch buffer per device, shared by calls that pass ws=None.  The forward
+    kernels leave it zero-filled, so stream-ordered calls can share it; calls on different streams
+    that may overlap must pass their own."""
+    dev = torch.device(device)
+    key = dev.index if dev.index is not None else torch.cuda.current_device()
+    if key not in _workspaces:
+        nbytes = ssconv_sizes(make_desc(1, 8, 8, 8, 8, 1, 1)).ws_bytes_sparse
+        _workspaces[key] = torch.zeros((nbytes,), dtype=torch.uint8, device=torch.device("cuda", key))
+    return _workspaces[key]
+
+
 def _alloc_y(desc: Desc, x: torch.Tensor) -> torch.Tensor:
     ho, wo = ssconv_out_shape(desc)
     return torch.empty((desc.N, ho, wo, desc.C_out), dtype=torch.bfloat16, device=x.device)
@@ -184,6 +199,8 @@ def ssconv_forward(desc: Desc, x: torch.Tensor, w_comp: torch.Tensor, meta: torc
     _need_cuda(x, w_comp, meta, bias, y, ws, dev_status)
     if y is None:
         y = _alloc_y(desc, x)
+    if ws is None:
+        ws = default_workspace(x.device)
     _check("ssconv_forward", lib().ssconv_forward(
         ctypes.byref(desc), _ptr(x), _ptr(w_comp), _ptr(meta), _ptr(bias), _ptr(y), _ptr(ws),
         0 if ws is None else ws.numel() * ws.element_size(), _ptr(dev_status), _stream(stream)))
@@ -197,6 +214,8 @@ def ssconv_forward_dense(desc: Desc, x: torch.Tensor, w: torch.Tensor, bias: Opt
     _need_cuda(x, w, bias, y, ws, dev_status)
     if y is None:
         y = _alloc_y(desc, x)
+    if ws is None:
+        ws = default_workspace(x.device)
     _check("ssconv_forward_dense", lib().ssconv_forward_dense(
         ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _ptr(ws),
         0 if ws is None else ws.numel() * ws.element_size(), _ptr(dev_status), _stream(stream)))

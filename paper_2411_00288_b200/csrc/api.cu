@@ -12,9 +12,11 @@ cudaError_t launch_compress(const ssconv_desc_t& d, const void* w, const uint8_t
 cudaError_t launch_decompress(const ssconv_desc_t& d, const void* w_comp, const void* meta, void* w_out,
                               uint8_t* pattern_out, cudaStream_t st);
 int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
-                              const float* bias, void* y, int32_t* dev_status, cudaStream_t stream);
+                              const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
+                              cudaStream_t stream);
 int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias, void* y,
-                             int32_t* dev_status, cudaStream_t stream);
+                             void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream);
+size_t workspace_bytes();
 }  // namespace ssconv
 
 namespace {
@@ -93,8 +95,8 @@ int32_t ssconv_sizes(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes
   if (G) *G = (int64_t)desc->C_out * geo.taps * (desc->C_in / 4);
   if (w_comp_bytes) *w_comp_bytes = (size_t)geo.Mp * geo.KC * 2;
   if (meta_bytes) *meta_bytes = (size_t)geo.m_tiles * geo.stages * ssconv::kMetaImageBytes;
-  if (ws_bytes_sparse) *ws_bytes_sparse = 0;
-  if (ws_bytes_dense) *ws_bytes_dense = 0;
+  if (ws_bytes_sparse) *ws_bytes_sparse = ssconv::workspace_bytes();
+  if (ws_bytes_dense) *ws_bytes_dense = ssconv::workspace_bytes();
   return SSCONV_OK;
 }
 
@@ -135,26 +137,23 @@ int32_t ssconv_decompress(const ssconv_desc_t* desc, const void* w_comp, const v
 
 int32_t ssconv_forward(const ssconv_desc_t* desc, const void* x, const void* w_comp, const void* meta,
                        const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
-  (void)ws;
-  (void)ws_bytes;
   int32_t rc = check_desc(desc, true);
   if (rc != SSCONV_OK) return rc;
   if (!x || !w_comp || !meta || !y) return SSCONV_ERR_NULL;
   if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
   if (!aligned16(x) || !aligned16(w_comp) || !aligned16(meta) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
-  return ssconv::launch_forward_sparse(*desc, x, w_comp, meta, bias, y, dev_status, (cudaStream_t)stream);
+  return ssconv::launch_forward_sparse(*desc, x, w_comp, meta, bias, y, ws, ws_bytes, dev_status,
+                                       (cudaStream_t)stream);
 }
 
 int32_t ssconv_forward_dense(const ssconv_desc_t* desc, const void* x, const void* w_bf16, const float* bias,
                              void* y, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
-  (void)ws;
-  (void)ws_bytes;
   int32_t rc = check_desc(desc, true);
   if (rc != SSCONV_OK) return rc;
   if (!x || !w_bf16 || !y) return SSCONV_ERR_NULL;
   if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
   if (!aligned16(x) || !aligned16(w_bf16) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
-  return ssconv::launch_forward_dense(*desc, x, w_bf16, bias, y, dev_status, (cudaStream_t)stream);
+  return ssconv::launch_forward_dense(*desc, x, w_bf16, bias, y, ws, ws_bytes, dev_status, (cudaStream_t)stream);
 }
 
 }  // extern "C"

@@ -14,9 +14,17 @@
 //               sparse weight tile spans two activation tiles (128 dense columns).
 //   warp 1      owns TMEM; one thread copies metadata smem->TMEM and issues the MMAs into one of
 //               two fp32 accumulators (128 lanes x 240 columns each).
-//   warps 2-5   epilogue: TMEM -> registers, + bias, ReLU, bf16, transpose through shared
-//               memory to pixel-major rows, TMA stores of 80-pixel pieces (clipped at the
-//               tensor edge) from a double-buffered staging area.
+//   warps 2-9   epilogue, two groups of four warps, each owning half of the tile's pixel columns:
+//               TMEM -> registers, + bias, ReLU, bf16, transpose through shared memory to
+//               pixel-major rows, TMA stores of 40-pixel pieces (clipped at the tensor edge)
+//               from a double-buffered staging area per group.
+// Work partition: the unit of work is one weight tile's worth of K for one output tile.  Either
+// every CTA takes a contiguous block of whole output tiles, or (when whole tiles would leave many
+// SMs idle) the units are dealt out evenly, so a CTA's range may start and end inside an
+// output tile ("stream-K").  A CTA writes a partly computed tile (fp32) to a scratch region of its
+// own in global memory and bumps the tile's counter; the last CTA to arrive sums the regions of all
+// contributors in a fixed order, finishes the epilogue and resets the counter.  No CTA ever waits
+// for another, and the result does not depend on the order of arrival.
 // All mbarrier waits are bounded; when one runs out the CTA raises a flag, every role leaves
 // its loop, TMEM is freed and SSCONV_ERR_TIMEOUT is stored to *dev_status.
 #include <cuda.h>
@@ -30,15 +38,17 @@
 namespace ssconv {
 
 constexpr int kBN = 240;                 // pixels per tile (N of the MMA)
-constexpr int kPiece = 80;               // pixels per epilogue store
-constexpr int kThreads = 192;
+constexpr int kGroups = 2;               // epilogue warp groups, each owning kBN / kGroups pixel columns
+constexpr int kGroupCols = kBN / kGroups;
+constexpr int kPiece = 40;               // pixels per epilogue store
+constexpr int kThreads = 64 + 128 * kGroups;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kAccCol1 = 256;       // second accumulator; the first starts at column 0
 constexpr uint32_t kMetaCol = kBN;       // metadata: 2 slots x 4 columns in [240, 248)
 constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 1.9 GHz
 constexpr uint32_t kATileBytes = 128 * 128;          // 128 rows x 128 B
 constexpr uint32_t kBTileBytes = kBN * 128;          // 240 pixels x 64 channels bf16
-constexpr uint32_t kPieceBytes = kPiece * 256;       // 80 pixels x 128 channels bf16
+constexpr uint32_t kPieceBytes = kPiece * 256;       // 40 pixels x 128 channels bf16
 constexpr int kNA = 3;                               // weight ring depth
 constexpr int kNB = 4;                               // activation ring depth
 
@@ -49,7 +59,7 @@ struct Cfg {
   static constexpr uint32_t kAEntryBytes = kATileBytes + kMetaBytes;
   static constexpr uint32_t kBarrierBytes = 256;
   static constexpr uint32_t kSmemBytes =
-      kNA * kAEntryBytes + kNB * kBTileBytes + 2 * kPieceBytes + kBarrierBytes + 1024;
+      kNA * kAEntryBytes + kNB * kBTileBytes + 2 * kGroups * kPieceBytes + kBarrierBytes + 1024;
 };
 
 struct FwdParams {
@@ -58,13 +68,73 @@ struct FwdParams {
   int cblocks, kblocks;
   int m_tiles, num_tiles;
   int a_tiles;  // weight tiles per output tile
+  int split;    // 1: units dealt out evenly across CTAs (stream-K); 0: whole tiles per CTA
+  long long units;  // num_tiles * a_tiles
+  float4* ws_regions;  // [2 * gridDim.x] regions of 128 x 240 fp32: a CTA's partial tiles
+  int* ws_counters;    // [gridDim.x][2] arrivals per split tile and epilogue group, zero between launches
   uint32_t flags;
   const float* bias;
   const uint8_t* meta;
   int32_t* dev_status;
 };
 
-__device__ __forceinline__ void epilogue_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Weight-tile range [a0, a1) of one output tile: what a CTA computes in one accumulator pass.
+struct Segment {
+  int tile, a0, a1;
+};
+
+// Walks the segments of this CTA's contiguous range of work units.
+struct WorkIter {
+  long long u, u_end;
+  int A;
+  __device__ WorkIter(const FwdParams& p) {
+    A = p.a_tiles;
+    const long long c = blockIdx.x, G = gridDim.x;
+    if (p.split) {
+      u = c * p.units / G;
+      u_end = (c + 1) * p.units / G;
+    } else {
+      u = (c * p.num_tiles / G) * A;
+      u_end = ((c + 1) * p.num_tiles / G) * A;
+    }
+  }
+  __device__ bool next(Segment& s) {
+    if (u >= u_end) return false;
+    s.tile = (int)(u / A);
+    s.a0 = (int)(u - (long long)s.tile * A);
+    const long long left = u_end - u;
+    s.a1 = (left >= A - s.a0) ? A : s.a0 + (int)left;
+    u += s.a1 - s.a0;
+    return true;
+  }
+};
+
+// CTA that owns work unit u under the even split: the c with c*U/G <= u < (c+1)*U/G.
+__device__ __forceinline__ int unit_owner(long long u, long long U, long long G) {
+  return (int)(((u + 1) * G - 1) / U);
+}
+
+// A scratch region holds one 128 x 240 fp32 partial tile as float4s ordered [4-column group][row],
+// so that a warp reads or writes 512 contiguous bytes at a time.
+constexpr int kRegionVecs = kTileM * kBN / 4;
+__device__ __forceinline__ int region_vec(int col4, int row) { return col4 * kTileM + row; }
+// Region of CTA c for a split tile: its range starts inside the tile (0) or the tile starts inside
+// its range (1).  A range has at most one segment of each kind.
+__device__ __forceinline__ size_t region_index(int c, bool tile_starts_here) { return 2 * (size_t)c + (tile_starts_here ? 1 : 0); }
+
+__device__ __forceinline__ void epilogue_bar_sync(int group) {
+  asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory");
+}
+// One epilogue piece (40 accumulator columns of this thread's lane) from TMEM; no wait.
+__device__ __forceinline__ void tc_ld_piece(uint32_t taddr, uint32_t (&r)[kPiece]) {
+  uint32_t a[32], b[8];
+  tc_ld_32x32(taddr, a);
+  tc_ld_32x8(taddr + 32, b);
+#pragma unroll
+  for (int j = 0; j < 32; ++j) r[j] = a[j];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) r[32 + j] = b[j];
+}
 
 template <bool SPARSE>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -78,7 +148,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   uint8_t* a_ring = smem;
   uint8_t* b_ring = a_ring + kNA * C::kAEntryBytes;
   uint8_t* out_stage = b_ring + kNB * kBTileBytes;
-  uint64_t* bar_a_full = reinterpret_cast<uint64_t*>(out_stage + 2 * kPieceBytes);
+  uint64_t* bar_a_full = reinterpret_cast<uint64_t*>(out_stage + 2 * kGroups * kPieceBytes);
   uint64_t* bar_a_empty = bar_a_full + kNA;
   uint64_t* bar_b_full = bar_a_empty + kNA;
   uint64_t* bar_b_empty = bar_b_full + kNB;
@@ -86,7 +156,8 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   uint64_t* bar_acc_empty = bar_acc_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* epi_go = abort_flag + 1;  // two slots: the epilogue leader's go/stop verdict per tile
+  volatile int* epi_go = abort_flag + 1;         // per group two slots: the leader's go/stop verdict per tile
+  volatile int* epi_last = epi_go + 2 * kGroups;  // per group: partial tile, is this CTA the last to arrive?
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -102,7 +173,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bar_acc_full[b], 1);
-      mbar_init(&bar_acc_empty[b], 4);
+      mbar_init(&bar_acc_empty[b], 4 * kGroups);
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -125,9 +196,11 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       int sa = 0, sb = 0;
       uint32_t pha = 0, phb = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
-        const int pt = tile / p.m_tiles;
-        const int m = tile - pt * p.m_tiles;
+      WorkIter work(p);
+      Segment seg;
+      while (ok && work.next(seg)) {
+        const int pt = seg.tile / p.m_tiles;
+        const int m = seg.tile - pt * p.m_tiles;
         const int p0 = pt * kBN;
         const int n0 = p0 / p.HoWo;
         const int rem = p0 - n0 * p.HoWo;
@@ -135,9 +208,16 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         const int wo0 = rem - ho0 * p.Wo;
         const int base_w = wo0 * p.stride_w - p.pad_w;
         const int base_h = ho0 * p.stride_h - p.pad_h;
-        const uint8_t* meta_src = p.meta + (size_t)m * p.a_tiles * kMetaImageBytes;
-        int cc = 0, tap = 0, off_w = 0, off_h = 0, kw = 0, a_idx = 0, a_sub = 0;
-        for (int kb = 0; kb < p.kblocks; ++kb) {
+        const uint8_t* meta_src = p.meta + ((size_t)m * p.a_tiles + seg.a0) * kMetaImageBytes;
+        const int kb0 = seg.a0 * APER;
+        const int kb1 = (seg.a1 * APER < p.kblocks) ? seg.a1 * APER : p.kblocks;
+        int tap = kb0 / p.cblocks;
+        int cc = kb0 - tap * p.cblocks;
+        const int kh0 = tap / p.KW;
+        int kw = tap - kh0 * p.KW;
+        int off_w = kw * p.dil_w, off_h = kh0 * p.dil_h;
+        int a_idx = seg.a0, a_sub = 0;
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (a_sub == 0) {
             if (!mbar_wait_bounded(&bar_a_empty[sa], pha ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
             uint8_t* st = a_ring + sa * C::kAEntryBytes;
@@ -195,17 +275,21 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       uint32_t tcount = 0;
       uint32_t mslot = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x, ++tcount) {
+      WorkIter work(p);
+      Segment seg;
+      for (; ok && work.next(seg); ++tcount) {
         const uint32_t buf = tcount & 1u;
         const uint32_t aph = (tcount >> 1) & 1u;
         if (!mbar_wait_bounded(&bar_acc_empty[buf], aph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kAccCol1;
         uint32_t accumulate = 0;
-        int cc = 0, a_sub = 0;
+        const int kb0 = seg.a0 * APER;
+        const int kb1 = (seg.a1 * APER < p.kblocks) ? seg.a1 * APER : p.kblocks;
+        int cc = kb0 % p.cblocks, a_sub = 0;
         uint64_t a_desc = 0;
         uint32_t meta_tmem = 0;
-        for (int kb = 0; kb < p.kblocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (a_sub == 0) {
             if (!mbar_wait_bounded(&bar_a_full[sa], pha, abort_flag, kWaitLimitCycles)) { ok = false; break; }
             tc_fence_after();
@@ -239,7 +323,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             phb ^= 1u;
           }
           if (++cc == p.cblocks) cc = 0;
-          if (++a_sub == APER || kb == p.kblocks - 1) {
+          if (++a_sub == APER || kb == kb1 - 1) {
             a_sub = 0;
             tc_commit(&bar_a_empty[sa]);
             if (++sa == kNA) {
@@ -253,60 +337,120 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     }
   } else {
     // ------------------------------------------------------------------ epilogue
+    // Two independent groups of four warps; group g owns pixel columns [120 g, 120 g + 120) of
+    // every tile, with its own staging buffers, named barrier, leader and TMA stores.
+    const int grp = (warp - 2) >> 2;
     const int q = warp & 3;  // TMEM lane quadrant this warp may read
     const int row = q * 32 + lane;
-    const bool leader = (warp == 2 && lane == 0);
+    const bool leader = (q == 2 && lane == 0);  // first warp of each group
     const bool relu = (p.flags & SSCONV_FLAG_RELU) != 0;
+    const int col_base = grp * kGroupCols;
+    uint8_t* my_stage = out_stage + grp * 2 * kPieceBytes;
+    volatile int* my_go = epi_go + 2 * grp;
+    volatile int* my_last = epi_last + grp;
     uint32_t tcount = 0;
     uint32_t piece_count = 0;
-    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++tcount) {
-      const int pt = tile / p.m_tiles;
-      const int m = tile - pt * p.m_tiles;
-      const int p0 = pt * kBN;
+    WorkIter work(p);
+    Segment seg;
+    for (; work.next(seg); ++tcount) {
+      const int pt = seg.tile / p.m_tiles;
+      const int m = seg.tile - pt * p.m_tiles;
+      const int p0 = pt * kBN + col_base;
       const uint32_t buf = tcount & 1u;
       const uint32_t aph = (tcount >> 1) & 1u;
       const bool got = mbar_wait_bounded(&bar_acc_full[buf], aph, abort_flag, kWaitLimitCycles);
-      // All 128 epilogue threads must take the same branch (they meet at named barriers below):
+      // All threads of a group must take the same branch (they meet at named barriers below):
       // the leader publishes one verdict, everybody reads it after the barrier.
-      if (leader) epi_go[tcount & 1u] = (got && *abort_flag == 0) ? 1 : 0;
-      epilogue_bar_sync();
-      if (epi_go[tcount & 1u] == 0) break;
+      if (leader) my_go[tcount & 1u] = (got && *abort_flag == 0) ? 1 : 0;
+      epilogue_bar_sync(grp);
+      if (my_go[tcount & 1u] == 0) break;
       tc_fence_after();
       const int co = m * kTileM + row;
       const float bias_v = ((p.flags & SSCONV_FLAG_BIAS) && co < p.C_out) ? p.bias[co] : 0.0f;
-      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCol1;
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCol1 + col_base;
+      const bool whole = (seg.a0 == 0 && seg.a1 == p.a_tiles);
+      int c_first = 0, c_last = 0;
+      if (!whole) {
+        // ---- partial tile: park this CTA's share in its own scratch region --------------------
+        const long long u_first = (long long)seg.tile * p.a_tiles;
+        c_first = unit_owner(u_first, p.units, gridDim.x);
+        c_last = unit_owner(u_first + p.a_tiles - 1, p.units, gridDim.x);
+        float4* mine = p.ws_regions + region_index(blockIdx.x, seg.a0 == 0) * kRegionVecs;
 #pragma unroll 1
-      for (int piece = 0; piece < kBN / kPiece; ++piece, ++piece_count) {
-        uint8_t* stage = out_stage + (piece_count & 1u) * kPieceBytes;
-        // the store issued two pieces ago has finished reading this staging buffer
-        if (leader) bulk_wait_group_read1();
-        epilogue_bar_sync();
-        uint16_t* stage_col = reinterpret_cast<uint16_t*>(stage) + row;
-#pragma unroll 1
-        for (int c0 = 0; c0 < kPiece; c0 += 16) {
-          uint32_t r[16];
-          tc_ld_32x16(t_row + piece * kPiece + c0, r);
+        for (int c0 = 0; c0 < kGroupCols; c0 += kPiece) {
+          uint32_t r[kPiece];
+          tc_ld_piece(t_row + c0, r);
           tc_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            float v = __uint_as_float(r[j]) + bias_v;
-            if (relu) v = fmaxf(v, 0.0f);
-            stage_col[(c0 + j) * 128] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+          for (int j = 0; j < kPiece / 4; ++j)
+            __stcg(mine + region_vec((col_base + c0) / 4 + j, row),
+                   make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                               __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3])));
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
+        __threadfence();
+        epilogue_bar_sync(grp);
+        if (leader) {
+          const int arrived = atomicAdd(p.ws_counters + 2 * c_first + grp, 1);
+          *my_last = (arrived == c_last - c_first) ? 1 : 0;
+        }
+        epilogue_bar_sync(grp);
+        if (*my_last == 0) continue;  // someone else finishes this half tile
+        __threadfence();
+      }
+      // ---- finish the tile: bias, activation, bf16, transpose through smem, TMA store -----------
+#pragma unroll 1
+      for (int piece = 0; piece < kGroupCols / kPiece; ++piece, ++piece_count) {
+        uint8_t* stage = my_stage + (piece_count & 1u) * kPieceBytes;
+        uint32_t r[kPiece];
+        if (whole) {
+          tc_ld_piece(t_row + piece * kPiece, r);
+        } else {
+          // sum the contributors' regions in CTA order (reads bypass L1: the data came from other SMs)
+#pragma unroll
+          for (int j = 0; j < kPiece; ++j) r[j] = 0u;
+          const int v0 = (col_base + piece * kPiece) / 4;
+          for (int c = c_first; c <= c_last; ++c) {
+            const float4* src = p.ws_regions + region_index(c, c == c_first) * kRegionVecs;
+            float4 v[kPiece / 4];
+#pragma unroll
+            for (int j = 0; j < kPiece / 4; ++j) v[j] = __ldcg(src + region_vec(v0 + j, row));
+#pragma unroll
+            for (int j = 0; j < kPiece / 4; ++j) {
+              r[4 * j] = __float_as_uint(__uint_as_float(r[4 * j]) + v[j].x);
+              r[4 * j + 1] = __float_as_uint(__uint_as_float(r[4 * j + 1]) + v[j].y);
+              r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + v[j].z);
+              r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + v[j].w);
+            }
           }
         }
-        if (piece == kBN / kPiece - 1) {
-          // accumulator fully read: hand it back to the MMA thread
+        // the store issued two pieces ago has finished reading this staging buffer
+        if (leader) bulk_wait_group_read1();
+        if (whole) tc_wait_ld();
+        epilogue_bar_sync(grp);
+        uint16_t* stage_col = reinterpret_cast<uint16_t*>(stage) + row;
+#pragma unroll
+        for (int j = 0; j < kPiece; ++j) {
+          float v = __uint_as_float(r[j]) + bias_v;
+          if (relu) v = fmaxf(v, 0.0f);
+          stage_col[j * 128] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+        }
+        if (whole && piece == kGroupCols / kPiece - 1) {
+          // this warp's part of the accumulator is read: hand it back to the MMA thread
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
         }
         fence_proxy_async_smem();
-        epilogue_bar_sync();
+        epilogue_bar_sync(grp);
         if (leader) {
           tma_store_2d(&tm_y, stage, m * kTileM, p0 + piece * kPiece);
           bulk_commit_group();
         }
       }
+      if (!whole && leader) p.ws_counters[2 * c_first + grp] = 0;
     }
     if (leader) bulk_wait_group0();
   }
@@ -359,12 +503,20 @@ static int out_extent(int in, int k, int stride, int pad, int dil) {
   return span < 0 ? 0 : span / stride + 1;
 }
 
+// Scratch for partly computed tiles: two fp32 regions (128 x 240) and two counters per CTA.
+constexpr int kMaxWorkers = 148;
+constexpr size_t kRegionBytes = (size_t)kTileM * kBN * sizeof(float);
+constexpr double kCyclesPerATile = 1200.0;
+constexpr double kSplitFixedCycles = 18000.0;
+size_t workspace_bytes() { return 2 * (size_t)kMaxWorkers * kRegionBytes + 2 * (size_t)kMaxWorkers * sizeof(int); }
+
 static int g_sm_count[64] = {0};
 static bool g_attr_set[64][2] = {{false}};
 
 template <bool SPARSE>
 static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const void* weights, const void* meta,
-                                   const float* bias, void* y, int32_t* dev_status, cudaStream_t stream) {
+                                   const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
+                                   cudaStream_t stream) {
   if (!load_driver_entry_points()) return SSCONV_ERR_CUDA;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SSCONV_ERR_CUDA;
@@ -459,18 +611,39 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.meta = static_cast<const uint8_t*>(meta);
   p.dev_status = dev_status;
 
-  int grid = p.num_tiles < g_sm_count[dev] ? p.num_tiles : g_sm_count[dev];
+  p.units = (long long)p.num_tiles * p.a_tiles;
+  int workers = g_sm_count[dev] < kMaxWorkers ? g_sm_count[dev] : kMaxWorkers;
+  // Whole tiles per CTA, unless dealing the K range out evenly is clearly faster by a simple
+  // cost model: cycles per weight tile in the main loop, and a fixed cost for parking, summing
+  // and finishing partial tiles (both measured on B200).
+  const int waves = (p.num_tiles + workers - 1) / workers;
+  const double whole_cost = (double)waves * p.a_tiles * kCyclesPerATile;
+  const double split_cost = (double)p.units / workers * kCyclesPerATile + kSplitFixedCycles;
+  p.split = (p.a_tiles > 1 && whole_cost > 1.15 * split_cost) ? 1 : 0;
+  int grid;
+  if (p.split) {
+    grid = p.units < workers ? (int)p.units : workers;
+    if (ws == nullptr || ws_bytes < workspace_bytes()) return SSCONV_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(ws) & 15u) return SSCONV_ERR_ALIGNMENT;
+    p.ws_regions = static_cast<float4*>(ws);
+    p.ws_counters = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + 2 * (size_t)kMaxWorkers * kRegionBytes);
+  } else {
+    grid = p.num_tiles < workers ? p.num_tiles : workers;
+    p.ws_regions = nullptr;
+    p.ws_counters = nullptr;
+  }
   ssconv_fwd_kernel<SPARSE><<<grid, kThreads, C::kSmemBytes, stream>>>(tm_a, tm_b, tm_y, p);
   return cudaGetLastError() == cudaSuccess ? SSCONV_OK : SSCONV_ERR_CUDA;
 }
 
 int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
-                              const float* bias, void* y, int32_t* dev_status, cudaStream_t stream) {
-  return launch_forward_impl<true>(d, x, w_comp, meta, bias, y, dev_status, stream);
+                              const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
+                              cudaStream_t stream) {
+  return launch_forward_impl<true>(d, x, w_comp, meta, bias, y, ws, ws_bytes, dev_status, stream);
 }
 int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias, void* y,
-                             int32_t* dev_status, cudaStream_t stream) {
-  return launch_forward_impl<false>(d, x, w, nullptr, bias, y, dev_status, stream);
+                             void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream) {
+  return launch_forward_impl<false>(d, x, w, nullptr, bias, y, ws, ws_bytes, dev_status, stream);
 }
 
 }  // namespace ssconv
