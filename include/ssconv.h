@@ -137,6 +137,34 @@ int32_t ssconv_forward_dense(const ssconv_desc_t* desc, const void* x, const voi
                              const float* bias, void* y, void* ws, size_t ws_bytes,
                              int32_t* dev_status, void* stream);
 
+/* ssconv_forward for callers that have no way to provide scratch memory.  (The paper has no
+ * counterpart to this call; it exists for integration only.)
+ *
+ * Some hosts of this library may not allocate on the device at all once they are running: an
+ * inference server that hands every component a fixed arena at start-up, a real-time loop where
+ * cudaMalloc's implicit synchronisation is unacceptable, a plug-in inside a process whose memory
+ * pool is owned by someone else.  For them the scratch that ssconv_forward takes as `ws` is
+ * compiled into the library: a fixed device array of about 15.7 MB (room for 64 thread blocks),
+ * which every GPU that loads the library holds until the process exits.  The call allocates
+ * nothing: no cudaMalloc, no cudaFree, no allocating library routine.
+ *
+ * Same arguments, formula, layouts and error codes as ssconv_forward, without ws.  Differences:
+ *  - Only small layers are accepted, the ones whose K range is worth splitting across thread
+ *    blocks: at most 64 output tiles (a tile is 128 output channels x 240 pixels); larger layers
+ *    return SSCONV_ERR_UNSUPPORTED_SHAPE and should go through ssconv_forward, which needs no
+ *    scratch for them (ws = NULL is accepted there).
+ *  - The K range is always split, over at most 64 thread blocks, so the fp32 summation order,
+ *    and with it the last bits of y, can differ from ssconv_forward's.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call outside any stream capture.
+ *  - All calls share the one array, and it keeps what the previous call left in it.  Each call
+ *    clears the arrival counters it relies on before its kernel runs (stream-ordered), so calls
+ *    issued one after another on one stream are safe; two calls that can overlap on the GPU
+ *    (different streams, no dependency) race on the array and give wrong results. */
+int32_t ssconv_forward_static_ws(const ssconv_desc_t* desc, const void* x, const void* w_comp,
+                                 const void* meta, const float* bias, void* y, int32_t* dev_status,
+                                 void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,8 @@ ERR_TIMEOUT = 8
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.so")
 EXPORTS = ("ssconv_version", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes", "ssconv_select_mask",
-           "ssconv_compress", "ssconv_decompress", "ssconv_forward", "ssconv_forward_dense")
+           "ssconv_compress", "ssconv_decompress", "ssconv_forward", "ssconv_forward_dense",
+           "ssconv_forward_static_ws")
 
 
 class SsconvError(RuntimeError):
@@ -84,6 +85,8 @@ def lib():
         L.ssconv_forward.argtypes = [dp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         L.ssconv_forward_dense.restype = i32
         L.ssconv_forward_dense.argtypes = [dp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.ssconv_forward_static_ws.restype = i32
+        L.ssconv_forward_static_ws.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -219,4 +222,17 @@ def ssconv_forward_dense(desc: Desc, x: torch.Tensor, w: torch.Tensor, bias: Opt
     _check("ssconv_forward_dense", lib().ssconv_forward_dense(
         ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _ptr(ws),
         0 if ws is None else ws.numel() * ws.element_size(), _ptr(dev_status), _stream(stream)))
+    return y
+
+
+def ssconv_forward_static_ws(desc: Desc, x: torch.Tensor, w_comp: torch.Tensor, meta: torch.Tensor,
+                             bias: Optional[torch.Tensor], y: torch.Tensor,
+                             dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """ssconv_forward with the library's built-in scratch: for callers that must not allocate device
+    memory.  Nothing is allocated here either, so the caller passes the output tensor y.  Small
+    layers only (at most 64 output tiles); calls that overlap on the GPU race on the shared scratch."""
+    _need_cuda(x, w_comp, meta, bias, y, dev_status)
+    _check("ssconv_forward_static_ws", lib().ssconv_forward_static_ws(
+        ctypes.byref(desc), _ptr(x), _ptr(w_comp), _ptr(meta), _ptr(bias), _ptr(y), _ptr(dev_status),
+        _stream(stream)))
     return y

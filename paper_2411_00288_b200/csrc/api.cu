@@ -17,6 +17,8 @@ int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void*
 int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias, void* y,
                              void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream);
 size_t workspace_bytes();
+int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
+                                 const float* bias, void* y, int32_t* dev_status, cudaStream_t stream);
 }  // namespace ssconv
 
 namespace {
@@ -154,6 +156,16 @@ int32_t ssconv_forward_dense(const ssconv_desc_t* desc, const void* x, const voi
   if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
   if (!aligned16(x) || !aligned16(w_bf16) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
   return ssconv::launch_forward_dense(*desc, x, w_bf16, bias, y, ws, ws_bytes, dev_status, (cudaStream_t)stream);
+}
+
+int32_t ssconv_forward_static_ws(const ssconv_desc_t* desc, const void* x, const void* w_comp, const void* meta,
+                                 const float* bias, void* y, int32_t* dev_status, void* stream) {
+  int32_t rc = check_desc(desc, true);
+  if (rc != SSCONV_OK) return rc;
+  if (!x || !w_comp || !meta || !y) return SSCONV_ERR_NULL;
+  if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
+  if (!aligned16(x) || !aligned16(w_comp) || !aligned16(meta) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_forward_static_ws(*desc, x, w_comp, meta, bias, y, dev_status, (cudaStream_t)stream);
 }
 
 }  // extern "C"

@@ -508,7 +508,10 @@ constexpr int kMaxWorkers = 148;
 constexpr size_t kRegionBytes = (size_t)kTileM * kBN * sizeof(float);
 constexpr double kCyclesPerATile = 1200.0;
 constexpr double kSplitFixedCycles = 18000.0;
-size_t workspace_bytes() { return 2 * (size_t)kMaxWorkers * kRegionBytes + 2 * (size_t)kMaxWorkers * sizeof(int); }
+constexpr size_t scratch_bytes(int workers) {
+  return 2 * (size_t)workers * kRegionBytes + 2 * (size_t)workers * sizeof(int);
+}
+size_t workspace_bytes() { return scratch_bytes(kMaxWorkers); }
 
 static int g_sm_count[64] = {0};
 static bool g_attr_set[64][2] = {{false}};
@@ -516,7 +519,7 @@ static bool g_attr_set[64][2] = {{false}};
 template <bool SPARSE>
 static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const void* weights, const void* meta,
                                    const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
-                                   cudaStream_t stream) {
+                                   cudaStream_t stream, int worker_cap = kMaxWorkers, bool force_split = false) {
   if (!load_driver_entry_points()) return SSCONV_ERR_CUDA;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SSCONV_ERR_CUDA;
@@ -612,21 +615,21 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.dev_status = dev_status;
 
   p.units = (long long)p.num_tiles * p.a_tiles;
-  int workers = g_sm_count[dev] < kMaxWorkers ? g_sm_count[dev] : kMaxWorkers;
+  int workers = g_sm_count[dev] < worker_cap ? g_sm_count[dev] : worker_cap;
   // Whole tiles per CTA, unless dealing the K range out evenly is clearly faster by a simple
   // cost model: cycles per weight tile in the main loop, and a fixed cost for parking, summing
   // and finishing partial tiles (both measured on B200).
   const int waves = (p.num_tiles + workers - 1) / workers;
   const double whole_cost = (double)waves * p.a_tiles * kCyclesPerATile;
   const double split_cost = (double)p.units / workers * kCyclesPerATile + kSplitFixedCycles;
-  p.split = (p.a_tiles > 1 && whole_cost > 1.15 * split_cost) ? 1 : 0;
+  p.split = (p.a_tiles > 1 && (force_split || whole_cost > 1.15 * split_cost)) ? 1 : 0;
   int grid;
   if (p.split) {
     grid = p.units < workers ? (int)p.units : workers;
-    if (ws == nullptr || ws_bytes < workspace_bytes()) return SSCONV_ERR_WORKSPACE;
+    if (ws == nullptr || ws_bytes < scratch_bytes(worker_cap)) return SSCONV_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(ws) & 15u) return SSCONV_ERR_ALIGNMENT;
     p.ws_regions = static_cast<float4*>(ws);
-    p.ws_counters = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + 2 * (size_t)kMaxWorkers * kRegionBytes);
+    p.ws_counters = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + 2 * (size_t)worker_cap * kRegionBytes);
   } else {
     grid = p.num_tiles < workers ? p.num_tiles : workers;
     p.ws_regions = nullptr;
@@ -644,6 +647,43 @@ int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void*
 int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias, void* y,
                              void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream) {
   return launch_forward_impl<false>(d, x, w, nullptr, bias, y, ws, ws_bytes, dev_status, stream);
+}
+
+// ---------------------------------------------------------------------------------------
+// Variant with built-in scratch, for callers that cannot allocate device memory
+// ---------------------------------------------------------------------------------------
+// The scratch of the split-K path lives in this file-scope device array instead of a caller
+// buffer.  It is sized for kStaticWorkers thread blocks; every GPU that loads the library keeps
+// it (about 15.7 MB) until the process exits.  In host code the array's name is only a handle:
+// the device address comes from cudaGetSymbolAddress, once per device.
+constexpr int kStaticWorkers = 64;
+constexpr int kStaticMaxTiles = 64;
+static __device__ __align__(256) unsigned char g_static_scratch[scratch_bytes(kStaticWorkers)];
+static unsigned char* g_static_scratch_ptr[64] = {nullptr};
+
+int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
+                                 const float* bias, void* y, int32_t* dev_status, cudaStream_t stream) {
+  const Geometry geo = make_geometry(d);
+  const long long P = (long long)d.N * out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h) *
+                      out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
+  const long long tiles = ((P + kBN - 1) / kBN) * geo.m_tiles;
+  if (tiles > kStaticMaxTiles) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SSCONV_ERR_CUDA;
+  if (g_static_scratch_ptr[dev] == nullptr) {
+    unsigned char* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess || ptr == nullptr)
+      return SSCONV_ERR_CUDA;
+    g_static_scratch_ptr[dev] = ptr;
+  }
+  unsigned char* scratch = g_static_scratch_ptr[dev];
+  // The arrival counters must start at zero; the partial-sum regions are overwritten before use.
+  // The array keeps whatever the previous call left (an aborted call can leave counts behind).
+  const size_t counters_at = 2 * (size_t)kStaticWorkers * kRegionBytes;
+  if (cudaMemsetAsync(scratch + counters_at, 0, 2 * (size_t)kStaticWorkers * sizeof(int), stream) != cudaSuccess)
+    return SSCONV_ERR_CUDA;
+  return launch_forward_impl<true>(d, x, w_comp, meta, bias, y, scratch, scratch_bytes(kStaticWorkers), dev_status,
+                                   stream, kStaticWorkers, true);
 }
 
 }  // namespace ssconv
