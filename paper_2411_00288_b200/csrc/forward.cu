@@ -8,10 +8,12 @@
 // tiles (persistent kernel).  The pixel extent is as wide as two fp32 accumulators plus the
 // metadata columns allow in the 512 TMEM columns: one thread issues every MMA, and the cost of
 // issuing one is what bounds narrow tiles.  Warp roles:
-//   warp 0      TMA producer.  Two rings: weight tiles (128 rows x 128 B, plus the 2 KB
-//               metadata image for the sparse kernel) and activation tiles (240 pixels x 64
-//               channels at one filter tap, im2col mode, zero-filled outside the image).  A
-//               sparse weight tile spans two activation tiles (128 dense columns).
+//   warp 0      TMA producer.  One ring of stages, a stage = one k-block of 64 dense columns: an
+//               activation tile (240 pixels x 64 channels at one filter tap, im2col mode,
+//               zero-filled outside the image) and, with the first stage of each weight tile, that
+//               weight tile (128 rows x 128 B, plus the 2 KB metadata image for the sparse kernel,
+//               where it spans two stages).  One full and one empty barrier per stage: every
+//               barrier operation of the two single-thread loops costs tens of cycles.
 //   warp 1      owns TMEM; one thread copies metadata smem->TMEM and issues the MMAs into one of
 //               two fp32 accumulators (128 lanes x 240 columns each).
 //   warps 2-9   epilogue, two groups of four warps, each owning half of the tile's pixel columns:
@@ -49,8 +51,7 @@ constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 1.9 GHz
 constexpr uint32_t kATileBytes = 128 * 128;          // 128 rows x 128 B
 constexpr uint32_t kBTileBytes = kBN * 128;          // 240 pixels x 64 channels bf16
 constexpr uint32_t kPieceBytes = kPiece * 256;       // 40 pixels x 128 channels bf16
-constexpr int kNA = 3;                               // weight ring depth
-constexpr int kNB = 4;                               // activation ring depth
+constexpr int kNB = 4;                               // stages in the ring
 
 template <bool SPARSE>
 struct Cfg {
@@ -58,6 +59,7 @@ struct Cfg {
   static constexpr uint32_t kMetaBytes = SPARSE ? (uint32_t)kMetaImageBytes : 0u;
   static constexpr uint32_t kAEntryBytes = kATileBytes + kMetaBytes;
   static constexpr uint32_t kBarrierBytes = 256;
+  static constexpr int kNA = kNB / kBlocksPerA;       // weight slots: one per group of stages sharing a tile
   static constexpr uint32_t kSmemBytes =
       kNA * kAEntryBytes + kNB * kBTileBytes + 2 * kGroups * kPieceBytes + kBarrierBytes + 1024;
 };
@@ -91,8 +93,18 @@ struct WorkIter {
     A = p.a_tiles;
     const long long c = blockIdx.x, G = gridDim.x;
     if (p.split) {
-      u = c * p.units / G;
-      u_end = (c + 1) * p.units / G;
+      if (p.units < (1LL << 31) / (G + 1)) {  // 32-bit divisions: this runs before the first load
+        const uint32_t U = (uint32_t)p.units, g = (uint32_t)G, cc = (uint32_t)c;
+        u = cc * U / g;
+        u_end = (cc + 1) * U / g;
+      } else {
+        u = c * p.units / G;
+        u_end = (c + 1) * p.units / G;
+      }
+    } else if (p.num_tiles < (1 << 23)) {
+      const uint32_t T = (uint32_t)p.num_tiles, g = (uint32_t)G, cc = (uint32_t)c;
+      u = (long long)(cc * T / g) * A;
+      u_end = (long long)((cc + 1) * T / g) * A;
     } else {
       u = (c * p.num_tiles / G) * A;
       u_end = ((c + 1) * p.num_tiles / G) * A;
@@ -100,7 +112,7 @@ struct WorkIter {
   }
   __device__ bool next(Segment& s) {
     if (u >= u_end) return false;
-    s.tile = (int)(u / A);
+    s.tile = (u < (1LL << 31)) ? (int)((uint32_t)u / (uint32_t)A) : (int)(u / A);
     s.a0 = (int)(u - (long long)s.tile * A);
     const long long left = u_end - u;
     s.a1 = (left >= A - s.a0) ? A : s.a0 + (int)left;
@@ -146,13 +158,12 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* a_ring = smem;
+  constexpr int kNA = C::kNA;
   uint8_t* b_ring = a_ring + kNA * C::kAEntryBytes;
   uint8_t* out_stage = b_ring + kNB * kBTileBytes;
-  uint64_t* bar_a_full = reinterpret_cast<uint64_t*>(out_stage + 2 * kGroups * kPieceBytes);
-  uint64_t* bar_a_empty = bar_a_full + kNA;
-  uint64_t* bar_b_full = bar_a_empty + kNA;
-  uint64_t* bar_b_empty = bar_b_full + kNB;
-  uint64_t* bar_acc_full = bar_b_empty + kNB;
+  uint64_t* bar_full = reinterpret_cast<uint64_t*>(out_stage + 2 * kGroups * kPieceBytes);
+  uint64_t* bar_empty = bar_full + kNB;
+  uint64_t* bar_acc_full = bar_empty + kNB;
   uint64_t* bar_acc_empty = bar_acc_full + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -163,13 +174,9 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kNA; ++s) {
-      mbar_init(&bar_a_full[s], 1);
-      mbar_init(&bar_a_empty[s], 1);
-    }
     for (int s = 0; s < kNB; ++s) {
-      mbar_init(&bar_b_full[s], 1);
-      mbar_init(&bar_b_empty[s], 1);
+      mbar_init(&bar_full[s], 1);
+      mbar_init(&bar_empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bar_acc_full[b], 1);
@@ -191,10 +198,11 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      // All index arithmetic in the k loop is incremental: this single thread's instruction
+      // Index arithmetic in the k loop is incremental and 32-bit: this single thread's instruction
       // stream is on the critical path of every stage.
-      int sa = 0, sb = 0;
-      uint32_t pha = 0, phb = 0;
+      const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty);
+      const uint32_t a_smem0 = smem_u32(a_ring), b_smem0 = smem_u32(b_ring);
+      uint32_t s = 0, ph = 0;  // stage and its phase parity
       bool ok = true;
       WorkIter work(p);
       Segment seg;
@@ -216,43 +224,52 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         const int kh0 = tap / p.KW;
         int kw = tap - kh0 * p.KW;
         int off_w = kw * p.dil_w, off_h = kh0 * p.dil_h;
-        int a_idx = seg.a0, a_sub = 0;
-        for (int kb = kb0; kb < kb1; ++kb) {
-          if (a_sub == 0) {
-            if (!mbar_wait_bounded(&bar_a_empty[sa], pha ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-            uint8_t* st = a_ring + sa * C::kAEntryBytes;
-            mbar_expect_tx(&bar_a_full[sa], C::kAEntryBytes);
-            if (SPARSE) {
-              tma_load_2d(st, &tm_a, &bar_a_full[sa], a_idx * 64, m * kTileM);
-              bulk_load(st + kATileBytes, meta_src, kMetaImageBytes, &bar_a_full[sa]);
-              meta_src += kMetaImageBytes;
+        int a_idx = seg.a0;
+        // whole weight tiles: a tile whose second k-block does not exist still takes two stages
+        for (int left = (seg.a1 - seg.a0) * APER, kb = kb0; left > 0; --left, ++kb) {
+          const bool first_of_tile = (APER == 1) || ((s & 1u) == 0u);
+          if (first_of_tile) {
+            // the weight slot is shared by the APER stages that follow: all of them must be free
+            if (!mbar_wait_a(empty0 + 8u * s, ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+            if (APER == 2 && !mbar_wait_a(empty0 + 8u * (s + 1u), ph ^ 1u, abort_flag, kWaitLimitCycles)) {
+              ok = false;
+              break;
+            }
+          }
+          const uint32_t full = full0 + 8u * s;
+          if (kb < kb1) {
+            if (first_of_tile) {
+              const uint32_t a_dst = a_smem0 + (s / APER) * C::kAEntryBytes;
+              mbar_expect_tx_a(full, C::kAEntryBytes + kBTileBytes);
+              if (SPARSE) {
+                tma_load_2d_a(a_dst, &tm_a, full, a_idx * 64, m * kTileM);
+                bulk_load_a(a_dst + kATileBytes, meta_src, kMetaImageBytes, full);
+                meta_src += kMetaImageBytes;
+              } else {
+                tma_load_3d_a(a_dst, &tm_a, full, cc * kBlockK, tap, m * kTileM);
+              }
+              ++a_idx;
             } else {
-              tma_load_3d(st, &tm_a, &bar_a_full[sa], cc * kBlockK, tap, m * kTileM);
+              mbar_expect_tx_a(full, kBTileBytes);
             }
-            ++a_idx;
-            if (++sa == kNA) {
-              sa = 0;
-              pha ^= 1u;
+            tma_load_im2col_4d_a(b_smem0 + s * kBTileBytes, &tm_b, full, cc * kBlockK, base_w, base_h, n0,
+                                 (uint16_t)off_w, (uint16_t)off_h);
+            if (++cc == p.cblocks) {  // next filter tap
+              cc = 0;
+              ++tap;
+              off_w += p.dil_w;
+              if (++kw == p.KW) {
+                kw = 0;
+                off_w = 0;
+                off_h += p.dil_h;
+              }
             }
+          } else {
+            mbar_arrive_a(full);  // stage without a k-block: keeps the ring's phases in step
           }
-          if (++a_sub == APER) a_sub = 0;
-          if (!mbar_wait_bounded(&bar_b_empty[sb], phb ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-          mbar_expect_tx(&bar_b_full[sb], kBTileBytes);
-          tma_load_im2col_4d(b_ring + sb * kBTileBytes, &tm_b, &bar_b_full[sb], cc * kBlockK, base_w, base_h, n0,
-                             (uint16_t)off_w, (uint16_t)off_h);
-          if (++sb == kNB) {
-            sb = 0;
-            phb ^= 1u;
-          }
-          if (++cc == p.cblocks) {  // next filter tap
-            cc = 0;
-            ++tap;
-            off_w += p.dil_w;
-            if (++kw == p.KW) {
-              kw = 0;
-              off_w = 0;
-              off_h += p.dil_h;
-            }
+          if (++s == (uint32_t)kNB) {
+            s = 0;
+            ph ^= 1u;
           }
         }
       }
@@ -263,15 +280,16 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       constexpr uint32_t idesc = make_idesc_bf16(kTileM, kBN, SPARSE);
       constexpr uint32_t kAEntryDesc = C::kAEntryBytes >> 4;  // descriptor address units are 16 B
       constexpr uint32_t kBTileDesc = kBTileBytes >> 4;
-      const uint64_t a_desc0 = smem_desc_sw128(smem_u32(a_ring));
-      const uint64_t b_desc0 = smem_desc_sw128(smem_u32(b_ring));
-      const uint64_t m_desc0 = smem_desc_noswizzle(smem_u32(a_ring) + kATileBytes, 16, 128);
+      const uint32_t a_lo0 = desc_lo(smem_u32(a_ring));
+      const uint32_t b_lo0 = desc_lo(smem_u32(b_ring));
+      const uint32_t m_lo0 = desc_lo(smem_u32(a_ring) + kATileBytes);
+      const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty);
+      const uint32_t meta_tmem0 = tmem_base + kMetaCol;
       // channels left in the last k-block of a tap decide how many MMAs it needs
       const int tail_c = p.C_in - (p.cblocks - 1) * kBlockK;
-      const int mma_full = SPARSE ? 2 : 4;
       const int mma_tail = SPARSE ? ((tail_c + 31) >> 5) : ((tail_c + 15) >> 4);
-      int sa = 0, sb = 0;
-      uint32_t pha = 0, phb = 0;
+      const int last_cc = p.cblocks - 1;
+      uint32_t s = 0, ph = 0;
       uint32_t tcount = 0;
       uint32_t mslot = 0;
       bool ok = true;
@@ -286,50 +304,49 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         uint32_t accumulate = 0;
         const int kb0 = seg.a0 * APER;
         const int kb1 = (seg.a1 * APER < p.kblocks) ? seg.a1 * APER : p.kblocks;
-        int cc = kb0 % p.cblocks, a_sub = 0;
-        uint64_t a_desc = 0;
-        uint32_t meta_tmem = 0;
-        for (int kb = kb0; kb < kb1; ++kb) {
-          if (a_sub == 0) {
-            if (!mbar_wait_bounded(&bar_a_full[sa], pha, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-            tc_fence_after();
-            a_desc = a_desc0 + (uint64_t)(sa * kAEntryDesc);
-            if (SPARSE) {
-              // two metadata slots of 4 TMEM columns, alternating per weight tile
-              meta_tmem = tmem_base + kMetaCol + 4u * mslot;
-              mslot ^= 1u;
-              tc_cp_128x128b(meta_tmem, m_desc0 + (uint64_t)(sa * kAEntryDesc));
-            }
-          }
-          if (!mbar_wait_bounded(&bar_b_full[sb], phb, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+        int cc = kb0 % p.cblocks;
+        uint32_t a_lo = 0, meta_tmem = 0;
+        for (int left = (seg.a1 - seg.a0) * APER, kb = kb0; left > 0; --left, ++kb) {
+          if (!mbar_wait_a(full0 + 8u * s, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t b_desc = b_desc0 + (uint64_t)(sb * kBTileDesc);
-          const int n_mma = (cc == p.cblocks - 1) ? mma_tail : mma_full;
-          if (SPARSE) {
-            // k-block a_sub of the weight tile: kept values start 64 B in, metadata 2 columns in;
-            // per MMA A advances 16 kept values = 32 B, B 32 channels = 64 B (descriptor units of 16 B)
-            const uint64_t a_kb = a_desc + 4 * a_sub;
-            const uint32_t meta_kb = meta_tmem + 2 * a_sub;
-            tc_mma_sparse(d_tmem, a_kb, b_desc, meta_kb, idesc, accumulate);
-            if (n_mma > 1) tc_mma_sparse(d_tmem, a_kb + 2, b_desc + 4, meta_kb, idesc | 1u, 1);
-          } else {
-            tc_mma_dense(d_tmem, a_desc, b_desc, idesc, accumulate);
-            for (int kk = 1; kk < n_mma; ++kk) tc_mma_dense(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, 1);
-          }
-          accumulate = 1;
-          tc_commit(&bar_b_empty[sb]);
-          if (++sb == kNB) {
-            sb = 0;
-            phb ^= 1u;
-          }
-          if (++cc == p.cblocks) cc = 0;
-          if (++a_sub == APER || kb == kb1 - 1) {
-            a_sub = 0;
-            tc_commit(&bar_a_empty[sa]);
-            if (++sa == kNA) {
-              sa = 0;
-              pha ^= 1u;
+          if (kb < kb1) {
+            const uint32_t a_sub = (APER == 2) ? (s & 1u) : 0u;
+            if (a_sub == 0) {
+              a_lo = a_lo0 + (s / APER) * kAEntryDesc;
+              if (SPARSE) {
+                // two metadata slots of 4 TMEM columns, alternating per weight tile
+                meta_tmem = meta_tmem0 + 4u * mslot;
+                mslot ^= 1u;
+                tc_cp_128x128b_lo(meta_tmem, m_lo0 + (s / APER) * kAEntryDesc);
+              }
             }
+            const uint32_t b_lo = b_lo0 + s * kBTileDesc;
+            const bool tail = (cc == last_cc);
+            if (SPARSE) {
+              // k-block a_sub of the weight tile: kept values start 64 B in, metadata 2 columns in;
+              // per MMA A advances 16 kept values = 32 B, B 32 channels = 64 B (descriptor units of 16 B)
+              const uint32_t a_kb = a_lo + 4u * a_sub;
+              const uint32_t meta_kb = meta_tmem + 2u * a_sub;
+              tc_mma_sparse_lo(d_tmem, a_kb, b_lo, meta_kb, idesc, accumulate);
+              if (!tail || mma_tail > 1) tc_mma_sparse_lo(d_tmem, a_kb + 2u, b_lo + 4u, meta_kb, idesc | 1u, 1u);
+            } else {
+              tc_mma_dense_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
+              if (!tail) {
+                tc_mma_dense_lo(d_tmem, a_lo + 2u, b_lo + 2u, idesc, 1u);
+                tc_mma_dense_lo(d_tmem, a_lo + 4u, b_lo + 4u, idesc, 1u);
+                tc_mma_dense_lo(d_tmem, a_lo + 6u, b_lo + 6u, idesc, 1u);
+              } else {
+                for (int kk = 1; kk < mma_tail; ++kk)
+                  tc_mma_dense_lo(d_tmem, a_lo + 2u * kk, b_lo + 2u * kk, idesc, 1u);
+              }
+            }
+            accumulate = 1;
+            cc = tail ? 0 : cc + 1;
+          }
+          tc_commit_a(empty0 + 8u * s);
+          if (++s == (uint32_t)kNB) {
+            s = 0;
+            ph ^= 1u;
           }
         }
         if (ok) tc_commit(&bar_acc_full[buf]);
