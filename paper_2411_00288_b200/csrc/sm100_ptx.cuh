@@ -39,25 +39,56 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Wait for a phase of an mbarrier, but never forever: after `limit_cycles` SM clock
-// cycles without completion, or as soon as another thread of the CTA has raised
-// *abort_flag, the wait gives up and returns false.  The caller then leaves its loop
-// and the CTA drains (see the kernels' tail).
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                                  long long limit_cycles) {
-  if (mbar_try_wait(bar, parity)) return true;
+// Spin on a phase of an mbarrier for at most `spins` tries, entirely inside one asm block: the
+// common short wait costs a few instructions and no call.  Returns whether the phase completed.
+__device__ __forceinline__ bool mbar_spin_a(uint32_t bar_addr, uint32_t parity, uint32_t spins) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+      "mov.u32 n, %3;\n"
+      "SPIN:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra DONE;\n\t"
+      "sub.u32 n, n, 1;\n\t"
+      "setp.ne.u32 q, n, 0;\n\t"
+      "@q bra SPIN;\n"
+      "DONE:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar_addr), "r"(parity), "r"(spins)
+      : "memory");
+  return ok != 0;
+}
+
+// Out-of-line continuation of a wait that outlasted the fast spin: polls on, but never forever.
+// After `limit_cycles` SM clock cycles without completion, or as soon as another thread of the
+// CTA has raised *abort_flag, it gives up and returns false.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t parity, volatile int* abort_flag,
+                                            long long limit_cycles, uint32_t backoff_ns) {
   const long long t0 = clock64();
-  uint32_t polls = 0;
   while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((++polls & 63u) == 0u) {
-      if (*abort_flag != 0) return false;
-      if (clock64() - t0 > limit_cycles) {
-        *abort_flag = 1;
-        return false;
-      }
+    if (mbar_spin_a(bar_addr, parity, 64)) return true;
+    if (*abort_flag != 0) return false;
+    if (clock64() - t0 > limit_cycles) {
+      *abort_flag = 1;
+      return false;
     }
+    if (backoff_ns) __nanosleep(backoff_ns);
   }
+}
+
+// Wait for a phase of an mbarrier, but never forever (see mbar_wait_slow).  The caller then leaves
+// its loop and the CTA drains (see the kernels' tail).  `backoff_ns` > 0 makes a long wait sleep
+// between polls: for roles whose waits are long and not latency critical.
+constexpr uint32_t kFastSpins = 2048;
+__device__ __forceinline__ bool mbar_wait_a(uint32_t bar_addr, uint32_t parity, volatile int* abort_flag,
+                                            long long limit_cycles, uint32_t backoff_ns = 0) {
+  if (mbar_spin_a(bar_addr, parity, kFastSpins)) return true;
+  return mbar_wait_slow(bar_addr, parity, abort_flag, limit_cycles, backoff_ns);
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                  long long limit_cycles, uint32_t backoff_ns = 0) {
+  return mbar_wait_a(smem_u32(bar), parity, abort_flag, limit_cycles, backoff_ns);
 }
 
 // ---------------------------------------------------------------- proxies / fences
@@ -238,38 +269,6 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 // The producer and the MMA issuer are single threads whose instruction streams sit on the critical
 // path of every k-block, so their helpers take 32-bit shared-memory addresses and 32-bit descriptor
 // halves that the caller keeps in registers, and the slow path of a wait is kept out of line.
-__device__ __forceinline__ bool mbar_try_wait_a(uint32_t bar_addr, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar_addr), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t parity, volatile int* abort_flag,
-                                            long long limit_cycles) {
-  const long long t0 = clock64();
-  uint32_t polls = 0;
-  while (true) {
-    if (mbar_try_wait_a(bar_addr, parity)) return true;
-    if ((++polls & 63u) == 0u) {
-      if (*abort_flag != 0) return false;
-      if (clock64() - t0 > limit_cycles) {
-        *abort_flag = 1;
-        return false;
-      }
-    }
-  }
-}
-// Bounded wait (same contract as mbar_wait_bounded) on a barrier given by its shared address.
-__device__ __forceinline__ bool mbar_wait_a(uint32_t bar_addr, uint32_t parity, volatile int* abort_flag,
-                                            long long limit_cycles) {
-  if (mbar_try_wait_a(bar_addr, parity)) return true;
-  return mbar_wait_slow(bar_addr, parity, abort_flag, limit_cycles);
-}
 __device__ __forceinline__ void mbar_expect_tx_a(uint32_t bar_addr, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(bytes) : "memory");
 }
