@@ -28,8 +28,10 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "dense-equiv TFLOP/s of 2:4 sparse conv fwd (bf16), % of sparse-TC roofline, xdense"
-WORKLOAD = "resnet18_3x3_sweep_bf16_nhwc_batch32"
-CONFIG_ID = 2
+WORKLOADS = {2: "resnet18_3x3_sweep_bf16_nhwc_batch32", 3: "resnet50_bottleneck_layers_bf16_nhwc_batch64",
+             4: "convnext_t_pointwise_layers_bf16_nhwc_batch128"}
+CONFIG_ID = 2          # the benchmarked workload; --workload-config picks another for layer tables
+WORKLOAD = WORKLOADS[CONFIG_ID]
 L2_BYTES = 126 * 2 ** 20
 
 
@@ -171,6 +173,7 @@ def reference_arm(args):
 
 # ----------------------------------------------------------------------------- GPU arm
 def main():
+    global CONFIG_ID, WORKLOAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=4000)
@@ -181,7 +184,11 @@ def main():
     ap.add_argument("--only-layer", type=int, default=None,
                     help="profiling aid: launch just this layer of the sweep --layer-iters times and exit")
     ap.add_argument("--dense", action="store_true", help="with --only-layer: use the dense kernel")
+    ap.add_argument("--workload-config", type=int, default=CONFIG_ID, choices=sorted(WORKLOADS),
+                    help="layer set to run (default: the benchmarked ResNet-18 sweep)")
     args = ap.parse_args()
+    CONFIG_ID = args.workload_config
+    WORKLOAD = WORKLOADS[CONFIG_ID]
     if args.impl == "reference":
         reference_arm(args)
         return
@@ -382,7 +389,7 @@ def main():
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps,
             "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "layers": len(layers), "batch_per_gpu": 32,
+            "config": {"workload": WORKLOAD, "layers": len(layers), "batch_per_gpu": layers[0].N,
                        "l2": f"rotating {n_sets} buffer sets of {set_bytes / 2**20:.0f} MiB (> L2) per rank",
                        "masks": "magnitude top-2 of 4, selected and compressed once before timing",
                        "launch": "the C-ABI calls of one step recorded into a CUDA graph per buffer set and replayed",
