@@ -1,10 +1,13 @@
 // Geometry of the compressed 2:4 operand as the forward kernel consumes it.
 //
 // The weight matrix W [C_out x K], K ordered (kh, kw, c_in), is cut along K into "k-blocks"
-// of 64 dense columns that never straddle a filter tap: each tap contributes
-// ceil(C_in/64) k-blocks, the last of which may be partly (or, after rounding the block
-// count up to even, wholly) padding.  Two consecutive k-blocks form one pipeline stage of
-// the sparse kernel (128 dense columns = 64 kept values per row).
+// of 64 dense columns that never straddle a filter tap: a k-block is 64 consecutive input
+// channels (a "channel chunk", the last one possibly partly padding) at one tap.  K-blocks are
+// numbered chunk-major, b = chunk * taps + tap, so that all taps of one channel chunk are
+// consecutive: the forward kernel can then serve them from one staged run of activations.
+// The block count is rounded up to even (the extra block is padding).  Two consecutive
+// k-blocks share one weight tile of the sparse kernel (128 dense columns = 64 kept values
+// per row).
 //
 // Value blob:    bf16 [Mp][KC], Mp = C_out rounded up to 128, KC = 32 * n_kblocks_padded.
 //                Column 32*b + 2*q + s holds kept value s (0 = lower position) of the q-th
@@ -31,7 +34,7 @@ constexpr int kMetaImageBytes = 2048;
 struct Geometry {
   int taps;          // KH*KW
   int cblocks;       // k-blocks per tap = ceil(C_in/64)
-  int kblocks;       // taps*cblocks
+  int kblocks;       // taps*cblocks, numbered chunk * taps + tap
   int kblocks_pad;   // rounded up to even
   int stages;        // kblocks_pad/2 (sparse pipeline stages per tile)
   int m_tiles;       // ceil(C_out/128)

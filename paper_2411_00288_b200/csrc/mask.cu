@@ -76,8 +76,8 @@ __global__ void compress_values_kernel(ssconv_desc_t d, Geometry geo, const uint
   int co = (int)(t / (16 * (int64_t)geo.kblocks_pad));
   uint32_t out = 0;
   if (co < d.C_out && b < geo.kblocks) {
-    int tap = b / geo.cblocks;
-    int c = (b % geo.cblocks) * kBlockK + 4 * q;
+    int tap = b % geo.taps;
+    int c = (b / geo.taps) * kBlockK + 4 * q;
     if (c < d.C_in) {
       int64_t g = ((int64_t)co * geo.taps + tap) * (d.C_in / 4) + c / 4;
       uint2 v = w[g];
@@ -104,8 +104,8 @@ __global__ void compress_meta_kernel(ssconv_desc_t d, Geometry geo, const uint8_
   int s = (int)((t / 512) % geo.stages);
   int mt = (int)(t / (512 * (int64_t)geo.stages));
   int b = 2 * s + (j >> 1);
-  int tap = b / geo.cblocks;
-  int cbase = (b % geo.cblocks) * kBlockK + (j & 1) * 32 + 16 * ((L >> 3) & 1);
+  int tap = b % geo.taps;
+  int cbase = (b / geo.taps) * kBlockK + (j & 1) * 32 + 16 * ((L >> 3) & 1);
   uint32_t word = 0;
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
@@ -138,7 +138,7 @@ __global__ void decompress_kernel(ssconv_desc_t d, Geometry geo, const uint32_t*
   int c = (int)(g % groups_per_tap) * 4;
   int tap = (int)((g / groups_per_tap) % geo.taps);
   int co = (int)(g / ((int64_t)groups_per_tap * geo.taps));
-  int b = tap * geo.cblocks + c / kBlockK;
+  int b = (c / kBlockK) * geo.taps + tap;
   int cl = c % kBlockK;
   // metadata word and nibble of this group
   int mt = co / kTileM, r = co % kTileM;

@@ -72,7 +72,7 @@ def test_compress_roundtrip_bit_exact(shape):
     vals = vals.reshape(Co, KH * KW, Ci // 4, 2)
     total_kept = 0
     for b in range(kb):
-        tap, cc = divmod(b, cblocks)
+        cc, tap = divmod(b, KH * KW)  # k-blocks are numbered chunk-major
         ng = min(16, Ci // 4 - 16 * cc)
         assert np.array_equal(blob[:Co, b, :2 * ng], vals[:, tap, 16 * cc:16 * cc + ng, :].reshape(Co, -1))
         total_kept += blob[:Co, b, :2 * ng].size
