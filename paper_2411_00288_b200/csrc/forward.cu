@@ -8,22 +8,17 @@
 // tiles (persistent kernel).  240 is as wide as two fp32 accumulators plus the metadata columns
 // allow in the 512 TMEM columns: one thread issues every MMA, and wide MMAs amortise its cost.
 //
-// Two ways of staging activations (template parameter HALO):
-//  * im2col mode (any stride): positions are the output pixels (n, ho, wo) in row-major order.
-//    Per k-block (64 input channels at one filter tap) one im2col-mode TMA load brings the 240
-//    pixels' channels at that tap, zero-filled outside the image.  A 3x3 filter therefore stages
-//    every input pixel nine times, and shared-memory bandwidth bounds the main loop.
-//  * halo mode (stride 1): positions are the pixels of the zero-padded input, (n, r, c) with
-//    c < W + 2 pad, r < H + 2 pad, row-major; an output exists where r < H_out and c < W_out, the
-//    rest of a tile is computed and dropped.  In this space the activation a tap (kh, kw) needs
-//    for position q is the one at q + kh*dil*(W+2pad) + kw*dil, for every q.  So ONE staged run
-//    of 240 + (KH-1)*dil*(W+2pad) + (KW-1)*dil consecutive padded pixels per 64-channel chunk
-//    serves all KH*KW taps: the MMA of a tap reads the run through a descriptor that starts a
-//    few rows later (a 128-byte-swizzled K-major operand may start at any 128-byte row).
+// Positions are the output pixels (n, ho, wo) in row-major order.  Per k-block (64 input channels
+// at one filter tap) one im2col-mode TMA load brings the 240 pixels' channels at that tap,
+// zero-filled outside the image.  (Staging one run of padded input per channel chunk and serving
+// all taps from it through row-shifted descriptors was built and measured: the MMA's operand
+// fetch, about 64 B/clk, bounds the main loop either way, so the simpler scheme stays.)
 //
 // Warp roles: warp 0 TMA producer, warp 1 MMA issuer (one thread; owns TMEM), warps 2-9 epilogue
 // in two groups of four warps that each own half of a tile's positions: TMEM -> registers,
-// + bias, ReLU, bf16, transpose through shared memory, 16-byte coalesced stores to NHWC.
+// + bias, ReLU, bf16; neighbouring lanes (channels c, c+1) swap one value per position pair so
+// that every lane holds two adjacent channels of one position, and stores them as one 32-bit
+// word: a warp writes two 64-byte runs of NHWC per instruction, with no shared-memory staging.
 //
 // Work partition: the unit of work is one weight tile's worth of K for one output tile.  Either
 // every CTA takes a contiguous block of whole output tiles, or (when whole tiles would leave many
@@ -47,7 +42,7 @@ namespace ssconv {
 constexpr int kBN = 240;                 // positions per tile (N of the MMA)
 constexpr int kGroups = 2;               // epilogue warp groups, each owning kBN / kGroups positions
 constexpr int kGroupCols = kBN / kGroups;
-constexpr int kPiece = 40;               // positions per epilogue staging piece
+constexpr int kPiece = 40;               // accumulator columns the epilogue handles at a time
 constexpr int kThreads = 64 + 128 * kGroups;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kAccCol1 = 256;       // second accumulator; the first starts at column 0
@@ -55,37 +50,29 @@ constexpr uint32_t kMetaCol = kBN;       // metadata: 2 slots x 4 columns in [24
 constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 1.9 GHz
 constexpr uint32_t kATileBytes = 128 * 128;          // 128 rows x 128 B
 constexpr uint32_t kBTileBytes = kBN * 128;          // 240 positions x 64 channels bf16
-constexpr uint32_t kPieceBytes = kPiece * 256;       // 40 positions x 128 channels bf16
-constexpr uint32_t kStagingBytes = 2 * kGroups * kPieceBytes;
-constexpr int kNB = 4;                               // im2col mode: stages in the ring
-constexpr int kNAHalo = 3;                           // halo mode: weight tiles in flight
-constexpr int kNRuns = 2;                            // halo mode: activation runs in flight
 constexpr uint32_t kBarrierBytes = 256;
-constexpr uint32_t kMaxSmemBytes = 232448;           // 227 KB per CTA
 
 template <bool SPARSE>
 struct Cfg {
   static constexpr int kBlocksPerA = SPARSE ? 2 : 1;  // k-blocks of 64 dense columns per weight tile
   static constexpr uint32_t kMetaBytes = SPARSE ? (uint32_t)kMetaImageBytes : 0u;
   static constexpr uint32_t kAEntryBytes = kATileBytes + kMetaBytes;
-  static constexpr int kNA = kNB / kBlocksPerA;       // im2col mode: weight slots, one per group of stages
-  static constexpr uint32_t kSmemIm2col =
-      kNA * kAEntryBytes + kNB * kBTileBytes + kStagingBytes + kBarrierBytes + 1024;
-  static constexpr uint32_t kSmemHaloFixed = kNAHalo * kAEntryBytes + kStagingBytes + kBarrierBytes + 1024;
+  static constexpr int kNB = 4;                       // stages in the ring
+  static constexpr int kNA = kNB / kBlocksPerA;       // weight slots, one per group of stages sharing a tile
+  static constexpr uint32_t kSmemBytes = kNA * kAEntryBytes + kNB * kBTileBytes + kBarrierBytes + 1024;
+  static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 };
 
 struct FwdParams {
   int C_in, C_out;
-  int N_img, Ho, Wo;        // output extent
-  int Hq, Wq;               // extent of the position space (= Ho, Wo in im2col mode; padded input in halo mode)
+  int Ho, Wo;               // output extent
+  int Q;                    // positions = N * Ho * Wo
   int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
   int taps, cblocks, kblocks;
   int m_tiles, num_tiles;
   int a_tiles;              // weight tiles per output tile
   int split;                // 1: units dealt out evenly across CTAs (stream-K); 0: whole tiles per CTA
   long long units;          // num_tiles * a_tiles
-  int run_rows;             // halo mode: padded pixels per staged run
-  uint32_t run_bytes;       // halo mode: run_rows * 128 rounded up to 1024
   float4* ws_regions;       // [2 * gridDim.x] regions of 128 x 240 fp32: a CTA's partial tiles
   int* ws_counters;         // [gridDim.x][2] arrivals per split tile and epilogue group, zero between launches
   uint32_t flags;
@@ -165,7 +152,7 @@ __device__ __forceinline__ void tc_ld_piece(uint32_t taddr, uint32_t (&r)[kPiece
   for (int j = 0; j < 8; ++j) r[32 + j] = b[j];
 }
 
-// Position q of the position space -> (image, row, column).
+// Position q -> (image, output row, output column).
 struct Pos {
   int n, r, c;
 };
@@ -178,29 +165,26 @@ __device__ __forceinline__ Pos decode_pos(int q, int Wq, int Hq) {
   return s;
 }
 
-template <bool SPARSE, bool HALO>
+template <bool SPARSE>
 __global__ void __launch_bounds__(kThreads, 1)
 ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                   const FwdParams p) {
   using C = Cfg<SPARSE>;
   constexpr int APER = C::kBlocksPerA;
-  constexpr int kNA = HALO ? kNAHalo : C::kNA;
+  constexpr int kNA = C::kNA;
+  constexpr int kNB = C::kNB;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* a_ring = smem;                                        // kNA weight tiles (+ metadata)
-  uint8_t* b_ring = a_ring + kNA * C::kAEntryBytes;              // im2col: kNB stages; halo: kNRuns runs
-  uint8_t* out_stage = b_ring + (HALO ? kNRuns * p.run_bytes : kNB * kBTileBytes);
-  // 16 barrier slots: [0,4) full / weight-full, [4,8) empty / weight-empty, [8,10) run-full,
-  // [10,12) run-empty, [12,14) accumulator-full, [14,16) accumulator-empty
-  uint64_t* bars = reinterpret_cast<uint64_t*>(out_stage + kStagingBytes);
+  uint8_t* b_ring = a_ring + kNA * C::kAEntryBytes;              // kNB activation tiles
+  // barrier slots: [0,8) stage full, [8,16) stage empty, [16,18) accumulator full, [18,20) accumulator empty
+  uint64_t* bars = reinterpret_cast<uint64_t*>(b_ring + kNB * kBTileBytes);
   uint64_t* bar_full = bars;
-  uint64_t* bar_empty = bars + 4;
-  uint64_t* bar_run_full = bars + 8;
-  uint64_t* bar_run_empty = bars + 10;
-  uint64_t* bar_acc_full = bars + 12;
-  uint64_t* bar_acc_empty = bars + 14;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint64_t* bar_empty = bars + 8;
+  uint64_t* bar_acc_full = bars + 16;
+  uint64_t* bar_acc_empty = bars + 18;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = abort_flag + 1;         // per group two slots: the leader's go/stop verdict per tile
   volatile int* epi_last = epi_go + 2 * kGroups;  // per group: partial tile, is this CTA the last to arrive?
@@ -209,7 +193,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < 12; ++s) mbar_init(&bars[s], 1);
+    for (int s = 0; s < 16; ++s) mbar_init(&bars[s], 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(&bar_acc_full[b], 1);
       mbar_init(&bar_acc_empty[b], 4 * kGroups);
@@ -233,17 +217,15 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       // Index arithmetic in the k loop is incremental and 32-bit: this single thread's instruction
       // stream is on the critical path of every stage.
       const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty);
-      const uint32_t rfull0 = smem_u32(bar_run_full), rempty0 = smem_u32(bar_run_empty);
       const uint32_t a_smem0 = smem_u32(a_ring), b_smem0 = smem_u32(b_ring);
-      uint32_t s = 0, ph = 0;    // im2col: stage and parity; halo: weight-tile slot and parity
-      uint32_t rs = 0, rph = 0;  // halo: run slot and parity
+      uint32_t s = 0, ph = 0;  // stage and its phase parity
       bool ok = true;
       WorkIter work(p);
       Segment seg;
       while (ok && work.next(seg)) {
         const int pt = seg.tile / p.m_tiles;
         const int m = seg.tile - pt * p.m_tiles;
-        const Pos q0 = decode_pos(pt * kBN, p.Wq, p.Hq);
+        const Pos q0 = decode_pos(pt * kBN, p.Wo, p.Ho);
         const int base_w = q0.c * p.stride_w - p.pad_w;
         const int base_h = q0.r * p.stride_h - p.pad_h;
         const uint8_t* meta_src = p.meta + ((size_t)m * p.a_tiles + seg.a0) * kMetaImageBytes;
@@ -252,45 +234,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         int cc = kb0 / p.taps;          // channel chunk
         int tap = kb0 - cc * p.taps;
         int a_idx = seg.a0;
-        if (HALO) {
-          bool need_run = true;
-          for (int kb = kb0; kb < kb1; ++kb) {
-            if (need_run) {
-              if (!mbar_wait_a(rempty0 + 8u * rs, rph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-              mbar_expect_tx_a(rfull0 + 8u * rs, (uint32_t)p.run_rows * 128u);
-              tma_load_im2col_4d_a(b_smem0 + rs * p.run_bytes, &tm_b, rfull0 + 8u * rs, cc * kBlockK, base_w, base_h,
-                                   q0.n, 0, 0);
-              if (++rs == (uint32_t)kNRuns) {
-                rs = 0;
-                rph ^= 1u;
-              }
-              need_run = false;
-            }
-            if (APER == 1 || (kb & 1) == 0) {
-              if (!mbar_wait_a(empty0 + 8u * s, ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-              const uint32_t a_dst = a_smem0 + s * C::kAEntryBytes;
-              const uint32_t full = full0 + 8u * s;
-              mbar_expect_tx_a(full, C::kAEntryBytes);
-              if (SPARSE) {
-                tma_load_2d_a(a_dst, &tm_a, full, a_idx * 64, m * kTileM);
-                bulk_load_a(a_dst + kATileBytes, meta_src, kMetaImageBytes, full);
-                meta_src += kMetaImageBytes;
-              } else {
-                tma_load_3d_a(a_dst, &tm_a, full, cc * kBlockK, tap, m * kTileM);
-              }
-              ++a_idx;
-              if (++s == (uint32_t)kNA) {
-                s = 0;
-                ph ^= 1u;
-              }
-            }
-            if (++tap == p.taps) {  // next channel chunk needs its own run
-              tap = 0;
-              ++cc;
-              need_run = true;
-            }
-          }
-        } else {
+        {
           const int kh0 = tap / p.KW;
           int kw = tap - kh0 * p.KW;
           int off_w = kw * p.dil_w, off_h = kh0 * p.dil_h;
@@ -356,18 +300,12 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       const uint32_t b_lo0 = desc_lo(smem_u32(b_ring));
       const uint32_t m_lo0 = desc_lo(smem_u32(a_ring) + kATileBytes);
       const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty);
-      const uint32_t rfull0 = smem_u32(bar_run_full), rempty0 = smem_u32(bar_run_empty);
       const uint32_t meta_tmem0 = tmem_base + kMetaCol;
-      const uint32_t run_desc = p.run_bytes >> 4;
       // channels left in the last chunk decide how many MMAs its k-blocks need
       const int tail_c = p.C_in - (p.cblocks - 1) * kBlockK;
       const int mma_tail = SPARSE ? ((tail_c + 31) >> 5) : ((tail_c + 15) >> 4);
       const int last_cc = p.cblocks - 1;
-      // halo mode: descriptor steps (16-byte units; a position row is 128 B) between taps
-      const uint32_t step_kw = 8u * (uint32_t)p.dil_w;
-      const uint32_t step_kh = 8u * (uint32_t)(p.dil_h * p.Wq);
-      uint32_t s = 0, ph = 0;    // im2col: stage and parity; halo: weight-tile slot and parity
-      uint32_t rs = 0, rph = 0;  // halo: run slot and parity
+      uint32_t s = 0, ph = 0;  // stage and its phase parity
       uint32_t tcount = 0;
       uint32_t mslot = 0;
       bool ok = true;
@@ -385,85 +323,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         int cc = kb0 / p.taps;
         int tap = kb0 - cc * p.taps;
         uint32_t a_lo = 0, meta_tmem = 0;
-        if (HALO) {
-          int kh = tap / p.KW;
-          int kw = tap - kh * p.KW;
-          uint32_t shift = (uint32_t)kh * step_kh + (uint32_t)kw * step_kw;
-          bool run_active = false;
-          uint32_t run_lo = 0;
-          for (int kb = kb0; kb < kb1; ++kb) {
-            if (!run_active) {
-              if (!mbar_wait_a(rfull0 + 8u * rs, rph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-              tc_fence_after();
-              run_lo = b_lo0 + rs * run_desc;
-              run_active = true;
-            }
-            const uint32_t a_sub = (APER == 2) ? (uint32_t)(kb & 1) : 0u;
-            if (a_sub == 0) {
-              if (!mbar_wait_a(full0 + 8u * s, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-              tc_fence_after();
-              a_lo = a_lo0 + s * kAEntryDesc;
-              if (SPARSE) {
-                // two metadata slots of 4 TMEM columns, alternating per weight tile
-                meta_tmem = meta_tmem0 + 4u * mslot;
-                mslot ^= 1u;
-                tc_cp_128x128b_lo(meta_tmem, m_lo0 + s * kAEntryDesc);
-              }
-            }
-            const uint32_t b_lo = run_lo + shift;  // the tap's window into the staged run
-            const bool tail = (cc == last_cc);
-            if (SPARSE) {
-              const uint32_t a_kb = a_lo + 4u * a_sub;
-              const uint32_t meta_kb = meta_tmem + 2u * a_sub;
-              tc_mma_sparse_lo(d_tmem, a_kb, b_lo, meta_kb, idesc, accumulate);
-              if (!tail || mma_tail > 1) tc_mma_sparse_lo(d_tmem, a_kb + 2u, b_lo + 4u, meta_kb, idesc | 1u, 1u);
-            } else {
-              tc_mma_dense_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
-              if (!tail) {
-                tc_mma_dense_lo(d_tmem, a_lo + 2u, b_lo + 2u, idesc, 1u);
-                tc_mma_dense_lo(d_tmem, a_lo + 4u, b_lo + 4u, idesc, 1u);
-                tc_mma_dense_lo(d_tmem, a_lo + 6u, b_lo + 6u, idesc, 1u);
-              } else {
-                for (int kk = 1; kk < mma_tail; ++kk)
-                  tc_mma_dense_lo(d_tmem, a_lo + 2u * kk, b_lo + 2u * kk, idesc, 1u);
-              }
-            }
-            accumulate = 1;
-            if (APER == 1 || a_sub == 1 || kb == kb1 - 1) {  // last k-block of this weight tile
-              tc_commit_a(empty0 + 8u * s);
-              if (++s == (uint32_t)kNA) {
-                s = 0;
-                ph ^= 1u;
-              }
-            }
-            // next tap, or next channel chunk
-            shift += step_kw;
-            if (++kw == p.KW) {
-              kw = 0;
-              shift += step_kh - (uint32_t)p.KW * step_kw;
-              ++kh;
-            }
-            if (++tap == p.taps) {
-              tap = 0;
-              kh = 0;
-              shift = 0;
-              ++cc;
-              tc_commit_a(rempty0 + 8u * rs);  // the run's last reader has been issued
-              if (++rs == (uint32_t)kNRuns) {
-                rs = 0;
-                rph ^= 1u;
-              }
-              run_active = false;
-            }
-          }
-          if (run_active) {  // segment ended inside a chunk: the producer stages that run again
-            tc_commit_a(rempty0 + 8u * rs);
-            if (++rs == (uint32_t)kNRuns) {
-              rs = 0;
-              rph ^= 1u;
-            }
-          }
-        } else {
+        {
           for (int left = (seg.a1 - seg.a0) * APER, kb = kb0; left > 0; --left, ++kb) {
             if (!mbar_wait_a(full0 + 8u * s, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
             tc_fence_after();
@@ -516,22 +376,19 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   } else {
     // ------------------------------------------------------------------ epilogue
     // Two independent groups of four warps; group g owns positions [120 g, 120 g + 120) of every
-    // tile, with its own staging buffers and named barrier.
+    // tile and has its own named barrier.  A thread reads accumulator lane `row` (one output
+    // channel) for 40 positions at a time.
     const int grp = (warp - 2) >> 2;
     const int q = warp & 3;  // TMEM lane quadrant this warp may read
     const int row = q * 32 + lane;
-    const int gtid = row;    // thread index within the group (the group's warps have q = 2, 3, 0, 1)
     const bool leader = (q == 2 && lane == 0);  // first warp of each group
     const bool relu = (p.flags & SSCONV_FLAG_RELU) != 0;
     const int col_base = grp * kGroupCols;
-    uint8_t* my_stage = out_stage + grp * 2 * kPieceBytes;
+    const int odd = lane & 1;
+    const size_t pos_step_bytes = (size_t)p.C_out * 2;  // one position further in NHWC
     volatile int* my_go = epi_go + 2 * grp;
     volatile int* my_last = epi_last + grp;
-    // store duty: 16 threads cover the 256 bytes of one staged position, 8 positions at a time
-    const int part = gtid & 15;
-    const int jb = gtid >> 4;
     uint32_t tcount = 0;
-    uint32_t piece_count = 0;
     WorkIter work(p);
     Segment seg;
     for (; work.next(seg); ++tcount) {
@@ -581,17 +438,26 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         if (*my_last == 0) continue;  // someone else finishes this half tile
         __threadfence();
       }
-      // ---- finish the tile: bias, activation, bf16, transpose through smem, coalesced stores -----
-      // first position this thread stores, then it advances by 8 positions per step
-      Pos sp = decode_pos(pt * kBN + col_base + jb, p.Wq, p.Hq);
-      const int co_part = m * kTileM + part * 8;
+      // ---- finish the tile: bias, activation, bf16, lane-pair exchange, 32-bit stores -----------
+      // Lanes 2t and 2t+1 hold channels c and c+1 of the same positions.  Per position pair
+      // (j, j+1) they swap one value, after which the even lane has both channels of position j and
+      // the odd lane both channels of position j+1.
+      const int q_lane = pt * kBN + col_base + odd;  // first position this lane stores
+      const int co_pair = m * kTileM + (row & ~1);
+      int q_left = (co_pair < p.C_out) ? p.Q - q_lane : 0;  // positions q_lane + j with j < q_left exist
+      uint8_t* y_lane = reinterpret_cast<uint8_t*>(p.y + (size_t)q_lane * p.C_out + co_pair);
 #pragma unroll 1
-      for (int piece = 0; piece < kGroupCols / kPiece; ++piece, ++piece_count) {
-        uint8_t* stage = my_stage + (piece_count & 1u) * kPieceBytes;
+      for (int piece = 0; piece < kGroupCols / kPiece; ++piece) {
         uint32_t r[kPiece];
         if (whole) {
           tc_ld_piece(t_row + piece * kPiece, r);
           tc_wait_ld();
+          if (piece == kGroupCols / kPiece - 1) {
+            // this warp's part of the accumulator is read: hand it back to the MMA thread
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
+          }
         } else {
           // sum the contributors' regions in CTA order (reads bypass L1: the data came from other SMs)
 #pragma unroll
@@ -611,42 +477,23 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             }
           }
         }
-        // staging buffer [position][channel]; the buffer used two pieces ago is free again because
-        // every thread has passed the barrier of the piece in between
-        uint16_t* stage_col = reinterpret_cast<uint16_t*>(stage) + row;
 #pragma unroll
-        for (int j = 0; j < kPiece; ++j) {
-          float v = __uint_as_float(r[j]) + bias_v;
-          if (relu) v = fmaxf(v, 0.0f);
-          stage_col[j * 128] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
-        }
-        if (whole && piece == kGroupCols / kPiece - 1) {
-          // this warp's part of the accumulator is read: hand it back to the MMA thread
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
-        }
-        epilogue_bar_sync(grp);
-        // 16-byte stores: 16 consecutive threads write the 256 contiguous bytes of one position
-#pragma unroll
-        for (int k = 0; k < kPiece / 8; ++k) {
-          const bool valid = sp.c < p.Wo && sp.r < p.Ho && sp.n < p.N_img && co_part < p.C_out;
-          if (valid) {
-            const uint4 v = *reinterpret_cast<const uint4*>(stage + (jb + 8 * k) * 256 + part * 16);
-            const size_t pix = ((size_t)sp.n * p.Ho + sp.r) * p.Wo + sp.c;
-            *reinterpret_cast<uint4*>(p.y + pix * p.C_out + co_part) = v;
+        for (int i = 0; i < kPiece / 2; ++i) {
+          float v0 = __uint_as_float(r[2 * i]) + bias_v;
+          float v1 = __uint_as_float(r[2 * i + 1]) + bias_v;
+          if (relu) {
+            v0 = fmaxf(v0, 0.0f);
+            v1 = fmaxf(v1, 0.0f);
           }
-          sp.c += 8;
-          while (sp.c >= p.Wq) {
-            sp.c -= p.Wq;
-            if (++sp.r == p.Hq) {
-              sp.r = 0;
-              ++sp.n;
-            }
-          }
+          const float got_v = __shfl_xor_sync(0xFFFFFFFFu, odd ? v0 : v1, 1);
+          const __nv_bfloat162 pair = __floats2bfloat162_rn(odd ? got_v : v0, odd ? v1 : got_v);
+          if (2 * i < q_left)
+            *reinterpret_cast<__nv_bfloat162*>(y_lane + (size_t)(2 * i) * pos_step_bytes) = pair;
         }
+        q_left -= kPiece;
+        y_lane += (size_t)kPiece * pos_step_bytes;
       }
-      if (!whole && leader) p.ws_counters[2 * c_first + grp] = 0;
+      if (!whole && leader) p.ws_counters[2 * c_first + grp] = 0;  // zero again for the next launch
     }
   }
 
@@ -708,70 +555,49 @@ constexpr size_t scratch_bytes(int workers) {
 }
 size_t workspace_bytes() { return scratch_bytes(kMaxWorkers); }
 
-// Halo mode pays for positions that produce no output (the padding ring of every image); it is
-// used when at least this share of the positions is real and the staged run fits.
-constexpr double kHaloMinValidShare = 0.7;
-
-struct HaloPlan {
-  bool use;
-  int Wq, Hq, run_rows;
-  uint32_t run_bytes;
-};
+static int g_sm_count[64] = {0};
+static bool g_attr_set[64][2] = {{false}};
 
 template <bool SPARSE>
-static HaloPlan plan_halo(const ssconv_desc_t& d, int Ho, int Wo) {
-  HaloPlan h{};
-  h.use = false;
-  if (d.stride_h != 1 || d.stride_w != 1 || d.KH * d.KW == 1) return h;
-  h.Wq = d.W + 2 * d.pad_w;
-  h.Hq = d.H + 2 * d.pad_h;
-  h.run_rows = kBN + (d.KH - 1) * d.dil_h * h.Wq + (d.KW - 1) * d.dil_w;
-  h.run_bytes = ((uint32_t)h.run_rows * 128u + 1023u) & ~1023u;
-  if (h.run_rows > 1024) return h;
-  if (Cfg<SPARSE>::kSmemHaloFixed + kNRuns * h.run_bytes > kMaxSmemBytes) return h;
-  if ((double)Ho * Wo < kHaloMinValidShare * (double)h.Hq * h.Wq) return h;
-  h.use = true;
-  return h;
-}
-
-static int g_sm_count[64] = {0};
-static bool g_attr_set[64][2][2] = {{{false}}};
-
-template <bool SPARSE, bool HALO>
-static int32_t launch_variant(int dev, const ssconv_desc_t& d, const Geometry& geo, int Ho, int Wo,
-                              const HaloPlan& hp, const void* x, const void* weights, const void* meta,
-                              const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
-                              cudaStream_t stream, int worker_cap, bool force_split) {
+static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const void* weights, const void* meta,
+                                   const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
+                                   cudaStream_t stream, int worker_cap = kMaxWorkers, bool force_split = false) {
   using C = Cfg<SPARSE>;
-  if (!g_attr_set[dev][SPARSE ? 1 : 0][HALO ? 1 : 0]) {
-    if (cudaFuncSetAttribute(ssconv_fwd_kernel<SPARSE, HALO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kMaxSmemBytes) != cudaSuccess)
+  if (!load_driver_entry_points()) return SSCONV_ERR_CUDA;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SSCONV_ERR_CUDA;
+  if (g_sm_count[dev] == 0) {
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SSCONV_ERR_CUDA;
+    if (major != 10) return SSCONV_ERR_ARCH;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
       return SSCONV_ERR_CUDA;
-    g_attr_set[dev][SPARSE ? 1 : 0][HALO ? 1 : 0] = true;
+    g_sm_count[dev] = sms;
   }
-  const int Wq = HALO ? hp.Wq : Wo;
-  const int Hq = HALO ? hp.Hq : Ho;
-  const long long Q = (long long)d.N * Hq * Wq;  // positions
+  if (!g_attr_set[dev][SPARSE ? 1 : 0]) {
+    if (cudaFuncSetAttribute(ssconv_fwd_kernel<SPARSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)C::kSmemBytes) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
+    g_attr_set[dev][SPARSE ? 1 : 0] = true;
+  }
+  const Geometry geo = make_geometry(d);
+  const int Ho = out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h);
+  const int Wo = out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
+  const long long Q = (long long)d.N * Ho * Wo;  // positions
   if (Q > 0x7FFFFF00LL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
 
   CUtensorMap tm_a, tm_b;
   // activations: NHWC seen as (c, w, h, n), im2col mode; elements outside the image read as zero
-  // (= the zero padding of Eq. 4).  im2col mode: base pixels are the filter placements and each
-  // load adds a tap offset.  Halo mode: base pixels are all pixels of the padded image, no offset.
+  // (= the zero padding of Eq. 4); base pixels are the filter placements, each load adds a tap offset
   {
     cuuint64_t dims[4] = {(cuuint64_t)d.C_in, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
     cuuint64_t strides[3] = {(cuuint64_t)d.C_in * 2, (cuuint64_t)d.W * d.C_in * 2,
                              (cuuint64_t)d.H * d.W * d.C_in * 2};
     int lower[2] = {-d.pad_w, -d.pad_h};
     int upper[2] = {d.pad_w - (d.KW - 1) * d.dil_w, d.pad_h - (d.KH - 1) * d.dil_h};
-    if (HALO) {
-      upper[0] = d.pad_w;
-      upper[1] = d.pad_h;
-    }
     cuuint32_t estr[4] = {1, (cuuint32_t)d.stride_w, (cuuint32_t)d.stride_h, 1};
-    const cuuint32_t pixels = HALO ? (cuuint32_t)hp.run_rows : (cuuint32_t)kBN;
     CUresult r = g_encode_im2col(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), dims, strides,
-                                 lower, upper, (cuuint32_t)kBlockK, pixels, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 lower, upper, (cuuint32_t)kBlockK, (cuuint32_t)kBN, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
@@ -799,11 +625,9 @@ static int32_t launch_variant(int dev, const ssconv_desc_t& d, const Geometry& g
   FwdParams p;
   p.C_in = d.C_in;
   p.C_out = d.C_out;
-  p.N_img = d.N;
   p.Ho = Ho;
   p.Wo = Wo;
-  p.Hq = Hq;
-  p.Wq = Wq;
+  p.Q = (int)Q;
   p.stride_h = d.stride_h;
   p.stride_w = d.stride_w;
   p.pad_h = d.pad_h;
@@ -818,8 +642,6 @@ static int32_t launch_variant(int dev, const ssconv_desc_t& d, const Geometry& g
   const long long q_tiles = (Q + kBN - 1) / kBN;
   p.num_tiles = (int)(q_tiles * geo.m_tiles);
   p.a_tiles = SPARSE ? geo.stages : geo.kblocks;
-  p.run_rows = HALO ? hp.run_rows : 0;
-  p.run_bytes = HALO ? hp.run_bytes : 0;
   p.flags = d.flags;
   p.bias = bias;
   p.meta = static_cast<const uint8_t*>(meta);
@@ -847,35 +669,8 @@ static int32_t launch_variant(int dev, const ssconv_desc_t& d, const Geometry& g
     p.ws_regions = nullptr;
     p.ws_counters = nullptr;
   }
-  const uint32_t smem_bytes = HALO ? (C::kSmemHaloFixed + kNRuns * hp.run_bytes) : C::kSmemIm2col;
-  ssconv_fwd_kernel<SPARSE, HALO><<<grid, kThreads, smem_bytes, stream>>>(tm_a, tm_b, p);
+  ssconv_fwd_kernel<SPARSE><<<grid, kThreads, C::kSmemBytes, stream>>>(tm_a, tm_b, p);
   return cudaGetLastError() == cudaSuccess ? SSCONV_OK : SSCONV_ERR_CUDA;
-}
-
-template <bool SPARSE>
-static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const void* weights, const void* meta,
-                                   const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
-                                   cudaStream_t stream, int worker_cap = kMaxWorkers, bool force_split = false) {
-  if (!load_driver_entry_points()) return SSCONV_ERR_CUDA;
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SSCONV_ERR_CUDA;
-  if (g_sm_count[dev] == 0) {
-    int major = 0, sms = 0;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SSCONV_ERR_CUDA;
-    if (major != 10) return SSCONV_ERR_ARCH;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-      return SSCONV_ERR_CUDA;
-    g_sm_count[dev] = sms;
-  }
-  const Geometry geo = make_geometry(d);
-  const int Ho = out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h);
-  const int Wo = out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
-  const HaloPlan hp = plan_halo<SPARSE>(d, Ho, Wo);
-  if (hp.use)
-    return launch_variant<SPARSE, true>(dev, d, geo, Ho, Wo, hp, x, weights, meta, bias, y, ws, ws_bytes, dev_status,
-                                        stream, worker_cap, force_split);
-  return launch_variant<SPARSE, false>(dev, d, geo, Ho, Wo, hp, x, weights, meta, bias, y, ws, ws_bytes, dev_status,
-                                       stream, worker_cap, force_split);
 }
 
 int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
