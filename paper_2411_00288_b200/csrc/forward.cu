@@ -15,10 +15,13 @@
 // fetch, about 64 B/clk, bounds the main loop either way, so the simpler scheme stays.)
 //
 // Warp roles: warp 0 TMA producer, warp 1 MMA issuer (one thread; owns TMEM), warps 2-9 epilogue
-// in two groups of four warps that each own half of a tile's positions: TMEM -> registers,
-// + bias, ReLU, bf16; neighbouring lanes (channels c, c+1) swap one value per position pair so
-// that every lane holds two adjacent channels of one position, and stores them as one 32-bit
-// word: a warp writes two 64-byte runs of NHWC per instruction, with no shared-memory staging.
+// in two groups of four warps that each own half of a tile's positions.  The accumulator has
+// channels on TMEM lanes and positions on columns, NHWC wants the transpose: the epilogue reads
+// TMEM in the MMA-fragment layout (tcgen05.ld 16x256b), adds the bias, converts pairs to bf16
+// (with ReLU in the conversion), and stmatrix.trans writes 8x8 blocks transposed into a 128-byte
+// swizzled staging buffer [position][channel], which TMA stores write to NHWC asynchronously.
+// That is about 2.5 instructions per thread and element pair; an epilogue of scalar shared-memory
+// stores or lane shuffles is issue-bound at several times that.
 //
 // Work partition: the unit of work is one weight tile's worth of K for one output tile.  Either
 // every CTA takes a contiguous block of whole output tiles, or (when whole tiles would leave many
@@ -42,7 +45,7 @@ namespace ssconv {
 constexpr int kBN = 240;                 // positions per tile (N of the MMA)
 constexpr int kGroups = 2;               // epilogue warp groups, each owning kBN / kGroups positions
 constexpr int kGroupCols = kBN / kGroups;
-constexpr int kPiece = 40;               // accumulator columns the epilogue handles at a time
+constexpr int kPiece = 40;               // positions per epilogue piece (one staging buffer)
 constexpr int kThreads = 64 + 128 * kGroups;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kAccCol1 = 256;       // second accumulator; the first starts at column 0
@@ -50,6 +53,9 @@ constexpr uint32_t kMetaCol = kBN;       // metadata: 2 slots x 4 columns in [24
 constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 1.9 GHz
 constexpr uint32_t kATileBytes = 128 * 128;          // 128 rows x 128 B
 constexpr uint32_t kBTileBytes = kBN * 128;          // 240 positions x 64 channels bf16
+constexpr uint32_t kHalfPieceBytes = kPiece * 128;    // 40 positions x 64 channels bf16, 128-byte swizzled
+constexpr uint32_t kPieceBytes = 2 * kHalfPieceBytes; // channels [0,64) then [64,128) of the tile
+constexpr uint32_t kStagingBytes = 2 * kGroups * kPieceBytes;  // two buffers per group
 constexpr uint32_t kBarrierBytes = 256;
 
 template <bool SPARSE>
@@ -59,7 +65,8 @@ struct Cfg {
   static constexpr uint32_t kAEntryBytes = kATileBytes + kMetaBytes;
   static constexpr int kNB = 4;                       // stages in the ring
   static constexpr int kNA = kNB / kBlocksPerA;       // weight slots, one per group of stages sharing a tile
-  static constexpr uint32_t kSmemBytes = kNA * kAEntryBytes + kNB * kBTileBytes + kBarrierBytes + 1024;
+  static constexpr uint32_t kSmemBytes =
+      kNA * kAEntryBytes + kNB * kBTileBytes + kStagingBytes + kBarrierBytes + 1024;
   static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 };
 
@@ -128,28 +135,53 @@ __device__ __forceinline__ int unit_owner(long long u, long long U, long long G)
   return (int)(((u + 1) * G - 1) / U);
 }
 
-// A scratch region holds one 128 x 240 fp32 partial tile as float4s ordered [4-column group][row],
-// so that a warp reads or writes 512 contiguous bytes at a time.
+// A scratch region holds one 128 x 240 fp32 partial tile in the order the epilogue threads hold it:
+// float4 number j (of 10) of piece `piece` of thread `gtid` of group `grp`, consecutive threads
+// adjacent, so that a warp reads or writes 512 contiguous bytes at a time.
 constexpr int kRegionVecs = kTileM * kBN / 4;
-__device__ __forceinline__ int region_vec(int col4, int row) { return col4 * kTileM + row; }
+constexpr int kPiecesPerGroup = kGroupCols / kPiece;
+__device__ __forceinline__ int region_vec(int grp, int piece, int j, int gtid) {
+  return ((grp * kPiecesPerGroup + piece) * (kPiece / 4) + j) * 128 + gtid;
+}
 // Region of CTA c for a split tile: its range starts inside the tile (0) or the tile starts inside
 // its range (1).  A range has at most one segment of each kind.
 __device__ __forceinline__ size_t region_index(int c, bool tile_starts_here) {
   return 2 * (size_t)c + (tile_starts_here ? 1 : 0);
 }
 
+// Named barriers: 1 and 2 for the epilogue groups, 3 for the setup (warp 0 arrives without waiting).
 __device__ __forceinline__ void epilogue_bar_sync(int group) {
   asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory");
 }
-// One epilogue piece (40 accumulator columns of this thread's lane) from TMEM; no wait.
+__device__ __forceinline__ void setup_bar_arrive() {
+  __threadfence_block();
+  asm volatile("bar.arrive 3, %0;" ::"n"(kThreads) : "memory");
+}
+__device__ __forceinline__ void setup_bar_sync() { asm volatile("bar.sync 3, %0;" ::"n"(kThreads) : "memory"); }
+// One epilogue piece of this warp's 32 lanes x 40 columns in fragment layout: register
+// r[20 h + 4 k + 2 s + e] = lane (16 h + 8 s + t/4), column (8 k + 2 (t%4) + e).  No wait.
 __device__ __forceinline__ void tc_ld_piece(uint32_t taddr, uint32_t (&r)[kPiece]) {
-  uint32_t a[32], b[8];
-  tc_ld_32x32(taddr, a);
-  tc_ld_32x8(taddr + 32, b);
 #pragma unroll
-  for (int j = 0; j < 32; ++j) r[j] = a[j];
+  for (int h = 0; h < 2; ++h) {
+    const uint32_t a = taddr + ((uint32_t)(16 * h) << 16);
+    tc_ld_16x256b_x4(a, &r[20 * h]);
+    tc_ld_16x256b_x1(a + 32, &r[20 * h + 16]);
+  }
+}
+// bias, activation and bf16 for one piece, written transposed to its staging buffer.  st_addr is
+// this thread's address for the first 8 positions; each further 8 positions are 1024 bytes on.
+template <bool RELU>
+__device__ __forceinline__ void stage_piece(const uint32_t (&r)[kPiece], const float (&bias)[4], uint32_t st_addr) {
 #pragma unroll
-  for (int j = 0; j < 8; ++j) r[32 + j] = b[j];
+  for (int k = 0; k < kPiece / 8; ++k) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {  // channel block i = 2 h + s of the warp's 32 channels
+      const int at = 20 * (i >> 1) + 4 * k + 2 * (i & 1);
+      w[i] = pack_bf16x2<RELU>(__uint_as_float(r[at]) + bias[i], __uint_as_float(r[at + 1]) + bias[i]);
+    }
+    stmatrix_x4_trans(st_addr + 1024u * k, w[0], w[1], w[2], w[3]);
+  }
 }
 
 // Position q -> (image, output row, output column).
@@ -168,7 +200,7 @@ __device__ __forceinline__ Pos decode_pos(int q, int Wq, int Hq) {
 template <bool SPARSE>
 __global__ void __launch_bounds__(kThreads, 1)
 ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                  const FwdParams p) {
+                  const __grid_constant__ CUtensorMap tm_y, const FwdParams p) {
   using C = Cfg<SPARSE>;
   constexpr int APER = C::kBlocksPerA;
   constexpr int kNA = C::kNA;
@@ -179,7 +211,8 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   uint8_t* a_ring = smem;                                        // kNA weight tiles (+ metadata)
   uint8_t* b_ring = a_ring + kNA * C::kAEntryBytes;              // kNB activation tiles
   // barrier slots: [0,8) stage full, [8,16) stage empty, [16,18) accumulator full, [18,20) accumulator empty
-  uint64_t* bars = reinterpret_cast<uint64_t*>(b_ring + kNB * kBTileBytes);
+  uint8_t* out_stage = b_ring + kNB * kBTileBytes;               // per group two staging buffers
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_stage + kStagingBytes);
   uint64_t* bar_full = bars;
   uint64_t* bar_empty = bars + 8;
   uint64_t* bar_acc_full = bars + 16;
@@ -192,24 +225,38 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < 16; ++s) mbar_init(&bars[s], 1);
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(&bar_acc_full[b], 1);
-      mbar_init(&bar_acc_empty[b], 4 * kGroups);
+  // Warp 0 initialises the barriers and goes straight on to load; everybody else also waits for
+  // the TMEM allocation (which the producer does not need).
+  if (warp == 0) {
+    if (lane == 0) {
+      grid_launch_dependents();  // the next grid in the stream may set itself up as SMs become free
+      prefetch_tensormap(&tm_a);
+      prefetch_tensormap(&tm_b);
+      for (int s = 0; s < kNB; ++s) {
+        mbar_init(&bar_full[s], 1);
+        mbar_init(&bar_empty[s], 1);
+      }
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(&bar_acc_full[b], 1);
+        mbar_init(&bar_acc_empty[b], 4 * kGroups);
+      }
+      *abort_flag = 0;
+      mbar_fence_init();
+      fence_proxy_async_smem();
     }
-    *abort_flag = 0;
-    mbar_fence_init();
-    fence_proxy_async_smem();
+    __syncwarp();
+    setup_bar_arrive();
+  } else {
+    if (warp == 1) {
+      tmem_alloc(tmem_slot, kTmemCols);
+      tmem_relinquish();
+    }
+    if (warp == 2 && lane == 0) prefetch_tensormap(&tm_y);
+    tc_fence_before();
+    setup_bar_sync();
+    tc_fence_after();
   }
-  if (warp == 1) {
-    tmem_alloc(tmem_slot, kTmemCols);
-    tmem_relinquish();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_base = (warp == 0) ? 0u : *tmem_slot;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -220,6 +267,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       const uint32_t a_smem0 = smem_u32(a_ring), b_smem0 = smem_u32(b_ring);
       uint32_t s = 0, ph = 0;  // stage and its phase parity
       bool ok = true;
+      bool first_segment = true;
       WorkIter work(p);
       Segment seg;
       while (ok && work.next(seg)) {
@@ -234,6 +282,12 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         int cc = kb0 / p.taps;          // channel chunk
         int tap = kb0 - cc * p.taps;
         int a_idx = seg.a0;
+        if (first_segment) {
+          // everything above ran concurrently with the tail of the previous grid in the stream;
+          // its results (our inputs) are complete from here on
+          grid_dependency_wait();
+          first_segment = false;
+        }
         {
           const int kh0 = tap / p.KW;
           int kw = tap - kh0 * p.KW;
@@ -376,19 +430,24 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   } else {
     // ------------------------------------------------------------------ epilogue
     // Two independent groups of four warps; group g owns positions [120 g, 120 g + 120) of every
-    // tile and has its own named barrier.  A thread reads accumulator lane `row` (one output
-    // channel) for 40 positions at a time.
+    // tile, with its own staging buffers and named barrier, and handles them 40 at a time.
     const int grp = (warp - 2) >> 2;
-    const int q = warp & 3;  // TMEM lane quadrant this warp may read
-    const int row = q * 32 + lane;
+    const int q = warp & 3;  // TMEM lane quadrant this warp may read: channels [32 q, 32 q + 32) of the tile
+    const int gtid = q * 32 + lane;
     const bool leader = (q == 2 && lane == 0);  // first warp of each group
     const bool relu = (p.flags & SSCONV_FLAG_RELU) != 0;
     const int col_base = grp * kGroupCols;
-    const int odd = lane & 1;
-    const size_t pos_step_bytes = (size_t)p.C_out * 2;  // one position further in NHWC
+    uint8_t* my_stage = out_stage + grp * 2 * kPieceBytes;
     volatile int* my_go = epi_go + 2 * grp;
     volatile int* my_last = epi_last + grp;
+    // stmatrix duty of this thread: 16 bytes = 8 channels of block (lane / 8) of the warp's four, at
+    // position (lane % 8) of each run of 8 positions; the 16-byte chunks of a 128-byte staging row
+    // are permuted by the row number (the swizzle the TMA store undoes)
+    const uint32_t st_offset = (uint32_t)(q >> 1) * kHalfPieceBytes + (uint32_t)(lane & 7) * 128u +
+                               ((((uint32_t)(q & 1) * 4u + (uint32_t)(lane >> 3)) ^ (uint32_t)(lane & 7)) << 4);
     uint32_t tcount = 0;
+    uint32_t piece_count = 0;
+    grid_dependency_wait();  // before the first access to global memory (bias, scratch, output)
     WorkIter work(p);
     Segment seg;
     for (; work.next(seg); ++tcount) {
@@ -403,8 +462,13 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       epilogue_bar_sync(grp);
       if (my_go[tcount & 1u] == 0) break;
       tc_fence_after();
-      const int co = m * kTileM + row;
-      const float bias_v = ((p.flags & SSCONV_FLAG_BIAS) && co < p.C_out) ? p.bias[co] : 0.0f;
+      // the four channels whose accumulators this thread receives: 8 i + lane / 4 of the warp's 32
+      float bias_v[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int co = m * kTileM + q * 32 + 8 * i + (lane >> 2);
+        bias_v[i] = ((p.flags & SSCONV_FLAG_BIAS) && co < p.C_out) ? p.bias[co] : 0.0f;
+      }
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCol1 + col_base;
       const bool whole = (seg.a0 == 0 && seg.a1 == p.a_tiles);
       int c_first = 0, c_last = 0;
@@ -415,13 +479,13 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         c_last = unit_owner(u_first + p.a_tiles - 1, p.units, gridDim.x);
         float4* mine = p.ws_regions + region_index(blockIdx.x, seg.a0 == 0) * kRegionVecs;
 #pragma unroll 1
-        for (int c0 = 0; c0 < kGroupCols; c0 += kPiece) {
+        for (int piece = 0; piece < kPiecesPerGroup; ++piece) {
           uint32_t r[kPiece];
-          tc_ld_piece(t_row + c0, r);
+          tc_ld_piece(t_row + piece * kPiece, r);
           tc_wait_ld();
 #pragma unroll
           for (int j = 0; j < kPiece / 4; ++j)
-            __stcg(mine + region_vec((col_base + c0) / 4 + j, row),
+            __stcg(mine + region_vec(grp, piece, j, gtid),
                    make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
                                __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3])));
         }
@@ -438,21 +502,15 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         if (*my_last == 0) continue;  // someone else finishes this half tile
         __threadfence();
       }
-      // ---- finish the tile: bias, activation, bf16, lane-pair exchange, 32-bit stores -----------
-      // Lanes 2t and 2t+1 hold channels c and c+1 of the same positions.  Per position pair
-      // (j, j+1) they swap one value, after which the even lane has both channels of position j and
-      // the odd lane both channels of position j+1.
-      const int q_lane = pt * kBN + col_base + odd;  // first position this lane stores
-      const int co_pair = m * kTileM + (row & ~1);
-      int q_left = (co_pair < p.C_out) ? p.Q - q_lane : 0;  // positions q_lane + j with j < q_left exist
-      uint8_t* y_lane = reinterpret_cast<uint8_t*>(p.y + (size_t)q_lane * p.C_out + co_pair);
+      // ---- finish the tile: bias, activation, bf16, transposed staging, TMA stores ---------------
 #pragma unroll 1
-      for (int piece = 0; piece < kGroupCols / kPiece; ++piece) {
+      for (int piece = 0; piece < kPiecesPerGroup; ++piece, ++piece_count) {
+        uint8_t* stage = my_stage + (piece_count & 1u) * kPieceBytes;
         uint32_t r[kPiece];
         if (whole) {
           tc_ld_piece(t_row + piece * kPiece, r);
           tc_wait_ld();
-          if (piece == kGroupCols / kPiece - 1) {
+          if (piece == kPiecesPerGroup - 1) {
             // this warp's part of the accumulator is read: hand it back to the MMA thread
             tc_fence_before();
             __syncwarp();
@@ -462,12 +520,11 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
           // sum the contributors' regions in CTA order (reads bypass L1: the data came from other SMs)
 #pragma unroll
           for (int j = 0; j < kPiece; ++j) r[j] = 0u;
-          const int v0 = (col_base + piece * kPiece) / 4;
           for (int c = c_first; c <= c_last; ++c) {
             const float4* src = p.ws_regions + region_index(c, c == c_first) * kRegionVecs;
             float4 v[kPiece / 4];
 #pragma unroll
-            for (int j = 0; j < kPiece / 4; ++j) v[j] = __ldcg(src + region_vec(v0 + j, row));
+            for (int j = 0; j < kPiece / 4; ++j) v[j] = __ldcg(src + region_vec(grp, piece, j, gtid));
 #pragma unroll
             for (int j = 0; j < kPiece / 4; ++j) {
               r[4 * j] = __float_as_uint(__uint_as_float(r[4 * j]) + v[j].x);
@@ -477,24 +534,31 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             }
           }
         }
-#pragma unroll
-        for (int i = 0; i < kPiece / 2; ++i) {
-          float v0 = __uint_as_float(r[2 * i]) + bias_v;
-          float v1 = __uint_as_float(r[2 * i + 1]) + bias_v;
-          if (relu) {
-            v0 = fmaxf(v0, 0.0f);
-            v1 = fmaxf(v1, 0.0f);
+        // The buffer was last the source of the store issued two pieces ago; the leader saw that
+        // store finish reading before it entered the barrier of the previous piece.
+        const uint32_t st_addr = smem_u32(stage) + st_offset;
+        if (relu)
+          stage_piece<true>(r, bias_v, st_addr);
+        else
+          stage_piece<false>(r, bias_v, st_addr);
+        fence_proxy_async_smem();           // generic-proxy writes -> visible to the TMA store
+        if (leader) bulk_wait_group_read0();  // the previous piece's store no longer reads its buffer
+        epilogue_bar_sync(grp);
+        if (leader) {
+          const int q_piece = pt * kBN + col_base + piece * kPiece;
+          if (q_piece < p.Q) {
+            // positions beyond Q and channels beyond C_out fall outside the tensor map and are dropped
+            tma_store_2d(&tm_y, stage, m * kTileM, q_piece);
+            if (m * kTileM + 64 < p.C_out) tma_store_2d(&tm_y, stage + kHalfPieceBytes, m * kTileM + 64, q_piece);
           }
-          const float got_v = __shfl_xor_sync(0xFFFFFFFFu, odd ? v0 : v1, 1);
-          const __nv_bfloat162 pair = __floats2bfloat162_rn(odd ? got_v : v0, odd ? v1 : got_v);
-          if (2 * i < q_left)
-            *reinterpret_cast<__nv_bfloat162*>(y_lane + (size_t)(2 * i) * pos_step_bytes) = pair;
+          bulk_commit_group();
         }
-        q_left -= kPiece;
-        y_lane += (size_t)kPiece * pos_step_bytes;
       }
       if (!whole && leader) p.ws_counters[2 * c_first + grp] = 0;  // zero again for the next launch
     }
+    // the stores have read their staging buffers before shared memory is released; the writes
+    // themselves complete with the grid
+    if (leader) bulk_wait_group_read0();
   }
 
   // ------------------------------------------------------------------ teardown
@@ -586,7 +650,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   const long long Q = (long long)d.N * Ho * Wo;  // positions
   if (Q > 0x7FFFFF00LL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
 
-  CUtensorMap tm_a, tm_b;
+  CUtensorMap tm_a, tm_b, tm_y;
   // activations: NHWC seen as (c, w, h, n), im2col mode; elements outside the image read as zero
   // (= the zero padding of Eq. 4); base pixels are the filter placements, each load adds a tap offset
   {
@@ -619,6 +683,17 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     CUresult r = g_encode_tiled(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(weights), dims, strides,
                                 box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
+  }
+  // output: NHWC seen as (c, position); a box is one staging half piece, 64 channels x 40 positions
+  {
+    cuuint64_t dims[2] = {(cuuint64_t)d.C_out, (cuuint64_t)Q};
+    cuuint64_t strides[1] = {(cuuint64_t)d.C_out * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kPiece};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode_tiled(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
   }
 
@@ -669,8 +744,21 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     p.ws_regions = nullptr;
     p.ws_counters = nullptr;
   }
-  ssconv_fwd_kernel<SPARSE><<<grid, kThreads, C::kSmemBytes, stream>>>(tm_a, tm_b, p);
-  return cudaGetLastError() == cudaSuccess ? SSCONV_OK : SSCONV_ERR_CUDA;
+  // Programmatic stream serialisation: this grid's set-up (barriers, TMEM, tensor-map fetch, index
+  // arithmetic) may overlap the tail of the previous kernel in the stream; the kernel itself
+  // waits for that kernel's completion before it touches global memory.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)kThreads);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE>, tm_a, tm_b, tm_y, p) == cudaSuccess ? SSCONV_OK
+                                                                                                 : SSCONV_ERR_CUDA;
 }
 
 int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
