@@ -116,12 +116,11 @@ int32_t ssconv_decompress(const ssconv_desc_t* desc, const void* w_comp, const v
  * pad <= 127, dil*(K-1) <= 255, stride <= 8.
  * ws: device scratch of at least the size ssconv_sizes reports, 16-byte aligned.  It is used
  * only by layers with too few output tiles to fill the GPU, whose K range is then split over
- * several thread blocks that park fp32 partial results there and sum them in a fixed order,
- * so results are reproducible.  Contract: the caller zero-fills ws once (only the counters at
- * its end must be zero, the rest is overwritten before it is read); every call that completes
- * leaves the counters zero, so ws can be reused by later calls on the same stream.  Calls
- * that may overlap on the GPU need separate workspaces.  After SSCONV_ERR_TIMEOUT zero-fill
- * it again.  If ws is NULL or too small and
+ * several thread blocks that park fp32 partial results there; a second small kernel, launched
+ * by the same call, sums them in a fixed order, so results are reproducible.  ws needs no
+ * initialisation: every part is written before it is read.  Calls issued one after another on
+ * one stream may share it; calls that may overlap on the GPU need separate workspaces.
+ * If ws is NULL or too small and
  * the layer needs it, SSCONV_ERR_WORKSPACE is returned and nothing is launched.
  * dev_status (nullable): device int32; a kernel whose bounded wait expires stores
  * SSCONV_ERR_TIMEOUT there and drains instead of hanging; it is never written on success,
@@ -157,9 +156,9 @@ int32_t ssconv_forward_dense(const ssconv_desc_t* desc, const void* x, const voi
  *    and with it the last bits of y, can differ from ssconv_forward's.
  *  - The first call on each device looks up the array's device address (with that device
  *    current); make that first call outside any stream capture.
- *  - All calls share the one array, and it keeps what the previous call left in it.  Each call
- *    clears the arrival counters it relies on before its kernel runs (stream-ordered), so calls
- *    issued one after another on one stream are safe; two calls that can overlap on the GPU
+ *  - All calls share the one array, and it keeps what the previous call left in it.  Nothing in
+ *    it has to be cleared (every partial sum is written before it is read), so calls issued one
+ *    after another on one stream are safe; two calls that can overlap on the GPU
  *    (different streams, no dependency) race on the array and give wrong results. */
 int32_t ssconv_forward_static_ws(const ssconv_desc_t* desc, const void* x, const void* w_comp,
                                  const void* meta, const float* bias, void* y, int32_t* dev_status,

@@ -178,14 +178,14 @@ _workspaces = {}
 
 
 def default_workspace(device) -> torch.Tensor:
-    """One zero-filled scratch buffer per device, shared by calls that pass ws=None.  The forward
-    kernels leave it zero-filled, so stream-ordered calls can share it; calls on different streams
-    that may overlap must pass their own."""
+    """One scratch buffer per device, shared by calls that pass ws=None.  It needs no initialisation
+    (the kernels write every part before reading it), so stream-ordered calls can share it; calls
+    on different streams that may overlap must pass their own."""
     dev = torch.device(device)
     key = dev.index if dev.index is not None else torch.cuda.current_device()
     if key not in _workspaces:
         nbytes = ssconv_sizes(make_desc(1, 8, 8, 8, 8, 1, 1)).ws_bytes_sparse
-        _workspaces[key] = torch.zeros((nbytes,), dtype=torch.uint8, device=torch.device("cuda", key))
+        _workspaces[key] = torch.empty((nbytes,), dtype=torch.uint8, device=torch.device("cuda", key))
     return _workspaces[key]
 
 

@@ -27,9 +27,9 @@
 // every CTA takes a contiguous block of whole output tiles, or (when whole tiles would leave many
 // SMs idle) the units are dealt out evenly, so a CTA's range may start and end inside an
 // output tile ("stream-K").  A CTA writes a partly computed tile (fp32) to a scratch region of its
-// own in global memory and bumps the tile's counter; the last CTA to arrive sums the regions of all
-// contributors in a fixed order, finishes the epilogue and resets the counter.  No CTA ever waits
-// for another, and the result does not depend on the order of arrival.
+// own in global memory; a second, small kernel (ssconv_split_finish_kernel) then sums the regions
+// of every split tile in a fixed order on all SMs and applies the same epilogue.  No CTA ever
+// waits for another, and the result does not depend on timing.
 // All mbarrier waits are bounded; when one runs out the CTA raises a flag, every role leaves
 // its loop, TMEM is freed and SSCONV_ERR_TIMEOUT is stored to *dev_status.
 #include <cuda.h>
@@ -81,7 +81,6 @@ struct FwdParams {
   int split;                // 1: units dealt out evenly across CTAs (stream-K); 0: whole tiles per CTA
   long long units;          // num_tiles * a_tiles
   float4* ws_regions;       // [2 * gridDim.x] regions of 128 x 240 fp32: a CTA's partial tiles
-  int* ws_counters;         // [gridDim.x][2] arrivals per split tile and epilogue group, zero between launches
   uint32_t flags;
   const float* bias;
   const uint8_t* meta;
@@ -220,7 +219,6 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = abort_flag + 1;         // per group two slots: the leader's go/stop verdict per tile
-  volatile int* epi_last = epi_go + 2 * kGroups;  // per group: partial tile, is this CTA the last to arrive?
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -439,7 +437,6 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     const int col_base = grp * kGroupCols;
     uint8_t* my_stage = out_stage + grp * 2 * kPieceBytes;
     volatile int* my_go = epi_go + 2 * grp;
-    volatile int* my_last = epi_last + grp;
     // stmatrix duty of this thread: 16 bytes = 8 channels of block (lane / 8) of the warp's four, at
     // position (lane % 8) of each run of 8 positions; the 16-byte chunks of a 128-byte staging row
     // are permuted by the row number (the swizzle the TMA store undoes)
@@ -462,21 +459,11 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       epilogue_bar_sync(grp);
       if (my_go[tcount & 1u] == 0) break;
       tc_fence_after();
-      // the four channels whose accumulators this thread receives: 8 i + lane / 4 of the warp's 32
-      float bias_v[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int co = m * kTileM + q * 32 + 8 * i + (lane >> 2);
-        bias_v[i] = ((p.flags & SSCONV_FLAG_BIAS) && co < p.C_out) ? p.bias[co] : 0.0f;
-      }
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCol1 + col_base;
       const bool whole = (seg.a0 == 0 && seg.a1 == p.a_tiles);
-      int c_first = 0, c_last = 0;
       if (!whole) {
-        // ---- partial tile: park this CTA's share in its own scratch region --------------------
-        const long long u_first = (long long)seg.tile * p.a_tiles;
-        c_first = unit_owner(u_first, p.units, gridDim.x);
-        c_last = unit_owner(u_first + p.a_tiles - 1, p.units, gridDim.x);
+        // ---- partial tile: park this CTA's share in its own scratch region; the finishing kernel
+        // sums the shares of all contributors
         float4* mine = p.ws_regions + region_index(blockIdx.x, seg.a0 == 0) * kRegionVecs;
 #pragma unroll 1
         for (int piece = 0; piece < kPiecesPerGroup; ++piece) {
@@ -492,47 +479,27 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
-        __threadfence();
-        epilogue_bar_sync(grp);
-        if (leader) {
-          const int arrived = atomicAdd(p.ws_counters + 2 * c_first + grp, 1);
-          *my_last = (arrived == c_last - c_first) ? 1 : 0;
-        }
-        epilogue_bar_sync(grp);
-        if (*my_last == 0) continue;  // someone else finishes this half tile
-        __threadfence();
+        continue;
       }
       // ---- finish the tile: bias, activation, bf16, transposed staging, TMA stores ---------------
+      // the four channels whose accumulators this thread receives: 8 i + lane / 4 of the warp's 32
+      float bias_v[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int co = m * kTileM + q * 32 + 8 * i + (lane >> 2);
+        bias_v[i] = ((p.flags & SSCONV_FLAG_BIAS) && co < p.C_out) ? p.bias[co] : 0.0f;
+      }
 #pragma unroll 1
       for (int piece = 0; piece < kPiecesPerGroup; ++piece, ++piece_count) {
         uint8_t* stage = my_stage + (piece_count & 1u) * kPieceBytes;
         uint32_t r[kPiece];
-        if (whole) {
-          tc_ld_piece(t_row + piece * kPiece, r);
-          tc_wait_ld();
-          if (piece == kPiecesPerGroup - 1) {
-            // this warp's part of the accumulator is read: hand it back to the MMA thread
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
-          }
-        } else {
-          // sum the contributors' regions in CTA order (reads bypass L1: the data came from other SMs)
-#pragma unroll
-          for (int j = 0; j < kPiece; ++j) r[j] = 0u;
-          for (int c = c_first; c <= c_last; ++c) {
-            const float4* src = p.ws_regions + region_index(c, c == c_first) * kRegionVecs;
-            float4 v[kPiece / 4];
-#pragma unroll
-            for (int j = 0; j < kPiece / 4; ++j) v[j] = __ldcg(src + region_vec(grp, piece, j, gtid));
-#pragma unroll
-            for (int j = 0; j < kPiece / 4; ++j) {
-              r[4 * j] = __float_as_uint(__uint_as_float(r[4 * j]) + v[j].x);
-              r[4 * j + 1] = __float_as_uint(__uint_as_float(r[4 * j + 1]) + v[j].y);
-              r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + v[j].z);
-              r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + v[j].w);
-            }
-          }
+        tc_ld_piece(t_row + piece * kPiece, r);
+        tc_wait_ld();
+        if (piece == kPiecesPerGroup - 1) {
+          // this warp's part of the accumulator is read: hand it back to the MMA thread
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
         }
         // The buffer was last the source of the store issued two pieces ago; the leader saw that
         // store finish reading before it entered the barrier of the previous piece.
@@ -554,7 +521,6 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
           bulk_commit_group();
         }
       }
-      if (!whole && leader) p.ws_counters[2 * c_first + grp] = 0;  // zero again for the next launch
     }
     // the stores have read their staging buffers before shared memory is released; the writes
     // themselves complete with the grid
@@ -576,6 +542,103 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     tmem_dealloc(tmem_base, kTmemCols);
   }
 }
+
+// ---------------------------------------------------------------------------------------
+// Finishing kernel of the split-K path
+// ---------------------------------------------------------------------------------------
+// One CTA of 128 threads finishes 128 channels x 8 positions of one split tile: thread gtid sums,
+// in CTA order, the two float4s it would have held in the main kernel's epilogue (fragment
+// layout, see region_vec), applies bias / ReLU / bf16, and the block is transposed through shared
+// memory by stmatrix.trans exactly as in the main kernel before 16-byte stores write NHWC.
+struct FinishParams {
+  int C_out, Q;
+  int m_tiles, a_tiles;
+  int workers;            // grid size of the main kernel
+  long long units;
+  const float4* ws_regions;
+  uint32_t flags;
+  const float* bias;
+  __nv_bfloat16* y;
+};
+constexpr int kFinishThreads = 128;
+constexpr int kFinishItemsPerTile = kGroups * kPiecesPerGroup * (kPiece / 8);
+constexpr int kFinishBatch = 8;  // contributors whose loads are in flight together
+
+__global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(const FinishParams f) {
+  __shared__ __align__(128) uint8_t stage[8 * 256];  // [position][128 channels], 16-byte chunks permuted per row
+  const int gtid = threadIdx.x, lane = gtid & 31, q = gtid >> 5;
+  int item = blockIdx.x;
+  const int k = item % (kPiece / 8);
+  item /= (kPiece / 8);
+  const int piece = item % kPiecesPerGroup;
+  item /= kPiecesPerGroup;
+  const int grp = item % kGroups;
+  const int tile = item / kGroups;
+  if (gtid == 0) grid_launch_dependents();
+  const long long u_first = (long long)tile * f.a_tiles;
+  const int c_first = unit_owner(u_first, f.units, f.workers);
+  const int c_last = unit_owner(u_first + f.a_tiles - 1, f.units, f.workers);
+  if (c_first == c_last) return;  // the tile was computed whole by one CTA, which also finished it
+  const int pt = tile / f.m_tiles;
+  const int m = tile - pt * f.m_tiles;
+  grid_dependency_wait();  // the main kernel's partial tiles are complete and visible
+
+  float4 acc0 = make_float4(0.f, 0.f, 0.f, 0.f), acc1 = acc0;
+  const int at0 = region_vec(grp, piece, k, gtid);               // lanes 0-15 of the warp's quadrant
+  const int at1 = region_vec(grp, piece, kPiece / 8 + k, gtid);  // lanes 16-31
+  for (int c0 = c_first; c0 <= c_last; c0 += kFinishBatch) {
+    float4 v0[kFinishBatch], v1[kFinishBatch];
+#pragma unroll
+    for (int i = 0; i < kFinishBatch; ++i) {
+      const int c = c0 + i;
+      if (c <= c_last) {
+        const float4* src = f.ws_regions + region_index(c, c == c_first) * kRegionVecs;
+        v0[i] = __ldcg(src + at0);
+        v1[i] = __ldcg(src + at1);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kFinishBatch; ++i) {
+      if (c0 + i <= c_last) {
+        acc0.x += v0[i].x; acc0.y += v0[i].y; acc0.z += v0[i].z; acc0.w += v0[i].w;
+        acc1.x += v1[i].x; acc1.y += v1[i].y; acc1.z += v1[i].z; acc1.w += v1[i].w;
+      }
+    }
+  }
+  float bias_v[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int co = m * kTileM + q * 32 + 8 * i + (lane >> 2);
+    bias_v[i] = ((f.flags & SSCONV_FLAG_BIAS) && co < f.C_out) ? f.bias[co] : 0.0f;
+  }
+  uint32_t w[4];
+  if (f.flags & SSCONV_FLAG_RELU) {
+    w[0] = pack_bf16x2<true>(acc0.x + bias_v[0], acc0.y + bias_v[0]);
+    w[1] = pack_bf16x2<true>(acc0.z + bias_v[1], acc0.w + bias_v[1]);
+    w[2] = pack_bf16x2<true>(acc1.x + bias_v[2], acc1.y + bias_v[2]);
+    w[3] = pack_bf16x2<true>(acc1.z + bias_v[3], acc1.w + bias_v[3]);
+  } else {
+    w[0] = pack_bf16x2<false>(acc0.x + bias_v[0], acc0.y + bias_v[0]);
+    w[1] = pack_bf16x2<false>(acc0.z + bias_v[1], acc0.w + bias_v[1]);
+    w[2] = pack_bf16x2<false>(acc1.x + bias_v[2], acc1.y + bias_v[2]);
+    w[3] = pack_bf16x2<false>(acc1.z + bias_v[3], acc1.w + bias_v[3]);
+  }
+  // thread 8 i + j of a warp addresses position j of channel block i of the warp's four
+  const uint32_t row = (uint32_t)(lane & 7);
+  const uint32_t chunk = (uint32_t)(4 * q + (lane >> 3));
+  stmatrix_x4_trans(smem_u32(stage) + row * 256u + ((chunk ^ row) << 4), w[0], w[1], w[2], w[3]);
+  __syncthreads();
+  {
+    const int pos = gtid >> 4, ch16 = gtid & 15;  // 16 threads write the 256 contiguous bytes of one position
+    const int q_pos = pt * kBN + grp * kGroupCols + piece * kPiece + 8 * k + pos;
+    const int co = m * kTileM + 8 * ch16;
+    if (q_pos < f.Q && co < f.C_out) {
+      const uint4 v = *reinterpret_cast<const uint4*>(stage + pos * 256 + ((ch16 ^ pos) << 4));
+      *reinterpret_cast<uint4*>(f.y + (size_t)q_pos * f.C_out + co) = v;
+    }
+  }
+}
+
 
 // ---------------------------------------------------------------------------------------
 // host side
@@ -609,13 +672,13 @@ static int out_extent(int in, int k, int stride, int pad, int dil) {
   return span < 0 ? 0 : span / stride + 1;
 }
 
-// Scratch for partly computed tiles: two fp32 regions (128 x 240) and two counters per CTA.
+// Scratch for partly computed tiles: two fp32 regions (128 x 240) per CTA.
 constexpr int kMaxWorkers = 148;
 constexpr size_t kRegionBytes = (size_t)kTileM * kBN * sizeof(float);
 constexpr double kCyclesPerATile = 1200.0;
 constexpr double kSplitFixedCycles = 18000.0;
 constexpr size_t scratch_bytes(int workers) {
-  return 2 * (size_t)workers * kRegionBytes + 2 * (size_t)workers * sizeof(int);
+  return 2 * (size_t)workers * kRegionBytes;
 }
 size_t workspace_bytes() { return scratch_bytes(kMaxWorkers); }
 
@@ -726,8 +789,8 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.units = (long long)p.num_tiles * p.a_tiles;
   int workers = g_sm_count[dev] < worker_cap ? g_sm_count[dev] : worker_cap;
   // Whole tiles per CTA, unless dealing the K range out evenly is clearly faster by a simple
-  // cost model: cycles per weight tile in the main loop, and a fixed cost for parking, summing
-  // and finishing partial tiles (both measured on B200).
+  // cost model: cycles per weight tile in the main loop, and a fixed cost for parking partial tiles
+  // and for the finishing kernel (both measured on B200).
   const int waves = (p.num_tiles + workers - 1) / workers;
   const double whole_cost = (double)waves * p.a_tiles * kCyclesPerATile;
   const double split_cost = (double)p.units / workers * kCyclesPerATile + kSplitFixedCycles;
@@ -738,11 +801,9 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     if (ws == nullptr || ws_bytes < scratch_bytes(worker_cap)) return SSCONV_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(ws) & 15u) return SSCONV_ERR_ALIGNMENT;
     p.ws_regions = static_cast<float4*>(ws);
-    p.ws_counters = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + 2 * (size_t)worker_cap * kRegionBytes);
   } else {
     grid = p.num_tiles < workers ? p.num_tiles : workers;
     p.ws_regions = nullptr;
-    p.ws_counters = nullptr;
   }
   // Programmatic stream serialisation: this grid's set-up (barriers, TMEM, tensor-map fetch, index
   // arithmetic) may overlap the tail of the previous kernel in the stream; the kernel itself
@@ -757,8 +818,25 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE>, tm_a, tm_b, tm_y, p) == cudaSuccess ? SSCONV_OK
-                                                                                                 : SSCONV_ERR_CUDA;
+  if (cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE>, tm_a, tm_b, tm_y, p) != cudaSuccess) return SSCONV_ERR_CUDA;
+  if (p.split) {
+    FinishParams f;
+    f.C_out = d.C_out;
+    f.Q = (int)Q;
+    f.m_tiles = geo.m_tiles;
+    f.a_tiles = p.a_tiles;
+    f.workers = grid;
+    f.units = p.units;
+    f.ws_regions = p.ws_regions;
+    f.flags = d.flags;
+    f.bias = bias;
+    f.y = p.y;
+    cfg.gridDim = dim3((unsigned)p.num_tiles * kFinishItemsPerTile);
+    cfg.blockDim = dim3((unsigned)kFinishThreads);
+    cfg.dynamicSmemBytes = 0;
+    if (cudaLaunchKernelEx(&cfg, ssconv_split_finish_kernel, f) != cudaSuccess) return SSCONV_ERR_CUDA;
+  }
+  return SSCONV_OK;
 }
 
 int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
@@ -799,11 +877,8 @@ int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const vo
     g_static_scratch_ptr[dev] = ptr;
   }
   unsigned char* scratch = g_static_scratch_ptr[dev];
-  // The arrival counters must start at zero; the partial-sum regions are overwritten before use.
-  // The array keeps whatever the previous call left (an aborted call can leave counts behind).
-  const size_t counters_at = 2 * (size_t)kStaticWorkers * kRegionBytes;
-  if (cudaMemsetAsync(scratch + counters_at, 0, 2 * (size_t)kStaticWorkers * sizeof(int), stream) != cudaSuccess)
-    return SSCONV_ERR_CUDA;
+  // Nothing in the array has to be cleared: it keeps whatever the previous call left, and every
+  // partial-sum region is written by this call's main kernel before its finishing kernel reads it.
   return launch_forward_impl<true>(d, x, w_comp, meta, bias, y, scratch, scratch_bytes(kStaticWorkers), dev_status,
                                    stream, kStaticWorkers, true);
 }
