@@ -675,8 +675,15 @@ static int out_extent(int in, int k, int stride, int pad, int dil) {
 // Scratch for partly computed tiles: two fp32 regions (128 x 240) per CTA.
 constexpr int kMaxWorkers = 148;
 constexpr size_t kRegionBytes = (size_t)kTileM * kBN * sizeof(float);
-constexpr double kCyclesPerATile = 1200.0;
-constexpr double kSplitFixedCycles = 18000.0;
+// Cost model of the choice between whole tiles and an even split of K (cycles, measured on B200):
+// a k-block of 64 dense columns takes about 600 cycles sparse and 720 dense; an epilogue that
+// nothing overlaps about 3500; and every parked partial tile costs the chip about 90 cycles of
+// L2 traffic (123 KB written by the main kernel and read again by the finishing kernel).
+constexpr double kCyclesPerKBlockSparse = 600.0;
+constexpr double kCyclesPerKBlockDense = 720.0;
+constexpr double kEpilogueCycles = 3500.0;
+constexpr double kCyclesPerParkedTile = 90.0;
+constexpr double kSplitAdvantage = 1.1;  // split only if the model predicts at least this gain
 constexpr size_t scratch_bytes(int workers) {
   return 2 * (size_t)workers * kRegionBytes;
 }
@@ -788,13 +795,14 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
 
   p.units = (long long)p.num_tiles * p.a_tiles;
   int workers = g_sm_count[dev] < worker_cap ? g_sm_count[dev] : worker_cap;
-  // Whole tiles per CTA, unless dealing the K range out evenly is clearly faster by a simple
-  // cost model: cycles per weight tile in the main loop, and a fixed cost for parking partial tiles
-  // and for the finishing kernel (both measured on B200).
+  // Whole tiles per CTA, unless dealing the K range out evenly is clearly faster by the cost model.
+  const double a_tile_cycles = SPARSE ? 2.0 * kCyclesPerKBlockSparse : kCyclesPerKBlockDense;
   const int waves = (p.num_tiles + workers - 1) / workers;
-  const double whole_cost = (double)waves * p.a_tiles * kCyclesPerATile;
-  const double split_cost = (double)p.units / workers * kCyclesPerATile + kSplitFixedCycles;
-  p.split = (p.a_tiles > 1 && (force_split || whole_cost > 1.15 * split_cost)) ? 1 : 0;
+  const double whole_cost = (double)waves * p.a_tiles * a_tile_cycles + kEpilogueCycles;
+  const double split_ctas = p.units < workers ? (double)p.units : (double)workers;
+  const double split_cost =
+      (double)p.units / split_ctas * a_tile_cycles + (split_ctas + p.num_tiles) * kCyclesPerParkedTile;
+  p.split = (p.a_tiles > 1 && (force_split || whole_cost > kSplitAdvantage * split_cost)) ? 1 : 0;
   int grid;
   if (p.split) {
     grid = p.units < workers ? (int)p.units : workers;
