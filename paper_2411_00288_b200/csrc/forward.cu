@@ -372,54 +372,76 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         uint32_t accumulate = 0;
         const int kb0 = seg.a0 * APER;
         const int kb1 = (seg.a1 * APER < p.kblocks) ? seg.a1 * APER : p.kblocks;
-        int cc = kb0 / p.taps;
-        int tap = kb0 - cc * p.taps;
         uint32_t a_lo = 0, meta_tmem = 0;
-        {
-          for (int left = (seg.a1 - seg.a0) * APER, kb = kb0; left > 0; --left, ++kb) {
-            if (!mbar_wait_a(full0 + 8u * s, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-            tc_fence_after();
-            if (kb < kb1) {
-              const uint32_t a_sub = (APER == 2) ? (s & 1u) : 0u;
+        const int n_stages = (seg.a1 - seg.a0) * APER;  // stages this segment occupies
+        // k-blocks before the last channel chunk need the full number of MMAs: they take the lean
+        // loop.  This thread's instruction stream paces the tensor pipe (its queue is shallow), so
+        // the loop holds nothing but the wait, the MMAs and the commit.
+        const int tail_start = (tail_c == kBlockK) ? p.kblocks : last_cc * p.taps;
+        int n_lean = ((kb1 < tail_start) ? kb1 : tail_start) - kb0;
+        if (n_lean < 0) n_lean = 0;
+        int done_stages = 0;
+        for (; done_stages < n_lean; ++done_stages) {
+          if (!mbar_wait_a(full0 + 8u * s, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+          const uint32_t b_lo = b_lo0 + s * kBTileDesc;
+          if (SPARSE) {
+            const uint32_t a_sub = s & 1u;
+            if (a_sub == 0) {
+              a_lo = a_lo0 + (s >> 1) * kAEntryDesc;
+              meta_tmem = meta_tmem0 + 4u * mslot;
+              mslot ^= 1u;
+              tc_cp_128x128b_lo(meta_tmem, m_lo0 + (s >> 1) * kAEntryDesc);
+            }
+            // k-block a_sub of the weight tile: kept values start 64 B in, metadata 2 columns in;
+            // per MMA A advances 16 kept values = 32 B, B 32 channels = 64 B (descriptor units of 16 B)
+            const uint32_t a_kb = a_lo + 4u * a_sub;
+            const uint32_t meta_kb = meta_tmem + 2u * a_sub;
+            tc_mma_sparse_lo(d_tmem, a_kb, b_lo, meta_kb, idesc, accumulate);
+            tc_mma_sparse_lo(d_tmem, a_kb + 2u, b_lo + 4u, meta_kb, idesc | 1u, 1u);
+          } else {
+            a_lo = a_lo0 + s * kAEntryDesc;
+            tc_mma_dense_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
+            tc_mma_dense_lo(d_tmem, a_lo + 2u, b_lo + 2u, idesc, 1u);
+            tc_mma_dense_lo(d_tmem, a_lo + 4u, b_lo + 4u, idesc, 1u);
+            tc_mma_dense_lo(d_tmem, a_lo + 6u, b_lo + 6u, idesc, 1u);
+          }
+          accumulate = 1;
+          tc_commit_a(empty0 + 8u * s);
+          if (++s == (uint32_t)kNB) {
+            s = 0;
+            ph ^= 1u;
+          }
+        }
+        // the rest: k-blocks of the last channel chunk (possibly fewer MMAs) and, for a weight tile
+        // whose second k-block does not exist, a stage that only keeps the ring's phases in step
+        for (int kb = kb0 + done_stages; ok && done_stages < n_stages; ++done_stages, ++kb) {
+          if (!mbar_wait_a(full0 + 8u * s, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+          if (kb < kb1) {
+            const uint32_t b_lo = b_lo0 + s * kBTileDesc;
+            const int n_mma = (kb >= tail_start) ? mma_tail : (SPARSE ? 2 : 4);
+            if (SPARSE) {
+              const uint32_t a_sub = s & 1u;
               if (a_sub == 0) {
-                a_lo = a_lo0 + (s / APER) * kAEntryDesc;
-                if (SPARSE) {
-                  meta_tmem = meta_tmem0 + 4u * mslot;
-                  mslot ^= 1u;
-                  tc_cp_128x128b_lo(meta_tmem, m_lo0 + (s / APER) * kAEntryDesc);
-                }
+                a_lo = a_lo0 + (s >> 1) * kAEntryDesc;
+                meta_tmem = meta_tmem0 + 4u * mslot;
+                mslot ^= 1u;
+                tc_cp_128x128b_lo(meta_tmem, m_lo0 + (s >> 1) * kAEntryDesc);
               }
-              const uint32_t b_lo = b_lo0 + s * kBTileDesc;
-              const bool tail = (cc == last_cc);
-              if (SPARSE) {
-                // k-block a_sub of the weight tile: kept values start 64 B in, metadata 2 columns in;
-                // per MMA A advances 16 kept values = 32 B, B 32 channels = 64 B (descriptor units of 16 B)
-                const uint32_t a_kb = a_lo + 4u * a_sub;
-                const uint32_t meta_kb = meta_tmem + 2u * a_sub;
-                tc_mma_sparse_lo(d_tmem, a_kb, b_lo, meta_kb, idesc, accumulate);
-                if (!tail || mma_tail > 1) tc_mma_sparse_lo(d_tmem, a_kb + 2u, b_lo + 4u, meta_kb, idesc | 1u, 1u);
-              } else {
-                tc_mma_dense_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
-                if (!tail) {
-                  tc_mma_dense_lo(d_tmem, a_lo + 2u, b_lo + 2u, idesc, 1u);
-                  tc_mma_dense_lo(d_tmem, a_lo + 4u, b_lo + 4u, idesc, 1u);
-                  tc_mma_dense_lo(d_tmem, a_lo + 6u, b_lo + 6u, idesc, 1u);
-                } else {
-                  for (int kk = 1; kk < mma_tail; ++kk)
-                    tc_mma_dense_lo(d_tmem, a_lo + 2u * kk, b_lo + 2u * kk, idesc, 1u);
-                }
-              }
-              accumulate = 1;
-              if (++tap == p.taps) {
-                tap = 0;
-                ++cc;
-              }
+              const uint32_t a_kb = a_lo + 4u * a_sub;
+              const uint32_t meta_kb = meta_tmem + 2u * a_sub;
+              tc_mma_sparse_lo(d_tmem, a_kb, b_lo, meta_kb, idesc, accumulate);
+              if (n_mma > 1) tc_mma_sparse_lo(d_tmem, a_kb + 2u, b_lo + 4u, meta_kb, idesc | 1u, 1u);
+            } else {
+              a_lo = a_lo0 + s * kAEntryDesc;
+              tc_mma_dense_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
+              for (int kk = 1; kk < n_mma; ++kk) tc_mma_dense_lo(d_tmem, a_lo + 2u * kk, b_lo + 2u * kk, idesc, 1u);
             }
-            tc_commit_a(empty0 + 8u * s);
-            if (++s == (uint32_t)kNB) {
-              s = 0;
-              ph ^= 1u;
-            }
+            accumulate = 1;
+          }
+          tc_commit_a(empty0 + 8u * s);
+          if (++s == (uint32_t)kNB) {
+            s = 0;
+            ph ^= 1u;
           }
         }
         if (ok) tc_commit(&bar_acc_full[buf]);
