@@ -296,8 +296,11 @@ def main():
         return max_over_ranks(e0.elapsed_time(e1))
 
     # eager warm-up (also performs every one-time host set-up before any capture)
+    launches_per_step = 0
     for i in range(warmup):
+        c0 = api.ssconv_launch_count()
         step(i % n_sets, True)
+        launches_per_step = api.ssconv_launch_count() - c0
         step(i % n_sets, False)
     torch.cuda.synchronize()
 
@@ -404,7 +407,7 @@ def main():
             "per_layer": per_layer,
             "e2e": {"value": world * total_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-            "gpu_launches": steps * len(layers),
+            "gpu_launches": steps * launches_per_step,
             "clocks": clocks, "dev_status": dev_status,
         }
         if cpu is not None:

@@ -63,6 +63,12 @@ enum {
 /* Library version (major*10000 + minor*100 + patch). */
 int32_t ssconv_version(void);
 
+/* Number of GPU kernels this library has launched in this process so far (all devices and
+ * threads; memsets and copies are not counted).  A diagnostic with no counterpart in the paper:
+ * it lets a caller verify that a call ran on the GPU and how many kernels it took (a layer whose
+ * K range is split launches two, see ssconv_forward).  Host only, never fails. */
+uint64_t ssconv_launch_count(void);
+
 /* Static string for a status code. */
 const char* ssconv_status_string(int32_t status);
 

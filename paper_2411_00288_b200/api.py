@@ -21,7 +21,8 @@ OK = 0
 ERR_TIMEOUT = 8
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.so")
-EXPORTS = ("ssconv_version", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes", "ssconv_select_mask",
+EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes",
+           "ssconv_select_mask",
            "ssconv_compress", "ssconv_decompress", "ssconv_forward", "ssconv_forward_dense",
            "ssconv_forward_static_ws")
 
@@ -69,6 +70,8 @@ def lib():
         dp = ctypes.POINTER(Desc)
         L.ssconv_version.restype = i32
         L.ssconv_version.argtypes = []
+        L.ssconv_launch_count.restype = ctypes.c_uint64
+        L.ssconv_launch_count.argtypes = []
         L.ssconv_status_string.restype = ctypes.c_char_p
         L.ssconv_status_string.argtypes = [i32]
         L.ssconv_out_shape.restype = i32
@@ -117,6 +120,11 @@ def _need_cuda(*tensors):
 
 def ssconv_version() -> int:
     return int(lib().ssconv_version())
+
+
+def ssconv_launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return int(lib().ssconv_launch_count())
 
 
 def ssconv_out_shape(desc: Desc) -> Tuple[int, int]:

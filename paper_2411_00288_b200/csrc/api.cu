@@ -21,6 +21,12 @@ int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const vo
                                  const float* bias, void* y, int32_t* dev_status, cudaStream_t stream);
 }  // namespace ssconv
 
+#include <atomic>
+namespace ssconv {
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+}  // namespace ssconv
+
 namespace {
 
 using ssconv::Geometry;
@@ -63,6 +69,8 @@ int32_t check_desc(const ssconv_desc_t* d, bool need_tma_shape) {
 extern "C" {
 
 int32_t ssconv_version(void) { return 100; }
+
+uint64_t ssconv_launch_count(void) { return ssconv::g_launches.load(std::memory_order_relaxed); }
 
 const char* ssconv_status_string(int32_t status) {
   switch (status) {

@@ -849,6 +849,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE>, tm_a, tm_b, tm_y, p) != cudaSuccess) return SSCONV_ERR_CUDA;
+  count_launch();
   if (p.split) {
     FinishParams f;
     f.C_out = d.C_out;
@@ -865,6 +866,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     cfg.blockDim = dim3((unsigned)kFinishThreads);
     cfg.dynamicSmemBytes = 0;
     if (cudaLaunchKernelEx(&cfg, ssconv_split_finish_kernel, f) != cudaSuccess) return SSCONV_ERR_CUDA;
+    count_launch();
   }
   return SSCONV_OK;
 }

@@ -74,4 +74,7 @@ __host__ __device__ inline uint32_t code_pattern(uint32_t code) {
   }
 }
 
+// Kernels launched by this library in this process (all devices, all threads); see ssconv_launch_count.
+void count_launch();
+
 }  // namespace ssconv

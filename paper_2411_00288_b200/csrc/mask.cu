@@ -165,6 +165,7 @@ static inline unsigned blocks_for(int64_t n, int threads) { return (unsigned)((n
 cudaError_t launch_select(int mode, const void* scores, int64_t G, uint8_t* pattern, cudaStream_t st) {
   if (G == 0) return cudaSuccess;
   const int T = 256;
+  count_launch();
   if (mode == SSCONV_MASK_LOGITS_F32)
     select_logits_kernel<<<blocks_for(G, T), T, 0, st>>>((const float2*)scores, G, pattern);
   else
@@ -177,10 +178,12 @@ cudaError_t launch_compress(const ssconv_desc_t& d, const void* w, const uint8_t
   Geometry geo = make_geometry(d);
   const int T = 256;
   int64_t nv = (int64_t)geo.Mp * geo.kblocks_pad * 16;
+  count_launch();
   compress_values_kernel<<<blocks_for(nv, T), T, 0, st>>>(d, geo, (const uint2*)w, pattern, (uint32_t*)w_comp);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   int64_t nm = (int64_t)geo.m_tiles * geo.stages * 512;
+  count_launch();
   compress_meta_kernel<<<blocks_for(nm, T), T, 0, st>>>(d, geo, pattern, (uint32_t*)meta);
   return cudaGetLastError();
 }
@@ -190,6 +193,7 @@ cudaError_t launch_decompress(const ssconv_desc_t& d, const void* w_comp, const 
   Geometry geo = make_geometry(d);
   const int T = 256;
   int64_t G = (int64_t)d.C_out * geo.taps * (d.C_in / 4);
+  count_launch();
   decompress_kernel<<<blocks_for(G, T), T, 0, st>>>(d, geo, (const uint32_t*)w_comp, (const uint32_t*)meta,
                                                     (uint2*)w_out, pattern_out);
   return cudaGetLastError();

@@ -27,6 +27,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_version_and_status_strings(lib):
     assert api.ssconv_version() >= 100
+    assert api.ssconv_launch_count() >= 0  # host-only counter, callable without a GPU
     assert api.status_string(0) == "ok"
     assert "timed out" in api.status_string(api.ERR_TIMEOUT)
 
