@@ -4,9 +4,11 @@
 //   D[C_out x Q] = A[C_out x K] * B[K x Q],   Q = output positions, K = KH*KW*C_in
 //
 // A = weights (the only operand tcgen05.mma.sp accepts in 2:4 form), B = activations.  A CTA
-// owns a 128 (output channels) x 240 (positions) tile of D at a time and walks a static list of
-// tiles (persistent kernel).  240 is as wide as two fp32 accumulators plus the metadata columns
-// allow in the 512 TMEM columns: one thread issues every MMA, and wide MMAs amortise its cost.
+// owns a 128 (output channels) x BN (positions) tile of D at a time and walks a static list of
+// tiles (persistent kernel).  BN is chosen per layer by the host, a multiple of 16 up to 240: 240
+// is as wide as two fp32 accumulators plus the metadata columns allow in the 512 TMEM columns, and
+// wide MMAs amortise the cost of issuing them; narrower tiles are used when 240-wide ones would
+// leave most SMs without work.
 //
 // Positions are the output pixels (n, ho, wo) in row-major order.  Per k-block (64 input channels
 // at one filter tap) one im2col-mode TMA load brings the 240 pixels' channels at that tap,
@@ -14,8 +16,8 @@
 // all taps from it through row-shifted descriptors was built and measured: the MMA's operand
 // fetch, about 64 B/clk, bounds the main loop either way, so the simpler scheme stays.)
 //
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer (one thread; owns TMEM), warps 2-9 epilogue
-// in two groups of four warps that each own half of a tile's positions.  The accumulator has
+// Warp roles: warps 0, 10 and 11 TMA producers (one thread each: activations of even stages, of
+// odd stages, weights), warp 1 MMA issuer (one thread; owns TMEM), warps 2-9 epilogue in two groups of four warps that each own half of a tile's positions.  The accumulator has
 // channels on TMEM lanes and positions on columns, NHWC wants the transpose: the epilogue reads
 // TMEM in the MMA-fragment layout (tcgen05.ld 16x256b), adds the bias, converts pairs to bf16
 // (with ReLU in the conversion), and stmatrix.trans writes 8x8 blocks transposed into a 128-byte
@@ -42,11 +44,12 @@
 
 namespace ssconv {
 
-constexpr int kBN = 240;                 // positions per tile (N of the MMA)
-constexpr int kGroups = 2;               // epilogue warp groups, each owning kBN / kGroups positions
+constexpr int kBN = 240;                 // most positions per tile (N of the MMA); a layer's tile may be narrower
+constexpr int kGroups = 2;               // epilogue warp groups, each owning half of a tile's positions
 constexpr int kGroupCols = kBN / kGroups;
 constexpr int kPiece = 40;               // positions per epilogue piece (one staging buffer)
-constexpr int kThreads = 64 + 128 * kGroups;
+constexpr int kFirstExtraProducerWarp = 2 + 4 * kGroups;  // warps 10 and 11: two more TMA producers
+constexpr int kThreads = 64 + 128 * kGroups + 64;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kAccCol1 = 256;       // second accumulator; the first starts at column 0
 constexpr uint32_t kMetaCol = kBN;       // metadata: 2 slots x 4 columns in [240, 248)
@@ -74,6 +77,9 @@ struct FwdParams {
   int C_in, C_out;
   int Ho, Wo;               // output extent
   int Q;                    // positions = N * Ho * Wo
+  int BN;                   // positions per tile, a multiple of 16, at most kBN
+  int pieces;               // epilogue pieces per group: ceil(BN / 2 / kPiece)
+  int tail_cols;            // positions in a group's last piece (a multiple of 8, at most kPiece)
   int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
   int taps, cblocks, kblocks;
   int m_tiles, num_tiles;
@@ -196,10 +202,109 @@ __device__ __forceinline__ Pos decode_pos(int q, int Wq, int Hq) {
   return s;
 }
 
+// One of the three TMA producer threads.  All of them walk the same sequence of stages; role 0
+// loads the activation tiles of the even stages, role 1 those of the odd stages, role 2 the
+// weight tiles (with their metadata).  A TMA instruction occupies its issuing thread for a few
+// hundred cycles, so one thread issuing everything (three to four loads per pair of k-blocks, plus
+// the waits) cannot keep up with the tensor pipe; three can.
+constexpr int kRoleActEven = 0, kRoleActOdd = 1, kRoleWeights = 2;
+template <bool SPARSE, int ROLE>
+__device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUtensorMap* tm_b, const FwdParams& p,
+                                              uint32_t full0, uint32_t empty0, uint32_t a_smem0, uint32_t b_smem0,
+                                              volatile int* abort_flag) {
+  using C = Cfg<SPARSE>;
+  constexpr int APER = C::kBlocksPerA;
+  constexpr int kNB = C::kNB;
+  const uint32_t b_bytes = (uint32_t)p.BN * 128u;  // one activation tile: BN positions x 64 channels
+  uint32_t s = 0, ph = 0;  // stage and its phase parity
+  bool ok = true;
+  bool first_segment = true;
+  WorkIter work(p);
+  Segment seg;
+  while (ok && work.next(seg)) {
+    const int pt = seg.tile / p.m_tiles;
+    const int m = seg.tile - pt * p.m_tiles;
+    const Pos q0 = decode_pos(pt * p.BN, p.Wo, p.Ho);
+    const int base_w = q0.c * p.stride_w - p.pad_w;
+    const int base_h = q0.r * p.stride_h - p.pad_h;
+    const uint8_t* meta_src = p.meta + ((size_t)m * p.a_tiles + seg.a0) * kMetaImageBytes;
+    const int kb0 = seg.a0 * APER;
+    const int kb1 = (seg.a1 * APER < p.kblocks) ? seg.a1 * APER : p.kblocks;
+    int cc = kb0 / p.taps;  // channel chunk
+    int tap = kb0 - cc * p.taps;
+    int a_idx = seg.a0;
+    const int kh0 = tap / p.KW;
+    int kw = tap - kh0 * p.KW;
+    int off_w = kw * p.dil_w, off_h = kh0 * p.dil_h;
+    if (first_segment) {
+      // everything above ran concurrently with the tail of the previous grid in the stream; its
+      // results (our inputs) are complete from here on
+      grid_dependency_wait();
+      first_segment = false;
+    }
+    // whole weight tiles: a tile whose second k-block does not exist still takes two stages
+    for (int left = (seg.a1 - seg.a0) * APER, kb = kb0; left > 0; --left, ++kb) {
+      const uint32_t full = full0 + 8u * s;
+      if (ROLE == kRoleWeights) {
+        if (APER == 1 || (s & 1u) == 0u) {
+          // the weight slot is shared by the APER stages that follow: all of them must be free
+          if (!mbar_wait_a(empty0 + 8u * s, ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+          if (APER == 2 && !mbar_wait_a(empty0 + 8u * (s + 1u), ph ^ 1u, abort_flag, kWaitLimitCycles)) {
+            ok = false;
+            break;
+          }
+          if (kb < kb1) {
+            const uint32_t a_dst = a_smem0 + (s / APER) * C::kAEntryBytes;
+            mbar_expect_tx_a(full, C::kAEntryBytes);
+            if (SPARSE) {
+              tma_load_2d_a(a_dst, tm_a, full, a_idx * 64, m * kTileM);
+              bulk_load_a(a_dst + kATileBytes, meta_src, kMetaImageBytes, full);
+              meta_src += kMetaImageBytes;
+            } else {
+              tma_load_3d_a(a_dst, tm_a, full, cc * kBlockK, tap, m * kTileM);
+            }
+            ++a_idx;
+          } else {
+            mbar_arrive_a(full);  // stage without a k-block: keeps the ring's phases in step
+          }
+        }
+      } else if ((s & 1u) == (uint32_t)ROLE) {
+        if (!mbar_wait_a(empty0 + 8u * s, ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+        if (kb < kb1) {
+          mbar_expect_tx_a(full, b_bytes);
+          tma_load_im2col_4d_a(b_smem0 + s * kBTileBytes, tm_b, full, cc * kBlockK, base_w, base_h, q0.n,
+                               (uint16_t)off_w, (uint16_t)off_h);
+        } else {
+          mbar_arrive_a(full);
+        }
+      }
+      if (kb < kb1) {
+        ++tap;
+        off_w += p.dil_w;
+        if (++kw == p.KW) {
+          kw = 0;
+          off_w = 0;
+          off_h += p.dil_h;
+          if (tap == p.taps) {  // next channel chunk
+            tap = 0;
+            off_h = 0;
+            ++cc;
+          }
+        }
+      }
+      if (++s == (uint32_t)kNB) {
+        s = 0;
+        ph ^= 1u;
+      }
+    }
+  }
+}
+
 template <bool SPARSE>
 __global__ void __launch_bounds__(kThreads, 1)
 ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                  const __grid_constant__ CUtensorMap tm_y, const FwdParams p) {
+                  const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_y_tail,
+                  const FwdParams p) {
   using C = Cfg<SPARSE>;
   constexpr int APER = C::kBlocksPerA;
   constexpr int kNA = C::kNA;
@@ -231,7 +336,9 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       prefetch_tensormap(&tm_a);
       prefetch_tensormap(&tm_b);
       for (int s = 0; s < kNB; ++s) {
-        mbar_init(&bar_full[s], 1);
+        // a stage is full once its activation producer and, where the stage starts a weight tile,
+        // the weight producer have both arrived and their bytes have landed
+        mbar_init(&bar_full[s], (APER == 1 || (s & 1) == 0) ? 2 : 1);
         mbar_init(&bar_empty[s], 1);
       }
       for (int b = 0; b < 2; ++b) {
@@ -249,103 +356,32 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       tmem_alloc(tmem_slot, kTmemCols);
       tmem_relinquish();
     }
-    if (warp == 2 && lane == 0) prefetch_tensormap(&tm_y);
+    if (warp == 2 && lane == 0) {
+      prefetch_tensormap(&tm_y);
+      prefetch_tensormap(&tm_y_tail);
+    }
     tc_fence_before();
     setup_bar_sync();
     tc_fence_after();
   }
   const uint32_t tmem_base = (warp == 0) ? 0u : *tmem_slot;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+  if (warp == 0 || warp >= kFirstExtraProducerWarp) {
+    // ------------------------------------------------------------------ TMA producers
     if (lane == 0) {
-      // Index arithmetic in the k loop is incremental and 32-bit: this single thread's instruction
-      // stream is on the critical path of every stage.
       const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty);
       const uint32_t a_smem0 = smem_u32(a_ring), b_smem0 = smem_u32(b_ring);
-      uint32_t s = 0, ph = 0;  // stage and its phase parity
-      bool ok = true;
-      bool first_segment = true;
-      WorkIter work(p);
-      Segment seg;
-      while (ok && work.next(seg)) {
-        const int pt = seg.tile / p.m_tiles;
-        const int m = seg.tile - pt * p.m_tiles;
-        const Pos q0 = decode_pos(pt * kBN, p.Wo, p.Ho);
-        const int base_w = q0.c * p.stride_w - p.pad_w;
-        const int base_h = q0.r * p.stride_h - p.pad_h;
-        const uint8_t* meta_src = p.meta + ((size_t)m * p.a_tiles + seg.a0) * kMetaImageBytes;
-        const int kb0 = seg.a0 * APER;
-        const int kb1 = (seg.a1 * APER < p.kblocks) ? seg.a1 * APER : p.kblocks;
-        int cc = kb0 / p.taps;          // channel chunk
-        int tap = kb0 - cc * p.taps;
-        int a_idx = seg.a0;
-        if (first_segment) {
-          // everything above ran concurrently with the tail of the previous grid in the stream;
-          // its results (our inputs) are complete from here on
-          grid_dependency_wait();
-          first_segment = false;
-        }
-        {
-          const int kh0 = tap / p.KW;
-          int kw = tap - kh0 * p.KW;
-          int off_w = kw * p.dil_w, off_h = kh0 * p.dil_h;
-          // whole weight tiles: a tile whose second k-block does not exist still takes two stages
-          for (int left = (seg.a1 - seg.a0) * APER, kb = kb0; left > 0; --left, ++kb) {
-            const bool first_of_tile = (APER == 1) || ((s & 1u) == 0u);
-            if (first_of_tile) {
-              // the weight slot is shared by the APER stages that follow: all of them must be free
-              if (!mbar_wait_a(empty0 + 8u * s, ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-              if (APER == 2 && !mbar_wait_a(empty0 + 8u * (s + 1u), ph ^ 1u, abort_flag, kWaitLimitCycles)) {
-                ok = false;
-                break;
-              }
-            }
-            const uint32_t full = full0 + 8u * s;
-            if (kb < kb1) {
-              if (first_of_tile) {
-                const uint32_t a_dst = a_smem0 + (s / APER) * C::kAEntryBytes;
-                mbar_expect_tx_a(full, C::kAEntryBytes + kBTileBytes);
-                if (SPARSE) {
-                  tma_load_2d_a(a_dst, &tm_a, full, a_idx * 64, m * kTileM);
-                  bulk_load_a(a_dst + kATileBytes, meta_src, kMetaImageBytes, full);
-                  meta_src += kMetaImageBytes;
-                } else {
-                  tma_load_3d_a(a_dst, &tm_a, full, cc * kBlockK, tap, m * kTileM);
-                }
-                ++a_idx;
-              } else {
-                mbar_expect_tx_a(full, kBTileBytes);
-              }
-              tma_load_im2col_4d_a(b_smem0 + s * kBTileBytes, &tm_b, full, cc * kBlockK, base_w, base_h, q0.n,
-                                   (uint16_t)off_w, (uint16_t)off_h);
-              ++tap;
-              off_w += p.dil_w;
-              if (++kw == p.KW) {
-                kw = 0;
-                off_w = 0;
-                off_h += p.dil_h;
-                if (tap == p.taps) {  // next channel chunk
-                  tap = 0;
-                  off_h = 0;
-                  ++cc;
-                }
-              }
-            } else {
-              mbar_arrive_a(full);  // stage without a k-block: keeps the ring's phases in step
-            }
-            if (++s == (uint32_t)kNB) {
-              s = 0;
-              ph ^= 1u;
-            }
-          }
-        }
-      }
+      if (warp == 0)
+        producer_role<SPARSE, kRoleActEven>(&tm_a, &tm_b, p, full0, empty0, a_smem0, b_smem0, abort_flag);
+      else if (warp == kFirstExtraProducerWarp)
+        producer_role<SPARSE, kRoleActOdd>(&tm_a, &tm_b, p, full0, empty0, a_smem0, b_smem0, abort_flag);
+      else
+        producer_role<SPARSE, kRoleWeights>(&tm_a, &tm_b, p, full0, empty0, a_smem0, b_smem0, abort_flag);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(kTileM, kBN, SPARSE);
+      const uint32_t idesc = make_idesc_bf16(kTileM, (uint32_t)p.BN, SPARSE);
       constexpr uint32_t kAEntryDesc = C::kAEntryBytes >> 4;  // descriptor address units are 16 B
       constexpr uint32_t kBTileDesc = kBTileBytes >> 4;
       const uint32_t a_lo0 = desc_lo(smem_u32(a_ring));
@@ -447,16 +483,17 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         if (ok) tc_commit(&bar_acc_full[buf]);
       }
     }
-  } else {
+  } else if (warp < kFirstExtraProducerWarp) {
     // ------------------------------------------------------------------ epilogue
-    // Two independent groups of four warps; group g owns positions [120 g, 120 g + 120) of every
-    // tile, with its own staging buffers and named barrier, and handles them 40 at a time.
+    // Two independent groups of four warps; group g owns positions [g BN/2, (g + 1) BN/2) of every
+    // tile, with its own staging buffers and named barrier, and handles them 40 at a time (the last
+    // piece of a group may hold fewer).
     const int grp = (warp - 2) >> 2;
     const int q = warp & 3;  // TMEM lane quadrant this warp may read: channels [32 q, 32 q + 32) of the tile
     const int gtid = q * 32 + lane;
     const bool leader = (q == 2 && lane == 0);  // first warp of each group
     const bool relu = (p.flags & SSCONV_FLAG_RELU) != 0;
-    const int col_base = grp * kGroupCols;
+    const int col_base = grp * (p.BN >> 1);
     uint8_t* my_stage = out_stage + grp * 2 * kPieceBytes;
     volatile int* my_go = epi_go + 2 * grp;
     // stmatrix duty of this thread: 16 bytes = 8 channels of block (lane / 8) of the warp's four, at
@@ -512,12 +549,13 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         bias_v[i] = ((p.flags & SSCONV_FLAG_BIAS) && co < p.C_out) ? p.bias[co] : 0.0f;
       }
 #pragma unroll 1
-      for (int piece = 0; piece < kPiecesPerGroup; ++piece, ++piece_count) {
+      for (int piece = 0; piece < p.pieces; ++piece, ++piece_count) {
         uint8_t* stage = my_stage + (piece_count & 1u) * kPieceBytes;
         uint32_t r[kPiece];
+        // (a short last piece still reads and stages 40 columns; the surplus is never stored)
         tc_ld_piece(t_row + piece * kPiece, r);
         tc_wait_ld();
-        if (piece == kPiecesPerGroup - 1) {
+        if (piece == p.pieces - 1) {
           // this warp's part of the accumulator is read: hand it back to the MMA thread
           tc_fence_before();
           __syncwarp();
@@ -534,11 +572,13 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         if (leader) bulk_wait_group_read0();  // the previous piece's store no longer reads its buffer
         epilogue_bar_sync(grp);
         if (leader) {
-          const int q_piece = pt * kBN + col_base + piece * kPiece;
+          const int q_piece = pt * p.BN + col_base + piece * kPiece;
           if (q_piece < p.Q) {
-            // positions beyond Q and channels beyond C_out fall outside the tensor map and are dropped
-            tma_store_2d(&tm_y, stage, m * kTileM, q_piece);
-            if (m * kTileM + 64 < p.C_out) tma_store_2d(&tm_y, stage + kHalfPieceBytes, m * kTileM + 64, q_piece);
+            // positions beyond Q and channels beyond C_out fall outside the tensor map and are dropped;
+            // a short last piece goes through the map whose box holds just its positions
+            const CUtensorMap* map = (piece == p.pieces - 1 && p.tail_cols != kPiece) ? &tm_y_tail : &tm_y;
+            tma_store_2d(map, stage, m * kTileM, q_piece);
+            if (m * kTileM + 64 < p.C_out) tma_store_2d(map, stage + kHalfPieceBytes, m * kTileM + 64, q_piece);
           }
           bulk_commit_group();
         }
@@ -697,15 +737,62 @@ static int out_extent(int in, int k, int stride, int pad, int dil) {
 // Scratch for partly computed tiles: two fp32 regions (128 x 240) per CTA.
 constexpr int kMaxWorkers = 148;
 constexpr size_t kRegionBytes = (size_t)kTileM * kBN * sizeof(float);
-// Cost model of the choice between whole tiles and an even split of K (cycles, measured on B200):
-// a k-block of 64 dense columns takes about 600 cycles sparse and 720 dense; an epilogue that
-// nothing overlaps about 3500; and every parked partial tile costs the chip about 90 cycles of
-// L2 traffic (123 KB written by the main kernel and read again by the finishing kernel).
-constexpr double kCyclesPerKBlockSparse = 600.0;
-constexpr double kCyclesPerKBlockDense = 720.0;
-constexpr double kEpilogueCycles = 3500.0;
+// Cost model behind the choice of tile width and of splitting K (cycles, measured on B200).
+// A k-block of 64 dense columns takes the longer of two things.  The issuing thread: a fixed
+// cost per k-block (wait, commit, metadata copy) plus MMAs whose time grows with the tile width
+// BN.  The fill of shared memory from L2, about 68 bytes per cycle and SM: the weight tile's share
+// plus 128 BN bytes of activations.  For BN = 240 that is about 590 cycles sparse, 690 dense.  An
+// epilogue that nothing overlaps takes about 1200 cycles per 40 positions of the widest group, and
+// every parked partial tile costs the chip about 90 cycles of L2 traffic (123 KB written by the
+// main kernel and read again by the finishing kernel).
+constexpr double kFillBytesPerCycle = 68.0;
+constexpr double kIssueFixedSparse = 242.0, kIssuePerColSparse = 1.0;   // 2 MMAs of about 35 + 0.5 BN, + 172
+constexpr double kIssueFixedDense = 170.0, kIssuePerColDense = 1.96;    // 4 MMAs of about 5 + 0.49 BN, + 150
+constexpr double kEpiloguePieceCycles = 1200.0;
 constexpr double kCyclesPerParkedTile = 90.0;
 constexpr double kSplitAdvantage = 1.1;  // split only if the model predicts at least this gain
+
+template <bool SPARSE>
+static double kblock_cycles(int BN) {
+  const double a_bytes = SPARSE ? (kATileBytes + kMetaImageBytes) / 2.0 : (double)kATileBytes;
+  const double fill = (a_bytes + 128.0 * BN) / kFillBytesPerCycle;
+  const double issue = SPARSE ? kIssueFixedSparse + kIssuePerColSparse * BN : kIssueFixedDense + kIssuePerColDense * BN;
+  return fill > issue ? fill : issue;
+}
+
+// Tile width and partition of a layer.
+struct Plan {
+  int BN;
+  bool split;
+};
+template <bool SPARSE>
+static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force_split) {
+  Plan best{kBN, false};
+  if (force_split) return Plan{kBN, true};
+  double best_cost = 0.0;
+  for (int BN = kBN; BN >= 48; BN -= 16) {
+    const long long tiles = ((Q + BN - 1) / BN) * geo.m_tiles;
+    const long long per_cta = (tiles + workers - 1) / workers;
+    const int pieces = (BN / 2 + kPiece - 1) / kPiece;
+    const double cost = (double)per_cta * geo.kblocks * kblock_cycles<SPARSE>(BN) + pieces * kEpiloguePieceCycles;
+    if (BN == kBN || cost < 0.97 * best_cost) {  // a narrower tile has to earn its extra weight traffic
+      best_cost = cost;
+      best.BN = BN;
+    }
+  }
+  // Even split of K at full width, when many SMs would still idle and K is deep.
+  const int a_tiles = SPARSE ? geo.stages : geo.kblocks;
+  if (a_tiles > 1) {
+    const long long tiles = ((Q + kBN - 1) / kBN) * geo.m_tiles;
+    const double units = (double)tiles * a_tiles;
+    const double ctas = units < workers ? units : (double)workers;
+    const double per_a_tile = kblock_cycles<SPARSE>(kBN) * (SPARSE ? 2.0 : 1.0);
+    const double split_cost = units / ctas * per_a_tile + (ctas + tiles) * kCyclesPerParkedTile;
+    if (best_cost > kSplitAdvantage * split_cost) return Plan{kBN, true};
+  }
+  return best;
+}
+
 constexpr size_t scratch_bytes(int workers) {
   return 2 * (size_t)workers * kRegionBytes;
 }
@@ -741,8 +828,13 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   const int Wo = out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
   const long long Q = (long long)d.N * Ho * Wo;  // positions
   if (Q > 0x7FFFFF00LL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  const int workers = g_sm_count[dev] < worker_cap ? g_sm_count[dev] : worker_cap;
+  const Plan plan = plan_layer<SPARSE>(Q, geo, workers, force_split);
+  const int BN = plan.BN;
+  const int pieces = (BN / 2 + kPiece - 1) / kPiece;
+  const int tail_cols = BN / 2 - (pieces - 1) * kPiece;
 
-  CUtensorMap tm_a, tm_b, tm_y;
+  CUtensorMap tm_a, tm_b, tm_y, tm_y_tail;
   // activations: NHWC seen as (c, w, h, n), im2col mode; elements outside the image read as zero
   // (= the zero padding of Eq. 4); base pixels are the filter placements, each load adds a tap offset
   {
@@ -753,7 +845,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     int upper[2] = {d.pad_w - (d.KW - 1) * d.dil_w, d.pad_h - (d.KH - 1) * d.dil_h};
     cuuint32_t estr[4] = {1, (cuuint32_t)d.stride_w, (cuuint32_t)d.stride_h, 1};
     CUresult r = g_encode_im2col(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), dims, strides,
-                                 lower, upper, (cuuint32_t)kBlockK, (cuuint32_t)kBN, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 lower, upper, (cuuint32_t)kBlockK, (cuuint32_t)BN, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
@@ -787,6 +879,12 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
+    // the last piece of a group may hold fewer positions: same view, shorter box
+    box[1] = (cuuint32_t)tail_cols;
+    r = g_encode_tiled(&tm_y_tail, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
   }
 
   FwdParams p;
@@ -795,6 +893,9 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.Ho = Ho;
   p.Wo = Wo;
   p.Q = (int)Q;
+  p.BN = BN;
+  p.pieces = pieces;
+  p.tail_cols = tail_cols;
   p.stride_h = d.stride_h;
   p.stride_w = d.stride_w;
   p.pad_h = d.pad_h;
@@ -806,7 +907,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.cblocks = geo.cblocks;
   p.kblocks = geo.kblocks;
   p.m_tiles = geo.m_tiles;
-  const long long q_tiles = (Q + kBN - 1) / kBN;
+  const long long q_tiles = (Q + BN - 1) / BN;
   p.num_tiles = (int)(q_tiles * geo.m_tiles);
   p.a_tiles = SPARSE ? geo.stages : geo.kblocks;
   p.flags = d.flags;
@@ -816,15 +917,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.dev_status = dev_status;
 
   p.units = (long long)p.num_tiles * p.a_tiles;
-  int workers = g_sm_count[dev] < worker_cap ? g_sm_count[dev] : worker_cap;
-  // Whole tiles per CTA, unless dealing the K range out evenly is clearly faster by the cost model.
-  const double a_tile_cycles = SPARSE ? 2.0 * kCyclesPerKBlockSparse : kCyclesPerKBlockDense;
-  const int waves = (p.num_tiles + workers - 1) / workers;
-  const double whole_cost = (double)waves * p.a_tiles * a_tile_cycles + kEpilogueCycles;
-  const double split_ctas = p.units < workers ? (double)p.units : (double)workers;
-  const double split_cost =
-      (double)p.units / split_ctas * a_tile_cycles + (split_ctas + p.num_tiles) * kCyclesPerParkedTile;
-  p.split = (p.a_tiles > 1 && (force_split || whole_cost > kSplitAdvantage * split_cost)) ? 1 : 0;
+  p.split = (plan.split && p.a_tiles > 1) ? 1 : 0;
   int grid;
   if (p.split) {
     grid = p.units < workers ? (int)p.units : workers;
@@ -848,7 +941,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE>, tm_a, tm_b, tm_y, p) != cudaSuccess) return SSCONV_ERR_CUDA;
+  if (cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE>, tm_a, tm_b, tm_y, tm_y_tail, p) != cudaSuccess) return SSCONV_ERR_CUDA;
   count_launch();
   if (p.split) {
     FinishParams f;
