@@ -55,23 +55,25 @@ constexpr uint32_t kAccCol1 = 256;       // second accumulator; the first starts
 constexpr uint32_t kMetaCol = kBN;       // metadata: 2 slots x 4 columns in [240, 248)
 constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 1.9 GHz
 constexpr uint32_t kATileBytes = 128 * 128;          // 128 rows x 128 B
-constexpr uint32_t kBTileBytes = kBN * 128;          // 240 positions x 64 channels bf16
 constexpr uint32_t kHalfPieceBytes = kPiece * 128;    // 40 positions x 64 channels bf16, 128-byte swizzled
 constexpr uint32_t kPieceBytes = 2 * kHalfPieceBytes; // channels [0,64) then [64,128) of the tile
 constexpr uint32_t kStagingBytes = 2 * kGroups * kPieceBytes;  // two buffers per group
 constexpr uint32_t kBarrierBytes = 256;
 
+// The ring's unit is a group: the operands of one pair of k-blocks (128 dense columns of K).
+// Layout of a group in shared memory: weights (sparse: one 128 x 128 B tile of kept values, which
+// spans both k-blocks, + its metadata image; dense: two tiles), then the two activation tiles of
+// BN x 128 B.  One full and one empty barrier per group: the issuing thread pays about 200 cycles
+// per wait and 80 per tcgen05 instruction, so the handshake is per pair of k-blocks, not per k-block.
 template <bool SPARSE>
 struct Cfg {
-  static constexpr int kBlocksPerA = SPARSE ? 2 : 1;  // k-blocks of 64 dense columns per weight tile
-  static constexpr uint32_t kMetaBytes = SPARSE ? (uint32_t)kMetaImageBytes : 0u;
-  static constexpr uint32_t kAEntryBytes = kATileBytes + kMetaBytes;
-  static constexpr int kNB = 4;                       // stages in the ring
-  static constexpr int kNA = kNB / kBlocksPerA;       // weight slots, one per group of stages sharing a tile
-  static constexpr uint32_t kSmemBytes =
-      kNA * kAEntryBytes + kNB * kBTileBytes + kStagingBytes + kBarrierBytes + 1024;
-  static_assert(kSmemBytes <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+  static constexpr uint32_t kAGroupBytes = SPARSE ? kATileBytes + (uint32_t)kMetaImageBytes : 2 * kATileBytes;
 };
+constexpr int kMaxGroups = 4;                  // groups in the ring: as many as fit, 2 to 4
+constexpr uint32_t kMaxSmemBytes = 232448;     // 227 KB per CTA
+__host__ __device__ constexpr uint32_t group_bytes(uint32_t a_group_bytes, int BN) {
+  return a_group_bytes + 2u * (uint32_t)BN * 128u;
+}
 
 struct FwdParams {
   int C_in, C_out;
@@ -80,10 +82,11 @@ struct FwdParams {
   int BN;                   // positions per tile, a multiple of 16, at most kBN
   int pieces;               // epilogue pieces per group: ceil(BN / 2 / kPiece)
   int tail_cols;            // positions in a group's last piece (a multiple of 8, at most kPiece)
+  int ring_groups;          // groups in the shared-memory ring
   int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
   int taps, cblocks, kblocks;
   int m_tiles, num_tiles;
-  int a_tiles;              // weight tiles per output tile
+  int a_tiles;              // pairs of k-blocks (groups) per output tile
   int split;                // 1: units dealt out evenly across CTAs (stream-K); 0: whole tiles per CTA
   long long units;          // num_tiles * a_tiles
   float4* ws_regions;       // [2 * gridDim.x] regions of 128 x 240 fp32: a CTA's partial tiles
@@ -202,21 +205,46 @@ __device__ __forceinline__ Pos decode_pos(int q, int Wq, int Hq) {
   return s;
 }
 
-// One of the three TMA producer threads.  All of them walk the same sequence of stages; role 0
-// loads the activation tiles of the even stages, role 1 those of the odd stages, role 2 the
-// weight tiles (with their metadata).  A TMA instruction occupies its issuing thread for a few
-// hundred cycles, so one thread issuing everything (three to four loads per pair of k-blocks, plus
-// the waits) cannot keep up with the tensor pipe; three can.
-constexpr int kRoleActEven = 0, kRoleActOdd = 1, kRoleWeights = 2;
+// Filter tap and channel chunk of a k-block (numbered chunk * taps + tap), advanced incrementally.
+struct TapIter {
+  int cc, tap, kw, off_w, off_h;
+  __device__ void init(int kb, const FwdParams& p) {
+    cc = kb / p.taps;
+    tap = kb - cc * p.taps;
+    const int kh = tap / p.KW;
+    kw = tap - kh * p.KW;
+    off_w = kw * p.dil_w;
+    off_h = kh * p.dil_h;
+  }
+  __device__ void advance(const FwdParams& p) {
+    ++tap;
+    off_w += p.dil_w;
+    if (++kw == p.KW) {
+      kw = 0;
+      off_w = 0;
+      off_h += p.dil_h;
+      if (tap == p.taps) {  // next channel chunk
+        tap = 0;
+        off_h = 0;
+        ++cc;
+      }
+    }
+  }
+};
+
+// One of the three TMA producer threads.  All of them walk the same sequence of groups; role 0
+// loads the activation tile of each group's first k-block, role 1 that of the second, role 2 the
+// weights (with their metadata).  A TMA instruction occupies its issuing thread for a few hundred
+// cycles, so one thread issuing everything cannot keep up with the tensor pipe; three can.
+constexpr int kRoleActFirst = 0, kRoleActSecond = 1, kRoleWeights = 2;
 template <bool SPARSE, int ROLE>
 __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUtensorMap* tm_b, const FwdParams& p,
-                                              uint32_t full0, uint32_t empty0, uint32_t a_smem0, uint32_t b_smem0,
+                                              uint32_t full0, uint32_t empty0, uint32_t ring0,
                                               volatile int* abort_flag) {
   using C = Cfg<SPARSE>;
-  constexpr int APER = C::kBlocksPerA;
-  constexpr int kNB = C::kNB;
   const uint32_t b_bytes = (uint32_t)p.BN * 128u;  // one activation tile: BN positions x 64 channels
-  uint32_t s = 0, ph = 0;  // stage and its phase parity
+  const uint32_t grp_bytes = group_bytes(C::kAGroupBytes, p.BN);
+  uint32_t g = 0, ph = 0;  // group slot and its phase parity
   bool ok = true;
   bool first_segment = true;
   WorkIter work(p);
@@ -228,72 +256,43 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
     const int base_w = q0.c * p.stride_w - p.pad_w;
     const int base_h = q0.r * p.stride_h - p.pad_h;
     const uint8_t* meta_src = p.meta + ((size_t)m * p.a_tiles + seg.a0) * kMetaImageBytes;
-    const int kb0 = seg.a0 * APER;
-    const int kb1 = (seg.a1 * APER < p.kblocks) ? seg.a1 * APER : p.kblocks;
-    int cc = kb0 / p.taps;  // channel chunk
-    int tap = kb0 - cc * p.taps;
-    int a_idx = seg.a0;
-    const int kh0 = tap / p.KW;
-    int kw = tap - kh0 * p.KW;
-    int off_w = kw * p.dil_w, off_h = kh0 * p.dil_h;
+    TapIter it;
+    it.init(2 * seg.a0 + (ROLE == kRoleActSecond ? 1 : 0), p);
     if (first_segment) {
       // everything above ran concurrently with the tail of the previous grid in the stream; its
       // results (our inputs) are complete from here on
       grid_dependency_wait();
       first_segment = false;
     }
-    // whole weight tiles: a tile whose second k-block does not exist still takes two stages
-    for (int left = (seg.a1 - seg.a0) * APER, kb = kb0; left > 0; --left, ++kb) {
-      const uint32_t full = full0 + 8u * s;
+    for (int a = seg.a0; a < seg.a1; ++a) {
+      if (!mbar_wait_a(empty0 + 8u * g, ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+      const uint32_t full = full0 + 8u * g;
+      const uint32_t dst = ring0 + g * grp_bytes;
+      const bool has_second = 2 * a + 1 < p.kblocks;
       if (ROLE == kRoleWeights) {
-        if (APER == 1 || (s & 1u) == 0u) {
-          // the weight slot is shared by the APER stages that follow: all of them must be free
-          if (!mbar_wait_a(empty0 + 8u * s, ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-          if (APER == 2 && !mbar_wait_a(empty0 + 8u * (s + 1u), ph ^ 1u, abort_flag, kWaitLimitCycles)) {
-            ok = false;
-            break;
-          }
-          if (kb < kb1) {
-            const uint32_t a_dst = a_smem0 + (s / APER) * C::kAEntryBytes;
-            mbar_expect_tx_a(full, C::kAEntryBytes);
-            if (SPARSE) {
-              tma_load_2d_a(a_dst, tm_a, full, a_idx * 64, m * kTileM);
-              bulk_load_a(a_dst + kATileBytes, meta_src, kMetaImageBytes, full);
-              meta_src += kMetaImageBytes;
-            } else {
-              tma_load_3d_a(a_dst, tm_a, full, cc * kBlockK, tap, m * kTileM);
-            }
-            ++a_idx;
-          } else {
-            mbar_arrive_a(full);  // stage without a k-block: keeps the ring's phases in step
-          }
-        }
-      } else if ((s & 1u) == (uint32_t)ROLE) {
-        if (!mbar_wait_a(empty0 + 8u * s, ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-        if (kb < kb1) {
-          mbar_expect_tx_a(full, b_bytes);
-          tma_load_im2col_4d_a(b_smem0 + s * kBTileBytes, tm_b, full, cc * kBlockK, base_w, base_h, q0.n,
-                               (uint16_t)off_w, (uint16_t)off_h);
+        if (SPARSE) {
+          mbar_expect_tx_a(full, C::kAGroupBytes);
+          tma_load_2d_a(dst, tm_a, full, a * 64, m * kTileM);
+          bulk_load_a(dst + kATileBytes, meta_src, kMetaImageBytes, full);
+          meta_src += kMetaImageBytes;
         } else {
-          mbar_arrive_a(full);
+          mbar_expect_tx_a(full, has_second ? 2 * kATileBytes : kATileBytes);
+          tma_load_3d_a(dst, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+          it.advance(p);
+          if (has_second) tma_load_3d_a(dst + kATileBytes, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+          it.advance(p);
         }
+      } else if (ROLE == kRoleActFirst || has_second) {
+        mbar_expect_tx_a(full, b_bytes);
+        tma_load_im2col_4d_a(dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? b_bytes : 0u), tm_b, full,
+                             it.cc * kBlockK, base_w, base_h, q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
+        it.advance(p);
+        it.advance(p);
+      } else {
+        mbar_arrive_a(full);  // the group has no second k-block: only keep the barrier's count
       }
-      if (kb < kb1) {
-        ++tap;
-        off_w += p.dil_w;
-        if (++kw == p.KW) {
-          kw = 0;
-          off_w = 0;
-          off_h += p.dil_h;
-          if (tap == p.taps) {  // next channel chunk
-            tap = 0;
-            off_h = 0;
-            ++cc;
-          }
-        }
-      }
-      if (++s == (uint32_t)kNB) {
-        s = 0;
+      if (++g == (uint32_t)p.ring_groups) {
+        g = 0;
         ph ^= 1u;
       }
     }
@@ -306,22 +305,18 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                   const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_y_tail,
                   const FwdParams p) {
   using C = Cfg<SPARSE>;
-  constexpr int APER = C::kBlocksPerA;
-  constexpr int kNA = C::kNA;
-  constexpr int kNB = C::kNB;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* a_ring = smem;                                        // kNA weight tiles (+ metadata)
-  uint8_t* b_ring = a_ring + kNA * C::kAEntryBytes;              // kNB activation tiles
-  // barrier slots: [0,8) stage full, [8,16) stage empty, [16,18) accumulator full, [18,20) accumulator empty
-  uint8_t* out_stage = b_ring + kNB * kBTileBytes;               // per group two staging buffers
+  uint8_t* ring = smem;                                                    // ring_groups groups
+  uint8_t* out_stage = ring + p.ring_groups * group_bytes(C::kAGroupBytes, p.BN);  // per epilogue group two buffers
+  // barrier slots: [0,4) group full, [4,8) group empty, [8,10) accumulator full, [10,12) accumulator empty
   uint64_t* bars = reinterpret_cast<uint64_t*>(out_stage + kStagingBytes);
   uint64_t* bar_full = bars;
-  uint64_t* bar_empty = bars + 8;
-  uint64_t* bar_acc_full = bars + 16;
-  uint64_t* bar_acc_empty = bars + 18;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
+  uint64_t* bar_empty = bars + 4;
+  uint64_t* bar_acc_full = bars + 8;
+  uint64_t* bar_acc_empty = bars + 10;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = abort_flag + 1;         // per group two slots: the leader's go/stop verdict per tile
 
@@ -335,11 +330,9 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       grid_launch_dependents();  // the next grid in the stream may set itself up as SMs become free
       prefetch_tensormap(&tm_a);
       prefetch_tensormap(&tm_b);
-      for (int s = 0; s < kNB; ++s) {
-        // a stage is full once its activation producer and, where the stage starts a weight tile,
-        // the weight producer have both arrived and their bytes have landed
-        mbar_init(&bar_full[s], (APER == 1 || (s & 1) == 0) ? 2 : 1);
-        mbar_init(&bar_empty[s], 1);
+      for (int g = 0; g < kMaxGroups; ++g) {
+        mbar_init(&bar_full[g], 3);   // the three producers each arrive once per group
+        mbar_init(&bar_empty[g], 1);  // one commit by the MMA thread
       }
       for (int b = 0; b < 2; ++b) {
         mbar_init(&bar_acc_full[b], 1);
@@ -369,31 +362,31 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   if (warp == 0 || warp >= kFirstExtraProducerWarp) {
     // ------------------------------------------------------------------ TMA producers
     if (lane == 0) {
-      const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty);
-      const uint32_t a_smem0 = smem_u32(a_ring), b_smem0 = smem_u32(b_ring);
+      const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty), ring0 = smem_u32(ring);
       if (warp == 0)
-        producer_role<SPARSE, kRoleActEven>(&tm_a, &tm_b, p, full0, empty0, a_smem0, b_smem0, abort_flag);
+        producer_role<SPARSE, kRoleActFirst>(&tm_a, &tm_b, p, full0, empty0, ring0, abort_flag);
       else if (warp == kFirstExtraProducerWarp)
-        producer_role<SPARSE, kRoleActOdd>(&tm_a, &tm_b, p, full0, empty0, a_smem0, b_smem0, abort_flag);
+        producer_role<SPARSE, kRoleActSecond>(&tm_a, &tm_b, p, full0, empty0, ring0, abort_flag);
       else
-        producer_role<SPARSE, kRoleWeights>(&tm_a, &tm_b, p, full0, empty0, a_smem0, b_smem0, abort_flag);
+        producer_role<SPARSE, kRoleWeights>(&tm_a, &tm_b, p, full0, empty0, ring0, abort_flag);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = make_idesc_bf16(kTileM, (uint32_t)p.BN, SPARSE);
-      constexpr uint32_t kAEntryDesc = C::kAEntryBytes >> 4;  // descriptor address units are 16 B
-      constexpr uint32_t kBTileDesc = kBTileBytes >> 4;
-      const uint32_t a_lo0 = desc_lo(smem_u32(a_ring));
-      const uint32_t b_lo0 = desc_lo(smem_u32(b_ring));
-      const uint32_t m_lo0 = desc_lo(smem_u32(a_ring) + kATileBytes);
+      // descriptor address units are 16 B
+      const uint32_t grp_desc = group_bytes(C::kAGroupBytes, p.BN) >> 4;
+      const uint32_t b_desc = ((uint32_t)p.BN * 128u) >> 4;
+      const uint32_t ring_lo0 = desc_lo(smem_u32(ring));
       const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty);
       const uint32_t meta_tmem0 = tmem_base + kMetaCol;
       // channels left in the last chunk decide how many MMAs its k-blocks need
       const int tail_c = p.C_in - (p.cblocks - 1) * kBlockK;
+      const int mma_full = SPARSE ? 2 : 4;
       const int mma_tail = SPARSE ? ((tail_c + 31) >> 5) : ((tail_c + 15) >> 4);
-      const int last_cc = p.cblocks - 1;
-      uint32_t s = 0, ph = 0;  // stage and its phase parity
+      const int tail_start = (tail_c == kBlockK) ? p.kblocks : (p.cblocks - 1) * p.taps;  // first k-block of the tail
+      const int a_lean_end = tail_start >> 1;  // groups before this one hold two full k-blocks
+      uint32_t g = 0, ph = 0;  // group slot and its phase parity
       uint32_t tcount = 0;
       uint32_t mslot = 0;
       bool ok = true;
@@ -406,77 +399,56 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kAccCol1;
         uint32_t accumulate = 0;
-        const int kb0 = seg.a0 * APER;
-        const int kb1 = (seg.a1 * APER < p.kblocks) ? seg.a1 * APER : p.kblocks;
-        uint32_t a_lo = 0, meta_tmem = 0;
-        const int n_stages = (seg.a1 - seg.a0) * APER;  // stages this segment occupies
-        // k-blocks before the last channel chunk need the full number of MMAs: they take the lean
-        // loop.  This thread's instruction stream paces the tensor pipe (its queue is shallow), so
-        // the loop holds nothing but the wait, the MMAs and the commit.
-        const int tail_start = (tail_c == kBlockK) ? p.kblocks : last_cc * p.taps;
-        int n_lean = ((kb1 < tail_start) ? kb1 : tail_start) - kb0;
-        if (n_lean < 0) n_lean = 0;
-        int done_stages = 0;
-        for (; done_stages < n_lean; ++done_stages) {
-          if (!mbar_wait_a(full0 + 8u * s, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-          const uint32_t b_lo = b_lo0 + s * kBTileDesc;
+        // This thread's instruction stream paces the tensor pipe (its queue is shallow): per group
+        // one wait, the MMAs, one commit, and as little else as possible.
+        for (int a = seg.a0; a < seg.a1; ++a) {
+          if (!mbar_wait_a(full0 + 8u * g, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+          const uint32_t a_lo = ring_lo0 + g * grp_desc;
+          const uint32_t b0_lo = a_lo + (C::kAGroupBytes >> 4);
+          const uint32_t b1_lo = b0_lo + b_desc;
           if (SPARSE) {
-            const uint32_t a_sub = s & 1u;
-            if (a_sub == 0) {
-              a_lo = a_lo0 + (s >> 1) * kAEntryDesc;
-              meta_tmem = meta_tmem0 + 4u * mslot;
-              mslot ^= 1u;
-              tc_cp_128x128b_lo(meta_tmem, m_lo0 + (s >> 1) * kAEntryDesc);
+            // metadata image -> 4 TMEM columns: 2 per k-block.  Kept values of the second k-block
+            // start 64 B into the tile's rows; per MMA A advances 16 kept values = 32 B, B 32
+            // channels = 64 B (descriptor units of 16 B).
+            const uint32_t meta_tmem = meta_tmem0 + 4u * mslot;
+            mslot ^= 1u;
+            tc_cp_128x128b_lo(meta_tmem, a_lo + (kATileBytes >> 4));
+            if (a < a_lean_end) {
+              tc_mma_sparse_lo(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
+              tc_mma_sparse_lo(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
+              tc_mma_sparse_lo(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
+              tc_mma_sparse_lo(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
+            } else {
+              const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
+              const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
+              tc_mma_sparse_lo(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
+              if (n0 > 1) tc_mma_sparse_lo(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
+              if (n1 > 0) tc_mma_sparse_lo(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
+              if (n1 > 1) tc_mma_sparse_lo(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
             }
-            // k-block a_sub of the weight tile: kept values start 64 B in, metadata 2 columns in;
-            // per MMA A advances 16 kept values = 32 B, B 32 channels = 64 B (descriptor units of 16 B)
-            const uint32_t a_kb = a_lo + 4u * a_sub;
-            const uint32_t meta_kb = meta_tmem + 2u * a_sub;
-            tc_mma_sparse_lo(d_tmem, a_kb, b_lo, meta_kb, idesc, accumulate);
-            tc_mma_sparse_lo(d_tmem, a_kb + 2u, b_lo + 4u, meta_kb, idesc | 1u, 1u);
           } else {
-            a_lo = a_lo0 + s * kAEntryDesc;
-            tc_mma_dense_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
-            tc_mma_dense_lo(d_tmem, a_lo + 2u, b_lo + 2u, idesc, 1u);
-            tc_mma_dense_lo(d_tmem, a_lo + 4u, b_lo + 4u, idesc, 1u);
-            tc_mma_dense_lo(d_tmem, a_lo + 6u, b_lo + 6u, idesc, 1u);
+            const uint32_t a1_lo = a_lo + (kATileBytes >> 4);
+            if (a < a_lean_end) {
+              tc_mma_dense_lo(d_tmem, a_lo, b0_lo, idesc, accumulate);
+              tc_mma_dense_lo(d_tmem, a_lo + 2u, b0_lo + 2u, idesc, 1u);
+              tc_mma_dense_lo(d_tmem, a_lo + 4u, b0_lo + 4u, idesc, 1u);
+              tc_mma_dense_lo(d_tmem, a_lo + 6u, b0_lo + 6u, idesc, 1u);
+              tc_mma_dense_lo(d_tmem, a1_lo, b1_lo, idesc, 1u);
+              tc_mma_dense_lo(d_tmem, a1_lo + 2u, b1_lo + 2u, idesc, 1u);
+              tc_mma_dense_lo(d_tmem, a1_lo + 4u, b1_lo + 4u, idesc, 1u);
+              tc_mma_dense_lo(d_tmem, a1_lo + 6u, b1_lo + 6u, idesc, 1u);
+            } else {
+              const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
+              const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
+              for (int kk = 0; kk < n0; ++kk)
+                tc_mma_dense_lo(d_tmem, a_lo + 2u * kk, b0_lo + 2u * kk, idesc, (kk > 0) ? 1u : accumulate);
+              for (int kk = 0; kk < n1; ++kk) tc_mma_dense_lo(d_tmem, a1_lo + 2u * kk, b1_lo + 2u * kk, idesc, 1u);
+            }
           }
           accumulate = 1;
-          tc_commit_a(empty0 + 8u * s);
-          if (++s == (uint32_t)kNB) {
-            s = 0;
-            ph ^= 1u;
-          }
-        }
-        // the rest: k-blocks of the last channel chunk (possibly fewer MMAs) and, for a weight tile
-        // whose second k-block does not exist, a stage that only keeps the ring's phases in step
-        for (int kb = kb0 + done_stages; ok && done_stages < n_stages; ++done_stages, ++kb) {
-          if (!mbar_wait_a(full0 + 8u * s, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-          if (kb < kb1) {
-            const uint32_t b_lo = b_lo0 + s * kBTileDesc;
-            const int n_mma = (kb >= tail_start) ? mma_tail : (SPARSE ? 2 : 4);
-            if (SPARSE) {
-              const uint32_t a_sub = s & 1u;
-              if (a_sub == 0) {
-                a_lo = a_lo0 + (s >> 1) * kAEntryDesc;
-                meta_tmem = meta_tmem0 + 4u * mslot;
-                mslot ^= 1u;
-                tc_cp_128x128b_lo(meta_tmem, m_lo0 + (s >> 1) * kAEntryDesc);
-              }
-              const uint32_t a_kb = a_lo + 4u * a_sub;
-              const uint32_t meta_kb = meta_tmem + 2u * a_sub;
-              tc_mma_sparse_lo(d_tmem, a_kb, b_lo, meta_kb, idesc, accumulate);
-              if (n_mma > 1) tc_mma_sparse_lo(d_tmem, a_kb + 2u, b_lo + 4u, meta_kb, idesc | 1u, 1u);
-            } else {
-              a_lo = a_lo0 + s * kAEntryDesc;
-              tc_mma_dense_lo(d_tmem, a_lo, b_lo, idesc, accumulate);
-              for (int kk = 1; kk < n_mma; ++kk) tc_mma_dense_lo(d_tmem, a_lo + 2u * kk, b_lo + 2u * kk, idesc, 1u);
-            }
-            accumulate = 1;
-          }
-          tc_commit_a(empty0 + 8u * s);
-          if (++s == (uint32_t)kNB) {
-            s = 0;
+          tc_commit_a(empty0 + 8u * g);
+          if (++g == (uint32_t)p.ring_groups) {
+            g = 0;
             ph ^= 1u;
           }
         }
@@ -781,12 +753,12 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
     }
   }
   // Even split of K at full width, when many SMs would still idle and K is deep.
-  const int a_tiles = SPARSE ? geo.stages : geo.kblocks;
+  const int a_tiles = geo.stages;
   if (a_tiles > 1) {
     const long long tiles = ((Q + kBN - 1) / kBN) * geo.m_tiles;
     const double units = (double)tiles * a_tiles;
     const double ctas = units < workers ? units : (double)workers;
-    const double per_a_tile = kblock_cycles<SPARSE>(kBN) * (SPARSE ? 2.0 : 1.0);
+    const double per_a_tile = 2.0 * kblock_cycles<SPARSE>(kBN);
     const double split_cost = units / ctas * per_a_tile + (ctas + tiles) * kCyclesPerParkedTile;
     if (best_cost > kSplitAdvantage * split_cost) return Plan{kBN, true};
   }
@@ -819,7 +791,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   }
   if (!g_attr_set[dev][SPARSE ? 1 : 0]) {
     if (cudaFuncSetAttribute(ssconv_fwd_kernel<SPARSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)C::kSmemBytes) != cudaSuccess)
+                             (int)kMaxSmemBytes) != cudaSuccess)
       return SSCONV_ERR_CUDA;
     g_attr_set[dev][SPARSE ? 1 : 0] = true;
   }
@@ -833,6 +805,11 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   const int BN = plan.BN;
   const int pieces = (BN / 2 + kPiece - 1) / kPiece;
   const int tail_cols = BN / 2 - (pieces - 1) * kPiece;
+  // as many groups in the ring as fit beside the staging buffers, at most kMaxGroups (at least 2 fit)
+  const uint32_t grp_bytes = group_bytes(C::kAGroupBytes, BN);
+  int ring_groups = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - kStagingBytes) / grp_bytes);
+  if (ring_groups > kMaxGroups) ring_groups = kMaxGroups;
+  const uint32_t smem_bytes = 1024 + (uint32_t)ring_groups * grp_bytes + kStagingBytes + kBarrierBytes;
 
   CUtensorMap tm_a, tm_b, tm_y, tm_y_tail;
   // activations: NHWC seen as (c, w, h, n), im2col mode; elements outside the image read as zero
@@ -896,6 +873,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.BN = BN;
   p.pieces = pieces;
   p.tail_cols = tail_cols;
+  p.ring_groups = ring_groups;
   p.stride_h = d.stride_h;
   p.stride_w = d.stride_w;
   p.pad_h = d.pad_h;
@@ -909,7 +887,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.m_tiles = geo.m_tiles;
   const long long q_tiles = (Q + BN - 1) / BN;
   p.num_tiles = (int)(q_tiles * geo.m_tiles);
-  p.a_tiles = SPARSE ? geo.stages : geo.kblocks;
+  p.a_tiles = geo.stages;
   p.flags = d.flags;
   p.bias = bias;
   p.meta = static_cast<const uint8_t*>(meta);
@@ -934,7 +912,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3((unsigned)kThreads);
-  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
