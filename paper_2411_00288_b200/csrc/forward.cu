@@ -710,26 +710,29 @@ static int out_extent(int in, int k, int stride, int pad, int dil) {
 constexpr int kMaxWorkers = 148;
 constexpr size_t kRegionBytes = (size_t)kTileM * kBN * sizeof(float);
 // Cost model behind the choice of tile width and of splitting K (cycles, measured on B200).
-// A k-block of 64 dense columns takes the longer of two things.  The issuing thread: a fixed
-// cost per k-block (wait, commit, metadata copy) plus MMAs whose time grows with the tile width
-// BN.  The fill of shared memory from L2, about 68 bytes per cycle and SM: the weight tile's share
-// plus 128 BN bytes of activations.  For BN = 240 that is about 590 cycles sparse, 690 dense.  An
-// epilogue that nothing overlaps takes about 1200 cycles per 40 positions of the widest group, and
-// every parked partial tile costs the chip about 90 cycles of L2 traffic (123 KB written by the
-// main kernel and read again by the finishing kernel).
+// A k-block of 64 dense columns takes the longest of three things.  The issuing thread: per pair
+// of k-blocks one wait (about 200 cycles even on a complete barrier), about 76 per tcgen05
+// instruction (metadata copy, MMAs, commit) and some loop overhead: 365 per k-block sparse, 480
+// dense, whatever the tile width BN.  The tensor pipe: MMAs of about 35 + 0.5 BN (sparse, two per
+// k-block) or 5 + 0.49 BN (dense, four).  The fill of shared memory from L2, about 68 bytes per
+// cycle and SM when all SMs load: the weight tile's share plus 128 BN bytes of activations.  An
+// epilogue that nothing overlaps takes about 900 cycles per 40 positions of a group, and every
+// parked partial tile costs the chip about 90 cycles of L2 traffic (123 KB written by the main
+// kernel and read again by the finishing kernel).
 constexpr double kFillBytesPerCycle = 68.0;
-constexpr double kIssueFixedSparse = 242.0, kIssuePerColSparse = 1.0;   // 2 MMAs of about 35 + 0.5 BN, + 172
-constexpr double kIssueFixedDense = 170.0, kIssuePerColDense = 1.96;    // 4 MMAs of about 5 + 0.49 BN, + 150
-constexpr double kEpiloguePieceCycles = 1200.0;
+constexpr double kIssueSparse = 365.0, kIssueDense = 480.0;
+constexpr double kEpiloguePieceCycles = 900.0;
 constexpr double kCyclesPerParkedTile = 90.0;
 constexpr double kSplitAdvantage = 1.1;  // split only if the model predicts at least this gain
 
 template <bool SPARSE>
 static double kblock_cycles(int BN) {
-  const double a_bytes = SPARSE ? (kATileBytes + kMetaImageBytes) / 2.0 : (double)kATileBytes;
+  const double a_bytes = Cfg<SPARSE>::kAGroupBytes / 2.0;
   const double fill = (a_bytes + 128.0 * BN) / kFillBytesPerCycle;
-  const double issue = SPARSE ? kIssueFixedSparse + kIssuePerColSparse * BN : kIssueFixedDense + kIssuePerColDense * BN;
-  return fill > issue ? fill : issue;
+  const double issue = SPARSE ? kIssueSparse : kIssueDense;
+  const double pipe = SPARSE ? 2.0 * (35.0 + 0.5 * BN) + 11.0 : 4.0 * (5.0 + 0.49 * BN);
+  double t = fill > issue ? fill : issue;
+  return t > pipe ? t : pipe;
 }
 
 // Tile width and partition of a layer.
