@@ -356,7 +356,8 @@ def main():
         per_layer.append({"layer": spec.name, "us_sparse": round(t_s * 1e3, 2), "us_dense": round(t_d * 1e3, 2),
                           "tflops": round(flops / t_s / 1e9, 1), "gbs": round(bytes_alg / t_s / 1e6, 1),
                           "bound": "tensor" if t_c >= t_m else "hbm", "us_roofline": round(roof * 1e3, 2),
-                          "roofline_frac": round(roof / t_s, 4), "x_dense": round(t_d / t_s, 3)})
+                          "roofline_frac": round(roof / t_s, 4), "x_dense": round(t_d / t_s, 3),
+                          "plan": api.ssconv_plan(L["desc"], True)})
 
     # ---- end to end through the public API with host buffers (H2D of inputs, D2H of outputs)
     def e2e_step():

@@ -85,6 +85,16 @@ int32_t ssconv_out_shape(const ssconv_desc_t* desc, int32_t* H_out, int32_t* W_o
 int32_t ssconv_sizes(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes,
                      size_t* meta_bytes, size_t* ws_bytes_sparse, size_t* ws_bytes_dense);
 
+/* How ssconv_forward (sparse != 0) or ssconv_forward_dense (sparse == 0) would run this layer on
+ * the current device: positions per output tile (the N of the tensor-core instruction, a multiple
+ * of 16 up to 240, chosen so that the tiles fill the SMs), whether the K range is split across
+ * thread blocks (then a second, finishing kernel runs and ws is used), the number of thread
+ * blocks, and the depth of the shared-memory ring in pairs of 64-column k-blocks.  A tuning aid
+ * with no counterpart in the paper; nothing is launched.  Needs a device of compute capability
+ * 10.x to be current (SSCONV_ERR_ARCH / SSCONV_ERR_CUDA otherwise).  Any output may be NULL. */
+int32_t ssconv_plan(const ssconv_desc_t* desc, int32_t sparse, int32_t* tile_positions, int32_t* split,
+                    int32_t* ctas, int32_t* ring_groups);
+
 /* Hard pattern choice per group (Eq. 1 of Sec. 3.1 without the one-hot: the index of the
  * winning pattern).
  *   mode LOGITS:    pattern[g] = argmax_i scores[g][i]; the caller has already added any

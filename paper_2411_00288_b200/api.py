@@ -22,6 +22,7 @@ ERR_TIMEOUT = 8
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.so")
 EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes",
+           "ssconv_plan",
            "ssconv_select_mask",
            "ssconv_compress", "ssconv_decompress", "ssconv_forward", "ssconv_forward_dense",
            "ssconv_forward_static_ws")
@@ -183,6 +184,16 @@ def ssconv_decompress(desc: Desc, w_comp: torch.Tensor, meta: torch.Tensor, want
 
 
 _workspaces = {}
+
+
+def ssconv_plan(desc: Desc, sparse: bool = True) -> dict:
+    """Tile width, K split, thread blocks and ring depth the forward call would use on the current device."""
+    out = [ctypes.c_int32(0) for _ in range(4)]
+    f = lib().ssconv_plan
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_int32] + [ctypes.POINTER(ctypes.c_int32)] * 4
+    _check("ssconv_plan", f(ctypes.byref(desc), 1 if sparse else 0, *[ctypes.byref(o) for o in out]))
+    return dict(tile_positions=out[0].value, split=bool(out[1].value), ctas=out[2].value, ring_groups=out[3].value)
 
 
 def default_workspace(device) -> torch.Tensor:

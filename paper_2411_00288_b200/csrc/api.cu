@@ -17,6 +17,8 @@ int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void*
 int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias, void* y,
                              void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream);
 size_t workspace_bytes();
+int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* split, int32_t* ctas,
+                   int32_t* ring_groups);
 int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
                                  const float* bias, void* y, int32_t* dev_status, cudaStream_t stream);
 }  // namespace ssconv
@@ -108,6 +110,13 @@ int32_t ssconv_sizes(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes
   if (ws_bytes_sparse) *ws_bytes_sparse = ssconv::workspace_bytes();
   if (ws_bytes_dense) *ws_bytes_dense = ssconv::workspace_bytes();
   return SSCONV_OK;
+}
+
+int32_t ssconv_plan(const ssconv_desc_t* desc, int32_t sparse, int32_t* tile_positions, int32_t* split,
+                    int32_t* ctas, int32_t* ring_groups) {
+  int32_t st = check_desc(desc, true);
+  if (st != SSCONV_OK) return st;
+  return ssconv::plan_query(*desc, sparse != 0, tile_positions, split, ctas, ring_groups);
 }
 
 int32_t ssconv_select_mask(int32_t mode, const void* scores, int64_t G, uint8_t* pattern, void* stream) {

@@ -776,12 +776,8 @@ size_t workspace_bytes() { return scratch_bytes(kMaxWorkers); }
 static int g_sm_count[64] = {0};
 static bool g_attr_set[64][2] = {{false}};
 
-template <bool SPARSE>
-static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const void* weights, const void* meta,
-                                   const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
-                                   cudaStream_t stream, int worker_cap = kMaxWorkers, bool force_split = false) {
-  using C = Cfg<SPARSE>;
-  if (!load_driver_entry_points()) return SSCONV_ERR_CUDA;
+// Current device and its SM count (checked once per device: must be compute capability 10.x).
+static int32_t current_device(int* dev_out) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SSCONV_ERR_CUDA;
   if (g_sm_count[dev] == 0) {
@@ -791,6 +787,49 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
       return SSCONV_ERR_CUDA;
     g_sm_count[dev] = sms;
+  }
+  *dev_out = dev;
+  return SSCONV_OK;
+}
+
+static int ring_groups_for(uint32_t a_group_bytes, int BN) {
+  // as many groups in the ring as fit beside the staging buffers, at most kMaxGroups (at least 2 fit)
+  const int n = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - kStagingBytes) / group_bytes(a_group_bytes, BN));
+  return n > kMaxGroups ? kMaxGroups : n;
+}
+
+// What launch_forward_impl would do for this layer on the current device.
+int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* split, int32_t* ctas,
+                   int32_t* ring_groups) {
+  int dev = 0;
+  const int32_t st = current_device(&dev);
+  if (st != SSCONV_OK) return st;
+  const Geometry geo = make_geometry(d);
+  const long long Q = (long long)d.N * out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h) *
+                      out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
+  const int workers = g_sm_count[dev] < kMaxWorkers ? g_sm_count[dev] : kMaxWorkers;
+  const Plan plan = sparse ? plan_layer<true>(Q, geo, workers, false) : plan_layer<false>(Q, geo, workers, false);
+  const long long tiles = ((Q + plan.BN - 1) / plan.BN) * geo.m_tiles;
+  const bool do_split = plan.split && geo.stages > 1;
+  const long long work = do_split ? tiles * geo.stages : tiles;
+  if (bn) *bn = plan.BN;
+  if (split) *split = do_split ? 1 : 0;
+  if (ctas) *ctas = (int32_t)(work < workers ? work : workers);
+  if (ring_groups)
+    *ring_groups = ring_groups_for(sparse ? Cfg<true>::kAGroupBytes : Cfg<false>::kAGroupBytes, plan.BN);
+  return SSCONV_OK;
+}
+
+template <bool SPARSE>
+static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const void* weights, const void* meta,
+                                   const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
+                                   cudaStream_t stream, int worker_cap = kMaxWorkers, bool force_split = false) {
+  using C = Cfg<SPARSE>;
+  if (!load_driver_entry_points()) return SSCONV_ERR_CUDA;
+  int dev = 0;
+  {
+    const int32_t st = current_device(&dev);
+    if (st != SSCONV_OK) return st;
   }
   if (!g_attr_set[dev][SPARSE ? 1 : 0]) {
     if (cudaFuncSetAttribute(ssconv_fwd_kernel<SPARSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -808,10 +847,8 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   const int BN = plan.BN;
   const int pieces = (BN / 2 + kPiece - 1) / kPiece;
   const int tail_cols = BN / 2 - (pieces - 1) * kPiece;
-  // as many groups in the ring as fit beside the staging buffers, at most kMaxGroups (at least 2 fit)
   const uint32_t grp_bytes = group_bytes(C::kAGroupBytes, BN);
-  int ring_groups = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - kStagingBytes) / grp_bytes);
-  if (ring_groups > kMaxGroups) ring_groups = kMaxGroups;
+  const int ring_groups = ring_groups_for(C::kAGroupBytes, BN);
   const uint32_t smem_bytes = 1024 + (uint32_t)ring_groups * grp_bytes + kStagingBytes + kBarrierBytes;
 
   CUtensorMap tm_a, tm_b, tm_y, tm_y_tail;
