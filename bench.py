@@ -171,6 +171,28 @@ def reference_arm(args):
     print(json.dumps(line))
 
 
+# DRAM traffic of the sparse forward kernels of one step (7 launches of ssconv_fwd_kernel<sparse> and
+# the finishing kernel of the one split layer), dram__bytes_read.sum + dram__bytes_write.sum from an
+# ncu capture of this workload (summary and command: profiles/bench_resnet18_sweep_dram_traffic.md).
+# It belongs to the kernel sources with the digest below; with other sources the bench reports null.
+TRAFFIC_BYTES_PER_STEP = 72.97e6
+TRAFFIC_SOURCES = ("forward.cu", "sm100_ptx.cuh", "layout.cuh")
+TRAFFIC_SOURCES_SHA256 = "85521aa19fcd9c00238220c1dd6d674ed3fa262ce6a3edae3dd7678e3251d798"
+
+
+def measured_traffic():
+    import hashlib
+    h = hashlib.sha256()
+    root = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2411_00288_b200", "csrc")
+    try:
+        for name in TRAFFIC_SOURCES:
+            with open(os.path.join(root, name), "rb") as fh:
+                h.update(fh.read())
+    except OSError:
+        return None
+    return TRAFFIC_BYTES_PER_STEP if h.hexdigest() == TRAFFIC_SOURCES_SHA256 else None
+
+
 # ----------------------------------------------------------------------------- GPU arm
 def main():
     global CONFIG_ID, WORKLOAD
@@ -404,7 +426,11 @@ def main():
                          "peak_source": f"2 x dense bf16 burst of {peaks['source']} peaks (nominal sparse:dense ratio)",
                          "layer_mix_ceiling": total_flops / (sum_roof_ms * 1e-3) / 1e12,
                          "frac_of_layer_mix_ceiling": sum_roof_ms / sum_kernel_ms,
-                         "hbm_peak_gbs": peaks["hbm_gbs"], "traffic": None},
+                         "hbm_peak_gbs": peaks["hbm_gbs"],
+                         "traffic": measured_traffic() if CONFIG_ID == 2 else None,
+                         "traffic_unit": "bytes per step (DRAM read + write of the sparse forward and finishing "
+                                         "kernels, ncu)",
+                         "algorithmic_bytes_per_step": sum(L["spec"].algorithmic_bytes(sparse=True) for L in prep)},
             "per_layer": per_layer,
             "e2e": {"value": world * total_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
