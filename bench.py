@@ -217,11 +217,9 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2411_00288_b200 import api, synth, build as libbuild
+    from paper_2411_00288_b200 import api, synth, ranks, build as libbuild
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank, local_rank, world = ranks.env_ranks()
     distributed = world > 1
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -290,11 +288,7 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if not distributed:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return ranks.max_over_ranks(ms, dev)
 
     def capture(fn):
         """Record fn()'s launches into a CUDA graph (the launches are the same C-ABI calls; the
@@ -337,7 +331,7 @@ def main():
     time_replays(g_sparse, warmup)
     ms_total = time_replays(g_sparse, steps)
     ms_per_step = ms_total / steps
-    value = world * total_flops / (ms_per_step * 1e-3) / 1e12
+    value = ranks.job_throughput(total_flops, world, ms_per_step) / 1e12
 
     # ---- dense counterpart (S4) on the same buffers, same rotation
     time_replays(g_dense, warmup)
