@@ -88,7 +88,7 @@ struct FwdParams {
   int m_tiles, num_tiles;
   int a_tiles;              // pairs of k-blocks (groups) per output tile
   int split;                // 1: units dealt out evenly across CTAs (stream-K); 0: whole tiles per CTA
-  long long units;          // num_tiles * a_tiles
+  int work_quot, work_rem;  // work items per CTA: quotient and remainder of (tiles or units) / grid
   float4* ws_regions;       // [2 * gridDim.x] regions of 128 x 240 fp32: a CTA's partial tiles
   uint32_t flags;
   const float* bias;
@@ -102,45 +102,42 @@ struct Segment {
   int tile, a0, a1;
 };
 
-// Walks the segments of this CTA's contiguous range of work units.
+// The W work items (whole tiles, or (tile, group) units when K is split) are dealt out to the G
+// CTAs in contiguous, near-equal ranges: CTA c gets [c q + min(c, r), ...) of length q + (c < r)
+// with q = W / G, r = W % G, both computed on the host: the device needs no division for it.
 struct WorkIter {
-  long long u, u_end;
-  int A;
+  int tile, a0, left, A;  // next tile, first group of it, units left in this CTA's range, groups per tile
   __device__ WorkIter(const FwdParams& p) {
     A = p.a_tiles;
-    const long long c = blockIdx.x, G = gridDim.x;
+    const uint32_t c = blockIdx.x;
+    const uint32_t start = c * (uint32_t)p.work_quot + (c < (uint32_t)p.work_rem ? c : (uint32_t)p.work_rem);
+    const int count = p.work_quot + (c < (uint32_t)p.work_rem ? 1 : 0);
     if (p.split) {
-      if (p.units < (1LL << 31) / (G + 1)) {  // 32-bit divisions: this runs before the first load
-        const uint32_t U = (uint32_t)p.units, g = (uint32_t)G, cc = (uint32_t)c;
-        u = cc * U / g;
-        u_end = (cc + 1) * U / g;
-      } else {
-        u = c * p.units / G;
-        u_end = (c + 1) * p.units / G;
-      }
-    } else if (p.num_tiles < (1 << 23)) {
-      const uint32_t T = (uint32_t)p.num_tiles, g = (uint32_t)G, cc = (uint32_t)c;
-      u = (long long)(cc * T / g) * A;
-      u_end = (long long)((cc + 1) * T / g) * A;
+      tile = (int)(start / (uint32_t)A);  // the one division of the split path
+      a0 = (int)(start - (uint32_t)tile * (uint32_t)A);
+      left = count;
     } else {
-      u = (c * p.num_tiles / G) * A;
-      u_end = ((c + 1) * p.num_tiles / G) * A;
+      tile = (int)start;
+      a0 = 0;
+      left = count * A;
     }
   }
   __device__ bool next(Segment& s) {
-    if (u >= u_end) return false;
-    s.tile = (u < (1LL << 31)) ? (int)((uint32_t)u / (uint32_t)A) : (int)(u / A);
-    s.a0 = (int)(u - (long long)s.tile * A);
-    const long long left = u_end - u;
-    s.a1 = (left >= A - s.a0) ? A : s.a0 + (int)left;
-    u += s.a1 - s.a0;
+    if (left <= 0) return false;
+    s.tile = tile;
+    s.a0 = a0;
+    s.a1 = (left >= A - a0) ? A : a0 + left;
+    left -= s.a1 - s.a0;
+    ++tile;
+    a0 = 0;
     return true;
   }
 };
 
-// CTA that owns work unit u under the even split: the c with c*U/G <= u < (c+1)*U/G.
-__device__ __forceinline__ int unit_owner(long long u, long long U, long long G) {
-  return (int)(((u + 1) * G - 1) / U);
+// CTA that owns work unit u under that dealing: inverse of start(c) = c q + min(c, r).
+__device__ __forceinline__ int unit_owner(uint32_t u, uint32_t q, uint32_t r) {
+  const uint32_t big = r * (q + 1);  // units held by the r CTAs with one extra
+  return (u < big) ? (int)(u / (q + 1)) : (int)(r + (u - big) / q);
 }
 
 // A scratch region holds one 128 x 240 fp32 partial tile in the order the epilogue threads hold it:
@@ -326,19 +323,19 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   // Warp 0 initialises the barriers and goes straight on to load; everybody else also waits for
   // the TMEM allocation (which the producer does not need).
   if (warp == 0) {
+    // barrier slots in memory order: 4 group full (3 arrivals: the three producers), 4 group empty (one
+    // commit by the MMA thread), 2 accumulator full, 2 accumulator empty (one arrival per epilogue
+    // warp); lane i initialises slot i
+    if (lane < 12) {
+      const uint32_t count = (lane < 4) ? 3u : (lane < 10) ? 1u : (uint32_t)(4 * kGroups);
+      mbar_init(&bars[lane], count);
+    }
     if (lane == 0) {
       grid_launch_dependents();  // the next grid in the stream may set itself up as SMs become free
-      prefetch_tensormap(&tm_a);
-      prefetch_tensormap(&tm_b);
-      for (int g = 0; g < kMaxGroups; ++g) {
-        mbar_init(&bar_full[g], 3);   // the three producers each arrive once per group
-        mbar_init(&bar_empty[g], 1);  // one commit by the MMA thread
-      }
-      for (int b = 0; b < 2; ++b) {
-        mbar_init(&bar_acc_full[b], 1);
-        mbar_init(&bar_acc_empty[b], 4 * kGroups);
-      }
       *abort_flag = 0;
+    }
+    __syncwarp();
+    if (lane == 0) {
       mbar_fence_init();
       fence_proxy_async_smem();
     }
@@ -349,9 +346,13 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       tmem_alloc(tmem_slot, kTmemCols);
       tmem_relinquish();
     }
-    if (warp == 2 && lane == 0) {
-      prefetch_tensormap(&tm_y);
-      prefetch_tensormap(&tm_y_tail);
+    if (lane == 0) {  // tensor maps are fetched while thread 0 initialises the barriers
+      if (warp == kFirstExtraProducerWarp) prefetch_tensormap(&tm_b);
+      if (warp == kFirstExtraProducerWarp + 1) prefetch_tensormap(&tm_a);
+      if (warp == 2) {
+        prefetch_tensormap(&tm_y);
+        prefetch_tensormap(&tm_y_tail);
+      }
     }
     tc_fence_before();
     setup_bar_sync();
@@ -587,8 +588,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
 struct FinishParams {
   int C_out, Q;
   int m_tiles, a_tiles;
-  int workers;            // grid size of the main kernel
-  long long units;
+  int work_quot, work_rem;  // the main kernel's dealing of (tile, group) units to its CTAs
   const float4* ws_regions;
   uint32_t flags;
   const float* bias;
@@ -609,9 +609,9 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
   const int grp = item % kGroups;
   const int tile = item / kGroups;
   if (gtid == 0) grid_launch_dependents();
-  const long long u_first = (long long)tile * f.a_tiles;
-  const int c_first = unit_owner(u_first, f.units, f.workers);
-  const int c_last = unit_owner(u_first + f.a_tiles - 1, f.units, f.workers);
+  const uint32_t u_first = (uint32_t)tile * (uint32_t)f.a_tiles;
+  const int c_first = unit_owner(u_first, f.work_quot, f.work_rem);
+  const int c_last = unit_owner(u_first + f.a_tiles - 1, f.work_quot, f.work_rem);
   if (c_first == c_last) return;  // the tile was computed whole by one CTA, which also finished it
   const int pt = tile / f.m_tiles;
   const int m = tile - pt * f.m_tiles;
@@ -934,17 +934,23 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.y = static_cast<__nv_bfloat16*>(y);
   p.dev_status = dev_status;
 
-  p.units = (long long)p.num_tiles * p.a_tiles;
+  const long long units = q_tiles * geo.m_tiles * geo.stages;
+  if (units >= (1LL << 31)) return SSCONV_ERR_UNSUPPORTED_SHAPE;  // 32-bit work indices on the device
   p.split = (plan.split && p.a_tiles > 1) ? 1 : 0;
   int grid;
   if (p.split) {
-    grid = p.units < workers ? (int)p.units : workers;
+    grid = units < workers ? (int)units : workers;
     if (ws == nullptr || ws_bytes < scratch_bytes(worker_cap)) return SSCONV_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(ws) & 15u) return SSCONV_ERR_ALIGNMENT;
     p.ws_regions = static_cast<float4*>(ws);
   } else {
     grid = p.num_tiles < workers ? p.num_tiles : workers;
     p.ws_regions = nullptr;
+  }
+  {
+    const long long work = p.split ? units : (long long)p.num_tiles;
+    p.work_quot = (int)(work / grid);
+    p.work_rem = (int)(work % grid);
   }
   // Programmatic stream serialisation: this grid's set-up (barriers, TMEM, tensor-map fetch, index
   // arithmetic) may overlap the tail of the previous kernel in the stream; the kernel itself
@@ -967,8 +973,8 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     f.Q = (int)Q;
     f.m_tiles = geo.m_tiles;
     f.a_tiles = p.a_tiles;
-    f.workers = grid;
-    f.units = p.units;
+    f.work_quot = p.work_quot;
+    f.work_rem = p.work_rem;
     f.ws_regions = p.ws_regions;
     f.flags = d.flags;
     f.bias = bias;
