@@ -29,7 +29,8 @@ if ROOT not in sys.path:
 
 METRIC = "dense-equiv TFLOP/s of 2:4 sparse conv fwd (bf16), % of sparse-TC roofline, xdense"
 WORKLOADS = {2: "resnet18_3x3_sweep_bf16_nhwc_batch32", 3: "resnet50_bottleneck_layers_bf16_nhwc_batch64",
-             4: "convnext_t_pointwise_layers_bf16_nhwc_batch128"}
+             4: "convnext_t_pointwise_layers_bf16_nhwc_batch128",
+           5: "resnet50_conv_stack_end_to_end_bf16_nhwc_batch256"}
 CONFIG_ID = 2          # the benchmarked workload; --workload-config picks another for layer tables
 WORKLOAD = WORKLOADS[CONFIG_ID]
 L2_BYTES = 126 * 2 ** 20
@@ -193,6 +194,88 @@ def measured_traffic():
     return TRAFFIC_BYTES_PER_STEP if h.hexdigest() == TRAFFIC_SOURCES_SHA256 else None
 
 
+# ----------------------------------------------------------------------------- conv stack, end to end
+def stack_arm(args):
+    """ResNet-50-shaped convolution stack (dense stem, max-pool, 52 masked convolutions) at batch 256
+    per GPU: images per second of the whole stack, recorded into one CUDA graph and replayed, with
+    the same stack on the dense kernel for comparison.  One JSON line on rank 0."""
+    import torch
+    import torch.distributed as dist
+    from paper_2411_00288_b200 import api, synth, stack, ranks, build as libbuild
+
+    rank, local_rank, world = ranks.env_ranks()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        libbuild.build()
+    if world > 1:
+        dist.barrier()
+    api.lib()
+    batch = args.batch or 256
+    steps_def = synth.resnet50_stack(batch)
+    net = stack.ConvStack(steps_def, dev, with_dense=True)
+    g = torch.Generator().manual_seed(synth.SEED_BASE + 577 + rank)
+    x = torch.zeros((batch, 224, 224, 8), dtype=torch.bfloat16)
+    x[..., :3] = torch.randn((batch, 224, 224, 3), generator=g, dtype=torch.float32).to(torch.bfloat16)
+    xd = x.to(dev)
+    warmup, steps = max(3, args.warmup), min(args.steps, 200)
+
+    def timed(sparse):
+        for _ in range(2):
+            net.forward(xd, sparse=sparse)
+        torch.cuda.synchronize()
+        c0 = api.ssconv_launch_count()
+        net.forward(xd, sparse=sparse)
+        launches = api.ssconv_launch_count() - c0
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            net.forward(xd, sparse=sparse)
+        for _ in range(warmup):
+            graph.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            graph.replay()
+        e1.record()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        return ranks.max_over_ranks(e0.elapsed_time(e1) / steps, dev), launches
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms_sparse, launches = timed(True)
+    ms_dense, _ = timed(False)
+    clocks = sampler.stop() if rank == 0 else None
+    status = int(net.status.item())
+    if rank == 0:
+        flops = net.conv_flops()
+        print(json.dumps({
+            "metric": "end-to-end images/s of the ResNet-50-shaped convolution stack, 2:4 masked (bf16)",
+            "value": ranks.job_throughput(batch, world, ms_sparse), "unit": "images/s", "n_gpus": world,
+            "steps": steps, "warmup": warmup, "ms_per_step": ms_sparse, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "batch_per_gpu": batch,
+                       "stack": "stem 7x7 s2 (dense, input padded 3 -> 8 channels), 3x3 s2 max-pool (torch op), 16 "
+                                "bottlenecks as reduce -> 3x3 -> expand with bias + ReLU, 4 downsample convolutions on "
+                                "their block's input; no residual additions",
+                       "l2": "activations of a step total several GB (> L2)",
+                       "launch": "the stack's calls recorded into one CUDA graph and replayed"},
+            "dense_equiv_tflops": ranks.job_throughput(flops, world, ms_sparse) / 1e12,
+            "x_dense": ms_dense / ms_sparse, "ms_per_step_dense": ms_dense,
+            "images_per_s_dense": ranks.job_throughput(batch, world, ms_dense),
+            "gpu_launches": steps * launches, "clocks": clocks, "dev_status": status}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ----------------------------------------------------------------------------- GPU arm
 def main():
     global CONFIG_ID, WORKLOAD
@@ -206,6 +289,7 @@ def main():
     ap.add_argument("--only-layer", type=int, default=None,
                     help="profiling aid: launch just this layer of the sweep --layer-iters times and exit")
     ap.add_argument("--dense", action="store_true", help="with --only-layer: use the dense kernel")
+    ap.add_argument("--batch", type=int, default=None, help="with --workload-config 5: images per GPU (default 256)")
     ap.add_argument("--workload-config", type=int, default=CONFIG_ID, choices=sorted(WORKLOADS),
                     help="layer set to run (default: the benchmarked ResNet-18 sweep)")
     args = ap.parse_args()
@@ -213,6 +297,9 @@ def main():
     WORKLOAD = WORKLOADS[CONFIG_ID]
     if args.impl == "reference":
         reference_arm(args)
+        return
+    if CONFIG_ID == 5:
+        stack_arm(args)
         return
 
     import torch

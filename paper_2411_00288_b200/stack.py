@@ -1,0 +1,70 @@
+"""Run a stack of convolutions (synth.StackStep) through the library, layer by layer.
+
+Only marshalling: weights are masked and compressed once with the library's own calls, output
+buffers are allocated once, and forward() issues one C-ABI call per convolution on the current
+stream (so it can be recorded into a CUDA graph).  The 3x3 stride-2 max-pool between the stem and
+the first block is not part of the library; it runs as a torch op on the same stream.
+"""
+from __future__ import annotations
+
+from typing import List, Optional
+
+import torch
+
+from . import api, synth
+
+
+class ConvStack:
+    def __init__(self, steps: List[synth.StackStep], device, with_dense: bool = False):
+        self.steps = steps
+        self.device = torch.device(device)
+        self.layers = []
+        self.outputs: List[Optional[torch.Tensor]] = []
+        self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
+        shape = None
+        shapes = []
+        for st in steps:
+            if st.kind == "maxpool":
+                n, h, w, c = shapes[st.src]
+                shape = (n, (h + 2 - 3) // 2 + 1, (w + 2 - 3) // 2 + 1, c)
+                self.layers.append(None)
+            else:
+                spec = st.spec
+                inp = synth.make_weights(spec)
+                desc = api.desc_from_spec(spec)
+                w = inp.w.to(self.device)
+                bias = inp.bias.to(self.device) if inp.bias is not None else None
+                entry = dict(desc=desc, w=None, bias=bias, w_comp=None, meta=None, w_host=inp.w, bias_host=inp.bias)
+                if st.kind == "conv":
+                    pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
+                    entry["w_comp"], entry["meta"] = api.ssconv_compress(desc, w, pat)
+                    entry["pattern"] = pat
+                if st.kind == "dense" or with_dense:
+                    entry["w"] = w
+                self.layers.append(entry)
+                shape = (spec.N, spec.H_out, spec.W_out, spec.C_out)
+            shapes.append(shape)
+            self.outputs.append(torch.empty(shape, dtype=torch.bfloat16, device=self.device))
+        torch.cuda.synchronize(self.device)
+
+    def forward(self, x: torch.Tensor, sparse: bool = True) -> torch.Tensor:
+        """Enqueue the whole stack; returns the last chained output (not synchronised)."""
+        last = None
+        for i, st in enumerate(self.steps):
+            src = x if st.src < 0 else self.outputs[st.src]
+            y = self.outputs[i]
+            if st.kind == "maxpool":
+                pooled = torch.nn.functional.max_pool2d(src.permute(0, 3, 1, 2), 3, 2, 1)
+                y.copy_(pooled.permute(0, 2, 3, 1))
+            else:
+                L = self.layers[i]
+                if st.kind == "conv" and sparse:
+                    api.ssconv_forward(L["desc"], src, L["w_comp"], L["meta"], L["bias"], y=y, dev_status=self.status)
+                else:
+                    api.ssconv_forward_dense(L["desc"], src, L["w"], L["bias"], y=y, dev_status=self.status)
+            if st.feeds_next:
+                last = y
+        return last
+
+    def conv_flops(self) -> int:
+        return sum(st.spec.dense_equiv_flops for st in self.steps if st.kind != "maxpool")

@@ -138,6 +138,57 @@ def config_layers(config: int, batch: Optional[int] = None) -> List[LayerSpec]:
     raise ValueError(f"unknown config {config}")
 
 
+@dataclass(frozen=True)
+class StackStep:
+    """One step of a convolution stack: `kind` is "conv" (masked), "dense" (unmasked convolution)
+    or "maxpool" (3x3, stride 2, pad 1).  `src` is the index of the step whose output it reads (-1:
+    the stack's input); `feeds_next` is False for branches whose output nothing consumes."""
+    kind: str
+    spec: Optional[LayerSpec]
+    src: int
+    feeds_next: bool = True
+
+
+def resnet50_stack(batch: int = 256) -> List[StackStep]:
+    """The convolution stack of a Torchvision-shaped ResNet-50 as a residual-free chain: stem
+    (7x7 stride 2, dense, on an input padded from 3 to 8 channels), 3x3 stride-2 max-pool, then per
+    bottleneck reduce -> 3x3 -> expand, each with bias and ReLU, the expand output feeding the next
+    block; the four downsample convolutions read their block's input and feed nothing.  Every
+    convolution has exactly the shape, traffic and FLOPs of the network's; residual additions and
+    batch-norm statistics are left out (batch norm counts as folded into the bias)."""
+    steps: List[StackStep] = []
+    stem = LayerSpec("r50_stem", batch, 224, 224, 8, 64, 7, 7, 2, 3, w_std="he", config=5, index=90)
+    steps.append(StackStep("dense", stem, -1))
+    steps.append(StackStep("maxpool", None, 0))
+    src = 1
+    specs = config_layers(5, batch)
+    i = 0
+    while i < len(specs):
+        block_in = src
+        reduce_, conv3 = specs[i], specs[i + 1]
+        steps.append(StackStep("conv", reduce_, block_in))
+        steps.append(StackStep("conv", conv3, len(steps) - 1))
+        after3 = len(steps) - 1
+        i += 2
+        if specs[i].name.endswith("_down"):
+            steps.append(StackStep("conv", specs[i], block_in, feeds_next=False))
+            i += 1
+        steps.append(StackStep("conv", specs[i], after3))
+        src = len(steps) - 1
+        i += 1
+    return steps
+
+
+def make_weights(spec: LayerSpec, seed: Optional[int] = None) -> "LayerInputs":
+    """Weights and bias only (no activations are drawn): for layers whose input comes from the
+    layer before.  Its own seed stream, so the bits differ from make_inputs' for the same spec."""
+    g = torch.Generator().manual_seed((spec.seed if seed is None else seed) + 50_000_000)
+    w = (torch.randn((spec.C_out, spec.KH, spec.KW, spec.C_in), generator=g, dtype=torch.float32)
+         * _std(spec)).to(torch.bfloat16)
+    bias = (torch.randn((spec.C_out,), generator=g, dtype=torch.float32) * 0.1) if spec.has_bias else None
+    return LayerInputs(spec, None, w, bias, None, None)
+
+
 def _std(spec: LayerSpec) -> float:
     fan_in = spec.K
     if spec.w_std == "fan_in":
