@@ -263,7 +263,7 @@ def stack_arm(args):
             "steps": steps, "warmup": warmup, "ms_per_step": ms_sparse, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "batch_per_gpu": batch,
-                       "stack": "stem 7x7 s2 (dense, input padded 3 -> 8 channels), 3x3 s2 max-pool (torch op), 16 "
+                       "stack": "stem 7x7 s2 (dense, input padded 3 -> 8 channels), 3x3 s2 max-pool, 16 "
                                 "bottlenecks as reduce -> 3x3 -> expand with bias + ReLU, 4 downsample convolutions on "
                                 "their block's input; no residual additions",
                        "l2": "activations of a step total several GB (> L2)",

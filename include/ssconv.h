@@ -122,6 +122,14 @@ int32_t ssconv_compress(const ssconv_desc_t* desc, const void* w_bf16, const uin
 int32_t ssconv_decompress(const ssconv_desc_t* desc, const void* w_comp, const void* meta,
                           void* w_masked_bf16, uint8_t* pattern_out, void* stream);
 
+/* Max-pooling of NHWC bf16 activations with a k x k window, given stride and padding (padding
+ * never wins): y[n,ho,wo,c] = max over the window of x.  H_out = (H + 2 pad - k)/stride + 1.  Not
+ * part of the paper's method: the pooling step between the stem and the first block of the
+ * ResNet-shaped convolution stacks the paper evaluates on (Sec. 4), here so that such a stack runs
+ * without any other library.  x, y: device, 16-byte aligned; C % 8 == 0; pad < k. */
+int32_t ssconv_maxpool(const void* x, void* y, int32_t N, int32_t H, int32_t W, int32_t C, int32_t k,
+                       int32_t stride, int32_t pad, void* stream);
+
 /* Masked convolution forward (Eq. 6 with the direct definition Eq. 4):
  *   y[n,ho,wo,co] = act( bias[co] + sum_{kh,kw,ci} x[n, ho*s-p+kh*d, wo*s-p+kw*d, ci]
  *                                                  * (M .* W)[co,kh,kw,ci] ),

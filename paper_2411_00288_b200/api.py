@@ -24,7 +24,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.
 EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes",
            "ssconv_plan",
            "ssconv_select_mask",
-           "ssconv_compress", "ssconv_decompress", "ssconv_forward", "ssconv_forward_dense",
+           "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_forward", "ssconv_forward_dense",
            "ssconv_forward_static_ws")
 
 
@@ -241,6 +241,21 @@ def ssconv_forward_dense(desc: Desc, x: torch.Tensor, w: torch.Tensor, bias: Opt
     _check("ssconv_forward_dense", lib().ssconv_forward_dense(
         ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _ptr(ws),
         0 if ws is None else ws.numel() * ws.element_size(), _ptr(dev_status), _stream(stream)))
+    return y
+
+
+def ssconv_maxpool(x: torch.Tensor, k: int = 3, stride: int = 2, pad: int = 1, y: Optional[torch.Tensor] = None,
+                   stream=None) -> torch.Tensor:
+    """k x k max-pooling of NHWC bf16 activations; returns y [N,H_out,W_out,C] (enqueued, not synchronised)."""
+    _need_cuda(x, y)
+    n, h, w, c = x.shape
+    if y is None:
+        y = torch.empty((n, (h + 2 * pad - k) // stride + 1, (w + 2 * pad - k) // stride + 1, c),
+                        dtype=torch.bfloat16, device=x.device)
+    f = lib().ssconv_maxpool
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int32] * 7 + [ctypes.c_void_p]
+    _check("ssconv_maxpool", f(_ptr(x), _ptr(y), n, h, w, c, k, stride, pad, _stream(stream)))
     return y
 
 

@@ -17,6 +17,8 @@ int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void*
 int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias, void* y,
                              void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream);
 size_t workspace_bytes();
+cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad,
+                           cudaStream_t st);
 int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* split, int32_t* ctas,
                    int32_t* ring_groups);
 int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
@@ -150,6 +152,19 @@ int32_t ssconv_decompress(const ssconv_desc_t* desc, const void* w_comp, const v
   if (!aligned16(w_comp) || !aligned16(meta) || !aligned16(w_masked_bf16)) return SSCONV_ERR_ALIGNMENT;
   return ssconv::launch_decompress(*desc, w_comp, meta, w_masked_bf16, pattern_out, (cudaStream_t)stream) ==
                  cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_maxpool(const void* x, void* y, int32_t N, int32_t H, int32_t W, int32_t C, int32_t k, int32_t stride,
+                       int32_t pad, void* stream) {
+  if (!x || !y) return SSCONV_ERR_NULL;
+  if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || k <= 0 || stride <= 0 || pad < 0) return SSCONV_ERR_BAD_DESC;
+  if (2 * pad >= 2 * k || H + 2 * pad < k || W + 2 * pad < k) return SSCONV_ERR_BAD_DESC;  // every window meets the image
+  if (C % 8 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned16(x) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  if ((long long)N * H * W * C > 0x7FFFFFFFFFLL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  return ssconv::launch_maxpool(x, y, N, H, W, C, k, stride, pad, (cudaStream_t)stream) == cudaSuccess
              ? SSCONV_OK
              : SSCONV_ERR_CUDA;
 }

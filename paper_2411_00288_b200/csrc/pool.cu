@@ -1,0 +1,66 @@
+// Max-pooling over NHWC bf16 activations: the pooling step between the stem and the first block of
+// a ResNet-shaped stack.  Purely HBM-bound: every input element is read once (neighbouring windows
+// overlap in L1/L2), every output element written once.  One thread per 8 channels (16 bytes) of
+// one output pixel; consecutive threads take consecutive channel groups, so a warp reads and writes
+// whole 128-byte lines whenever C >= 64.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "layout.cuh"
+#include "ssconv.h"
+
+namespace ssconv {
+
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+  __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&a);
+  __nv_bfloat162 y = *reinterpret_cast<__nv_bfloat162*>(&b);
+  __nv_bfloat162 m = __hmax2(x, y);
+  return *reinterpret_cast<uint32_t*>(&m);
+}
+
+__global__ void __launch_bounds__(256) maxpool_nhwc_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int N,
+                                                           int H, int W, int C8, int Ho, int Wo, int k, int stride,
+                                                           int pad) {
+  const long long total = (long long)N * Ho * Wo * C8;
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int c = (int)(i % C8);
+  long long pix = i / C8;
+  const int wo = (int)(pix % Wo);
+  pix /= Wo;
+  const int ho = (int)(pix % Ho);
+  const int n = (int)(pix / Ho);
+  const uint32_t neg_inf2 = 0xFF80FF80u;  // bf16 -inf twice: padding never wins
+  uint4 m = make_uint4(neg_inf2, neg_inf2, neg_inf2, neg_inf2);
+  for (int kh = 0; kh < k; ++kh) {
+    const int h = ho * stride - pad + kh;
+    if (h < 0 || h >= H) continue;
+    for (int kw = 0; kw < k; ++kw) {
+      const int w = wo * stride - pad + kw;
+      if (w < 0 || w >= W) continue;
+      const uint4 v = __ldg(x + ((long long)(n * H + h) * W + w) * C8 + c);
+      m.x = max_bf16x2(m.x, v.x);
+      m.y = max_bf16x2(m.y, v.y);
+      m.z = max_bf16x2(m.z, v.z);
+      m.w = max_bf16x2(m.w, v.w);
+    }
+  }
+  y[i] = m;
+}
+
+cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad,
+                           cudaStream_t st) {
+  const int Ho = (H + 2 * pad - k) / stride + 1, Wo = (W + 2 * pad - k) / stride + 1;
+  const long long total = (long long)N * Ho * Wo * (C / 8);
+  if (total == 0) return cudaSuccess;
+  const int T = 256;
+  count_launch();
+  maxpool_nhwc_kernel<<<(unsigned)((total + T - 1) / T), T, 0, st>>>(static_cast<const uint4*>(x),
+                                                                     static_cast<uint4*>(y), N, H, W, C / 8, Ho, Wo,
+                                                                     k, stride, pad);
+  return cudaGetLastError();
+}
+
+}  // namespace ssconv

@@ -2,8 +2,8 @@
 
 Only marshalling: weights are masked and compressed once with the library's own calls, output
 buffers are allocated once, and forward() issues one C-ABI call per convolution on the current
-stream (so it can be recorded into a CUDA graph).  The 3x3 stride-2 max-pool between the stem and
-the first block is not part of the library; it runs as a torch op on the same stream.
+stream (so it can be recorded into a CUDA graph); the 3x3 stride-2 max-pool between the stem and
+the first block is the library's ssconv_maxpool.
 """
 from __future__ import annotations
 
@@ -54,8 +54,7 @@ class ConvStack:
             src = x if st.src < 0 else self.outputs[st.src]
             y = self.outputs[i]
             if st.kind == "maxpool":
-                pooled = torch.nn.functional.max_pool2d(src.permute(0, 3, 1, 2), 3, 2, 1)
-                y.copy_(pooled.permute(0, 2, 3, 1))
+                api.ssconv_maxpool(src, 3, 2, 1, y=y)
             else:
                 L = self.layers[i]
                 if st.kind == "conv" and sparse:
