@@ -83,6 +83,7 @@ struct FwdParams {
   int pieces;               // epilogue pieces per group: ceil(BN / 2 / kPiece)
   int tail_cols;            // positions in a group's last piece (a multiple of 8, at most kPiece)
   int ring_groups;          // groups in the shared-memory ring
+  int small_c;              // dense layers with C_in == 8: a k-block is 8 filter taps (see producer_role)
   int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
   int taps, cblocks, kblocks;
   int m_tiles, num_tiles;
@@ -266,7 +267,38 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
       const uint32_t full = full0 + 8u * g;
       const uint32_t dst = ring0 + g * grp_bytes;
       const bool has_second = 2 * a + 1 < p.kblocks;
-      if (ROLE == kRoleWeights) {
+      if (!SPARSE && p.small_c) {
+        // 8 input channels (16 bytes per pixel): a k-block is 8 filter taps, held in shared memory as
+        // 8 unswizzled chunks, each 16 bytes wide (chunk after chunk, rows every 16 bytes).
+        // One load per tap and operand (im2col for the activations, a 8 x 1 x 128 box for the
+        // weights; a single box over 8 taps was measured slower).  MMAs take chunks in pairs, so an
+        // odd tail is padded with a tap beyond the filter, whose channel coordinate lies outside
+        // the tensor: TMA fills zeros on both operands.
+        const int first_tap = 16 * a + (ROLE == kRoleActSecond ? 8 : 0);
+        int left_taps = p.taps - first_tap;
+        const int most = (ROLE == kRoleWeights) ? 16 : 8;
+        left_taps = left_taps < 0 ? 0 : (left_taps > most ? most : left_taps);
+        const int chunks = (left_taps + 1) & ~1;
+        it.init(first_tap, p);  // counted in taps here
+        if (chunks == 0) {
+          mbar_arrive_a(full);
+        } else if (ROLE == kRoleWeights) {
+          mbar_expect_tx_a(full, (uint32_t)chunks * 2048u);
+          for (int j = 0; j < chunks; ++j) {  // chunks 8.. belong to the second k-block: 16 KB further on = 8 x 2048
+            tma_load_3d_a(dst + (uint32_t)j * 2048u, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+            it.advance(p);
+          }
+        } else {
+          const uint32_t chunk_bytes = (uint32_t)p.BN * 16u;
+          mbar_expect_tx_a(full, (uint32_t)chunks * chunk_bytes);
+          const uint32_t b_dst = dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? b_bytes : 0u);
+          for (int j = 0; j < chunks; ++j) {
+            tma_load_im2col_4d_a(b_dst + (uint32_t)j * chunk_bytes, tm_b, full, it.cc * kBlockK, base_w, base_h,
+                                 q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
+            it.advance(p);
+          }
+        }
+      } else if (ROLE == kRoleWeights) {
         if (SPARSE) {
           mbar_expect_tx_a(full, C::kAGroupBytes);
           tma_load_2d_a(dst, tm_a, full, a * 64, m * kTileM);
@@ -426,6 +458,22 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
               if (n0 > 1) tc_mma_sparse_lo(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
               if (n1 > 0) tc_mma_sparse_lo(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
               if (n1 > 1) tc_mma_sparse_lo(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
+            }
+          } else if (p.small_c) {
+            // chunked operands (see producer_role): chunk stride 2048 B for the weights, 16 BN for the
+            // activations; an MMA takes two chunks (K = 16) of each
+            const uint32_t a_ns = (a_lo & 0xFFFFu) | (128u << 16);
+            const uint32_t b_ns = (b0_lo & 0xFFFFu) | ((uint32_t)p.BN << 16);
+#pragma unroll 1
+            for (int kb = 0; kb < 2; ++kb) {
+              int left_taps = p.taps - (16 * a + 8 * kb);
+              left_taps = left_taps < 0 ? 0 : (left_taps > 8 ? 8 : left_taps);
+              const int n_mma = (left_taps + 1) >> 1;
+              for (int i = 0; i < n_mma; ++i) {
+                tc_mma_dense_chunked(d_tmem, a_ns + (uint32_t)kb * (kATileBytes >> 4) + (uint32_t)i * 256u,
+                                     b_ns + (uint32_t)kb * b_desc + (uint32_t)i * (uint32_t)(2 * p.BN), idesc, accumulate);
+                accumulate = 1;
+              }
             }
           } else {
             const uint32_t a1_lo = a_lo + (kATileBytes >> 4);
@@ -776,6 +824,19 @@ size_t workspace_bytes() { return scratch_bytes(kMaxWorkers); }
 static int g_sm_count[64] = {0};
 static bool g_attr_set[64][2] = {{false}};
 
+// Dense layers with 8 input channels (a channel-padded RGB stem): a k-block of 64 K-elements is 8
+// filter taps instead of 64 channels of one tap, which would be 7/8 padding.
+static bool small_channel_mode(const ssconv_desc_t& d, bool sparse) { return !sparse && d.C_in == 8; }
+static Geometry layer_geometry(const ssconv_desc_t& d, bool sparse) {
+  Geometry g = make_geometry(d);
+  if (small_channel_mode(d, sparse)) {
+    g.kblocks = (g.taps + 7) / 8;
+    g.kblocks_pad = (g.kblocks + 1) & ~1;
+    g.stages = g.kblocks_pad / 2;
+  }
+  return g;
+}
+
 // Current device and its SM count (checked once per device: must be compute capability 10.x).
 static int32_t current_device(int* dev_out) {
   int dev = 0;
@@ -804,7 +865,7 @@ int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* sp
   int dev = 0;
   const int32_t st = current_device(&dev);
   if (st != SSCONV_OK) return st;
-  const Geometry geo = make_geometry(d);
+  const Geometry geo = layer_geometry(d, sparse);
   const long long Q = (long long)d.N * out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h) *
                       out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
   const int workers = g_sm_count[dev] < kMaxWorkers ? g_sm_count[dev] : kMaxWorkers;
@@ -837,7 +898,8 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
       return SSCONV_ERR_CUDA;
     g_attr_set[dev][SPARSE ? 1 : 0] = true;
   }
-  const Geometry geo = make_geometry(d);
+  const Geometry geo = layer_geometry(d, SPARSE);
+  const bool small_c = small_channel_mode(d, SPARSE);
   const int Ho = out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h);
   const int Wo = out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
   const long long Q = (long long)d.N * Ho * Wo;  // positions
@@ -861,10 +923,12 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     int lower[2] = {-d.pad_w, -d.pad_h};
     int upper[2] = {d.pad_w - (d.KW - 1) * d.dil_w, d.pad_h - (d.KH - 1) * d.dil_h};
     cuuint32_t estr[4] = {1, (cuuint32_t)d.stride_w, (cuuint32_t)d.stride_h, 1};
+    // (8-channel mode: 16-byte-wide unswizzled chunks, one per filter tap)
     CUresult r = g_encode_im2col(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), dims, strides,
-                                 lower, upper, (cuuint32_t)kBlockK, (cuuint32_t)BN, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                                 lower, upper, small_c ? 8u : (cuuint32_t)kBlockK, (cuuint32_t)BN, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 small_c ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
   }
   if (SPARSE) {
@@ -877,12 +941,15 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
   } else {
+    // dense weights [C_out][taps][C_in] seen as (c, tap, output channel); 8-channel mode: one tap's
+    // 8 channels of 128 rows per load, unswizzled
     cuuint64_t dims[3] = {(cuuint64_t)d.C_in, (cuuint64_t)geo.taps, (cuuint64_t)d.C_out};
     cuuint64_t strides[2] = {(cuuint64_t)d.C_in * 2, (cuuint64_t)geo.taps * d.C_in * 2};
-    cuuint32_t box[3] = {(cuuint32_t)kBlockK, 1, (cuuint32_t)kTileM};
+    cuuint32_t box[3] = {small_c ? 8u : (cuuint32_t)kBlockK, 1, (cuuint32_t)kTileM};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = g_encode_tiled(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(weights), dims, strides,
-                                box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                small_c ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
   }
@@ -914,6 +981,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.pieces = pieces;
   p.tail_cols = tail_cols;
   p.ring_groups = ring_groups;
+  p.small_c = small_c ? 1 : 0;
   p.stride_h = d.stride_h;
   p.stride_w = d.stride_w;
   p.pad_h = d.pad_h;

@@ -376,6 +376,21 @@ __device__ __forceinline__ void tc_mma_dense_lo(uint32_t d_tmem, uint32_t a_lo, 
       ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHiSw128)
       : "memory");
 }
+// Dense MMA on unswizzled K-major operands: 16-byte chunks of 8 K-elements; within a chunk the
+// rows follow each other every 16 bytes (8 rows = one 128-byte core matrix, stride-dimension offset
+// 128), chunks follow each other every `chunk stride` bytes, which goes into bits 16-29 of the low
+// word as the leading-dimension offset: lo = (address >> 4) | ((chunk stride >> 4) << 16).
+__device__ __forceinline__ void tc_mma_dense_chunked(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                                     uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %5};\n\t"
+      "mov.b64 db, {%2, %5};\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHiNoSwizzle128)
+      : "memory");
+}
 __device__ __forceinline__ void tc_mma_sparse_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t meta_tmem,
                                                  uint32_t idesc, uint32_t accumulate) {
   asm volatile(

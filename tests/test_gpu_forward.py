@@ -33,6 +33,10 @@ SWEEP = [
     ("c3_small_channels",       2, 8,  8,  8,   8,  3, 3, 1, 1, 1),
     ("c3_7x7_maps_wrap_images", 9, 7,  7,  128, 256, 3, 3, 1, 1, 1),
     ("pw_deepK",                1, 6,  6,  1024, 64, 1, 1, 1, 0, 1),
+    # 8 input channels: the dense kernel packs 8 filter taps into a k-block (a channel-padded RGB stem)
+    ("stem_7x7_s2_c8",          2, 30, 34, 8,  64,  7, 7, 2, 3, 1),
+    ("pw_c8",                   2, 9,  9,  8,  16,  1, 1, 1, 0, 1),
+    ("c4x4_c8_even_taps",       1, 12, 12, 8,  136, 4, 4, 1, 1, 1),
 ]
 
 
