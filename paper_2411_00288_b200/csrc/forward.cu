@@ -10,28 +10,38 @@
 // wide MMAs amortise the cost of issuing them; narrower tiles are used when 240-wide ones would
 // leave most SMs without work.
 //
-// Positions are the output pixels (n, ho, wo) in row-major order.  Per k-block (64 input channels
-// at one filter tap) one im2col-mode TMA load brings the 240 pixels' channels at that tap,
-// zero-filled outside the image.  (Staging one run of padded input per channel chunk and serving
-// all taps from it through row-shifted descriptors was built and measured: the MMA's operand
-// fetch, about 64 B/clk, bounds the main loop either way, so the simpler scheme stays.)
+// Positions are the output pixels (n, ho, wo) in row-major order.  K is cut into k-blocks of 64
+// input channels at one filter tap; per k-block one im2col-mode TMA load brings the tile's pixels'
+// channels at that tap, zero-filled outside the image.  The shared-memory ring's unit is a group
+// of two k-blocks (see Cfg).  Dense layers with 8 input channels pack 8 taps into a k-block instead
+// (see producer_role).
 //
-// Warp roles: warps 0, 10 and 11 TMA producers (one thread each: activations of even stages, of
-// odd stages, weights), warp 1 MMA issuer (one thread; owns TMEM), warps 2-9 epilogue in two groups of four warps that each own half of a tile's positions.  The accumulator has
-// channels on TMEM lanes and positions on columns, NHWC wants the transpose: the epilogue reads
+// Warp roles: warps 0, 10 and 11 TMA producers (one thread each: the activations of a group's
+// first k-block, of its second, the weights), warp 1 MMA issuer (one thread; owns TMEM), warps 2-9
+// epilogue in two groups of four warps that each own half of a tile's positions.  The accumulator
+// has channels on TMEM lanes and positions on columns, NHWC wants the transpose: the epilogue reads
 // TMEM in the MMA-fragment layout (tcgen05.ld 16x256b), adds the bias, converts pairs to bf16
 // (with ReLU in the conversion), and stmatrix.trans writes 8x8 blocks transposed into a 128-byte
 // swizzled staging buffer [position][channel], which TMA stores write to NHWC asynchronously.
 // That is about 2.5 instructions per thread and element pair; an epilogue of scalar shared-memory
 // stores or lane shuffles is issue-bound at several times that.
 //
-// Work partition: the unit of work is one weight tile's worth of K for one output tile.  Either
-// every CTA takes a contiguous block of whole output tiles, or (when whole tiles would leave many
-// SMs idle) the units are dealt out evenly, so a CTA's range may start and end inside an
-// output tile ("stream-K").  A CTA writes a partly computed tile (fp32) to a scratch region of its
-// own in global memory; a second, small kernel (ssconv_split_finish_kernel) then sums the regions
-// of every split tile in a fixed order on all SMs and applies the same epilogue.  No CTA ever
-// waits for another, and the result does not depend on timing.
+// What paces the main loop (measured): the issuing thread pays about 200 cycles per mbarrier wait,
+// even on a complete barrier, and about 76 per tcgen05 instruction, and the tensor pipe's queue is
+// shallow, so every instruction between MMAs is exposed: hence one handshake per group and nothing
+// else in that loop (365 cycles per k-block).  The other bound is the rate at which an SM takes
+// loads in from L2, about 68 bytes per cycle when all SMs load.  Staging one run of padded input per
+// channel chunk and serving all taps of a 3x3 filter from it through row-shifted descriptors (which
+// would cut the activation loads ninefold) was built and measured before the issue loop was lean,
+// and dropped; it remains the way past the fill bound for large feature maps.
+//
+// Work partition: the unit of work is one group's worth of K for one output tile.  Either every CTA
+// takes a contiguous block of whole output tiles, or (when whole tiles would leave many SMs idle)
+// the units are dealt out evenly, so a CTA's range may start and end inside an output tile
+// ("stream-K").  A CTA writes a partly computed tile (fp32) to a scratch region of its own in
+// global memory; a second, small kernel (ssconv_split_finish_kernel) then sums the regions of
+// every split tile in a fixed order on all SMs and applies the same epilogue.  No CTA ever waits
+// for another, and the result does not depend on timing.
 // All mbarrier waits are bounded; when one runs out the CTA raises a flag, every role leaves
 // its loop, TMEM is freed and SSCONV_ERR_TIMEOUT is stored to *dev_status.
 #include <cuda.h>
