@@ -176,9 +176,9 @@ def reference_arm(args):
 # the finishing kernel of the one split layer), dram__bytes_read.sum + dram__bytes_write.sum from an
 # ncu capture of this workload (summary and command: profiles/bench_resnet18_sweep_dram_traffic.md).
 # It belongs to the kernel sources with the digest below; with other sources the bench reports null.
-TRAFFIC_BYTES_PER_STEP = 72.97e6
+TRAFFIC_BYTES_PER_STEP = 72.81e6
 TRAFFIC_SOURCES = ("forward.cu", "sm100_ptx.cuh", "layout.cuh")
-TRAFFIC_SOURCES_SHA256 = "85521aa19fcd9c00238220c1dd6d674ed3fa262ce6a3edae3dd7678e3251d798"
+TRAFFIC_SOURCES_SHA256 = "e935a88a8d1e7479fc92b564c590c56b81c2a40194c7d6c6208ac7a26e9ab107"
 
 
 def measured_traffic():

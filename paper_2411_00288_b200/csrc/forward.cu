@@ -108,7 +108,8 @@ struct FwdParams {
   int32_t* dev_status;
 };
 
-// Weight-tile range [a0, a1) of one output tile: what a CTA computes in one accumulator pass.
+// Range [a0, a1) of groups (pairs of k-blocks) of one output tile: what a CTA computes in one
+// accumulator pass.
 struct Segment {
   int tile, a0, a1;
 };
