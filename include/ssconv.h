@@ -160,6 +160,20 @@ int32_t ssconv_forward_dense(const ssconv_desc_t* desc, const void* x, const voi
                              const float* bias, void* y, void* ws, size_t ws_bytes,
                              int32_t* dev_status, void* stream);
 
+/* Both forward calls with a residual tensor added before the activation:
+ *   y = act(bias + conv(x, .) + residual),   residual: bf16 NHWC, the shape of y,
+ * the sum taken in fp32 and rounded once.  This is the last convolution of a ResNet bottleneck
+ * fused with the block's skip connection (the architectures of Sec. 4); the paper's method itself
+ * has no such step.  residual may be y's own buffer only if nothing else reads y concurrently (each
+ * element is read before it is written, by the same thread block).  Otherwise as the calls above;
+ * residual: device, 16-byte aligned, not NULL. */
+int32_t ssconv_forward_res(const ssconv_desc_t* desc, const void* x, const void* w_comp,
+                           const void* meta, const float* bias, const void* residual, void* y,
+                           void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+int32_t ssconv_forward_dense_res(const ssconv_desc_t* desc, const void* x, const void* w_bf16,
+                                 const float* bias, const void* residual, void* y, void* ws,
+                                 size_t ws_bytes, int32_t* dev_status, void* stream);
+
 /* ssconv_forward for callers that have no way to provide scratch memory.  (The paper has no
  * counterpart to this call; it exists for integration only.)
  *

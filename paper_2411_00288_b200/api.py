@@ -24,7 +24,8 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.
 EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes",
            "ssconv_plan",
            "ssconv_select_mask",
-           "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_forward", "ssconv_forward_dense",
+           "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_forward", "ssconv_forward_res",
+           "ssconv_forward_dense_res", "ssconv_forward_dense",
            "ssconv_forward_static_ws")
 
 
@@ -216,31 +217,54 @@ def _alloc_y(desc: Desc, x: torch.Tensor) -> torch.Tensor:
 def ssconv_forward(desc: Desc, x: torch.Tensor, w_comp: torch.Tensor, meta: torch.Tensor,
                    bias: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None,
                    ws: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
-                   stream=None) -> torch.Tensor:
-    """2:4 masked convolution forward; returns y bf16 [N,H_out,W_out,C_out] (enqueued, not synchronised)."""
-    _need_cuda(x, w_comp, meta, bias, y, ws, dev_status)
+                   stream=None, residual: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """2:4 masked convolution forward; returns y bf16 [N,H_out,W_out,C_out] (enqueued, not synchronised).
+    With `residual` (bf16, the shape of y) the call is ssconv_forward_res: y = act(bias + conv + residual)."""
+    _need_cuda(x, w_comp, meta, bias, y, ws, dev_status, residual)
     if y is None:
         y = _alloc_y(desc, x)
     if ws is None:
         ws = default_workspace(x.device)
-    _check("ssconv_forward", lib().ssconv_forward(
-        ctypes.byref(desc), _ptr(x), _ptr(w_comp), _ptr(meta), _ptr(bias), _ptr(y), _ptr(ws),
-        0 if ws is None else ws.numel() * ws.element_size(), _ptr(dev_status), _stream(stream)))
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    if residual is None:
+        _check("ssconv_forward", lib().ssconv_forward(
+            ctypes.byref(desc), _ptr(x), _ptr(w_comp), _ptr(meta), _ptr(bias), _ptr(y), _ptr(ws), ws_bytes,
+            _ptr(dev_status), _stream(stream)))
+    else:
+        assert residual.shape == y.shape and residual.dtype == torch.bfloat16 and residual.is_contiguous()
+        f = lib().ssconv_forward_res
+        f.restype = ctypes.c_int32
+        f.argtypes = [ctypes.POINTER(Desc)] + [ctypes.c_void_p] * 7 + [ctypes.c_size_t, ctypes.c_void_p,
+                                                                     ctypes.c_void_p]
+        _check("ssconv_forward_res", f(ctypes.byref(desc), _ptr(x), _ptr(w_comp), _ptr(meta), _ptr(bias),
+                                       _ptr(residual), _ptr(y), _ptr(ws), ws_bytes, _ptr(dev_status),
+                                       _stream(stream)))
     return y
 
 
 def ssconv_forward_dense(desc: Desc, x: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor] = None,
                          y: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None,
-                         dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-    """Dense counterpart with bf16 weights [C_out,KH,KW,C_in]."""
-    _need_cuda(x, w, bias, y, ws, dev_status)
+                         dev_status: Optional[torch.Tensor] = None, stream=None,
+                         residual: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Dense counterpart with bf16 weights [C_out,KH,KW,C_in]; `residual` as in ssconv_forward."""
+    _need_cuda(x, w, bias, y, ws, dev_status, residual)
     if y is None:
         y = _alloc_y(desc, x)
     if ws is None:
         ws = default_workspace(x.device)
-    _check("ssconv_forward_dense", lib().ssconv_forward_dense(
-        ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _ptr(ws),
-        0 if ws is None else ws.numel() * ws.element_size(), _ptr(dev_status), _stream(stream)))
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    if residual is None:
+        _check("ssconv_forward_dense", lib().ssconv_forward_dense(
+            ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _ptr(ws), ws_bytes, _ptr(dev_status),
+            _stream(stream)))
+    else:
+        assert residual.shape == y.shape and residual.dtype == torch.bfloat16 and residual.is_contiguous()
+        f = lib().ssconv_forward_dense_res
+        f.restype = ctypes.c_int32
+        f.argtypes = [ctypes.POINTER(Desc)] + [ctypes.c_void_p] * 6 + [ctypes.c_size_t, ctypes.c_void_p,
+                                                                     ctypes.c_void_p]
+        _check("ssconv_forward_dense_res", f(ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(residual),
+                                             _ptr(y), _ptr(ws), ws_bytes, _ptr(dev_status), _stream(stream)))
     return y
 
 

@@ -12,10 +12,11 @@ cudaError_t launch_compress(const ssconv_desc_t& d, const void* w, const uint8_t
 cudaError_t launch_decompress(const ssconv_desc_t& d, const void* w_comp, const void* meta, void* w_out,
                               uint8_t* pattern_out, cudaStream_t st);
 int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
-                              const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
-                              cudaStream_t stream);
-int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias, void* y,
-                             void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream);
+                              const float* bias, const void* residual, void* y, void* ws, size_t ws_bytes,
+                              int32_t* dev_status, cudaStream_t stream);
+int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias,
+                             const void* residual, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
+                             cudaStream_t stream);
 size_t workspace_bytes();
 cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad,
                            cudaStream_t st);
@@ -176,9 +177,23 @@ int32_t ssconv_forward(const ssconv_desc_t* desc, const void* x, const void* w_c
   if (!x || !w_comp || !meta || !y) return SSCONV_ERR_NULL;
   if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
   if (!aligned16(x) || !aligned16(w_comp) || !aligned16(meta) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
-  return ssconv::launch_forward_sparse(*desc, x, w_comp, meta, bias, y, ws, ws_bytes, dev_status,
+  return ssconv::launch_forward_sparse(*desc, x, w_comp, meta, bias, nullptr, y, ws, ws_bytes, dev_status,
                                        (cudaStream_t)stream);
 }
+
+int32_t ssconv_forward_res(const ssconv_desc_t* desc, const void* x, const void* w_comp, const void* meta,
+                           const float* bias, const void* residual, void* y, void* ws, size_t ws_bytes,
+                           int32_t* dev_status, void* stream) {
+  int32_t rc = check_desc(desc, true);
+  if (rc != SSCONV_OK) return rc;
+  if (!x || !w_comp || !meta || !y || !residual) return SSCONV_ERR_NULL;
+  if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
+  if (!aligned16(x) || !aligned16(w_comp) || !aligned16(meta) || !aligned16(y) || !aligned16(residual))
+    return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_forward_sparse(*desc, x, w_comp, meta, bias, residual, y, ws, ws_bytes, dev_status,
+                                       (cudaStream_t)stream);
+}
+
 
 int32_t ssconv_forward_dense(const ssconv_desc_t* desc, const void* x, const void* w_bf16, const float* bias,
                              void* y, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
@@ -187,7 +202,20 @@ int32_t ssconv_forward_dense(const ssconv_desc_t* desc, const void* x, const voi
   if (!x || !w_bf16 || !y) return SSCONV_ERR_NULL;
   if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
   if (!aligned16(x) || !aligned16(w_bf16) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
-  return ssconv::launch_forward_dense(*desc, x, w_bf16, bias, y, ws, ws_bytes, dev_status, (cudaStream_t)stream);
+  return ssconv::launch_forward_dense(*desc, x, w_bf16, bias, nullptr, y, ws, ws_bytes, dev_status,
+                                      (cudaStream_t)stream);
+}
+
+int32_t ssconv_forward_dense_res(const ssconv_desc_t* desc, const void* x, const void* w_bf16, const float* bias,
+                                 const void* residual, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
+                                 void* stream) {
+  int32_t rc = check_desc(desc, true);
+  if (rc != SSCONV_OK) return rc;
+  if (!x || !w_bf16 || !y || !residual) return SSCONV_ERR_NULL;
+  if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
+  if (!aligned16(x) || !aligned16(w_bf16) || !aligned16(y) || !aligned16(residual)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_forward_dense(*desc, x, w_bf16, bias, residual, y, ws, ws_bytes, dev_status,
+                                      (cudaStream_t)stream);
 }
 
 int32_t ssconv_forward_static_ws(const ssconv_desc_t* desc, const void* x, const void* w_comp, const void* meta,

@@ -93,6 +93,7 @@ struct FwdParams {
   int pieces;               // epilogue pieces per group: ceil(BN / 2 / kPiece)
   int tail_cols;            // positions in a group's last piece (a multiple of 8, at most kPiece)
   int ring_groups;          // groups in the shared-memory ring
+  int has_res;              // a residual tensor is added before the activation (see stage_piece)
   int small_c;              // dense layers with C_in == 8: a k-block is 8 filter taps (see producer_role)
   int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
   int taps, cblocks, kblocks;
@@ -187,15 +188,25 @@ __device__ __forceinline__ void tc_ld_piece(uint32_t taddr, uint32_t (&r)[kPiece
 }
 // bias, activation and bf16 for one piece, written transposed to its staging buffer.  st_addr is
 // this thread's address for the first 8 positions; each further 8 positions are 1024 bytes on.
-template <bool RELU>
+// With RES the staging buffer already holds the residual tile (bf16, same layout): it is read back
+// in fragment layout (ldmatrix.trans, the inverse of the store), added in fp32 before the one
+// rounding, and overwritten in place (a warp only touches its own 16-byte columns).
+template <bool RELU, bool RES>
 __device__ __forceinline__ void stage_piece(const uint32_t (&r)[kPiece], const float (&bias)[4], uint32_t st_addr) {
 #pragma unroll
   for (int k = 0; k < kPiece / 8; ++k) {
     uint32_t w[4];
+    uint32_t res[4] = {0u, 0u, 0u, 0u};
+    if (RES) ldmatrix_x4_trans(st_addr + 1024u * k, res);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {  // channel block i = 2 h + s of the warp's 32 channels
       const int at = 20 * (i >> 1) + 4 * k + 2 * (i & 1);
-      w[i] = pack_bf16x2<RELU>(__uint_as_float(r[at]) + bias[i], __uint_as_float(r[at + 1]) + bias[i]);
+      float lo = __uint_as_float(r[at]) + bias[i], hi = __uint_as_float(r[at + 1]) + bias[i];
+      if (RES) {
+        lo += bf16_lo(res[i]);
+        hi += bf16_hi(res[i]);
+      }
+      w[i] = pack_bf16x2<RELU>(lo, hi);
     }
     stmatrix_x4_trans(st_addr + 1024u * k, w[0], w[1], w[2], w[3]);
   }
@@ -343,6 +354,7 @@ template <bool SPARSE>
 __global__ void __launch_bounds__(kThreads, 1)
 ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                   const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_y_tail,
+                  const __grid_constant__ CUtensorMap tm_r, const __grid_constant__ CUtensorMap tm_r_tail,
                   const FwdParams p) {
   using C = Cfg<SPARSE>;
 
@@ -350,13 +362,15 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* ring = smem;                                                    // ring_groups groups
   uint8_t* out_stage = ring + p.ring_groups * group_bytes(C::kAGroupBytes, p.BN);  // per epilogue group two buffers
-  // barrier slots: [0,4) group full, [4,8) group empty, [8,10) accumulator full, [10,12) accumulator empty
+  // barrier slots: [0,4) group full, [4,8) group empty, [8,10) accumulator full, [10,12) accumulator empty,
+  // [12,16) residual piece landed (per epilogue group and staging buffer)
   uint64_t* bars = reinterpret_cast<uint64_t*>(out_stage + kStagingBytes);
   uint64_t* bar_full = bars;
   uint64_t* bar_empty = bars + 4;
   uint64_t* bar_acc_full = bars + 8;
   uint64_t* bar_acc_empty = bars + 10;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
+  uint64_t* bar_res = bars + 12;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = abort_flag + 1;         // per group two slots: the leader's go/stop verdict per tile
 
@@ -368,9 +382,9 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   if (warp == 0) {
     // barrier slots in memory order: 4 group full (3 arrivals: the three producers), 4 group empty (one
     // commit by the MMA thread), 2 accumulator full, 2 accumulator empty (one arrival per epilogue
-    // warp); lane i initialises slot i
-    if (lane < 12) {
-      const uint32_t count = (lane < 4) ? 3u : (lane < 10) ? 1u : (uint32_t)(4 * kGroups);
+    // warp), 4 residual (one arrival with bytes); lane i initialises slot i
+    if (lane < 16) {
+      const uint32_t count = (lane < 4) ? 3u : (lane < 10) ? 1u : (lane < 12) ? (uint32_t)(4 * kGroups) : 1u;
       mbar_init(&bars[lane], count);
     }
     if (lane == 0) {
@@ -395,6 +409,10 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       if (warp == 2) {
         prefetch_tensormap(&tm_y);
         prefetch_tensormap(&tm_y_tail);
+        if (p.has_res) {
+          prefetch_tensormap(&tm_r);
+          prefetch_tensormap(&tm_r_tail);
+        }
       }
     }
     tc_fence_before();
@@ -580,6 +598,29 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         const int co = m * kTileM + q * 32 + 8 * i + (lane >> 2);
         bias_v[i] = ((p.flags & SSCONV_FLAG_BIAS) && co < p.C_out) ? p.bias[co] : 0.0f;
       }
+      // Residual pieces are brought into the staging buffers by TMA, one piece ahead: the leader
+      // issues the load of piece i + 1 once the store that last read that buffer has finished.
+      auto load_residual = [&](int pp, uint32_t count) {  // leader only; count = running piece number
+        const uint32_t b = count & 1u;
+        const uint32_t bar = smem_u32(&bar_res[2 * grp + b]);
+        const int q_piece = pt * p.BN + col_base + pp * kPiece;
+        if (q_piece >= p.Q) {  // nothing of this piece is stored: only keep the barrier's phases in step
+          mbar_arrive_a(bar);
+          return;
+        }
+        const bool tail = (pp == p.pieces - 1 && p.tail_cols != kPiece);
+        const CUtensorMap* map = tail ? &tm_r_tail : &tm_r;
+        const uint32_t half_bytes = (uint32_t)(tail ? p.tail_cols : kPiece) * 128u;
+        const bool two = m * kTileM + 64 < p.C_out;
+        const uint32_t dst = smem_u32(my_stage + b * kPieceBytes);
+        mbar_expect_tx_a(bar, two ? 2u * half_bytes : half_bytes);
+        tma_load_2d_a(dst, map, bar, m * kTileM, q_piece);
+        if (two) tma_load_2d_a(dst + kHalfPieceBytes, map, bar, m * kTileM + 64, q_piece);
+      };
+      if (p.has_res && leader) {
+        bulk_wait_group_read1();  // the store of two pieces ago has finished reading this buffer
+        load_residual(0, piece_count);
+      }
 #pragma unroll 1
       for (int piece = 0; piece < p.pieces; ++piece, ++piece_count) {
         uint8_t* stage = my_stage + (piece_count & 1u) * kPieceBytes;
@@ -596,10 +637,20 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         // The buffer was last the source of the store issued two pieces ago; the leader saw that
         // store finish reading before it entered the barrier of the previous piece.
         const uint32_t st_addr = smem_u32(stage) + st_offset;
-        if (relu)
-          stage_piece<true>(r, bias_v, st_addr);
-        else
-          stage_piece<false>(r, bias_v, st_addr);
+        if (p.has_res) {
+          // the residual piece has landed in this buffer (a wait that runs out raises the abort flag;
+          // the group still goes on to its barrier and stops at the next tile)
+          mbar_wait_bounded(&bar_res[2 * grp + (piece_count & 1u)], (piece_count >> 1) & 1u, abort_flag,
+                            kWaitLimitCycles);
+          if (relu)
+            stage_piece<true, true>(r, bias_v, st_addr);
+          else
+            stage_piece<false, true>(r, bias_v, st_addr);
+        } else if (relu) {
+          stage_piece<true, false>(r, bias_v, st_addr);
+        } else {
+          stage_piece<false, false>(r, bias_v, st_addr);
+        }
         fence_proxy_async_smem();           // generic-proxy writes -> visible to the TMA store
         if (leader) bulk_wait_group_read0();  // the previous piece's store no longer reads its buffer
         epilogue_bar_sync(grp);
@@ -613,6 +664,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             if (m * kTileM + 64 < p.C_out) tma_store_2d(map, stage + kHalfPieceBytes, m * kTileM + 64, q_piece);
           }
           bulk_commit_group();
+          if (p.has_res && piece + 1 < p.pieces) load_residual(piece + 1, piece_count + 1);
         }
       }
     }
@@ -651,6 +703,7 @@ struct FinishParams {
   const float4* ws_regions;
   uint32_t flags;
   const float* bias;
+  const __nv_bfloat16* residual;  // nullable
   __nv_bfloat16* y;
 };
 constexpr int kFinishThreads = 128;
@@ -704,6 +757,25 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
     const int co = m * kTileM + q * 32 + 8 * i + (lane >> 2);
     bias_v[i] = ((f.flags & SSCONV_FLAG_BIAS) && co < f.C_out) ? f.bias[co] : 0.0f;
   }
+  // thread 8 i + j of a warp addresses position j of channel block i of the warp's four
+  const uint32_t row = (uint32_t)(lane & 7);
+  const uint32_t chunk = (uint32_t)(4 * q + (lane >> 3));
+  const uint32_t st_addr = smem_u32(stage) + row * 256u + ((chunk ^ row) << 4);
+  const int pos = gtid >> 4, ch16 = gtid & 15;  // 16 threads cover the 256 contiguous bytes of one position
+  const int q_pos = pt * kBN + grp * kGroupCols + piece * kPiece + 8 * k + pos;
+  const int co16 = m * kTileM + 8 * ch16;
+  const bool in_range = q_pos < f.Q && co16 < f.C_out;
+  if (f.residual != nullptr) {
+    // residual block -> staging buffer (same layout), read back in fragment layout, added in fp32
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (in_range) v = *reinterpret_cast<const uint4*>(f.residual + (size_t)q_pos * f.C_out + co16);
+    *reinterpret_cast<uint4*>(stage + pos * 256 + ((ch16 ^ pos) << 4)) = v;
+    __syncthreads();
+    uint32_t res[4];
+    ldmatrix_x4_trans(st_addr, res);
+    acc0.x += bf16_lo(res[0]); acc0.y += bf16_hi(res[0]); acc0.z += bf16_lo(res[1]); acc0.w += bf16_hi(res[1]);
+    acc1.x += bf16_lo(res[2]); acc1.y += bf16_hi(res[2]); acc1.z += bf16_lo(res[3]); acc1.w += bf16_hi(res[3]);
+  }
   uint32_t w[4];
   if (f.flags & SSCONV_FLAG_RELU) {
     w[0] = pack_bf16x2<true>(acc0.x + bias_v[0], acc0.y + bias_v[0]);
@@ -716,19 +788,11 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
     w[2] = pack_bf16x2<false>(acc1.x + bias_v[2], acc1.y + bias_v[2]);
     w[3] = pack_bf16x2<false>(acc1.z + bias_v[3], acc1.w + bias_v[3]);
   }
-  // thread 8 i + j of a warp addresses position j of channel block i of the warp's four
-  const uint32_t row = (uint32_t)(lane & 7);
-  const uint32_t chunk = (uint32_t)(4 * q + (lane >> 3));
-  stmatrix_x4_trans(smem_u32(stage) + row * 256u + ((chunk ^ row) << 4), w[0], w[1], w[2], w[3]);
+  stmatrix_x4_trans(st_addr, w[0], w[1], w[2], w[3]);
   __syncthreads();
-  {
-    const int pos = gtid >> 4, ch16 = gtid & 15;  // 16 threads write the 256 contiguous bytes of one position
-    const int q_pos = pt * kBN + grp * kGroupCols + piece * kPiece + 8 * k + pos;
-    const int co = m * kTileM + 8 * ch16;
-    if (q_pos < f.Q && co < f.C_out) {
-      const uint4 v = *reinterpret_cast<const uint4*>(stage + pos * 256 + ((ch16 ^ pos) << 4));
-      *reinterpret_cast<uint4*>(f.y + (size_t)q_pos * f.C_out + co) = v;
-    }
+  if (in_range) {
+    const uint4 v = *reinterpret_cast<const uint4*>(stage + pos * 256 + ((ch16 ^ pos) << 4));
+    *reinterpret_cast<uint4*>(f.y + (size_t)q_pos * f.C_out + co16) = v;
   }
 }
 
@@ -894,8 +958,9 @@ int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* sp
 
 template <bool SPARSE>
 static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const void* weights, const void* meta,
-                                   const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
-                                   cudaStream_t stream, int worker_cap = kMaxWorkers, bool force_split = false) {
+                                   const float* bias, const void* residual, void* y, void* ws, size_t ws_bytes,
+                                   int32_t* dev_status, cudaStream_t stream, int worker_cap = kMaxWorkers,
+                                   bool force_split = false) {
   using C = Cfg<SPARSE>;
   if (!load_driver_entry_points()) return SSCONV_ERR_CUDA;
   int dev = 0;
@@ -924,7 +989,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   const int ring_groups = ring_groups_for(C::kAGroupBytes, BN);
   const uint32_t smem_bytes = 1024 + (uint32_t)ring_groups * grp_bytes + kStagingBytes + kBarrierBytes;
 
-  CUtensorMap tm_a, tm_b, tm_y, tm_y_tail;
+  CUtensorMap tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail;
   // activations: NHWC seen as (c, w, h, n), im2col mode; elements outside the image read as zero
   // (= the zero padding of Eq. 4); base pixels are the filter placements, each load adds a tap offset
   {
@@ -980,6 +1045,22 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
+    // the residual tensor, when there is one, is read through the same two views
+    tm_r = tm_y;
+    tm_r_tail = tm_y_tail;
+    if (residual != nullptr) {
+      void* res = const_cast<void*>(residual);
+      box[1] = (cuuint32_t)kPiece;
+      r = g_encode_tiled(&tm_r, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, res, dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
+      box[1] = (cuuint32_t)tail_cols;
+      r = g_encode_tiled(&tm_r_tail, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, res, dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
+    }
   }
 
   FwdParams p;
@@ -993,6 +1074,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.tail_cols = tail_cols;
   p.ring_groups = ring_groups;
   p.small_c = small_c ? 1 : 0;
+  p.has_res = residual != nullptr ? 1 : 0;
   p.stride_h = d.stride_h;
   p.stride_w = d.stride_w;
   p.pad_h = d.pad_h;
@@ -1044,7 +1126,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE>, tm_a, tm_b, tm_y, tm_y_tail, p) != cudaSuccess) return SSCONV_ERR_CUDA;
+  if (cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p) != cudaSuccess) return SSCONV_ERR_CUDA;
   count_launch();
   if (p.split) {
     FinishParams f;
@@ -1057,6 +1139,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     f.ws_regions = p.ws_regions;
     f.flags = d.flags;
     f.bias = bias;
+    f.residual = static_cast<const __nv_bfloat16*>(residual);
     f.y = p.y;
     cfg.gridDim = dim3((unsigned)p.num_tiles * kFinishItemsPerTile);
     cfg.blockDim = dim3((unsigned)kFinishThreads);
@@ -1068,13 +1151,14 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
 }
 
 int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
-                              const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
-                              cudaStream_t stream) {
-  return launch_forward_impl<true>(d, x, w_comp, meta, bias, y, ws, ws_bytes, dev_status, stream);
+                              const float* bias, const void* residual, void* y, void* ws, size_t ws_bytes,
+                              int32_t* dev_status, cudaStream_t stream) {
+  return launch_forward_impl<true>(d, x, w_comp, meta, bias, residual, y, ws, ws_bytes, dev_status, stream);
 }
-int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias, void* y,
-                             void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream) {
-  return launch_forward_impl<false>(d, x, w, nullptr, bias, y, ws, ws_bytes, dev_status, stream);
+int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias,
+                             const void* residual, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
+                             cudaStream_t stream) {
+  return launch_forward_impl<false>(d, x, w, nullptr, bias, residual, y, ws, ws_bytes, dev_status, stream);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -1107,7 +1191,7 @@ int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const vo
   unsigned char* scratch = g_static_scratch_ptr[dev];
   // Nothing in the array has to be cleared: it keeps whatever the previous call left, and every
   // partial-sum region is written by this call's main kernel before its finishing kernel reads it.
-  return launch_forward_impl<true>(d, x, w_comp, meta, bias, y, scratch, scratch_bytes(kStaticWorkers), dev_status,
+  return launch_forward_impl<true>(d, x, w_comp, meta, bias, nullptr, y, scratch, scratch_bytes(kStaticWorkers), dev_status,
                                    stream, kStaticWorkers, true);
 }
 

@@ -141,6 +141,17 @@ __device__ __forceinline__ void stmatrix_x4_trans(uint32_t addr, uint32_t r0, ui
                "r"(r2), "r"(r3)
                : "memory");
 }
+// The inverse: thread t receives in register i elements (row t/4, columns 2(t%4), 2(t%4)+1) of
+// matrix i, read transposed from the 16-byte rows whose addresses threads 8i+j supply.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
+// Low and high bf16 of a packed pair as floats (exact).
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
 // Two floats -> packed bf16 pair (lo in the low half), round to nearest even, optionally max(., 0).
 template <bool RELU>
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {

@@ -1,5 +1,7 @@
 """Helpers shared by the GPU parity tests: run one layer through the CUDA library (via the
 C ABI binding) and through the CPU oracle on the same seeded bits, and compare."""
+import dataclasses
+
 import numpy as np
 import torch
 
@@ -48,7 +50,7 @@ def errors(y_gpu_f64: np.ndarray, y_ref: np.ndarray):
     return rel, float(np.abs(diff).max())
 
 
-def run_layer_gpu(inp, dev, sparse=True, pattern=None):
+def run_layer_gpu(inp, dev, sparse=True, pattern=None, residual=None):
     """Returns (y bf16 on device, dev_status int).  Dense path uses the raw (unmasked) weights
     unless `pattern` is given, in which case it gets the masked weights from decompress."""
     spec = inp.spec
@@ -60,29 +62,48 @@ def run_layer_gpu(inp, dev, sparse=True, pattern=None):
     if sparse:
         pat = gpu_pattern(inp, dev) if pattern is None else pattern
         w_comp, meta = api.ssconv_compress(desc, w, pat)
-        y = api.ssconv_forward(desc, x, w_comp, meta, bias, dev_status=status)
+        y = api.ssconv_forward(desc, x, w_comp, meta, bias, dev_status=status, residual=residual)
     else:
-        y = api.ssconv_forward_dense(desc, x, w, bias, dev_status=status)
+        y = api.ssconv_forward_dense(desc, x, w, bias, dev_status=status, residual=residual)
     torch.cuda.synchronize()
     return y, int(status.item())
 
 
-def check_layer(spec, dev, sparse=True, sample=None, seed=None):
-    """Full (or sampled) parity of one layer against the oracle; returns (rel_fro, max_abs)."""
+def make_residual(spec, seed=None) -> torch.Tensor:
+    """Seeded bf16 tensor of the layer's output shape (its own stream of the layer's seed)."""
+    g = torch.Generator().manual_seed((spec.seed if seed is None else seed) + 90_000_000)
+    return torch.randn((spec.N, spec.H_out, spec.W_out, spec.C_out), generator=g, dtype=torch.float32).to(torch.bfloat16)
+
+
+def check_layer(spec, dev, sparse=True, sample=None, seed=None, residual=False):
+    """Full (or sampled) parity of one layer against the oracle; returns (rel_fro, max_abs).
+    With residual=True the fused call y = act(bias + conv + residual) is checked: the oracle computes
+    the convolution without activation, the test adds the residual and applies the activation in fp64."""
     inp = synth.make_inputs(spec, seed=seed)
-    y, st = run_layer_gpu(inp, dev, sparse=sparse)
+    res = make_residual(spec, seed) if residual else None
+    y, st = run_layer_gpu(inp, dev, sparse=sparse, residual=res.to(dev) if residual else None)
     assert st == 0, f"device status {st}"
     pat = oracle_pattern(inp)
     w_bits = synth.bf16_bits(inp.w)
     mask = masks.mask_from_pattern(pat, w_bits.shape) if sparse else None
     bias = inp.bias.numpy() if inp.bias is not None else None
     shp = oracle_shape(spec)
+    if residual:
+        shp = dataclasses.replace(shp, relu=False)
     yg = bf16_tensor_to_f64(y)
+
+    def finish(ref, idx=None):
+        if not residual:
+            return ref
+        r = bf16_tensor_to_f64(res).reshape(-1)
+        ref = ref + (r.reshape(ref.shape) if idx is None else r[idx])
+        return np.maximum(ref, 0.0) if spec.relu else ref
+
     if sample is None:
-        ref = conv2d_f64(shp, synth.bf16_bits(inp.x), w_bits, mask=mask, bias=bias)
+        ref = finish(conv2d_f64(shp, synth.bf16_bits(inp.x), w_bits, mask=mask, bias=bias))
         assert ref.shape == yg.shape
         return errors(yg, ref)
     rng = np.random.default_rng(spec.seed & 0xFFFFFFFF)
     idx = rng.choice(yg.size, size=min(sample, yg.size), replace=False)
-    ref = conv2d_f64_sample(shp, synth.bf16_bits(inp.x), w_bits, idx, mask=mask, bias=bias)
+    ref = finish(conv2d_f64_sample(shp, synth.bf16_bits(inp.x), w_bits, idx, mask=mask, bias=bias), idx)
     return errors(yg.reshape(-1)[idx], ref)

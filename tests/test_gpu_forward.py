@@ -83,3 +83,44 @@ def test_all_ones_input_closed_form_borders():
         for wo in range(W):
             taps = sum(1 for kh in range(K) for kw in range(K) if 0 <= ho - 1 + kh < H and 0 <= wo - 1 + kw < W)
             assert (y[0, ho, wo, :] == 0.125 * (C // 2) * taps).all()
+
+
+# ---------------------------------------------------------------------------------------------
+# fused residual: y = act(bias + conv + residual)
+RES_CASES = [
+    # name                      N  H   W   Ci   Co  KH KW s  p  d
+    ("res_pw_256to64",          2, 14, 14, 256, 64,  1, 1, 1, 0, 1),
+    ("res_pw_64to256",          3, 9,  11, 64,  256, 1, 1, 1, 0, 1),
+    ("res_c3_ragged_136",       2, 12, 9,  64,  136, 3, 3, 1, 1, 1),
+    ("res_c3_s2",               2, 13, 12, 128, 64,  3, 3, 2, 1, 1),
+    ("res_small_channels",      2, 8,  8,  8,   8,   3, 3, 1, 1, 1),
+]
+
+
+@pytest.mark.parametrize("case", RES_CASES, ids=[c[0] for c in RES_CASES])
+@pytest.mark.parametrize("sparse", [True, False], ids=["sparse", "dense"])
+def test_residual_epilogue(case, sparse):
+    name, N, H, W, Ci, Co, KH, KW, s, p, d = case
+    spec = synth.LayerSpec(name, N, H, W, Ci, Co, KH, KW, s, p, d, relu=(Co != 136), w_std="fan_in",
+                           mask_source="magnitude", config=9, index=60 + RES_CASES.index(case))
+    _assert_ok(*parity.check_layer(spec, DEV, sparse=sparse, residual=True), name)
+
+
+def test_residual_in_place_and_wide_tiles():
+    """A layer wide enough for 240-position tiles and several pieces per group, with the residual
+    read from the output buffer itself (y += conv, as a skip connection updated in place)."""
+    spec = synth.LayerSpec("res_inplace", 1, 188, 188, 64, 64, 3, 3, 1, 1, 1, relu=True, w_std="fan_in",
+                           mask_source="magnitude", config=9, index=70)
+    inp = synth.make_inputs(spec)
+    res = parity.make_residual(spec)
+    desc = api.desc_from_spec(spec)
+    x, w, b = inp.x.to(DEV), inp.w.to(DEV), inp.bias.to(DEV)
+    pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
+    w_comp, meta = api.ssconv_compress(desc, w, pat)
+    y_sep = api.ssconv_forward(desc, x, w_comp, meta, b, residual=res.to(DEV))
+    y_inplace = res.to(DEV).clone()
+    api.ssconv_forward(desc, x, w_comp, meta, b, y=y_inplace, residual=y_inplace)
+    torch.cuda.synchronize()
+    assert torch.equal(y_sep, y_inplace)
+    assert api.ssconv_plan(desc, True)["tile_positions"] == 240
+    _assert_ok(*parity.check_layer(spec, DEV, sparse=True, sample=30000, residual=True), "res_inplace")

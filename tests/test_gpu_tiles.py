@@ -45,6 +45,8 @@ def test_split_plan_deep_k_few_tiles():
         c0 = api.ssconv_launch_count()
         rel, mx = parity.check_layer(spec, DEV, sparse=sparse)
         assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"split {sparse}: rel={rel:.3e} max={mx:.3e}"
+        rel, mx = parity.check_layer(spec, DEV, sparse=sparse, residual=True)  # the finishing kernel adds it
+        assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"split+res {sparse}: rel={rel:.3e} max={mx:.3e}"
         assert api.ssconv_launch_count() - c0 >= 2  # main + finishing kernel (+ select/compress when sparse)
 
 
