@@ -214,7 +214,7 @@ def stack_arm(args):
         dist.barrier()
     api.lib()
     batch = args.batch or 256
-    steps_def = synth.resnet50_stack(batch)
+    steps_def = synth.resnet50_stack(batch, residual=args.residual)
     net = stack.ConvStack(steps_def, dev, with_dense=True)
     g = torch.Generator().manual_seed(synth.SEED_BASE + 577 + rank)
     x = torch.zeros((batch, 224, 224, 8), dtype=torch.bfloat16)
@@ -262,10 +262,12 @@ def stack_arm(args):
             "value": ranks.job_throughput(batch, world, ms_sparse), "unit": "images/s", "n_gpus": world,
             "steps": steps, "warmup": warmup, "ms_per_step": ms_sparse, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "batch_per_gpu": batch,
+            "config": {"workload": WORKLOAD + ("_with_skip_connections" if args.residual else ""),
+                       "batch_per_gpu": batch,
                        "stack": "stem 7x7 s2 (dense, input padded 3 -> 8 channels), 3x3 s2 max-pool, 16 "
                                 "bottlenecks as reduce -> 3x3 -> expand with bias + ReLU, 4 downsample convolutions on "
-                                "their block's input; no residual additions",
+                                "their block's input; " + ("skip connections fused into the expand convolutions"
+                                                            if args.residual else "no residual additions"),
                        "l2": "activations of a step total several GB (> L2)",
                        "launch": "the stack's calls recorded into one CUDA graph and replayed"},
             "dense_equiv_tflops": ranks.job_throughput(flops, world, ms_sparse) / 1e12,
@@ -289,6 +291,8 @@ def main():
     ap.add_argument("--only-layer", type=int, default=None,
                     help="profiling aid: launch just this layer of the sweep --layer-iters times and exit")
     ap.add_argument("--dense", action="store_true", help="with --only-layer: use the dense kernel")
+    ap.add_argument("--residual", action="store_true",
+                    help="with --workload-config 5: fuse the network's skip connections into the expand convolutions")
     ap.add_argument("--batch", type=int, default=None, help="with --workload-config 5: images per GPU (default 256)")
     ap.add_argument("--workload-config", type=int, default=CONFIG_ID, choices=sorted(WORKLOADS),
                     help="layer set to run (default: the benchmarked ResNet-18 sweep)")

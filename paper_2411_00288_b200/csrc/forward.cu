@@ -67,7 +67,7 @@ constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 1.9 GHz
 constexpr uint32_t kATileBytes = 128 * 128;          // 128 rows x 128 B
 constexpr uint32_t kHalfPieceBytes = kPiece * 128;    // 40 positions x 64 channels bf16, 128-byte swizzled
 constexpr uint32_t kPieceBytes = 2 * kHalfPieceBytes; // channels [0,64) then [64,128) of the tile
-constexpr uint32_t kStagingBytes = 2 * kGroups * kPieceBytes;  // two buffers per group
+__host__ __device__ constexpr uint32_t staging_bytes(int bufs) { return (uint32_t)bufs * kGroups * kPieceBytes; }  // per group 2 or 4 buffers
 constexpr uint32_t kBarrierBytes = 256;
 
 // The ring's unit is a group: the operands of one pair of k-blocks (128 dense columns of K).
@@ -94,6 +94,7 @@ struct FwdParams {
   int tail_cols;            // positions in a group's last piece (a multiple of 8, at most kPiece)
   int ring_groups;          // groups in the shared-memory ring
   int has_res;              // a residual tensor is added before the activation (see stage_piece)
+  int stage_bufs;           // staging buffers per epilogue group: 2, or 4 when residual pieces are prefetched
   int small_c;              // dense layers with C_in == 8: a k-block is 8 filter taps (see producer_role)
   int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
   int taps, cblocks, kblocks;
@@ -143,6 +144,26 @@ struct WorkIter {
     left -= s.a1 - s.a0;
     ++tile;
     a0 = 0;
+    return true;
+  }
+};
+
+// Walks the epilogue pieces of this CTA's whole tiles in the order the epilogue meets them, ahead of
+// it: used to prefetch residual pieces.
+struct PieceAhead {
+  WorkIter it;
+  Segment seg;
+  int piece, pieces, a_tiles;
+  bool have;
+  __device__ PieceAhead(const FwdParams& p) : it(p), piece(0), pieces(p.pieces), a_tiles(p.a_tiles), have(false) {}
+  __device__ bool next(int& tile, int& piece_out) {
+    while (!have || piece == pieces) {
+      if (!it.next(seg)) return false;
+      have = (seg.a0 == 0 && seg.a1 == a_tiles);
+      piece = 0;
+    }
+    tile = seg.tile;
+    piece_out = piece++;
     return true;
   }
 };
@@ -363,14 +384,14 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   uint8_t* ring = smem;                                                    // ring_groups groups
   uint8_t* out_stage = ring + p.ring_groups * group_bytes(C::kAGroupBytes, p.BN);  // per epilogue group two buffers
   // barrier slots: [0,4) group full, [4,8) group empty, [8,10) accumulator full, [10,12) accumulator empty,
-  // [12,16) residual piece landed (per epilogue group and staging buffer)
-  uint64_t* bars = reinterpret_cast<uint64_t*>(out_stage + kStagingBytes);
+  // [12,20) residual piece landed (per epilogue group and staging buffer)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_stage + staging_bytes(p.stage_bufs));
   uint64_t* bar_full = bars;
   uint64_t* bar_empty = bars + 4;
   uint64_t* bar_acc_full = bars + 8;
   uint64_t* bar_acc_empty = bars + 10;
   uint64_t* bar_res = bars + 12;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = abort_flag + 1;         // per group two slots: the leader's go/stop verdict per tile
 
@@ -382,8 +403,8 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   if (warp == 0) {
     // barrier slots in memory order: 4 group full (3 arrivals: the three producers), 4 group empty (one
     // commit by the MMA thread), 2 accumulator full, 2 accumulator empty (one arrival per epilogue
-    // warp), 4 residual (one arrival with bytes); lane i initialises slot i
-    if (lane < 16) {
+    // warp), 8 residual (one arrival with bytes); lane i initialises slot i
+    if (lane < 20) {
       const uint32_t count = (lane < 4) ? 3u : (lane < 10) ? 1u : (lane < 12) ? (uint32_t)(4 * kGroups) : 1u;
       mbar_init(&bars[lane], count);
     }
@@ -544,7 +565,9 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     const bool leader = (q == 2 && lane == 0);  // first warp of each group
     const bool relu = (p.flags & SSCONV_FLAG_RELU) != 0;
     const int col_base = grp * (p.BN >> 1);
-    uint8_t* my_stage = out_stage + grp * 2 * kPieceBytes;
+    const uint32_t nbuf = (uint32_t)p.stage_bufs;  // 2 or 4
+    const uint32_t nbuf_shift = nbuf == 4 ? 2u : 1u;
+    uint8_t* my_stage = out_stage + grp * nbuf * kPieceBytes;
     volatile int* my_go = epi_go + 2 * grp;
     // stmatrix duty of this thread: 16 bytes = 8 channels of block (lane / 8) of the warp's four, at
     // position (lane % 8) of each run of 8 positions; the 16-byte chunks of a 128-byte staging row
@@ -554,6 +577,33 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     uint32_t tcount = 0;
     uint32_t piece_count = 0;
     grid_dependency_wait();  // before the first access to global memory (bias, scratch, output)
+    // Residual pieces are brought into the staging buffers by TMA, nbuf - 1 pieces ahead of the
+    // epilogue (they come from HBM: one piece of latency would be exposed on every piece).  The
+    // leader walks the same sequence of pieces with an iterator of its own.
+    PieceAhead ahead(p);
+    auto load_residual = [&](uint32_t count) {  // leader only; count = running number of the piece to load
+      int tile_a, piece_a;
+      if (!ahead.next(tile_a, piece_a)) return;  // no such piece: nobody will wait for it
+      const uint32_t b = count & (nbuf - 1u);
+      const uint32_t bar = smem_u32(&bar_res[4 * grp + b]);
+      const int pt_a = tile_a / p.m_tiles;
+      const int m_a = tile_a - pt_a * p.m_tiles;
+      const int q_piece = pt_a * p.BN + col_base + piece_a * kPiece;
+      if (q_piece >= p.Q) {  // nothing of this piece is stored: only keep the barrier's phases in step
+        mbar_arrive_a(bar);
+        return;
+      }
+      const bool tail = (piece_a == p.pieces - 1 && p.tail_cols != kPiece);
+      const CUtensorMap* map = tail ? &tm_r_tail : &tm_r;
+      const uint32_t half_bytes = (uint32_t)(tail ? p.tail_cols : kPiece) * 128u;
+      const bool two = m_a * kTileM + 64 < p.C_out;
+      const uint32_t dst = smem_u32(my_stage + b * kPieceBytes);
+      mbar_expect_tx_a(bar, two ? 2u * half_bytes : half_bytes);
+      tma_load_2d_a(dst, map, bar, m_a * kTileM, q_piece);
+      if (two) tma_load_2d_a(dst + kHalfPieceBytes, map, bar, m_a * kTileM + 64, q_piece);
+    };
+    if (p.has_res && leader)
+      for (uint32_t c = 0; c + 1 < nbuf; ++c) load_residual(c);
     WorkIter work(p);
     Segment seg;
     for (; work.next(seg); ++tcount) {
@@ -598,32 +648,10 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         const int co = m * kTileM + q * 32 + 8 * i + (lane >> 2);
         bias_v[i] = ((p.flags & SSCONV_FLAG_BIAS) && co < p.C_out) ? p.bias[co] : 0.0f;
       }
-      // Residual pieces are brought into the staging buffers by TMA, one piece ahead: the leader
-      // issues the load of piece i + 1 once the store that last read that buffer has finished.
-      auto load_residual = [&](int pp, uint32_t count) {  // leader only; count = running piece number
-        const uint32_t b = count & 1u;
-        const uint32_t bar = smem_u32(&bar_res[2 * grp + b]);
-        const int q_piece = pt * p.BN + col_base + pp * kPiece;
-        if (q_piece >= p.Q) {  // nothing of this piece is stored: only keep the barrier's phases in step
-          mbar_arrive_a(bar);
-          return;
-        }
-        const bool tail = (pp == p.pieces - 1 && p.tail_cols != kPiece);
-        const CUtensorMap* map = tail ? &tm_r_tail : &tm_r;
-        const uint32_t half_bytes = (uint32_t)(tail ? p.tail_cols : kPiece) * 128u;
-        const bool two = m * kTileM + 64 < p.C_out;
-        const uint32_t dst = smem_u32(my_stage + b * kPieceBytes);
-        mbar_expect_tx_a(bar, two ? 2u * half_bytes : half_bytes);
-        tma_load_2d_a(dst, map, bar, m * kTileM, q_piece);
-        if (two) tma_load_2d_a(dst + kHalfPieceBytes, map, bar, m * kTileM + 64, q_piece);
-      };
-      if (p.has_res && leader) {
-        bulk_wait_group_read1();  // the store of two pieces ago has finished reading this buffer
-        load_residual(0, piece_count);
-      }
 #pragma unroll 1
       for (int piece = 0; piece < p.pieces; ++piece, ++piece_count) {
-        uint8_t* stage = my_stage + (piece_count & 1u) * kPieceBytes;
+        const uint32_t sbuf = piece_count & (nbuf - 1u);
+        uint8_t* stage = my_stage + sbuf * kPieceBytes;
         uint32_t r[kPiece];
         // (a short last piece still reads and stages 40 columns; the surplus is never stored)
         tc_ld_piece(t_row + piece * kPiece, r);
@@ -640,8 +668,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         if (p.has_res) {
           // the residual piece has landed in this buffer (a wait that runs out raises the abort flag;
           // the group still goes on to its barrier and stops at the next tile)
-          mbar_wait_bounded(&bar_res[2 * grp + (piece_count & 1u)], (piece_count >> 1) & 1u, abort_flag,
-                            kWaitLimitCycles);
+          mbar_wait_bounded(&bar_res[4 * grp + sbuf], (piece_count >> nbuf_shift) & 1u, abort_flag, kWaitLimitCycles);
           if (relu)
             stage_piece<true, true>(r, bias_v, st_addr);
           else
@@ -651,8 +678,11 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         } else {
           stage_piece<false, false>(r, bias_v, st_addr);
         }
-        fence_proxy_async_smem();           // generic-proxy writes -> visible to the TMA store
-        if (leader) bulk_wait_group_read0();  // the previous piece's store no longer reads its buffer
+        fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA store
+        // Without a residual the next piece overwrites the other buffer: its store (the previous
+        // piece's) must have read it.  With one, the buffers are refilled by the residual loads
+        // below, which wait for the stores themselves.
+        if (leader && !p.has_res) bulk_wait_group_read0();
         epilogue_bar_sync(grp);
         if (leader) {
           const int q_piece = pt * p.BN + col_base + piece * kPiece;
@@ -664,7 +694,11 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             if (m * kTileM + 64 < p.C_out) tma_store_2d(map, stage + kHalfPieceBytes, m * kTileM + 64, q_piece);
           }
           bulk_commit_group();
-          if (p.has_res && piece + 1 < p.pieces) load_residual(piece + 1, piece_count + 1);
+          if (p.has_res) {
+            // refill the buffer the previous piece's store read: residual piece (count + nbuf - 1)
+            bulk_wait_group_read1();
+            load_residual(piece_count + nbuf - 1u);
+          }
         }
       }
     }
@@ -864,16 +898,16 @@ struct Plan {
   bool split;
 };
 template <bool SPARSE>
-static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force_split) {
-  Plan best{kBN, false};
+static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force_split, int max_bn = kBN) {
+  Plan best{max_bn, false};
   if (force_split) return Plan{kBN, true};
   double best_cost = 0.0;
-  for (int BN = kBN; BN >= 48; BN -= 16) {
+  for (int BN = max_bn; BN >= 48; BN -= 16) {
     const long long tiles = ((Q + BN - 1) / BN) * geo.m_tiles;
     const long long per_cta = (tiles + workers - 1) / workers;
     const int pieces = (BN / 2 + kPiece - 1) / kPiece;
     const double cost = (double)per_cta * geo.kblocks * kblock_cycles<SPARSE>(BN) + pieces * kEpiloguePieceCycles;
-    if (BN == kBN || cost < 0.97 * best_cost) {  // a narrower tile has to earn its extra weight traffic
+    if (BN == max_bn || cost < 0.97 * best_cost) {  // a narrower tile has to earn its extra weight traffic
       best_cost = cost;
       best.BN = BN;
     }
@@ -928,10 +962,17 @@ static int32_t current_device(int* dev_out) {
   return SSCONV_OK;
 }
 
-static int ring_groups_for(uint32_t a_group_bytes, int BN) {
-  // as many groups in the ring as fit beside the staging buffers, at most kMaxGroups (at least 2 fit)
-  const int n = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - kStagingBytes) / group_bytes(a_group_bytes, BN));
+static int ring_groups_for(uint32_t a_group_bytes, int BN, int stage_bufs) {
+  // as many groups in the ring as fit beside the staging buffers, at most kMaxGroups
+  const int n =
+      (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(stage_bufs)) / group_bytes(a_group_bytes, BN));
   return n > kMaxGroups ? kMaxGroups : n;
+}
+// Widest tile for which two groups fit beside the staging buffers.
+static int widest_tile(uint32_t a_group_bytes, int stage_bufs) {
+  int BN = kBN;
+  while (BN > 48 && ring_groups_for(a_group_bytes, BN, stage_bufs) < 2) BN -= 16;
+  return BN;
 }
 
 // What launch_forward_impl would do for this layer on the current device.
@@ -952,7 +993,7 @@ int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* sp
   if (split) *split = do_split ? 1 : 0;
   if (ctas) *ctas = (int32_t)(work < workers ? work : workers);
   if (ring_groups)
-    *ring_groups = ring_groups_for(sparse ? Cfg<true>::kAGroupBytes : Cfg<false>::kAGroupBytes, plan.BN);
+    *ring_groups = ring_groups_for(sparse ? Cfg<true>::kAGroupBytes : Cfg<false>::kAGroupBytes, plan.BN, 2);
   return SSCONV_OK;
 }
 
@@ -981,13 +1022,26 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   const long long Q = (long long)d.N * Ho * Wo;  // positions
   if (Q > 0x7FFFFF00LL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
   const int workers = g_sm_count[dev] < worker_cap ? g_sm_count[dev] : worker_cap;
-  const Plan plan = plan_layer<SPARSE>(Q, geo, workers, force_split);
+  // With a residual the epilogue prefetches residual pieces three ahead into four staging buffers
+  // per group, which narrows the widest tile that still leaves room for two ring groups.  (When K
+  // is split the finishing kernel adds the residual to the split tiles; the main kernel then keeps
+  // two buffers and one piece of lookahead for the whole tiles it may also own.)
+  Plan plan = plan_layer<SPARSE>(Q, geo, workers, force_split);
+  int stage_bufs = 2;
+  if (residual != nullptr && !plan.split) {
+    stage_bufs = 4;
+    plan = plan_layer<SPARSE>(Q, geo, workers, false, widest_tile(C::kAGroupBytes, 4));
+    if (plan.split) {  // the narrower limit made splitting look better: stay unsplit at the limit
+      plan.split = false;
+      plan.BN = widest_tile(C::kAGroupBytes, 4);
+    }
+  }
   const int BN = plan.BN;
   const int pieces = (BN / 2 + kPiece - 1) / kPiece;
   const int tail_cols = BN / 2 - (pieces - 1) * kPiece;
   const uint32_t grp_bytes = group_bytes(C::kAGroupBytes, BN);
-  const int ring_groups = ring_groups_for(C::kAGroupBytes, BN);
-  const uint32_t smem_bytes = 1024 + (uint32_t)ring_groups * grp_bytes + kStagingBytes + kBarrierBytes;
+  const int ring_groups = ring_groups_for(C::kAGroupBytes, BN, stage_bufs);
+  const uint32_t smem_bytes = 1024 + (uint32_t)ring_groups * grp_bytes + staging_bytes(stage_bufs) + kBarrierBytes;
 
   CUtensorMap tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail;
   // activations: NHWC seen as (c, w, h, n), im2col mode; elements outside the image read as zero
@@ -1075,6 +1129,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.ring_groups = ring_groups;
   p.small_c = small_c ? 1 : 0;
   p.has_res = residual != nullptr ? 1 : 0;
+  p.stage_bufs = stage_bufs;
   p.stride_h = d.stride_h;
   p.stride_w = d.stride_w;
   p.pad_h = d.pad_h;

@@ -57,10 +57,13 @@ class ConvStack:
                 api.ssconv_maxpool(src, 3, 2, 1, y=y)
             else:
                 L = self.layers[i]
+                res = self.outputs[st.res] if st.res >= 0 else None
                 if st.kind == "conv" and sparse:
-                    api.ssconv_forward(L["desc"], src, L["w_comp"], L["meta"], L["bias"], y=y, dev_status=self.status)
+                    api.ssconv_forward(L["desc"], src, L["w_comp"], L["meta"], L["bias"], y=y, dev_status=self.status,
+                                       residual=res)
                 else:
-                    api.ssconv_forward_dense(L["desc"], src, L["w"], L["bias"], y=y, dev_status=self.status)
+                    api.ssconv_forward_dense(L["desc"], src, L["w"], L["bias"], y=y, dev_status=self.status,
+                                             residual=res)
             if st.feeds_next:
                 last = y
         return last

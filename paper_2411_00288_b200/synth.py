@@ -147,15 +147,19 @@ class StackStep:
     spec: Optional[LayerSpec]
     src: int
     feeds_next: bool = True
+    res: int = -2  # index of the step whose output is added before the activation (-2: none)
 
 
-def resnet50_stack(batch: int = 256) -> List[StackStep]:
-    """The convolution stack of a Torchvision-shaped ResNet-50 as a residual-free chain: stem
-    (7x7 stride 2, dense, on an input padded from 3 to 8 channels), 3x3 stride-2 max-pool, then per
-    bottleneck reduce -> 3x3 -> expand, each with bias and ReLU, the expand output feeding the next
-    block; the four downsample convolutions read their block's input and feed nothing.  Every
-    convolution has exactly the shape, traffic and FLOPs of the network's; residual additions and
-    batch-norm statistics are left out (batch norm counts as folded into the bias)."""
+def resnet50_stack(batch: int = 256, residual: bool = False) -> List[StackStep]:
+    """The convolution stack of a Torchvision-shaped ResNet-50: stem (7x7 stride 2, dense, on an
+    input padded from 3 to 8 channels), 3x3 stride-2 max-pool, then per bottleneck reduce -> 3x3 ->
+    expand with bias and ReLU, the expand output feeding the next block.  Every convolution has
+    exactly the shape, traffic and FLOPs of the network's; batch norm counts as folded into the bias.
+    residual=False: a residual-free chain, the four downsample convolutions read their block's
+    input and feed nothing.  residual=True: the network's skip connections: the expand convolution
+    adds the block's input (the downsample convolution's output in the first block of a stage)
+    before its ReLU; the expand and downsample weights are scaled down so that activations stay
+    O(1) over the 16 blocks without batch-norm statistics."""
     steps: List[StackStep] = []
     stem = LayerSpec("r50_stem", batch, 224, 224, 8, 64, 7, 7, 2, 3, w_std="he", config=5, index=90)
     steps.append(StackStep("dense", stem, -1))
@@ -170,10 +174,19 @@ def resnet50_stack(batch: int = 256) -> List[StackStep]:
         steps.append(StackStep("conv", conv3, len(steps) - 1))
         after3 = len(steps) - 1
         i += 2
+        identity = block_in
         if specs[i].name.endswith("_down"):
-            steps.append(StackStep("conv", specs[i], block_in, feeds_next=False))
+            down = specs[i]
+            if residual:
+                down = replace(down, w_std=str(0.5 * math.sqrt(1.0 / down.K)))
+            steps.append(StackStep("conv", down, block_in, feeds_next=False))
+            identity = len(steps) - 1
             i += 1
-        steps.append(StackStep("conv", specs[i], after3))
+        if residual:
+            expand = replace(specs[i], w_std=str(0.25 * math.sqrt(2.0 / specs[i].K)))
+            steps.append(StackStep("conv", expand, after3, res=identity))
+        else:
+            steps.append(StackStep("conv", specs[i], after3))
         src = len(steps) - 1
         i += 1
     return steps

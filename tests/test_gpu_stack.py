@@ -4,6 +4,8 @@ the GPU, checked layer by layer against the fp64 oracle.
 The check is teacher-forced: every layer's oracle receives the bf16 input that the GPU layer before
 it actually produced, so errors do not compound over the 53 convolutions and each layer meets the
 same gates as a stand-alone layer."""
+import dataclasses
+
 import numpy as np
 import pytest
 import torch
@@ -37,8 +39,8 @@ def _maxpool_reference(x):
     return out
 
 
-def _check_stack(n, sample):
-    steps = synth.resnet50_stack(n)
+def _check_stack(n, sample, residual=False):
+    steps = synth.resnet50_stack(n, residual=residual)
     net = stack.ConvStack(steps, DEV)
     x = _stack_input(n)
     xd = x.to(DEV)
@@ -48,6 +50,7 @@ def _check_stack(n, sample):
     assert api.ssconv_launch_count() - c0 >= 53
     assert int(net.status.item()) == 0
     worst = (0.0, 0.0, "")
+    peak = 0.0
     for i, st in enumerate(steps):
         src = x if st.src < 0 else net.outputs[st.src].cpu()
         y = net.outputs[i].cpu()
@@ -65,19 +68,30 @@ def _check_stack(n, sample):
             mask = masks.mask_from_pattern(pat, w_bits.shape)
         bias = L["bias_host"].numpy() if L["bias_host"] is not None else None
         shp = parity.oracle_shape(spec)
+        res = net.outputs[st.res].cpu() if st.res >= 0 else None
+        if res is not None:
+            shp = dataclasses.replace(shp, relu=False)  # residual first, then the activation, in fp64 below
         if sample is None:
             yg = parity.bf16_tensor_to_f64(y)
             ref = conv2d_f64(shp, synth.bf16_bits(src), w_bits, mask=mask, bias=bias)
+            if res is not None:
+                ref = ref + parity.bf16_tensor_to_f64(res)
         else:
             rng = np.random.default_rng(spec.seed & 0xFFFFFFFF)
             idx = rng.choice(y.numel(), size=min(sample, y.numel()), replace=False)
             yg = parity.bf16_tensor_to_f64(y.reshape(-1)[torch.from_numpy(idx)])
             ref = conv2d_f64_sample(shp, synth.bf16_bits(src), w_bits, idx, mask=mask, bias=bias)
+            if res is not None:
+                ref = ref + parity.bf16_tensor_to_f64(res.reshape(-1)[torch.from_numpy(idx)])
+        if res is not None and spec.relu:
+            ref = np.maximum(ref, 0.0)
         rel, mx = parity.errors(yg, ref)
         assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"{spec.name}: rel={rel:.3e} max={mx:.3e}"
         assert np.abs(yg).max() > 0, f"{spec.name}: all-zero output"
         if rel > worst[0]:
             worst = (rel, mx, spec.name)
+        peak = max(peak, float(np.abs(yg).max()))
+    print("largest |activation|", peak)
     return worst
 
 
@@ -88,6 +102,17 @@ def test_resnet50_stack_batch4_every_layer_full():
 
 def test_resnet50_stack_batch32_sampled():
     worst = _check_stack(32, 65536)
+    print("worst layer", worst)
+
+
+def test_resnet50_stack_with_skip_connections_batch4_full():
+    """The same stack with the network's skip connections fused into the expand convolutions."""
+    worst = _check_stack(4, None, residual=True)
+    print("worst layer", worst)
+
+
+def test_resnet50_stack_with_skip_connections_batch32_sampled():
+    worst = _check_stack(32, 65536, residual=True)
     print("worst layer", worst)
 
 
