@@ -93,7 +93,6 @@ struct FwdParams {
   int pieces;               // epilogue pieces per group: ceil(BN / 2 / kPiece)
   int tail_cols;            // positions in a group's last piece (a multiple of 8, at most kPiece)
   int ring_groups;          // groups in the shared-memory ring
-  int has_res;              // a residual tensor is added before the activation (see stage_piece)
   int stage_bufs;           // staging buffers per epilogue group: 2, or 4 when residual pieces are prefetched
   int small_c;              // dense layers with C_in == 8: a k-block is 8 filter taps (see producer_role)
   int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
@@ -371,7 +370,9 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
   }
 }
 
-template <bool SPARSE>
+// RES: a residual tensor is added in the epilogue (its own instantiation, so that the plain kernel's
+// epilogue loop carries none of that code).
+template <bool SPARSE, bool RES>
 __global__ void __launch_bounds__(kThreads, 1)
 ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                   const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_y_tail,
@@ -430,7 +431,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       if (warp == 2) {
         prefetch_tensormap(&tm_y);
         prefetch_tensormap(&tm_y_tail);
-        if (p.has_res) {
+        if (RES) {
           prefetch_tensormap(&tm_r);
           prefetch_tensormap(&tm_r_tail);
         }
@@ -602,7 +603,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       tma_load_2d_a(dst, map, bar, m_a * kTileM, q_piece);
       if (two) tma_load_2d_a(dst + kHalfPieceBytes, map, bar, m_a * kTileM + 64, q_piece);
     };
-    if (p.has_res && leader)
+    if (RES && leader)
       for (uint32_t c = 0; c + 1 < nbuf; ++c) load_residual(c);
     WorkIter work(p);
     Segment seg;
@@ -665,7 +666,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         // The buffer was last the source of the store issued two pieces ago; the leader saw that
         // store finish reading before it entered the barrier of the previous piece.
         const uint32_t st_addr = smem_u32(stage) + st_offset;
-        if (p.has_res) {
+        if (RES) {
           // the residual piece has landed in this buffer (a wait that runs out raises the abort flag;
           // the group still goes on to its barrier and stops at the next tile)
           mbar_wait_bounded(&bar_res[4 * grp + sbuf], (piece_count >> nbuf_shift) & 1u, abort_flag, kWaitLimitCycles);
@@ -682,7 +683,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         // Without a residual the next piece overwrites the other buffer: its store (the previous
         // piece's) must have read it.  With one, the buffers are refilled by the residual loads
         // below, which wait for the stores themselves.
-        if (leader && !p.has_res) bulk_wait_group_read0();
+        if (leader && !RES) bulk_wait_group_read0();
         epilogue_bar_sync(grp);
         if (leader) {
           const int q_piece = pt * p.BN + col_base + piece * kPiece;
@@ -694,7 +695,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             if (m * kTileM + 64 < p.C_out) tma_store_2d(map, stage + kHalfPieceBytes, m * kTileM + 64, q_piece);
           }
           bulk_commit_group();
-          if (p.has_res) {
+          if (RES) {
             // refill the buffer the previous piece's store read: residual piece (count + nbuf - 1)
             bulk_wait_group_read1();
             load_residual(piece_count + nbuf - 1u);
@@ -931,7 +932,7 @@ constexpr size_t scratch_bytes(int workers) {
 size_t workspace_bytes() { return scratch_bytes(kMaxWorkers); }
 
 static int g_sm_count[64] = {0};
-static bool g_attr_set[64][2] = {{false}};
+static bool g_attr_set[64][2][2] = {{{false}}};
 
 // Dense layers with 8 input channels (a channel-padded RGB stem): a k-block of 64 K-elements is 8
 // filter taps instead of 64 channels of one tap, which would be 7/8 padding.
@@ -1009,11 +1010,14 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     const int32_t st = current_device(&dev);
     if (st != SSCONV_OK) return st;
   }
-  if (!g_attr_set[dev][SPARSE ? 1 : 0]) {
-    if (cudaFuncSetAttribute(ssconv_fwd_kernel<SPARSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kMaxSmemBytes) != cudaSuccess)
-      return SSCONV_ERR_CUDA;
-    g_attr_set[dev][SPARSE ? 1 : 0] = true;
+  for (int res = 0; res < 2; ++res) {
+    if (g_attr_set[dev][SPARSE ? 1 : 0][res]) continue;
+    const cudaError_t e = res ? cudaFuncSetAttribute(ssconv_fwd_kernel<SPARSE, true>,
+                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmemBytes)
+                              : cudaFuncSetAttribute(ssconv_fwd_kernel<SPARSE, false>,
+                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxSmemBytes);
+    if (e != cudaSuccess) return SSCONV_ERR_CUDA;
+    g_attr_set[dev][SPARSE ? 1 : 0][res] = true;
   }
   const Geometry geo = layer_geometry(d, SPARSE);
   const bool small_c = small_channel_mode(d, SPARSE);
@@ -1128,7 +1132,6 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.tail_cols = tail_cols;
   p.ring_groups = ring_groups;
   p.small_c = small_c ? 1 : 0;
-  p.has_res = residual != nullptr ? 1 : 0;
   p.stage_bufs = stage_bufs;
   p.stride_h = d.stride_h;
   p.stride_w = d.stride_w;
@@ -1181,7 +1184,11 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p) != cudaSuccess) return SSCONV_ERR_CUDA;
+  const cudaError_t launched =
+      residual != nullptr
+          ? cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, true>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p)
+          : cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, false>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p);
+  if (launched != cudaSuccess) return SSCONV_ERR_CUDA;
   count_launch();
   if (p.split) {
     FinishParams f;
