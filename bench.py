@@ -178,7 +178,7 @@ def reference_arm(args):
 # It belongs to the kernel sources with the digest below; with other sources the bench reports null.
 TRAFFIC_BYTES_PER_STEP = 72.81e6
 TRAFFIC_SOURCES = ("forward.cu", "sm100_ptx.cuh", "layout.cuh")
-TRAFFIC_SOURCES_SHA256 = "e935a88a8d1e7479fc92b564c590c56b81c2a40194c7d6c6208ac7a26e9ab107"
+TRAFFIC_SOURCES_SHA256 = "1507f6f00133d2b193e61d7a9c7e0f467f53f9346ce80c45c045a9b5fb99b4e6"
 
 
 def measured_traffic():
