@@ -53,7 +53,9 @@ typedef struct {
   uint32_t flags; /* SSCONV_FLAG_* */
 } ssconv_desc_t;
 
-enum { SSCONV_FLAG_BIAS = 1u, SSCONV_FLAG_RELU = 2u };
+/* GELU (exact form, x Phi(x)) is not part of the paper's method: it is the activation of the
+ * ConvNeXt point-wise layers the paper evaluates on (Sec. 4).  At most one of RELU and GELU. */
+enum { SSCONV_FLAG_BIAS = 1u, SSCONV_FLAG_RELU = 2u, SSCONV_FLAG_GELU = 4u };
 
 enum {
   SSCONV_MASK_LOGITS_F32 = 0,    /* scores: float [G,6], one score per pattern            */
@@ -134,7 +136,7 @@ int32_t ssconv_maxpool(const void* x, void* y, int32_t N, int32_t H, int32_t W, 
  *   y[n,ho,wo,co] = act( bias[co] + sum_{kh,kw,ci} x[n, ho*s-p+kh*d, wo*s-p+kw*d, ci]
  *                                                  * (M .* W)[co,kh,kw,ci] ),
  * taps outside the image contribute 0, products are exact, accumulation is fp32, the
- * result is rounded once to bf16 (nearest even).  act = ReLU if SSCONV_FLAG_RELU, bias is
+ * result is rounded once to bf16 (nearest even).  act = ReLU if SSCONV_FLAG_RELU, GELU if SSCONV_FLAG_GELU, bias is
  * read only if SSCONV_FLAG_BIAS.
  * x, y, w_comp, meta: device, 16-byte aligned.  Needs C_in % 8 == 0, C_out % 8 == 0,
  * pad <= 127, dil*(K-1) <= 255, stride <= 8.

@@ -15,6 +15,7 @@ import torch
 
 FLAG_BIAS = 1
 FLAG_RELU = 2
+FLAG_GELU = 4
 MASK_LOGITS_F32 = 0
 MASK_MAGNITUDE_BF16 = 1
 OK = 0
@@ -42,18 +43,18 @@ class Desc(ctypes.Structure):
         ("flags", ctypes.c_uint32)]
 
 
-def make_desc(N, H, W, C_in, C_out, KH, KW, stride=1, pad=0, dil=1, bias=True, relu=False) -> Desc:
+def make_desc(N, H, W, C_in, C_out, KH, KW, stride=1, pad=0, dil=1, bias=True, relu=False, gelu=False) -> Desc:
     def pair(v):
         return (v, v) if isinstance(v, int) else tuple(v)
     (sh, sw), (ph, pw), (dh, dw) = pair(stride), pair(pad), pair(dil)
-    flags = (FLAG_BIAS if bias else 0) | (FLAG_RELU if relu else 0)
+    flags = (FLAG_BIAS if bias else 0) | (FLAG_RELU if relu else 0) | (FLAG_GELU if gelu else 0)
     return Desc(N, H, W, C_in, C_out, KH, KW, sh, sw, ph, pw, dh, dw, flags)
 
 
 def desc_from_spec(spec) -> Desc:
     """Descriptor for a synth.LayerSpec."""
     return make_desc(spec.N, spec.H, spec.W, spec.C_in, spec.C_out, spec.KH, spec.KW, spec.stride, spec.pad,
-                     spec.dil, bias=spec.has_bias, relu=spec.relu)
+                     spec.dil, bias=spec.has_bias, relu=spec.relu and not spec.gelu, gelu=spec.gelu)
 
 
 _lib = None

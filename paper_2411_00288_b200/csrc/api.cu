@@ -51,7 +51,8 @@ int32_t check_desc(const ssconv_desc_t* d, bool need_tma_shape) {
     return SSCONV_ERR_BAD_DESC;
   if (d->stride_h <= 0 || d->stride_w <= 0 || d->dil_h <= 0 || d->dil_w <= 0 || d->pad_h < 0 || d->pad_w < 0)
     return SSCONV_ERR_BAD_DESC;
-  if (d->flags & ~(SSCONV_FLAG_BIAS | SSCONV_FLAG_RELU)) return SSCONV_ERR_BAD_DESC;
+  if (d->flags & ~(SSCONV_FLAG_BIAS | SSCONV_FLAG_RELU | SSCONV_FLAG_GELU)) return SSCONV_ERR_BAD_DESC;
+  if ((d->flags & SSCONV_FLAG_RELU) && (d->flags & SSCONV_FLAG_GELU)) return SSCONV_ERR_BAD_DESC;  // one activation
   int Ho = out_extent(d->H, d->KH, d->stride_h, d->pad_h, d->dil_h);
   int Wo = out_extent(d->W, d->KW, d->stride_w, d->pad_w, d->dil_w);
   if (Ho <= 0 || Wo <= 0) return SSCONV_ERR_BAD_DESC;

@@ -211,7 +211,22 @@ __device__ __forceinline__ void tc_ld_piece(uint32_t taddr, uint32_t (&r)[kPiece
 // With RES the staging buffer already holds the residual tile (bf16, same layout): it is read back
 // in fragment layout (ldmatrix.trans, the inverse of the store), added in fp32 before the one
 // rounding, and overwritten in place (a warp only touches its own 16-byte columns).
-template <bool RELU, bool RES>
+// ACT: 0 identity, 1 ReLU (inside the bf16 conversion), 2 GELU in its exact form x Phi(x) =
+// 0.5 x (1 + erf(x / sqrt 2)), evaluated in fp32 before the rounding.
+constexpr int kActNone = 0, kActRelu = 1, kActGelu = 2;
+__device__ __forceinline__ float gelu_f32(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
+template <int ACT>
+__device__ __forceinline__ uint32_t activate_pack(float lo, float hi) {
+  if (ACT == kActGelu) {
+    lo = gelu_f32(lo);
+    hi = gelu_f32(hi);
+  }
+  return pack_bf16x2<ACT == kActRelu>(lo, hi);
+}
+__host__ __device__ inline int activation_of(uint32_t flags) {
+  return (flags & SSCONV_FLAG_GELU) ? kActGelu : (flags & SSCONV_FLAG_RELU) ? kActRelu : kActNone;
+}
+template <int ACT, bool RES>
 __device__ __forceinline__ void stage_piece(const uint32_t (&r)[kPiece], const float (&bias)[4], uint32_t st_addr) {
 #pragma unroll
   for (int k = 0; k < kPiece / 8; ++k) {
@@ -226,7 +241,7 @@ __device__ __forceinline__ void stage_piece(const uint32_t (&r)[kPiece], const f
         lo += bf16_lo(res[i]);
         hi += bf16_hi(res[i]);
       }
-      w[i] = pack_bf16x2<RELU>(lo, hi);
+      w[i] = activate_pack<ACT>(lo, hi);
     }
     stmatrix_x4_trans(st_addr + 1024u * k, w[0], w[1], w[2], w[3]);
   }
@@ -564,7 +579,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     const int q = warp & 3;  // TMEM lane quadrant this warp may read: channels [32 q, 32 q + 32) of the tile
     const int gtid = q * 32 + lane;
     const bool leader = (q == 2 && lane == 0);  // first warp of each group
-    const bool relu = (p.flags & SSCONV_FLAG_RELU) != 0;
+    const int act = activation_of(p.flags);
     const int col_base = grp * (p.BN >> 1);
     const uint32_t nbuf = (uint32_t)p.stage_bufs;  // 2 or 4
     const uint32_t nbuf_shift = nbuf == 4 ? 2u : 1u;
@@ -670,14 +685,18 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
           // the residual piece has landed in this buffer (a wait that runs out raises the abort flag;
           // the group still goes on to its barrier and stops at the next tile)
           mbar_wait_bounded(&bar_res[4 * grp + sbuf], (piece_count >> nbuf_shift) & 1u, abort_flag, kWaitLimitCycles);
-          if (relu)
-            stage_piece<true, true>(r, bias_v, st_addr);
+          if (act == kActRelu)
+            stage_piece<kActRelu, true>(r, bias_v, st_addr);
+          else if (act == kActGelu)
+            stage_piece<kActGelu, true>(r, bias_v, st_addr);
           else
-            stage_piece<false, true>(r, bias_v, st_addr);
-        } else if (relu) {
-          stage_piece<true, false>(r, bias_v, st_addr);
+            stage_piece<kActNone, true>(r, bias_v, st_addr);
+        } else if (act == kActRelu) {
+          stage_piece<kActRelu, false>(r, bias_v, st_addr);
+        } else if (act == kActGelu) {
+          stage_piece<kActGelu, false>(r, bias_v, st_addr);
         } else {
-          stage_piece<false, false>(r, bias_v, st_addr);
+          stage_piece<kActNone, false>(r, bias_v, st_addr);
         }
         fence_proxy_async_smem();  // generic-proxy writes -> visible to the TMA store
         // Without a residual the next piece overwrites the other buffer: its store (the previous
@@ -812,17 +831,14 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
     acc1.x += bf16_lo(res[2]); acc1.y += bf16_hi(res[2]); acc1.z += bf16_lo(res[3]); acc1.w += bf16_hi(res[3]);
   }
   uint32_t w[4];
-  if (f.flags & SSCONV_FLAG_RELU) {
-    w[0] = pack_bf16x2<true>(acc0.x + bias_v[0], acc0.y + bias_v[0]);
-    w[1] = pack_bf16x2<true>(acc0.z + bias_v[1], acc0.w + bias_v[1]);
-    w[2] = pack_bf16x2<true>(acc1.x + bias_v[2], acc1.y + bias_v[2]);
-    w[3] = pack_bf16x2<true>(acc1.z + bias_v[3], acc1.w + bias_v[3]);
-  } else {
-    w[0] = pack_bf16x2<false>(acc0.x + bias_v[0], acc0.y + bias_v[0]);
-    w[1] = pack_bf16x2<false>(acc0.z + bias_v[1], acc0.w + bias_v[1]);
-    w[2] = pack_bf16x2<false>(acc1.x + bias_v[2], acc1.y + bias_v[2]);
-    w[3] = pack_bf16x2<false>(acc1.z + bias_v[3], acc1.w + bias_v[3]);
-  }
+  const float v[8] = {acc0.x + bias_v[0], acc0.y + bias_v[0], acc0.z + bias_v[1], acc0.w + bias_v[1],
+                      acc1.x + bias_v[2], acc1.y + bias_v[2], acc1.z + bias_v[3], acc1.w + bias_v[3]};
+  const int act = activation_of(f.flags);
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    w[i] = (act == kActRelu)   ? activate_pack<kActRelu>(v[2 * i], v[2 * i + 1])
+           : (act == kActGelu) ? activate_pack<kActGelu>(v[2 * i], v[2 * i + 1])
+                               : activate_pack<kActNone>(v[2 * i], v[2 * i + 1]);
   stmatrix_x4_trans(st_addr, w[0], w[1], w[2], w[3]);
   __syncthreads();
   if (in_range) {

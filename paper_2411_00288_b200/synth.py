@@ -35,6 +35,7 @@ class LayerSpec:
     dil: int = 1
     relu: bool = True
     has_bias: bool = True
+    gelu: bool = False             # GELU instead of ReLU (takes precedence)
     w_std: str = "fan_in"          # "fan_in": 1/sqrt(fan_in); "he": sqrt(2/fan_in); or a float as str
     mask_source: str = "magnitude"  # "magnitude" | "gumbel_logits" | "uniform_pattern"
     config: int = 0

@@ -1,6 +1,7 @@
 """Helpers shared by the GPU parity tests: run one layer through the CUDA library (via the
 C ABI binding) and through the CPU oracle on the same seeded bits, and compare."""
 import dataclasses
+import math
 
 import numpy as np
 import torch
@@ -16,7 +17,8 @@ MAX_ABS_TOL = 2e-2
 
 def oracle_shape(spec) -> ConvShape:
     return ConvShape(spec.N, spec.H, spec.W, spec.C_in, spec.C_out, spec.KH, spec.KW,
-                     (spec.stride, spec.stride), (spec.pad, spec.pad), (spec.dil, spec.dil), relu=spec.relu)
+                     (spec.stride, spec.stride), (spec.pad, spec.pad), (spec.dil, spec.dil),
+                     relu=spec.relu and not spec.gelu)
 
 
 def oracle_pattern(inp) -> np.ndarray:
@@ -41,6 +43,12 @@ def gpu_pattern(inp, dev) -> torch.Tensor:
 
 def bf16_tensor_to_f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().to(torch.float32).numpy().astype(np.float64)
+
+
+def gelu_f64(x: np.ndarray) -> np.ndarray:
+    """GELU in its defining form x * Phi(x), Phi the standard normal distribution function."""
+    erf = np.vectorize(math.erf, otypes=[np.float64])
+    return 0.5 * x * (1.0 + erf(x / math.sqrt(2.0)))
 
 
 def errors(y_gpu_f64: np.ndarray, y_ref: np.ndarray):
@@ -88,15 +96,18 @@ def check_layer(spec, dev, sparse=True, sample=None, seed=None, residual=False):
     mask = masks.mask_from_pattern(pat, w_bits.shape) if sparse else None
     bias = inp.bias.numpy() if inp.bias is not None else None
     shp = oracle_shape(spec)
-    if residual:
-        shp = dataclasses.replace(shp, relu=False)
+    if residual or spec.gelu:
+        shp = dataclasses.replace(shp, relu=False)  # the test finishes the epilogue in fp64 itself
     yg = bf16_tensor_to_f64(y)
 
     def finish(ref, idx=None):
-        if not residual:
+        if not residual and not spec.gelu:
             return ref
-        r = bf16_tensor_to_f64(res).reshape(-1)
-        ref = ref + (r.reshape(ref.shape) if idx is None else r[idx])
+        if residual:
+            r = bf16_tensor_to_f64(res).reshape(-1)
+            ref = ref + (r.reshape(ref.shape) if idx is None else r[idx])
+        if spec.gelu:
+            return gelu_f64(ref)
         return np.maximum(ref, 0.0) if spec.relu else ref
 
     if sample is None:

@@ -124,3 +124,42 @@ def test_residual_in_place_and_wide_tiles():
     assert torch.equal(y_sep, y_inplace)
     assert api.ssconv_plan(desc, True)["tile_positions"] == 240
     _assert_ok(*parity.check_layer(spec, DEV, sparse=True, sample=30000, residual=True), "res_inplace")
+
+
+# ---------------------------------------------------------------------------------------------
+# GELU epilogue (the activation of ConvNeXt's point-wise expand layers)
+GELU_CASES = [
+    ("gelu_pw_96to384",   2, 14, 14, 96,  384, 1, 1, 1, 0, 1),
+    ("gelu_c3_64to136",   2, 12, 9,  64,  136, 3, 3, 1, 1, 1),
+]
+
+
+@pytest.mark.parametrize("case", GELU_CASES, ids=[c[0] for c in GELU_CASES])
+@pytest.mark.parametrize("sparse", [True, False], ids=["sparse", "dense"])
+@pytest.mark.parametrize("residual", [False, True], ids=["plain", "residual"])
+def test_gelu_epilogue(case, sparse, residual):
+    name, N, H, W, Ci, Co, KH, KW, s, p, d = case
+    spec = synth.LayerSpec(name, N, H, W, Ci, Co, KH, KW, s, p, d, gelu=True, w_std="fan_in",
+                           mask_source="magnitude", config=9, index=80 + GELU_CASES.index(case))
+    _assert_ok(*parity.check_layer(spec, DEV, sparse=sparse, residual=residual), name)
+
+
+def test_gelu_matches_closed_values_and_flag_rules():
+    """x == 1, one kept weight w per output channel and zero bias give y = GELU(w) exactly enough to tell
+    GELU from ReLU and identity; RELU and GELU together are refused."""
+    import ctypes
+    import math
+    N, H, W, C, Co = 1, 4, 4, 8, 8
+    desc = api.make_desc(N, H, W, C, Co, 1, 1, bias=False, gelu=True)
+    x = torch.ones((N, H, W, C), dtype=torch.bfloat16, device=DEV)
+    w = torch.zeros((Co, 1, 1, C), dtype=torch.bfloat16, device=DEV)
+    vals = [-3.0, -1.0, -0.5, 0.0, 0.5, 1.0, 2.0, 4.0]
+    for co, v in enumerate(vals):
+        w[co, 0, 0, 0] = v
+    y = api.ssconv_forward_dense(desc, x, w, None).float().cpu().numpy()
+    for co, v in enumerate(vals):
+        want = 0.5 * v * (1.0 + math.erf(v / math.sqrt(2.0)))
+        assert abs(y[0, 0, 0, co] - want) <= 2 ** -8 * max(1.0, abs(want)), (v, y[0, 0, 0, co], want)
+    both = api.make_desc(N, H, W, C, Co, 1, 1, bias=False, relu=True, gelu=True)
+    ho, wo = ctypes.c_int32(), ctypes.c_int32()
+    assert api.lib().ssconv_out_shape(ctypes.byref(both), ctypes.byref(ho), ctypes.byref(wo)) == 2  # bad descriptor
