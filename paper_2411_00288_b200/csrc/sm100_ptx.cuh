@@ -20,23 +20,8 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_fence_init() {
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-               : "memory");
-}
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
 }
 
 // Spin on a phase of an mbarrier for at most `spins` tries, entirely inside one asm block: the
@@ -97,40 +82,6 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 }
 
 // ---------------------------------------------------------------- TMA loads
-__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int32_t x,
-                                            int32_t y) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
-      : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int32_t x,
-                                            int32_t y, int32_t z) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
-      : "memory");
-}
-// im2col mode over an NHWC tensor seen as (c, w, h, n): loads `pixelsPerColumn` consecutive
-// filter placements starting at base pixel (w, h, n), `channelsPerPixel` channels from c,
-// each read at base + (off_w, off_h); out-of-image elements arrive as zeros.
-__device__ __forceinline__ void tma_load_im2col_4d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int32_t c,
-                                                   int32_t w, int32_t h, int32_t n, uint16_t off_w,
-                                                   uint16_t off_h) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
-      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w),
-      "h"(off_h)
-      : "memory");
-}
-// Untiled bulk copy global -> shared; both addresses 16-byte aligned, bytes % 16 == 0.
-__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-      ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
-      : "memory");
-}
 
 // ---------------------------------------------------------------- fragment -> shared memory
 // Four 8x8 matrices of 16-bit elements, each stored transposed: register i of thread t holds
@@ -190,7 +141,6 @@ __device__ __forceinline__ void bulk_wait_group_read0() {
 __device__ __forceinline__ void bulk_wait_group_read1() {
   asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
 }
-__device__ __forceinline__ void bulk_wait_group0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // ---------------------------------------------------------------- tcgen05: TMEM management
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t ncols) {
@@ -216,32 +166,6 @@ __device__ __forceinline__ void tc_commit(uint64_t* bar) {
 }
 
 // ---------------------------------------------------------------- tcgen05: descriptors
-// Shared-memory matrix descriptor for a K-major operand tile whose rows are 128 bytes and
-// swizzled with the 128-byte pattern (what a TMA load with SWIZZLE_128B produces):
-//   bits  0-13  start address >> 4
-//   bits 16-29  leading-dimension byte offset >> 4 (not used by swizzled K-major tiles)
-//   bits 32-45  stride-dimension byte offset >> 4 = distance between 8-row groups (1024 B)
-//   bits 46-47  descriptor version (1 on sm_100)
-//   bits 61-63  swizzle mode (2 = 128 B)
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
-  d |= static_cast<uint64_t>(1) << 16;
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= static_cast<uint64_t>(2) << 61;
-  return d;
-}
-// Descriptor for an unswizzled tile of 16-byte rows, 8 rows (128 B) per core matrix, core
-// matrices stacked every `sbo_bytes`: the source format of the metadata copy below.
-__device__ __forceinline__ uint64_t smem_desc_noswizzle(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
-  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFF) << 16;
-  d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFF) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  return d;
-}
 
 // Instruction descriptor of tcgen05.mma kind::f16 with bf16 A and B (both K-major) and an
 // fp32 accumulator:
@@ -253,60 +177,7 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(uint32_t M, uint32_t N, b
 }
 
 // ---------------------------------------------------------------- tcgen05: mma / cp / ld
-__device__ __forceinline__ void tc_mma_dense(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                             uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// Sparse form: A holds the kept half of a 2:4 sparse matrix, `meta_tmem` the TMEM column
-// pair with its position indices; the sparsity selector in idesc picks the column.
-__device__ __forceinline__ void tc_mma_sparse(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t meta_tmem,
-                                              uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %5, 0;\n\t"
-      "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(meta_tmem), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// Copy 128 rows x 128 bits from shared memory (descriptor) into 4 TMEM columns, row r -> lane r.
-__device__ __forceinline__ void tc_cp_128x128b(uint32_t dst_tmem, uint64_t src_desc) {
-  asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(dst_tmem), "l"(src_desc) : "memory");
-}
 
-// 32 lanes x 32 consecutive 32-bit columns: thread t of the warp receives lane (base+t).
-__device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-// Same for 16 columns.
-__device__ __forceinline__ void tc_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tc_ld_32x8(uint32_t taddr, uint32_t (&r)[8]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "r"(taddr)
-               : "memory");
-}
 // 16 lanes x 8N consecutive 32-bit columns in the layout of an MMA accumulator fragment: per
 // group of 8 columns thread t receives 4 registers: lane (base + t/4), columns 2(t%4) and 2(t%4)+1,
 // then lane (base + t/4 + 8), same columns.  base is the first or the 17th lane of the warp's quadrant.
@@ -370,12 +241,23 @@ __device__ __forceinline__ void bulk_load_a(uint32_t dst, const void* gsrc, uint
       : "memory");
 }
 
-// Upper 32 bits of the two shared-memory descriptor kinds used here (see smem_desc_sw128 and
-// smem_desc_noswizzle); the lower 32 bits are (address >> 4) | (1 << 16).
+// A shared-memory matrix descriptor is 64 bits:
+//   bits  0-13  start address >> 4
+//   bits 16-29  leading-dimension byte offset >> 4 (distance between 16-byte K-chunks of an
+//               unswizzled tile; not used by swizzled K-major tiles, set to 1)
+//   bits 32-45  stride-dimension byte offset >> 4 = distance between groups of 8 rows
+//   bits 46-47  descriptor version (1 on sm_100)
+//   bits 61-63  swizzle mode (0 = none, 2 = 128 B)
+// The kernels build it from two 32-bit halves.  The high half is one of two constants: for a
+// K-major tile with 128-byte rows in the 128-byte swizzle (what a TMA load with SWIZZLE_128B
+// produces; 8-row groups 1024 B apart), and for an unswizzled tile of 16-byte-wide chunks (8 rows =
+// one 128-byte core matrix).  The low half is (address >> 4) | (leading-dimension offset << 16).
 constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
 constexpr uint32_t kDescHiNoSwizzle128 = (128u >> 4) | (1u << 14);
 __device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
 
+// D[128 x N] (+)= A[128 x 16] B[N x 16]^T, bf16 operands in swizzled K-major shared-memory tiles, fp32
+// accumulator at TMEM address d_tmem; `accumulate` == 0 overwrites D.  Issued by one thread.
 __device__ __forceinline__ void tc_mma_dense_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
                                                 uint32_t accumulate) {
   asm volatile(
@@ -402,6 +284,9 @@ __device__ __forceinline__ void tc_mma_dense_chunked(uint32_t d_tmem, uint32_t a
       ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHiNoSwizzle128)
       : "memory");
 }
+// 2:4 sparse form: A holds the 16 kept values of 32 dense K-columns per row, B the 32 columns;
+// meta_tmem is the TMEM column with the 2-bit indices of those columns (bit 0 of the column
+// address is passed in the instruction descriptor's selector bits by the caller).
 __device__ __forceinline__ void tc_mma_sparse_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t meta_tmem,
                                                  uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -413,6 +298,8 @@ __device__ __forceinline__ void tc_mma_sparse_lo(uint32_t d_tmem, uint32_t a_lo,
       ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(meta_tmem), "r"(idesc), "r"(accumulate), "r"(kDescHiSw128)
       : "memory");
 }
+// Copy 128 rows x 128 bits from shared memory (unswizzled, 16-byte rows) into 4 TMEM columns, row r
+// to lane r: one weight tile's metadata image.  Ordered with the MMAs of the issuing thread.
 __device__ __forceinline__ void tc_cp_128x128b_lo(uint32_t dst_tmem, uint32_t src_lo) {
   asm volatile(
       "{\n\t.reg .b64 ds;\n\t"
