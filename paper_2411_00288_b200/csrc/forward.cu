@@ -641,7 +641,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         // sums the shares of all contributors
         float4* mine = p.ws_regions + region_index(blockIdx.x, seg.a0 == 0) * kRegionVecs;
 #pragma unroll 1
-        for (int piece = 0; piece < kPiecesPerGroup; ++piece) {
+        for (int piece = 0; piece < p.pieces; ++piece) {  // (a short last piece is parked whole)
           uint32_t r[kPiece];
           tc_ld_piece(t_row + piece * kPiece, r);
           tc_wait_ld();
@@ -752,6 +752,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
 // memory by stmatrix.trans exactly as in the main kernel before 16-byte stores write NHWC.
 struct FinishParams {
   int C_out, Q;
+  int BN, pieces, tail_cols;  // the main kernel's tile width and epilogue pieces per group
   int m_tiles, a_tiles;
   int work_quot, work_rem;  // the main kernel's dealing of (tile, group) units to its CTAs
   const float4* ws_regions;
@@ -761,7 +762,8 @@ struct FinishParams {
   __nv_bfloat16* y;
 };
 constexpr int kFinishThreads = 128;
-constexpr int kFinishItemsPerTile = kGroups * kPiecesPerGroup * (kPiece / 8);
+// work items per tile: epilogue groups x pieces per group x blocks of 8 positions per piece
+__host__ __device__ constexpr int finish_items_per_tile(int pieces) { return kGroups * pieces * (kPiece / 8); }
 constexpr int kFinishBatch = 8;  // contributors whose loads are in flight together
 
 __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(const FinishParams f) {
@@ -770,8 +772,8 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
   int item = blockIdx.x;
   const int k = item % (kPiece / 8);
   item /= (kPiece / 8);
-  const int piece = item % kPiecesPerGroup;
-  item /= kPiecesPerGroup;
+  const int piece = item % f.pieces;
+  item /= f.pieces;
   const int grp = item % kGroups;
   const int tile = item / kGroups;
   if (gtid == 0) grid_launch_dependents();
@@ -779,6 +781,7 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
   const int c_first = unit_owner(u_first, f.work_quot, f.work_rem);
   const int c_last = unit_owner(u_first + f.a_tiles - 1, f.work_quot, f.work_rem);
   if (c_first == c_last) return;  // the tile was computed whole by one CTA, which also finished it
+  if (piece == f.pieces - 1 && 8 * k >= f.tail_cols) return;  // beyond a short last piece
   const int pt = tile / f.m_tiles;
   const int m = tile - pt * f.m_tiles;
   grid_dependency_wait();  // the main kernel's partial tiles are complete and visible
@@ -816,7 +819,7 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
   const uint32_t chunk = (uint32_t)(4 * q + (lane >> 3));
   const uint32_t st_addr = smem_u32(stage) + row * 256u + ((chunk ^ row) << 4);
   const int pos = gtid >> 4, ch16 = gtid & 15;  // 16 threads cover the 256 contiguous bytes of one position
-  const int q_pos = pt * kBN + grp * kGroupCols + piece * kPiece + 8 * k + pos;
+  const int q_pos = pt * f.BN + grp * (f.BN >> 1) + piece * kPiece + 8 * k + pos;
   const int co16 = m * kTileM + 8 * ch16;
   const bool in_range = q_pos < f.Q && co16 < f.C_out;
   if (f.residual != nullptr) {
@@ -929,15 +932,25 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
       best.BN = BN;
     }
   }
-  // Even split of K at full width, when many SMs would still idle and K is deep.
+  // Even split of K ("stream-K"), when many SMs would still idle and K is deep: every CTA gets the
+  // same number of groups; parked partial tiles cost L2 traffic in proportion to the tile width.
   const int a_tiles = geo.stages;
   if (a_tiles > 1) {
-    const long long tiles = ((Q + kBN - 1) / kBN) * geo.m_tiles;
-    const double units = (double)tiles * a_tiles;
-    const double ctas = units < workers ? units : (double)workers;
-    const double per_a_tile = 2.0 * kblock_cycles<SPARSE>(kBN);
-    const double split_cost = units / ctas * per_a_tile + (ctas + tiles) * kCyclesPerParkedTile;
-    if (best_cost > kSplitAdvantage * split_cost) return Plan{kBN, true};
+    Plan best_split{kBN, true};
+    double best_split_cost = 0.0;
+    for (int BN = max_bn; BN >= 48; BN -= 16) {
+      const long long tiles = ((Q + BN - 1) / BN) * geo.m_tiles;
+      const double units = (double)tiles * a_tiles;
+      const double ctas = units < workers ? units : (double)workers;
+      const int pieces = (BN / 2 + kPiece - 1) / kPiece;
+      const double cost = units / ctas * 2.0 * kblock_cycles<SPARSE>(BN) +
+                          (ctas + tiles) * kCyclesPerParkedTile * (pieces * 2.0 * kPiece / kBN);
+      if (BN == max_bn || cost < 0.97 * best_split_cost) {
+        best_split_cost = cost;
+        best_split.BN = BN;
+      }
+    }
+    if (best_cost > kSplitAdvantage * best_split_cost) return best_split;
   }
   return best;
 }
@@ -1210,6 +1223,9 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     FinishParams f;
     f.C_out = d.C_out;
     f.Q = (int)Q;
+    f.BN = BN;
+    f.pieces = pieces;
+    f.tail_cols = tail_cols;
     f.m_tiles = geo.m_tiles;
     f.a_tiles = p.a_tiles;
     f.work_quot = p.work_quot;
@@ -1219,7 +1235,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     f.bias = bias;
     f.residual = static_cast<const __nv_bfloat16*>(residual);
     f.y = p.y;
-    cfg.gridDim = dim3((unsigned)p.num_tiles * kFinishItemsPerTile);
+    cfg.gridDim = dim3((unsigned)p.num_tiles * finish_items_per_tile(pieces));
     cfg.blockDim = dim3((unsigned)kFinishThreads);
     cfg.dynamicSmemBytes = 0;
     if (cudaLaunchKernelEx(&cfg, ssconv_split_finish_kernel, f) != cudaSuccess) return SSCONV_ERR_CUDA;
