@@ -37,6 +37,11 @@ SWEEP = [
     ("stem_7x7_s2_c8",          2, 30, 34, 8,  64,  7, 7, 2, 3, 1),
     ("pw_c8",                   2, 9,  9,  8,  16,  1, 1, 1, 0, 1),
     ("c4x4_c8_even_taps",       1, 12, 12, 8,  136, 4, 4, 1, 1, 1),
+    # degenerate extents: a single pixel, a single row, a filter larger than the image
+    ("one_pixel",               1, 1,  1,  8,   8,  1, 1, 1, 0, 1),
+    ("one_row_wide",            1, 1,  301, 64, 64, 1, 1, 1, 0, 1),
+    ("filter_exceeds_image",    2, 2,  3,  16,  24, 5, 5, 1, 2, 1),
+    ("stride3_pad0",            1, 10, 13, 32,  40, 3, 3, 3, 0, 1),
 ]
 
 
