@@ -176,9 +176,9 @@ def reference_arm(args):
 # the finishing kernel of the one split layer), dram__bytes_read.sum + dram__bytes_write.sum from an
 # ncu capture of this workload (summary and command: profiles/bench_resnet18_sweep_dram_traffic.md).
 # It belongs to the kernel sources with the digest below; with other sources the bench reports null.
-TRAFFIC_BYTES_PER_STEP = 72.81e6
+TRAFFIC_BYTES_PER_STEP = 66.38e6
 TRAFFIC_SOURCES = ("forward.cu", "sm100_ptx.cuh", "layout.cuh")
-TRAFFIC_SOURCES_SHA256 = "1507f6f00133d2b193e61d7a9c7e0f467f53f9346ce80c45c045a9b5fb99b4e6"
+TRAFFIC_SOURCES_SHA256 = "a80b01042e59b76d202800b8b36e1c3b196dad8e237508538eea2d164988d0f2"
 
 
 def measured_traffic():
