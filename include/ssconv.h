@@ -176,6 +176,48 @@ int32_t ssconv_forward_dense_res(const ssconv_desc_t* desc, const void* x, const
                                  const float* bias, const void* residual, void* y, void* ws,
                                  size_t ws_bytes, int32_t* dev_status, void* stream);
 
+/* ---- Learning the mask (Sec. 3.1): one training step's kernels for one layer ----------------
+ * Only the choice weights (one logit per pattern and group) are trained; the pretrained weights W
+ * stay as they are (Sec. 4.1).  A step for one layer is: ssconv_soft_mask -> ssconv_forward_dense
+ * with the effective weights -> (the caller's loss and its gradient dL/dy) -> ssconv_wgrad ->
+ * ssconv_mask_grad -> the caller's optimiser on the logits. */
+
+/* Relaxed choice and soft mask of every group:
+ *   z[g][i]   = softmax_i((logits[g][i] + noise[g][i]) / tau)                      (Eq. 3)
+ *   b[g][j]   = sum_i D[j][i] z[g][i],   D the 4 x 6 pattern matrix of Eq. 2       (b = D z)
+ *   w_eff     = b .* w  (Eq. 6 with the soft mask), rounded once to bf16 (nearest even).
+ * logits = log pi up to a constant per group; noise = the caller's Gumbel(0,1) sample per logit
+ * (NULL: none); tau > 0.  All arithmetic is fp32.  Pattern order as in ssconv_select_mask.
+ * logits, noise, z: device fp32 [G][6], 8-byte aligned; w, w_eff: device bf16 [C_out,KH,KW,C_in]
+ * read as G groups of 4, 8-byte aligned.  z (nullable) is kept for ssconv_mask_grad; w_eff
+ * (nullable, then w may be NULL too) feeds ssconv_forward_dense.  G >= 0 (0 is a no-op). */
+int32_t ssconv_soft_mask(const float* logits, const float* noise, float tau, const void* w_bf16,
+                         int64_t G, float* z, void* w_eff_bf16, void* stream);
+
+/* Gradient of the loss with respect to the choice weights, from G = dL/dw_eff (chain rule through
+ * Eq. 6, Eq. 2 and Eq. 3; the paper prints no gradient):
+ *   dL/db[g][j] = G[g][j] w[g][j],   dL/dz[g][i] = sum_j D[j][i] dL/db[g][j],
+ *   g_logits[g][i] = z[g][i] (dL/dz[g][i] - sum_k z[g][k] dL/dz[g][k]) / tau.
+ * z: what ssconv_soft_mask stored; g_w_eff: device fp32 [C_out,KH,KW,C_in] (what ssconv_wgrad
+ * writes), 16-byte aligned; g_logits: device fp32 [G][6], 8-byte aligned.  fp32 arithmetic. */
+int32_t ssconv_mask_grad(const float* z, float tau, const void* w_bf16, const float* g_w_eff,
+                         int64_t G, float* g_logits, void* stream);
+
+/* Weight gradient of the convolution (Eq. 4 differentiated in the weights):
+ *   dw[co,kh,kw,ci] = sum_{n,ho,wo} dy[n,ho,wo,co] * x[n, ho*s-p+kh*d, wo*s-p+kw*d, ci],
+ * pixels outside the image contributing nothing.  x: bf16 NHWC input of the layer; dy: bf16 NHWC
+ * gradient of its output [N,H_out,W_out,C_out]; dw: fp32 [C_out,KH,KW,C_in], every element written.
+ * Products are exact, accumulation is fp32 on the tensor cores.  flags of desc are ignored.
+ * Shape rules as ssconv_forward_dense.  x, dy, dw, ws: device, 16-byte aligned.
+ * ws: scratch of at least ssconv_wgrad_ws_bytes (0 for layers with enough work per SM; ws may then
+ * be NULL): layers with few weights and many positions split the positions over thread blocks,
+ * which store partial gradients there; a second kernel adds them in a fixed order.  Needs no
+ * initialisation.  dev_status: as in ssconv_forward. */
+int32_t ssconv_wgrad(const ssconv_desc_t* desc, const void* x, const void* dy, float* dw, void* ws,
+                     size_t ws_bytes, int32_t* dev_status, void* stream);
+/* Scratch bytes ssconv_wgrad needs for this layer on the current device. */
+int32_t ssconv_wgrad_ws_bytes(const ssconv_desc_t* desc, size_t* bytes);
+
 /* ssconv_forward for callers that have no way to provide scratch memory.  (The paper has no
  * counterpart to this call; it exists for integration only.)
  *

@@ -27,6 +27,7 @@ EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssc
            "ssconv_select_mask",
            "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense",
+           "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
            "ssconv_forward_static_ws")
 
 
@@ -295,3 +296,64 @@ def ssconv_forward_static_ws(desc: Desc, x: torch.Tensor, w_comp: torch.Tensor, 
         ctypes.byref(desc), _ptr(x), _ptr(w_comp), _ptr(meta), _ptr(bias), _ptr(y), _ptr(dev_status),
         _stream(stream)))
     return y
+
+
+def ssconv_soft_mask(logits: torch.Tensor, noise: Optional[torch.Tensor], tau: float, w: Optional[torch.Tensor],
+                     want_z: bool = True, want_w_eff: bool = True, stream=None):
+    """(z fp32 [G,6] or None, w_eff bf16 shaped like w or None): relaxed choice (Eq. 3) and effective
+    weights (Eq. 6 with the soft mask) of every group of four weights."""
+    _need_cuda(logits, noise, w)
+    G = logits.shape[0]
+    z = torch.empty((G, 6), dtype=torch.float32, device=logits.device) if want_z else None
+    w_eff = torch.empty_like(w) if want_w_eff else None
+    f = lib().ssconv_soft_mask
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p, ctypes.c_int64,
+                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    _check("ssconv_soft_mask", f(_ptr(logits), _ptr(noise), float(tau), _ptr(w), G, _ptr(z), _ptr(w_eff),
+                                 _stream(stream)))
+    return z, w_eff
+
+
+def ssconv_mask_grad(z: torch.Tensor, tau: float, w: torch.Tensor, g_w_eff: torch.Tensor,
+                     g_logits: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """dL/dlogits fp32 [G,6] from dL/dw_eff (fp32, the shape of w)."""
+    _need_cuda(z, w, g_w_eff, g_logits)
+    G = z.shape[0]
+    if g_logits is None:
+        g_logits = torch.empty((G, 6), dtype=torch.float32, device=z.device)
+    f = lib().ssconv_mask_grad
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                  ctypes.c_void_p, ctypes.c_void_p]
+    _check("ssconv_mask_grad", f(_ptr(z), float(tau), _ptr(w), _ptr(g_w_eff), G, _ptr(g_logits), _stream(stream)))
+    return g_logits
+
+
+def ssconv_wgrad_ws_bytes(desc: Desc) -> int:
+    n = ctypes.c_size_t()
+    f = lib().ssconv_wgrad_ws_bytes
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.POINTER(ctypes.c_size_t)]
+    _check("ssconv_wgrad_ws_bytes", f(ctypes.byref(desc), ctypes.byref(n)))
+    return int(n.value)
+
+
+def ssconv_wgrad(desc: Desc, x: torch.Tensor, dy: torch.Tensor, dw: Optional[torch.Tensor] = None,
+                 ws: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                 stream=None) -> torch.Tensor:
+    """Weight gradient fp32 [C_out,KH,KW,C_in] of the layer from its bf16 input x and output gradient dy."""
+    _need_cuda(x, dy, dw, ws, dev_status)
+    if dw is None:
+        dw = torch.empty((desc.C_out, desc.KH, desc.KW, desc.C_in), dtype=torch.float32, device=x.device)
+    if ws is None:
+        need = ssconv_wgrad_ws_bytes(desc)
+        ws = torch.empty((need,), dtype=torch.uint8, device=x.device) if need else None
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    f = lib().ssconv_wgrad
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                  ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p]
+    _check("ssconv_wgrad", f(ctypes.byref(desc), _ptr(x), _ptr(dy), _ptr(dw), _ptr(ws), ws_bytes, _ptr(dev_status),
+                             _stream(stream)))
+    return dw

@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libssconv.so")
-SOURCES = ["api.cu", "mask.cu", "pool.cu", "forward.cu"]
+SOURCES = ["api.cu", "mask.cu", "pool.cu", "train.cu", "wgrad.cu", "forward.cu"]
 HEADERS = ["layout.cuh", "sm100_ptx.cuh"]
 
 

@@ -24,6 +24,13 @@ int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* sp
                    int32_t* ring_groups);
 int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
                                  const float* bias, void* y, int32_t* dev_status, cudaStream_t stream);
+cudaError_t launch_soft_mask(const float* logits, const float* noise, float tau, const void* w, int64_t G, float* z,
+                             void* w_eff, cudaStream_t st);
+cudaError_t launch_mask_grad(const float* z, float tau, const void* w, const float* g_w_eff, int64_t G,
+                             float* g_logits, cudaStream_t st);
+int32_t launch_wgrad(const ssconv_desc_t& d, const void* x, const void* dy, float* dw, void* ws, size_t ws_bytes,
+                     int32_t* dev_status, cudaStream_t stream);
+int32_t wgrad_workspace_bytes(const ssconv_desc_t& d, size_t* bytes);
 }  // namespace ssconv
 
 #include <atomic>
@@ -217,6 +224,59 @@ int32_t ssconv_forward_dense_res(const ssconv_desc_t* desc, const void* x, const
   if (!aligned16(x) || !aligned16(w_bf16) || !aligned16(y) || !aligned16(residual)) return SSCONV_ERR_ALIGNMENT;
   return ssconv::launch_forward_dense(*desc, x, w_bf16, bias, residual, y, ws, ws_bytes, dev_status,
                                       (cudaStream_t)stream);
+}
+
+int32_t ssconv_soft_mask(const float* logits, const float* noise, float tau, const void* w_bf16, int64_t G, float* z,
+                         void* w_eff_bf16, void* stream) {
+  if (G < 0 || !(tau > 0.0f)) return SSCONV_ERR_BAD_DESC;
+  if (G == 0) return SSCONV_OK;
+  if (!logits || (w_eff_bf16 && !w_bf16) || (!z && !w_eff_bf16)) return SSCONV_ERR_NULL;
+  const uintptr_t all = reinterpret_cast<uintptr_t>(logits) | reinterpret_cast<uintptr_t>(noise) |
+                        reinterpret_cast<uintptr_t>(w_bf16) | reinterpret_cast<uintptr_t>(z) |
+                        reinterpret_cast<uintptr_t>(w_eff_bf16);
+  if (all & 7u) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_soft_mask(logits, noise, tau, w_bf16, G, z, w_eff_bf16, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_mask_grad(const float* z, float tau, const void* w_bf16, const float* g_w_eff, int64_t G,
+                         float* g_logits, void* stream) {
+  if (G < 0 || !(tau > 0.0f)) return SSCONV_ERR_BAD_DESC;
+  if (G == 0) return SSCONV_OK;
+  if (!z || !w_bf16 || !g_w_eff || !g_logits) return SSCONV_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(z) | reinterpret_cast<uintptr_t>(w_bf16) | reinterpret_cast<uintptr_t>(g_logits)) & 7u)
+    return SSCONV_ERR_ALIGNMENT;
+  if (!aligned16(g_w_eff)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_mask_grad(z, tau, w_bf16, g_w_eff, G, g_logits, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_wgrad_ws_bytes(const ssconv_desc_t* desc, size_t* bytes) {
+  if (!bytes) return SSCONV_ERR_NULL;
+  ssconv_desc_t d;
+  if (desc) {
+    d = *desc;
+    d.flags = 0;
+  }
+  int32_t rc = check_desc(desc ? &d : nullptr, true);
+  if (rc != SSCONV_OK) return rc;
+  return ssconv::wgrad_workspace_bytes(d, bytes);
+}
+
+int32_t ssconv_wgrad(const ssconv_desc_t* desc, const void* x, const void* dy, float* dw, void* ws, size_t ws_bytes,
+                     int32_t* dev_status, void* stream) {
+  ssconv_desc_t d;
+  if (desc) {
+    d = *desc;
+    d.flags = 0;  // bias and activation play no part in this gradient
+  }
+  int32_t rc = check_desc(desc ? &d : nullptr, true);
+  if (rc != SSCONV_OK) return rc;
+  if (!x || !dy || !dw) return SSCONV_ERR_NULL;
+  if (!aligned16(x) || !aligned16(dy) || !aligned16(dw) || !aligned16(ws)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_wgrad(d, x, dy, dw, ws, ws_bytes, dev_status, (cudaStream_t)stream);
 }
 
 int32_t ssconv_forward_static_ws(const ssconv_desc_t* desc, const void* x, const void* w_comp, const void* meta,

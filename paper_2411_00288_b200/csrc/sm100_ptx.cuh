@@ -48,7 +48,7 @@ __device__ __forceinline__ bool mbar_spin_a(uint32_t bar_addr, uint32_t parity, 
 // Out-of-line continuation of a wait that outlasted the fast spin: polls on, but never forever.
 // After `limit_cycles` SM clock cycles without completion, or as soon as another thread of the
 // CTA has raised *abort_flag, it gives up and returns false.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t parity, volatile int* abort_flag,
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar_addr, uint32_t parity, volatile int* abort_flag,
                                             long long limit_cycles, uint32_t backoff_ns) {
   const long long t0 = clock64();
   while (true) {

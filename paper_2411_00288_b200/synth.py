@@ -247,3 +247,22 @@ def make_inputs(spec: LayerSpec, seed: Optional[int] = None, x_only: bool = Fals
     elif spec.mask_source == "uniform_pattern":
         pattern = torch.randint(0, 6, (spec.G,), generator=g, dtype=torch.int64).to(torch.uint8)
     return LayerInputs(spec, x, w, bias, scores, pattern)
+
+
+@dataclass
+class TrainInputs:
+    logits: torch.Tensor   # fp32 [G,6]: the trainable choice weights (log pi up to a constant)
+    noise: torch.Tensor    # fp32 [G,6]: one Gumbel(0,1) draw per logit (the method's randomness, drawn here)
+    dy: torch.Tensor       # bf16 [N,H_out,W_out,C_out]: a stand-in for the loss gradient at the layer's output
+
+
+def make_train_inputs(spec: LayerSpec, seed: Optional[int] = None) -> TrainInputs:
+    """Seeded inputs of one mask-learning step for a layer (its own stream of the layer's seed).
+    The upstream gradient is N(0, 1/P) so that weight gradients stay O(1)."""
+    g = torch.Generator().manual_seed((spec.seed if seed is None else seed) + 70_000_000)
+    logits = torch.randn((spec.G, 6), generator=g, dtype=torch.float32)
+    u = torch.rand((spec.G, 6), generator=g, dtype=torch.float64).clamp_(1e-12, 1.0 - 1e-12)
+    noise = (-torch.log(-torch.log(u))).float()
+    dy = (torch.randn((spec.N, spec.H_out, spec.W_out, spec.C_out), generator=g, dtype=torch.float32)
+          / math.sqrt(spec.P)).to(torch.bfloat16)
+    return TrainInputs(logits, noise, dy)

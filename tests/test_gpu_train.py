@@ -1,0 +1,160 @@
+"""GPU parity of the mask-learning step's kernels (soft mask, weight gradient, gradient to the
+choice weights) against the fp64 oracle, on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import train as otrain
+from oracle.conv import ConvShape, conv2d_f64
+from paper_2411_00288_b200 import api, synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+# fp32 softmax against fp64: exp of an argument of magnitude a carries a relative error of about
+# a * 2^-24; z <= 1
+Z_ATOL, Z_RTOL = 1e-6, 3e-5
+# one rounding to bf16 (8 significant bits: half an ulp is at most 2^-8 of the value) on top of fp32 arithmetic
+WEFF_RTOL = 2.0 ** -8 * 1.01
+# fp32 accumulation of exact products over up to 1e5 positions
+WGRAD_REL_FRO, WGRAD_MAX_REL = 1e-4, 2e-4
+LGRAD_REL_FRO = 1e-4
+
+
+def _rel_fro(a, b):
+    d = np.linalg.norm(b.reshape(-1))
+    return float(np.linalg.norm((a - b).reshape(-1)) / d) if d > 0 else float(np.abs(a - b).max())
+
+
+@pytest.mark.parametrize("G,tau,with_noise", [(1, 1.0, True), (255, 0.1, True), (4097, 0.5, False),
+                                               (147456, 0.1, True), (589824, 2.0, True)])
+def test_soft_mask_matches_oracle(G, tau, with_noise):
+    g = torch.Generator().manual_seed(synth.SEED_BASE + 800 + G)
+    logits = torch.randn((G, 6), generator=g)
+    u = torch.rand((G, 6), generator=g, dtype=torch.float64).clamp_(1e-12, 1 - 1e-12)
+    noise = (-torch.log(-torch.log(u))).float() if with_noise else None
+    w = (torch.randn((G, 4), generator=g) * 0.05).to(torch.bfloat16)
+    z, w_eff = api.ssconv_soft_mask(logits.to(DEV), None if noise is None else noise.to(DEV), tau, w.to(DEV))
+    torch.cuda.synchronize()
+    z_ref = otrain.soft_choice(logits.numpy(), None if noise is None else noise.numpy(), tau)
+    zg = z.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(zg - z_ref) <= Z_ATOL + Z_RTOL * z_ref), float(np.abs(zg - z_ref).max())
+    we_ref = otrain.effective_weights(synth.bf16_bits(w), z_ref)
+    we = parity.bf16_tensor_to_f64(w_eff)
+    assert np.all(np.abs(we - we_ref) <= WEFF_RTOL * np.abs(we_ref) + 1e-30), float(np.abs(we - we_ref).max())
+
+
+def test_soft_mask_outputs_are_optional_and_tau_is_checked():
+    logits = torch.randn((64, 6)).to(DEV)
+    w = torch.randn((64, 4)).to(torch.bfloat16).to(DEV)
+    z, none = api.ssconv_soft_mask(logits, None, 0.3, w, want_w_eff=False)
+    assert none is None and z.shape == (64, 6)
+    none, w_eff = api.ssconv_soft_mask(logits, None, 0.3, w, want_z=False)
+    assert none is None and w_eff.shape == w.shape
+    with pytest.raises(api.SsconvError):
+        api.ssconv_soft_mask(logits, None, 0.0, w)
+
+
+@pytest.mark.parametrize("G,tau", [(3, 1.0), (1000, 0.1), (147456, 0.5)])
+def test_mask_grad_matches_oracle(G, tau):
+    g = torch.Generator().manual_seed(4242 + G)
+    logits = torch.randn((G, 6), generator=g)
+    w = (torch.randn((G, 4), generator=g) * 0.05).to(torch.bfloat16)
+    up = torch.randn((G, 4), generator=g)
+    z, _ = api.ssconv_soft_mask(logits.to(DEV), None, tau, w.to(DEV), want_w_eff=False)
+    gl = api.ssconv_mask_grad(z, tau, w.to(DEV), up.to(DEV))
+    torch.cuda.synchronize()
+    # the kernel alone: same z on both sides
+    ref_same_z = otrain.logit_grad(z.cpu().numpy(), tau, synth.bf16_bits(w), up.numpy())
+    assert _rel_fro(gl.cpu().numpy().astype(np.float64), ref_same_z) <= 1e-5
+    # the two kernels in sequence against the oracle's own z
+    ref = otrain.logit_grad(otrain.soft_choice(logits.numpy(), None, tau), tau, synth.bf16_bits(w), up.numpy())
+    assert _rel_fro(gl.cpu().numpy().astype(np.float64), ref) <= LGRAD_REL_FRO
+
+
+WG_SWEEP = [
+    # name                    N  H   W   Ci   Co  KH KW s  p  d
+    ("pw_64",                 2, 9,  7,  64,  64, 1, 1, 1, 0, 1),
+    ("pw_ragged_96to136",     3, 11, 5,  96, 136, 1, 1, 1, 0, 1),
+    ("pw_s2",                 2, 10, 10, 64, 128, 1, 1, 2, 0, 1),
+    ("c3_s1p1",               2, 12, 9,  64, 128, 3, 3, 1, 1, 1),
+    ("c3_s2p1",               2, 13, 12, 128, 64, 3, 3, 2, 1, 1),
+    ("c3_dil2",               1, 12, 12, 64,  64, 3, 3, 1, 2, 2),
+    ("c5_p2_c32",             1, 9,  9,  32,  40, 5, 5, 1, 2, 1),
+    ("c3_c8",                 2, 8,  8,  8,   8,  3, 3, 1, 1, 1),
+    ("c3_7x7_maps",           9, 7,  7,  128, 256, 3, 3, 1, 1, 1),
+    ("pw_deepK",              1, 6,  6,  1024, 64, 1, 1, 1, 0, 1),
+    ("one_pixel",             1, 1,  1,  8,   8,  1, 1, 1, 0, 1),
+    ("many_positions_split",  4, 40, 40, 64,  64, 3, 3, 1, 1, 1),
+    ("pw_many_positions",     2, 64, 50, 64,  128, 1, 1, 1, 0, 1),
+]
+
+
+def _check_wgrad(spec, seed=None):
+    inp = synth.make_inputs(spec, seed=seed, x_only=True)
+    tr = synth.make_train_inputs(spec, seed=seed)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    dw = api.ssconv_wgrad(api.desc_from_spec(spec), inp.x.to(DEV), tr.dy.to(DEV), dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = otrain.wgrad_f64(synth.bf16_bits(inp.x), synth.bf16_bits(tr.dy), spec.KH, spec.KW, spec.stride, spec.pad,
+                           spec.dil)
+    got = dw.cpu().numpy().astype(np.float64)
+    assert got.shape == ref.shape
+    return _rel_fro(got, ref), float(np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-30))
+
+
+@pytest.mark.parametrize("case", WG_SWEEP, ids=[c[0] for c in WG_SWEEP])
+def test_wgrad_shape_sweep(case):
+    name, N, H, W, Ci, Co, KH, KW, s, p, d = case
+    spec = synth.LayerSpec(name, N, H, W, Ci, Co, KH, KW, s, p, d, config=8, index=WG_SWEEP.index(case))
+    rel, mx = _check_wgrad(spec)
+    assert rel <= WGRAD_REL_FRO and mx <= WGRAD_MAX_REL, f"{name}: rel_fro={rel:.3e} max_rel={mx:.3e}"
+
+
+@pytest.mark.parametrize("index", [0, 1, 3, 4])
+def test_wgrad_resnet18_layers_full_size(index):
+    spec = [s for s in synth.config_layers(2) if not s.extra][index]
+    rel, mx = _check_wgrad(spec)
+    assert rel <= WGRAD_REL_FRO and mx <= WGRAD_MAX_REL, f"{spec.name}: rel_fro={rel:.3e} max_rel={mx:.3e}"
+
+
+def test_wgrad_workspace_is_required_when_positions_are_split():
+    spec = synth.config_layers(2)[0]
+    desc = api.desc_from_spec(spec)
+    assert api.ssconv_wgrad_ws_bytes(desc) > 0
+    x = torch.zeros((spec.N, spec.H, spec.W, spec.C_in), dtype=torch.bfloat16, device=DEV)
+    dy = torch.zeros((spec.N, spec.H_out, spec.W_out, spec.C_out), dtype=torch.bfloat16, device=DEV)
+    tiny = torch.empty((16,), dtype=torch.uint8, device=DEV)
+    with pytest.raises(api.SsconvError) as e:
+        api.ssconv_wgrad(desc, x, dy, ws=tiny)
+    assert e.value.status == 5
+
+
+def test_one_mask_learning_step_of_a_layer():
+    """soft mask -> dense forward with the effective weights -> weight gradient -> gradient of the
+    choice weights, each stage against the oracle fed with the same bits."""
+    spec = synth.LayerSpec("step", 4, 14, 14, 128, 128, 3, 3, 1, 1, 1, relu=False, has_bias=True, w_std="he",
+                           config=8, index=60)
+    tau = 0.5
+    inp = synth.make_inputs(spec)
+    tr = synth.make_train_inputs(spec)
+    desc = api.desc_from_spec(spec)
+    x, w = inp.x.to(DEV), inp.w.to(DEV)
+    z, w_eff = api.ssconv_soft_mask(tr.logits.to(DEV), tr.noise.to(DEV), tau, w)
+    y = api.ssconv_forward_dense(desc, x, w_eff, inp.bias.to(DEV))
+    dw = api.ssconv_wgrad(desc, x, tr.dy.to(DEV))
+    gl = api.ssconv_mask_grad(z, tau, w, dw)
+    torch.cuda.synchronize()
+    # forward: the oracle convolves with the effective weights the GPU rounded to bf16
+    shp = ConvShape(spec.N, spec.H, spec.W, spec.C_in, spec.C_out, 3, 3, (1, 1), (1, 1), (1, 1), relu=False)
+    y_ref = conv2d_f64(shp, synth.bf16_bits(inp.x), synth.bf16_bits(w_eff.cpu()), bias=inp.bias.numpy())
+    rel, mx = parity.errors(parity.bf16_tensor_to_f64(y), y_ref)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL
+    # backward: entirely from the oracle's own fp64 chain
+    z_ref = otrain.soft_choice(tr.logits.numpy(), tr.noise.numpy(), tau)
+    dw_ref = otrain.wgrad_f64(synth.bf16_bits(inp.x), synth.bf16_bits(tr.dy), 3, 3, 1, 1, 1)
+    gl_ref = otrain.logit_grad(z_ref, tau, synth.bf16_bits(inp.w), dw_ref)
+    assert _rel_fro(dw.cpu().numpy().astype(np.float64), dw_ref) <= WGRAD_REL_FRO
+    assert _rel_fro(gl.cpu().numpy().astype(np.float64), gl_ref) <= LGRAD_REL_FRO
