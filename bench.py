@@ -278,6 +278,143 @@ def stack_arm(args):
         dist.destroy_process_group()
 
 
+def train_arm(args):
+    """One mask-learning step per layer of the chosen layer set (Sec. 3.1): soft mask -> dense forward
+    with the effective weights -> weight gradient -> gradient of the choice weights, with a seeded
+    stand-in for the loss gradient.  Dense-equivalent TFLOP/s over the two convolutions' FLOPs, and a
+    per-layer table of the four kernels' device times.  One JSON line on rank 0."""
+    import torch
+    import torch.distributed as dist
+    from paper_2411_00288_b200 import api, synth, ranks, build as libbuild
+
+    rank, local_rank, world = ranks.env_ranks()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        libbuild.build()
+    if world > 1:
+        dist.barrier()
+    api.lib()
+    peaks = load_peaks()
+    tau = 0.5
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    prep = []
+    for spec in timed_layers():
+        inp = synth.make_inputs(spec)
+        tr = synth.make_train_inputs(spec)
+        desc = api.desc_from_spec(spec)
+        need = api.ssconv_wgrad_ws_bytes(desc)
+        prep.append(dict(
+            spec=spec, desc=desc, x=inp.x.to(dev), w=inp.w.to(dev), bias=inp.bias.to(dev),
+            logits=tr.logits.to(dev), noise=tr.noise.to(dev), dy=tr.dy.to(dev),
+            z=torch.empty((spec.G, 6), dtype=torch.float32, device=dev), w_eff=torch.empty_like(inp.w, device=dev),
+            y=torch.empty((spec.N, spec.H_out, spec.W_out, spec.C_out), dtype=torch.bfloat16, device=dev),
+            dw=torch.empty((spec.C_out, spec.KH, spec.KW, spec.C_in), dtype=torch.float32, device=dev),
+            ws=torch.empty((max(need, 16),), dtype=torch.uint8, device=dev),
+            gl=torch.empty((spec.G, 6), dtype=torch.float32, device=dev)))
+
+    kernels = {
+        "soft_mask": lambda L: api.ssconv_soft_mask(L["logits"], L["noise"], tau, L["w"], z=L["z"], w_eff=L["w_eff"]),
+        "forward": lambda L: api.ssconv_forward_dense(L["desc"], L["x"], L["w_eff"], L["bias"], y=L["y"],
+                                                      dev_status=status),
+        "wgrad": lambda L: api.ssconv_wgrad(L["desc"], L["x"], L["dy"], dw=L["dw"], ws=L["ws"], dev_status=status),
+        "mask_grad": lambda L: api.ssconv_mask_grad(L["z"], tau, L["w"], L["dw"], g_logits=L["gl"]),
+    }
+
+    def step():
+        for L in prep:
+            for k in kernels.values():
+                k(L)
+
+    warmup, steps = max(3, args.warmup), min(args.steps, 2000)
+    c0 = api.ssconv_launch_count()
+    step()
+    launches = api.ssconv_launch_count() - c0
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+
+    def replay_ms(fn, reps):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        g.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        return ranks.max_over_ranks(e0.elapsed_time(e1) / reps, dev)
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms_step = replay_ms(step, steps)
+    clocks = sampler.stop() if rank == 0 else None
+    per_layer = []
+    iters = 50
+    for L in prep:
+        spec = L["spec"]
+        row = {"layer": spec.name}
+        for name, k in kernels.items():
+            row["us_" + name] = round(replay_ms(lambda: [k(L) for _ in range(iters)], 5) / iters * 1e3, 2)
+        row["wgrad_tflops"] = round(spec.dense_equiv_flops / row["us_wgrad"] / 1e6, 1)
+        row["wgrad_frac_of_dense_peak"] = round(row["wgrad_tflops"] / peaks["bf16_tflops"], 4)
+        # soft_mask moves 88 bytes per group (logits, noise, weights in; z, effective weights out),
+        # mask_grad 72 (z, weights, weight gradient in; logit gradient out)
+        row["soft_mask_gbs"] = round(88 * spec.G / row["us_soft_mask"] / 1e3, 1)
+        row["mask_grad_gbs"] = round(72 * spec.G / row["us_mask_grad"] / 1e3, 1)
+        per_layer.append(row)
+    # the two elementwise kernels on as many groups as a whole ResNet-50 has (5.9 M: 0.5 GB of
+    # traffic, beyond L2), where their HBM roofline applies
+    Gb = 5_900_000
+    gen = torch.Generator().manual_seed(synth.SEED_BASE + 4711)
+    big = dict(logits=torch.randn((Gb, 6), generator=gen).to(dev), noise=torch.randn((Gb, 6), generator=gen).to(dev),
+               w=torch.randn((Gb, 4), generator=gen).to(torch.bfloat16).to(dev),
+               dw=torch.randn((Gb, 4), generator=gen).to(dev),
+               z=torch.empty((Gb, 6), dtype=torch.float32, device=dev),
+               w_eff=torch.empty((Gb, 4), dtype=torch.bfloat16, device=dev),
+               gl=torch.empty((Gb, 6), dtype=torch.float32, device=dev))
+    us_sm = replay_ms(lambda: [api.ssconv_soft_mask(big["logits"], big["noise"], tau, big["w"], z=big["z"],
+                                                    w_eff=big["w_eff"]) for _ in range(10)], 5) / 10 * 1e3
+    us_mg = replay_ms(lambda: [api.ssconv_mask_grad(big["z"], tau, big["w"], big["dw"], g_logits=big["gl"])
+                               for _ in range(10)], 5) / 10 * 1e3
+    elementwise = {"groups": Gb, "us_soft_mask": round(us_sm, 1), "us_mask_grad": round(us_mg, 1),
+                   "soft_mask_gbs": round(88 * Gb / us_sm / 1e3, 1), "mask_grad_gbs": round(72 * Gb / us_mg / 1e3, 1),
+                   "soft_mask_frac_of_hbm_peak": round(88 * Gb / us_sm / 1e3 / peaks["hbm_gbs"], 4),
+                   "mask_grad_frac_of_hbm_peak": round(72 * Gb / us_mg / 1e3 / peaks["hbm_gbs"], 4),
+                   "bytes_per_group": {"soft_mask": 88, "mask_grad": 72}}
+    flops = 2 * sum(L["spec"].dense_equiv_flops for L in prep)
+    if rank == 0:
+        wg_ms = sum(r["us_wgrad"] for r in per_layer) * 1e-3
+        wg_tflops = sum(L["spec"].dense_equiv_flops for L in prep) / (wg_ms * 1e-3) / 1e12
+        print(json.dumps({
+            "metric": "TFLOP/s of one mask-learning step per layer (dense forward with soft-masked weights + weight "
+                      "gradient; bf16, fp32 accumulate)",
+            "value": ranks.job_throughput(flops, world, ms_step) / 1e12, "unit": "TFLOP/s", "n_gpus": world,
+            "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD + "_mask_learning_step", "layers": len(prep), "tau": tau,
+                       "batch_per_gpu": prep[0]["spec"].N,
+                       "launch": "the step's C-ABI calls recorded into one CUDA graph and replayed",
+                       "l2": "one buffer set (the step's tensors total more than L2 only for the larger layer sets)"},
+            "roofline": {"bound": "tensor", "kernel": "ssconv_wgrad_kernel", "achieved": wg_tflops,
+                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": wg_tflops / peaks["bf16_tflops"],
+                         "peak_source": f"dense bf16 burst of {peaks['source']} peaks", "traffic": None},
+            "per_layer": per_layer, "elementwise_at_resnet50_size": elementwise,
+            "gpu_launches": steps * launches, "clocks": clocks, "dev_status": int(status.item())}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ----------------------------------------------------------------------------- GPU arm
 def main():
     global CONFIG_ID, WORKLOAD
@@ -293,6 +430,9 @@ def main():
     ap.add_argument("--dense", action="store_true", help="with --only-layer: use the dense kernel")
     ap.add_argument("--residual", action="store_true",
                     help="with --workload-config 5: fuse the network's skip connections into the expand convolutions")
+    ap.add_argument("--train", action="store_true",
+                    help="time one mask-learning step per layer (soft mask, dense forward, weight gradient, "
+                         "choice-weight gradient) instead of the inference sweep")
     ap.add_argument("--batch", type=int, default=None, help="with --workload-config 5: images per GPU (default 256)")
     ap.add_argument("--workload-config", type=int, default=CONFIG_ID, choices=sorted(WORKLOADS),
                     help="layer set to run (default: the benchmarked ResNet-18 sweep)")
@@ -304,6 +444,9 @@ def main():
         return
     if CONFIG_ID == 5:
         stack_arm(args)
+        return
+    if args.train:
+        train_arm(args)
         return
 
     import torch

@@ -209,10 +209,10 @@ int32_t ssconv_mask_grad(const float* z, float tau, const void* w_bf16, const fl
  * gradient of its output [N,H_out,W_out,C_out]; dw: fp32 [C_out,KH,KW,C_in], every element written.
  * Products are exact, accumulation is fp32 on the tensor cores.  flags of desc are ignored.
  * Shape rules as ssconv_forward_dense.  x, dy, dw, ws: device, 16-byte aligned.
- * ws: scratch of at least ssconv_wgrad_ws_bytes (0 for layers with enough work per SM; ws may then
- * be NULL): layers with few weights and many positions split the positions over thread blocks,
- * which store partial gradients there; a second kernel adds them in a fixed order.  Needs no
- * initialisation.  dev_status: as in ssconv_forward. */
+ * ws: scratch of at least ssconv_wgrad_ws_bytes, always needed: thread blocks store partial
+ * gradients there (one slice per range of positions; layers with few weights and many positions
+ * split the positions over thread blocks), and a second kernel adds the slices in a fixed order
+ * and writes dw.  Needs no initialisation.  dev_status: as in ssconv_forward. */
 int32_t ssconv_wgrad(const ssconv_desc_t* desc, const void* x, const void* dy, float* dw, void* ws,
                      size_t ws_bytes, int32_t* dev_status, void* stream);
 /* Scratch bytes ssconv_wgrad needs for this layer on the current device. */

@@ -299,13 +299,16 @@ def ssconv_forward_static_ws(desc: Desc, x: torch.Tensor, w_comp: torch.Tensor, 
 
 
 def ssconv_soft_mask(logits: torch.Tensor, noise: Optional[torch.Tensor], tau: float, w: Optional[torch.Tensor],
-                     want_z: bool = True, want_w_eff: bool = True, stream=None):
+                     want_z: bool = True, want_w_eff: bool = True, stream=None,
+                     z: Optional[torch.Tensor] = None, w_eff: Optional[torch.Tensor] = None):
     """(z fp32 [G,6] or None, w_eff bf16 shaped like w or None): relaxed choice (Eq. 3) and effective
-    weights (Eq. 6 with the soft mask) of every group of four weights."""
-    _need_cuda(logits, noise, w)
+    weights (Eq. 6 with the soft mask) of every group of four weights.  Output tensors may be passed in."""
+    _need_cuda(logits, noise, w, z, w_eff)
     G = logits.shape[0]
-    z = torch.empty((G, 6), dtype=torch.float32, device=logits.device) if want_z else None
-    w_eff = torch.empty_like(w) if want_w_eff else None
+    if z is None and want_z:
+        z = torch.empty((G, 6), dtype=torch.float32, device=logits.device)
+    if w_eff is None and want_w_eff:
+        w_eff = torch.empty_like(w)
     f = lib().ssconv_soft_mask
     f.restype = ctypes.c_int32
     f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p, ctypes.c_int64,

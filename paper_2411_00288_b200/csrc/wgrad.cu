@@ -16,11 +16,14 @@
 // to four taps.
 //
 // A CTA owns one work item: 128 output channels x T k-blocks x one range of positions, and walks
-// its positions 64 at a time through a 4-stage TMA ring (two producer threads, one MMA thread,
-// four epilogue warps, fp32 accumulator of 64 T columns in TMEM).  When the position range is
-// split (few items, many positions) every CTA writes its partial dW to a slice of the scratch
-// buffer and a second kernel adds the slices in a fixed order: the result does not depend on
-// timing.  All mbarrier waits are bounded (see sm100_ptx.cuh).
+// its positions 64 at a time through a 4-stage TMA ring (four producer threads, one MMA thread,
+// four epilogue warps, fp32 accumulator of 64 T columns in TMEM).  The accumulator has output
+// channels on TMEM lanes, so an epilogue thread holds one row of dW: it writes to a scratch slice
+// laid out [tile of 128 output channels][K][128], where the 32 lanes of a warp store 128 contiguous
+// bytes and a CTA's whole output is one contiguous block.  A second kernel
+// adds the slices of all position ranges in a fixed order (the result does not depend on timing)
+// and transposes 32 x 32 tiles through shared memory into dW [C_out][K].  All mbarrier waits are
+// bounded (see sm100_ptx.cuh).
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -30,7 +33,7 @@
 
 namespace ssconv {
 
-constexpr int kWgThreads = 224;        // warp 0 and 6: TMA producers, warp 1: MMA, warps 2-5: epilogue
+constexpr int kWgThreads = 288;        // warps 0, 6, 7, 8: TMA producers, warp 1: MMA, warps 2-5: epilogue
 constexpr int kWgPos = 64;             // positions per ring stage
 constexpr int kWgMaxT = 4;             // k-blocks per work item (N = 64 T <= 256)
 constexpr int kWgStages = 4;
@@ -48,7 +51,8 @@ struct WgParams {
   int m_tiles;
   int splits;              // position ranges
   int ksteps, ksteps_per_split;  // steps of 64 positions: in all, per range
-  float* out;              // dW [C_out][taps][C_in] when splits == 1, else `splits` such slices
+  int dy_one_load;         // C_out % 64 == 0: both halves of a gradient tile come with one 3-D load
+  float* out;              // `splits` slices [m_tiles][taps * C_in][128] of partial gradients
   int32_t* dev_status;
 };
 
@@ -104,12 +108,12 @@ ssconv_wgrad_kernel(const __grid_constant__ CUtensorMap tm_dy, const __grid_cons
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const WgItem item = wg_item(p);
-  const bool second_producer = item.nb > 1;
+  const uint32_t producers = 1u + (uint32_t)min(item.nb, 3);  // roles that load something
 
   if (warp == 0) {
     if (lane == 0) {
       for (int s = 0; s < kWgStages; ++s) {
-        mbar_init(&bar_full[s], second_producer ? 2u : 1u);
+        mbar_init(&bar_full[s], producers);
         mbar_init(&bar_empty[s], 1u);
       }
       mbar_init(bar_acc, 1u);
@@ -130,39 +134,46 @@ ssconv_wgrad_kernel(const __grid_constant__ CUtensorMap tm_dy, const __grid_cons
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty), ring0 = smem_u32(smem);
 
-  if (warp == 0 || warp == 6) {
+  if (warp == 0 || warp >= 6) {
     // ------------------------------------------------------------------ TMA producers
-    // warp 0: both halves of the gradient tile and the first activation tile; warp 6: the other
-    // activation tiles (a TMA instruction occupies its thread for a few hundred cycles)
-    if (lane == 0 && (warp == 0 || second_producer)) {
-      const int first = (warp == 0) ? 0 : 1;
-      const int last = (warp == 0) ? 1 : item.nb;
+    // A TMA instruction occupies its thread for a few hundred cycles, so the loads of a stage are
+    // spread over four threads: role 0 the gradient tile, roles 1-3 the activation tiles
+    // (role 1 also the fourth one).
+    const int role = (warp == 0) ? 0 : warp - 5;
+    if (lane == 0 && role < (int)producers) {
       uint32_t s = 0, ph = 0;
       for (int ks = item.ks0; ks < item.ks1; ++ks) {
         if (!mbar_wait_a(empty0 + 8u * s, ph ^ 1u, abort_flag, kWgWaitLimitCycles)) break;
         const uint32_t full = full0 + 8u * s;
         const uint32_t dst = ring0 + s * kWgStageBytes;
         const int q0 = ks * kWgPos;
-        const int rho = q0 / p.Wo;
-        const int wo = q0 - rho * p.Wo;
-        const int n = rho / p.Ho;
-        const int ho = rho - n * p.Ho;
-        const int base_w = wo * p.stride_w - p.pad_w;
-        const int base_h = ho * p.stride_h - p.pad_h;
-        mbar_expect_tx_a(full, (uint32_t)(last - first + (warp == 0 ? 2 : 0)) * kWgTileBytes);
-        if (warp == 0) {
+        if (role == 0) {
           // channels beyond C_out and positions beyond Q lie outside the tensor map: zeros
-          tma_load_2d_a(dst, &tm_dy, full, item.m * kTileM, q0);
-          tma_load_2d_a(dst + kWgTileBytes, &tm_dy, full, item.m * kTileM + 64, q0);
-        }
-        for (int t = first; t < last; ++t) {
-          const int b = item.b0 + t;
-          const int cc = b / p.taps;
-          const int tap = b - cc * p.taps;
-          const int kh = tap / p.KW;
-          const int kw = tap - kh * p.KW;
-          tma_load_im2col_4d_a(dst + (uint32_t)(2 + t) * kWgTileBytes, &tm_x, full, cc * kBlockK, base_w, base_h, n,
-                               (uint16_t)(kw * p.dil_w), (uint16_t)(kh * p.dil_h));
+          mbar_expect_tx_a(full, 2u * kWgTileBytes);
+          if (p.dy_one_load) {
+            tma_load_3d_a(dst, &tm_dy, full, 0, q0, 2 * item.m);
+          } else {
+            tma_load_2d_a(dst, &tm_dy, full, item.m * kTileM, q0);
+            tma_load_2d_a(dst + kWgTileBytes, &tm_dy, full, item.m * kTileM + 64, q0);
+          }
+        } else {
+          const int rho = q0 / p.Wo;
+          const int wo = q0 - rho * p.Wo;
+          const int n = rho / p.Ho;
+          const int ho = rho - n * p.Ho;
+          const int base_w = wo * p.stride_w - p.pad_w;
+          const int base_h = ho * p.stride_h - p.pad_h;
+          const bool two = (role == 1 && item.nb > 3);
+          mbar_expect_tx_a(full, two ? 2u * kWgTileBytes : kWgTileBytes);
+          for (int t = role - 1; t < item.nb; t += 3) {
+            const int b = item.b0 + t;
+            const int cc = b / p.taps;
+            const int tap = b - cc * p.taps;
+            const int kh = tap / p.KW;
+            const int kw = tap - kh * p.KW;
+            tma_load_im2col_4d_a(dst + (uint32_t)(2 + t) * kWgTileBytes, &tm_x, full, cc * kBlockK, base_w, base_h,
+                                 n, (uint16_t)(kw * p.dil_w), (uint16_t)(kh * p.dil_h));
+          }
         }
         if (++s == kWgStages) {
           s = 0;
@@ -198,33 +209,29 @@ ssconv_wgrad_kernel(const __grid_constant__ CUtensorMap tm_dy, const __grid_cons
   } else if (warp < 6) {
     // ------------------------------------------------------------------ epilogue
     const int qd = warp & 3;  // TMEM lane quadrant of this warp
-    const int co = item.m * kTileM + qd * 32 + lane;
     // the TMEM loads below are warp-wide: the warp goes on only if every lane saw the barrier complete
     const bool got =
         __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar_acc, 0u, abort_flag, kWgWaitLimitCycles, 64) ? 1 : 0) != 0;
     if (got) {
       tc_fence_after();
-      const size_t slice = (size_t)p.C_out * p.taps * p.C_in;
-      float* out = p.out + (size_t)item.split * slice;
+      const size_t K = (size_t)p.taps * p.C_in;
+      float* out = p.out + ((size_t)item.split * p.m_tiles + item.m) * K * kTileM + qd * 32 + lane;
       for (int t = 0; t < item.nb; ++t) {
         const int b = item.b0 + t;
         const int cc = b / p.taps;
         const int tap = b - cc * p.taps;
-        float* row = out + ((size_t)co * p.taps + tap) * p.C_in + cc * kBlockK;
+        // column c of this k-block is row tap * C_in + 64 cc + c of the tile's [K][128] block
+        // (rows of output channels beyond C_out hold zeros: their gradient rows were zero-filled)
+        float* col0 = out + ((size_t)tap * p.C_in + cc * kBlockK) * kTileM;
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
           uint32_t r[32];
           tc_ld_32x32b_x32(tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(64 * t + 32 * half), r);
           tc_wait_ld();
-          if (co < p.C_out) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const int ci = cc * kBlockK + 32 * half + 4 * j;
-              if (ci < p.C_in)  // C_in is a multiple of 8: a float4 never straddles the end
-                *reinterpret_cast<float4*>(row + 32 * half + 4 * j) =
-                    make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
-            }
+          for (int j = 0; j < 32; ++j) {
+            const int c = 32 * half + j;
+            if (cc * kBlockK + c < p.C_in) col0[(size_t)c * kTileM] = __uint_as_float(r[j]);
           }
         }
       }
@@ -246,19 +253,34 @@ ssconv_wgrad_kernel(const __grid_constant__ CUtensorMap tm_dy, const __grid_cons
   }
 }
 
-// dW = sum over the position ranges' slices, in slice order.
-__global__ void wgrad_reduce_kernel(const float4* __restrict__ slices, int splits, size_t vecs, float4* __restrict__ dw) {
-  const size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x;
-  if (i >= vecs) return;
-  float4 acc = slices[i];
-  for (int s = 1; s < splits; ++s) {
-    const float4 v = slices[(size_t)s * vecs + i];
-    acc.x += v.x;
-    acc.y += v.y;
-    acc.z += v.z;
-    acc.w += v.w;
+// dW [C_out][K] = transpose of the sum, in slice order, of the slices [m_tiles][K][128].  A block
+// of 32 x 8 threads handles 32 output channels x 8 columns of K, one element per thread: reads are
+// contiguous along the output channels, writes go out as 32-byte runs along K.  With many slices
+// the sums are latency-bound, hence the small tiles (many blocks) and eight loads in flight.
+__global__ void wgrad_reduce_kernel(const float* __restrict__ slices, int splits, int K, int C_out, int m_tiles,
+                                    float* __restrict__ dw) {
+  __shared__ float tile[8][33];
+  const int k0 = blockIdx.x * 8, c0 = blockIdx.y * 32;
+  const size_t slice = (size_t)m_tiles * K * kTileM;
+  const int c = c0 + threadIdx.x, k = k0 + threadIdx.y;
+  float acc = 0.0f;
+  if (k < K && c < C_out) {
+    const float* src = slices + ((size_t)(c / kTileM) * K + k) * kTileM + (c % kTileM);
+    int s = 0;
+    for (; s + 8 <= splits; s += 8) {  // eight loads in flight, added in slice order
+      float v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = src[(size_t)(s + j) * slice];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc += v[j];
+    }
+    for (; s < splits; ++s) acc += src[(size_t)s * slice];
   }
-  dw[i] = acc;
+  tile[threadIdx.y][threadIdx.x] = acc;
+  __syncthreads();
+  const int t = threadIdx.y * 32 + threadIdx.x;
+  const int cl = t >> 3, kl = t & 7;
+  if (k0 + kl < K && c0 + cl < C_out) dw[(size_t)(c0 + cl) * K + k0 + kl] = tile[kl][cl];
 }
 
 // ---------------------------------------------------------------------------------------
@@ -336,13 +358,13 @@ int wg_sm_count(int* sms) {
 
 }  // namespace
 
-// Scratch the layer's weight gradient needs on the current device (0 when positions are not split).
+// Scratch the layer's weight gradient needs on the current device: one slice per position range.
 int32_t wgrad_workspace_bytes(const ssconv_desc_t& d, size_t* bytes) {
   int sms = 0;
   const int32_t st = wg_sm_count(&sms);
   if (st != SSCONV_OK) return st;
   const WgPlan w = wg_plan(d, sms);
-  *bytes = w.splits > 1 ? (size_t)w.splits * d.C_out * w.taps * d.C_in * sizeof(float) : 0;
+  *bytes = (size_t)w.splits * w.m_tiles * kTileM * w.taps * d.C_in * sizeof(float);
   return SSCONV_OK;
 }
 
@@ -364,22 +386,36 @@ int32_t launch_wgrad(const ssconv_desc_t& d, const void* x, const void* dy, floa
   }
   const WgPlan w = wg_plan(d, sms);
   if (w.Q > 0x7FFFFF00LL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
-  const size_t slice_bytes = (size_t)d.C_out * w.taps * d.C_in * sizeof(float);
-  if (w.splits > 1 && (ws == nullptr || ws_bytes < (size_t)w.splits * slice_bytes)) return SSCONV_ERR_WORKSPACE;
+  const size_t slice_bytes = (size_t)w.m_tiles * kTileM * w.taps * d.C_in * sizeof(float);
+  if (ws == nullptr || ws_bytes < (size_t)w.splits * slice_bytes) return SSCONV_ERR_WORKSPACE;
   const int Ho = wg_out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h);
   const int Wo = wg_out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
 
   CUtensorMap tm_dy, tm_x;
   {
-    // gradient of the output, NHWC seen as (c, position); a box is 64 channels x 64 positions
-    cuuint64_t dims[2] = {(cuuint64_t)d.C_out, (cuuint64_t)w.Q};
-    cuuint64_t strides[1] = {(cuuint64_t)d.C_out * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kWgPos};
-    cuuint32_t estr[2] = {1, 1};
-    if (wg_encode_tiled(&tm_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(dy), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return SSCONV_ERR_CUDA;
+    // gradient of the output, NHWC seen as (c, position); a box is 64 channels x 64 positions.  When
+    // C_out is a multiple of 64 the view is (64 channels, position, block of 64 channels) instead, so
+    // that one box of 64 x 64 x 2 brings both halves of a 128-channel tile, half after half.
+    const bool one_load = d.C_out % 64 == 0;
+    CUresult r;
+    if (one_load) {
+      cuuint64_t dims[3] = {64, (cuuint64_t)w.Q, (cuuint64_t)(d.C_out / 64)};
+      cuuint64_t strides[2] = {(cuuint64_t)d.C_out * 2, 128};
+      cuuint32_t box[3] = {64, (cuuint32_t)kWgPos, 2};
+      cuuint32_t estr[3] = {1, 1, 1};
+      r = wg_encode_tiled(&tm_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(dy), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+      cuuint64_t dims[2] = {(cuuint64_t)d.C_out, (cuuint64_t)w.Q};
+      cuuint64_t strides[1] = {(cuuint64_t)d.C_out * 2};
+      cuuint32_t box[2] = {64, (cuuint32_t)kWgPos};
+      cuuint32_t estr[2] = {1, 1};
+      r = wg_encode_tiled(&tm_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(dy), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
   }
   {
     // activations: NHWC seen as (c, w, h, n) in im2col mode, as in the forward kernel: base pixels
@@ -419,17 +455,19 @@ int32_t launch_wgrad(const ssconv_desc_t& d, const void* x, const void* dy, floa
   p.splits = w.splits;
   p.ksteps = w.ksteps;
   p.ksteps_per_split = w.ksteps_per_split;
-  p.out = w.splits > 1 ? static_cast<float*>(ws) : dw;
+  p.dy_one_load = (d.C_out % 64 == 0) ? 1 : 0;
+  p.out = static_cast<float*>(ws);
   p.dev_status = dev_status;
 
   const unsigned grid = (unsigned)(w.splits * w.m_tiles * w.items_b);
   ssconv_wgrad_kernel<<<grid, kWgThreads, kWgSmemBytes, stream>>>(tm_dy, tm_x, p);
   count_launch();
   if (cudaGetLastError() != cudaSuccess) return SSCONV_ERR_CUDA;
-  if (w.splits > 1) {
-    const size_t vecs = slice_bytes / sizeof(float4);
-    wgrad_reduce_kernel<<<(unsigned)((vecs + 255) / 256), 256, 0, stream>>>(static_cast<const float4*>(ws), w.splits,
-                                                                             vecs, reinterpret_cast<float4*>(dw));
+  {
+    const int K = w.taps * d.C_in;
+    const dim3 rgrid((unsigned)((K + 7) / 8), (unsigned)((d.C_out + 31) / 32));
+    wgrad_reduce_kernel<<<rgrid, dim3(32, 8), 0, stream>>>(static_cast<const float*>(ws), w.splits, K, d.C_out,
+                                                           w.m_tiles, dw);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return SSCONV_ERR_CUDA;
   }
