@@ -23,6 +23,10 @@ What it restates (Sec. 3.1 and Sec. 3.3 of the paper):
   sum over images and output pixels of dL/dy[n, ho, wo, co] x[n, ho s - p + kh d,
   wo s - p + kw d, ci], pixels outside the image contributing nothing (they are the zero
   padding).
+* The choice weights are updated with AdamW (Appendix, training details: learning rate 1.0,
+  momentum 0.9, weight decay 1e-4).  The update is the published one (decoupled weight decay):
+  m <- b1 m + (1 - b1) g,  v <- b2 v + (1 - b2) g^2,  theta <- theta - lr (mhat / (sqrt(vhat) + eps)
+  + wd theta) with the bias-corrected mhat = m / (1 - b1^t), vhat = v / (1 - b2^t).
 """
 from __future__ import annotations
 
@@ -98,3 +102,15 @@ def wgrad_f64(x_bits: np.ndarray, dy_bits: np.ndarray, KH: int, KW: int, stride:
             xs = xp[:, h0:h0 + stride * (Ho - 1) + 1:stride, w0:w0 + stride * (Wo - 1) + 1:stride, :]
             dw[:, kh, kw, :] = dy2.T @ xs.reshape(-1, C_in)
     return dw
+
+
+def adamw_step(theta, g, m, v, step: int, lr: float, beta1: float, beta2: float, eps: float, wd: float):
+    """One AdamW update in fp64; `step` counts from 1.  Returns (theta, m, v) as new arrays."""
+    theta = np.asarray(theta, dtype=np.float64)
+    g = np.asarray(g, dtype=np.float64)
+    m = beta1 * np.asarray(m, dtype=np.float64) + (1.0 - beta1) * g
+    v = beta2 * np.asarray(v, dtype=np.float64) + (1.0 - beta2) * g * g
+    mhat = m / (1.0 - beta1 ** step)
+    vhat = v / (1.0 - beta2 ** step)
+    theta = theta - lr * (mhat / (np.sqrt(vhat) + eps) + wd * theta)
+    return theta, m, v

@@ -209,3 +209,28 @@ def test_wgrad_of_a_1x1_filter_is_a_plain_matrix_product():
     dw = train.wgrad_f64(x, dy, 1, 1, 1, 0, 1)
     ref = bf16_to_f64(dy).reshape(-1, 6).T @ bf16_to_f64(x).reshape(-1, 8)
     np.testing.assert_allclose(dw.reshape(6, 8), ref, rtol=1e-13)
+
+
+# ---------------------------------------------------------------- optimiser of the choice weights
+def test_adamw_step_matches_the_library_optimiser_over_several_steps():
+    import torch
+    rng = np.random.default_rng(11)
+    theta0 = rng.normal(size=(40, 6))
+    grads = [rng.normal(size=(40, 6)) * (0.1 + 0.3 * i) for i in range(5)]
+    lr, b1, b2, eps, wd = 0.05, 0.9, 0.999, 1e-8, 1e-2
+    t = torch.tensor(theta0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.AdamW([t], lr=lr, betas=(b1, b2), eps=eps, weight_decay=wd)
+    theta, m, v = theta0, np.zeros_like(theta0), np.zeros_like(theta0)
+    for i, g in enumerate(grads, start=1):
+        t.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        theta, m, v = train.adamw_step(theta, g, m, v, i, lr, b1, b2, eps, wd)
+        np.testing.assert_allclose(theta, t.detach().numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_adamw_first_step_is_a_signed_unit_step_without_decay():
+    g = np.array([3.0, -0.2, 1e-3])
+    theta, m, v = train.adamw_step(np.zeros(3), g, np.zeros(3), np.zeros(3), 1, 0.5, 0.9, 0.999, 0.0, 0.0)
+    np.testing.assert_allclose(theta, -0.5 * np.sign(g), rtol=1e-12)
+    np.testing.assert_allclose(m, 0.1 * g, rtol=1e-12)
+    np.testing.assert_allclose(v, 0.001 * g * g, rtol=1e-9)
