@@ -280,8 +280,8 @@ def stack_arm(args):
 
 def train_arm(args):
     """One mask-learning step per layer of the chosen layer set (Sec. 3.1): soft mask -> dense forward
-    with the effective weights -> weight gradient -> gradient of the choice weights, with a seeded
-    stand-in for the loss gradient.  Dense-equivalent TFLOP/s over the two convolutions' FLOPs, and a
+    with the effective weights -> weight gradient -> gradient of the choice weights -> AdamW on them,
+    with a seeded stand-in for the loss gradient.  Dense-equivalent TFLOP/s over the two convolutions' FLOPs, and a
     per-layer table of the four kernels' device times.  One JSON line on rank 0."""
     import torch
     import torch.distributed as dist
@@ -313,7 +313,9 @@ def train_arm(args):
             y=torch.empty((spec.N, spec.H_out, spec.W_out, spec.C_out), dtype=torch.bfloat16, device=dev),
             dw=torch.empty((spec.C_out, spec.KH, spec.KW, spec.C_in), dtype=torch.float32, device=dev),
             ws=torch.empty((max(need, 16),), dtype=torch.uint8, device=dev),
-            gl=torch.empty((spec.G, 6), dtype=torch.float32, device=dev)))
+            gl=torch.empty((spec.G, 6), dtype=torch.float32, device=dev),
+            m=torch.zeros((spec.G, 6), dtype=torch.float32, device=dev),
+            v=torch.zeros((spec.G, 6), dtype=torch.float32, device=dev)))
 
     kernels = {
         "soft_mask": lambda L: api.ssconv_soft_mask(L["logits"], L["noise"], tau, L["w"], z=L["z"], w_eff=L["w_eff"]),
@@ -321,6 +323,8 @@ def train_arm(args):
                                                       dev_status=status),
         "wgrad": lambda L: api.ssconv_wgrad(L["desc"], L["x"], L["dy"], dw=L["dw"], ws=L["ws"], dev_status=status),
         "mask_grad": lambda L: api.ssconv_mask_grad(L["z"], tau, L["w"], L["dw"], g_logits=L["gl"]),
+        # (a small learning rate: the timed replays repeat the update hundreds of times on the same gradient)
+        "adamw": lambda L: api.ssconv_adamw(L["logits"], L["gl"], L["m"], L["v"], 1, lr=1e-3),
     }
 
     def step():
@@ -372,6 +376,7 @@ def train_arm(args):
         # mask_grad 72 (z, weights, weight gradient in; logit gradient out)
         row["soft_mask_gbs"] = round(88 * spec.G / row["us_soft_mask"] / 1e3, 1)
         row["mask_grad_gbs"] = round(72 * spec.G / row["us_mask_grad"] / 1e3, 1)
+        row["adamw_gbs"] = round(28 * 6 * spec.G / row["us_adamw"] / 1e3, 1)
         per_layer.append(row)
     # the two elementwise kernels on as many groups as a whole ResNet-50 has (5.9 M: 0.5 GB of
     # traffic, beyond L2), where their HBM roofline applies
@@ -382,16 +387,22 @@ def train_arm(args):
                dw=torch.randn((Gb, 4), generator=gen).to(dev),
                z=torch.empty((Gb, 6), dtype=torch.float32, device=dev),
                w_eff=torch.empty((Gb, 4), dtype=torch.bfloat16, device=dev),
-               gl=torch.empty((Gb, 6), dtype=torch.float32, device=dev))
+               gl=torch.randn((Gb, 6), generator=gen).to(dev),
+               m=torch.zeros((Gb, 6), dtype=torch.float32, device=dev),
+               v=torch.zeros((Gb, 6), dtype=torch.float32, device=dev))
     us_sm = replay_ms(lambda: [api.ssconv_soft_mask(big["logits"], big["noise"], tau, big["w"], z=big["z"],
                                                     w_eff=big["w_eff"]) for _ in range(10)], 5) / 10 * 1e3
     us_mg = replay_ms(lambda: [api.ssconv_mask_grad(big["z"], tau, big["w"], big["dw"], g_logits=big["gl"])
                                for _ in range(10)], 5) / 10 * 1e3
+    us_ad = replay_ms(lambda: [api.ssconv_adamw(big["logits"], big["gl"], big["m"], big["v"], 1, lr=1e-3)
+                               for _ in range(10)], 5) / 10 * 1e3
     elementwise = {"groups": Gb, "us_soft_mask": round(us_sm, 1), "us_mask_grad": round(us_mg, 1),
+                   "us_adamw": round(us_ad, 1), "adamw_gbs": round(28 * 6 * Gb / us_ad / 1e3, 1),
+                   "adamw_frac_of_hbm_peak": round(28 * 6 * Gb / us_ad / 1e3 / peaks["hbm_gbs"], 4),
                    "soft_mask_gbs": round(88 * Gb / us_sm / 1e3, 1), "mask_grad_gbs": round(72 * Gb / us_mg / 1e3, 1),
                    "soft_mask_frac_of_hbm_peak": round(88 * Gb / us_sm / 1e3 / peaks["hbm_gbs"], 4),
                    "mask_grad_frac_of_hbm_peak": round(72 * Gb / us_mg / 1e3 / peaks["hbm_gbs"], 4),
-                   "bytes_per_group": {"soft_mask": 88, "mask_grad": 72}}
+                   "bytes_per_group": {"soft_mask": 88, "mask_grad": 72, "adamw": 168}}
     flops = 2 * sum(L["spec"].dense_equiv_flops for L in prep)
     if rank == 0:
         wg_ms = sum(r["us_wgrad"] for r in per_layer) * 1e-3

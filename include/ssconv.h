@@ -180,7 +180,7 @@ int32_t ssconv_forward_dense_res(const ssconv_desc_t* desc, const void* x, const
  * Only the choice weights (one logit per pattern and group) are trained; the pretrained weights W
  * stay as they are (Sec. 4.1).  A step for one layer is: ssconv_soft_mask -> ssconv_forward_dense
  * with the effective weights -> (the caller's loss and its gradient dL/dy) -> ssconv_wgrad ->
- * ssconv_mask_grad -> the caller's optimiser on the logits. */
+ * ssconv_mask_grad -> ssconv_adamw on the logits. */
 
 /* Relaxed choice and soft mask of every group:
  *   z[g][i]   = softmax_i((logits[g][i] + noise[g][i]) / tau)                      (Eq. 3)
@@ -202,6 +202,15 @@ int32_t ssconv_soft_mask(const float* logits, const float* noise, float tau, con
  * writes), 16-byte aligned; g_logits: device fp32 [G][6], 8-byte aligned.  fp32 arithmetic. */
 int32_t ssconv_mask_grad(const float* z, float tau, const void* w_bf16, const float* g_w_eff,
                          int64_t G, float* g_logits, void* stream);
+
+/* One AdamW update (decoupled weight decay; the optimiser of the Appendix's training details, there
+ * with learning rate 1.0, momentum 0.9, weight decay 1e-4) of n fp32 parameters in place:
+ *   m <- beta1 m + (1 - beta1) g,   v <- beta2 v + (1 - beta2) g^2,
+ *   theta <- theta - lr ( (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps) + weight_decay theta ).
+ * step counts from 1.  theta (the logits), g (from ssconv_mask_grad), m, v: device fp32 [n]; m and v
+ * start as zeros and belong to the caller; all four 16-byte aligned.  fp32 arithmetic. */
+int32_t ssconv_adamw(float* theta, const float* g, float* m, float* v, int64_t n, int32_t step, float lr,
+                     float beta1, float beta2, float eps, float weight_decay, void* stream);
 
 /* Weight gradient of the convolution (Eq. 4 differentiated in the weights):
  *   dw[co,kh,kw,ci] = sum_{n,ho,wo} dy[n,ho,wo,co] * x[n, ho*s-p+kh*d, wo*s-p+kw*d, ci],

@@ -27,7 +27,7 @@ EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssc
            "ssconv_select_mask",
            "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense",
-           "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
+           "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
            "ssconv_forward_static_ws")
 
 
@@ -360,3 +360,18 @@ def ssconv_wgrad(desc: Desc, x: torch.Tensor, dy: torch.Tensor, dw: Optional[tor
     _check("ssconv_wgrad", f(ctypes.byref(desc), _ptr(x), _ptr(dy), _ptr(dw), _ptr(ws), ws_bytes, _ptr(dev_status),
                              _stream(stream)))
     return dw
+
+
+def ssconv_adamw(theta: torch.Tensor, g: torch.Tensor, m: torch.Tensor, v: torch.Tensor, step: int, lr: float = 1.0,
+                 beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, weight_decay: float = 1e-4,
+                 stream=None) -> torch.Tensor:
+    """One AdamW update of fp32 parameters in place (theta, m, v are modified); step counts from 1."""
+    _need_cuda(theta, g, m, v)
+    assert theta.dtype == g.dtype == m.dtype == v.dtype == torch.float32
+    assert theta.numel() == g.numel() == m.numel() == v.numel()
+    f = lib().ssconv_adamw
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int64, ctypes.c_int32] + [ctypes.c_float] * 5 + [ctypes.c_void_p]
+    _check("ssconv_adamw", f(_ptr(theta), _ptr(g), _ptr(m), _ptr(v), theta.numel(), int(step), float(lr),
+                             float(beta1), float(beta2), float(eps), float(weight_decay), _stream(stream)))
+    return theta

@@ -28,12 +28,15 @@ cudaError_t launch_soft_mask(const float* logits, const float* noise, float tau,
                              void* w_eff, cudaStream_t st);
 cudaError_t launch_mask_grad(const float* z, float tau, const void* w, const float* g_w_eff, int64_t G,
                              float* g_logits, cudaStream_t st);
+cudaError_t launch_adamw(float* theta, const float* g, float* m, float* v, int64_t n, float lr, float beta1,
+                         float beta2, float eps, float wd, float c1, float c2, cudaStream_t st);
 int32_t launch_wgrad(const ssconv_desc_t& d, const void* x, const void* dy, float* dw, void* ws, size_t ws_bytes,
                      int32_t* dev_status, cudaStream_t stream);
 int32_t wgrad_workspace_bytes(const ssconv_desc_t& d, size_t* bytes);
 }  // namespace ssconv
 
 #include <atomic>
+#include <cmath>
 namespace ssconv {
 static std::atomic<unsigned long long> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
@@ -249,6 +252,23 @@ int32_t ssconv_mask_grad(const float* z, float tau, const void* w_bf16, const fl
     return SSCONV_ERR_ALIGNMENT;
   if (!aligned16(g_w_eff)) return SSCONV_ERR_ALIGNMENT;
   return ssconv::launch_mask_grad(z, tau, w_bf16, g_w_eff, G, g_logits, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_adamw(float* theta, const float* g, float* m, float* v, int64_t n, int32_t step, float lr, float beta1,
+                     float beta2, float eps, float weight_decay, void* stream) {
+  if (n < 0 || step < 1) return SSCONV_ERR_BAD_DESC;
+  if (!(beta1 >= 0.0f && beta1 < 1.0f && beta2 >= 0.0f && beta2 < 1.0f) || !(eps >= 0.0f)) return SSCONV_ERR_BAD_DESC;
+  if (n == 0) return SSCONV_OK;
+  if (!theta || !g || !m || !v) return SSCONV_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(theta) | reinterpret_cast<uintptr_t>(g) | reinterpret_cast<uintptr_t>(m) |
+       reinterpret_cast<uintptr_t>(v)) & 15u)
+    return SSCONV_ERR_ALIGNMENT;
+  const double c1 = 1.0 / (1.0 - std::pow((double)beta1, (double)step));
+  const double c2 = 1.0 / (1.0 - std::pow((double)beta2, (double)step));
+  return ssconv::launch_adamw(theta, g, m, v, n, lr, beta1, beta2, eps, weight_decay, (float)c1, (float)c2,
+                              (cudaStream_t)stream) == cudaSuccess
              ? SSCONV_OK
              : SSCONV_ERR_CUDA;
 }

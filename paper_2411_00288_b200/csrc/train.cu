@@ -98,6 +98,52 @@ __global__ void mask_grad_kernel(const float* __restrict__ z_in, float inv_tau, 
   store6(g_logits, g, out);
 }
 
+// AdamW on the choice weights (Appendix, training details): decoupled weight decay, bias-corrected
+// moments; c1 = 1 / (1 - beta1^t) and c2 = 1 / (1 - beta2^t) come from the host.  28 bytes per
+// element: HBM-bound.
+__device__ __forceinline__ void adamw_one(float& t, float g, float& m, float& v, float lr, float beta1, float beta2,
+                                          float eps, float wd, float c1, float c2) {
+  m = beta1 * m + (1.0f - beta1) * g;
+  v = beta2 * v + (1.0f - beta2) * g * g;
+  t = t - lr * (m * c1 / (sqrtf(v * c2) + eps) + wd * t);
+}
+// Four elements per thread (16-byte accesses); the last n % 4 elements are handled one by one.
+__global__ void adamw_kernel(float* __restrict__ theta, const float* __restrict__ g, float* __restrict__ m,
+                             float* __restrict__ v, int64_t n, float lr, float beta1, float beta2, float eps,
+                             float wd, float c1, float c2) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  const int64_t n4 = n >> 2;
+  if (i < n4) {
+    float4 t = reinterpret_cast<float4*>(theta)[i];
+    const float4 gi = reinterpret_cast<const float4*>(g)[i];
+    float4 mi = reinterpret_cast<float4*>(m)[i], vi = reinterpret_cast<float4*>(v)[i];
+    adamw_one(t.x, gi.x, mi.x, vi.x, lr, beta1, beta2, eps, wd, c1, c2);
+    adamw_one(t.y, gi.y, mi.y, vi.y, lr, beta1, beta2, eps, wd, c1, c2);
+    adamw_one(t.z, gi.z, mi.z, vi.z, lr, beta1, beta2, eps, wd, c1, c2);
+    adamw_one(t.w, gi.w, mi.w, vi.w, lr, beta1, beta2, eps, wd, c1, c2);
+    reinterpret_cast<float4*>(m)[i] = mi;
+    reinterpret_cast<float4*>(v)[i] = vi;
+    reinterpret_cast<float4*>(theta)[i] = t;
+  } else if (i < n4 + (n & 3)) {
+    const int64_t j = 4 * n4 + (i - n4);
+    float t = theta[j], mi = m[j], vi = v[j];
+    adamw_one(t, g[j], mi, vi, lr, beta1, beta2, eps, wd, c1, c2);
+    m[j] = mi;
+    v[j] = vi;
+    theta[j] = t;
+  }
+}
+
+cudaError_t launch_adamw(float* theta, const float* g, float* m, float* v, int64_t n, float lr, float beta1,
+                         float beta2, float eps, float wd, float c1, float c2, cudaStream_t st) {
+  const int threads = 256;
+  const int64_t work = (n >> 2) + (n & 3);
+  adamw_kernel<<<(unsigned)((work + threads - 1) / threads), threads, 0, st>>>(theta, g, m, v, n, lr, beta1, beta2,
+                                                                                 eps, wd, c1, c2);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_soft_mask(const float* logits, const float* noise, float tau, const void* w, int64_t G, float* z,
                              void* w_eff, cudaStream_t st) {
   const int threads = 256;

@@ -158,3 +158,59 @@ def test_one_mask_learning_step_of_a_layer():
     gl_ref = otrain.logit_grad(z_ref, tau, synth.bf16_bits(inp.w), dw_ref)
     assert _rel_fro(dw.cpu().numpy().astype(np.float64), dw_ref) <= WGRAD_REL_FRO
     assert _rel_fro(gl.cpu().numpy().astype(np.float64), gl_ref) <= LGRAD_REL_FRO
+
+
+@pytest.mark.parametrize("n", [6, 6 * 1000 + 6, 6 * 147456])
+def test_adamw_matches_oracle_over_several_steps(n):
+    g = torch.Generator().manual_seed(999 + n)
+    theta = torch.randn((n,), generator=g)
+    m = torch.zeros(n)
+    v = torch.zeros(n)
+    th_d, m_d, v_d = theta.to(DEV), m.to(DEV), v.to(DEV)
+    th_r, m_r, v_r = theta.numpy().astype(np.float64), np.zeros(n), np.zeros(n)
+    # the call takes fp32 hyper-parameters: the oracle gets the values they round to
+    lr, b1, b2, eps, wd = (float(np.float32(h)) for h in (1.0, 0.9, 0.999, 1e-8, 1e-4))
+    for step in range(1, 5):
+        grad = torch.randn((n,), generator=g) * (10.0 ** (step - 3))
+        api.ssconv_adamw(th_d, grad.to(DEV), m_d, v_d, step, lr, b1, b2, eps, wd)
+        th_r, m_r, v_r = otrain.adamw_step(th_r, grad.numpy(), m_r, v_r, step, lr, b1, b2, eps, wd)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(th_d.cpu().numpy(), th_r, rtol=2e-5, atol=2e-5)
+    np.testing.assert_allclose(m_d.cpu().numpy(), m_r, rtol=1e-5, atol=1e-7)
+    np.testing.assert_allclose(v_d.cpu().numpy(), v_r, rtol=1e-5, atol=1e-10)
+
+
+def test_learning_the_mask_of_a_layer_reduces_its_distillation_loss():
+    """Thirty steps of the whole loop on one layer, every kernel the library's own: the choice weights
+    move so that the soft-masked layer reproduces the dense layer's output better, and the hard mask
+    read off them afterwards beats the one read off the initial choice weights."""
+    spec = synth.LayerSpec("learn", 2, 12, 12, 64, 64, 3, 3, 1, 1, 1, relu=False, has_bias=False, w_std="he",
+                           config=8, index=70)
+    inp = synth.make_inputs(spec)
+    desc = api.desc_from_spec(spec)
+    x, w = inp.x.to(DEV), inp.w.to(DEV)
+    y_dense = api.ssconv_forward_dense(desc, x, w).float()
+    g = torch.Generator().manual_seed(spec.seed + 1)
+    logits = (torch.randn((spec.G, 6), generator=g) * 0.01).to(DEV)
+    m, v = torch.zeros_like(logits), torch.zeros_like(logits)
+    tau = 1.0
+
+    def hard_loss(lg):
+        pat = api.ssconv_select_mask(api.MASK_LOGITS_F32, lg, spec.G)
+        wc, meta = api.ssconv_compress(desc, w, pat)
+        return float(((api.ssconv_forward(desc, x, wc, meta).float() - y_dense) ** 2).mean())
+
+    first_hard = hard_loss(logits)
+    losses = []
+    for step in range(1, 31):
+        z, w_eff = api.ssconv_soft_mask(logits, None, tau, w)
+        y = api.ssconv_forward_dense(desc, x, w_eff).float()
+        diff = y - y_dense
+        losses.append(float((diff ** 2).mean()))
+        dy = (diff * (2.0 / diff.numel())).to(torch.bfloat16)  # the caller's loss gradient
+        dw = api.ssconv_wgrad(desc, x, dy)
+        gl = api.ssconv_mask_grad(z, tau, w, dw)
+        api.ssconv_adamw(logits, gl, m, v, step, lr=0.3, weight_decay=1e-4)
+    torch.cuda.synchronize()
+    assert losses[-1] < 0.5 * losses[0], (losses[0], losses[-1])
+    assert hard_loss(logits) < 0.8 * first_hard
