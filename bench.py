@@ -327,6 +327,15 @@ def train_arm(args):
         "adamw": lambda L: api.ssconv_adamw(L["logits"], L["gl"], L["m"], L["v"], 1, lr=1e-3),
     }
 
+    if args.only_layer is not None:  # profiling aid: the weight gradient of one layer, launched repeatedly
+        L = prep[args.only_layer]
+        for _ in range(args.layer_iters):
+            kernels["wgrad"](L)
+        torch.cuda.synchronize()
+        print(json.dumps({"only_layer": L["spec"].name, "kernel": "wgrad", "launches": args.layer_iters,
+                          "dev_status": int(status.item())}))
+        return
+
     def step():
         for L in prep:
             for k in kernels.values():
