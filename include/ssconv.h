@@ -132,6 +132,21 @@ int32_t ssconv_decompress(const ssconv_desc_t* desc, const void* w_comp, const v
 int32_t ssconv_maxpool(const void* x, void* y, int32_t N, int32_t H, int32_t W, int32_t C, int32_t k,
                        int32_t stride, int32_t pad, void* stream);
 
+/* Partial unfold along the width: the unfold U(X) of Eq. 5 restricted to one filter row.  For every
+ * row of pixels (rows = N*H of them, each W pixels of C channels, bf16) and every horizontal filter
+ * placement wo:
+ *   y[row, wo, kw*C + c] = x[row, wo*stride_w - pad_w + kw*dil_w, c],   0 <= kw < KW,
+ * zero outside the row and in the padding channels [KW*C, C_pad).  y: bf16 [rows, W_out, C_pad] with
+ * W_out = (W + 2 pad_w - dil_w (KW-1) - 1)/stride_w + 1.  A KH x KW convolution over x then equals a
+ * KH x 1 convolution over y with horizontal stride 1, no horizontal padding and C_pad input channels,
+ * with weights unfolded by the same call (weights [C_out,KH,KW,C] are rows = C_out*KH "pixel rows" of
+ * width KW: stride 1, pad 0 gives [C_out,KH,1,C_pad]).  Meant for dense layers with very few input
+ * channels (an RGB stem padded to C = 8: KW = 7 gives C_pad = 64), whose 16-byte pixels the
+ * convolution kernels load slowly.  x, y: device, 16-byte aligned; C % 8 == 0, C_pad % 8 == 0,
+ * C_pad >= KW*C. */
+int32_t ssconv_unfold_w(const void* x, void* y, int64_t rows, int32_t W, int32_t C, int32_t KW,
+                        int32_t stride_w, int32_t pad_w, int32_t dil_w, int32_t C_pad, void* stream);
+
 /* Masked convolution forward (Eq. 6 with the direct definition Eq. 4):
  *   y[n,ho,wo,co] = act( bias[co] + sum_{kh,kw,ci} x[n, ho*s-p+kh*d, wo*s-p+kw*d, ci]
  *                                                  * (M .* W)[co,kh,kw,ci] ),

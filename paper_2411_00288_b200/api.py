@@ -25,7 +25,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.
 EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes",
            "ssconv_plan",
            "ssconv_select_mask",
-           "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_forward", "ssconv_forward_res",
+           "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_unfold_w", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense",
            "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
            "ssconv_forward_static_ws")
@@ -375,3 +375,24 @@ def ssconv_adamw(theta: torch.Tensor, g: torch.Tensor, m: torch.Tensor, v: torch
     _check("ssconv_adamw", f(_ptr(theta), _ptr(g), _ptr(m), _ptr(v), theta.numel(), int(step), float(lr),
                              float(beta1), float(beta2), float(eps), float(weight_decay), _stream(stream)))
     return theta
+
+
+def ssconv_unfold_w(x: torch.Tensor, KW: int, stride: int = 1, pad: int = 0, dil: int = 1, C_pad: Optional[int] = None,
+                    y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Partial unfold along the width of x [..., W, C] bf16: y [..., W_out, C_pad] with
+    y[..., wo, kw*C + c] = x[..., wo*stride - pad + kw*dil, c] (zeros outside and in padding channels)."""
+    _need_cuda(x, y)
+    *lead, w, c = x.shape
+    rows = 1
+    for d in lead:
+        rows *= d
+    if C_pad is None:
+        C_pad = -(-KW * c // 64) * 64
+    wo = (w + 2 * pad - dil * (KW - 1) - 1) // stride + 1
+    if y is None:
+        y = torch.empty((*lead, wo, C_pad), dtype=torch.bfloat16, device=x.device)
+    f = lib().ssconv_unfold_w
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64] + [ctypes.c_int32] * 7 + [ctypes.c_void_p]
+    _check("ssconv_unfold_w", f(_ptr(x), _ptr(y), rows, w, c, KW, stride, pad, dil, C_pad, _stream(stream)))
+    return y

@@ -20,6 +20,8 @@ int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* 
 size_t workspace_bytes();
 cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad,
                            cudaStream_t st);
+cudaError_t launch_unfold_w(const void* x, void* y, long long rows, int W, int C, int KW, int stride, int pad, int dil,
+                            int C_pad, cudaStream_t st);
 int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* split, int32_t* ctas,
                    int32_t* ring_groups);
 int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
@@ -177,6 +179,20 @@ int32_t ssconv_maxpool(const void* x, void* y, int32_t N, int32_t H, int32_t W, 
   if (!aligned16(x) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
   if ((long long)N * H * W * C > 0x7FFFFFFFFFLL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
   return ssconv::launch_maxpool(x, y, N, H, W, C, k, stride, pad, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_unfold_w(const void* x, void* y, int64_t rows, int32_t W, int32_t C, int32_t KW, int32_t stride_w,
+                        int32_t pad_w, int32_t dil_w, int32_t C_pad, void* stream) {
+  if (!x || !y) return SSCONV_ERR_NULL;
+  if (rows <= 0 || W <= 0 || C <= 0 || KW <= 0 || stride_w <= 0 || dil_w <= 0 || pad_w < 0) return SSCONV_ERR_BAD_DESC;
+  if (C % 8 != 0 || C_pad % 8 != 0 || (long long)KW * C > C_pad) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)W + 2LL * pad_w - (long long)dil_w * (KW - 1) - 1 < 0) return SSCONV_ERR_BAD_DESC;
+  if (!aligned16(x) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  if (rows > 0x7FFFFFFFLL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  return ssconv::launch_unfold_w(x, y, rows, W, C, KW, stride_w, pad_w, dil_w, C_pad, (cudaStream_t)stream) ==
+                 cudaSuccess
              ? SSCONV_OK
              : SSCONV_ERR_CUDA;
 }

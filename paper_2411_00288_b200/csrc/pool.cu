@@ -1,4 +1,6 @@
-// Max-pooling over NHWC bf16 activations: the pooling step between the stem and the first block of
+// Max-pooling and a partial unfold over NHWC bf16 activations.
+//
+// Max-pooling: the pooling step between the stem and the first block of
 // a ResNet-shaped stack.  Purely HBM-bound: every input element is read once (neighbouring windows
 // overlap in L1/L2), every output element written once.  One thread per 8 channels (16 bytes) of
 // one output pixel; consecutive threads take consecutive channel groups, so a warp reads and writes
@@ -48,6 +50,42 @@ __global__ void __launch_bounds__(256) maxpool_nhwc_kernel(const uint4* __restri
     }
   }
   y[i] = m;
+}
+
+// Partial unfold along the width (the unfold U(X) of Eq. 5 restricted to one filter row): the KW
+// taps of a filter row become channels,
+//   y[n, h, wo, kw C + c] = x[n, h, wo s - p + kw d, c]   (0 outside the image and for channels >= KW C),
+// so that a KH x KW convolution over C channels equals a KH x 1 convolution with unit horizontal
+// stride over C_pad channels of y.  For layers with very few input channels (an RGB stem padded to 8)
+// this turns 16-byte pixels into 128-byte ones, which the convolution's loads handle at full rate.
+// One thread per 16 bytes of y; HBM-bound on the write of y.
+__global__ void __launch_bounds__(256) unfold_w_kernel(const uint4* __restrict__ x, uint4* __restrict__ y,
+                                                       long long total, int W, int C8, int Wo, int Cp8, int KW,
+                                                       int stride, int pad, int dil) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int ch = (int)(i % Cp8);       // 16-byte chunk of the output pixel
+  const long long pix = i / Cp8;       // (n h) * Wo + wo
+  const int wo = (int)(pix % Wo);
+  const long long row = pix / Wo;      // n * H + h
+  const int kw = ch / C8, c = ch - kw * C8;
+  const int w = wo * stride - pad + kw * dil;
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  if (kw < KW && w >= 0 && w < W) v = __ldg(x + (row * W + w) * C8 + c);
+  y[i] = v;
+}
+
+cudaError_t launch_unfold_w(const void* x, void* y, long long rows, int W, int C, int KW, int stride, int pad, int dil,
+                            int C_pad, cudaStream_t st) {
+  const int span = W + 2 * pad - dil * (KW - 1) - 1;
+  const int Wo = span < 0 ? 0 : span / stride + 1;
+  const long long total = rows * Wo * (C_pad / 8);
+  if (total == 0) return cudaSuccess;
+  const int T = 256;
+  count_launch();
+  unfold_w_kernel<<<(unsigned)((total + T - 1) / T), T, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(y),
+                                                                 total, W, C / 8, Wo, C_pad / 8, KW, stride, pad, dil);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad,

@@ -3,7 +3,8 @@
 Only marshalling: weights are masked and compressed once with the library's own calls, output
 buffers are allocated once, and forward() issues one C-ABI call per convolution on the current
 stream (so it can be recorded into a CUDA graph); the 3x3 stride-2 max-pool between the stem and
-the first block is the library's ssconv_maxpool.
+the first block is the library's ssconv_maxpool.  A dense layer with 8 input channels (the stem) runs
+as ssconv_unfold_w followed by the equivalent KH x 1 convolution over the unfolded taps.
 """
 from __future__ import annotations
 
@@ -41,6 +42,15 @@ class ConvStack:
                     entry["pattern"] = pat
                 if st.kind == "dense" or with_dense:
                     entry["w"] = w
+                if st.kind == "dense" and spec.C_in == 8 and spec.KW > 1:
+                    # the filter row's taps as channels: x -> [N,H,W_out,C_pad], weights -> [C_out,KH,1,C_pad]
+                    c_pad = -(-spec.KW * spec.C_in // 64) * 64
+                    entry["unfold"] = dict(
+                        c_pad=c_pad, w=api.ssconv_unfold_w(w, spec.KW, C_pad=c_pad),
+                        x=torch.empty((spec.N, spec.H, spec.W_out, c_pad), dtype=torch.bfloat16, device=self.device),
+                        desc=api.make_desc(spec.N, spec.H, spec.W_out, c_pad, spec.C_out, spec.KH, 1,
+                                           stride=(spec.stride, 1), pad=(spec.pad, 0), dil=(spec.dil, 1),
+                                           bias=spec.has_bias, relu=spec.relu and not spec.gelu, gelu=spec.gelu))
                 self.layers.append(entry)
                 shape = (spec.N, spec.H_out, spec.W_out, spec.C_out)
             shapes.append(shape)
@@ -61,6 +71,12 @@ class ConvStack:
                 if st.kind == "conv" and sparse:
                     api.ssconv_forward(L["desc"], src, L["w_comp"], L["meta"], L["bias"], y=y, dev_status=self.status,
                                        residual=res)
+                elif "unfold" in L:
+                    U = L["unfold"]
+                    sp = st.spec
+                    api.ssconv_unfold_w(src, sp.KW, sp.stride, sp.pad, sp.dil, C_pad=U["c_pad"], y=U["x"])
+                    api.ssconv_forward_dense(U["desc"], U["x"], U["w"], L["bias"], y=y, dev_status=self.status,
+                                             residual=res)
                 else:
                     api.ssconv_forward_dense(L["desc"], src, L["w"], L["bias"], y=y, dev_status=self.status,
                                              residual=res)
