@@ -242,6 +242,32 @@ int32_t ssconv_wgrad(const ssconv_desc_t* desc, const void* x, const void* dy, f
 /* Scratch bytes ssconv_wgrad needs for this layer on the current device. */
 int32_t ssconv_wgrad_ws_bytes(const ssconv_desc_t* desc, size_t* bytes);
 
+/* ---- Stability quantities (Sec. 3.2) -----------------------------------------------------------
+ * A masking B of a weight matrix W is the additive perturbation dW = (B - 1) .* W (Lemma 3.3).  In the
+ * maximum-absolute-row-sum norm over W in R^{C_out x K} (a row is one output channel):
+ *   out3[0] = ||W||_inf,   out3[1] = ||(B - 1) .* W||_inf  (<= out3[0], Lemma 3.3),   out3[2] = ||B .* W||_inf.
+ * w_bf16: device bf16 [C_out][K], 8-byte aligned; pattern: device uint8 [C_out*K/4], as from
+ * ssconv_select_mask; out3: device fp32 [3] (cleared and written by the call).  K % 4 == 0.
+ * Magnitudes are summed in fp32 in a fixed order. */
+int32_t ssconv_mask_norms(const void* w_bf16, const uint8_t* pattern, int32_t C_out, int64_t K,
+                          float* out3, void* stream);
+
+/* ||x||_inf = the largest magnitude among n bf16 values (exact).  x: device, 16-byte aligned; out:
+ * device fp32 [1] (cleared and written by the call).  n >= 0 (0 gives 0). */
+int32_t ssconv_absmax(const void* x_bf16, int64_t n, float* out, void* stream);
+
+/* The confidence above which a depth-`depth` classifier with L-Lipschitz activations keeps its
+ * prediction on a sample of norm x_norm (host arithmetic in double; returns a negative value for bad
+ * arguments).  layer_norms[i] = ||W_i||, j = the layer that is masked or perturbed:
+ *   SSCONV_LEMMA_PERTURBATION  (Lemma 3.4): L^depth * extra_norm * x_norm * prod_{i != j} ||W_i||,
+ *                              extra_norm = ||dW_j|| (e.g. out3[1] of ssconv_mask_norms);
+ *   SSCONV_LEMMA_ANY_MASK      (Lemma 3.5): L^depth * x_norm * prod_i ||W_i||  (extra_norm unused);
+ *   SSCONV_LEMMA_MASKED_UPDATE (Lemma 3.6): L^depth * (||W_j|| + extra_norm) * x_norm * prod_{i != j} ||W_i||,
+ *                              extra_norm = ||U_j||, the norm of the weight update. */
+enum { SSCONV_LEMMA_PERTURBATION = 34, SSCONV_LEMMA_ANY_MASK = 35, SSCONV_LEMMA_MASKED_UPDATE = 36 };
+double ssconv_stability_threshold(int32_t lemma, double L, const double* layer_norms, int32_t depth,
+                                  int32_t j, double extra_norm, double x_norm);
+
 /* ssconv_forward for callers that have no way to provide scratch memory.  (The paper has no
  * counterpart to this call; it exists for integration only.)
  *

@@ -27,7 +27,7 @@ EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssc
            "ssconv_select_mask",
            "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_unfold_w", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense",
-           "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
+           "ssconv_mask_norms", "ssconv_absmax", "ssconv_stability_threshold", "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
            "ssconv_forward_static_ws")
 
 
@@ -396,3 +396,48 @@ def ssconv_unfold_w(x: torch.Tensor, KW: int, stride: int = 1, pad: int = 0, dil
     f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64] + [ctypes.c_int32] * 7 + [ctypes.c_void_p]
     _check("ssconv_unfold_w", f(_ptr(x), _ptr(y), rows, w, c, KW, stride, pad, dil, C_pad, _stream(stream)))
     return y
+
+
+LEMMA_PERTURBATION, LEMMA_ANY_MASK, LEMMA_MASKED_UPDATE = 34, 35, 36
+
+
+def ssconv_mask_norms(w: torch.Tensor, pattern: torch.Tensor, out: Optional[torch.Tensor] = None,
+                      stream=None) -> torch.Tensor:
+    """fp32 [3] on the device: ||W||_inf, ||(B-1).*W||_inf, ||B.*W||_inf (max absolute row sums; rows are
+    output channels) for bf16 weights [C_out, ...] and one 2:4 pattern per group."""
+    _need_cuda(w, pattern, out)
+    c_out = w.shape[0]
+    k = w.numel() // c_out
+    if out is None:
+        out = torch.empty((3,), dtype=torch.float32, device=w.device)
+    f = lib().ssconv_mask_norms
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
+    _check("ssconv_mask_norms", f(_ptr(w), _ptr(pattern), c_out, k, _ptr(out), _stream(stream)))
+    return out
+
+
+def ssconv_absmax(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """fp32 [1] on the device: the largest magnitude in a bf16 tensor."""
+    _need_cuda(x, out)
+    if out is None:
+        out = torch.empty((1,), dtype=torch.float32, device=x.device)
+    f = lib().ssconv_absmax
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
+    _check("ssconv_absmax", f(_ptr(x), x.numel(), _ptr(out), _stream(stream)))
+    return out
+
+
+def ssconv_stability_threshold(lemma: int, L: float, layer_norms, j: int, extra_norm: float, x_norm: float) -> float:
+    """Confidence threshold of Lemma 3.4 / 3.5 / 3.6 (host arithmetic in the library)."""
+    n = len(layer_norms)
+    arr = (ctypes.c_double * n)(*[float(v) for v in layer_norms])
+    f = lib().ssconv_stability_threshold
+    f.restype = ctypes.c_double
+    f.argtypes = [ctypes.c_int32, ctypes.c_double, ctypes.POINTER(ctypes.c_double), ctypes.c_int32, ctypes.c_int32,
+                  ctypes.c_double, ctypes.c_double]
+    v = float(f(lemma, float(L), arr, n, j, float(extra_norm), float(x_norm)))
+    if v < 0:
+        raise ValueError("bad arguments to ssconv_stability_threshold")
+    return v

@@ -32,6 +32,8 @@ cudaError_t launch_mask_grad(const float* z, float tau, const void* w, const flo
                              float* g_logits, cudaStream_t st);
 cudaError_t launch_adamw(float* theta, const float* g, float* m, float* v, int64_t n, float lr, float beta1,
                          float beta2, float eps, float wd, float c1, float c2, cudaStream_t st);
+cudaError_t launch_mask_norms(const void* w, const uint8_t* pattern, int C_out, int64_t K, float* out, cudaStream_t st);
+cudaError_t launch_absmax(const void* x, int64_t n, float* out, cudaStream_t st);
 int32_t launch_wgrad(const ssconv_desc_t& d, const void* x, const void* dy, float* dw, void* ws, size_t ws_bytes,
                      int32_t* dev_status, cudaStream_t stream);
 int32_t wgrad_workspace_bytes(const ssconv_desc_t& d, size_t* bytes);
@@ -287,6 +289,39 @@ int32_t ssconv_adamw(float* theta, const float* g, float* m, float* v, int64_t n
                               (cudaStream_t)stream) == cudaSuccess
              ? SSCONV_OK
              : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_mask_norms(const void* w_bf16, const uint8_t* pattern, int32_t C_out, int64_t K, float* out3,
+                          void* stream) {
+  if (C_out <= 0 || K <= 0) return SSCONV_ERR_BAD_DESC;
+  if (K % 4 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if (!w_bf16 || !pattern || !out3) return SSCONV_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(w_bf16) & 7u) || (reinterpret_cast<uintptr_t>(out3) & 3u)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_mask_norms(w_bf16, pattern, C_out, K, out3, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_absmax(const void* x_bf16, int64_t n, float* out, void* stream) {
+  if (n < 0) return SSCONV_ERR_BAD_DESC;
+  if (!out || (n > 0 && !x_bf16)) return SSCONV_ERR_NULL;
+  if (!aligned16(x_bf16) || (reinterpret_cast<uintptr_t>(out) & 3u)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_absmax(x_bf16, n, out, (cudaStream_t)stream) == cudaSuccess ? SSCONV_OK : SSCONV_ERR_CUDA;
+}
+
+double ssconv_stability_threshold(int32_t lemma, double L, const double* layer_norms, int32_t depth, int32_t j,
+                                  double extra_norm, double x_norm) {
+  if (!layer_norms || depth <= 0 || j < 0 || j >= depth) return -1.0;
+  if (lemma != SSCONV_LEMMA_PERTURBATION && lemma != SSCONV_LEMMA_ANY_MASK && lemma != SSCONV_LEMMA_MASKED_UPDATE)
+    return -1.0;
+  double others = 1.0;
+  for (int32_t i = 0; i < depth; ++i)
+    if (i != j) others *= layer_norms[i];
+  const double lip = std::pow(L, (double)depth);
+  const double own = lemma == SSCONV_LEMMA_PERTURBATION   ? extra_norm
+                     : lemma == SSCONV_LEMMA_ANY_MASK     ? layer_norms[j]
+                                                          : layer_norms[j] + extra_norm;
+  return lip * own * x_norm * others;
 }
 
 int32_t ssconv_wgrad_ws_bytes(const ssconv_desc_t* desc, size_t* bytes) {

@@ -144,6 +144,90 @@ cudaError_t launch_adamw(float* theta, const float* g, float* m, float* v, int64
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------
+// Stability quantities of Sec. 3.2
+// ---------------------------------------------------------------------------------------
+// Maximum absolute row sums of W [C_out x K], of the part a 2:4 mask drops, (B - 1) .* W (the additive
+// perturbation of Lemma 3.3), and of the part it keeps, B .* W.  One block per row (output channel);
+// a thread adds the magnitudes of its groups in fp32, the block sums them in a fixed order, and the
+// row's three sums go into the result by an integer maximum (non-negative floats order like their bit
+// patterns), so the result does not depend on timing.  out must be zero when the kernel starts.
+__device__ __forceinline__ float block_sum_256(float v, float* scratch) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, o);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __syncthreads();
+  if (lane == 0) scratch[warp] = v;
+  __syncthreads();
+  float total = 0.0f;
+  if (threadIdx.x == 0)
+    for (int i = 0; i < 8; ++i) total += scratch[i];
+  return total;  // valid in thread 0
+}
+__global__ void __launch_bounds__(256) mask_norms_kernel(const uint2* __restrict__ w, const uint8_t* __restrict__ pattern,
+                                                         int64_t groups_per_row, float* __restrict__ out) {
+  __shared__ float scratch[8];
+  const int64_t row0 = (int64_t)blockIdx.x * groups_per_row;
+  float all = 0.0f, kept = 0.0f, dropped = 0.0f;
+  for (int64_t g = threadIdx.x; g < groups_per_row; g += 256) {
+    const uint2 v = w[row0 + g];
+    const float a[4] = {fabsf(bf16_bits_to_f32(v.x & 0xFFFFu)), fabsf(bf16_bits_to_f32(v.x >> 16)),
+                        fabsf(bf16_bits_to_f32(v.y & 0xFFFFu)), fabsf(bf16_bits_to_f32(v.y >> 16))};
+    const uint32_t code = pattern_code(pattern[row0 + g]);  // pos0 | pos1 << 2
+    const float grp_all = (a[0] + a[1]) + (a[2] + a[3]);
+    const float grp_kept = a[code & 3u] + a[(code >> 2) & 3u];
+    all += grp_all;
+    kept += grp_kept;
+    dropped += grp_all - grp_kept;
+  }
+  const float s_all = block_sum_256(all, scratch);
+  const float s_drop = block_sum_256(dropped, scratch);
+  const float s_kept = block_sum_256(kept, scratch);
+  if (threadIdx.x == 0) {
+    atomicMax(reinterpret_cast<int*>(out), __float_as_int(s_all));
+    atomicMax(reinterpret_cast<int*>(out) + 1, __float_as_int(fmaxf(s_drop, 0.0f)));
+    atomicMax(reinterpret_cast<int*>(out) + 2, __float_as_int(s_kept));
+  }
+}
+
+// ||x||_inf of n bf16 values (n a multiple of 8 handled 16 bytes at a time, the rest one by one).
+__global__ void __launch_bounds__(256) absmax_kernel(const uint16_t* __restrict__ x, int64_t n, float* __restrict__ out) {
+  uint32_t m = 0;  // largest magnitude as the 15 bits below the sign, which order like |x|
+  const int64_t n8 = n >> 3;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n8; i += (int64_t)gridDim.x * blockDim.x) {
+    const uint4 v = reinterpret_cast<const uint4*>(x)[i];
+    const uint32_t words[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      m = max(m, words[k] & 0x7FFFu);
+      m = max(m, (words[k] >> 16) & 0x7FFFu);
+    }
+  }
+  if (blockIdx.x == 0)
+    for (int64_t i = 8 * n8 + threadIdx.x; i < n; i += blockDim.x) m = max(m, (uint32_t)x[i] & 0x7FFFu);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_down_sync(0xFFFFFFFFu, m, o));
+  if ((threadIdx.x & 31) == 0 && m != 0) atomicMax(reinterpret_cast<int*>(out), (int)(m << 16));
+}
+
+cudaError_t launch_mask_norms(const void* w, const uint8_t* pattern, int C_out, int64_t K, float* out, cudaStream_t st) {
+  cudaError_t e = cudaMemsetAsync(out, 0, 3 * sizeof(float), st);
+  if (e != cudaSuccess) return e;
+  mask_norms_kernel<<<(unsigned)C_out, 256, 0, st>>>((const uint2*)w, pattern, K / 4, out);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_absmax(const void* x, int64_t n, float* out, cudaStream_t st) {
+  cudaError_t e = cudaMemsetAsync(out, 0, sizeof(float), st);
+  if (e != cudaSuccess) return e;
+  int64_t blocks = ((n >> 3) + 255) / 256;
+  blocks = blocks < 1 ? 1 : (blocks > 148 * 8 ? 148 * 8 : blocks);
+  absmax_kernel<<<(unsigned)blocks, 256, 0, st>>>((const uint16_t*)x, n, out);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_soft_mask(const float* logits, const float* noise, float tau, const void* w, int64_t G, float* z,
                              void* w_eff, cudaStream_t st) {
   const int threads = 256;
