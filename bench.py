@@ -405,7 +405,15 @@ def train_arm(args):
                                for _ in range(10)], 5) / 10 * 1e3
     us_ad = replay_ms(lambda: [api.ssconv_adamw(big["logits"], big["gl"], big["m"], big["v"], 1, lr=1e-3)
                                for _ in range(10)], 5) / 10 * 1e3
+    # the norms of Sec. 3.2 over the same number of groups, as one matrix of 2048 rows (9 bytes per group)
+    rows_n = 2048
+    Gn = Gb // rows_n * rows_n
+    pat_n = torch.randint(0, 6, (Gn,), generator=gen, dtype=torch.int64).to(torch.uint8).to(dev)
+    w_n = big["w"][:Gn].reshape(rows_n, -1).contiguous()
+    out_n = torch.empty((3,), dtype=torch.float32, device=dev)
+    us_nm = replay_ms(lambda: [api.ssconv_mask_norms(w_n, pat_n, out=out_n) for _ in range(10)], 5) / 10 * 1e3
     elementwise = {"groups": Gb, "us_soft_mask": round(us_sm, 1), "us_mask_grad": round(us_mg, 1),
+                   "us_mask_norms": round(us_nm, 1), "mask_norms_gbs": round(9 * Gn / us_nm / 1e3, 1),
                    "us_adamw": round(us_ad, 1), "adamw_gbs": round(28 * 6 * Gb / us_ad / 1e3, 1),
                    "adamw_frac_of_hbm_peak": round(28 * 6 * Gb / us_ad / 1e3 / peaks["hbm_gbs"], 4),
                    "soft_mask_gbs": round(88 * Gb / us_sm / 1e3, 1), "mask_grad_gbs": round(72 * Gb / us_mg / 1e3, 1),
