@@ -23,6 +23,7 @@ What it restates (Sec. 3.1 and Sec. 3.3 of the paper):
   sum over images and output pixels of dL/dy[n, ho, wo, co] x[n, ho s - p + kh d,
   wo s - p + kw d, ci], pixels outside the image contributing nothing (they are the zero
   padding).
+* The gradient with respect to the layer's input is the adjoint of the same linear map in x.
 * The choice weights are updated with AdamW (Appendix, training details: learning rate 1.0,
   momentum 0.9, weight decay 1e-4).  The update is the published one (decoupled weight decay):
   m <- b1 m + (1 - b1) g,  v <- b2 v + (1 - b2) g^2,  theta <- theta - lr (mhat / (sqrt(vhat) + eps)
@@ -102,6 +103,25 @@ def wgrad_f64(x_bits: np.ndarray, dy_bits: np.ndarray, KH: int, KW: int, stride:
             xs = xp[:, h0:h0 + stride * (Ho - 1) + 1:stride, w0:w0 + stride * (Wo - 1) + 1:stride, :]
             dw[:, kh, kw, :] = dy2.T @ xs.reshape(-1, C_in)
     return dw
+
+
+def dgrad_f64(dy_bits: np.ndarray, w: np.ndarray, H: int, W: int, stride: int, pad: int, dil: int) -> np.ndarray:
+    """dL/dx [N, H, W, C_in] in fp64 from dL/dy [N, Ho, Wo, C_out] (bf16 bit patterns) and weights
+    [C_out, KH, KW, C_in] (fp64): every product x * w that enters y[n, ho, wo, co] hands dy * w back to
+    that x (Eq. 4 differentiated in the input); one matrix product per filter tap, scattered to the
+    input pixels the tap reads."""
+    dy = bf16_bits_to_f64(dy_bits)
+    w = np.asarray(w, dtype=np.float64)
+    N, Ho, Wo, C_out = dy.shape
+    _, KH, KW, C_in = w.shape
+    dxp = np.zeros((N, H + 2 * pad, W + 2 * pad, C_in), dtype=np.float64)
+    for kh in range(KH):
+        for kw in range(KW):
+            h0, w0 = kh * dil, kw * dil
+            contrib = dy.reshape(-1, C_out) @ w[:, kh, kw, :]  # [N Ho Wo, C_in]
+            dxp[:, h0:h0 + stride * (Ho - 1) + 1:stride, w0:w0 + stride * (Wo - 1) + 1:stride, :] += contrib.reshape(
+                N, Ho, Wo, C_in)
+    return dxp[:, pad:pad + H, pad:pad + W, :]
 
 
 def adamw_step(theta, g, m, v, step: int, lr: float, beta1: float, beta2: float, eps: float, wd: float):

@@ -211,6 +211,36 @@ def test_wgrad_of_a_1x1_filter_is_a_plain_matrix_product():
     np.testing.assert_allclose(dw.reshape(6, 8), ref, rtol=1e-13)
 
 
+# ---------------------------------------------------------------- gradient with respect to the input
+@pytest.mark.parametrize("case", WG_CASES)
+def test_dgrad_is_the_adjoint_of_the_convolution_oracle_in_x(case):
+    """<dy, conv(e, w)> = <dgrad(dy, w), e> for any input e: the convolution is linear in its input."""
+    N, H, W, C, Co, KH, KW, s, p, d = case
+    rng = np.random.default_rng(hash(case) % (2 ** 32) + 2)
+    Ho, Wo = train.conv_out_extent(H, KH, s, p, d), train.conv_out_extent(W, KW, s, p, d)
+    dy = _bits(rng, (N, Ho, Wo, Co))
+    w = _bits(rng, (Co, KH, KW, C))
+    e = _bits(rng, (N, H, W, C))
+    y = conv2d_f64(ConvShape(N, H, W, C, Co, KH, KW, (s, s), (p, p), (d, d), relu=False), e, w)
+    lhs = float((bf16_to_f64(dy) * y).sum())
+    dx = train.dgrad_f64(dy, bf16_to_f64(w), H, W, s, p, d)
+    assert dx.shape == (N, H, W, C)
+    assert lhs == pytest.approx(float((dx * bf16_to_f64(e)).sum()), rel=1e-11, abs=1e-11)
+
+
+def test_dgrad_of_an_impulse_gradient_is_the_filter_placed_at_that_pixel():
+    rng = np.random.default_rng(12)
+    w = _bits(rng, (3, 3, 3, 4))
+    dy = np.zeros((1, 5, 5, 3), dtype=np.uint16)
+    dy[0, 2, 3, 1] = 0x3F80  # 1.0 at output pixel (2, 3), channel 1
+    dx = train.dgrad_f64(dy, bf16_to_f64(w), 5, 5, 1, 1, 1)
+    wf = bf16_to_f64(w)
+    # output pixel (2, 3) read input pixels (1..3, 2..4) through taps (0..2, 0..2) of filter 1
+    np.testing.assert_array_equal(dx[0, 1:4, 2:5, :], wf[1])
+    dx[0, 1:4, 2:5, :] = 0
+    assert not dx.any()
+
+
 # ---------------------------------------------------------------- optimiser of the choice weights
 def test_adamw_step_matches_the_library_optimiser_over_several_steps():
     import torch
