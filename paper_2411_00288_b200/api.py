@@ -27,7 +27,7 @@ EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssc
            "ssconv_select_mask",
            "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_unfold_w", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense",
-           "ssconv_mask_norms", "ssconv_absmax", "ssconv_stability_threshold", "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
+           "ssconv_mask_norms", "ssconv_absmax", "ssconv_stability_threshold", "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_dgrad_prepare", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
            "ssconv_forward_static_ws")
 
 
@@ -441,3 +441,18 @@ def ssconv_stability_threshold(lemma: int, L: float, layer_norms, j: int, extra_
     if v < 0:
         raise ValueError("bad arguments to ssconv_stability_threshold")
     return v
+
+
+def ssconv_dgrad_prepare(desc: Desc, w: Optional[torch.Tensor], stream=None):
+    """(desc_dx, w_t) for the input gradient of a unit-stride layer: dx = ssconv_forward_dense(desc_dx, dy, w_t).
+    w_t bf16 [C_in,KH,KW,C_out] holds the reversed, channel-exchanged filter (None if w is None)."""
+    _need_cuda(w)
+    out = Desc()
+    w_t = None
+    if w is not None:
+        w_t = torch.empty((desc.C_in, desc.KH, desc.KW, desc.C_out), dtype=torch.bfloat16, device=w.device)
+    f = lib().ssconv_dgrad_prepare
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(Desc), ctypes.c_void_p]
+    _check("ssconv_dgrad_prepare", f(ctypes.byref(desc), _ptr(w), _ptr(w_t), ctypes.byref(out), _stream(stream)))
+    return out, w_t

@@ -228,6 +228,35 @@ cudaError_t launch_absmax(const void* x, int64_t n, float* out, cudaStream_t st)
   return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------
+// Gradient with respect to a layer's input (unit stride)
+// ---------------------------------------------------------------------------------------
+// For unit stride, dL/dx is itself a convolution of dL/dy: with the filter taps reversed and the roles
+// of input and output channels exchanged, padded by dil (K - 1) - pad.  This kernel writes those
+// weights, w_t[ci][KH-1-kh][KW-1-kw][co] = w[co][kh][kw][ci]; the dense forward kernel then does the
+// work.  One thread per element of w_t (writes contiguous; the strided reads hit L2: weights are small).
+__global__ void __launch_bounds__(256) dgrad_weights_kernel(const uint16_t* __restrict__ w, uint16_t* __restrict__ w_t,
+                                                            int C_out, int KH, int KW, int C_in) {
+  const int64_t total = (int64_t)C_in * KH * KW * C_out;
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int co = (int)(i % C_out);
+  int64_t r = i / C_out;
+  const int kw = (int)(r % KW);
+  r /= KW;
+  const int kh = (int)(r % KH);
+  const int ci = (int)(r / KH);
+  w_t[i] = w[(((int64_t)co * KH + (KH - 1 - kh)) * KW + (KW - 1 - kw)) * C_in + ci];
+}
+
+cudaError_t launch_dgrad_weights(const void* w, void* w_t, int C_out, int KH, int KW, int C_in, cudaStream_t st) {
+  const int64_t total = (int64_t)C_in * KH * KW * C_out;
+  dgrad_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>((const uint16_t*)w, (uint16_t*)w_t, C_out, KH,
+                                                                        KW, C_in);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_soft_mask(const float* logits, const float* noise, float tau, const void* w, int64_t G, float* z,
                              void* w_eff, cudaStream_t st) {
   const int threads = 256;

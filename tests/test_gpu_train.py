@@ -214,3 +214,40 @@ def test_learning_the_mask_of_a_layer_reduces_its_distillation_loss():
     torch.cuda.synchronize()
     assert losses[-1] < 0.5 * losses[0], (losses[0], losses[-1])
     assert hard_loss(logits) < 0.8 * first_hard
+
+
+DG_SWEEP = [
+    # name          N  H   W   Ci   Co  KH KW p  d
+    ("c3_p1",       2, 12, 9,  64,  128, 3, 3, 1, 1),
+    ("pw",          2, 9,  7,  96,  136, 1, 1, 0, 1),
+    ("c3_nopad",    1, 10, 10, 64,  64,  3, 3, 0, 1),
+    ("c3_dil2",     1, 12, 12, 64,  64,  3, 3, 2, 2),
+    ("c5_p2",       1, 9,  9,  32,  40,  5, 5, 2, 1),
+    ("r18_128_28",  4, 28, 28, 128, 128, 3, 3, 1, 1),
+]
+
+
+@pytest.mark.parametrize("case", DG_SWEEP, ids=[c[0] for c in DG_SWEEP])
+def test_input_gradient_through_the_dense_kernel_matches_oracle(case):
+    name, N, H, W, Ci, Co, KH, KW, p, d = case
+    spec = synth.LayerSpec(name, N, H, W, Ci, Co, KH, KW, 1, p, d, config=8, index=80 + DG_SWEEP.index(case))
+    inp = synth.make_inputs(spec)
+    g = torch.Generator().manual_seed(spec.seed + 5)
+    dy = torch.randn((N, spec.H_out, spec.W_out, Co), generator=g).to(torch.bfloat16)
+    desc = api.desc_from_spec(spec)
+    desc_dx, w_t = api.ssconv_dgrad_prepare(desc, inp.w.to(DEV))
+    assert (desc_dx.H, desc_dx.W, desc_dx.C_in, desc_dx.C_out) == (spec.H_out, spec.W_out, Co, Ci)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    dx = api.ssconv_forward_dense(desc_dx, dy.to(DEV), w_t, None, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and tuple(dx.shape) == (N, H, W, Ci)
+    ref = otrain.dgrad_f64(synth.bf16_bits(dy), parity.bf16_tensor_to_f64(inp.w), H, W, 1, p, d)
+    rel, mx = parity.errors(parity.bf16_tensor_to_f64(dx), ref)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL * max(1.0, float(np.abs(ref).max()) / 4.0), (rel, mx)
+
+
+def test_input_gradient_is_refused_for_strided_layers():
+    desc = api.make_desc(1, 8, 8, 64, 64, 3, 3, stride=2, pad=1)
+    with pytest.raises(api.SsconvError) as e:
+        api.ssconv_dgrad_prepare(desc, None)
+    assert e.value.status == 3
