@@ -251,3 +251,37 @@ def test_input_gradient_is_refused_for_strided_layers():
     with pytest.raises(api.SsconvError) as e:
         api.ssconv_dgrad_prepare(desc, None)
     assert e.value.status == 3
+
+
+def test_learning_the_masks_of_two_chained_layers():
+    """Two unit-stride layers trained together: the loss gradient reaches the first layer's choice
+    weights through the second layer's input gradient.  Twenty-five steps must lower the loss."""
+    s1 = synth.LayerSpec("chain1", 2, 12, 12, 64, 64, 3, 3, 1, 1, 1, relu=False, has_bias=False, w_std="he",
+                         config=8, index=71)
+    s2 = synth.LayerSpec("chain2", 2, 12, 12, 64, 128, 1, 1, 1, 0, 1, relu=False, has_bias=False, w_std="he",
+                         config=8, index=72)
+    i1, i2 = synth.make_inputs(s1), synth.make_inputs(s2)
+    d1, d2 = api.desc_from_spec(s1), api.desc_from_spec(s2)
+    x, w1, w2 = i1.x.to(DEV), i1.w.to(DEV), i2.w.to(DEV)
+    target = api.ssconv_forward_dense(d2, api.ssconv_forward_dense(d1, x, w1), w2).float()
+    g = torch.Generator().manual_seed(s1.seed + 9)
+    l1 = (torch.randn((s1.G, 6), generator=g) * 0.01).to(DEV)
+    l2 = (torch.randn((s2.G, 6), generator=g) * 0.01).to(DEV)
+    m1, v1, m2, v2 = (torch.zeros_like(t) for t in (l1, l1, l2, l2))
+    tau, losses = 1.0, []
+    for step in range(1, 26):
+        z1, e1 = api.ssconv_soft_mask(l1, None, tau, w1)
+        z2, e2 = api.ssconv_soft_mask(l2, None, tau, w2)
+        h = api.ssconv_forward_dense(d1, x, e1)
+        y = api.ssconv_forward_dense(d2, h, e2).float()
+        diff = y - target
+        losses.append(float((diff ** 2).mean()))
+        dy = (diff * (2.0 / diff.numel()) * 1e4).to(torch.bfloat16)  # scaled so that bf16 keeps it; Adam is scale-free
+        g2 = api.ssconv_mask_grad(z2, tau, w2, api.ssconv_wgrad(d2, h, dy))
+        dd, wt = api.ssconv_dgrad_prepare(d2, e2)
+        dh = api.ssconv_forward_dense(dd, dy, wt, None)
+        g1 = api.ssconv_mask_grad(z1, tau, w1, api.ssconv_wgrad(d1, x, dh))
+        api.ssconv_adamw(l1, g1, m1, v1, step, lr=0.3)
+        api.ssconv_adamw(l2, g2, m2, v2, step, lr=0.3)
+    torch.cuda.synchronize()
+    assert losses[-1] < 0.6 * losses[0], (losses[0], losses[-1])
