@@ -195,8 +195,8 @@ int32_t ssconv_forward_dense_res(const ssconv_desc_t* desc, const void* x, const
  * Only the choice weights (one logit per pattern and group) are trained; the pretrained weights W
  * stay as they are (Sec. 4.1).  A step for one layer is: ssconv_soft_mask -> ssconv_forward_dense
  * with the effective weights -> (the caller's loss and its gradient dL/dy) -> ssconv_wgrad ->
- * ssconv_mask_grad -> ssconv_adamw on the logits; ssconv_dgrad_prepare + ssconv_forward_dense hand
- * dL/dx to the layer before (unit-stride layers). */
+ * ssconv_mask_grad -> ssconv_adamw on the logits; ssconv_dgrad_prepare (+ ssconv_dgrad_spread for a
+ * strided layer) + ssconv_forward_dense hand dL/dx to the layer before. */
 
 /* Relaxed choice and soft mask of every group:
  *   z[g][i]   = softmax_i((logits[g][i] + noise[g][i]) / tau)                      (Eq. 3)
@@ -219,20 +219,31 @@ int32_t ssconv_soft_mask(const float* logits, const float* noise, float tau, con
 int32_t ssconv_mask_grad(const float* z, float tau, const void* w_bf16, const float* g_w_eff,
                          int64_t G, float* g_logits, void* stream);
 
-/* Gradient with respect to a layer's input, for layers with unit stride: dL/dx is the convolution of
- * dL/dy with the filter taps reversed and input and output channels exchanged,
+/* Gradient with respect to a layer's input.  With unit stride, dL/dx is the convolution of dL/dy with
+ * the filter taps reversed and input and output channels exchanged,
  *   dx[n,h,w,ci] = sum_{kh,kw,co} dy[n, h + pad - kh*dil, w + pad - kw*dil, co] * w[co,kh,kw,ci]
- * (Eq. 4 differentiated in the input), so it runs on the dense forward kernel.  This call prepares
- * that: it writes w_t [C_in,KH,KW,C_out] bf16 with w_t[ci][KH-1-kh][KW-1-kw][co] = w[co][kh][kw][ci]
- * (for the mask-learning step w is the effective weights of ssconv_soft_mask) and fills *desc_dx with
- * the descriptor of the equivalent convolution (input = dy [N,H_out,W_out,C_out], output = dx
- * [N,H,W,C_in], padding dil*(K-1) - pad, no bias, no activation).  Then
- *   ssconv_forward_dense(desc_dx, dy, w_t, NULL, dx, ws, ws_bytes, dev_status, stream)
- * computes dx in bf16.  w_bf16 = w_t_bf16 = NULL fills only the descriptor.  Layers with a stride
- * above 1, or with padding beyond dil*(K-1), return SSCONV_ERR_UNSUPPORTED_SHAPE.  w, w_t: device,
- * 16-byte aligned. */
+ * (Eq. 4 differentiated in the input), so it runs on the dense forward kernel.  With a stride s above 1
+ * the same sum runs over the gradient spread out with zeros, dyz[n, ho*s, wo*s, :] = dy[n, ho, wo, :],
+ * of extents Hz = H + 2 pad - dil (KH - 1) and Wz likewise (ssconv_dgrad_spread below writes it).
+ * This call prepares the convolution: it writes w_t [C_in,KH,KW,C_out] bf16 with
+ * w_t[ci][KH-1-kh][KW-1-kw][co] = w[co][kh][kw][ci] (for the mask-learning step w is the effective
+ * weights of ssconv_soft_mask) and fills *desc_dx with the descriptor of the equivalent convolution
+ * (input = dy, or dyz for a strided layer, [N,Hz,Wz,C_out]; output = dx [N,H,W,C_in]; unit stride,
+ * padding dil*(K-1) - pad, no bias, no activation).  Then
+ *   ssconv_forward_dense(desc_dx, dy or dyz, w_t, NULL, dx, ws, ws_bytes, dev_status, stream)
+ * computes dx in bf16.  w_bf16 = w_t_bf16 = NULL fills only the descriptor.  Layers with padding
+ * beyond dil*(K-1) return SSCONV_ERR_UNSUPPORTED_SHAPE.  w, w_t: device, 16-byte aligned. */
 int32_t ssconv_dgrad_prepare(const ssconv_desc_t* desc, const void* w_bf16, void* w_t_bf16,
                              ssconv_desc_t* desc_dx, void* stream);
+
+/* The output gradient of a strided layer spread out for ssconv_dgrad_prepare's convolution:
+ *   dy_spread[n, hz, wz, :] = dy[n, hz / stride_h, wz / stride_w, :] where both divisions are exact and
+ *   land inside dy, zero elsewhere;  dy_spread is [N, Hz, Wz, C_out] with Hz = H + 2 pad_h - dil_h (KH - 1),
+ *   Wz = W + 2 pad_w - dil_w (KW - 1)  (desc_dx->H and desc_dx->W of ssconv_dgrad_prepare).
+ * desc is the layer's own descriptor.  dy: device bf16 [N,H_out,W_out,C_out]; dy_spread: device bf16,
+ * caller-owned, every element written; both 16-byte aligned.  With unit stride it is a plain copy and
+ * not needed.  Values are moved bit-exactly. */
+int32_t ssconv_dgrad_spread(const ssconv_desc_t* desc, const void* dy, void* dy_spread, void* stream);
 
 /* One AdamW update (decoupled weight decay; the optimiser of the Appendix's training details, there
  * with learning rate 1.0, momentum 0.9, weight decay 1e-4) of n fp32 parameters in place:

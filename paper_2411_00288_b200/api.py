@@ -27,7 +27,7 @@ EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssc
            "ssconv_select_mask",
            "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_unfold_w", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense",
-           "ssconv_mask_norms", "ssconv_absmax", "ssconv_stability_threshold", "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_dgrad_prepare", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
+           "ssconv_mask_norms", "ssconv_absmax", "ssconv_stability_threshold", "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_dgrad_prepare", "ssconv_dgrad_spread", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
            "ssconv_forward_static_ws")
 
 
@@ -444,7 +444,8 @@ def ssconv_stability_threshold(lemma: int, L: float, layer_norms, j: int, extra_
 
 
 def ssconv_dgrad_prepare(desc: Desc, w: Optional[torch.Tensor], stream=None):
-    """(desc_dx, w_t) for the input gradient of a unit-stride layer: dx = ssconv_forward_dense(desc_dx, dy, w_t).
+    """(desc_dx, w_t) for the input gradient of a layer: dx = ssconv_forward_dense(desc_dx, dy, w_t), with dy
+    passed through ssconv_dgrad_spread first when the layer's stride is above 1.
     w_t bf16 [C_in,KH,KW,C_out] holds the reversed, channel-exchanged filter (None if w is None)."""
     _need_cuda(w)
     out = Desc()
@@ -456,3 +457,17 @@ def ssconv_dgrad_prepare(desc: Desc, w: Optional[torch.Tensor], stream=None):
     f.argtypes = [ctypes.POINTER(Desc), ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(Desc), ctypes.c_void_p]
     _check("ssconv_dgrad_prepare", f(ctypes.byref(desc), _ptr(w), _ptr(w_t), ctypes.byref(out), _stream(stream)))
     return out, w_t
+
+
+def ssconv_dgrad_spread(desc: Desc, dy: torch.Tensor, stream=None) -> torch.Tensor:
+    """dy [N,H_out,W_out,C_out] of a strided layer spread out with zeros to [N,Hz,Wz,C_out],
+    Hz = H + 2 pad - dil (KH - 1): the input of the convolution ssconv_dgrad_prepare describes."""
+    _need_cuda(dy)
+    Hz = desc.H + 2 * desc.pad_h - desc.dil_h * (desc.KH - 1)
+    Wz = desc.W + 2 * desc.pad_w - desc.dil_w * (desc.KW - 1)
+    out = torch.empty((desc.N, Hz, Wz, desc.C_out), dtype=torch.bfloat16, device=dy.device)
+    f = lib().ssconv_dgrad_spread
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    _check("ssconv_dgrad_spread", f(ctypes.byref(desc), _ptr(dy), _ptr(out), _stream(stream)))
+    return out

@@ -35,6 +35,8 @@ cudaError_t launch_adamw(float* theta, const float* g, float* m, float* v, int64
 cudaError_t launch_mask_norms(const void* w, const uint8_t* pattern, int C_out, int64_t K, float* out, cudaStream_t st);
 cudaError_t launch_absmax(const void* x, int64_t n, float* out, cudaStream_t st);
 cudaError_t launch_dgrad_weights(const void* w, void* w_t, int C_out, int KH, int KW, int C_in, cudaStream_t st);
+cudaError_t launch_dgrad_spread(const void* dy, void* dyz, int N, int Ho, int Wo, int C, int Hz, int Wz, int sh, int sw,
+                                cudaStream_t st);
 int32_t launch_wgrad(const ssconv_desc_t& d, const void* x, const void* dy, float* dw, void* ws, size_t ws_bytes,
                      int32_t* dev_status, cudaStream_t stream);
 int32_t wgrad_workspace_bytes(const ssconv_desc_t& d, size_t* bytes);
@@ -325,6 +327,25 @@ double ssconv_stability_threshold(int32_t lemma, double L, const double* layer_n
   return lip * own * x_norm * others;
 }
 
+int32_t ssconv_dgrad_spread(const ssconv_desc_t* desc, const void* dy, void* dy_spread, void* stream) {
+  ssconv_desc_t d;
+  if (desc) {
+    d = *desc;
+    d.flags = 0;
+  }
+  int32_t rc = check_desc(desc ? &d : nullptr, true);
+  if (rc != SSCONV_OK) return rc;
+  if (!dy || !dy_spread) return SSCONV_ERR_NULL;
+  if (!aligned16(dy) || !aligned16(dy_spread)) return SSCONV_ERR_ALIGNMENT;
+  const int Hz = d.H + 2 * d.pad_h - d.dil_h * (d.KH - 1), Wz = d.W + 2 * d.pad_w - d.dil_w * (d.KW - 1);
+  const int Ho = out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h);
+  const int Wo = out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
+  return ssconv::launch_dgrad_spread(dy, dy_spread, d.N, Ho, Wo, d.C_out, Hz, Wz, d.stride_h, d.stride_w,
+                                     (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
 int32_t ssconv_dgrad_prepare(const ssconv_desc_t* desc, const void* w_bf16, void* w_t_bf16, ssconv_desc_t* desc_dx,
                              void* stream) {
   ssconv_desc_t d;
@@ -335,12 +356,14 @@ int32_t ssconv_dgrad_prepare(const ssconv_desc_t* desc, const void* w_bf16, void
   int32_t rc = check_desc(desc ? &d : nullptr, true);
   if (rc != SSCONV_OK) return rc;
   if (!desc_dx) return SSCONV_ERR_NULL;
-  if (d.stride_h != 1 || d.stride_w != 1) return SSCONV_ERR_UNSUPPORTED_SHAPE;
   const int pad_h = d.dil_h * (d.KH - 1) - d.pad_h, pad_w = d.dil_w * (d.KW - 1) - d.pad_w;
   if (pad_h < 0 || pad_w < 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;  // padding wider than the filter's reach
   ssconv_desc_t t = d;
-  t.H = out_extent(d.H, d.KH, 1, d.pad_h, d.dil_h);
-  t.W = out_extent(d.W, d.KW, 1, d.pad_w, d.dil_w);
+  // Extents of the (spread) gradient: all filter placements at unit stride.  With unit stride this is
+  // the layer's own output extent.
+  t.H = d.H + 2 * d.pad_h - d.dil_h * (d.KH - 1);
+  t.W = d.W + 2 * d.pad_w - d.dil_w * (d.KW - 1);
+  t.stride_h = t.stride_w = 1;
   t.C_in = d.C_out;
   t.C_out = d.C_in;
   t.pad_h = pad_h;

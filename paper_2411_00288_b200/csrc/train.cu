@@ -229,7 +229,7 @@ cudaError_t launch_absmax(const void* x, int64_t n, float* out, cudaStream_t st)
 }
 
 // ---------------------------------------------------------------------------------------
-// Gradient with respect to a layer's input (unit stride)
+// Gradient with respect to a layer's input
 // ---------------------------------------------------------------------------------------
 // For unit stride, dL/dx is itself a convolution of dL/dy: with the filter taps reversed and the roles
 // of input and output channels exchanged, padded by dil (K - 1) - pad.  This kernel writes those
@@ -253,6 +253,37 @@ cudaError_t launch_dgrad_weights(const void* w, void* w_t, int C_out, int KH, in
   const int64_t total = (int64_t)C_in * KH * KW * C_out;
   dgrad_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>((const uint16_t*)w, (uint16_t*)w_t, C_out, KH,
                                                                         KW, C_in);
+  count_launch();
+  return cudaGetLastError();
+}
+
+// For a stride above 1 the same holds once dL/dy is spread out: dyz[n][ho sh][wo sw][:] = dy[n][ho][wo][:],
+// zeros elsewhere, with extents Hz = H + 2 pad - dil (KH - 1) (at least sh (Ho - 1) + 1: input rows past the
+// last filter placement get their zero gradient from the zero rows at the end).  One thread per 16 bytes
+// of dyz; HBM-bound on the write.
+__global__ void __launch_bounds__(256) dgrad_spread_kernel(const uint4* __restrict__ dy, uint4* __restrict__ dyz,
+                                                           long long total, int Ho, int Wo, int C8, int Hz, int Wz,
+                                                           int sh, int sw) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int c = (int)(i % C8);
+  long long r = i / C8;
+  const int wz = (int)(r % Wz);
+  r /= Wz;
+  const int hz = (int)(r % Hz);
+  const long long n = r / Hz;
+  const int ho = hz / sh, wo = wz / sw;
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  if (ho * sh == hz && wo * sw == wz && ho < Ho && wo < Wo) v = __ldg(dy + ((n * Ho + ho) * Wo + wo) * C8 + c);
+  dyz[i] = v;
+}
+
+cudaError_t launch_dgrad_spread(const void* dy, void* dyz, int N, int Ho, int Wo, int C, int Hz, int Wz, int sh, int sw,
+                                cudaStream_t st) {
+  const long long total = (long long)N * Hz * Wz * (C / 8);
+  if (total == 0) return cudaSuccess;
+  dgrad_spread_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>((const uint4*)dy, (uint4*)dyz, total, Ho, Wo,
+                                                                       C / 8, Hz, Wz, sh, sw);
   count_launch();
   return cudaGetLastError();
 }

@@ -246,19 +246,73 @@ def test_input_gradient_through_the_dense_kernel_matches_oracle(case):
     assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL * max(1.0, float(np.abs(ref).max()) / 4.0), (rel, mx)
 
 
-def test_input_gradient_is_refused_for_strided_layers():
-    desc = api.make_desc(1, 8, 8, 64, 64, 3, 3, stride=2, pad=1)
+def test_input_gradient_is_refused_when_the_padding_exceeds_the_filters_reach():
+    desc = api.make_desc(1, 8, 8, 64, 64, 1, 1, stride=1, pad=1)
     with pytest.raises(api.SsconvError) as e:
         api.ssconv_dgrad_prepare(desc, None)
     assert e.value.status == 3
 
 
-def test_learning_the_masks_of_two_chained_layers():
-    """Two unit-stride layers trained together: the loss gradient reaches the first layer's choice
-    weights through the second layer's input gradient.  Twenty-five steps must lower the loss."""
+# Strided layers: the gradient is first spread out with zeros.  H and W are chosen so that some
+# sizes leave input rows and columns beyond the last filter placement (they must get zero gradient).
+#              name            N  H   W   Ci   Co   KH KW s  p  d
+DG_STRIDED = [
+    ("s2_3x3",        2, 16, 16, 64,  64,  3, 3, 2, 1, 1),
+    ("s2_3x3_odd",    2, 15, 18, 64,  96,  3, 3, 2, 1, 1),
+    ("s2_1x1",        2, 14, 14, 128, 64,  1, 1, 2, 0, 1),
+    ("s2_1x1_odd",    1, 13, 11, 64,  128, 1, 1, 2, 0, 1),
+    ("s3_5x5",        1, 20, 17, 32,  40,  5, 5, 3, 2, 1),
+    ("s2_3x3_dil2",   1, 18, 18, 64,  32,  3, 3, 2, 2, 2),
+    ("s2_3x3_p0",     1, 12, 13, 32,  64,  3, 3, 2, 0, 1),
+    ("r18_s2_64to128", 4, 56, 56, 64, 128, 3, 3, 2, 1, 1),
+]
+
+
+@pytest.mark.parametrize("case", DG_STRIDED, ids=[c[0] for c in DG_STRIDED])
+def test_spread_gradient_is_bit_exact(case):
+    name, N, H, W, Ci, Co, KH, KW, s, p, d = case
+    spec = synth.LayerSpec(name, N, H, W, Ci, Co, KH, KW, s, p, d, config=8, index=90 + DG_STRIDED.index(case))
+    g = torch.Generator().manual_seed(spec.seed + 5)
+    dy = torch.randn((N, spec.H_out, spec.W_out, Co), generator=g).to(torch.bfloat16)
+    desc = api.desc_from_spec(spec)
+    got = api.ssconv_dgrad_spread(desc, dy.to(DEV)).cpu()
+    Hz, Wz = H + 2 * p - d * (KH - 1), W + 2 * p - d * (KW - 1)
+    ref = np.zeros((N, Hz, Wz, Co), dtype=np.uint16)
+    ref[:, 0:s * (spec.H_out - 1) + 1:s, 0:s * (spec.W_out - 1) + 1:s, :] = synth.bf16_bits(dy)
+    assert tuple(got.shape) == ref.shape
+    np.testing.assert_array_equal(synth.bf16_bits(got), ref)
+
+
+@pytest.mark.parametrize("case", DG_STRIDED, ids=[c[0] for c in DG_STRIDED])
+def test_input_gradient_of_strided_layers_matches_oracle(case):
+    name, N, H, W, Ci, Co, KH, KW, s, p, d = case
+    spec = synth.LayerSpec(name, N, H, W, Ci, Co, KH, KW, s, p, d, config=8, index=90 + DG_STRIDED.index(case))
+    inp = synth.make_inputs(spec)
+    g = torch.Generator().manual_seed(spec.seed + 5)
+    dy = torch.randn((N, spec.H_out, spec.W_out, Co), generator=g).to(torch.bfloat16)
+    desc = api.desc_from_spec(spec)
+    desc_dx, w_t = api.ssconv_dgrad_prepare(desc, inp.w.to(DEV))
+    assert (desc_dx.stride_h, desc_dx.stride_w, desc_dx.C_in, desc_dx.C_out) == (1, 1, Co, Ci)
+    dyz = api.ssconv_dgrad_spread(desc, dy.to(DEV))
+    assert tuple(dyz.shape) == (N, desc_dx.H, desc_dx.W, Co)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    dx = api.ssconv_forward_dense(desc_dx, dyz, w_t, None, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and tuple(dx.shape) == (N, H, W, Ci)
+    ref = otrain.dgrad_f64(synth.bf16_bits(dy), parity.bf16_tensor_to_f64(inp.w), H, W, s, p, d)
+    rel, mx = parity.errors(parity.bf16_tensor_to_f64(dx), ref)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL * max(1.0, float(np.abs(ref).max()) / 4.0), (rel, mx)
+
+
+@pytest.mark.parametrize("second", [(1, 1, 1, 0), (3, 3, 2, 1)], ids=["1x1", "3x3_stride2"])
+def test_learning_the_masks_of_two_chained_layers(second):
+    """Two layers trained together: the loss gradient reaches the first layer's choice weights through
+    the second layer's input gradient (spread out first when that layer is strided).  Twenty-five steps
+    must lower the loss."""
+    KH2, KW2, st2, p2 = second
     s1 = synth.LayerSpec("chain1", 2, 12, 12, 64, 64, 3, 3, 1, 1, 1, relu=False, has_bias=False, w_std="he",
                          config=8, index=71)
-    s2 = synth.LayerSpec("chain2", 2, 12, 12, 64, 128, 1, 1, 1, 0, 1, relu=False, has_bias=False, w_std="he",
+    s2 = synth.LayerSpec("chain2", 2, 12, 12, 64, 128, KH2, KW2, st2, p2, 1, relu=False, has_bias=False, w_std="he",
                          config=8, index=72)
     i1, i2 = synth.make_inputs(s1), synth.make_inputs(s2)
     d1, d2 = api.desc_from_spec(s1), api.desc_from_spec(s2)
@@ -279,7 +333,7 @@ def test_learning_the_masks_of_two_chained_layers():
         dy = (diff * (2.0 / diff.numel()) * 1e4).to(torch.bfloat16)  # scaled so that bf16 keeps it; Adam is scale-free
         g2 = api.ssconv_mask_grad(z2, tau, w2, api.ssconv_wgrad(d2, h, dy))
         dd, wt = api.ssconv_dgrad_prepare(d2, e2)
-        dh = api.ssconv_forward_dense(dd, dy, wt, None)
+        dh = api.ssconv_forward_dense(dd, api.ssconv_dgrad_spread(d2, dy) if st2 > 1 else dy, wt, None)
         g1 = api.ssconv_mask_grad(z1, tau, w1, api.ssconv_wgrad(d1, x, dh))
         api.ssconv_adamw(l1, g1, m1, v1, step, lr=0.3)
         api.ssconv_adamw(l2, g2, m2, v2, step, lr=0.3)
