@@ -887,29 +887,45 @@ static int out_extent(int in, int k, int stride, int pad, int dil) {
 constexpr int kMaxWorkers = 148;
 constexpr size_t kRegionBytes = (size_t)kTileM * kBN * sizeof(float);
 // Cost model behind the choice of tile width and of splitting K (cycles, measured on B200).
-// A k-block of 64 dense columns takes the longest of three things.  The issuing thread: per pair
+// A k-block of 64 dense columns takes the longest of four things.  The issuing thread: per pair
 // of k-blocks one wait (about 200 cycles even on a complete barrier), about 76 per tcgen05
 // instruction (metadata copy, MMAs, commit) and some loop overhead: 365 per k-block sparse, 480
 // dense, whatever the tile width BN.  The tensor pipe: MMAs of about 35 + 0.5 BN (sparse, two per
-// k-block) or 5 + 0.49 BN (dense, four).  The fill of shared memory from L2, about 68 bytes per
-// cycle and SM when all SMs load: the weight tile's share plus 128 BN bytes of activations.  An
+// k-block) or 5 + 0.49 BN (dense, four).  The fill of shared memory from L2: the weight tile's
+// share plus 128 BN bytes of activations at 56 bytes per cycle and SM (a probe with all SMs
+// loading reached 68; sweeps of forced tile widths over 27 layers fit 50-56 best).  The depth of
+// the ring: see kblock_cycles (load latency of about 1000 cycles, fitted by the same sweeps).  An
 // epilogue that nothing overlaps takes about 900 cycles per 40 positions of a group, and every
 // parked partial tile costs the chip about 90 cycles of L2 traffic (123 KB written by the main
 // kernel and read again by the finishing kernel).
-constexpr double kFillBytesPerCycle = 68.0;
+constexpr double kFillBytesPerCycle = 56.0;
+constexpr double kLoadLatencyCycles = 1000.0;
 constexpr double kIssueSparse = 365.0, kIssueDense = 480.0;
 constexpr double kEpiloguePieceCycles = 900.0;
 constexpr double kCyclesPerParkedTile = 90.0;
 constexpr double kSplitAdvantage = 1.1;  // split only if the model predicts at least this gain
 
+static int ring_groups_for(uint32_t a_group_bytes, int BN, int stage_bufs) {
+  // as many groups in the ring as fit beside the staging buffers, at most kMaxGroups
+  const int n =
+      (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(stage_bufs)) / group_bytes(a_group_bytes, BN));
+  return n > kMaxGroups ? kMaxGroups : n;
+}
+
 template <bool SPARSE>
-static double kblock_cycles(int BN) {
+static double kblock_cycles(int BN, int stage_bufs) {
   const double a_bytes = Cfg<SPARSE>::kAGroupBytes / 2.0;
   const double fill = (a_bytes + 128.0 * BN) / kFillBytesPerCycle;
   const double issue = SPARSE ? kIssueSparse : kIssueDense;
   const double pipe = SPARSE ? 2.0 * (35.0 + 0.5 * BN) + 11.0 : 4.0 * (5.0 + 0.49 * BN);
+  // A ring slot is refilled only once both of its k-blocks are consumed, so a slot's cycle is its
+  // MMAs plus the latency and transfer of its loads, and the ring completes one slot per
+  // (that cycle / slots): wide tiles with two slots are bound by this.
+  const int groups = ring_groups_for(Cfg<SPARSE>::kAGroupBytes, BN, stage_bufs);
+  const double ring = (kLoadLatencyCycles + 2.0 * fill + 2.0 * issue) / (2.0 * (groups < 1 ? 1 : groups));
   double t = fill > issue ? fill : issue;
-  return t > pipe ? t : pipe;
+  t = t > pipe ? t : pipe;
+  return t > ring ? t : ring;
 }
 
 // Tile width and partition of a layer.
@@ -918,7 +934,8 @@ struct Plan {
   bool split;
 };
 template <bool SPARSE>
-static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force_split, int max_bn = kBN) {
+static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force_split, int max_bn = kBN,
+                       int stage_bufs = 2) {
   Plan best{max_bn, false};
   if (force_split) return Plan{kBN, true};
   double best_cost = 0.0;
@@ -926,7 +943,8 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
     const long long tiles = ((Q + BN - 1) / BN) * geo.m_tiles;
     const long long per_cta = (tiles + workers - 1) / workers;
     const int pieces = (BN / 2 + kPiece - 1) / kPiece;
-    const double cost = (double)per_cta * geo.kblocks * kblock_cycles<SPARSE>(BN) + pieces * kEpiloguePieceCycles;
+    const double cost =
+        (double)per_cta * geo.kblocks * kblock_cycles<SPARSE>(BN, stage_bufs) + pieces * kEpiloguePieceCycles;
     if (BN == max_bn || cost < 0.97 * best_cost) {  // a narrower tile has to earn its extra weight traffic
       best_cost = cost;
       best.BN = BN;
@@ -943,7 +961,7 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
       const double units = (double)tiles * a_tiles;
       const double ctas = units < workers ? units : (double)workers;
       const int pieces = (BN / 2 + kPiece - 1) / kPiece;
-      const double cost = units / ctas * 2.0 * kblock_cycles<SPARSE>(BN) +
+      const double cost = units / ctas * 2.0 * kblock_cycles<SPARSE>(BN, stage_bufs) +
                           (ctas + tiles) * kCyclesPerParkedTile * (pieces * 2.0 * kPiece / kBN);
       if (BN == max_bn || cost < 0.97 * best_split_cost) {
         best_split_cost = cost;
@@ -992,12 +1010,6 @@ static int32_t current_device(int* dev_out) {
   return SSCONV_OK;
 }
 
-static int ring_groups_for(uint32_t a_group_bytes, int BN, int stage_bufs) {
-  // as many groups in the ring as fit beside the staging buffers, at most kMaxGroups
-  const int n =
-      (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(stage_bufs)) / group_bytes(a_group_bytes, BN));
-  return n > kMaxGroups ? kMaxGroups : n;
-}
 // Widest tile for which two groups fit beside the staging buffers.
 static int widest_tile(uint32_t a_group_bytes, int stage_bufs) {
   int BN = kBN;
@@ -1063,7 +1075,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   int stage_bufs = 2;
   if (residual != nullptr && !plan.split) {
     stage_bufs = 4;
-    plan = plan_layer<SPARSE>(Q, geo, workers, false, widest_tile(C::kAGroupBytes, 4));
+    plan = plan_layer<SPARSE>(Q, geo, workers, false, widest_tile(C::kAGroupBytes, 4), 4);
     if (plan.split) {  // the narrower limit made splitting look better: stay unsplit at the limit
       plan.split = false;
       plan.BN = widest_tile(C::kAGroupBytes, 4);
