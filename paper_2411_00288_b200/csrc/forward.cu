@@ -48,6 +48,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <type_traits>
+
 #include "layout.cuh"
 #include "sm100_ptx.cuh"
 #include "ssconv.h"
@@ -400,14 +402,16 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   uint8_t* ring = smem;                                                    // ring_groups groups
   uint8_t* out_stage = ring + p.ring_groups * group_bytes(C::kAGroupBytes, p.BN);  // per epilogue group two buffers
   // barrier slots: [0,4) group full, [4,8) group empty, [8,10) accumulator full, [10,12) accumulator empty,
-  // [12,20) residual piece landed (per epilogue group and staging buffer)
+  // [12,20) residual piece landed (per epilogue group and staging buffer), [20,24) first k-block of a
+  // group consumed (two-slot rings only: its activation tile may be refilled ahead of the rest)
   uint64_t* bars = reinterpret_cast<uint64_t*>(out_stage + staging_bytes(p.stage_bufs));
   uint64_t* bar_full = bars;
   uint64_t* bar_empty = bars + 4;
   uint64_t* bar_acc_full = bars + 8;
   uint64_t* bar_acc_empty = bars + 10;
   uint64_t* bar_res = bars + 12;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
+  uint64_t* bar_empty_first = bars + 20;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 24);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = abort_flag + 1;         // per group two slots: the leader's go/stop verdict per tile
 
@@ -419,8 +423,9 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   if (warp == 0) {
     // barrier slots in memory order: 4 group full (3 arrivals: the three producers), 4 group empty (one
     // commit by the MMA thread), 2 accumulator full, 2 accumulator empty (one arrival per epilogue
-    // warp), 8 residual (one arrival with bytes); lane i initialises slot i
-    if (lane < 20) {
+    // warp), 8 residual (one arrival with bytes), 4 first-k-block empty (one commit); lane i
+    // initialises slot i
+    if (lane < 24) {
       const uint32_t count = (lane < 4) ? 3u : (lane < 10) ? 1u : (lane < 12) ? (uint32_t)(4 * kGroups) : 1u;
       mbar_init(&bars[lane], count);
     }
@@ -463,7 +468,8 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     if (lane == 0) {
       const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty), ring0 = smem_u32(ring);
       if (warp == 0)
-        producer_role<SPARSE, kRoleActFirst>(&tm_a, &tm_b, p, full0, empty0, ring0, abort_flag);
+        producer_role<SPARSE, kRoleActFirst>(&tm_a, &tm_b, p, full0,
+                                             p.ring_groups == 2 ? smem_u32(bar_empty_first) : empty0, ring0, abort_flag);
       else if (warp == kFirstExtraProducerWarp)
         producer_role<SPARSE, kRoleActSecond>(&tm_a, &tm_b, p, full0, empty0, ring0, abort_flag);
       else
@@ -478,6 +484,10 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       const uint32_t b_desc = ((uint32_t)p.BN * 128u) >> 4;
       const uint32_t ring_lo0 = desc_lo(smem_u32(ring));
       const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty);
+      // With two ring slots the ring's depth bounds the main loop: the first k-block's activation
+      // tile is then released on its own, so that its reload starts one k-block earlier.
+      const uint32_t empty_first0 = smem_u32(bar_empty_first);
+      const bool early_release = p.ring_groups == 2;
       const uint32_t meta_tmem0 = tmem_base + kMetaCol;
       // channels left in the last chunk decide how many MMAs its k-blocks need
       const int tail_c = p.C_in - (p.cblocks - 1) * kBlockK;
@@ -500,73 +510,84 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         uint32_t accumulate = 0;
         // This thread's instruction stream paces the tensor pipe (its queue is shallow): per group
         // one wait, the MMAs, one commit, and as little else as possible.
-        for (int a = seg.a0; a < seg.a1; ++a) {
-          if (!mbar_wait_a(full0 + 8u * g, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-          const uint32_t a_lo = ring_lo0 + g * grp_desc;
-          const uint32_t b0_lo = a_lo + (C::kAGroupBytes >> 4);
-          const uint32_t b1_lo = b0_lo + b_desc;
-          if (SPARSE) {
-            // metadata image -> 4 TMEM columns: 2 per k-block.  Kept values of the second k-block
-            // start 64 B into the tile's rows; per MMA A advances 16 kept values = 32 B, B 32
-            // channels = 64 B (descriptor units of 16 B).
-            const uint32_t meta_tmem = meta_tmem0 + 4u * mslot;
-            mslot ^= 1u;
-            tc_cp_128x128b_lo(meta_tmem, a_lo + (kATileBytes >> 4));
-            if (a < a_lean_end) {
-              tc_mma_sparse_lo(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
-              tc_mma_sparse_lo(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
-              tc_mma_sparse_lo(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
-              tc_mma_sparse_lo(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
+        // The loop exists twice, with and without the early release, so that rings of more than two
+        // slots pay no branch for it in this thread's instruction stream.
+        auto run_groups = [&](auto early_tag) {
+          constexpr bool kEarly = decltype(early_tag)::value;
+          for (int a = seg.a0; a < seg.a1; ++a) {
+            if (!mbar_wait_a(full0 + 8u * g, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+            const uint32_t a_lo = ring_lo0 + g * grp_desc;
+            const uint32_t b0_lo = a_lo + (C::kAGroupBytes >> 4);
+            const uint32_t b1_lo = b0_lo + b_desc;
+            if (SPARSE) {
+              // metadata image -> 4 TMEM columns: 2 per k-block.  Kept values of the second k-block
+              // start 64 B into the tile's rows; per MMA A advances 16 kept values = 32 B, B 32
+              // channels = 64 B (descriptor units of 16 B).
+              const uint32_t meta_tmem = meta_tmem0 + 4u * mslot;
+              mslot ^= 1u;
+              tc_cp_128x128b_lo(meta_tmem, a_lo + (kATileBytes >> 4));
+              if (a < a_lean_end) {
+                tc_mma_sparse_lo(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
+                tc_mma_sparse_lo(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
+                if (kEarly) tc_commit_a(empty_first0 + 8u * g);
+                tc_mma_sparse_lo(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
+                tc_mma_sparse_lo(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
+              } else {
+                const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
+                const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
+                tc_mma_sparse_lo(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
+                if (n0 > 1) tc_mma_sparse_lo(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
+                if (kEarly) tc_commit_a(empty_first0 + 8u * g);
+                if (n1 > 0) tc_mma_sparse_lo(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
+                if (n1 > 1) tc_mma_sparse_lo(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
+              }
+            } else if (p.small_c) {
+              // chunked operands (see producer_role): chunk stride 2048 B for the weights, 16 BN for the
+              // activations; an MMA takes two chunks (K = 16) of each
+              const uint32_t a_ns = (a_lo & 0xFFFFu) | (128u << 16);
+              const uint32_t b_ns = (b0_lo & 0xFFFFu) | ((uint32_t)p.BN << 16);
+  #pragma unroll 1
+              for (int kb = 0; kb < 2; ++kb) {
+                int left_taps = p.taps - (16 * a + 8 * kb);
+                left_taps = left_taps < 0 ? 0 : (left_taps > 8 ? 8 : left_taps);
+                const int n_mma = (left_taps + 1) >> 1;
+                for (int i = 0; i < n_mma; ++i) {
+                  tc_mma_dense_chunked(d_tmem, a_ns + (uint32_t)kb * (kATileBytes >> 4) + (uint32_t)i * 256u,
+                                       b_ns + (uint32_t)kb * b_desc + (uint32_t)i * (uint32_t)(2 * p.BN), idesc, accumulate);
+                  accumulate = 1;
+                }
+                if (kEarly && kb == 0) tc_commit_a(empty_first0 + 8u * g);
+              }
             } else {
-              const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
-              const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
-              tc_mma_sparse_lo(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
-              if (n0 > 1) tc_mma_sparse_lo(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
-              if (n1 > 0) tc_mma_sparse_lo(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
-              if (n1 > 1) tc_mma_sparse_lo(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
-            }
-          } else if (p.small_c) {
-            // chunked operands (see producer_role): chunk stride 2048 B for the weights, 16 BN for the
-            // activations; an MMA takes two chunks (K = 16) of each
-            const uint32_t a_ns = (a_lo & 0xFFFFu) | (128u << 16);
-            const uint32_t b_ns = (b0_lo & 0xFFFFu) | ((uint32_t)p.BN << 16);
-#pragma unroll 1
-            for (int kb = 0; kb < 2; ++kb) {
-              int left_taps = p.taps - (16 * a + 8 * kb);
-              left_taps = left_taps < 0 ? 0 : (left_taps > 8 ? 8 : left_taps);
-              const int n_mma = (left_taps + 1) >> 1;
-              for (int i = 0; i < n_mma; ++i) {
-                tc_mma_dense_chunked(d_tmem, a_ns + (uint32_t)kb * (kATileBytes >> 4) + (uint32_t)i * 256u,
-                                     b_ns + (uint32_t)kb * b_desc + (uint32_t)i * (uint32_t)(2 * p.BN), idesc, accumulate);
-                accumulate = 1;
+              const uint32_t a1_lo = a_lo + (kATileBytes >> 4);
+              if (a < a_lean_end) {
+                tc_mma_dense_lo(d_tmem, a_lo, b0_lo, idesc, accumulate);
+                tc_mma_dense_lo(d_tmem, a_lo + 2u, b0_lo + 2u, idesc, 1u);
+                tc_mma_dense_lo(d_tmem, a_lo + 4u, b0_lo + 4u, idesc, 1u);
+                tc_mma_dense_lo(d_tmem, a_lo + 6u, b0_lo + 6u, idesc, 1u);
+                if (kEarly) tc_commit_a(empty_first0 + 8u * g);
+                tc_mma_dense_lo(d_tmem, a1_lo, b1_lo, idesc, 1u);
+                tc_mma_dense_lo(d_tmem, a1_lo + 2u, b1_lo + 2u, idesc, 1u);
+                tc_mma_dense_lo(d_tmem, a1_lo + 4u, b1_lo + 4u, idesc, 1u);
+                tc_mma_dense_lo(d_tmem, a1_lo + 6u, b1_lo + 6u, idesc, 1u);
+              } else {
+                const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
+                const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
+                for (int kk = 0; kk < n0; ++kk)
+                  tc_mma_dense_lo(d_tmem, a_lo + 2u * kk, b0_lo + 2u * kk, idesc, (kk > 0) ? 1u : accumulate);
+                if (kEarly) tc_commit_a(empty_first0 + 8u * g);
+                for (int kk = 0; kk < n1; ++kk) tc_mma_dense_lo(d_tmem, a1_lo + 2u * kk, b1_lo + 2u * kk, idesc, 1u);
               }
             }
-          } else {
-            const uint32_t a1_lo = a_lo + (kATileBytes >> 4);
-            if (a < a_lean_end) {
-              tc_mma_dense_lo(d_tmem, a_lo, b0_lo, idesc, accumulate);
-              tc_mma_dense_lo(d_tmem, a_lo + 2u, b0_lo + 2u, idesc, 1u);
-              tc_mma_dense_lo(d_tmem, a_lo + 4u, b0_lo + 4u, idesc, 1u);
-              tc_mma_dense_lo(d_tmem, a_lo + 6u, b0_lo + 6u, idesc, 1u);
-              tc_mma_dense_lo(d_tmem, a1_lo, b1_lo, idesc, 1u);
-              tc_mma_dense_lo(d_tmem, a1_lo + 2u, b1_lo + 2u, idesc, 1u);
-              tc_mma_dense_lo(d_tmem, a1_lo + 4u, b1_lo + 4u, idesc, 1u);
-              tc_mma_dense_lo(d_tmem, a1_lo + 6u, b1_lo + 6u, idesc, 1u);
-            } else {
-              const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
-              const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
-              for (int kk = 0; kk < n0; ++kk)
-                tc_mma_dense_lo(d_tmem, a_lo + 2u * kk, b0_lo + 2u * kk, idesc, (kk > 0) ? 1u : accumulate);
-              for (int kk = 0; kk < n1; ++kk) tc_mma_dense_lo(d_tmem, a1_lo + 2u * kk, b1_lo + 2u * kk, idesc, 1u);
+            accumulate = 1;
+            tc_commit_a(empty0 + 8u * g);
+            if (++g == (uint32_t)p.ring_groups) {
+              g = 0;
+              ph ^= 1u;
             }
           }
-          accumulate = 1;
-          tc_commit_a(empty0 + 8u * g);
-          if (++g == (uint32_t)p.ring_groups) {
-            g = 0;
-            ph ^= 1u;
-          }
-        }
+        };
+        if (early_release) run_groups(std::true_type{}); else run_groups(std::false_type{});
         if (ok) tc_commit(&bar_acc_full[buf]);
       }
     }
