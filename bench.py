@@ -176,9 +176,9 @@ def reference_arm(args):
 # the finishing kernel of the one split layer), dram__bytes_read.sum + dram__bytes_write.sum from an
 # ncu capture of this workload (summary and command: profiles/bench_resnet18_sweep_dram_traffic.md).
 # It belongs to the kernel sources with the digest below; with other sources the bench reports null.
-TRAFFIC_BYTES_PER_STEP = 66.38e6
+TRAFFIC_BYTES_PER_STEP = 66.42e6
 TRAFFIC_SOURCES = ("forward.cu", "sm100_ptx.cuh", "layout.cuh")
-TRAFFIC_SOURCES_SHA256 = "e9efe98dff5b5908a015cbd327e76efab1580627a6d8b3ba195732d849de5e11"
+TRAFFIC_SOURCES_SHA256 = "10e810a20457e9af8872c00178272fb66e51ae31a313be1f66ab4d4d005739c3"
 
 
 def measured_traffic():
