@@ -178,7 +178,7 @@ def reference_arm(args):
 # It belongs to the kernel sources with the digest below; with other sources the bench reports null.
 TRAFFIC_BYTES_PER_STEP = 66.42e6
 TRAFFIC_SOURCES = ("forward.cu", "sm100_ptx.cuh", "layout.cuh")
-TRAFFIC_SOURCES_SHA256 = "10e810a20457e9af8872c00178272fb66e51ae31a313be1f66ab4d4d005739c3"
+TRAFFIC_SOURCES_SHA256 = "80f7e881dd8530c122646168908a6b68fd7d7cbe3cdba0a13579523295a4a150"
 
 
 def measured_traffic():

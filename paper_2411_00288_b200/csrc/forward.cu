@@ -934,7 +934,7 @@ static int ring_groups_for(uint32_t a_group_bytes, int BN, int stage_bufs) {
 }
 
 template <bool SPARSE>
-static double kblock_cycles(int BN, int stage_bufs) {
+static double kblock_cycles(int BN, int stage_bufs, bool steady_ring = true) {
   const double a_bytes = Cfg<SPARSE>::kAGroupBytes / 2.0;
   const double fill = (a_bytes + 128.0 * BN) / kFillBytesPerCycle;
   const double issue = SPARSE ? kIssueSparse : kIssueDense;
@@ -946,7 +946,9 @@ static double kblock_cycles(int BN, int stage_bufs) {
   const double ring = (kLoadLatencyCycles + 2.0 * fill + 2.0 * issue) / (2.0 * (groups < 1 ? 1 : groups));
   double t = fill > issue ? fill : issue;
   t = t > pipe ? t : pipe;
-  return t > ring ? t : ring;
+  // (a CTA of a split layer works through a handful of groups per tile and never reaches that
+  // steady state: forced split plans measured fastest at the widths the other three terms choose)
+  return (steady_ring && ring > t) ? ring : t;
 }
 
 // Tile width and partition of a layer.
@@ -982,7 +984,7 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
       const double units = (double)tiles * a_tiles;
       const double ctas = units < workers ? units : (double)workers;
       const int pieces = (BN / 2 + kPiece - 1) / kPiece;
-      const double cost = units / ctas * 2.0 * kblock_cycles<SPARSE>(BN, stage_bufs) +
+      const double cost = units / ctas * 2.0 * kblock_cycles<SPARSE>(BN, stage_bufs, false) +
                           (ctas + tiles) * kCyclesPerParkedTile * (pieces * 2.0 * kPiece / kBN);
       if (BN == max_bn || cost < 0.97 * best_split_cost) {
         best_split_cost = cost;
