@@ -176,9 +176,9 @@ def reference_arm(args):
 # the finishing kernel of the one split layer), dram__bytes_read.sum + dram__bytes_write.sum from an
 # ncu capture of this workload (summary and command: profiles/bench_resnet18_sweep_dram_traffic.md).
 # It belongs to the kernel sources with the digest below; with other sources the bench reports null.
-TRAFFIC_BYTES_PER_STEP = 66.42e6
+TRAFFIC_BYTES_PER_STEP = 66.41e6
 TRAFFIC_SOURCES = ("forward.cu", "sm100_ptx.cuh", "layout.cuh")
-TRAFFIC_SOURCES_SHA256 = "80f7e881dd8530c122646168908a6b68fd7d7cbe3cdba0a13579523295a4a150"
+TRAFFIC_SOURCES_SHA256 = "f5473a3b686cfcf438dbd934658b158346017ede67fe2f4402739fec885f9b3f"
 
 
 def measured_traffic():

@@ -1122,11 +1122,15 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     int upper[2] = {d.pad_w - (d.KW - 1) * d.dil_w, d.pad_h - (d.KH - 1) * d.dil_h};
     cuuint32_t estr[4] = {1, (cuuint32_t)d.stride_w, (cuuint32_t)d.stride_h, 1};
     // (8-channel mode: 16-byte-wide unswizzled chunks, one per filter tap)
+    // L2 fetches 256 bytes per miss where a pixel is at least that long and every pixel is read
+    // (measured: up to 4 % faster on such layers, 4 % slower on a strided one, nothing elsewhere)
+    const bool wide_pixels = d.C_in >= 128 && d.stride_h == 1 && d.stride_w == 1;
     CUresult r = g_encode_im2col(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), dims, strides,
                                  lower, upper, small_c ? 8u : (cuuint32_t)kBlockK, (cuuint32_t)BN, estr,
                                  CU_TENSOR_MAP_INTERLEAVE_NONE,
                                  small_c ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
-                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                                 wide_pixels ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
   }
   if (SPARSE) {
