@@ -83,7 +83,7 @@ int32_t ssconv_out_shape(const ssconv_desc_t* desc, int32_t* H_out, int32_t* W_o
  * blob and of the metadata blob written by ssconv_compress, and workspace bytes the two
  * forward calls may need.  Any output pointer may be NULL.  The blobs are padded to whole
  * tiles, so they can be slightly larger than C_out*K and C_out*K/8 bytes.  The workspace
- * size is the same for every layer (about 36 MB), so one buffer serves a whole network. */
+ * size is the same for every layer (about 47 MB), so one buffer serves a whole network. */
 int32_t ssconv_sizes(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes,
                      size_t* meta_bytes, size_t* ws_bytes_sparse, size_t* ws_bytes_dense);
 
@@ -96,6 +96,15 @@ int32_t ssconv_sizes(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes
  * 10.x to be current (SSCONV_ERR_ARCH / SSCONV_ERR_CUDA otherwise).  Any output may be NULL. */
 int32_t ssconv_plan(const ssconv_desc_t* desc, int32_t sparse, int32_t* tile_positions, int32_t* split,
                     int32_t* ctas, int32_t* ring_groups);
+
+/* Process-wide override of a choice ssconv_plan reports, for tuning sweeps and tests (no counterpart
+ * in the paper).  SSCONV_TUNE_TILE_POSITIONS: 0 lets the planner choose (default), or a multiple of
+ * 16 in [48, 240] that every later forward call uses as its tile width where the layer allows it
+ * (calls with a residual are limited to 208 sparse / 160 dense and ignore a wider setting).  Not
+ * thread-safe against concurrent forward calls.  Returns SSCONV_ERR_BAD_DESC for an unknown option
+ * or a value out of range. */
+enum { SSCONV_TUNE_TILE_POSITIONS = 1 };
+int32_t ssconv_tune(int32_t option, int32_t value);
 
 /* Hard pattern choice per group (Eq. 1 of Sec. 3.1 without the one-hot: the index of the
  * winning pattern).

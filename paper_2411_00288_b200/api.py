@@ -23,7 +23,7 @@ ERR_TIMEOUT = 8
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.so")
 EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes",
-           "ssconv_plan",
+           "ssconv_plan", "ssconv_tune",
            "ssconv_select_mask",
            "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_unfold_w", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense",
@@ -197,6 +197,17 @@ def ssconv_plan(desc: Desc, sparse: bool = True) -> dict:
     f.argtypes = [ctypes.POINTER(Desc), ctypes.c_int32] + [ctypes.POINTER(ctypes.c_int32)] * 4
     _check("ssconv_plan", f(ctypes.byref(desc), 1 if sparse else 0, *[ctypes.byref(o) for o in out]))
     return dict(tile_positions=out[0].value, split=bool(out[1].value), ctas=out[2].value, ring_groups=out[3].value)
+
+
+TUNE_TILE_POSITIONS = 1
+
+
+def ssconv_tune(option: int, value: int) -> None:
+    """Process-wide planner override: TUNE_TILE_POSITIONS (0 = automatic, or a multiple of 16 in [48, 240])."""
+    f = lib().ssconv_tune
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_int32, ctypes.c_int32]
+    _check("ssconv_tune", f(int(option), int(value)))
 
 
 def default_workspace(device) -> torch.Tensor:

@@ -18,6 +18,7 @@ int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* 
                              const void* residual, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
                              cudaStream_t stream);
 size_t workspace_bytes();
+int32_t set_tuning(int32_t option, int32_t value);
 cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad,
                            cudaStream_t st);
 cudaError_t launch_unfold_w(const void* x, void* y, long long rows, int W, int C, int KW, int stride, int pad, int dil,
@@ -139,6 +140,8 @@ int32_t ssconv_plan(const ssconv_desc_t* desc, int32_t sparse, int32_t* tile_pos
   if (st != SSCONV_OK) return st;
   return ssconv::plan_query(*desc, sparse != 0, tile_positions, split, ctas, ring_groups);
 }
+
+int32_t ssconv_tune(int32_t option, int32_t value) { return ssconv::set_tuning(option, value); }
 
 int32_t ssconv_select_mask(int32_t mode, const void* scores, int64_t G, uint8_t* pattern, void* stream) {
   if (mode != SSCONV_MASK_LOGITS_F32 && mode != SSCONV_MASK_MAGNITUDE_BF16) return SSCONV_ERR_BAD_DESC;

@@ -26,10 +26,10 @@
 // That is about 2.5 instructions per thread and element pair; an epilogue of scalar shared-memory
 // stores or lane shuffles is issue-bound at several times that.
 //
-// What paces the main loop (measured): the issuing thread pays about 200 cycles per mbarrier wait,
-// even on a complete barrier, and about 76 per tcgen05 instruction, and the tensor pipe's queue is
+// What paces the main loop (measured): the issuing warp pays about 200 cycles per mbarrier wait,
+// even on a complete barrier, and 60-80 per tcgen05 instruction, and the tensor pipe's queue is
 // shallow, so every instruction between MMAs is exposed: hence one handshake per group and nothing
-// else in that loop (365 cycles per k-block).  The other bound is the rate at which an SM takes
+// else in that loop.  The other bound is the rate at which an SM takes
 // loads in from L2, about 68 bytes per cycle when all SMs load.  Staging one run of padded input per
 // channel chunk and serving all taps of a 3x3 filter from it through row-shifted descriptors (which
 // would cut the activation loads ninefold) was built and measured before the issue loop was lean,
@@ -289,7 +289,7 @@ struct TapIter {
   }
 };
 
-// One of the three TMA producer threads.  All of them walk the same sequence of groups; role 0
+// One of the three TMA producer warps.  All of them walk the same sequence of groups; role 0
 // loads the activation tile of each group's first k-block, role 1 that of the second, role 2 the
 // weights (with their metadata).  A TMA instruction occupies its issuing thread for a few hundred
 // cycles, so one thread issuing everything cannot keep up with the tensor pipe; three can.
@@ -340,44 +340,44 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
         const int chunks = (left_taps + 1) & ~1;
         it.init(first_tap, p);  // counted in taps here
         if (chunks == 0) {
-          mbar_arrive_a(full);
+          mbar_arrive_w(full);
         } else if (ROLE == kRoleWeights) {
-          mbar_expect_tx_a(full, (uint32_t)chunks * 2048u);
+          mbar_expect_tx_w(full, (uint32_t)chunks * 2048u);
           for (int j = 0; j < chunks; ++j) {  // chunks 8.. belong to the second k-block: 16 KB further on = 8 x 2048
-            tma_load_3d_a(dst + (uint32_t)j * 2048u, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+            tma_load_3d_w(dst + (uint32_t)j * 2048u, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
             it.advance(p);
           }
         } else {
           const uint32_t chunk_bytes = (uint32_t)p.BN * 16u;
-          mbar_expect_tx_a(full, (uint32_t)chunks * chunk_bytes);
+          mbar_expect_tx_w(full, (uint32_t)chunks * chunk_bytes);
           const uint32_t b_dst = dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? b_bytes : 0u);
           for (int j = 0; j < chunks; ++j) {
-            tma_load_im2col_4d_a(b_dst + (uint32_t)j * chunk_bytes, tm_b, full, it.cc * kBlockK, base_w, base_h,
+            tma_load_im2col_4d_w(b_dst + (uint32_t)j * chunk_bytes, tm_b, full, it.cc * kBlockK, base_w, base_h,
                                  q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
             it.advance(p);
           }
         }
       } else if (ROLE == kRoleWeights) {
         if (SPARSE) {
-          mbar_expect_tx_a(full, C::kAGroupBytes);
-          tma_load_2d_a(dst, tm_a, full, a * 64, m * kTileM);
-          bulk_load_a(dst + kATileBytes, meta_src, kMetaImageBytes, full);
+          mbar_expect_tx_w(full, C::kAGroupBytes);
+          tma_load_2d_w(dst, tm_a, full, a * 64, m * kTileM);
+          bulk_load_w(dst + kATileBytes, meta_src, kMetaImageBytes, full);
           meta_src += kMetaImageBytes;
         } else {
-          mbar_expect_tx_a(full, has_second ? 2 * kATileBytes : kATileBytes);
-          tma_load_3d_a(dst, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+          mbar_expect_tx_w(full, has_second ? 2 * kATileBytes : kATileBytes);
+          tma_load_3d_w(dst, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
           it.advance(p);
-          if (has_second) tma_load_3d_a(dst + kATileBytes, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+          if (has_second) tma_load_3d_w(dst + kATileBytes, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
           it.advance(p);
         }
       } else if (ROLE == kRoleActFirst || has_second) {
-        mbar_expect_tx_a(full, b_bytes);
-        tma_load_im2col_4d_a(dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? b_bytes : 0u), tm_b, full,
+        mbar_expect_tx_w(full, b_bytes);
+        tma_load_im2col_4d_w(dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? b_bytes : 0u), tm_b, full,
                              it.cc * kBlockK, base_w, base_h, q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
         it.advance(p);
         it.advance(p);
       } else {
-        mbar_arrive_a(full);  // the group has no second k-block: only keep the barrier's count
+        mbar_arrive_w(full);  // the group has no second k-block: only keep the barrier's count
       }
       if (++g == (uint32_t)p.ring_groups) {
         g = 0;
@@ -465,7 +465,8 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
 
   if (warp == 0 || warp >= kFirstExtraProducerWarp) {
     // ------------------------------------------------------------------ TMA producers
-    if (lane == 0) {
+    // (each a whole warp in lock step, one elected lane issuing: see the warp-wide forms)
+    {
       const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty), ring0 = smem_u32(ring);
       if (warp == 0)
         producer_role<SPARSE, kRoleActFirst>(&tm_a, &tm_b, p, full0,
@@ -477,7 +478,9 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // All 32 lanes run this loop in lock step and wait on the barriers together; the tcgen05
+    // instructions are issued by one elected lane (see the warp-wide forms in sm100_ptx.cuh).
+    {
       const uint32_t idesc = make_idesc_bf16(kTileM, (uint32_t)p.BN, SPARSE);
       // descriptor address units are 16 B
       const uint32_t grp_desc = group_bytes(C::kAGroupBytes, p.BN) >> 4;
@@ -525,21 +528,21 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
               // channels = 64 B (descriptor units of 16 B).
               const uint32_t meta_tmem = meta_tmem0 + 4u * mslot;
               mslot ^= 1u;
-              tc_cp_128x128b_lo(meta_tmem, a_lo + (kATileBytes >> 4));
+              tc_cp_128x128b_w(meta_tmem, a_lo + (kATileBytes >> 4));
               if (a < a_lean_end) {
-                tc_mma_sparse_lo(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
-                tc_mma_sparse_lo(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
-                if (kEarly) tc_commit_a(empty_first0 + 8u * g);
-                tc_mma_sparse_lo(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
-                tc_mma_sparse_lo(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
+                tc_mma_sparse_w(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
+                tc_mma_sparse_w(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
+                if (kEarly) tc_commit_w(empty_first0 + 8u * g);
+                tc_mma_sparse_w(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
+                tc_mma_sparse_w(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
               } else {
                 const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
                 const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
-                tc_mma_sparse_lo(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
-                if (n0 > 1) tc_mma_sparse_lo(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
-                if (kEarly) tc_commit_a(empty_first0 + 8u * g);
-                if (n1 > 0) tc_mma_sparse_lo(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
-                if (n1 > 1) tc_mma_sparse_lo(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
+                tc_mma_sparse_w(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
+                if (n0 > 1) tc_mma_sparse_w(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
+                if (kEarly) tc_commit_w(empty_first0 + 8u * g);
+                if (n1 > 0) tc_mma_sparse_w(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
+                if (n1 > 1) tc_mma_sparse_w(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
               }
             } else if (p.small_c) {
               // chunked operands (see producer_role): chunk stride 2048 B for the weights, 16 BN for the
@@ -552,35 +555,36 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                 left_taps = left_taps < 0 ? 0 : (left_taps > 8 ? 8 : left_taps);
                 const int n_mma = (left_taps + 1) >> 1;
                 for (int i = 0; i < n_mma; ++i) {
-                  tc_mma_dense_chunked(d_tmem, a_ns + (uint32_t)kb * (kATileBytes >> 4) + (uint32_t)i * 256u,
-                                       b_ns + (uint32_t)kb * b_desc + (uint32_t)i * (uint32_t)(2 * p.BN), idesc, accumulate);
+                  tc_mma_dense_w(d_tmem, a_ns + (uint32_t)kb * (kATileBytes >> 4) + (uint32_t)i * 256u,
+                                 b_ns + (uint32_t)kb * b_desc + (uint32_t)i * (uint32_t)(2 * p.BN), idesc, accumulate,
+                                 kDescHiNoSwizzle128);
                   accumulate = 1;
                 }
-                if (kEarly && kb == 0) tc_commit_a(empty_first0 + 8u * g);
+                if (kEarly && kb == 0) tc_commit_w(empty_first0 + 8u * g);
               }
             } else {
               const uint32_t a1_lo = a_lo + (kATileBytes >> 4);
               if (a < a_lean_end) {
-                tc_mma_dense_lo(d_tmem, a_lo, b0_lo, idesc, accumulate);
-                tc_mma_dense_lo(d_tmem, a_lo + 2u, b0_lo + 2u, idesc, 1u);
-                tc_mma_dense_lo(d_tmem, a_lo + 4u, b0_lo + 4u, idesc, 1u);
-                tc_mma_dense_lo(d_tmem, a_lo + 6u, b0_lo + 6u, idesc, 1u);
-                if (kEarly) tc_commit_a(empty_first0 + 8u * g);
-                tc_mma_dense_lo(d_tmem, a1_lo, b1_lo, idesc, 1u);
-                tc_mma_dense_lo(d_tmem, a1_lo + 2u, b1_lo + 2u, idesc, 1u);
-                tc_mma_dense_lo(d_tmem, a1_lo + 4u, b1_lo + 4u, idesc, 1u);
-                tc_mma_dense_lo(d_tmem, a1_lo + 6u, b1_lo + 6u, idesc, 1u);
+                tc_mma_dense_w(d_tmem, a_lo, b0_lo, idesc, accumulate);
+                tc_mma_dense_w(d_tmem, a_lo + 2u, b0_lo + 2u, idesc, 1u);
+                tc_mma_dense_w(d_tmem, a_lo + 4u, b0_lo + 4u, idesc, 1u);
+                tc_mma_dense_w(d_tmem, a_lo + 6u, b0_lo + 6u, idesc, 1u);
+                if (kEarly) tc_commit_w(empty_first0 + 8u * g);
+                tc_mma_dense_w(d_tmem, a1_lo, b1_lo, idesc, 1u);
+                tc_mma_dense_w(d_tmem, a1_lo + 2u, b1_lo + 2u, idesc, 1u);
+                tc_mma_dense_w(d_tmem, a1_lo + 4u, b1_lo + 4u, idesc, 1u);
+                tc_mma_dense_w(d_tmem, a1_lo + 6u, b1_lo + 6u, idesc, 1u);
               } else {
                 const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
                 const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
                 for (int kk = 0; kk < n0; ++kk)
-                  tc_mma_dense_lo(d_tmem, a_lo + 2u * kk, b0_lo + 2u * kk, idesc, (kk > 0) ? 1u : accumulate);
-                if (kEarly) tc_commit_a(empty_first0 + 8u * g);
-                for (int kk = 0; kk < n1; ++kk) tc_mma_dense_lo(d_tmem, a1_lo + 2u * kk, b1_lo + 2u * kk, idesc, 1u);
+                  tc_mma_dense_w(d_tmem, a_lo + 2u * kk, b0_lo + 2u * kk, idesc, (kk > 0) ? 1u : accumulate);
+                if (kEarly) tc_commit_w(empty_first0 + 8u * g);
+                for (int kk = 0; kk < n1; ++kk) tc_mma_dense_w(d_tmem, a1_lo + 2u * kk, b1_lo + 2u * kk, idesc, 1u);
               }
             }
             accumulate = 1;
-            tc_commit_a(empty0 + 8u * g);
+            tc_commit_w(empty0 + 8u * g);
             if (++g == (uint32_t)p.ring_groups) {
               g = 0;
               ph ^= 1u;
@@ -588,7 +592,7 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
           }
         };
         if (early_release) run_groups(std::true_type{}); else run_groups(std::false_type{});
-        if (ok) tc_commit(&bar_acc_full[buf]);
+        if (ok) tc_commit_w(smem_u32(&bar_acc_full[buf]));
       }
     }
   } else if (warp < kFirstExtraProducerWarp) {
@@ -904,8 +908,10 @@ static int out_extent(int in, int k, int stride, int pad, int dil) {
   return span < 0 ? 0 : span / stride + 1;
 }
 
-// Scratch for partly computed tiles: two fp32 regions (128 x 240) per CTA.
-constexpr int kMaxWorkers = 148;
+// Scratch for partly computed tiles: two fp32 regions (128 x 240) per CTA.  The grid is one CTA per SM
+// of the device the call runs on; this is only the largest grid the scratch size (which is fixed
+// without looking at a device, see ssconv_sizes) provides for.
+constexpr int kMaxWorkers = 192;
 constexpr size_t kRegionBytes = (size_t)kTileM * kBN * sizeof(float);
 // Cost model behind the choice of tile width and of splitting K (cycles, measured on B200).
 // A k-block of 64 dense columns takes the longest of four things.  The issuing thread: per pair
@@ -951,6 +957,17 @@ static double kblock_cycles(int BN, int stage_bufs, bool steady_ring = true) {
   return (steady_ring && ring > t) ? ring : t;
 }
 
+// Process-wide override of the planner's tile width (ssconv_tune): 0 lets the model choose.
+static int g_tune_bn = 0;
+int32_t set_tuning(int32_t option, int32_t value) {
+  if (option == SSCONV_TUNE_TILE_POSITIONS) {
+    if (value != 0 && (value < 48 || value > kBN || value % 16 != 0)) return SSCONV_ERR_BAD_DESC;
+    g_tune_bn = value;
+    return SSCONV_OK;
+  }
+  return SSCONV_ERR_BAD_DESC;
+}
+
 // Tile width and partition of a layer.
 struct Plan {
   int BN;
@@ -959,10 +976,12 @@ struct Plan {
 template <bool SPARSE>
 static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force_split, int max_bn = kBN,
                        int stage_bufs = 2) {
-  Plan best{max_bn, false};
   if (force_split) return Plan{kBN, true};
+  int min_bn = 48;
+  if (g_tune_bn != 0 && g_tune_bn <= max_bn) max_bn = min_bn = g_tune_bn;
+  Plan best{max_bn, false};
   double best_cost = 0.0;
-  for (int BN = max_bn; BN >= 48; BN -= 16) {
+  for (int BN = max_bn; BN >= min_bn; BN -= 16) {
     const long long tiles = ((Q + BN - 1) / BN) * geo.m_tiles;
     const long long per_cta = (tiles + workers - 1) / workers;
     const int pieces = (BN / 2 + kPiece - 1) / kPiece;
@@ -979,7 +998,7 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
   if (a_tiles > 1) {
     Plan best_split{kBN, true};
     double best_split_cost = 0.0;
-    for (int BN = max_bn; BN >= 48; BN -= 16) {
+    for (int BN = max_bn; BN >= min_bn; BN -= 16) {
       const long long tiles = ((Q + BN - 1) / BN) * geo.m_tiles;
       const double units = (double)tiles * a_tiles;
       const double ctas = units < workers ? units : (double)workers;

@@ -269,43 +269,109 @@ __device__ __forceinline__ void tc_mma_dense_lo(uint32_t d_tmem, uint32_t a_lo, 
       ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHiSw128)
       : "memory");
 }
-// Dense MMA on unswizzled K-major operands: 16-byte chunks of 8 K-elements; within a chunk the
-// rows follow each other every 16 bytes (8 rows = one 128-byte core matrix, stride-dimension offset
-// 128), chunks follow each other every `chunk stride` bytes, which goes into bits 16-29 of the low
-// word as the leading-dimension offset: lo = (address >> 4) | ((chunk stride >> 4) << 16).
-__device__ __forceinline__ void tc_mma_dense_chunked(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
-                                                     uint32_t accumulate) {
+// The 2:4 sparse form (warp-wide, below): A holds the 16 kept values of 32 dense K-columns per row, B
+// the 32 columns; meta_tmem is the TMEM column with the 2-bit indices of those columns (bit 0 of the
+// column address is passed in the instruction descriptor's selector bits by the caller).
+// tcgen05.cp 128x128b copies 128 rows x 128 bits from shared memory (unswizzled, 16-byte rows) into 4
+// TMEM columns, row r to lane r: one weight tile's metadata image; it is ordered with the MMAs of the
+// issuing thread.
+
+// ---------------------------------------------------------------- warp-wide forms
+// The same tcgen05 instructions for a loop that all 32 lanes of a warp execute in lock step, with one
+// elected lane issuing: the operands (descriptors, TMEM and barrier addresses) are then uniform over
+// the warp, which lets the compiler keep them in the uniform register file that these instructions
+// read; inside a branch taken by a single lane every operand has to be moved there per instruction
+// (measured on the forward kernel's issuing loop: 80 -> 62 cycles per tcgen05 instruction, 256 -> 205
+// per wait on a complete barrier).
+// desc_hi = kDescHiNoSwizzle128 selects unswizzled K-major operands: 16-byte chunks of 8 K-elements;
+// within a chunk the rows follow each other every 16 bytes (8 rows = one 128-byte core matrix), chunks
+// follow each other every `chunk stride` bytes, which goes into bits 16-29 of the low word as the
+// leading-dimension offset: lo = (address >> 4) | ((chunk stride >> 4) << 16).
+__device__ __forceinline__ void tc_mma_dense_w(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                               uint32_t accumulate, uint32_t desc_hi = kDescHiSw128) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "{\n\t.reg .pred p, e;\n\t.reg .b64 da, db;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
       "mov.b64 da, {%1, %5};\n\t"
       "mov.b64 db, {%2, %5};\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHiNoSwizzle128)
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(desc_hi)
       : "memory");
 }
-// 2:4 sparse form: A holds the 16 kept values of 32 dense K-columns per row, B the 32 columns;
-// meta_tmem is the TMEM column with the 2-bit indices of those columns (bit 0 of the column
-// address is passed in the instruction descriptor's selector bits by the caller).
-__device__ __forceinline__ void tc_mma_sparse_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t meta_tmem,
-                                                 uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void tc_mma_sparse_w(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t meta_tmem,
+                                                uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "{\n\t.reg .pred p, e;\n\t.reg .b64 da, db;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
       "mov.b64 da, {%1, %6};\n\t"
       "mov.b64 db, {%2, %6};\n\t"
       "setp.ne.b32 p, %5, 0;\n\t"
-      "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], da, db, [%3], %4, p;\n\t}"
+      "@e tcgen05.mma.sp.cta_group::1.kind::f16 [%0], da, db, [%3], %4, p;\n\t}"
       ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(meta_tmem), "r"(idesc), "r"(accumulate), "r"(kDescHiSw128)
       : "memory");
 }
-// Copy 128 rows x 128 bits from shared memory (unswizzled, 16-byte rows) into 4 TMEM columns, row r
-// to lane r: one weight tile's metadata image.  Ordered with the MMAs of the issuing thread.
-__device__ __forceinline__ void tc_cp_128x128b_lo(uint32_t dst_tmem, uint32_t src_lo) {
+__device__ __forceinline__ void tc_cp_128x128b_w(uint32_t dst_tmem, uint32_t src_lo) {
   asm volatile(
-      "{\n\t.reg .b64 ds;\n\t"
+      "{\n\t.reg .pred e;\n\t.reg .b64 ds;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
       "mov.b64 ds, {%1, %2};\n\t"
-      "tcgen05.cp.cta_group::1.128x128b [%0], ds;\n\t}"
+      "@e tcgen05.cp.cta_group::1.128x128b [%0], ds;\n\t}"
       ::"r"(dst_tmem), "r"(src_lo), "r"(kDescHiNoSwizzle128)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_w(uint32_t bar_addr) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
+      "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar_addr)
+      : "memory");
+}
+
+// Producer side, warp-wide: the whole warp waits and walks the loop, one elected lane arrives on the
+// barrier and issues the copies (their tensor-map, shared-memory and barrier operands are uniform).
+__device__ __forceinline__ void mbar_expect_tx_w(uint32_t bar_addr, uint32_t bytes) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+      "@e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}" ::"r"(bar_addr), "r"(bytes)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_w(uint32_t bar_addr) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+      "@e mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}" ::"r"(bar_addr)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_w(uint32_t dst, const CUtensorMap* map, uint32_t bar, int32_t x, int32_t y) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+      "@e cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n\t}"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_w(uint32_t dst, const CUtensorMap* map, uint32_t bar, int32_t x, int32_t y,
+                                              int32_t z) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+      "@e cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n\t}"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_4d_w(uint32_t dst, const CUtensorMap* map, uint32_t bar, int32_t c,
+                                                     int32_t w, int32_t h, int32_t n, uint16_t off_w, uint16_t off_h) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+      "@e cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};\n\t}"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_load_w(uint32_t dst, const void* gsrc, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+      "@e cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}"
+      ::"r"(dst), "l"(gsrc), "r"(bytes), "r"(bar)
       : "memory");
 }
 
