@@ -91,19 +91,22 @@ int32_t ssconv_sizes(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes
  * the current device: positions per output tile (the N of the tensor-core instruction, a multiple
  * of 16 up to 240, chosen so that the tiles fill the SMs), whether the K range is split across
  * thread blocks (then a second, finishing kernel runs and ws is used), the number of thread
- * blocks, and the depth of the shared-memory ring in pairs of 64-column k-blocks.  A tuning aid
- * with no counterpart in the paper; nothing is launched.  Needs a device of compute capability
- * 10.x to be current (SSCONV_ERR_ARCH / SSCONV_ERR_CUDA otherwise).  Any output may be NULL. */
+ * blocks, the depth of the shared-memory ring in pairs of 64-column k-blocks, and whether the layer
+ * runs on pairs of thread blocks that share tiles of 256 output channels (layers with more than 128
+ * output channels and enough tiles; ctas is then twice the number of pairs).  A tuning aid with no
+ * counterpart in the paper; nothing is launched.  Needs a device of compute capability 10.x to be
+ * current (SSCONV_ERR_ARCH / SSCONV_ERR_CUDA otherwise).  Any output may be NULL. */
 int32_t ssconv_plan(const ssconv_desc_t* desc, int32_t sparse, int32_t* tile_positions, int32_t* split,
-                    int32_t* ctas, int32_t* ring_groups);
+                    int32_t* ctas, int32_t* ring_groups, int32_t* pair);
 
-/* Process-wide override of a choice ssconv_plan reports, for tuning sweeps and tests (no counterpart
- * in the paper).  SSCONV_TUNE_TILE_POSITIONS: 0 lets the planner choose (default), or a multiple of
- * 16 in [48, 240] that every later forward call uses as its tile width where the layer allows it
- * (calls with a residual are limited to 208 sparse / 160 dense and ignore a wider setting).  Not
- * thread-safe against concurrent forward calls.  Returns SSCONV_ERR_BAD_DESC for an unknown option
- * or a value out of range. */
-enum { SSCONV_TUNE_TILE_POSITIONS = 1 };
+/* Process-wide overrides of the choices ssconv_plan reports, for tuning sweeps and tests (no
+ * counterpart in the paper).  SSCONV_TUNE_TILE_POSITIONS: 0 lets the planner choose (default), or a
+ * multiple of 16 in [48, 240] that every later forward call uses as its tile width where the layer
+ * allows it (calls with a residual are limited to 208 sparse / 160 dense and ignore a wider setting;
+ * the pair kernel takes 64 and up).  SSCONV_TUNE_PAIR: -1 lets the planner choose (default), 0 never
+ * uses pairs of thread blocks, 1 uses them wherever they apply.  Not thread-safe against concurrent
+ * forward calls.  Returns SSCONV_ERR_BAD_DESC for an unknown option or a value out of range. */
+enum { SSCONV_TUNE_TILE_POSITIONS = 1, SSCONV_TUNE_PAIR = 2 };
 int32_t ssconv_tune(int32_t option, int32_t value);
 
 /* Hard pattern choice per group (Eq. 1 of Sec. 3.1 without the one-hot: the index of the

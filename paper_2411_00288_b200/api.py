@@ -191,19 +191,21 @@ _workspaces = {}
 
 def ssconv_plan(desc: Desc, sparse: bool = True) -> dict:
     """Tile width, K split, thread blocks and ring depth the forward call would use on the current device."""
-    out = [ctypes.c_int32(0) for _ in range(4)]
+    out = [ctypes.c_int32(0) for _ in range(5)]
     f = lib().ssconv_plan
     f.restype = ctypes.c_int32
-    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_int32] + [ctypes.POINTER(ctypes.c_int32)] * 4
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_int32] + [ctypes.POINTER(ctypes.c_int32)] * 5
     _check("ssconv_plan", f(ctypes.byref(desc), 1 if sparse else 0, *[ctypes.byref(o) for o in out]))
-    return dict(tile_positions=out[0].value, split=bool(out[1].value), ctas=out[2].value, ring_groups=out[3].value)
+    return dict(tile_positions=out[0].value, split=bool(out[1].value), ctas=out[2].value, ring_groups=out[3].value,
+                pair=bool(out[4].value))
 
 
-TUNE_TILE_POSITIONS = 1
+TUNE_TILE_POSITIONS, TUNE_PAIR = 1, 2
 
 
 def ssconv_tune(option: int, value: int) -> None:
-    """Process-wide planner override: TUNE_TILE_POSITIONS (0 = automatic, or a multiple of 16 in [48, 240])."""
+    """Process-wide planner override: TUNE_TILE_POSITIONS (0 = automatic, or a multiple of 16 in [48, 240]),
+    TUNE_PAIR (-1 automatic, 0 never, 1 wherever thread-block pairs apply)."""
     f = lib().ssconv_tune
     f.restype = ctypes.c_int32
     f.argtypes = [ctypes.c_int32, ctypes.c_int32]

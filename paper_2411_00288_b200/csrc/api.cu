@@ -24,7 +24,7 @@ cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, i
 cudaError_t launch_unfold_w(const void* x, void* y, long long rows, int W, int C, int KW, int stride, int pad, int dil,
                             int C_pad, cudaStream_t st);
 int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* split, int32_t* ctas,
-                   int32_t* ring_groups);
+                   int32_t* ring_groups, int32_t* pair);
 int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const void* w_comp, const void* meta,
                                  const float* bias, void* y, int32_t* dev_status, cudaStream_t stream);
 cudaError_t launch_soft_mask(const float* logits, const float* noise, float tau, const void* w, int64_t G, float* z,
@@ -135,10 +135,10 @@ int32_t ssconv_sizes(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes
 }
 
 int32_t ssconv_plan(const ssconv_desc_t* desc, int32_t sparse, int32_t* tile_positions, int32_t* split,
-                    int32_t* ctas, int32_t* ring_groups) {
+                    int32_t* ctas, int32_t* ring_groups, int32_t* pair) {
   int32_t st = check_desc(desc, true);
   if (st != SSCONV_OK) return st;
-  return ssconv::plan_query(*desc, sparse != 0, tile_positions, split, ctas, ring_groups);
+  return ssconv::plan_query(*desc, sparse != 0, tile_positions, split, ctas, ring_groups, pair);
 }
 
 int32_t ssconv_tune(int32_t option, int32_t value) { return ssconv::set_tuning(option, value); }

@@ -99,7 +99,8 @@ struct FwdParams {
   int small_c;              // dense layers with C_in == 8: a k-block is 8 filter taps (see producer_role)
   int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
   int taps, cblocks, kblocks;
-  int m_tiles, num_tiles;
+  int m_tiles, num_tiles;   // (pair kernel: m_tiles counts pairs of 128-channel tiles, m_real the tiles themselves)
+  int m_real;
   int a_tiles;              // pairs of k-blocks (groups) per output tile
   int split;                // 1: units dealt out evenly across CTAs (stream-K); 0: whole tiles per CTA
   int work_quot, work_rem;  // work items per CTA: quotient and remainder of (tiles or units) / grid
@@ -122,9 +123,9 @@ struct Segment {
 // with q = W / G, r = W % G, both computed on the host: the device needs no division for it.
 struct WorkIter {
   int tile, a0, left, A;  // next tile, first group of it, units left in this CTA's range, groups per tile
-  __device__ WorkIter(const FwdParams& p) {
+  __device__ explicit WorkIter(const FwdParams& p) : WorkIter(p, blockIdx.x) {}
+  __device__ WorkIter(const FwdParams& p, uint32_t c) {  // c: this worker's number (CTA, or CTA pair)
     A = p.a_tiles;
-    const uint32_t c = blockIdx.x;
     const uint32_t start = c * (uint32_t)p.work_quot + (c < (uint32_t)p.work_rem ? c : (uint32_t)p.work_rem);
     const int count = p.work_quot + (c < (uint32_t)p.work_rem ? 1 : 0);
     if (p.split) {
@@ -877,6 +878,315 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
 
 
 // ---------------------------------------------------------------------------------------
+// Pair kernel: a tile of 256 output channels x BN positions on two CTAs (tcgen05 cta_group::2)
+// ---------------------------------------------------------------------------------------
+// What bounds the one-CTA kernel on compute-bound layers is shared-memory bandwidth: per k-block an
+// SM writes its weight and activation tiles once (TMA) and the MMAs read them once, 17 KB + 256 BN
+// bytes at about 140 bytes per cycle, against 240 cycles of sparse tensor time at BN = 240.  Two CTAs
+// of a cluster sharing one MMA of M = 256 halve the activation part: each CTA loads and holds its own
+// 128 weight rows (and their metadata) and only half of the tile's positions, and the tensor cores of
+// both SMs read both halves.  Per CTA nothing else changes: its TMEM holds its 128 channels x BN
+// positions, so the epilogue is the one-CTA kernel's.  Roles as there (three producer warps, one
+// issuing warp, eight epilogue warps), except that only the even CTA of a pair (the leader) issues
+// tcgen05.cp / mma / commit, for both.  Barriers: "full" lives in the leader and collects the bytes
+// of both CTAs' loads (the peer's copies signal it directly, the leader announces the sum); "empty"
+// and "accumulator full" exist in each CTA and the leader commits to both; "accumulator empty" lives
+// in the leader and counts the epilogue warps of both CTAs.  No load is multicast: each CTA fetches
+// what it needs itself.  Whole tiles only (no K split), no residual, no 8-channel mode.
+template <bool SPARSE, int ROLE>
+__device__ __forceinline__ void pair_producer_role(const CUtensorMap* tm_a, const CUtensorMap* tm_b,
+                                                   const CUtensorMap* tm_meta, const FwdParams& p, uint32_t rank,
+                                                   uint32_t pair, uint32_t full0_leader, uint32_t full0_local,
+                                                   uint32_t empty0, uint32_t ring0, volatile int* abort_flag) {
+  using C = Cfg<SPARSE>;
+  const uint32_t half_bytes = (uint32_t)(p.BN >> 1) * 128u;  // this CTA's half of an activation tile
+  const uint32_t grp_bytes = C::kAGroupBytes + 2u * half_bytes;
+  const bool leader = rank == 0;
+  uint32_t g = 0, ph = 0;
+  bool ok = true;
+  bool first_segment = true;
+  WorkIter work(p, pair);
+  Segment seg;
+  while (ok && work.next(seg)) {
+    const int pt = seg.tile / p.m_tiles;  // (m_tiles counts pairs of 128-channel tiles here)
+    const int m = 2 * (seg.tile - pt * p.m_tiles) + (int)rank;
+    const int m_meta = m < p.m_real ? m : p.m_real - 1;  // a CTA beyond the last channel tile multiplies zeros
+    const Pos q0 = decode_pos(pt * p.BN + (int)rank * (p.BN >> 1), p.Wo, p.Ho);
+    const int base_w = q0.c * p.stride_w - p.pad_w;
+    const int base_h = q0.r * p.stride_h - p.pad_h;
+    TapIter it;
+    it.init(ROLE == kRoleActSecond ? 1 : 0, p);
+    if (first_segment) {
+      grid_dependency_wait();
+      first_segment = false;
+    }
+    for (int a = 0; a < p.a_tiles; ++a) {
+      if (!mbar_wait_a(empty0 + 8u * g, ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+      const uint32_t full = full0_leader + 8u * g;  // cluster address of the leader's barrier
+      const uint32_t dst = ring0 + g * grp_bytes;
+      const bool has_second = 2 * a + 1 < p.kblocks;
+      if (ROLE == kRoleWeights) {
+        if (SPARSE) {
+          if (leader) mbar_expect_tx_w(full0_local + 8u * g, 2u * C::kAGroupBytes);
+          tma2_load_2d_w(dst, tm_a, full, a * 64, m * kTileM);
+          tma2_load_2d_w(dst + kATileBytes, tm_meta, full, 0, (m_meta * p.a_tiles + a) * kTileM);
+        } else {
+          if (leader) mbar_expect_tx_w(full0_local + 8u * g, (has_second ? 4u : 2u) * kATileBytes);
+          tma2_load_3d_w(dst, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+          it.advance(p);
+          if (has_second) tma2_load_3d_w(dst + kATileBytes, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+          it.advance(p);
+        }
+      } else if (ROLE == kRoleActFirst || has_second) {
+        if (leader) mbar_expect_tx_w(full0_local + 8u * g, 2u * half_bytes);
+        tma2_load_im2col_4d_w(dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? half_bytes : 0u), tm_b, full,
+                              it.cc * kBlockK, base_w, base_h, q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
+        it.advance(p);
+        it.advance(p);
+      } else if (leader) {
+        mbar_arrive_w(full0_local + 8u * g);  // the group has no second k-block: only keep the barrier's count
+      }
+      if (++g == (uint32_t)p.ring_groups) {
+        g = 0;
+        ph ^= 1u;
+      }
+    }
+  }
+}
+
+template <bool SPARSE>
+__global__ void __launch_bounds__(kThreads, 1)
+ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                       const __grid_constant__ CUtensorMap tm_meta, const __grid_constant__ CUtensorMap tm_y,
+                       const __grid_constant__ CUtensorMap tm_y_tail, const FwdParams p) {
+  using C = Cfg<SPARSE>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t half_bytes = (uint32_t)(p.BN >> 1) * 128u;
+  const uint32_t grp_bytes = C::kAGroupBytes + 2u * half_bytes;
+  uint8_t* ring = smem;
+  uint8_t* out_stage = ring + p.ring_groups * grp_bytes;
+  // barrier slots: [0,4) group full (used in the leader), [4,8) group empty, [8,10) accumulator full,
+  // [10,12) accumulator empty (used in the leader)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_stage + staging_bytes(2));
+  uint64_t* bar_full = bars;
+  uint64_t* bar_empty = bars + 4;
+  uint64_t* bar_acc_full = bars + 8;
+  uint64_t* bar_acc_empty = bars + 10;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* epi_go = abort_flag + 1;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const uint32_t pair = blockIdx.x >> 1;
+  const bool leader_cta = rank == 0;
+
+  if (warp == 0) {
+    if (lane < 12) {
+      // full: the leader's three producers; empty, accumulator full: one commit; accumulator empty: the
+      // epilogue warps of both CTAs
+      const uint32_t count = (lane < 4) ? 3u : (lane < 10) ? 1u : (uint32_t)(2 * 4 * kGroups);
+      mbar_init(&bars[lane], count);
+    }
+    if (lane == 0) {
+      grid_launch_dependents();
+      *abort_flag = 0;
+    }
+    __syncwarp();
+    if (lane == 0) {
+      mbar_fence_init();
+      fence_proxy_async_smem();
+    }
+  } else if (warp == 1) {
+    tmem_alloc2(tmem_slot, kTmemCols);
+    tmem_relinquish2();
+  } else if (lane == 0) {
+    if (warp == kFirstExtraProducerWarp) prefetch_tensormap(&tm_b);
+    if (warp == kFirstExtraProducerWarp + 1) {
+      prefetch_tensormap(&tm_a);
+      if (SPARSE) prefetch_tensormap(&tm_meta);
+    }
+    if (warp == 2) {
+      prefetch_tensormap(&tm_y);
+      prefetch_tensormap(&tm_y_tail);
+    }
+  }
+  // both CTAs' barriers and TMEM exist before either touches the other's
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0 || warp >= kFirstExtraProducerWarp) {
+    // ------------------------------------------------------------------ TMA producers (whole warps)
+    const uint32_t full0_local = smem_u32(bar_full);
+    const uint32_t full0_leader = map_to_cta(full0_local, 0);
+    const uint32_t empty0 = smem_u32(bar_empty), ring0 = smem_u32(ring);
+    if (warp == 0)
+      pair_producer_role<SPARSE, kRoleActFirst>(&tm_a, &tm_b, &tm_meta, p, rank, pair, full0_leader, full0_local, empty0,
+                                                ring0, abort_flag);
+    else if (warp == kFirstExtraProducerWarp)
+      pair_producer_role<SPARSE, kRoleActSecond>(&tm_a, &tm_b, &tm_meta, p, rank, pair, full0_leader, full0_local,
+                                                 empty0, ring0, abort_flag);
+    else
+      pair_producer_role<SPARSE, kRoleWeights>(&tm_a, &tm_b, &tm_meta, p, rank, pair, full0_leader, full0_local, empty0,
+                                               ring0, abort_flag);
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (leader_cta) {
+      const uint32_t idesc = make_idesc_bf16(2 * kTileM, (uint32_t)p.BN, SPARSE);
+      const uint32_t grp_desc = grp_bytes >> 4;
+      const uint32_t half_desc = half_bytes >> 4;
+      const uint32_t ring_lo0 = desc_lo(smem_u32(ring));
+      const uint32_t full0 = smem_u32(bar_full);
+      const uint32_t empty0 = smem_u32(bar_empty), accf0 = smem_u32(bar_acc_full);
+      const uint32_t meta_tmem0 = tmem_base + kMetaCol;
+      const int tail_c = p.C_in - (p.cblocks - 1) * kBlockK;
+      const int mma_full = SPARSE ? 2 : 4;
+      const int mma_tail = SPARSE ? ((tail_c + 31) >> 5) : ((tail_c + 15) >> 4);
+      const int tail_start = (tail_c == kBlockK) ? p.kblocks : (p.cblocks - 1) * p.taps;  // first k-block of the tail
+      uint32_t g = 0, ph = 0, tcount = 0, mslot = 0;
+      uint32_t ready = 0;  // the look-ahead saw the group in hand complete
+      bool ok = true;
+      WorkIter work(p, pair);
+      Segment seg;
+      for (; ok && work.next(seg); ++tcount) {
+        const uint32_t buf = tcount & 1u;
+        const uint32_t aph = (tcount >> 1) & 1u;
+        if (!mbar_wait_bounded(&bar_acc_empty[buf], aph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * kAccCol1;
+        uint32_t accumulate = 0;
+        for (int a = 0; a < p.a_tiles; ++a) {
+          if (!ready && !mbar_wait_a(full0 + 8u * g, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+          {  // look ahead at the next group's barrier (the ring runs on across tiles) while this group's
+             // MMAs are issued; the answer is used at the top of the next iteration
+            const uint32_t g_next = (g + 1u == (uint32_t)p.ring_groups) ? 0u : g + 1u;
+            ready = mbar_test_a(full0 + 8u * g_next, g_next == 0u ? ph ^ 1u : ph);
+          }
+          tc_fence_after();
+          const uint32_t a_lo = ring_lo0 + g * grp_desc;
+          const uint32_t b0_lo = a_lo + (C::kAGroupBytes >> 4);
+          const uint32_t b1_lo = b0_lo + half_desc;
+          const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
+          const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
+          if (SPARSE) {
+            const uint32_t meta_tmem = meta_tmem0 + 4u * mslot;
+            mslot ^= 1u;
+            tc2_cp_128x128b_w(meta_tmem, a_lo + (kATileBytes >> 4));
+            tc2_mma_sparse_w(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
+            if (n0 > 1) tc2_mma_sparse_w(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
+            if (n1 > 0) tc2_mma_sparse_w(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
+            if (n1 > 1) tc2_mma_sparse_w(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
+          } else {
+            const uint32_t a1_lo = a_lo + (kATileBytes >> 4);
+            for (int kk = 0; kk < n0; ++kk)
+              tc2_mma_dense_w(d_tmem, a_lo + 2u * kk, b0_lo + 2u * kk, idesc, (kk > 0) ? 1u : accumulate);
+            for (int kk = 0; kk < n1; ++kk) tc2_mma_dense_w(d_tmem, a1_lo + 2u * kk, b1_lo + 2u * kk, idesc, 1u);
+          }
+          accumulate = 1;
+          tc2_commit_both_w(empty0 + 8u * g);
+          if (++g == (uint32_t)p.ring_groups) {
+            g = 0;
+            ph ^= 1u;
+          }
+        }
+        if (ok) tc2_commit_both_w(accf0 + 8u * buf);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (as in the one-CTA kernel)
+    const int grp = (warp - 2) >> 2;
+    const int q = warp & 3;
+    const bool leader = (q == 2 && lane == 0);
+    const int act = activation_of(p.flags);
+    const int col_base = grp * (p.BN >> 1);
+    uint8_t* my_stage = out_stage + grp * 2 * kPieceBytes;
+    volatile int* my_go = epi_go + 2 * grp;
+    const uint32_t acc_empty0_leader = map_to_cta(smem_u32(bar_acc_empty), 0);
+    const uint32_t st_offset = (uint32_t)(q >> 1) * kHalfPieceBytes + (uint32_t)(lane & 7) * 128u +
+                               ((((uint32_t)(q & 1) * 4u + (uint32_t)(lane >> 3)) ^ (uint32_t)(lane & 7)) << 4);
+    uint32_t tcount = 0, piece_count = 0;
+    grid_dependency_wait();
+    WorkIter work(p, pair);
+    Segment seg;
+    for (; work.next(seg); ++tcount) {
+      const int pt = seg.tile / p.m_tiles;
+      const int m = 2 * (seg.tile - pt * p.m_tiles) + (int)rank;
+      const uint32_t buf = tcount & 1u;
+      const uint32_t aph = (tcount >> 1) & 1u;
+      const bool got = mbar_wait_bounded(&bar_acc_full[buf], aph, abort_flag, kWaitLimitCycles, 64);
+      if (leader) my_go[tcount & 1u] = (got && *abort_flag == 0) ? 1 : 0;
+      epilogue_bar_sync(grp);
+      if (my_go[tcount & 1u] == 0) break;
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCol1 + col_base;
+      const bool real = m < p.m_real;  // (the odd CTA of the last pair may have no channels at all)
+      float bias_v[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int co = m * kTileM + q * 32 + 8 * i + (lane >> 2);
+        bias_v[i] = ((p.flags & SSCONV_FLAG_BIAS) && co < p.C_out) ? p.bias[co] : 0.0f;
+      }
+#pragma unroll 1
+      for (int piece = 0; piece < p.pieces; ++piece, ++piece_count) {
+        uint8_t* stage = my_stage + (piece_count & 1u) * kPieceBytes;
+        uint32_t r[kPiece];
+        tc_ld_piece(t_row + piece * kPiece, r);
+        tc_wait_ld();
+        if (piece == p.pieces - 1) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(acc_empty0_leader + 8u * buf);
+        }
+        const uint32_t st_addr = smem_u32(stage) + st_offset;
+        if (act == kActRelu)
+          stage_piece<kActRelu, false>(r, bias_v, st_addr);
+        else if (act == kActGelu)
+          stage_piece<kActGelu, false>(r, bias_v, st_addr);
+        else
+          stage_piece<kActNone, false>(r, bias_v, st_addr);
+        fence_proxy_async_smem();
+        if (leader) bulk_wait_group_read0();
+        epilogue_bar_sync(grp);
+        if (leader) {
+          const int q_piece = pt * p.BN + col_base + piece * kPiece;
+          if (real && q_piece < p.Q) {
+            const CUtensorMap* map = (piece == p.pieces - 1 && p.tail_cols != kPiece) ? &tm_y_tail : &tm_y;
+            tma_store_2d(map, stage, m * kTileM, q_piece);
+            if (m * kTileM + 64 < p.C_out) tma_store_2d(map, stage + kHalfPieceBytes, m * kTileM + 64, q_piece);
+          }
+          bulk_commit_group();
+        }
+      }
+    }
+    if (leader) bulk_wait_group_read0();
+  }
+
+  // ------------------------------------------------------------------ teardown
+  // Neither CTA may leave while the other can still signal its barriers or read its shared memory.
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  if (*abort_flag != 0) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    if (threadIdx.x == 0 && p.dev_status != nullptr) atomicExch(p.dev_status, (int)SSCONV_ERR_TIMEOUT);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc2(tmem_base, kTmemCols);
+  }
+}
+
+
+// ---------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -957,9 +1267,16 @@ static double kblock_cycles(int BN, int stage_bufs, bool steady_ring = true) {
   return (steady_ring && ring > t) ? ring : t;
 }
 
-// Process-wide override of the planner's tile width (ssconv_tune): 0 lets the model choose.
+// Process-wide overrides of the planner (ssconv_tune): tile width (0 lets the model choose) and the
+// use of the pair kernel.
 static int g_tune_bn = 0;
+static int g_tune_pair = -1;  // -1: the model chooses; 0: never the pair kernel; 1: wherever it applies
 int32_t set_tuning(int32_t option, int32_t value) {
+  if (option == SSCONV_TUNE_PAIR) {
+    if (value < -1 || value > 1) return SSCONV_ERR_BAD_DESC;
+    g_tune_pair = value;
+    return SSCONV_OK;
+  }
   if (option == SSCONV_TUNE_TILE_POSITIONS) {
     if (value != 0 && (value < 48 || value > kBN || value % 16 != 0)) return SSCONV_ERR_BAD_DESC;
     g_tune_bn = value;
@@ -972,6 +1289,8 @@ int32_t set_tuning(int32_t option, int32_t value) {
 struct Plan {
   int BN;
   bool split;
+  double cost = 0.0;  // the model's cycles for the layer
+  bool pair = false;  // 256-channel tiles on CTA pairs (ssconv_fwd_pair_kernel)
 };
 template <bool SPARSE>
 static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force_split, int max_bn = kBN,
@@ -992,6 +1311,7 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
       best.BN = BN;
     }
   }
+  best.cost = best_cost;
   // Even split of K ("stream-K"), when many SMs would still idle and K is deep: every CTA gets the
   // same number of groups; parked partial tiles cost L2 traffic in proportion to the tile width.
   const int a_tiles = geo.stages;
@@ -1010,10 +1330,62 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
         best_split.BN = BN;
       }
     }
+    best_split.cost = best_split_cost;
     if (best_cost > kSplitAdvantage * best_split_cost) return best_split;
   }
   return best;
 }
+
+// Pair kernel: a CTA holds the group's weights and half of each activation tile.
+static int pair_ring_groups(uint32_t a_group_bytes, int BN) {
+  const int n = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(2)) / (a_group_bytes + (uint32_t)BN * 128u));
+  return n > kMaxGroups ? kMaxGroups : n;
+}
+// Plan for the pair kernel (whole tiles of 256 channels x BN positions dealt out to workers / 2
+// pairs), or BN = 0 where it does not apply.  Per k-block a CTA of a pair takes in its weights and
+// 64 BN bytes of activations (at a fitted 48 bytes per cycle) and the issuing warp does the work of
+// one CTA for two.  Measured on the ResNet-50 and ConvNeXt layer sets: layers with a deep K and
+// several tiles per pair gain 1.2-1.5x; layers with fewer than 12 k-blocks are bound by their
+// epilogues and output traffic, where two CTAs in lock step do worse than two independent ones
+// (0.6-0.9x), and with about one tile per pair the fixed costs decide: neither kind is paired
+// unless the override forces it.
+constexpr double kFillBytesPerCyclePair = 48.0;
+constexpr int kPairMinKBlocks = 12;
+constexpr double kPairMinTilesPerPair = 1.5;  // counted at the widest tile
+template <bool SPARSE>
+static Plan plan_pair(long long Q, const Geometry& geo, int workers, bool forced) {
+  Plan best{0, false};
+  best.pair = true;
+  const int pairs = workers / 2;
+  if (geo.m_tiles < 2 || pairs < 1) return best;
+  if (!forced && geo.kblocks < kPairMinKBlocks) return best;
+  const int mp_tiles = (geo.m_tiles + 1) / 2;
+  if (!forced && (double)(((Q + kBN - 1) / kBN) * mp_tiles) < kPairMinTilesPerPair * pairs) return best;
+  int max_bn = kBN, min_bn = 64;
+  if (g_tune_bn != 0) max_bn = min_bn = g_tune_bn < 64 ? 64 : g_tune_bn;
+  const double a_bytes = Cfg<SPARSE>::kAGroupBytes / 2.0;
+  const double issue = SPARSE ? kIssueSparse : kIssueDense;
+  for (int BN = max_bn; BN >= min_bn; BN -= 16) {
+    const int groups = pair_ring_groups(Cfg<SPARSE>::kAGroupBytes, BN);
+    if (groups < 2) continue;
+    const long long tiles = ((Q + BN - 1) / BN) * mp_tiles;
+    const long long per_pair = (tiles + pairs - 1) / pairs;
+    const int pieces = (BN / 2 + kPiece - 1) / kPiece;
+    const double fill = (a_bytes + 64.0 * BN) / kFillBytesPerCyclePair;
+    const double pipe = SPARSE ? 2.0 * (35.0 + 0.5 * BN) + 11.0 : 4.0 * (5.0 + 0.49 * BN);
+    const double ring = (kLoadLatencyCycles + 2.0 * fill + 2.0 * issue) / (2.0 * groups);
+    double t = fill > issue ? fill : issue;
+    t = t > pipe ? t : pipe;
+    t = t > ring ? t : ring;
+    const double cost = (double)per_pair * geo.kblocks * t + pieces * kEpiloguePieceCycles;
+    if (best.BN == 0 || cost < 0.97 * best.cost) {
+      best.BN = BN;
+      best.cost = cost;
+    }
+  }
+  return best;
+}
+constexpr double kPairAdvantage = 1.05;  // the pair kernel only if the model predicts at least this gain
 
 constexpr size_t scratch_bytes(int workers) {
   return 2 * (size_t)workers * kRegionBytes;
@@ -1022,6 +1394,7 @@ size_t workspace_bytes() { return scratch_bytes(kMaxWorkers); }
 
 static int g_sm_count[64] = {0};
 static bool g_attr_set[64][2][2] = {{{false}}};
+static bool g_pair_attr_set[64][2] = {{false}};
 
 // Dense layers with 8 input channels (a channel-padded RGB stem): a k-block of 64 K-elements is 8
 // filter taps instead of 64 channels of one tap, which would be 7/8 padding.
@@ -1059,9 +1432,19 @@ static int widest_tile(uint32_t a_group_bytes, int stage_bufs) {
   return BN;
 }
 
+// The plan for a layer without a residual: one-CTA tiles (whole or K split) or the pair kernel.
+template <bool SPARSE>
+static Plan choose_plan(const ssconv_desc_t& d, long long Q, const Geometry& geo, int workers, bool force_split) {
+  const Plan plan = plan_layer<SPARSE>(Q, geo, workers, force_split);
+  if (force_split || small_channel_mode(d, SPARSE) || g_tune_pair == 0) return plan;
+  const Plan pair = plan_pair<SPARSE>(Q, geo, workers, g_tune_pair == 1);
+  if (pair.BN != 0 && (g_tune_pair == 1 || plan.cost > kPairAdvantage * pair.cost)) return pair;
+  return plan;
+}
+
 // What launch_forward_impl would do for this layer on the current device.
 int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* split, int32_t* ctas,
-                   int32_t* ring_groups) {
+                   int32_t* ring_groups, int32_t* pair) {
   int dev = 0;
   const int32_t st = current_device(&dev);
   if (st != SSCONV_OK) return st;
@@ -1069,15 +1452,25 @@ int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* sp
   const long long Q = (long long)d.N * out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h) *
                       out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
   const int workers = g_sm_count[dev] < kMaxWorkers ? g_sm_count[dev] : kMaxWorkers;
-  const Plan plan = sparse ? plan_layer<true>(Q, geo, workers, false) : plan_layer<false>(Q, geo, workers, false);
-  const long long tiles = ((Q + plan.BN - 1) / plan.BN) * geo.m_tiles;
+  const Plan plan = sparse ? choose_plan<true>(d, Q, geo, workers, false) : choose_plan<false>(d, Q, geo, workers, false);
+  const uint32_t a_group_bytes = sparse ? Cfg<true>::kAGroupBytes : Cfg<false>::kAGroupBytes;
+  const long long q_tiles = (Q + plan.BN - 1) / plan.BN;
+  if (bn) *bn = plan.BN;
+  if (pair) *pair = plan.pair ? 1 : 0;
+  if (plan.pair) {
+    const long long tiles = q_tiles * ((geo.m_tiles + 1) / 2);
+    const long long pairs = workers / 2;
+    if (split) *split = 0;
+    if (ctas) *ctas = (int32_t)(2 * (tiles < pairs ? tiles : pairs));
+    if (ring_groups) *ring_groups = pair_ring_groups(a_group_bytes, plan.BN);
+    return SSCONV_OK;
+  }
+  const long long tiles = q_tiles * geo.m_tiles;
   const bool do_split = plan.split && geo.stages > 1;
   const long long work = do_split ? tiles * geo.stages : tiles;
-  if (bn) *bn = plan.BN;
   if (split) *split = do_split ? 1 : 0;
   if (ctas) *ctas = (int32_t)(work < workers ? work : workers);
-  if (ring_groups)
-    *ring_groups = ring_groups_for(sparse ? Cfg<true>::kAGroupBytes : Cfg<false>::kAGroupBytes, plan.BN, 2);
+  if (ring_groups) *ring_groups = ring_groups_for(a_group_bytes, plan.BN, 2);
   return SSCONV_OK;
 }
 
@@ -1113,7 +1506,8 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   // per group, which narrows the widest tile that still leaves room for two ring groups.  (When K
   // is split the finishing kernel adds the residual to the split tiles; the main kernel then keeps
   // two buffers and one piece of lookahead for the whole tiles it may also own.)
-  Plan plan = plan_layer<SPARSE>(Q, geo, workers, force_split);
+  Plan plan = residual != nullptr ? plan_layer<SPARSE>(Q, geo, workers, force_split)
+                                  : choose_plan<SPARSE>(d, Q, geo, workers, force_split);
   int stage_bufs = 2;
   if (residual != nullptr && !plan.split) {
     stage_bufs = 4;
@@ -1126,9 +1520,16 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   const int BN = plan.BN;
   const int pieces = (BN / 2 + kPiece - 1) / kPiece;
   const int tail_cols = BN / 2 - (pieces - 1) * kPiece;
-  const uint32_t grp_bytes = group_bytes(C::kAGroupBytes, BN);
-  const int ring_groups = ring_groups_for(C::kAGroupBytes, BN, stage_bufs);
+  const bool pair = plan.pair;  // a CTA of a pair holds half of each activation tile
+  const uint32_t grp_bytes = pair ? C::kAGroupBytes + (uint32_t)BN * 128u : group_bytes(C::kAGroupBytes, BN);
+  const int ring_groups = pair ? pair_ring_groups(C::kAGroupBytes, BN) : ring_groups_for(C::kAGroupBytes, BN, stage_bufs);
   const uint32_t smem_bytes = 1024 + (uint32_t)ring_groups * grp_bytes + staging_bytes(stage_bufs) + kBarrierBytes;
+  if (pair && !g_pair_attr_set[dev][SPARSE ? 1 : 0]) {
+    if (cudaFuncSetAttribute(ssconv_fwd_pair_kernel<SPARSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kMaxSmemBytes) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
+    g_pair_attr_set[dev][SPARSE ? 1 : 0] = true;
+  }
 
   CUtensorMap tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail;
   // activations: NHWC seen as (c, w, h, n), im2col mode; elements outside the image read as zero
@@ -1145,7 +1546,8 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     // (measured: up to 4 % faster on such layers, 4 % slower on a strided one, nothing elsewhere)
     const bool wide_pixels = d.C_in >= 128 && d.stride_h == 1 && d.stride_w == 1;
     CUresult r = g_encode_im2col(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), dims, strides,
-                                 lower, upper, small_c ? 8u : (cuuint32_t)kBlockK, (cuuint32_t)BN, estr,
+                                 lower, upper, small_c ? 8u : (cuuint32_t)kBlockK,
+                                 (cuuint32_t)(pair ? BN / 2 : BN), estr,
                                  CU_TENSOR_MAP_INTERLEAVE_NONE,
                                  small_c ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
                                  wide_pixels ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -1171,6 +1573,19 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     CUresult r = g_encode_tiled(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(weights), dims, strides,
                                 box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                 small_c ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
+  }
+  // pair kernel: the metadata images as rows of 16 bytes, one box per image (128 rows), so that they
+  // come in by a tensor copy, which unlike the plain bulk copy can signal a barrier in the peer CTA
+  CUtensorMap tm_meta = tm_a;
+  if (pair && SPARSE) {
+    cuuint64_t dims[2] = {16, (cuuint64_t)geo.m_tiles * geo.stages * kTileM};
+    cuuint64_t strides[1] = {16};
+    cuuint32_t box[2] = {16, (cuuint32_t)kTileM};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode_tiled(&tm_meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(meta), dims, strides, box,
+                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
   }
@@ -1230,9 +1645,10 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.taps = geo.taps;
   p.cblocks = geo.cblocks;
   p.kblocks = geo.kblocks;
-  p.m_tiles = geo.m_tiles;
+  p.m_real = geo.m_tiles;
+  p.m_tiles = pair ? (geo.m_tiles + 1) / 2 : geo.m_tiles;
   const long long q_tiles = (Q + BN - 1) / BN;
-  p.num_tiles = (int)(q_tiles * geo.m_tiles);
+  p.num_tiles = (int)(q_tiles * p.m_tiles);
   p.a_tiles = geo.stages;
   p.flags = d.flags;
   p.bias = bias;
@@ -1249,14 +1665,19 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     if (ws == nullptr || ws_bytes < scratch_bytes(worker_cap)) return SSCONV_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(ws) & 15u) return SSCONV_ERR_ALIGNMENT;
     p.ws_regions = static_cast<float4*>(ws);
+  } else if (pair) {
+    const int pairs = workers / 2;
+    grid = 2 * (p.num_tiles < pairs ? p.num_tiles : pairs);  // the tiles are dealt out to the pairs
+    p.ws_regions = nullptr;
   } else {
     grid = p.num_tiles < workers ? p.num_tiles : workers;
     p.ws_regions = nullptr;
   }
   {
     const long long work = p.split ? units : (long long)p.num_tiles;
-    p.work_quot = (int)(work / grid);
-    p.work_rem = (int)(work % grid);
+    const int dealt_to = pair ? grid / 2 : grid;
+    p.work_quot = (int)(work / dealt_to);
+    p.work_rem = (int)(work % dealt_to);
   }
   // Programmatic stream serialisation: this grid's set-up (barriers, TMEM, tensor-map fetch, index
   // arithmetic) may overlap the tail of the previous kernel in the stream; the kernel itself
@@ -1266,13 +1687,18 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   cfg.blockDim = dim3((unsigned)kThreads);
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;  // pair kernel: clusters of two CTAs
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pair ? 2 : 1;
   const cudaError_t launched =
-      residual != nullptr
+      pair ? cudaLaunchKernelEx(&cfg, ssconv_fwd_pair_kernel<SPARSE>, tm_a, tm_b, tm_meta, tm_y, tm_y_tail, p)
+      : residual != nullptr
           ? cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, true>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p)
           : cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, false>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p);
   if (launched != cudaSuccess) return SSCONV_ERR_CUDA;
