@@ -1,16 +1,21 @@
 #!/usr/bin/env python
 """Benchmark of the 2:4 sparse convolution forward on B200.
 
-A step is one pass of the masked-convolution forward over every layer of the ResNet-18-shaped
-3x3 sweep at batch 32 (seeded synthetic activations and weights, masks by magnitude selected
-and compressed once beforehand with the library's own kernels).  The reported value is
-dense-equivalent TFLOP/s (2*P*C_out*K per layer) over all ranks.  Each rank rotates over
-several input/output buffer sets whose total footprint exceeds the L2 cache, so every step
-reads its activations from HBM.
+Default workload: the convolution stack of a Torchvision-shaped ResNet-50 at batch 256 per GPU
+(the largest configuration: a dense 7x7 stem on 3-channel images, a 3x3 max-pool and 52 masked
+convolutions; seeded synthetic images and weights, masks by magnitude, selected and compressed
+once beforehand with the library's own kernels).  A step is one forward pass of the whole stack.
+The reported value is dense-equivalent TFLOP/s (2*P*C_out*K per convolution, the stem counted with
+its 3 real input channels) over all ranks; images per second, the dense counterpart, a per-layer
+table with each layer's roofline, the end-to-end figure with host buffers, the CPU oracle and
+short summaries of the three per-layer sweeps (ResNet-18 3x3 sweep, ResNet-50 bottleneck layers,
+ConvNeXt-T point-wise layers) ride in the same JSON line.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload-config 2|3|4|5] [--train]
 
-Prints exactly one JSON line on rank 0.
+Prints exactly one JSON line on rank 0.  With --gpus N > 1 and no torchrun environment it starts N
+ranks itself (one per GPU; the ranks share nothing but the timing barrier).
 """
 from __future__ import annotations
 
@@ -30,10 +35,10 @@ if ROOT not in sys.path:
 METRIC = "dense-equiv TFLOP/s of 2:4 sparse conv fwd (bf16), % of sparse-TC roofline, xdense"
 WORKLOADS = {2: "resnet18_3x3_sweep_bf16_nhwc_batch32", 3: "resnet50_bottleneck_layers_bf16_nhwc_batch64",
              4: "convnext_t_pointwise_layers_bf16_nhwc_batch128",
-           5: "resnet50_conv_stack_end_to_end_bf16_nhwc_batch256"}
-CONFIG_ID = 2          # the benchmarked workload; --workload-config picks another for layer tables
+             5: "resnet50_conv_stack_end_to_end_bf16_nhwc_batch256"}
+CONFIG_ID = 5          # the benchmarked workload; --workload-config picks one of the per-layer sweeps instead
 WORKLOAD = WORKLOADS[CONFIG_ID]
-L2_BYTES = 126 * 2 ** 20
+MIN_REGIONS = 30       # timed regions of --steps steps each; the median is reported
 
 
 def load_peaks():
@@ -47,14 +52,22 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-def timed_layers():
+def timed_layers(config_id=None):
     from paper_2411_00288_b200 import synth
-    return [s for s in synth.config_layers(CONFIG_ID) if not s.extra]
+    return [s for s in synth.config_layers(CONFIG_ID if config_id is None else config_id) if not s.extra]
+
+
+def spread(values):
+    """Median, extremes and the 10th / 90th percentiles of a list of region times."""
+    v = sorted(values)
+    n = len(v)
+    return {"median": statistics.median(v), "min": v[0], "max": v[-1], "p10": v[int(0.1 * (n - 1))],
+            "p90": v[int(round(0.9 * (n - 1)))], "regions": n}
 
 
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while a region runs."""
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the benchmark runs."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
@@ -64,6 +77,7 @@ class ClockSampler:
         self.proc = None
         self.lines = []
         self.thread = None
+        self.marks = {}
 
     def start(self):
         try:
@@ -80,70 +94,120 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
-    def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
+    def mark(self, name):
+        """Remember how many samples had arrived when leg `name` started."""
+        self.marks[name] = len(self.lines)
+
+    def _summary(self, lines):
+        sm, mx, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for ln in lines:
             parts = [p.strip() for p in ln.split(",")]
             if len(parts) < 7:
                 continue
             try:
                 sm.append(float(parts[0]))
                 mx.append(float(parts[1]))
+                power.append(float(parts[2]))
             except ValueError:
                 continue
             for name, val in zip(names, parts[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        # samples taken while the GPU was working (an idle GPU drops its clock between legs)
+        busy = [c for c, w in zip(sm, power) if w >= 0.5 * max(power)] if power else []
+        return {"sm_mhz": statistics.median(busy) if busy else (statistics.median(sm) if sm else None),
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "samples_under_load": len(busy),
+                "power_w_max": max(power) if power else None, "reasons": sorted(reasons)}
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)   # one more sampling period
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        out = self._summary(self.lines)
+        bounds = sorted(self.marks.items(), key=lambda kv: kv[1]) + [("end", len(self.lines))]
+        out["legs"] = {}
+        for (name, lo), (_, hi) in zip(bounds, bounds[1:]):
+            leg = self._summary(self.lines[lo:hi])
+            out["legs"][name] = {k: leg[k] for k in ("sm_mhz", "samples", "reasons")}
+        return out
 
 
 # ----------------------------------------------------------------------------- CPU oracle leg
-def oracle_leg(target_seconds: float = 15.0):
-    """Time the fp64 CPU oracle, as it stands, on a bounded sample of the same workload."""
-    import numpy as np  # noqa: F401
+_ORACLE_WEIGHTS = {}
+
+
+def stack_conv_specs(batch):
+    """The 53 convolutions of the benchmarked stack at the given batch: (spec, masked?)."""
+    from paper_2411_00288_b200 import synth
+    return [(st.spec, st.kind == "conv") for st in synth.resnet50_stack(batch) if st.kind != "maxpool"]
+
+
+def stack_flops(batch):
+    """Dense-equivalent FLOPs of one pass: 2*P*C_out*K per convolution; the stem with its 3 real channels."""
+    total = 0
+    for spec, masked in stack_conv_specs(batch):
+        total += spec.dense_equiv_flops if masked else spec.dense_equiv_flops * 3 // spec.C_in
+    return total
+
+
+def oracle_leg(target_seconds: float = 15.0, config_id=None):
+    """Time the fp64 CPU oracle, as it stands, on a bounded sample of the same workload: every
+    convolution of the workload on seeded inputs of its own shape, full output tensors, at the largest
+    batch that keeps the leg near `target_seconds`."""
+    import dataclasses
     from oracle import masks
     from oracle.conv import conv2d_f64, threads
     from paper_2411_00288_b200 import synth
     from tests import parity
-    import dataclasses
+
+    cfg = CONFIG_ID if config_id is None else config_id
+    full_batch = {2: 32, 3: 64, 4: 128, 5: 256}[cfg]
+
+    def layer_list(batch):
+        if cfg == 5:
+            return stack_conv_specs(batch)
+        return [(dataclasses.replace(s, N=batch), True) for s in timed_layers(cfg)]
 
     def run(batch):
         flops, secs = 0, 0.0
-        for spec in timed_layers():
-            spec_b = dataclasses.replace(spec, N=batch)
-            inp = synth.make_inputs(spec_b)
-            pat = parity.oracle_pattern(inp)
-            wb = synth.bf16_bits(inp.w)
-            m = masks.mask_from_pattern(pat, wb.shape)
-            xb = synth.bf16_bits(inp.x)
+        for idx, (spec, masked) in enumerate(layer_list(batch)):
+            key = (cfg, idx)
+            if key not in _ORACLE_WEIGHTS:   # weights, mask and bias do not depend on the batch: drawn once
+                inp = synth.make_inputs(dataclasses.replace(spec, N=1))
+                wb = synth.bf16_bits(inp.w)
+                m = masks.mask_from_pattern(parity.oracle_pattern(inp), wb.shape) if masked else None
+                _ORACLE_WEIGHTS[key] = (wb, m, inp.bias.numpy())
+            wb, m, bias = _ORACLE_WEIGHTS[key]
+            xb = synth.bf16_bits(synth.make_inputs(spec, x_only=True).x)
             t0 = time.perf_counter()
-            conv2d_f64(parity.oracle_shape(spec_b), xb, wb, mask=m, bias=inp.bias.numpy())
+            conv2d_f64(parity.oracle_shape(spec), xb, wb, mask=m, bias=bias)
             secs += time.perf_counter() - t0
-            flops += spec_b.dense_equiv_flops
+            flops += spec.dense_equiv_flops if masked else spec.dense_equiv_flops * 3 // spec.C_in
         return flops, secs
 
     f1, s1 = run(1)
     batch = 1
     for b in (32, 16, 8, 4, 2):
-        if s1 * b <= target_seconds * 1.5:
+        if b <= full_batch and s1 * b <= target_seconds * 1.5:
             batch = b
             break
     flops, secs = (f1, s1) if batch == 1 else run(batch)
+    what = ("the 53 convolutions of the stack" if cfg == 5 else f"all {len(layer_list(1))} layers of the sweep")
     return {"value": flops / secs / 1e12, "unit": "TFLOP/s", "cores": threads(), "kind": "oracle",
-            "sample": f"all {len(timed_layers())} layers of the sweep at batch {batch} (of 32), full output tensors, "
-                      f"{secs:.1f} s of CPU time", "seconds": secs, "batch": batch}
+            "sample": f"{what} at batch {batch} (of {full_batch}), each on seeded inputs of its own shape, full "
+                      f"output tensors, {secs:.1f} s of CPU time",
+            "seconds": secs, "batch": batch, "images_per_s": batch / secs if cfg == 5 else None}
 
 
 def reference_arm(args):
+    """The reference arm: the fp64 CPU oracle as it stands (the paper publishes no code to install), on
+    the same workload, metric and unit; each step is a bounded sample of it."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -172,112 +236,169 @@ def reference_arm(args):
     print(json.dumps(line))
 
 
-# DRAM traffic of the sparse forward kernels of one step (7 launches of ssconv_fwd_kernel<sparse> and
-# the finishing kernel of the one split layer), dram__bytes_read.sum + dram__bytes_write.sum from an
-# ncu capture of this workload (summary and command: profiles/bench_resnet18_sweep_dram_traffic.md).
-# It belongs to the kernel sources with the digest below; with other sources the bench reports null.
-TRAFFIC_BYTES_PER_STEP = 66.41e6
-TRAFFIC_SOURCES = ("forward.cu", "sm100_ptx.cuh", "layout.cuh")
-TRAFFIC_SOURCES_SHA256 = "f5473a3b686cfcf438dbd934658b158346017ede67fe2f4402739fec885f9b3f"
+# ----------------------------------------------------------------------------- timing helpers
+class Timer:
+    """CUDA-event timing of graph replays on the current stream, with the barrier / synchronise
+    bracket and the maximum over ranks."""
 
+    def __init__(self, torch, dist, ranks, dev, distributed):
+        self.torch, self.dist, self.ranks, self.dev, self.distributed = torch, dist, ranks, dev, distributed
 
-def measured_traffic():
-    import hashlib
-    h = hashlib.sha256()
-    root = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2411_00288_b200", "csrc")
-    try:
-        for name in TRAFFIC_SOURCES:
-            with open(os.path.join(root, name), "rb") as fh:
-                h.update(fh.read())
-    except OSError:
-        return None
-    return TRAFFIC_BYTES_PER_STEP if h.hexdigest() == TRAFFIC_SOURCES_SHA256 else None
+    def barrier(self):
+        if self.distributed:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
 
+    def capture(self, fn):
+        """Record fn()'s launches into a CUDA graph (the launches are the same C-ABI calls; the graph
+        only removes the host-side launch cost from the timed region)."""
+        g = self.torch.cuda.CUDAGraph()
+        with self.torch.cuda.graph(g):
+            fn()
+        return g
 
-# ----------------------------------------------------------------------------- conv stack, end to end
-def stack_arm(args):
-    """ResNet-50-shaped convolution stack (dense stem, max-pool, 52 masked convolutions) at batch 256
-    per GPU: images per second of the whole stack, recorded into one CUDA graph and replayed, with
-    the same stack on the dense kernel for comparison.  One JSON line on rank 0."""
-    import torch
-    import torch.distributed as dist
-    from paper_2411_00288_b200 import api, synth, stack, ranks, build as libbuild
-
-    rank, local_rank, world = ranks.env_ranks()
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    if rank == 0:
-        libbuild.build()
-    if world > 1:
-        dist.barrier()
-    api.lib()
-    batch = args.batch or 256
-    steps_def = synth.resnet50_stack(batch, residual=args.residual)
-    net = stack.ConvStack(steps_def, dev, with_dense=True)
-    g = torch.Generator().manual_seed(synth.SEED_BASE + 577 + rank)
-    x = torch.zeros((batch, 224, 224, 8), dtype=torch.bfloat16)
-    x[..., :3] = torch.randn((batch, 224, 224, 3), generator=g, dtype=torch.float32).to(torch.bfloat16)
-    xd = x.to(dev)
-    warmup, steps = max(3, args.warmup), min(args.steps, 200)
-
-    def timed(sparse):
-        for _ in range(2):
-            net.forward(xd, sparse=sparse)
-        torch.cuda.synchronize()
-        c0 = api.ssconv_launch_count()
-        net.forward(xd, sparse=sparse)
-        launches = api.ssconv_launch_count() - c0
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            net.forward(xd, sparse=sparse)
-        for _ in range(warmup):
-            graph.replay()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+    def region(self, graphs, replays):
+        """Replay graphs[i % len] for i < replays between two events; max over ranks, in ms."""
+        if not isinstance(graphs, (list, tuple)):
+            graphs = [graphs]
+        e0 = self.torch.cuda.Event(enable_timing=True)
+        e1 = self.torch.cuda.Event(enable_timing=True)
+        self.barrier()
         e0.record()
-        for _ in range(steps):
-            graph.replay()
+        for i in range(replays):
+            graphs[i % len(graphs)].replay()
         e1.record()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-        return ranks.max_over_ranks(e0.elapsed_time(e1) / steps, dev), launches
+        self.barrier()
+        return self.ranks.max_over_ranks(e0.elapsed_time(e1), self.dev)
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    ms_sparse, launches = timed(True)
-    ms_dense, _ = timed(False)
-    clocks = sampler.stop() if rank == 0 else None
-    status = int(net.status.item())
-    if rank == 0:
-        flops = net.conv_flops()
-        print(json.dumps({
-            "metric": "end-to-end images/s of the ResNet-50-shaped convolution stack, 2:4 masked (bf16)",
-            "value": ranks.job_throughput(batch, world, ms_sparse), "unit": "images/s", "n_gpus": world,
-            "steps": steps, "warmup": warmup, "ms_per_step": ms_sparse, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD + ("_with_skip_connections" if args.residual else ""),
-                       "batch_per_gpu": batch,
-                       "stack": "stem 7x7 s2 (dense, input padded 3 -> 8 channels), 3x3 s2 max-pool, 16 "
-                                "bottlenecks as reduce -> 3x3 -> expand with bias + ReLU, 4 downsample convolutions on "
-                                "their block's input; " + ("skip connections fused into the expand convolutions"
-                                                            if args.residual else "no residual additions"),
-                       "l2": "activations of a step total several GB (> L2)",
-                       "launch": "the stack's calls recorded into one CUDA graph and replayed"},
-            "dense_equiv_tflops": ranks.job_throughput(flops, world, ms_sparse) / 1e12,
-            "x_dense": ms_dense / ms_sparse, "ms_per_step_dense": ms_dense,
-            "images_per_s_dense": ranks.job_throughput(batch, world, ms_dense),
-            "gpu_launches": steps * launches, "clocks": clocks, "dev_status": status}))
-    if world > 1:
-        dist.destroy_process_group()
+    def regions(self, graphs, replays, count, budget_s=20.0):
+        """`count` regions of `replays` replays each (fewer if they would outlast the budget, never
+        fewer than 5); per-replay times in ms."""
+        out = []
+        t0 = time.perf_counter()
+        for i in range(count):
+            out.append(self.region(graphs, replays) / replays)
+            if i >= 4 and time.perf_counter() - t0 > budget_s:
+                break
+        return out
 
 
+def layer_roofline(spec, peaks, sparse=True, real_c_in=None):
+    """(flops, algorithmic bytes, compute roofline ms, memory roofline ms) of one convolution.  The
+    compute peak is 2 x the measured dense bf16 burst for a 2:4 layer (nominal sparse : dense ratio),
+    the measured dense burst for a dense one; the memory peak is the measured HBM copy bandwidth."""
+    flops = spec.dense_equiv_flops
+    bytes_alg = spec.algorithmic_bytes(sparse=sparse)
+    if real_c_in is not None:   # channel-padded input: count the real channels
+        flops = flops * real_c_in // spec.C_in
+        bytes_alg -= 2 * spec.N * spec.H * spec.W * (spec.C_in - real_c_in)
+        bytes_alg -= 2 * spec.C_out * spec.KH * spec.KW * (spec.C_in - real_c_in)
+    peak = (2.0 if sparse else 1.0) * peaks["bf16_tflops"]
+    return flops, bytes_alg, flops / (peak * 1e12) * 1e3, bytes_alg / (peaks["hbm_gbs"] * 1e9) * 1e3
+
+
+# ----------------------------------------------------------------------------- per-layer sweeps (configs 2-4)
+def sweep_measure(cfg, api, synth, torch, tm, dev, peaks, l2_bytes, steps, regions, layer_iters, status,
+                  only_layer=None, want_e2e=False):
+    """One of the per-layer workloads: every layer on its own seeded input (rotating over buffer sets
+    larger than L2), a step = all layers once; the dense counterpart; per-layer device times and
+    rooflines.  Returns a dict; the caller formats it."""
+    layers = timed_layers(cfg)
+    if only_layer is not None:
+        layers = [layers[only_layer]]
+    set_bytes = sum(2 * (s.N * s.H * s.W * s.C_in + s.P * s.C_out) for s in layers)
+    n_sets = max(2, -(-int(1.5 * l2_bytes) // set_bytes) + 1)
+    prep = []
+    t_prep0 = time.perf_counter()
+    gen = torch.Generator(device=dev).manual_seed(synth.SEED_BASE + 31 * cfg)
+    for spec in layers:
+        inp = synth.make_inputs(spec)
+        desc = api.desc_from_spec(spec)
+        w = inp.w.to(dev)
+        bias = inp.bias.to(dev)
+        if spec.mask_source == "gumbel_logits":
+            pat = api.ssconv_select_mask(api.MASK_LOGITS_F32, inp.scores.to(dev), spec.G)
+        else:
+            pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
+        w_comp, meta = api.ssconv_compress(desc, w, pat)
+        xs = [inp.x.to(dev)]
+        for _ in range(1, n_sets):   # further buffer sets only rotate the traffic: drawn on the device
+            xs.append(torch.randn(inp.x.shape, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16))
+        ys = [torch.empty((spec.N, spec.H_out, spec.W_out, spec.C_out), dtype=torch.bfloat16, device=dev)
+              for _ in range(n_sets)]
+        entry = dict(spec=spec, desc=desc, w=w, bias=bias, w_comp=w_comp, meta=meta, xs=xs, ys=ys)
+        if want_e2e:
+            entry["x_host"] = inp.x.pin_memory()
+            entry["y_host"] = torch.empty(ys[0].shape, dtype=torch.bfloat16).pin_memory()
+        prep.append(entry)
+    torch.cuda.synchronize()
+    prep_seconds = time.perf_counter() - t_prep0
+
+    def call(L, r, sparse):
+        if sparse:
+            api.ssconv_forward(L["desc"], L["xs"][r], L["w_comp"], L["meta"], L["bias"], y=L["ys"][r], dev_status=status)
+        else:
+            api.ssconv_forward_dense(L["desc"], L["xs"][r], L["w"], L["bias"], y=L["ys"][r], dev_status=status)
+
+    def step(r, sparse=True):
+        for L in prep:
+            call(L, r, sparse)
+
+    launches_per_step = 0
+    for i in range(3):   # eager warm-up (also performs every one-time host set-up before any capture)
+        c0 = api.ssconv_launch_count()
+        step(i % n_sets, True)
+        launches_per_step = api.ssconv_launch_count() - c0
+        step(i % n_sets, False)
+    torch.cuda.synchronize()
+    g_sparse = [tm.capture(lambda r=r: step(r, True)) for r in range(n_sets)]
+    g_dense = [tm.capture(lambda r=r: step(r, False)) for r in range(n_sets)]
+    tm.region(g_sparse, 2 * n_sets)
+    ms_sparse = tm.regions(g_sparse, steps, regions, budget_s=8.0)
+    tm.region(g_dense, 2 * n_sets)
+    ms_dense = tm.regions(g_dense, steps, max(5, regions // 3), budget_s=4.0)
+    del g_sparse, g_dense
+
+    per_layer, sum_t, sum_roof, sum_t_dense = [], 0.0, 0.0, 0.0
+    for L in prep:
+        spec = L["spec"]
+        res = {}
+        for sparse in (True, False):
+            g = tm.capture(lambda L=L, sparse=sparse: [call(L, i % n_sets, sparse) for i in range(layer_iters)])
+            tm.region(g, 1)
+            res[sparse] = min(tm.region(g, 2) / 2 for _ in range(3)) / layer_iters
+            del g
+        flops, bytes_alg, t_c, t_m = layer_roofline(spec, peaks, sparse=True)
+        roof = max(t_c, t_m)
+        sum_t += res[True]
+        sum_t_dense += res[False]
+        sum_roof += roof
+        per_layer.append({"layer": spec.name, "us_sparse": round(res[True] * 1e3, 2), "us_dense": round(res[False] * 1e3, 2),
+                          "tflops": round(flops / res[True] / 1e9, 1), "gbs": round(bytes_alg / res[True] / 1e6, 1),
+                          "bound": "tensor" if t_c >= t_m else "hbm", "us_roofline": round(roof * 1e3, 2),
+                          "roofline_frac": round(roof / res[True], 4), "x_dense": round(res[False] / res[True], 3),
+                          "plan": api.ssconv_plan(L["desc"], True)})
+    total_flops = sum(s.dense_equiv_flops for s in layers)
+    out = dict(layers=layers, prep=prep, n_sets=n_sets, set_bytes=set_bytes, prep_seconds=prep_seconds,
+               launches_per_step=launches_per_step, ms_sparse=ms_sparse, ms_dense=ms_dense, per_layer=per_layer,
+               sum_kernel_ms=sum_t, sum_kernel_ms_dense=sum_t_dense, sum_roof_ms=sum_roof, total_flops=total_flops,
+               bytes_alg=sum(s.algorithmic_bytes(sparse=True) for s in layers))
+    return out
+
+
+def sweep_summary(cfg, m, world, ranks):
+    """The short form of a sweep for the headline line."""
+    ms = statistics.median(m["ms_sparse"])
+    return {"workload": WORKLOADS[cfg], "layers": len(m["layers"]), "ms_per_step": round(ms, 5),
+            "tflops": round(ranks.job_throughput(m["total_flops"], world, ms) / 1e12, 1),
+            "x_dense": round(statistics.median(m["ms_dense"]) / ms, 3),
+            "roofline_frac": round(m["sum_roof_ms"] / m["sum_kernel_ms"], 4),
+            "min_layer_x_dense": min(r["x_dense"] for r in m["per_layer"]),
+            "per_layer": [{k: r[k] for k in ("layer", "us_sparse", "roofline_frac", "x_dense", "bound")}
+                          for r in m["per_layer"]]}
+
+
+# ----------------------------------------------------------------------------- mask-learning step
 def train_arm(args):
     """One mask-learning step per layer of the chosen layer set (Sec. 3.1): soft mask -> dense forward
     with the effective weights -> weight gradient -> gradient of the choice weights -> AdamW on them,
@@ -443,40 +564,261 @@ def train_arm(args):
         dist.destroy_process_group()
 
 
-# ----------------------------------------------------------------------------- GPU arm
-def main():
-    global CONFIG_ID, WORKLOAD
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=4000)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--layer-iters", type=int, default=200)
-    ap.add_argument("--only-layer", type=int, default=None,
-                    help="profiling aid: launch just this layer of the sweep --layer-iters times and exit")
-    ap.add_argument("--dense", action="store_true", help="with --only-layer: use the dense kernel")
-    ap.add_argument("--residual", action="store_true",
-                    help="with --workload-config 5: fuse the network's skip connections into the expand convolutions")
-    ap.add_argument("--train", action="store_true",
-                    help="time one mask-learning step per layer (soft mask, dense forward, weight gradient, "
-                         "choice-weight gradient) instead of the inference sweep")
-    ap.add_argument("--batch", type=int, default=None, help="with --workload-config 5: images per GPU (default 256)")
-    ap.add_argument("--workload-config", type=int, default=CONFIG_ID, choices=sorted(WORKLOADS),
-                    help="layer set to run (default: the benchmarked ResNet-18 sweep)")
-    args = ap.parse_args()
-    CONFIG_ID = args.workload_config
-    WORKLOAD = WORKLOADS[CONFIG_ID]
-    if args.impl == "reference":
-        reference_arm(args)
-        return
-    if CONFIG_ID == 5:
-        stack_arm(args)
-        return
-    if args.train:
-        train_arm(args)
-        return
+# ----------------------------------------------------------------------------- conv stack (the headline)
+def stack_arm(args):
+    """ResNet-50-shaped convolution stack at batch 256 per GPU, recorded into one CUDA graph and replayed."""
+    import torch
+    import torch.distributed as dist
+    from paper_2411_00288_b200 import api, synth, stack, ranks, build as libbuild
 
+    rank, local_rank, world = ranks.env_ranks()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    distributed = world > 1
+    if distributed:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        libbuild.build()
+    if distributed:
+        dist.barrier()
+    api.lib()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()          # before any warm-up: it runs through every leg below
+    peaks = load_peaks()
+    l2_bytes = int(torch.cuda.get_device_properties(dev).L2_cache_size)
+    tm = Timer(torch, dist, ranks, dev, distributed)
+    batch = args.batch or 256
+    warmup, steps = max(3, args.warmup), max(1, min(args.steps, 200))
+
+    t_prep0 = time.perf_counter()
+    steps_def = synth.resnet50_stack(batch, residual=args.residual)
+    net = stack.ConvStack(steps_def, dev, with_dense=True)
+    g = torch.Generator().manual_seed(synth.SEED_BASE + 577 + rank)
+    x3_host = torch.randn((batch, 224, 224, 3), generator=g, dtype=torch.float32).to(torch.bfloat16).pin_memory()
+    x_dev = x3_host.to(dev)   # (the stack takes the 3-channel images as they are: its stem starts with a space-to-depth)
+    torch.cuda.synchronize()
+    prep_seconds = time.perf_counter() - t_prep0
+    act_bytes = sum(o.numel() * 2 for o in net.outputs) + x_dev.numel() * 2
+
+    # ---- the step: whole stack, sparse; then the dense counterpart on the same buffers
+    sampler.mark("step")
+    for _ in range(2):
+        net.forward(x_dev, sparse=True)
+        net.forward(x_dev, sparse=False)
+    torch.cuda.synchronize()
+    c0 = api.ssconv_launch_count()
+    net.forward(x_dev, sparse=True)
+    launches = api.ssconv_launch_count() - c0
+    torch.cuda.synchronize()
+    g_sparse = tm.capture(lambda: net.forward(x_dev, sparse=True))
+    g_dense = tm.capture(lambda: net.forward(x_dev, sparse=False))
+    tm.region(g_sparse, warmup)
+    ms_regions = tm.regions(g_sparse, steps, max(MIN_REGIONS, args.regions), budget_s=25.0)
+    ms_step = statistics.median(ms_regions)
+    tm.region(g_dense, warmup)
+    ms_dense = statistics.median(tm.regions(g_dense, steps, 7, budget_s=8.0))
+    flops = stack_flops(batch)
+    value = ranks.job_throughput(flops, world, ms_step) / 1e12
+
+    # ---- per-layer device times: a graph of back-to-back launches of one step of the stack on the
+    # stack's own buffers (a layer whose tensors fit in L2 runs L2-warm here, as its input does inside
+    # the stack, where the layer before has just written it)
+    sampler.mark("per_layer")
+    iters = args.layer_iters
+    per_layer, sums = [], dict(t=0.0, roof=0.0, t_masked=0.0, roof_masked=0.0, flops_masked=0, bytes=0,
+                               t_dense_masked=0.0, t_tensor=0.0, roof_tensor=0.0, flops_tensor=0)
+    for i, st in enumerate(steps_def):
+        res = {}
+        for sparse in ((True, False) if st.kind == "conv" else (True,)):
+            gr = tm.capture(lambda i=i, sparse=sparse: [net.run_step(i, x_dev, sparse) for _ in range(iters)])
+            tm.region(gr, 1)
+            res[sparse] = min(tm.region(gr, 2) / 2 for _ in range(3)) / iters
+            del gr
+        t = res[True]
+        if st.kind == "maxpool":
+            n, h, w, c = net.outputs[st.src].shape
+            bytes_alg = 2 * (net.outputs[st.src].numel() + net.outputs[i].numel())
+            f, t_c, t_m, name, bound = 0, 0.0, bytes_alg / (peaks["hbm_gbs"] * 1e9) * 1e3, "maxpool_3x3s2", "hbm"
+            row = {"layer": name, "us": round(t * 1e3, 2)}
+        else:
+            spec = st.spec
+            masked = st.kind == "conv"
+            f, bytes_alg, t_c, t_m = layer_roofline(spec, peaks, sparse=masked, real_c_in=None if masked else 3)
+            if st.res >= 0:
+                bytes_alg += 2 * spec.P * spec.C_out
+                t_m = bytes_alg / (peaks["hbm_gbs"] * 1e9) * 1e3
+            bound = "tensor" if t_c >= t_m else "hbm"
+            row = {"layer": spec.name, "us": round(t * 1e3, 2), "tflops": round(f / t / 1e9, 1)}
+            if masked:
+                row["us_dense"] = round(res[False] * 1e3, 2)
+                row["x_dense"] = round(res[False] / t, 3)
+                row["plan"] = api.ssconv_plan(net.layers[i]["desc"], True)
+                sums["t_masked"] += t
+                sums["t_dense_masked"] += res[False]
+                sums["roof_masked"] += max(t_c, t_m)
+                sums["flops_masked"] += f
+                if bound == "tensor":
+                    sums["t_tensor"] += t
+                    sums["roof_tensor"] += max(t_c, t_m)
+                    sums["flops_tensor"] += f
+        roof = max(t_c, t_m)
+        row.update({"gbs": round(bytes_alg / t / 1e6, 1), "bound": bound, "us_roofline": round(roof * 1e3, 2),
+                    "roofline_frac": round(roof / t, 4)})
+        per_layer.append(row)
+        sums["t"] += t
+        sums["roof"] += roof
+        sums["bytes"] += bytes_alg
+
+    # ---- end to end with host buffers: every step copies the batch of 3-channel images from pinned
+    # host memory, pads them on the device, runs the stack and copies the last activation back.  Copy-in,
+    # compute and copy-out run on three streams chained by events, double-buffered on both ends, as a
+    # serving loop would do it.
+    sampler.mark("e2e")
+    s_in, s_run, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    x3_bufs = [torch.empty_like(x_dev) for _ in range(2)]
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s_run):
+        last = net.forward(x_dev, sparse=True)
+    torch.cuda.synchronize()
+    y_stage = [torch.empty_like(last) for _ in range(2)]
+    y_host = [torch.empty(last.shape, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_run = [torch.cuda.Event() for _ in range(2)]
+    ev_out = [torch.cuda.Event() for _ in range(2)]
+
+    def e2e_step(k):
+        b = k & 1
+        with torch.cuda.stream(s_in):
+            if k >= 2:
+                s_in.wait_event(ev_run[b])       # step k-2 has read this buffer
+            x3_bufs[b].copy_(x3_host, non_blocking=True)
+            ev_in[b].record(s_in)
+        with torch.cuda.stream(s_run):
+            s_run.wait_event(ev_in[b])
+            x_dev.copy_(x3_bufs[b], non_blocking=True)   # into the buffer the recorded graph reads (device to device)
+            g_sparse.replay()
+            if k >= 2:
+                s_run.wait_event(ev_out[b])      # the copy-out of step k-2 has read this staging buffer
+            y_stage[b].copy_(last, non_blocking=True)
+            ev_run[b].record(s_run)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_run[b])
+            y_host[b].copy_(y_stage[b], non_blocking=True)
+            ev_out[b].record(s_out)
+
+    for k in range(4):
+        e2e_step(k)
+    torch.cuda.synchronize()
+    k_e2e = max(6, min(20, steps))
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    tm.barrier()
+    t0.record(s_in)
+    for k in range(4, 4 + k_e2e):
+        e2e_step(k)
+    s_out.wait_stream(s_run)
+    s_out.wait_stream(s_in)
+    t1.record(s_out)
+    torch.cuda.synchronize()
+    e2e_ms = ranks.max_over_ranks(t0.elapsed_time(t1) / k_e2e, dev)
+    h2d, d2h = x3_host.numel() * 2, last.numel() * 2
+    e2e_launches = launches
+    dev_status = int(net.status.item())
+    del net, g_sparse, g_dense, x3_bufs, y_stage
+    torch.cuda.empty_cache()
+
+    # ---- the three per-layer sweeps, in short (one GPU only: they are parity-test workloads, reported as context)
+    summaries = {}
+    if world == 1 and not args.no_summaries:
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        for cfg in (2, 3, 4):
+            sampler.mark(f"summary_cfg{cfg}")
+            m = sweep_measure(cfg, api, synth, torch, tm, dev, peaks, l2_bytes, steps=50, regions=10, layer_iters=50,
+                              status=status)
+            summaries[f"summary_cfg{cfg}"] = sweep_summary(cfg, m, world, ranks)
+            del m
+            torch.cuda.empty_cache()
+        dev_status |= int(status.item())
+    clocks = sampler.stop() if rank == 0 else None
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import build as oracle_build
+        oracle_build.build()
+        leg = oracle_leg(15.0)
+        cpu = {k: leg[k] for k in ("value", "unit", "cores", "kind", "sample", "images_per_s")}
+
+    if rank == 0:
+        sp = spread(ms_regions)
+        n_hbm = sum(1 for r in per_layer if r["bound"] == "hbm")
+        achieved = flops / (sums["t"] * 1e-3) / 1e12
+        ceiling = flops / (sums["roof"] * 1e-3) / 1e12
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD + ("_with_skip_connections" if args.residual else ""),
+                       "batch_per_gpu": batch,
+                       "stack": "stem 7x7 s2 (dense, on the 3-channel images: space-to-depth + a 4x1 convolution over a "
+                                "sliding-window view), 3x3 s2 max-pool, 16 bottlenecks as reduce -> 3x3 -> expand with bias "
+                                "+ ReLU, 4 downsample convolutions on their block's input; "
+                                + ("skip connections fused into the expand convolutions" if args.residual
+                                   else "no residual additions"),
+                       "flops": "2*P*C_out*K per convolution (53 of them; the stem with its 3 real channels)",
+                       "l2": f"the activations of one step total {act_bytes / 2**30:.1f} GiB (> the {l2_bytes / 2**20:.0f} MiB "
+                             f"L2 read from the device): inputs larger than L2",
+                       "masks": "magnitude top-2 of 4, selected and compressed once before timing",
+                       "launch": "the stack's C-ABI calls recorded into one CUDA graph and replayed",
+                       "timing": f"{sp['regions']} regions of {steps} steps, CUDA events on the launching stream, barrier + "
+                                 f"synchronize on both sides of each region, max over ranks; ms_per_step is the median",
+                       "one_off_prepare_s": round(prep_seconds, 2)},
+            "ms_per_step_spread": {k: round(v, 5) if isinstance(v, float) else v for k, v in sp.items()},
+            "images_per_s": ranks.job_throughput(batch, world, ms_step),
+            "x_dense": ms_dense / ms_step, "ms_per_step_dense": ms_dense,
+            "images_per_s_dense": ranks.job_throughput(batch, world, ms_dense),
+            "roofline": {
+                "bound": "hbm", "kernel": "ssconv_fwd_kernel<sparse> / ssconv_fwd_pair_kernel<sparse> (52 of the 55 steps)",
+                "achieved": achieved, "peak": ceiling, "unit": "TFLOP/s", "frac": sums["roof"] / sums["t"],
+                "how": "per layer the roofline time is the slower of FLOPs / tensor peak and algorithmic bytes / HBM "
+                       "bandwidth; peak = the stack's FLOPs / the sum of those times, achieved = the stack's FLOPs / "
+                       "the sum of the measured per-layer CUDA-event times",
+                "peak_source": f"{peaks['source']} peaks: HBM {peaks['hbm_gbs']} GB/s; tensor 2 x the dense bf16 burst "
+                               f"({peaks['bf16_tflops']} TFLOP/s) for 2:4 layers, 1 x for the dense stem",
+                "layers_bound_by": {"hbm": n_hbm, "tensor": len(per_layer) - n_hbm},
+                "sum_layer_ms": sums["t"], "sum_roofline_ms": sums["roof"],
+                "algorithmic_bytes_per_step": sums["bytes"],
+                "achieved_gbs": sums["bytes"] / (sums["t"] * 1e-3) / 1e9, "hbm_peak_gbs": peaks["hbm_gbs"],
+                "masked_convolutions": {
+                    "sum_layer_ms": sums["t_masked"], "frac": sums["roof_masked"] / sums["t_masked"],
+                    "tflops": sums["flops_masked"] / (sums["t_masked"] * 1e-3) / 1e12,
+                    "x_dense": sums["t_dense_masked"] / sums["t_masked"]},
+                "tensor_bound_layers": {
+                    "sum_layer_ms": sums["t_tensor"], "tflops": sums["flops_tensor"] / max(sums["t_tensor"], 1e-9) / 1e9,
+                    "peak_tflops": 2.0 * peaks["bf16_tflops"],
+                    "frac": sums["roof_tensor"] / max(sums["t_tensor"], 1e-9)},
+                "traffic": None,
+                "traffic_note": "no ncu DRAM counters are committed for the current kernels at this batch"},
+            "per_layer": per_layer,
+            "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
+                    "images_per_s": ranks.job_throughput(batch, world, e2e_ms),
+                    "path": "pinned host images [N,224,224,3] bf16 -> device -> the stack -> last activation "
+                            "[N,7,7,2048] -> pinned host; three streams, double-buffered"},
+            "gpu_launches": len(ms_regions) * steps * launches, "gpu_launches_per_step": launches,
+            "gpu_launches_per_e2e_step": e2e_launches,
+            "clocks": clocks, "dev_status": dev_status,
+        }
+        line.update(summaries)
+        if cpu is not None:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line))
+    if distributed:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- per-layer sweep as its own line
+def sweep_arm(args):
+    """--workload-config 2|3|4: the full line for one of the per-layer sweeps."""
     import torch
     import torch.distributed as dist
     from paper_2411_00288_b200 import api, synth, ranks, build as libbuild
@@ -492,155 +834,48 @@ def main():
     if distributed:
         dist.barrier()
     api.lib()
-    peaks = load_peaks()
-    warmup = max(3, args.warmup)
-
-    layers = timed_layers()
-    if args.only_layer is not None:
-        layers = [layers[args.only_layer]]
-    # ---- one-off preparation with the library's own kernels: select -> compress (S1, S2)
-    prep = []
-    set_bytes = sum(2 * (s.N * s.H * s.W * s.C_in + s.P * s.C_out) for s in layers)
-    n_sets = max(2, -(-int(1.5 * L2_BYTES) // set_bytes) + 1)
-    t_prep0 = time.perf_counter()
-    for spec in layers:
-        inp = synth.make_inputs(spec)
-        desc = api.desc_from_spec(spec)
-        w = inp.w.to(dev)
-        bias = inp.bias.to(dev)
-        pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
-        w_comp, meta = api.ssconv_compress(desc, w, pat)
-        xs = [inp.x.to(dev)]
-        for r in range(1, n_sets):
-            xs.append(synth.make_inputs(spec, seed=spec.seed + 7919 * r, x_only=True).x.to(dev))
-        ys = [torch.empty((spec.N, spec.H_out, spec.W_out, spec.C_out), dtype=torch.bfloat16, device=dev)
-              for _ in range(n_sets)]
-        prep.append(dict(spec=spec, desc=desc, w=w, bias=bias, w_comp=w_comp, meta=meta, xs=xs, ys=ys,
-                         x_host=inp.x.pin_memory(),
-                         y_host=torch.empty(ys[0].shape, dtype=torch.bfloat16).pin_memory()))
-    status = torch.zeros(1, dtype=torch.int32, device=dev)
-    torch.cuda.synchronize()
-    prep_seconds = time.perf_counter() - t_prep0
-
-    if args.only_layer is not None:
-        L = prep[0]
-        for i in range(args.layer_iters):
-            r = i % n_sets
-            if args.dense:
-                api.ssconv_forward_dense(L["desc"], L["xs"][r], L["w"], L["bias"], y=L["ys"][r], dev_status=status)
-            else:
-                api.ssconv_forward(L["desc"], L["xs"][r], L["w_comp"], L["meta"], L["bias"], y=L["ys"][r],
-                                   dev_status=status)
-        torch.cuda.synchronize()
-        print(json.dumps({"only_layer": L["spec"].name, "launches": args.layer_iters, "dense": args.dense,
-                          "dev_status": int(status.item())}))
-        return
-
-    def step(r, sparse=True):
-        for L in prep:
-            if sparse:
-                api.ssconv_forward(L["desc"], L["xs"][r], L["w_comp"], L["meta"], L["bias"], y=L["ys"][r],
-                                   dev_status=status)
-            else:
-                api.ssconv_forward_dense(L["desc"], L["xs"][r], L["w"], L["bias"], y=L["ys"][r], dev_status=status)
-
-    def barrier():
-        if distributed:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(ms):
-        return ranks.max_over_ranks(ms, dev)
-
-    def capture(fn):
-        """Record fn()'s launches into a CUDA graph (the launches are the same C-ABI calls; the
-        graph only removes the host-side launch cost from the timed region)."""
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            fn()
-        return g
-
-    def time_replays(graphs, replays):
-        """Replay graphs[i % len] for i < replays between two events; max over ranks, in ms."""
-        if not isinstance(graphs, (list, tuple)):
-            graphs = [graphs]
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        e0.record()
-        for i in range(replays):
-            graphs[i % len(graphs)].replay()
-        e1.record()
-        barrier()
-        return max_over_ranks(e0.elapsed_time(e1))
-
-    # eager warm-up (also performs every one-time host set-up before any capture)
-    launches_per_step = 0
-    for i in range(warmup):
-        c0 = api.ssconv_launch_count()
-        step(i % n_sets, True)
-        launches_per_step = api.ssconv_launch_count() - c0
-        step(i % n_sets, False)
-    torch.cuda.synchronize()
-
-    # one graph per buffer set = one step; step i replays graph i % n_sets
-    g_sparse = [capture(lambda r=r: step(r, True)) for r in range(n_sets)]
-    g_dense = [capture(lambda r=r: step(r, False)) for r in range(n_sets)]
-    total_flops = sum(s.dense_equiv_flops for s in layers)
-    steps = args.steps
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    time_replays(g_sparse, warmup)
-    ms_total = time_replays(g_sparse, steps)
-    ms_per_step = ms_total / steps
-    value = ranks.job_throughput(total_flops, world, ms_per_step) / 1e12
+    peaks = load_peaks()
+    l2_bytes = int(torch.cuda.get_device_properties(dev).L2_cache_size)
+    tm = Timer(torch, dist, ranks, dev, distributed)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    steps = max(1, min(args.steps, 2000))
 
-    # ---- dense counterpart (S4) on the same buffers, same rotation
-    time_replays(g_dense, warmup)
-    ms_dense = time_replays(g_dense, steps) / steps
-    clocks = sampler.stop() if rank == 0 else None
+    if args.only_layer is not None:   # profiling aid: one layer, launched repeatedly, nothing timed
+        spec = timed_layers()[args.only_layer]
+        inp = synth.make_inputs(spec)
+        desc = api.desc_from_spec(spec)
+        w, bias = inp.w.to(dev), inp.bias.to(dev)
+        pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
+        w_comp, meta = api.ssconv_compress(desc, w, pat)
+        n_sets = max(2, -(-int(1.5 * l2_bytes) // (2 * (spec.N * spec.H * spec.W * spec.C_in + spec.P * spec.C_out))) + 1)
+        xs = [inp.x.to(dev)] + [torch.randn(inp.x.shape, device=dev).to(torch.bfloat16) for _ in range(n_sets - 1)]
+        ys = [torch.empty((spec.N, spec.H_out, spec.W_out, spec.C_out), dtype=torch.bfloat16, device=dev)
+              for _ in range(n_sets)]
+        for i in range(args.layer_iters):
+            r = i % n_sets
+            if args.dense:
+                api.ssconv_forward_dense(desc, xs[r], w, bias, y=ys[r], dev_status=status)
+            else:
+                api.ssconv_forward(desc, xs[r], w_comp, meta, bias, y=ys[r], dev_status=status)
+        torch.cuda.synchronize()
+        if rank == 0:
+            sampler.stop()
+        print(json.dumps({"only_layer": spec.name, "launches": args.layer_iters, "dense": args.dense,
+                          "plan": api.ssconv_plan(desc, not args.dense), "dev_status": int(status.item())}))
+        return
 
-    # ---- per-layer device times: a graph of `layer_iters` back-to-back launches of one layer,
-    # rotating buffer sets, timed with events on the launching stream
-    per_layer = []
-    sum_kernel_ms = 0.0
-    sum_roof_ms = 0.0
-    sparse_peak = 2.0 * peaks["bf16_tflops"]
-    for L in prep:
-        spec = L["spec"]
-        res = {}
-        for sparse in (True, False):
-            def many(L=L, sparse=sparse):
-                for i in range(args.layer_iters):
-                    r = i % n_sets
-                    if sparse:
-                        api.ssconv_forward(L["desc"], L["xs"][r], L["w_comp"], L["meta"], L["bias"], y=L["ys"][r],
-                                           dev_status=status)
-                    else:
-                        api.ssconv_forward_dense(L["desc"], L["xs"][r], L["w"], L["bias"], y=L["ys"][r],
-                                                 dev_status=status)
-            g = capture(many)
-            time_replays(g, 1)
-            res[sparse] = time_replays(g, 5) / (5 * args.layer_iters)
-            del g
-        t_s, t_d = res[True], res[False]
-        flops = spec.dense_equiv_flops
-        bytes_alg = spec.algorithmic_bytes(sparse=True)
-        t_c = flops / (sparse_peak * 1e12) * 1e3
-        t_m = bytes_alg / (peaks["hbm_gbs"] * 1e9) * 1e3
-        roof = max(t_c, t_m)
-        sum_kernel_ms += t_s
-        sum_roof_ms += roof
-        per_layer.append({"layer": spec.name, "us_sparse": round(t_s * 1e3, 2), "us_dense": round(t_d * 1e3, 2),
-                          "tflops": round(flops / t_s / 1e9, 1), "gbs": round(bytes_alg / t_s / 1e6, 1),
-                          "bound": "tensor" if t_c >= t_m else "hbm", "us_roofline": round(roof * 1e3, 2),
-                          "roofline_frac": round(roof / t_s, 4), "x_dense": round(t_d / t_s, 3),
-                          "plan": api.ssconv_plan(L["desc"], True)})
+    m = sweep_measure(CONFIG_ID, api, synth, torch, tm, dev, peaks, l2_bytes, steps=steps,
+                      regions=max(MIN_REGIONS, args.regions), layer_iters=args.layer_iters, status=status, want_e2e=True)
+    prep, layers = m["prep"], m["layers"]
+    ms_per_step = statistics.median(m["ms_sparse"])
+    ms_dense = statistics.median(m["ms_dense"])
+    total_flops = m["total_flops"]
 
     # ---- end to end through the public API with host buffers: every step copies each layer's input
-    # from pinned host memory, runs the layer, and copies its output back.  Three streams (copy in,
-    # compute, copy out) chained by events, so that the copies of one layer overlap the kernels
-    # and the opposite-direction copies of its neighbours, as a serving loop would do it.
+    # from pinned host memory, runs the layer, and copies its output back; three streams chained by events
     s_in, s_run, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
     ev_in = [torch.cuda.Event() for _ in prep]
     ev_run = [torch.cuda.Event() for _ in prep]
@@ -671,7 +906,7 @@ def main():
     torch.cuda.synchronize()
     k_e2e = 20
     e2e_t0, e2e_t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
+    tm.barrier()
     e2e_t0.record(s_in)
     for _ in range(k_e2e):
         e2e_step(False)
@@ -679,10 +914,11 @@ def main():
     s_out.wait_stream(s_in)
     e2e_t1.record(s_out)
     torch.cuda.synchronize()
-    e2e_ms = max_over_ranks(e2e_t0.elapsed_time(e2e_t1) / k_e2e)
+    e2e_ms = ranks.max_over_ranks(e2e_t0.elapsed_time(e2e_t1) / k_e2e, dev)
     h2d = sum(L["x_host"].numel() * 2 for L in prep)
     d2h = sum(L["y_host"].numel() * 2 for L in prep)
     dev_status = int(status.item())
+    clocks = sampler.stop() if rank == 0 else None
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -692,31 +928,33 @@ def main():
         cpu = {k: leg[k] for k in ("value", "unit", "cores", "kind", "sample")}
 
     if rank == 0:
-        achieved = total_flops / (sum_kernel_ms * 1e-3) / 1e12
+        sparse_peak = 2.0 * peaks["bf16_tflops"]
+        achieved = total_flops / (m["sum_kernel_ms"] * 1e-3) / 1e12
+        sp = spread(m["ms_sparse"])
         line = {
-            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps,
-            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "metric": METRIC, "value": ranks.job_throughput(total_flops, world, ms_per_step) / 1e12, "unit": "TFLOP/s",
+            "n_gpus": world, "steps": steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "layers": len(layers), "batch_per_gpu": layers[0].N,
-                       "l2": f"rotating {n_sets} buffer sets of {set_bytes / 2**20:.0f} MiB (> L2) per rank",
-                       "masks": "magnitude top-2 of 4, selected and compressed once before timing",
+                       "l2": f"rotating {m['n_sets']} buffer sets of {m['set_bytes'] / 2**20:.0f} MiB (> the "
+                             f"{l2_bytes / 2**20:.0f} MiB L2 read from the device) per rank",
+                       "masks": "selected and compressed once before timing",
                        "launch": "the C-ABI calls of one step recorded into a CUDA graph per buffer set and replayed",
-                       "one_off_prepare_s": round(prep_seconds, 3)},
+                       "timing": f"{sp['regions']} regions of {steps} steps; ms_per_step is the median",
+                       "one_off_prepare_s": round(m["prep_seconds"], 3)},
+            "ms_per_step_spread": {k: round(v, 6) if isinstance(v, float) else v for k, v in sp.items()},
             "x_dense": ms_dense / ms_per_step, "ms_per_step_dense": ms_dense,
             "roofline": {"bound": "tensor", "kernel": "ssconv_fwd_kernel<sparse>", "achieved": achieved,
                          "peak": sparse_peak, "unit": "TFLOP/s", "frac": achieved / sparse_peak,
                          "peak_source": f"2 x dense bf16 burst of {peaks['source']} peaks (nominal sparse:dense ratio)",
-                         "layer_mix_ceiling": total_flops / (sum_roof_ms * 1e-3) / 1e12,
-                         "frac_of_layer_mix_ceiling": sum_roof_ms / sum_kernel_ms,
-                         "hbm_peak_gbs": peaks["hbm_gbs"],
-                         "traffic": measured_traffic() if CONFIG_ID == 2 else None,
-                         "traffic_unit": "bytes per step (DRAM read + write of the sparse forward and finishing "
-                                         "kernels, ncu)",
-                         "algorithmic_bytes_per_step": sum(L["spec"].algorithmic_bytes(sparse=True) for L in prep)},
-            "per_layer": per_layer,
+                         "layer_mix_ceiling": total_flops / (m["sum_roof_ms"] * 1e-3) / 1e12,
+                         "frac_of_layer_mix_ceiling": m["sum_roof_ms"] / m["sum_kernel_ms"],
+                         "hbm_peak_gbs": peaks["hbm_gbs"], "traffic": None,
+                         "algorithmic_bytes_per_step": m["bytes_alg"]},
+            "per_layer": m["per_layer"],
             "e2e": {"value": world * total_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-            "gpu_launches": steps * launches_per_step,
+            "gpu_launches": len(m["ms_sparse"]) * steps * m["launches_per_step"],
             "clocks": clocks, "dev_status": dev_status,
         }
         if cpu is not None:
@@ -724,6 +962,60 @@ def main():
         print(json.dumps(line))
     if distributed:
         dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- entry
+def launch_ranks(args, argv):
+    """--gpus N > 1 without a torchrun environment: start N ranks of this script, one per GPU."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + argv
+    return subprocess.call(cmd)
+
+
+def main():
+    global CONFIG_ID, WORKLOAD
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20, help="steps per timed region")
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--regions", type=int, default=MIN_REGIONS, help="timed regions (at least 30)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-summaries", action="store_true", help="skip the short runs of the three per-layer sweeps")
+    ap.add_argument("--layer-iters", type=int, default=None,
+                    help="back-to-back launches per layer timing (default 10 for the stack, 100 for the sweeps)")
+    ap.add_argument("--only-layer", type=int, default=None,
+                    help="with --workload-config 2|3|4, a profiling aid: launch just this layer --layer-iters times and exit")
+    ap.add_argument("--dense", action="store_true", help="with --only-layer: use the dense kernel")
+    ap.add_argument("--residual", action="store_true",
+                    help="fuse the network's skip connections into the expand convolutions of the stack")
+    ap.add_argument("--train", action="store_true",
+                    help="time one mask-learning step per layer (soft mask, dense forward, weight gradient, "
+                         "choice-weight gradient) on one of the per-layer sweeps (default: the ResNet-18 sweep)")
+    ap.add_argument("--batch", type=int, default=None, help="images per GPU of the stack (default 256)")
+    ap.add_argument("--workload-config", type=int, default=None, choices=sorted(WORKLOADS),
+                    help="5 (default): the ResNet-50 stack; 2, 3, 4: one of the per-layer sweeps")
+    args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        sys.exit(launch_ranks(args, sys.argv[1:]))
+    CONFIG_ID = args.workload_config if args.workload_config is not None else (2 if args.train else 5)
+    WORKLOAD = WORKLOADS[CONFIG_ID]
+    if args.layer_iters is None:
+        args.layer_iters = 10 if CONFIG_ID == 5 else 100
+    if args.impl == "reference":
+        reference_arm(args)
+    elif args.train:
+        if CONFIG_ID == 5:
+            CONFIG_ID, WORKLOAD = 2, WORKLOADS[2]
+        train_arm(args)
+    elif CONFIG_ID == 5:
+        stack_arm(args)
+    else:
+        sweep_arm(args)
 
 
 if __name__ == "__main__":

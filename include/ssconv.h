@@ -144,6 +144,28 @@ int32_t ssconv_decompress(const ssconv_desc_t* desc, const void* w_comp, const v
 int32_t ssconv_maxpool(const void* x, void* y, int32_t N, int32_t H, int32_t W, int32_t C, int32_t k,
                        int32_t stride, int32_t pad, void* stream);
 
+/* Channel padding of NHWC bf16 activations: y[p, c] = x[p, c] for c < C and 0 for C <= c < C_pad,
+ * for `pixels` pixels.  Not part of the paper's method: the forward entry points want C_in % 8 == 0,
+ * and the networks of Sec. 4 start from 3-channel images; the zero channels meet zero-extended
+ * weights, so the convolution (Eq. 4) is unchanged.  x: device, 2-byte aligned; y: device, 16-byte
+ * aligned; C_pad % 8 == 0, C_pad >= C. */
+int32_t ssconv_pad_channels(const void* x, void* y, int64_t pixels, int32_t C, int32_t C_pad, void* stream);
+
+/* Space to depth of NHWC bf16 images: blocks of `block` x `block` pixels of the zero-padded image
+ * become the channels of one pixel,
+ *   y[n, r, q, (bh*block + bw)*C + c] = x[n, block*r - pad + bh, block*q - pad + bw, c],
+ * zero outside the image and in the channels [block*block*C, C_pad); y: bf16 [N, Hb, Wb, C_pad].
+ * Not part of the paper's method; it is how a strided convolution over very few channels (the
+ * 7x7 stride-2 stem of the ResNets of Sec. 4 on RGB images) reaches the tensor-core path: with
+ * T = ceil(K/block), Hb = H_out + T - 1 and Wb = W_out + T - 1, the K x K convolution of stride
+ * `block` and padding `pad` over x (Eq. 4) equals a T x T convolution of unit stride and no padding
+ * over y, and, reading T neighbouring pixels of y as one pixel of T*C_pad channels through
+ * ssconv_forward_dense_strided, a T x 1 convolution.  The weights are rearranged by the same call:
+ * [C_out, K, K, C] as C_out "images" with pad 0 and Hb = Wb = T gives [C_out, T, T, C_pad].
+ * x: device, 2-byte aligned; y: device, 16-byte aligned; C_pad % 8 == 0, C_pad >= block*block*C. */
+int32_t ssconv_space_to_depth(const void* x, void* y, int32_t N, int32_t H, int32_t W, int32_t C, int32_t block,
+                              int32_t pad, int32_t Hb, int32_t Wb, int32_t C_pad, void* stream);
+
 /* Partial unfold along the width: the unfold U(X) of Eq. 5 restricted to one filter row.  For every
  * row of pixels (rows = N*H of them, each W pixels of C channels, bf16) and every horizontal filter
  * placement wo:
@@ -306,6 +328,16 @@ int32_t ssconv_absmax(const void* x_bf16, int64_t n, float* out, void* stream);
 enum { SSCONV_LEMMA_PERTURBATION = 34, SSCONV_LEMMA_ANY_MASK = 35, SSCONV_LEMMA_MASKED_UPDATE = 36 };
 double ssconv_stability_threshold(int32_t lemma, double L, const double* layer_norms, int32_t depth,
                                   int32_t j, double extra_norm, double x_norm);
+
+/* ssconv_forward_dense on a strided view of the input: pixel (n, h, w) of the H x W x C_in input the
+ * descriptor names starts stride_n*n + stride_h*h + stride_w*w elements into x.  The strides are
+ * multiples of 8 elements and need not exceed C_in: with stride_w < C_in neighbouring pixels
+ * overlap, i.e. the input is a sliding window of C_in channels over a narrower tensor (the unfold of
+ * Eq. 5 along the width, taken by the loads themselves instead of being written out; see
+ * ssconv_space_to_depth).  Everything else as ssconv_forward_dense; C_in == 8 is not accepted. */
+int32_t ssconv_forward_dense_strided(const ssconv_desc_t* desc, const void* x, int64_t stride_w, int64_t stride_h,
+                                     int64_t stride_n, const void* w_bf16, const float* bias, void* y, void* ws,
+                                     size_t ws_bytes, int32_t* dev_status, void* stream);
 
 /* ssconv_forward for callers that have no way to provide scratch memory.  (The paper has no
  * counterpart to this call; it exists for integration only.)

@@ -25,8 +25,8 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.
 EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes",
            "ssconv_plan", "ssconv_tune",
            "ssconv_select_mask",
-           "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_unfold_w", "ssconv_forward", "ssconv_forward_res",
-           "ssconv_forward_dense_res", "ssconv_forward_dense",
+           "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_pad_channels", "ssconv_space_to_depth", "ssconv_unfold_w", "ssconv_forward", "ssconv_forward_res",
+           "ssconv_forward_dense_res", "ssconv_forward_dense", "ssconv_forward_dense_strided",
            "ssconv_mask_norms", "ssconv_absmax", "ssconv_stability_threshold", "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_dgrad_prepare", "ssconv_dgrad_spread", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
            "ssconv_forward_static_ws")
 
@@ -295,6 +295,60 @@ def ssconv_maxpool(x: torch.Tensor, k: int = 3, stride: int = 2, pad: int = 1, y
     f.restype = ctypes.c_int32
     f.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int32] * 7 + [ctypes.c_void_p]
     _check("ssconv_maxpool", f(_ptr(x), _ptr(y), n, h, w, c, k, stride, pad, _stream(stream)))
+    return y
+
+
+def ssconv_space_to_depth(x: torch.Tensor, block: int, pad: int, Hb: int, Wb: int, C_pad: int,
+                          y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """y [N,Hb,Wb,C_pad] with y[n,r,q,(bh*block+bw)*C+c] = x[n, block*r-pad+bh, block*q-pad+bw, c] (zeros outside
+    the image and in the padding channels) from x [N,H,W,C] bf16."""
+    _need_cuda(x, y)
+    n, h, w, c = x.shape
+    if y is None:
+        y = torch.empty((n, Hb, Wb, C_pad), dtype=torch.bfloat16, device=x.device)
+    f = lib().ssconv_space_to_depth
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int32] * 9 + [ctypes.c_void_p]
+    _check("ssconv_space_to_depth", f(_ptr(x), _ptr(y), n, h, w, c, block, pad, Hb, Wb, C_pad, _stream(stream)))
+    return y
+
+
+def ssconv_forward_dense_strided(desc: Desc, x: torch.Tensor, strides, w: torch.Tensor,
+                                 bias: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None,
+                                 ws: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                                 stream=None) -> torch.Tensor:
+    """ssconv_forward_dense on a strided (possibly overlapping) view of x: `strides` = element strides of
+    (w, h, n); pixel (n, h, w) of the input the descriptor names starts n*s_n + h*s_h + w*s_w elements into x."""
+    _need_cuda(x, w, bias, y, ws, dev_status)
+    if y is None:
+        y = _alloc_y(desc, x)
+    if ws is None:
+        ws = default_workspace(x.device)
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    s_w, s_h, s_n = (int(v) for v in strides)
+    f = lib().ssconv_forward_dense_strided
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
+                  ctypes.c_void_p, ctypes.c_void_p]
+    _check("ssconv_forward_dense_strided", f(ctypes.byref(desc), _ptr(x), s_w, s_h, s_n, _ptr(w), _ptr(bias), _ptr(y),
+                                             _ptr(ws), ws_bytes, _ptr(dev_status), _stream(stream)))
+    return y
+
+
+def ssconv_pad_channels(x: torch.Tensor, C_pad: int, y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Zero-pad the channels of x [..., C] bf16 to C_pad (a multiple of 8); returns y [..., C_pad]."""
+    _need_cuda(x, y)
+    *lead, c = x.shape
+    pixels = 1
+    for d in lead:
+        pixels *= d
+    if y is None:
+        y = torch.empty((*lead, C_pad), dtype=torch.bfloat16, device=x.device)
+    f = lib().ssconv_pad_channels
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
+    _check("ssconv_pad_channels", f(_ptr(x), _ptr(y), pixels, c, C_pad, _stream(stream)))
     return y
 
 

@@ -16,11 +16,14 @@ int32_t launch_forward_sparse(const ssconv_desc_t& d, const void* x, const void*
                               int32_t* dev_status, cudaStream_t stream);
 int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* w, const float* bias,
                              const void* residual, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
-                             cudaStream_t stream);
+                             cudaStream_t stream, const int64_t* x_strides = nullptr);
+cudaError_t launch_space_to_depth(const void* x, void* y, int N, int H, int W, int C, int s, int pad, int Hb, int Wb,
+                                  int C_pad, cudaStream_t st);
 size_t workspace_bytes();
 int32_t set_tuning(int32_t option, int32_t value);
 cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad,
                            cudaStream_t st);
+cudaError_t launch_pad_channels(const void* x, void* y, long long pixels, int C, int C_pad, cudaStream_t st);
 cudaError_t launch_unfold_w(const void* x, void* y, long long rows, int W, int C, int KW, int stride, int pad, int dil,
                             int C_pad, cudaStream_t st);
 int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* split, int32_t* ctas,
@@ -191,6 +194,16 @@ int32_t ssconv_maxpool(const void* x, void* y, int32_t N, int32_t H, int32_t W, 
              : SSCONV_ERR_CUDA;
 }
 
+int32_t ssconv_pad_channels(const void* x, void* y, int64_t pixels, int32_t C, int32_t C_pad, void* stream) {
+  if (!x || !y) return SSCONV_ERR_NULL;
+  if (pixels <= 0 || C <= 0 || C_pad < C) return SSCONV_ERR_BAD_DESC;
+  if (C_pad % 8 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(x) & 1u) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  if (pixels > 0x7FFFFFFFFFLL / C_pad) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  return ssconv::launch_pad_channels(x, y, pixels, C, C_pad, (cudaStream_t)stream) == cudaSuccess ? SSCONV_OK
+                                                                                                  : SSCONV_ERR_CUDA;
+}
+
 int32_t ssconv_unfold_w(const void* x, void* y, int64_t rows, int32_t W, int32_t C, int32_t KW, int32_t stride_w,
                         int32_t pad_w, int32_t dil_w, int32_t C_pad, void* stream) {
   if (!x || !y) return SSCONV_ERR_NULL;
@@ -239,6 +252,37 @@ int32_t ssconv_forward_dense(const ssconv_desc_t* desc, const void* x, const voi
   if (!aligned16(x) || !aligned16(w_bf16) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
   return ssconv::launch_forward_dense(*desc, x, w_bf16, bias, nullptr, y, ws, ws_bytes, dev_status,
                                       (cudaStream_t)stream);
+}
+
+int32_t ssconv_forward_dense_strided(const ssconv_desc_t* desc, const void* x, int64_t stride_w, int64_t stride_h,
+                                     int64_t stride_n, const void* w_bf16, const float* bias, void* y, void* ws,
+                                     size_t ws_bytes, int32_t* dev_status, void* stream) {
+  int32_t rc = check_desc(desc, true);
+  if (rc != SSCONV_OK) return rc;
+  if (!x || !w_bf16 || !y) return SSCONV_ERR_NULL;
+  if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
+  if (!aligned16(x) || !aligned16(w_bf16) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  if (desc->C_in == 8) return SSCONV_ERR_UNSUPPORTED_SHAPE;  // the 8-channel mode reads packed pixels
+  // tensor-map strides are multiples of 16 bytes below 2^40
+  if (stride_w <= 0 || stride_h <= 0 || stride_n <= 0 || stride_w % 8 || stride_h % 8 || stride_n % 8)
+    return SSCONV_ERR_BAD_DESC;
+  if (stride_n >= (1LL << 38) || stride_h >= (1LL << 38) || stride_w >= (1LL << 38)) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  const int64_t strides[3] = {stride_w, stride_h, stride_n};
+  return ssconv::launch_forward_dense(*desc, x, w_bf16, bias, nullptr, y, ws, ws_bytes, dev_status,
+                                      (cudaStream_t)stream, strides);
+}
+
+int32_t ssconv_space_to_depth(const void* x, void* y, int32_t N, int32_t H, int32_t W, int32_t C, int32_t block,
+                              int32_t pad, int32_t Hb, int32_t Wb, int32_t C_pad, void* stream) {
+  if (!x || !y) return SSCONV_ERR_NULL;
+  if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || block <= 0 || pad < 0 || Hb <= 0 || Wb <= 0) return SSCONV_ERR_BAD_DESC;
+  if (C_pad % 8 != 0 || (long long)block * block * C > C_pad) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(x) & 1u) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  if ((long long)N * Hb > 0x7FFFFFFFLL || (long long)Wb * C_pad > 0x7FFFFFFFLL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)Wb * (C_pad / 8) > 65535LL * 256) return SSCONV_ERR_UNSUPPORTED_SHAPE;  // grid limit along a row
+  return ssconv::launch_space_to_depth(x, y, N, H, W, C, block, pad, Hb, Wb, C_pad, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
 }
 
 int32_t ssconv_forward_dense_res(const ssconv_desc_t* desc, const void* x, const void* w_bf16, const float* bias,

@@ -75,6 +75,89 @@ __global__ void __launch_bounds__(256) unfold_w_kernel(const uint4* __restrict__
   y[i] = v;
 }
 
+// Channel padding: y[p, c] = x[p, c] for c < C, 0 for C <= c < C_pad (an RGB image into the 8-channel
+// form the dense entry point takes).  One thread per 16 bytes of y; the reads are scalar (a pixel of
+// 3 channels is 6 bytes), which is harmless at this size: the step moves about a quarter of the
+// bytes of the layer that follows it.
+__global__ void __launch_bounds__(256) pad_channels_kernel(const __nv_bfloat16* __restrict__ x, uint4* __restrict__ y,
+                                                           long long total, int C, int Cp8) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int ch = (int)(i % Cp8) * 8;
+  const long long pix = i / Cp8;
+  const unsigned short* src = reinterpret_cast<const unsigned short*>(x) + pix * C;
+  unsigned short v[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) v[j] = (ch + j < C) ? __ldg(src + ch + j) : (unsigned short)0;
+  uint4 o;
+  o.x = v[0] | ((uint32_t)v[1] << 16);
+  o.y = v[2] | ((uint32_t)v[3] << 16);
+  o.z = v[4] | ((uint32_t)v[5] << 16);
+  o.w = v[6] | ((uint32_t)v[7] << 16);
+  y[i] = o;
+}
+
+// Space to depth: blocks of `s` x `s` pixels of the zero-padded image become the channels of one
+// pixel,  y[n, r, q, (bh s + bw) C + c] = x[n, s r - pad + bh, s q - pad + bw, c]  (0 outside the image
+// and in the channels beyond s s C), for r < Hb, q < Wb.  A K x K convolution of stride s and padding
+// pad over x is then a ceil(K/s) x ceil(K/s) convolution of unit stride and no padding over y (with
+// weights rearranged by the same call, as K x K "images" with pad 0), when Hb = H_out + ceil(K/s) - 1
+// rows are produced: few-channel images turn into pixels wide enough for the tensor-core path without
+// the (K-fold) duplication of an unfold.  One thread per 16 bytes of y; scalar reads.
+__global__ void __launch_bounds__(256) space_to_depth_kernel(const unsigned short* __restrict__ x, uint4* __restrict__ y,
+                                                             int H, int W, int C, int s, int pad, int Hb, int Wb,
+                                                             int Cp8) {
+  // one grid row per row of y (n, r); threads along the row's 16-byte chunks (q, k)
+  const int col = blockIdx.y * blockDim.x + threadIdx.x;
+  if (col >= Wb * Cp8) return;
+  const int row = blockIdx.x;
+  const int n = row / Hb, r = row - n * Hb;
+  const int q = col / Cp8, k = col - q * Cp8;
+  // channel 8 k of the pixel = (block pixel blk = bh s + bw, channel c); the next seven follow incrementally
+  int blk = (8 * k) / C, c = 8 * k - blk * C;
+  int bh = blk / s, bw = blk - bh * s;
+  const unsigned short* img = x + (size_t)n * H * W * C;
+  unsigned short v[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int h = s * r - pad + bh, w = s * q - pad + bw;
+    v[j] = (bh < s && h >= 0 && h < H && w >= 0 && w < W) ? __ldg(img + ((size_t)h * W + w) * C + c) : (unsigned short)0;
+    if (++c == C) {
+      c = 0;
+      if (++bw == s) {
+        bw = 0;
+        ++bh;
+      }
+    }
+  }
+  uint4 o;
+  o.x = v[0] | ((uint32_t)v[1] << 16);
+  o.y = v[2] | ((uint32_t)v[3] << 16);
+  o.z = v[4] | ((uint32_t)v[5] << 16);
+  o.w = v[6] | ((uint32_t)v[7] << 16);
+  y[(size_t)row * Wb * Cp8 + col] = o;
+}
+
+cudaError_t launch_space_to_depth(const void* x, void* y, int N, int H, int W, int C, int s, int pad, int Hb, int Wb,
+                                  int C_pad, cudaStream_t st) {
+  const int T = 256;
+  const int per_row = Wb * (C_pad / 8);
+  count_launch();
+  space_to_depth_kernel<<<dim3((unsigned)(N * Hb), (unsigned)((per_row + T - 1) / T)), T, 0, st>>>(
+      static_cast<const unsigned short*>(x), static_cast<uint4*>(y), H, W, C, s, pad, Hb, Wb, C_pad / 8);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pad_channels(const void* x, void* y, long long pixels, int C, int C_pad, cudaStream_t st) {
+  const long long total = pixels * (C_pad / 8);
+  if (total == 0) return cudaSuccess;
+  const int T = 256;
+  count_launch();
+  pad_channels_kernel<<<(unsigned)((total + T - 1) / T), T, 0, st>>>(static_cast<const __nv_bfloat16*>(x),
+                                                                     static_cast<uint4*>(y), total, C, C_pad / 8);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_unfold_w(const void* x, void* y, long long rows, int W, int C, int KW, int stride, int pad, int dil,
                             int C_pad, cudaStream_t st) {
   const int span = W + 2 * pad - dil * (KW - 1) - 1;

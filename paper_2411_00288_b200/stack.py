@@ -3,8 +3,11 @@
 Only marshalling: weights are masked and compressed once with the library's own calls, output
 buffers are allocated once, and forward() issues one C-ABI call per convolution on the current
 stream (so it can be recorded into a CUDA graph); the 3x3 stride-2 max-pool between the stem and
-the first block is the library's ssconv_maxpool.  A dense layer with 8 input channels (the stem) runs
-as ssconv_unfold_w followed by the equivalent KH x 1 convolution over the unfolded taps.
+the first block is the library's ssconv_maxpool.  The stem (a dense strided convolution over very few
+channels) has two forms, chosen by the channel count of the tensor handed to forward(): raw images
+(fewer channels than the stem's padded C_in, e.g. RGB) go through ssconv_space_to_depth and the
+equivalent T x 1 convolution on a sliding-window view (ssconv_forward_dense_strided); images already
+padded to the stem's C_in go through ssconv_unfold_w and the equivalent KH x 1 convolution.
 """
 from __future__ import annotations
 
@@ -51,35 +54,63 @@ class ConvStack:
                         desc=api.make_desc(spec.N, spec.H, spec.W_out, c_pad, spec.C_out, spec.KH, 1,
                                            stride=(spec.stride, 1), pad=(spec.pad, 0), dil=(spec.dil, 1),
                                            bias=spec.has_bias, relu=spec.relu and not spec.gelu, gelu=spec.gelu))
+                if st.kind == "dense" and spec.C_in == 8 and spec.KH == spec.KW and spec.stride > 1 and st.src < 0:
+                    entry["s2d"] = self._prepare_s2d(spec, w, real_c=3)
                 self.layers.append(entry)
                 shape = (spec.N, spec.H_out, spec.W_out, spec.C_out)
             shapes.append(shape)
             self.outputs.append(torch.empty(shape, dtype=torch.bfloat16, device=self.device))
         torch.cuda.synchronize(self.device)
 
+    def _prepare_s2d(self, spec, w: torch.Tensor, real_c: int):
+        """Buffers, weights and descriptor of the space-to-depth form of a K x K stride-s layer on images
+        of `real_c` channels: blocks of s x s pixels become one pixel of C_pad channels, T = ceil(K/s)
+        neighbouring block pixels are read as one pixel of T*C_pad channels, and the layer is a T x 1
+        convolution of unit stride without padding over that view."""
+        s, K = spec.stride, spec.KH
+        T = -(-K // s)
+        c_pad = -(-s * s * real_c // 8) * 8
+        hb, wb = spec.H_out + T - 1, spec.W_out + T - 1
+        w_real = w[..., :real_c].contiguous()
+        w_s2d = api.ssconv_space_to_depth(w_real, s, 0, T, T, c_pad)          # [C_out, T, T, c_pad]
+        desc = api.make_desc(spec.N, hb, spec.W_out, T * c_pad, spec.C_out, T, 1, stride=1, pad=0, dil=1,
+                             bias=spec.has_bias, relu=spec.relu and not spec.gelu, gelu=spec.gelu)
+        return dict(block=s, pad=spec.pad, hb=hb, wb=wb, c_pad=c_pad, real_c=real_c, w=w_s2d, desc=desc,
+                    strides=(c_pad, wb * c_pad, hb * wb * c_pad),
+                    x=torch.empty((spec.N, hb, wb, c_pad), dtype=torch.bfloat16, device=self.device))
+
+    def run_step(self, i: int, x: torch.Tensor, sparse: bool = True) -> torch.Tensor:
+        """Enqueue step i alone (its input must already be in place); returns its output tensor."""
+        st = self.steps[i]
+        src = x if st.src < 0 else self.outputs[st.src]
+        y = self.outputs[i]
+        if st.kind == "maxpool":
+            api.ssconv_maxpool(src, 3, 2, 1, y=y)
+            return y
+        L = self.layers[i]
+        res = self.outputs[st.res] if st.res >= 0 else None
+        if st.kind == "conv" and sparse:
+            api.ssconv_forward(L["desc"], src, L["w_comp"], L["meta"], L["bias"], y=y, dev_status=self.status,
+                               residual=res)
+        elif "s2d" in L and src.shape[-1] == L["s2d"]["real_c"]:
+            S = L["s2d"]
+            api.ssconv_space_to_depth(src, S["block"], S["pad"], S["hb"], S["wb"], S["c_pad"], y=S["x"])
+            api.ssconv_forward_dense_strided(S["desc"], S["x"], S["strides"], S["w"], L["bias"], y=y,
+                                             dev_status=self.status)
+        elif "unfold" in L:
+            U = L["unfold"]
+            sp = st.spec
+            api.ssconv_unfold_w(src, sp.KW, sp.stride, sp.pad, sp.dil, C_pad=U["c_pad"], y=U["x"])
+            api.ssconv_forward_dense(U["desc"], U["x"], U["w"], L["bias"], y=y, dev_status=self.status, residual=res)
+        else:
+            api.ssconv_forward_dense(L["desc"], src, L["w"], L["bias"], y=y, dev_status=self.status, residual=res)
+        return y
+
     def forward(self, x: torch.Tensor, sparse: bool = True) -> torch.Tensor:
         """Enqueue the whole stack; returns the last chained output (not synchronised)."""
         last = None
         for i, st in enumerate(self.steps):
-            src = x if st.src < 0 else self.outputs[st.src]
-            y = self.outputs[i]
-            if st.kind == "maxpool":
-                api.ssconv_maxpool(src, 3, 2, 1, y=y)
-            else:
-                L = self.layers[i]
-                res = self.outputs[st.res] if st.res >= 0 else None
-                if st.kind == "conv" and sparse:
-                    api.ssconv_forward(L["desc"], src, L["w_comp"], L["meta"], L["bias"], y=y, dev_status=self.status,
-                                       residual=res)
-                elif "unfold" in L:
-                    U = L["unfold"]
-                    sp = st.spec
-                    api.ssconv_unfold_w(src, sp.KW, sp.stride, sp.pad, sp.dil, C_pad=U["c_pad"], y=U["x"])
-                    api.ssconv_forward_dense(U["desc"], U["x"], U["w"], L["bias"], y=y, dev_status=self.status,
-                                             residual=res)
-                else:
-                    api.ssconv_forward_dense(L["desc"], src, L["w"], L["bias"], y=y, dev_status=self.status,
-                                             residual=res)
+            y = self.run_step(i, x, sparse)
             if st.feeds_next:
                 last = y
         return last
