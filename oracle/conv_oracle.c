@@ -128,8 +128,9 @@ int32_t oracle_conv2d_f64(const oracle_conv_shape* s, const uint16_t* x_bf16,
 }
 
 /* Selected output elements only: idx holds flat indices into y [N,H_out,W_out,C_out].
- * Used where the full tensor would take too long; every element is evaluated by the
- * same per-element routine as above. */
+ * Used where the full tensor would take too long.  It has a loop of its own (the same sum of Eq. 4,
+ * term by term in the same order, over bf16 inputs widened on the fly instead of a widened copy of
+ * the whole input); a test pins it equal to the full-tensor routine. */
 int32_t oracle_conv2d_f64_sample(const oracle_conv_shape* s, const uint16_t* x_bf16,
                                  const uint16_t* w_bf16, const uint8_t* mask,
                                  const float* bias, const int64_t* idx, int64_t n_idx,

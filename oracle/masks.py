@@ -69,24 +69,14 @@ def select_from_magnitude(w_bits: np.ndarray) -> np.ndarray:
     kept first (a stable ordering), so the result is unique.
     """
     a = _abs_bits(w_bits).reshape(-1, 4)
-    G = a.shape[0]
-    # rank each position: position j beats position i when it is strictly larger, or
-    # equal and earlier.  The two positions beaten by fewer than two others are kept.
-    beaten_by = np.zeros((G, 4), dtype=np.int32)
-    for i in range(4):
-        for j in range(4):
-            if i == j:
-                continue
-            wins = (a[:, j] > a[:, i]) | ((a[:, j] == a[:, i]) & (j < i))
-            beaten_by[:, i] += wins
-    kept = beaten_by < 2  # exactly two per group
+    # the plain definition: sort the four positions by decreasing magnitude with a stable sort (equal
+    # magnitudes keep their order, so the lower position comes first) and keep the first two
+    order = np.argsort(-a, axis=1, kind="stable")
+    kept = np.sort(order[:, :2], axis=1)
     lut = {pos: p for p, pos in enumerate(KEPT_POSITIONS)}
-    out = np.empty(G, dtype=np.uint8)
-    # map the kept pair to its pattern index
-    first = np.argmax(kept, axis=1)
-    second = 3 - np.argmax(kept[:, ::-1], axis=1)
+    out = np.empty(a.shape[0], dtype=np.uint8)
     for (pa, pb), p in lut.items():
-        out[(first == pa) & (second == pb)] = p
+        out[(kept[:, 0] == pa) & (kept[:, 1] == pb)] = p
     return out
 
 

@@ -81,16 +81,30 @@ def _alphabet_bits():
     return f32_to_bf16_bits(vals)
 
 
-def test_select_magnitude_exhaustive_vs_stable_sort():
+def _best_pattern_by_enumeration(mags):
+    """Brute force over the six patterns, no sorting: the pattern whose kept pair has the largest
+    magnitude sum (exact: the magnitudes are small dyadic numbers); among equal sums the one whose kept
+    positions come first in lexicographic order, which is what "the lower position wins a tie" means."""
+    best, best_key = None, None
+    for p, (i, j) in enumerate(masks.KEPT_POSITIONS):
+        key = (-(mags[i] + mags[j]), i, j)
+        if best_key is None or key < best_key:
+            best, best_key = p, key
+    return best
+
+
+def test_select_magnitude_exhaustive_vs_enumeration():
     alpha = _alphabet_bits()
     groups = np.array(list(itertools.product(alpha, repeat=4)), dtype=np.uint16)
     got = masks.select_from_magnitude(groups)
     mags = np.abs(bf16_to_f64(groups))
     D = masks.pattern_matrix()
     for g in range(groups.shape[0]):
-        order = sorted(range(4), key=lambda i: (-mags[g, i], i))  # stable: ties -> lower position
-        kept = tuple(sorted(order[:2]))
-        assert masks.KEPT_POSITIONS[got[g]] == kept
+        assert got[g] == _best_pattern_by_enumeration(mags[g])
+        # the kept pair holds the two largest magnitudes: nothing dropped exceeds anything kept
+        kept = list(masks.KEPT_POSITIONS[got[g]])
+        dropped = [i for i in range(4) if i not in kept]
+        assert min(mags[g, kept]) >= max(mags[g, dropped])
         # optimality: no other pattern keeps a larger magnitude sum (exact in fp64)
         sums = mags[g] @ D
         assert sums[got[g]] >= sums.max()
@@ -169,5 +183,22 @@ def test_pins_catch_planted_mistakes(plant, monkeypatch):
         rows = _golden_patterns()
         assert any(list(D[:, p]) != bits for p, *bits in rows)
     else:
-        groups = np.tile(_alphabet_bits()[4], (1, 4)).astype(np.uint16)  # all equal magnitudes
-        assert masks.KEPT_POSITIONS[masks.select_from_magnitude(groups)[0]] == (0, 1)
+        # plant a tie-break that prefers the LATER position (an unstable sort would do this): the
+        # exhaustive enumeration pin must notice on the groups that hold equal magnitudes
+        def later_wins(w_bits):
+            a = masks._abs_bits(w_bits).reshape(-1, 4)
+            order = np.argsort(-a[:, ::-1], axis=1, kind="stable")   # ties -> higher position first
+            kept = np.sort(3 - order[:, :2], axis=1)
+            out = np.empty(a.shape[0], dtype=np.uint8)
+            for p, (pa, pb) in enumerate(masks.KEPT_POSITIONS):
+                out[(kept[:, 0] == pa) & (kept[:, 1] == pb)] = p
+            return out
+        monkeypatch.setattr(masks, "select_from_magnitude", later_wins)
+        alpha = _alphabet_bits()
+        groups = np.array(list(itertools.product(alpha, repeat=4)), dtype=np.uint16)
+        got = masks.select_from_magnitude(groups)
+        mags = np.abs(bf16_to_f64(groups))
+        wrong = [g for g in range(groups.shape[0]) if got[g] != _best_pattern_by_enumeration(mags[g])]
+        assert wrong, "the planted tie-break went unnoticed"
+        # and only tie groups are affected: where all four magnitudes differ both rules agree
+        assert all(len(set(mags[g])) < 4 for g in wrong)
