@@ -109,6 +109,24 @@ int32_t ssconv_plan(const ssconv_desc_t* desc, int32_t sparse, int32_t* tile_pos
 enum { SSCONV_TUNE_TILE_POSITIONS = 1, SSCONV_TUNE_PAIR = 2 };
 int32_t ssconv_tune(int32_t option, int32_t value);
 
+/* ssconv_plan for a device with `sm_count` SMs, without looking at any device (host arithmetic
+ * only; usable where no GPU is present, e.g. to pin the planner's choices in a test). */
+int32_t ssconv_plan_for_sms(const ssconv_desc_t* desc, int32_t sparse, int32_t sm_count, int32_t* tile_positions,
+                            int32_t* split, int32_t* ctas, int32_t* ring_groups, int32_t* pair);
+
+/* Extent of a sliding window: the number of placements of a window of k taps with the given stride,
+ * padding and dilation along an axis of `in` elements, floor((in + 2 pad - dil (k-1) - 1)/stride) + 1
+ * (0 if the window does not fit): the output-extent formula of Sec. 3.3 as the library computes it
+ * for the convolutions, the max-pool, the width unfold and the spread-out gradient.  Host only. */
+int32_t ssconv_window_extent(int32_t in, int32_t k, int32_t stride, int32_t pad, int32_t dil);
+
+/* Self-test of the bounded waits every kernel of this library relies on (no counterpart in the
+ * paper): launches a one-block kernel that waits, with a limit of `limit_cycles` SM clock cycles, on
+ * an mbarrier nobody ever arrives at.  The wait gives up, the kernel stores SSCONV_ERR_TIMEOUT to
+ * *dev_status (device int32, required) exactly as the convolution kernels do, and returns normally,
+ * so the context stays usable.  limit_cycles in [1000, 2e9]. */
+int32_t ssconv_selftest_wait_timeout(int64_t limit_cycles, int32_t* dev_status, void* stream);
+
 /* Hard pattern choice per group (Eq. 1 of Sec. 3.1 without the one-hot: the index of the
  * winning pattern).
  *   mode LOGITS:    pattern[g] = argmax_i scores[g][i]; the caller has already added any
@@ -126,7 +144,9 @@ int32_t ssconv_select_mask(int32_t mode, const void* scores, int64_t G, uint8_t*
  * two 2-bit position indices per group, laid out in the tile order the sparse tensor-core
  * instruction reads.  Needs C_in % 8 == 0 (else SSCONV_ERR_UNSUPPORTED_SHAPE: run such a
  * layer through ssconv_forward_dense).  w_comp / meta: device, 16-byte aligned, of the
- * sizes ssconv_sizes reports; every byte of both blobs is written. */
+ * sizes ssconv_sizes reports; every byte of both blobs is written.  pattern[g] must be in 0..5;
+ * the array lives on the device and is not checked: a value outside that range is treated as
+ * pattern 0, so the blobs stay well-formed whatever the array holds. */
 int32_t ssconv_compress(const ssconv_desc_t* desc, const void* w_bf16, const uint8_t* pattern,
                         void* w_comp, void* meta, void* stream);
 
@@ -195,8 +215,9 @@ int32_t ssconv_unfold_w(const void* x, void* y, int64_t rows, int32_t W, int32_t
  * by the same call, sums them in a fixed order, so results are reproducible.  ws needs no
  * initialisation: every part is written before it is read.  Calls issued one after another on
  * one stream may share it; calls that may overlap on the GPU need separate workspaces.
- * If ws is NULL or too small and
- * the layer needs it, SSCONV_ERR_WORKSPACE is returned and nothing is launched.
+ * If ws is NULL or too small
+ * the K range is never split: such layers then run on whole tiles (correct, slower where a layer has
+ * few tiles and a deep K), so a caller without scratch memory can pass ws = NULL for any layer.
  * dev_status (nullable): device int32; a kernel whose bounded wait expires stores
  * SSCONV_ERR_TIMEOUT there and drains instead of hanging; it is never written on success,
  * so the caller zeroes it once and reads it after its own synchronisation. */
@@ -358,7 +379,10 @@ int32_t ssconv_forward_dense_strided(const ssconv_desc_t* desc, const void* x, i
  *  - The K range is always split, over at most 64 thread blocks, so the fp32 summation order,
  *    and with it the last bits of y, can differ from ssconv_forward's.
  *  - The first call on each device looks up the array's device address (with that device
- *    current); make that first call outside any stream capture.
+ *    current); make that first call outside any stream capture.  The array itself comes into
+ *    being when the CUDA module that holds the forward kernels is loaded on the device, which
+ *    under CUDA's default lazy loading is the first forward call of any kind on that device:
+ *    until then its 15.7 MB are not yet taken.
  *  - All calls share the one array, and it keeps what the previous call left in it.  Nothing in
  *    it has to be cleared (every partial sum is written before it is read), so calls issued one
  *    after another on one stream are safe; two calls that can overlap on the GPU

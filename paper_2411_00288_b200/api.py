@@ -23,7 +23,7 @@ ERR_TIMEOUT = 8
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.so")
 EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes",
-           "ssconv_plan", "ssconv_tune",
+           "ssconv_plan", "ssconv_plan_for_sms", "ssconv_tune", "ssconv_window_extent", "ssconv_selftest_wait_timeout",
            "ssconv_select_mask",
            "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_pad_channels", "ssconv_space_to_depth", "ssconv_unfold_w", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense", "ssconv_forward_dense_strided",
@@ -189,6 +189,34 @@ def ssconv_decompress(desc: Desc, w_comp: torch.Tensor, meta: torch.Tensor, want
 _workspaces = {}
 
 
+def ssconv_window_extent(n: int, k: int, stride: int = 1, pad: int = 0, dil: int = 1) -> int:
+    """Placements of a k-tap window along an axis of n elements, as the library computes them."""
+    f = lib().ssconv_window_extent
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_int32] * 5
+    return int(f(int(n), int(k), int(stride), int(pad), int(dil)))
+
+
+def ssconv_plan_for_sms(desc: Desc, sparse: bool, sm_count: int) -> dict:
+    """ssconv_plan for a device with `sm_count` SMs; host arithmetic only, no GPU needed."""
+    out = [ctypes.c_int32(0) for _ in range(5)]
+    f = lib().ssconv_plan_for_sms
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_int32, ctypes.c_int32] + [ctypes.POINTER(ctypes.c_int32)] * 5
+    _check("ssconv_plan_for_sms", f(ctypes.byref(desc), 1 if sparse else 0, int(sm_count), *[ctypes.byref(o) for o in out]))
+    return dict(tile_positions=out[0].value, split=bool(out[1].value), ctas=out[2].value, ring_groups=out[3].value,
+                pair=bool(out[4].value))
+
+
+def ssconv_selftest_wait_timeout(limit_cycles: int, dev_status: torch.Tensor, stream=None) -> None:
+    """Launch the one-block kernel whose bounded wait runs out; it stores ERR_TIMEOUT to dev_status."""
+    _need_cuda(dev_status)
+    f = lib().ssconv_selftest_wait_timeout
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
+    _check("ssconv_selftest_wait_timeout", f(int(limit_cycles), _ptr(dev_status), _stream(stream)))
+
+
 def ssconv_plan(desc: Desc, sparse: bool = True) -> dict:
     """Tile width, K split, thread blocks and ring depth the forward call would use on the current device."""
     out = [ctypes.c_int32(0) for _ in range(5)]
@@ -289,7 +317,7 @@ def ssconv_maxpool(x: torch.Tensor, k: int = 3, stride: int = 2, pad: int = 1, y
     _need_cuda(x, y)
     n, h, w, c = x.shape
     if y is None:
-        y = torch.empty((n, (h + 2 * pad - k) // stride + 1, (w + 2 * pad - k) // stride + 1, c),
+        y = torch.empty((n, ssconv_window_extent(h, k, stride, pad), ssconv_window_extent(w, k, stride, pad), c),
                         dtype=torch.bfloat16, device=x.device)
     f = lib().ssconv_maxpool
     f.restype = ctypes.c_int32
@@ -455,9 +483,9 @@ def ssconv_unfold_w(x: torch.Tensor, KW: int, stride: int = 1, pad: int = 0, dil
         rows *= d
     if C_pad is None:
         C_pad = -(-KW * c // 64) * 64
-    wo = (w + 2 * pad - dil * (KW - 1) - 1) // stride + 1
     if y is None:
-        y = torch.empty((*lead, wo, C_pad), dtype=torch.bfloat16, device=x.device)
+        y = torch.empty((*lead, ssconv_window_extent(w, KW, stride, pad, dil), C_pad), dtype=torch.bfloat16,
+                        device=x.device)
     f = lib().ssconv_unfold_w
     f.restype = ctypes.c_int32
     f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64] + [ctypes.c_int32] * 7 + [ctypes.c_void_p]
@@ -530,8 +558,8 @@ def ssconv_dgrad_spread(desc: Desc, dy: torch.Tensor, stream=None) -> torch.Tens
     """dy [N,H_out,W_out,C_out] of a strided layer spread out with zeros to [N,Hz,Wz,C_out],
     Hz = H + 2 pad - dil (KH - 1): the input of the convolution ssconv_dgrad_prepare describes."""
     _need_cuda(dy)
-    Hz = desc.H + 2 * desc.pad_h - desc.dil_h * (desc.KH - 1)
-    Wz = desc.W + 2 * desc.pad_w - desc.dil_w * (desc.KW - 1)
+    Hz = ssconv_window_extent(desc.H, desc.KH, 1, desc.pad_h, desc.dil_h)   # all unit-stride filter placements
+    Wz = ssconv_window_extent(desc.W, desc.KW, 1, desc.pad_w, desc.dil_w)
     out = torch.empty((desc.N, Hz, Wz, desc.C_out), dtype=torch.bfloat16, device=dy.device)
     f = lib().ssconv_dgrad_spread
     f.restype = ctypes.c_int32

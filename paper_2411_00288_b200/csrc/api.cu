@@ -19,6 +19,9 @@ int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* 
                              cudaStream_t stream, const int64_t* x_strides = nullptr);
 cudaError_t launch_space_to_depth(const void* x, void* y, int N, int H, int W, int C, int s, int pad, int Hb, int Wb,
                                   int C_pad, cudaStream_t st);
+int32_t plan_query_sms(const ssconv_desc_t& d, bool sparse, int sm_count, int32_t* bn, int32_t* split, int32_t* ctas,
+                       int32_t* ring_groups, int32_t* pair);
+cudaError_t launch_wait_timeout_selftest(long long limit_cycles, int32_t* dev_status, cudaStream_t st);
 size_t workspace_bytes();
 int32_t set_tuning(int32_t option, int32_t value);
 cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad,
@@ -142,6 +145,26 @@ int32_t ssconv_plan(const ssconv_desc_t* desc, int32_t sparse, int32_t* tile_pos
   int32_t st = check_desc(desc, true);
   if (st != SSCONV_OK) return st;
   return ssconv::plan_query(*desc, sparse != 0, tile_positions, split, ctas, ring_groups, pair);
+}
+
+int32_t ssconv_plan_for_sms(const ssconv_desc_t* desc, int32_t sparse, int32_t sm_count, int32_t* tile_positions,
+                            int32_t* split, int32_t* ctas, int32_t* ring_groups, int32_t* pair) {
+  int32_t st = check_desc(desc, true);
+  if (st != SSCONV_OK) return st;
+  return ssconv::plan_query_sms(*desc, sparse != 0, sm_count, tile_positions, split, ctas, ring_groups, pair);
+}
+
+int32_t ssconv_window_extent(int32_t in, int32_t k, int32_t stride, int32_t pad, int32_t dil) {
+  if (in <= 0 || k <= 0 || stride <= 0 || pad < 0 || dil <= 0) return 0;
+  return out_extent(in, k, stride, pad, dil);
+}
+
+int32_t ssconv_selftest_wait_timeout(int64_t limit_cycles, int32_t* dev_status, void* stream) {
+  if (!dev_status) return SSCONV_ERR_NULL;
+  if (limit_cycles < 1000 || limit_cycles > 2000000000LL) return SSCONV_ERR_BAD_DESC;
+  return ssconv::launch_wait_timeout_selftest(limit_cycles, dev_status, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
 }
 
 int32_t ssconv_tune(int32_t option, int32_t value) { return ssconv::set_tuning(option, value); }

@@ -1294,7 +1294,7 @@ struct Plan {
 };
 template <bool SPARSE>
 static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force_split, int max_bn = kBN,
-                       int stage_bufs = 2) {
+                       int stage_bufs = 2, bool allow_split = true) {
   if (force_split) return Plan{kBN, true};
   int min_bn = 48;
   if (g_tune_bn != 0 && g_tune_bn <= max_bn) max_bn = min_bn = g_tune_bn;
@@ -1315,7 +1315,7 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
   // Even split of K ("stream-K"), when many SMs would still idle and K is deep: every CTA gets the
   // same number of groups; parked partial tiles cost L2 traffic in proportion to the tile width.
   const int a_tiles = geo.stages;
-  if (a_tiles > 1) {
+  if (a_tiles > 1 && allow_split) {
     Plan best_split{kBN, true};
     double best_split_cost = 0.0;
     for (int BN = max_bn; BN >= min_bn; BN -= 16) {
@@ -1434,24 +1434,32 @@ static int widest_tile(uint32_t a_group_bytes, int stage_bufs) {
 
 // The plan for a layer without a residual: one-CTA tiles (whole or K split) or the pair kernel.
 template <bool SPARSE>
-static Plan choose_plan(const ssconv_desc_t& d, long long Q, const Geometry& geo, int workers, bool force_split) {
-  const Plan plan = plan_layer<SPARSE>(Q, geo, workers, force_split);
+static Plan choose_plan(const ssconv_desc_t& d, long long Q, const Geometry& geo, int workers, bool force_split,
+                        bool allow_split = true) {
+  const Plan plan = plan_layer<SPARSE>(Q, geo, workers, force_split, kBN, 2, allow_split);
   if (force_split || small_channel_mode(d, SPARSE) || g_tune_pair == 0) return plan;
   const Plan pair = plan_pair<SPARSE>(Q, geo, workers, g_tune_pair == 1);
   if (pair.BN != 0 && (g_tune_pair == 1 || plan.cost > kPairAdvantage * pair.cost)) return pair;
   return plan;
 }
 
+int32_t plan_query_sms(const ssconv_desc_t& d, bool sparse, int sm_count, int32_t* bn, int32_t* split, int32_t* ctas,
+                       int32_t* ring_groups, int32_t* pair);
 // What launch_forward_impl would do for this layer on the current device.
 int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* split, int32_t* ctas,
                    int32_t* ring_groups, int32_t* pair) {
   int dev = 0;
   const int32_t st = current_device(&dev);
   if (st != SSCONV_OK) return st;
+  return plan_query_sms(d, sparse, g_sm_count[dev], bn, split, ctas, ring_groups, pair);
+}
+int32_t plan_query_sms(const ssconv_desc_t& d, bool sparse, int sm_count, int32_t* bn, int32_t* split, int32_t* ctas,
+                       int32_t* ring_groups, int32_t* pair) {
+  if (sm_count <= 0) return SSCONV_ERR_BAD_DESC;
   const Geometry geo = layer_geometry(d, sparse);
   const long long Q = (long long)d.N * out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h) *
                       out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
-  const int workers = g_sm_count[dev] < kMaxWorkers ? g_sm_count[dev] : kMaxWorkers;
+  const int workers = sm_count < kMaxWorkers ? sm_count : kMaxWorkers;
   const Plan plan = sparse ? choose_plan<true>(d, Q, geo, workers, false) : choose_plan<false>(d, Q, geo, workers, false);
   const uint32_t a_group_bytes = sparse ? Cfg<true>::kAGroupBytes : Cfg<false>::kAGroupBytes;
   const long long q_tiles = (Q + plan.BN - 1) / plan.BN;
@@ -1506,8 +1514,13 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   // per group, which narrows the widest tile that still leaves room for two ring groups.  (When K
   // is split the finishing kernel adds the residual to the split tiles; the main kernel then keeps
   // two buffers and one piece of lookahead for the whole tiles it may also own.)
-  Plan plan = residual != nullptr ? plan_layer<SPARSE>(Q, geo, workers, force_split)
-                                  : choose_plan<SPARSE>(d, Q, geo, workers, force_split);
+  // Without a usable workspace the K range is not split: the best plan of whole tiles runs instead
+  // (slower on layers with few tiles and a deep K, never wrong).
+  const bool have_ws = ws != nullptr && ws_bytes >= scratch_bytes(worker_cap);
+  if (have_ws && (reinterpret_cast<uintptr_t>(ws) & 15u)) return SSCONV_ERR_ALIGNMENT;
+  if (force_split && !have_ws) return SSCONV_ERR_WORKSPACE;
+  Plan plan = residual != nullptr ? plan_layer<SPARSE>(Q, geo, workers, force_split, kBN, 2, have_ws)
+                                  : choose_plan<SPARSE>(d, Q, geo, workers, force_split, have_ws);
   int stage_bufs = 2;
   if (residual != nullptr && !plan.split) {
     stage_bufs = 4;
@@ -1664,8 +1677,6 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   int grid;
   if (p.split) {
     grid = units < workers ? (int)units : workers;
-    if (ws == nullptr || ws_bytes < scratch_bytes(worker_cap)) return SSCONV_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(ws) & 15u) return SSCONV_ERR_ALIGNMENT;
     p.ws_regions = static_cast<float4*>(ws);
   } else if (pair) {
     const int pairs = workers / 2;
@@ -1774,6 +1785,31 @@ int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const vo
   // partial-sum region is written by this call's main kernel before its finishing kernel reads it.
   return launch_forward_impl<true>(d, x, w_comp, meta, bias, nullptr, y, scratch, scratch_bytes(kStaticWorkers), dev_status,
                                    stream, kStaticWorkers, true);
+}
+
+// ---------------------------------------------------------------------------------------
+// Self-test of the bounded wait
+// ---------------------------------------------------------------------------------------
+// One block; thread 0 waits on an mbarrier that nobody arrives at, with the same helper and the same
+// give-up path as the convolution kernels (abort flag, status word), only with a short limit.
+__global__ void wait_timeout_selftest_kernel(long long limit_cycles, int32_t* dev_status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(&bar, 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const bool done = mbar_wait_bounded(&bar, 0, &abort_flag, limit_cycles);
+    if (!done && abort_flag != 0) atomicExch(dev_status, (int)SSCONV_ERR_TIMEOUT);
+  }
+}
+cudaError_t launch_wait_timeout_selftest(long long limit_cycles, int32_t* dev_status, cudaStream_t st) {
+  count_launch();
+  wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(limit_cycles, dev_status);
+  return cudaGetLastError();
 }
 
 }  // namespace ssconv

@@ -56,10 +56,12 @@ __host__ __device__ inline Geometry make_geometry(const ssconv_desc_t& d) {
 }
 
 // 4-bit position code (pos0 | pos1 << 2) of the six patterns, lexicographic in the kept
-// positions: {0,1},{0,2},{0,3},{1,2},{1,3},{2,3}.
+// positions: {0,1},{0,2},{0,3},{1,2},{1,3},{2,3}.  A pattern index outside 0..5 (the array comes
+// from the caller's device memory and cannot be checked on the host) is treated as pattern 0, so that
+// whatever is in the array the metadata stays legal for the sparse MMA (two ascending positions).
 __host__ __device__ inline uint32_t pattern_code(uint32_t p) {
   const uint32_t codes = 0x4u | (0x8u << 4) | (0xCu << 8) | (0x9u << 12) | (0xDu << 16) | (0xEu << 20);
-  return (codes >> (4 * p)) & 0xFu;
+  return p < 6u ? (codes >> (4 * p)) & 0xFu : 0x4u;
 }
 // Inverse: 4-bit code -> pattern index, 0xFF for a code that is not two ascending positions.
 __host__ __device__ inline uint32_t code_pattern(uint32_t code) {

@@ -30,7 +30,7 @@ class ConvStack:
         for st in steps:
             if st.kind == "maxpool":
                 n, h, w, c = shapes[st.src]
-                shape = (n, (h + 2 - 3) // 2 + 1, (w + 2 - 3) // 2 + 1, c)
+                shape = (n, api.ssconv_window_extent(h, 3, 2, 1), api.ssconv_window_extent(w, 3, 2, 1), c)
                 self.layers.append(None)
             else:
                 spec = st.spec

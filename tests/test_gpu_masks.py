@@ -83,3 +83,27 @@ def test_compress_roundtrip_bit_exact(shape):
     m = meta.cpu().numpy()
     nib = np.concatenate([m & 0xF, m >> 4])
     assert set(np.unique(nib)) <= {0x4, 0x8, 0xC, 0x9, 0xD, 0xE}
+
+
+def test_compress_treats_out_of_range_patterns_as_pattern_zero():
+    """The pattern array lives on the device and cannot be checked on the host: values outside 0..5
+    must still give well-formed blobs (legal metadata, the kept values of pattern 0)."""
+    shape = (64, 1, 1, 64)
+    rng = np.random.default_rng(5)
+    w = f32_to_bf16_bits(rng.normal(size=shape).astype(np.float32))
+    G = 64 * 64 // 4
+    pat = rng.integers(0, 6, size=G).astype(np.uint8)
+    bad = pat.copy()
+    where = rng.choice(G, size=40, replace=False)
+    bad[where] = rng.choice(np.array([6, 7, 8, 31, 200, 255], dtype=np.uint8), size=40)
+    fixed = pat.copy()
+    fixed[where] = 0
+    desc = api.make_desc(1, 8, 8, 64, 64, 1, 1, 1, 0)
+    w_comp, meta = api.ssconv_compress(desc, _bits_to_bf16_tensor(w).to(DEV), torch.from_numpy(bad).to(DEV))
+    w_back, pat_back = api.ssconv_decompress(desc, w_comp, meta)
+    torch.cuda.synchronize()
+    m = meta.cpu().numpy()
+    assert set(np.unique(np.concatenate([m & 0xF, m >> 4]))) <= {0x4, 0x8, 0xC, 0x9, 0xD, 0xE}
+    assert np.array_equal(pat_back.cpu().numpy(), fixed)
+    expect = masks.apply_mask(w, masks.mask_from_pattern(fixed, shape))
+    assert np.array_equal(w_back.cpu().view(torch.int16).numpy().view(np.uint16), expect)
