@@ -844,7 +844,7 @@ def sweep_arm(args):
     steps = max(1, min(args.steps, 2000))
 
     if args.only_layer is not None:   # profiling aid: one layer, launched repeatedly, nothing timed
-        spec = timed_layers()[args.only_layer]
+        spec = (synth.config_layers(5, args.batch or 256) if CONFIG_ID == 5 else timed_layers())[args.only_layer]
         inp = synth.make_inputs(spec)
         desc = api.desc_from_spec(spec)
         w, bias = inp.w.to(dev), inp.bias.to(dev)
@@ -989,7 +989,8 @@ def main():
     ap.add_argument("--layer-iters", type=int, default=None,
                     help="back-to-back launches per layer timing (default 10 for the stack, 100 for the sweeps)")
     ap.add_argument("--only-layer", type=int, default=None,
-                    help="with --workload-config 2|3|4, a profiling aid: launch just this layer --layer-iters times and exit")
+                    help="a profiling aid: launch just this layer of the chosen configuration (for the stack: the i-th of "
+                         "its 52 masked convolutions, on seeded inputs of its own) --layer-iters times and exit")
     ap.add_argument("--dense", action="store_true", help="with --only-layer: use the dense kernel")
     ap.add_argument("--residual", action="store_true",
                     help="fuse the network's skip connections into the expand convolutions of the stack")
@@ -1012,7 +1013,7 @@ def main():
         if CONFIG_ID == 5:
             CONFIG_ID, WORKLOAD = 2, WORKLOADS[2]
         train_arm(args)
-    elif CONFIG_ID == 5:
+    elif CONFIG_ID == 5 and args.only_layer is None:
         stack_arm(args)
     else:
         sweep_arm(args)
