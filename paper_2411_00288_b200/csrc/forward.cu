@@ -1304,8 +1304,10 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
     const long long tiles = ((Q + BN - 1) / BN) * geo.m_tiles;
     const long long per_cta = (tiles + workers - 1) / workers;
     const int pieces = (BN / 2 + kPiece - 1) / kPiece;
-    const double cost =
-        (double)per_cta * geo.kblocks * kblock_cycles<SPARSE>(BN, stage_bufs) + pieces * kEpiloguePieceCycles;
+    // (with at most three groups per tile the ring never reaches its steady state: such layers are paced
+    // by their output stream, and measured fastest at the width the other terms choose)
+    const double cost = (double)per_cta * geo.kblocks * kblock_cycles<SPARSE>(BN, stage_bufs, geo.stages >= 4) +
+                        pieces * kEpiloguePieceCycles;
     if (BN == max_bn || cost < 0.97 * best_cost) {  // a narrower tile has to earn its extra weight traffic
       best_cost = cost;
       best.BN = BN;
