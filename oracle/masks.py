@@ -61,14 +61,15 @@ def _abs_bits(w_bits: np.ndarray) -> np.ndarray:
     return (np.asarray(w_bits, dtype=np.uint16) & np.uint16(0x7FFF)).astype(np.int32)
 
 
-def select_from_magnitude(w_bits: np.ndarray) -> np.ndarray:
+def select_from_magnitude(w_bits: np.ndarray, magnitudes: np.ndarray = None) -> np.ndarray:
     """Magnitude heuristic (Sec. 2, Sec. 3.2 closing remark): keep the two largest |w|.
 
     w_bits: uint16 bf16 bit patterns, any shape whose last axis is a multiple of 4 and
     whose flattening is the group order above.  Equal magnitudes: the lower position is
-    kept first (a stable ordering), so the result is unique.
+    kept first (a stable ordering), so the result is unique.  For weights of another type pass
+    `magnitudes` (integers that order like |w|) instead; w_bits is then ignored.
     """
-    a = _abs_bits(w_bits).reshape(-1, 4)
+    a = (_abs_bits(w_bits) if magnitudes is None else np.asarray(magnitudes, dtype=np.int32)).reshape(-1, 4)
     # the plain definition: sort the four positions by decreasing magnitude with a stable sort (equal
     # magnitudes keep their order, so the lower position comes first) and keep the first two
     order = np.argsort(-a, axis=1, kind="stable")
