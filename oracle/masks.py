@@ -118,3 +118,53 @@ def logical_decompress(values: np.ndarray, codes: np.ndarray, shape) -> np.ndarr
     out[rows, c & 3] = v[:, 0]
     out[rows, (c >> 2) & 3] = v[:, 1]
     return out.reshape(shape)
+
+
+# ---------------------------------------------------------------------------------------------------
+# General N:M masks (Sec. 3.1: "N:M sparsity", blocks of M consecutive entries of a row of W of which
+# N are kept, n = C(M, N) possible blocks as the columns of D).  The pattern order is lexicographic in
+# the kept positions, which for 2:4 is the order of KEPT_POSITIONS above.
+# ---------------------------------------------------------------------------------------------------
+def nm_kept_positions(N: int, M: int):
+    """The n = C(M, N) patterns as tuples of kept positions, lexicographic."""
+    from itertools import combinations
+    return tuple(combinations(range(M), N))
+
+
+def nm_pattern_matrix(N: int, M: int) -> np.ndarray:
+    """D in {0,1}^{M x n} of Eq. 2 for N:M blocks: column p has ones at the kept positions of pattern p."""
+    pats = nm_kept_positions(N, M)
+    D = np.zeros((M, len(pats)), dtype=np.uint8)
+    for p, kept in enumerate(pats):
+        D[list(kept), p] = 1
+    return D
+
+
+def nm_select_from_logits(scores: np.ndarray) -> np.ndarray:
+    """Eq. 1 for any number of patterns: first maximum of each row of scores [G, n]."""
+    s = np.asarray(scores, dtype=np.float32)
+    best = np.zeros(s.shape[0], dtype=np.int64)
+    best_val = s[:, 0].copy()
+    for i in range(1, s.shape[1]):
+        better = s[:, i] > best_val
+        best[better] = i
+        best_val[better] = s[better, i]
+    return best.astype(np.uint8)
+
+
+def nm_select_from_magnitude(magnitudes: np.ndarray, N: int) -> np.ndarray:
+    """Keep the N largest of each block's M magnitudes (integers that order like |w|, [G, M]); equal
+    magnitudes keep the lower position first: a stable sort by decreasing magnitude, first N kept."""
+    a = np.asarray(magnitudes, dtype=np.int64)
+    M = a.shape[1]
+    order = np.argsort(-a, axis=1, kind="stable")
+    kept = np.sort(order[:, :N], axis=1)
+    lut = {pos: p for p, pos in enumerate(nm_kept_positions(N, M))}
+    return np.array([lut[tuple(int(v) for v in row)] for row in kept], dtype=np.uint8)
+
+
+def nm_mask_from_pattern(pattern: np.ndarray, N: int, M: int, shape) -> np.ndarray:
+    """Eq. 2 for N:M blocks: 0/1 mask of the given weight shape, blocks of M along the last axis."""
+    D = nm_pattern_matrix(N, M)
+    blocks = D[:, np.asarray(pattern, dtype=np.int64)].T  # [G, M]
+    return blocks.reshape(shape).astype(np.uint8)
