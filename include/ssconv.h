@@ -59,7 +59,8 @@ enum { SSCONV_FLAG_BIAS = 1u, SSCONV_FLAG_RELU = 2u, SSCONV_FLAG_GELU = 4u };
 
 enum {
   SSCONV_MASK_LOGITS_F32 = 0,    /* scores: float [G,6], one score per pattern            */
-  SSCONV_MASK_MAGNITUDE_BF16 = 1 /* scores: bf16 weights [C_out,KH,KW,C_in] = [G,4]       */
+  SSCONV_MASK_MAGNITUDE_BF16 = 1,/* scores: bf16 weights [C_out,KH,KW,C_in] = [G,4]       */
+  SSCONV_MASK_MAGNITUDE_E4M3 = 2 /* scores: e4m3 weights [C_out,KH,KW,C_in] = [G,4] (bytes; 4-byte aligned) */
 };
 
 /* Library version (major*10000 + minor*100 + patch). */
@@ -349,6 +350,36 @@ int32_t ssconv_absmax(const void* x_bf16, int64_t n, float* out, void* stream);
 enum { SSCONV_LEMMA_PERTURBATION = 34, SSCONV_LEMMA_ANY_MASK = 35, SSCONV_LEMMA_MASKED_UPDATE = 36 };
 double ssconv_stability_threshold(int32_t lemma, double L, const double* layer_norms, int32_t depth,
                                   int32_t j, double extra_norm, double x_norm);
+
+/* ---- 8-bit (e4m3) operands.  The paper's method is stated for any operand type the 2:4 hardware
+ * operation supports (Sec. 2: the sparse operation halves storage and time; Sec. 3.1 defines the
+ * N:M masks on the weight matrix regardless of its number format); these calls run Eq. 6 / Eq. 4
+ * with activations and weights in the 8-bit floating-point format e4m3 (1 sign, 4 exponent bits of
+ * bias 7, 3 mantissa bits, no infinities, largest magnitude 448), fp32 accumulation and bf16
+ * output:   y = act( bias + out_scale * sum x_q * (M .* W)_q ),
+ * where x_q, W_q are the values the codes stand for and out_scale (> 0) undoes whatever scales the
+ * caller applied when quantising (ssconv_quantize_e4m3).  Layouts as for bf16 with one byte per
+ * element; C_in % 16 == 0; no residual form, no K split (no workspace), one-block tiles only. */
+
+/* y[i] = the e4m3 value nearest to x[i] * scale (the product rounded to fp32 first; ties to the even
+ * mantissa; magnitudes beyond 448 saturate to 448; the sign is kept).  x: bf16, 4-byte aligned;
+ * y: bytes, 2-byte aligned; n even. */
+int32_t ssconv_quantize_e4m3(const void* x_bf16, void* y_e4m3, int64_t n, float scale, void* stream);
+
+/* ssconv_sizes / ssconv_compress / ssconv_decompress for e4m3 weights [C_out,KH,KW,C_in] (bytes).
+ * The blobs differ from the bf16 ones (k-blocks of 128 channels, one byte per kept value, twice the
+ * metadata per pair of k-blocks) and only ssconv_forward_fp8 / ssconv_decompress_fp8 read them. */
+int32_t ssconv_sizes_fp8(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes, size_t* meta_bytes);
+int32_t ssconv_compress_fp8(const ssconv_desc_t* desc, const void* w_e4m3, const uint8_t* pattern, void* w_comp,
+                            void* meta, void* stream);
+int32_t ssconv_decompress_fp8(const ssconv_desc_t* desc, const void* w_comp, const void* meta, void* w_masked_e4m3,
+                              uint8_t* pattern_out, void* stream);
+
+/* The masked convolution on e4m3 operands (sparse tcgen05.mma kind::f8f6f4) and its dense counterpart. */
+int32_t ssconv_forward_fp8(const ssconv_desc_t* desc, const void* x_e4m3, const void* w_comp, const void* meta,
+                           const float* bias, float out_scale, void* y, int32_t* dev_status, void* stream);
+int32_t ssconv_forward_dense_fp8(const ssconv_desc_t* desc, const void* x_e4m3, const void* w_e4m3, const float* bias,
+                                 float out_scale, void* y, int32_t* dev_status, void* stream);
 
 /* ssconv_forward_dense on a strided view of the input: pixel (n, h, w) of the H x W x C_in input the
  * descriptor names starts stride_n*n + stride_h*h + stride_w*w elements into x.  The strides are

@@ -18,6 +18,7 @@ FLAG_RELU = 2
 FLAG_GELU = 4
 MASK_LOGITS_F32 = 0
 MASK_MAGNITUDE_BF16 = 1
+MASK_MAGNITUDE_E4M3 = 2
 OK = 0
 ERR_TIMEOUT = 8
 
@@ -28,7 +29,9 @@ EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssc
            "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_pad_channels", "ssconv_space_to_depth", "ssconv_unfold_w", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense", "ssconv_forward_dense_strided",
            "ssconv_mask_norms", "ssconv_absmax", "ssconv_stability_threshold", "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_dgrad_prepare", "ssconv_dgrad_spread", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
-           "ssconv_forward_static_ws")
+           "ssconv_forward_static_ws",
+           "ssconv_quantize_e4m3", "ssconv_sizes_fp8", "ssconv_compress_fp8", "ssconv_decompress_fp8",
+           "ssconv_forward_fp8", "ssconv_forward_dense_fp8")
 
 
 class SsconvError(RuntimeError):
@@ -390,6 +393,88 @@ def ssconv_forward_static_ws(desc: Desc, x: torch.Tensor, w_comp: torch.Tensor, 
     _check("ssconv_forward_static_ws", lib().ssconv_forward_static_ws(
         ctypes.byref(desc), _ptr(x), _ptr(w_comp), _ptr(meta), _ptr(bias), _ptr(y), _ptr(dev_status),
         _stream(stream)))
+    return y
+
+
+# ----------------------------------------------------------------------------- 8-bit (e4m3) operands
+def ssconv_quantize_e4m3(x: torch.Tensor, scale: float = 1.0, y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """uint8 e4m3 codes of x * scale (x bf16, an even number of elements), nearest even, saturating."""
+    _need_cuda(x, y)
+    assert x.dtype == torch.bfloat16
+    if y is None:
+        y = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+    f = lib().ssconv_quantize_e4m3
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_float, ctypes.c_void_p]
+    _check("ssconv_quantize_e4m3", f(_ptr(x), _ptr(y), x.numel(), float(scale), _stream(stream)))
+    return y
+
+
+def ssconv_sizes_fp8(desc: Desc):
+    """(G, w_comp_bytes, meta_bytes) of the e4m3 blobs."""
+    G = ctypes.c_int64()
+    a, b = ctypes.c_size_t(), ctypes.c_size_t()
+    f = lib().ssconv_sizes_fp8
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_size_t),
+                  ctypes.POINTER(ctypes.c_size_t)]
+    _check("ssconv_sizes_fp8", f(ctypes.byref(desc), ctypes.byref(G), ctypes.byref(a), ctypes.byref(b)))
+    return int(G.value), int(a.value), int(b.value)
+
+
+def ssconv_compress_fp8(desc: Desc, w: torch.Tensor, pattern: torch.Tensor, stream=None):
+    """(w_comp, meta) uint8 blobs from e4m3 weights [C_out,KH,KW,C_in] (uint8) and pattern [G]."""
+    _need_cuda(w, pattern)
+    _, nv, nm = ssconv_sizes_fp8(desc)
+    w_comp = torch.empty((nv,), dtype=torch.uint8, device=w.device)
+    meta = torch.empty((nm,), dtype=torch.uint8, device=w.device)
+    f = lib().ssconv_compress_fp8
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc)] + [ctypes.c_void_p] * 5
+    _check("ssconv_compress_fp8", f(ctypes.byref(desc), _ptr(w), _ptr(pattern), _ptr(w_comp), _ptr(meta), _stream(stream)))
+    return w_comp, meta
+
+
+def ssconv_decompress_fp8(desc: Desc, w_comp: torch.Tensor, meta: torch.Tensor, stream=None):
+    """(w_masked uint8 e4m3 [C_out,KH,KW,C_in], pattern uint8 [G]) read back from the e4m3 blobs."""
+    _need_cuda(w_comp, meta)
+    G, _, _ = ssconv_sizes_fp8(desc)
+    w_out = torch.empty((desc.C_out, desc.KH, desc.KW, desc.C_in), dtype=torch.uint8, device=w_comp.device)
+    pat = torch.empty((G,), dtype=torch.uint8, device=w_comp.device)
+    f = lib().ssconv_decompress_fp8
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc)] + [ctypes.c_void_p] * 5
+    _check("ssconv_decompress_fp8", f(ctypes.byref(desc), _ptr(w_comp), _ptr(meta), _ptr(w_out), _ptr(pat), _stream(stream)))
+    return w_out, pat
+
+
+def ssconv_forward_fp8(desc: Desc, x: torch.Tensor, w_comp: torch.Tensor, meta: torch.Tensor,
+                       bias: Optional[torch.Tensor] = None, out_scale: float = 1.0, y: Optional[torch.Tensor] = None,
+                       dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """2:4 masked convolution on e4m3 activations (uint8 NHWC) and compressed e4m3 weights; bf16 output."""
+    _need_cuda(x, w_comp, meta, bias, y, dev_status)
+    if y is None:
+        y = _alloc_y(desc, x)
+    f = lib().ssconv_forward_fp8
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc)] + [ctypes.c_void_p] * 4 + [ctypes.c_float] + [ctypes.c_void_p] * 3
+    _check("ssconv_forward_fp8", f(ctypes.byref(desc), _ptr(x), _ptr(w_comp), _ptr(meta), _ptr(bias), float(out_scale),
+                                   _ptr(y), _ptr(dev_status), _stream(stream)))
+    return y
+
+
+def ssconv_forward_dense_fp8(desc: Desc, x: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor] = None,
+                             out_scale: float = 1.0, y: Optional[torch.Tensor] = None,
+                             dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Dense counterpart on e4m3 weights [C_out,KH,KW,C_in] (uint8)."""
+    _need_cuda(x, w, bias, y, dev_status)
+    if y is None:
+        y = _alloc_y(desc, x)
+    f = lib().ssconv_forward_dense_fp8
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc)] + [ctypes.c_void_p] * 3 + [ctypes.c_float] + [ctypes.c_void_p] * 3
+    _check("ssconv_forward_dense_fp8", f(ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), float(out_scale), _ptr(y),
+                                         _ptr(dev_status), _stream(stream)))
     return y
 
 

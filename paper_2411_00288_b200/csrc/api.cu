@@ -22,6 +22,13 @@ cudaError_t launch_space_to_depth(const void* x, void* y, int N, int H, int W, i
 int32_t plan_query_sms(const ssconv_desc_t& d, bool sparse, int sm_count, int32_t* bn, int32_t* split, int32_t* ctas,
                        int32_t* ring_groups, int32_t* pair);
 cudaError_t launch_wait_timeout_selftest(long long limit_cycles, int32_t* dev_status, cudaStream_t st);
+int32_t launch_forward_fp8(const ssconv_desc_t& d, bool sparse, const void* x, const void* weights, const void* meta,
+                           const float* bias, float out_scale, void* y, int32_t* dev_status, cudaStream_t stream);
+cudaError_t launch_quantize_e4m3(const void* x, void* y, int64_t n, float scale, cudaStream_t st);
+cudaError_t launch_compress_e4m3(const ssconv_desc_t& d, const void* w, const uint8_t* pattern, void* w_comp, void* meta,
+                                 cudaStream_t st);
+cudaError_t launch_decompress_e4m3(const ssconv_desc_t& d, const void* w_comp, const void* meta, void* w_out,
+                                   uint8_t* pattern_out, cudaStream_t st);
 size_t workspace_bytes();
 int32_t set_tuning(int32_t option, int32_t value);
 cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad,
@@ -170,11 +177,12 @@ int32_t ssconv_selftest_wait_timeout(int64_t limit_cycles, int32_t* dev_status, 
 int32_t ssconv_tune(int32_t option, int32_t value) { return ssconv::set_tuning(option, value); }
 
 int32_t ssconv_select_mask(int32_t mode, const void* scores, int64_t G, uint8_t* pattern, void* stream) {
-  if (mode != SSCONV_MASK_LOGITS_F32 && mode != SSCONV_MASK_MAGNITUDE_BF16) return SSCONV_ERR_BAD_DESC;
+  if (mode != SSCONV_MASK_LOGITS_F32 && mode != SSCONV_MASK_MAGNITUDE_BF16 && mode != SSCONV_MASK_MAGNITUDE_E4M3)
+    return SSCONV_ERR_BAD_DESC;
   if (G < 0) return SSCONV_ERR_BAD_DESC;
   if (G == 0) return SSCONV_OK;
   if (!scores || !pattern) return SSCONV_ERR_NULL;
-  if (reinterpret_cast<uintptr_t>(scores) & 7u) return SSCONV_ERR_ALIGNMENT;
+  if (reinterpret_cast<uintptr_t>(scores) & (mode == SSCONV_MASK_MAGNITUDE_E4M3 ? 3u : 7u)) return SSCONV_ERR_ALIGNMENT;
   return ssconv::launch_select(mode, scores, G, pattern, (cudaStream_t)stream) == cudaSuccess ? SSCONV_OK
                                                                                               : SSCONV_ERR_CUDA;
 }
@@ -306,6 +314,82 @@ int32_t ssconv_space_to_depth(const void* x, void* y, int32_t N, int32_t H, int3
   return ssconv::launch_space_to_depth(x, y, N, H, W, C, block, pad, Hb, Wb, C_pad, (cudaStream_t)stream) == cudaSuccess
              ? SSCONV_OK
              : SSCONV_ERR_CUDA;
+}
+
+// Shape rules of the 8-bit entry points on top of check_desc: rows of 16 bytes for the copies.
+static int32_t check_fp8(const ssconv_desc_t* desc, float out_scale) {
+  int32_t rc = check_desc(desc, true);
+  if (rc != SSCONV_OK) return rc;
+  if (desc->C_in % 16 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if (!(out_scale > 0.0f) || !(out_scale < 3.0e38f)) return SSCONV_ERR_BAD_DESC;
+  return SSCONV_OK;
+}
+
+int32_t ssconv_quantize_e4m3(const void* x_bf16, void* y_e4m3, int64_t n, float scale, void* stream) {
+  if (n < 0 || n % 2 != 0 || !(scale > 0.0f) || !(scale < 3.0e38f)) return SSCONV_ERR_BAD_DESC;
+  if (n == 0) return SSCONV_OK;
+  if (!x_bf16 || !y_e4m3) return SSCONV_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(x_bf16) & 3u) || (reinterpret_cast<uintptr_t>(y_e4m3) & 1u)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_quantize_e4m3(x_bf16, y_e4m3, n, scale, (cudaStream_t)stream) == cudaSuccess ? SSCONV_OK
+                                                                                                      : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_sizes_fp8(const ssconv_desc_t* desc, int64_t* G, size_t* w_comp_bytes, size_t* meta_bytes) {
+  int32_t rc = check_desc(desc, false);
+  if (rc != SSCONV_OK) return rc;
+  if (desc->C_in % 16 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  Geometry geo = make_geometry(*desc, 128);
+  if (G) *G = (int64_t)desc->C_out * geo.taps * (desc->C_in / 4);
+  if (w_comp_bytes) *w_comp_bytes = (size_t)geo.Mp * geo.kblocks_pad * 64;
+  if (meta_bytes) *meta_bytes = (size_t)geo.m_tiles * geo.stages * 2 * ssconv::kMetaImageBytes;
+  return SSCONV_OK;
+}
+
+int32_t ssconv_compress_fp8(const ssconv_desc_t* desc, const void* w_e4m3, const uint8_t* pattern, void* w_comp,
+                            void* meta, void* stream) {
+  int32_t rc = check_desc(desc, false);
+  if (rc != SSCONV_OK) return rc;
+  if (desc->C_in % 16 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if (!w_e4m3 || !pattern || !w_comp || !meta) return SSCONV_ERR_NULL;
+  if (!aligned16(w_e4m3) || !aligned16(w_comp) || !aligned16(meta)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_compress_e4m3(*desc, w_e4m3, pattern, w_comp, meta, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_decompress_fp8(const ssconv_desc_t* desc, const void* w_comp, const void* meta, void* w_masked_e4m3,
+                              uint8_t* pattern_out, void* stream) {
+  int32_t rc = check_desc(desc, false);
+  if (rc != SSCONV_OK) return rc;
+  if (desc->C_in % 16 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if (!w_comp || !meta || !w_masked_e4m3) return SSCONV_ERR_NULL;
+  if (!aligned16(w_comp) || !aligned16(meta) || !aligned16(w_masked_e4m3)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_decompress_e4m3(*desc, w_comp, meta, w_masked_e4m3, pattern_out, (cudaStream_t)stream) ==
+                 cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_forward_fp8(const ssconv_desc_t* desc, const void* x_e4m3, const void* w_comp, const void* meta,
+                           const float* bias, float out_scale, void* y, int32_t* dev_status, void* stream) {
+  int32_t rc = check_fp8(desc, out_scale);
+  if (rc != SSCONV_OK) return rc;
+  if (!x_e4m3 || !w_comp || !meta || !y) return SSCONV_ERR_NULL;
+  if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
+  if (!aligned16(x_e4m3) || !aligned16(w_comp) || !aligned16(meta) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_forward_fp8(*desc, true, x_e4m3, w_comp, meta, bias, out_scale, y, dev_status,
+                                    (cudaStream_t)stream);
+}
+
+int32_t ssconv_forward_dense_fp8(const ssconv_desc_t* desc, const void* x_e4m3, const void* w_e4m3, const float* bias,
+                                 float out_scale, void* y, int32_t* dev_status, void* stream) {
+  int32_t rc = check_fp8(desc, out_scale);
+  if (rc != SSCONV_OK) return rc;
+  if (!x_e4m3 || !w_e4m3 || !y) return SSCONV_ERR_NULL;
+  if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
+  if (!aligned16(x_e4m3) || !aligned16(w_e4m3) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_forward_fp8(*desc, false, x_e4m3, w_e4m3, nullptr, bias, out_scale, y, dev_status,
+                                    (cudaStream_t)stream);
 }
 
 int32_t ssconv_forward_dense_res(const ssconv_desc_t* desc, const void* x, const void* w_bf16, const float* bias,

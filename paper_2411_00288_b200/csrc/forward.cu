@@ -77,9 +77,14 @@ constexpr uint32_t kBarrierBytes = 256;
 // spans both k-blocks, + its metadata image; dense: two tiles), then the two activation tiles of
 // BN x 128 B.  One full and one empty barrier per group: the issuing thread pays about 200 cycles
 // per wait and 80 per tcgen05 instruction, so the handshake is per pair of k-blocks, not per k-block.
-template <bool SPARSE>
+// FP8: e4m3 operands (tcgen05 kind::f8f6f4).  A 128-byte row then holds 128 channels, so a k-block is
+// 128 channels of one tap; in bytes every tile is what it is for bf16, only the metadata of a 2:4 group
+// of two k-blocks doubles (512 dense columns instead of 256: two images of 2048 bytes).
+template <bool SPARSE, bool FP8 = false>
 struct Cfg {
-  static constexpr uint32_t kAGroupBytes = SPARSE ? kATileBytes + (uint32_t)kMetaImageBytes : 2 * kATileBytes;
+  static constexpr uint32_t kMetaBytes = (FP8 ? 2u : 1u) * (uint32_t)kMetaImageBytes;
+  static constexpr uint32_t kAGroupBytes = SPARSE ? kATileBytes + kMetaBytes : 2 * kATileBytes;
+  static constexpr int kKbChannels = FP8 ? 2 * kBlockK : kBlockK;  // input channels per k-block
 };
 constexpr int kMaxGroups = 4;                  // groups in the ring: as many as fit, 2 to 4
 constexpr uint32_t kMaxSmemBytes = 232448;     // 227 KB per CTA
@@ -104,6 +109,7 @@ struct FwdParams {
   int a_tiles;              // pairs of k-blocks (groups) per output tile
   int split;                // 1: units dealt out evenly across CTAs (stream-K); 0: whole tiles per CTA
   int work_quot, work_rem;  // work items per CTA: quotient and remainder of (tiles or units) / grid
+  float out_scale;          // 8-bit operands: factor applied to the accumulators before the bias
   float4* ws_regions;       // [2 * gridDim.x] regions of 128 x 240 fp32: a CTA's partial tiles
   uint32_t flags;
   const float* bias;
@@ -295,11 +301,12 @@ struct TapIter {
 // weights (with their metadata).  A TMA instruction occupies its issuing thread for a few hundred
 // cycles, so one thread issuing everything cannot keep up with the tensor pipe; three can.
 constexpr int kRoleActFirst = 0, kRoleActSecond = 1, kRoleWeights = 2;
-template <bool SPARSE, int ROLE>
+template <bool SPARSE, int ROLE, bool FP8 = false>
 __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUtensorMap* tm_b, const FwdParams& p,
                                               uint32_t full0, uint32_t empty0, uint32_t ring0,
                                               volatile int* abort_flag) {
-  using C = Cfg<SPARSE>;
+  using C = Cfg<SPARSE, FP8>;
+  constexpr int kKb = C::kKbChannels;
   const uint32_t b_bytes = (uint32_t)p.BN * 128u;  // one activation tile: BN positions x 64 channels
   const uint32_t grp_bytes = group_bytes(C::kAGroupBytes, p.BN);
   uint32_t g = 0, ph = 0;  // group slot and its phase parity
@@ -313,7 +320,7 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
     const Pos q0 = decode_pos(pt * p.BN, p.Wo, p.Ho);
     const int base_w = q0.c * p.stride_w - p.pad_w;
     const int base_h = q0.r * p.stride_h - p.pad_h;
-    const uint8_t* meta_src = p.meta + ((size_t)m * p.a_tiles + seg.a0) * kMetaImageBytes;
+    const uint8_t* meta_src = p.meta + ((size_t)m * p.a_tiles + seg.a0) * C::kMetaBytes;
     TapIter it;
     it.init(2 * seg.a0 + (ROLE == kRoleActSecond ? 1 : 0), p);
     if (first_segment) {
@@ -345,7 +352,7 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
         } else if (ROLE == kRoleWeights) {
           mbar_expect_tx_w(full, (uint32_t)chunks * 2048u);
           for (int j = 0; j < chunks; ++j) {  // chunks 8.. belong to the second k-block: 16 KB further on = 8 x 2048
-            tma_load_3d_w(dst + (uint32_t)j * 2048u, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+            tma_load_3d_w(dst + (uint32_t)j * 2048u, tm_a, full, it.cc * kKb, it.tap, m * kTileM);
             it.advance(p);
           }
         } else {
@@ -353,7 +360,7 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
           mbar_expect_tx_w(full, (uint32_t)chunks * chunk_bytes);
           const uint32_t b_dst = dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? b_bytes : 0u);
           for (int j = 0; j < chunks; ++j) {
-            tma_load_im2col_4d_w(b_dst + (uint32_t)j * chunk_bytes, tm_b, full, it.cc * kBlockK, base_w, base_h,
+            tma_load_im2col_4d_w(b_dst + (uint32_t)j * chunk_bytes, tm_b, full, it.cc * kKb, base_w, base_h,
                                  q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
             it.advance(p);
           }
@@ -361,20 +368,20 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
       } else if (ROLE == kRoleWeights) {
         if (SPARSE) {
           mbar_expect_tx_w(full, C::kAGroupBytes);
-          tma_load_2d_w(dst, tm_a, full, a * 64, m * kTileM);
-          bulk_load_w(dst + kATileBytes, meta_src, kMetaImageBytes, full);
-          meta_src += kMetaImageBytes;
+          tma_load_2d_w(dst, tm_a, full, a * (FP8 ? 128 : 64), m * kTileM);  // 128 bytes of kept values per group
+          bulk_load_w(dst + kATileBytes, meta_src, C::kMetaBytes, full);
+          meta_src += C::kMetaBytes;
         } else {
           mbar_expect_tx_w(full, has_second ? 2 * kATileBytes : kATileBytes);
-          tma_load_3d_w(dst, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+          tma_load_3d_w(dst, tm_a, full, it.cc * kKb, it.tap, m * kTileM);
           it.advance(p);
-          if (has_second) tma_load_3d_w(dst + kATileBytes, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+          if (has_second) tma_load_3d_w(dst + kATileBytes, tm_a, full, it.cc * kKb, it.tap, m * kTileM);
           it.advance(p);
         }
       } else if (ROLE == kRoleActFirst || has_second) {
         mbar_expect_tx_w(full, b_bytes);
         tma_load_im2col_4d_w(dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? b_bytes : 0u), tm_b, full,
-                             it.cc * kBlockK, base_w, base_h, q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
+                             it.cc * kKb, base_w, base_h, q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
         it.advance(p);
         it.advance(p);
       } else {
@@ -390,13 +397,14 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
 
 // RES: a residual tensor is added in the epilogue (its own instantiation, so that the plain kernel's
 // epilogue loop carries none of that code).
-template <bool SPARSE, bool RES>
+template <bool SPARSE, bool RES, bool FP8 = false>
 __global__ void __launch_bounds__(kThreads, 1)
 ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                   const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_y_tail,
                   const __grid_constant__ CUtensorMap tm_r, const __grid_constant__ CUtensorMap tm_r_tail,
                   const FwdParams p) {
-  using C = Cfg<SPARSE>;
+  using C = Cfg<SPARSE, FP8>;
+  static_assert(!(FP8 && RES), "the residual epilogue is not built for 8-bit operands");
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -470,19 +478,21 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     {
       const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty), ring0 = smem_u32(ring);
       if (warp == 0)
-        producer_role<SPARSE, kRoleActFirst>(&tm_a, &tm_b, p, full0,
+        producer_role<SPARSE, kRoleActFirst, FP8>(&tm_a, &tm_b, p, full0,
                                              p.ring_groups == 2 ? smem_u32(bar_empty_first) : empty0, ring0, abort_flag);
       else if (warp == kFirstExtraProducerWarp)
-        producer_role<SPARSE, kRoleActSecond>(&tm_a, &tm_b, p, full0, empty0, ring0, abort_flag);
+        producer_role<SPARSE, kRoleActSecond, FP8>(&tm_a, &tm_b, p, full0, empty0, ring0, abort_flag);
       else
-        producer_role<SPARSE, kRoleWeights>(&tm_a, &tm_b, p, full0, empty0, ring0, abort_flag);
+        producer_role<SPARSE, kRoleWeights, FP8>(&tm_a, &tm_b, p, full0, empty0, ring0, abort_flag);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     // All 32 lanes run this loop in lock step and wait on the barriers together; the tcgen05
     // instructions are issued by one elected lane (see the warp-wide forms in sm100_ptx.cuh).
     {
-      const uint32_t idesc = make_idesc_bf16(kTileM, (uint32_t)p.BN, SPARSE);
+      const uint32_t idesc = FP8 ? make_idesc_e4m3(kTileM, (uint32_t)p.BN, SPARSE)
+                                 : make_idesc_bf16(kTileM, (uint32_t)p.BN, SPARSE);
+      constexpr int kKb = C::kKbChannels;
       // descriptor address units are 16 B
       const uint32_t grp_desc = group_bytes(C::kAGroupBytes, p.BN) >> 4;
       const uint32_t b_desc = ((uint32_t)p.BN * 128u) >> 4;
@@ -494,10 +504,11 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       const bool early_release = p.ring_groups == 2;
       const uint32_t meta_tmem0 = tmem_base + kMetaCol;
       // channels left in the last chunk decide how many MMAs its k-blocks need
-      const int tail_c = p.C_in - (p.cblocks - 1) * kBlockK;
+      const int tail_c = p.C_in - (p.cblocks - 1) * kKb;
       const int mma_full = SPARSE ? 2 : 4;
-      const int mma_tail = SPARSE ? ((tail_c + 31) >> 5) : ((tail_c + 15) >> 4);
-      const int tail_start = (tail_c == kBlockK) ? p.kblocks : (p.cblocks - 1) * p.taps;  // first k-block of the tail
+      // channels per MMA: bf16 32 sparse / 16 dense, e4m3 64 / 32
+      const int mma_tail = SPARSE ? ((tail_c + kKb / 2 - 1) / (kKb / 2)) : ((tail_c + kKb / 4 - 1) / (kKb / 4));
+      const int tail_start = (tail_c == kKb) ? p.kblocks : (p.cblocks - 1) * p.taps;  // first k-block of the tail
       const int a_lean_end = tail_start >> 1;  // groups before this one hold two full k-blocks
       uint32_t g = 0, ph = 0;  // group slot and its phase parity
       uint32_t tcount = 0;
@@ -523,7 +534,21 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             const uint32_t a_lo = ring_lo0 + g * grp_desc;
             const uint32_t b0_lo = a_lo + (C::kAGroupBytes >> 4);
             const uint32_t b1_lo = b0_lo + b_desc;
-            if (SPARSE) {
+            if (SPARSE && FP8) {
+              // two metadata images -> 8 TMEM columns: 2 per MMA of 64 dense columns; operand steps in
+              // bytes as for bf16 (A 32 kept bytes, B 64 bytes per MMA)
+              const uint32_t meta_tmem = meta_tmem0 + 8u * mslot;
+              mslot ^= 1u;
+              tc_cp_128x128b_w(meta_tmem, a_lo + (kATileBytes >> 4));
+              tc_cp_128x128b_w(meta_tmem + 4u, a_lo + ((kATileBytes + (uint32_t)kMetaImageBytes) >> 4));
+              const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
+              const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
+              tc_mma_f8_sparse_w(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
+              if (n0 > 1) tc_mma_f8_sparse_w(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem + 2u, idesc, 1u);
+              if (kEarly) tc_commit_w(empty_first0 + 8u * g);
+              if (n1 > 0) tc_mma_f8_sparse_w(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 4u, idesc, 1u);
+              if (n1 > 1) tc_mma_f8_sparse_w(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 6u, idesc, 1u);
+            } else if (SPARSE) {
               // metadata image -> 4 TMEM columns: 2 per k-block.  Kept values of the second k-block
               // start 64 B into the tile's rows; per MMA A advances 16 kept values = 32 B, B 32
               // channels = 64 B (descriptor units of 16 B).
@@ -563,6 +588,14 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                 }
                 if (kEarly && kb == 0) tc_commit_w(empty_first0 + 8u * g);
               }
+            } else if (FP8) {
+              const uint32_t a1_lo = a_lo + (kATileBytes >> 4);
+              const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
+              const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
+              for (int kk = 0; kk < n0; ++kk)
+                tc_mma_f8_dense_w(d_tmem, a_lo + 2u * kk, b0_lo + 2u * kk, idesc, (kk > 0) ? 1u : accumulate);
+              if (kEarly) tc_commit_w(empty_first0 + 8u * g);
+              for (int kk = 0; kk < n1; ++kk) tc_mma_f8_dense_w(d_tmem, a1_lo + 2u * kk, b1_lo + 2u * kk, idesc, 1u);
             } else {
               const uint32_t a1_lo = a_lo + (kATileBytes >> 4);
               if (a < a_lean_end) {
@@ -707,6 +740,10 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         // The buffer was last the source of the store issued two pieces ago; the leader saw that
         // store finish reading before it entered the barrier of the previous piece.
         const uint32_t st_addr = smem_u32(stage) + st_offset;
+        if (FP8) {  // the accumulators are sums of products of quantised values: undo the operands' scales
+#pragma unroll
+          for (int i = 0; i < kPiece; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * p.out_scale);
+        }
         if (RES) {
           // the residual piece has landed in this buffer (a wait that runs out raises the abort flag;
           // the group still goes on to its barrier and stops at the next tile)
@@ -1397,12 +1434,13 @@ size_t workspace_bytes() { return scratch_bytes(kMaxWorkers); }
 static int g_sm_count[64] = {0};
 static bool g_attr_set[64][2][2] = {{{false}}};
 static bool g_pair_attr_set[64][2] = {{false}};
+static bool g_fp8_attr_set[64][2] = {{false}};
 
 // Dense layers with 8 input channels (a channel-padded RGB stem): a k-block of 64 K-elements is 8
 // filter taps instead of 64 channels of one tap, which would be 7/8 padding.
 static bool small_channel_mode(const ssconv_desc_t& d, bool sparse) { return !sparse && d.C_in == 8; }
-static Geometry layer_geometry(const ssconv_desc_t& d, bool sparse) {
-  Geometry g = make_geometry(d);
+static Geometry layer_geometry(const ssconv_desc_t& d, bool sparse, bool fp8 = false) {
+  Geometry g = make_geometry(d, fp8 ? 2 * kBlockK : kBlockK);
   if (small_channel_mode(d, sparse)) {
     g.kblocks = (g.taps + 7) / 8;
     g.kblocks_pad = (g.kblocks + 1) & ~1;
@@ -1484,12 +1522,17 @@ int32_t plan_query_sms(const ssconv_desc_t& d, bool sparse, int sm_count, int32_
   return SSCONV_OK;
 }
 
-template <bool SPARSE>
+template <bool SPARSE, bool FP8 = false>
 static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const void* weights, const void* meta,
                                    const float* bias, const void* residual, void* y, void* ws, size_t ws_bytes,
                                    int32_t* dev_status, cudaStream_t stream, int worker_cap = kMaxWorkers,
-                                   bool force_split = false, const int64_t* x_strides = nullptr) {
-  using C = Cfg<SPARSE>;
+                                   bool force_split = false, const int64_t* x_strides = nullptr,
+                                   float out_scale = 1.0f) {
+  using C = Cfg<SPARSE, FP8>;
+  constexpr int kKb = C::kKbChannels;
+  constexpr size_t kElem = FP8 ? 1 : 2;  // bytes per operand element
+  constexpr CUtensorMapDataType kOperandType = FP8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  if (FP8 && residual != nullptr) return SSCONV_ERR_UNSUPPORTED_SHAPE;
   if (!load_driver_entry_points()) return SSCONV_ERR_CUDA;
   int dev = 0;
   {
@@ -1505,8 +1548,14 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     if (e != cudaSuccess) return SSCONV_ERR_CUDA;
     g_attr_set[dev][SPARSE ? 1 : 0][res] = true;
   }
-  const Geometry geo = layer_geometry(d, SPARSE);
-  const bool small_c = small_channel_mode(d, SPARSE);
+  if (FP8 && !g_fp8_attr_set[dev][SPARSE ? 1 : 0]) {
+    if (cudaFuncSetAttribute(ssconv_fwd_kernel<SPARSE, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kMaxSmemBytes) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
+    g_fp8_attr_set[dev][SPARSE ? 1 : 0] = true;
+  }
+  const Geometry geo = layer_geometry(d, SPARSE, FP8);
+  const bool small_c = !FP8 && small_channel_mode(d, SPARSE);
   const int Ho = out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h);
   const int Wo = out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
   const long long Q = (long long)d.N * Ho * Wo;  // positions
@@ -1518,11 +1567,11 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   // two buffers and one piece of lookahead for the whole tiles it may also own.)
   // Without a usable workspace the K range is not split: the best plan of whole tiles runs instead
   // (slower on layers with few tiles and a deep K, never wrong).
-  const bool have_ws = ws != nullptr && ws_bytes >= scratch_bytes(worker_cap);
+  const bool have_ws = !FP8 && ws != nullptr && ws_bytes >= scratch_bytes(worker_cap);  // (8-bit: whole tiles only)
   if (have_ws && (reinterpret_cast<uintptr_t>(ws) & 15u)) return SSCONV_ERR_ALIGNMENT;
   if (force_split && !have_ws) return SSCONV_ERR_WORKSPACE;
-  Plan plan = residual != nullptr ? plan_layer<SPARSE>(Q, geo, workers, force_split, kBN, 2, have_ws)
-                                  : choose_plan<SPARSE>(d, Q, geo, workers, force_split, have_ws);
+  Plan plan = (residual != nullptr || FP8) ? plan_layer<SPARSE>(Q, geo, workers, force_split, kBN, 2, have_ws)
+                                           : choose_plan<SPARSE>(d, Q, geo, workers, force_split, have_ws);
   int stage_bufs = 2;
   if (residual != nullptr && !plan.split) {
     stage_bufs = 4;
@@ -1551,19 +1600,19 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   // (= the zero padding of Eq. 4); base pixels are the filter placements, each load adds a tap offset
   {
     cuuint64_t dims[4] = {(cuuint64_t)d.C_in, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
-    cuuint64_t strides[3] = {(cuuint64_t)d.C_in * 2, (cuuint64_t)d.W * d.C_in * 2,
-                             (cuuint64_t)d.H * d.W * d.C_in * 2};
+    cuuint64_t strides[3] = {(cuuint64_t)d.C_in * kElem, (cuuint64_t)d.W * d.C_in * kElem,
+                             (cuuint64_t)d.H * d.W * d.C_in * kElem};
     if (x_strides != nullptr)  // a strided (possibly overlapping) view: element strides of w, h, n
-      for (int i = 0; i < 3; ++i) strides[i] = (cuuint64_t)x_strides[i] * 2;
+      for (int i = 0; i < 3; ++i) strides[i] = (cuuint64_t)x_strides[i] * kElem;
     int lower[2] = {-d.pad_w, -d.pad_h};
     int upper[2] = {d.pad_w - (d.KW - 1) * d.dil_w, d.pad_h - (d.KH - 1) * d.dil_h};
     cuuint32_t estr[4] = {1, (cuuint32_t)d.stride_w, (cuuint32_t)d.stride_h, 1};
     // (8-channel mode: 16-byte-wide unswizzled chunks, one per filter tap)
     // L2 fetches 256 bytes per miss where a pixel is at least that long and every pixel is read
     // (measured: up to 4 % faster on such layers, 4 % slower on a strided one, nothing elsewhere)
-    const bool wide_pixels = d.C_in >= 128 && d.stride_h == 1 && d.stride_w == 1 && x_strides == nullptr;
-    CUresult r = g_encode_im2col(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), dims, strides,
-                                 lower, upper, small_c ? 8u : (cuuint32_t)kBlockK,
+    const bool wide_pixels = d.C_in * kElem >= 256 && d.stride_h == 1 && d.stride_w == 1 && x_strides == nullptr;
+    CUresult r = g_encode_im2col(&tm_b, kOperandType, 4, const_cast<void*>(x), dims, strides,
+                                 lower, upper, small_c ? 8u : (cuuint32_t)kKb,
                                  (cuuint32_t)(pair ? BN / 2 : BN), estr,
                                  CU_TENSOR_MAP_INTERLEAVE_NONE,
                                  small_c ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
@@ -1572,11 +1621,12 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
   }
   if (SPARSE) {
-    cuuint64_t dims[2] = {(cuuint64_t)geo.KC, (cuuint64_t)geo.Mp};
+    // kept values: 64 bytes per row and k-block (KC counts 2-byte units); a box is 128 rows x 128 bytes
+    cuuint64_t dims[2] = {(cuuint64_t)geo.KC * 2 / kElem, (cuuint64_t)geo.Mp};
     cuuint64_t strides[1] = {(cuuint64_t)geo.KC * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kTileM};
+    cuuint32_t box[2] = {(cuuint32_t)(128 / kElem), (cuuint32_t)kTileM};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = g_encode_tiled(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(weights), dims, strides,
+    CUresult r = g_encode_tiled(&tm_a, kOperandType, 2, const_cast<void*>(weights), dims, strides,
                                 box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return SSCONV_ERR_CUDA;
@@ -1584,10 +1634,10 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     // dense weights [C_out][taps][C_in] seen as (c, tap, output channel); 8-channel mode: one tap's
     // 8 channels of 128 rows per load, unswizzled
     cuuint64_t dims[3] = {(cuuint64_t)d.C_in, (cuuint64_t)geo.taps, (cuuint64_t)d.C_out};
-    cuuint64_t strides[2] = {(cuuint64_t)d.C_in * 2, (cuuint64_t)geo.taps * d.C_in * 2};
-    cuuint32_t box[3] = {small_c ? 8u : (cuuint32_t)kBlockK, 1, (cuuint32_t)kTileM};
+    cuuint64_t strides[2] = {(cuuint64_t)d.C_in * kElem, (cuuint64_t)geo.taps * d.C_in * kElem};
+    cuuint32_t box[3] = {small_c ? 8u : (cuuint32_t)kKb, 1, (cuuint32_t)kTileM};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = g_encode_tiled(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(weights), dims, strides,
+    CUresult r = g_encode_tiled(&tm_a, kOperandType, 3, const_cast<void*>(weights), dims, strides,
                                 box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                 small_c ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -1672,6 +1722,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.meta = static_cast<const uint8_t*>(meta);
   p.y = static_cast<__nv_bfloat16*>(y);
   p.dev_status = dev_status;
+  p.out_scale = out_scale;
 
   const long long units = q_tiles * geo.m_tiles * geo.stages;
   if (units >= (1LL << 31)) return SSCONV_ERR_UNSUPPORTED_SHAPE;  // 32-bit work indices on the device
@@ -1712,7 +1763,8 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   cfg.attrs = attr;
   cfg.numAttrs = pair ? 2 : 1;
   const cudaError_t launched =
-      pair ? cudaLaunchKernelEx(&cfg, ssconv_fwd_pair_kernel<SPARSE>, tm_a, tm_b, tm_meta, tm_y, tm_y_tail, p)
+      FP8 ? cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, false, FP8>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p)
+      : pair ? cudaLaunchKernelEx(&cfg, ssconv_fwd_pair_kernel<SPARSE>, tm_a, tm_b, tm_meta, tm_y, tm_y_tail, p)
       : residual != nullptr
           ? cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, true>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p)
           : cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, false>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p);
@@ -1753,6 +1805,14 @@ int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* 
                              cudaStream_t stream, const int64_t* x_strides) {
   return launch_forward_impl<false>(d, x, w, nullptr, bias, residual, y, ws, ws_bytes, dev_status, stream, kMaxWorkers,
                                     false, x_strides);
+}
+
+int32_t launch_forward_fp8(const ssconv_desc_t& d, bool sparse, const void* x, const void* weights, const void* meta,
+                           const float* bias, float out_scale, void* y, int32_t* dev_status, cudaStream_t stream) {
+  return sparse ? launch_forward_impl<true, true>(d, x, weights, meta, bias, nullptr, y, nullptr, 0, dev_status, stream,
+                                                  kMaxWorkers, false, nullptr, out_scale)
+                : launch_forward_impl<false, true>(d, x, weights, nullptr, bias, nullptr, y, nullptr, 0, dev_status,
+                                                   stream, kMaxWorkers, false, nullptr, out_scale);
 }
 
 // ---------------------------------------------------------------------------------------

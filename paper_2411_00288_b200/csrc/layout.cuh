@@ -42,10 +42,13 @@ struct Geometry {
   int KC;            // 32*kblocks_pad: kept values per padded row
 };
 
-__host__ __device__ inline Geometry make_geometry(const ssconv_desc_t& d) {
+// kb_channels: input channels per k-block: 64 for bf16 (a 128-byte row of 16-bit elements), 128 for
+// 8-bit operands.  The byte sizes (KC kept values of 2 bytes, or 2 KC kept bytes... per row) work out
+// the same: 64 bytes of kept values per row and k-block either way.
+__host__ __device__ inline Geometry make_geometry(const ssconv_desc_t& d, int kb_channels = kBlockK) {
   Geometry g;
   g.taps = d.KH * d.KW;
-  g.cblocks = (d.C_in + kBlockK - 1) / kBlockK;
+  g.cblocks = (d.C_in + kb_channels - 1) / kb_channels;
   g.kblocks = g.taps * g.cblocks;
   g.kblocks_pad = (g.kblocks + 1) & ~1;
   g.stages = g.kblocks_pad / 2;

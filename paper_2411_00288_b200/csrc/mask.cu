@@ -34,8 +34,7 @@ __global__ void select_logits_kernel(const float2* __restrict__ scores, int64_t 
 // the 15-bit integers below the sign bit (monotone in |w|, +0 == -0); a position beats
 // another when it is larger, or equal and earlier, so exactly two positions are beaten by
 // fewer than two others.
-__device__ __forceinline__ uint32_t magnitude_pattern(uint32_t lo, uint32_t hi) {
-  uint32_t a[4] = {lo & 0x7FFFu, (lo >> 16) & 0x7FFFu, hi & 0x7FFFu, (hi >> 16) & 0x7FFFu};
+__device__ __forceinline__ uint32_t magnitude_pattern4(const uint32_t (&a)[4]) {
   int first = -1, second = -1;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -53,12 +52,118 @@ __device__ __forceinline__ uint32_t magnitude_pattern(uint32_t lo, uint32_t hi) 
   // {0,1}->0 {0,2}->1 {0,3}->2 {1,2}->3 {1,3}->4 {2,3}->5
   return (uint32_t)(first == 0 ? second - 1 : (first == 1 ? second + 1 : 5));
 }
+__device__ __forceinline__ uint32_t magnitude_pattern(uint32_t lo, uint32_t hi) {
+  const uint32_t a[4] = {lo & 0x7FFFu, (lo >> 16) & 0x7FFFu, hi & 0x7FFFu, (hi >> 16) & 0x7FFFu};
+  return magnitude_pattern4(a);
+}
 
 __global__ void select_magnitude_kernel(const uint2* __restrict__ w, int64_t G, uint8_t* __restrict__ pattern) {
   int64_t g = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
   if (g >= G) return;
   uint2 v = w[g];
   pattern[g] = (uint8_t)magnitude_pattern(v.x, v.y);
+}
+
+// The same for e4m3 weights: a group is four bytes, a magnitude the 7 bits below the sign bit.
+__global__ void select_magnitude_e4m3_kernel(const uint32_t* __restrict__ w, int64_t G, uint8_t* __restrict__ pattern) {
+  int64_t g = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (g >= G) return;
+  const uint32_t v = w[g];
+  const uint32_t a[4] = {v & 0x7Fu, (v >> 8) & 0x7Fu, (v >> 16) & 0x7Fu, (v >> 24) & 0x7Fu};
+  pattern[g] = (uint8_t)magnitude_pattern4(a);
+}
+
+// bf16 -> e4m3: y = nearest e4m3 value of x * scale (the product rounded to fp32 first), ties to even,
+// magnitudes beyond 448 saturate.  One thread per pair of elements.
+__global__ void quantize_e4m3_kernel(const uint32_t* __restrict__ x, uint16_t* __restrict__ y, int64_t pairs, float scale) {
+  int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= pairs) return;
+  const uint32_t v = x[i];
+  const float lo = __uint_as_float(v << 16) * scale, hi = __uint_as_float(v & 0xFFFF0000u) * scale;
+  uint16_t out;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(out) : "f"(hi), "f"(lo));
+  y[i] = out;
+}
+
+// ---------------------------------------------------------------------------------------
+// 8-bit (e4m3) weights: compress / decompress
+// ---------------------------------------------------------------------------------------
+// Geometry with k-blocks of 128 channels (make_geometry(d, 128)).  Value blob: bytes [Mp][64 * kblocks_pad]:
+// byte 64 b + 2 q + s holds kept value s (0 = lower position) of the q-th group of four channels of
+// k-block b.  Metadata: per (128-row tile, pair of k-blocks) two images of 2048 bytes, one per k-block,
+// each what one tcgen05.cp 128x128b moves into 4 TMEM columns: lane = row, its four words hold the 32
+// 4-bit codes of the row's groups in order (nibble n of word w = group 8 w + n); the sparse MMA over the
+// first 64 channels of a k-block reads the first two columns, the one over the second 64 the other two.
+// (Found by probing the instruction with an identity activation matrix and single flipped codes.)
+__global__ void compress_values_e4m3_kernel(ssconv_desc_t d, Geometry geo, const uint32_t* __restrict__ w,
+                                            const uint8_t* __restrict__ pattern, uint16_t* __restrict__ w_comp) {
+  int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  int64_t total = (int64_t)geo.Mp * geo.kblocks_pad * 32;
+  if (t >= total) return;
+  int q = (int)(t % 32);
+  int b = (int)((t / 32) % geo.kblocks_pad);
+  int co = (int)(t / (32 * (int64_t)geo.kblocks_pad));
+  uint32_t out = 0;
+  if (co < d.C_out && b < geo.kblocks) {
+    int tap = b % geo.taps;
+    int c = (b / geo.taps) * 128 + 4 * q;
+    if (c < d.C_in) {
+      int64_t g = ((int64_t)co * geo.taps + tap) * (d.C_in / 4) + c / 4;
+      uint32_t v = w[g];
+      uint32_t code = pattern_code(pattern[g]);
+      out = ((v >> (8 * (code & 3u))) & 0xFFu) | (((v >> (8 * ((code >> 2) & 3u))) & 0xFFu) << 8);
+    }
+  }
+  w_comp[(int64_t)co * (32 * geo.kblocks_pad) + 32 * b + q] = (uint16_t)out;
+}
+
+__global__ void compress_meta_e4m3_kernel(ssconv_desc_t d, Geometry geo, const uint8_t* __restrict__ pattern,
+                                          uint32_t* __restrict__ meta) {
+  // one thread per metadata word: (tile, stage, image i, lane L, word j)
+  int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  int64_t total = (int64_t)geo.m_tiles * geo.stages * 2 * 128 * 4;
+  if (t >= total) return;
+  int j = (int)(t % 4);
+  int L = (int)((t / 4) % 128);
+  int i = (int)((t / 512) % 2);
+  int s = (int)((t / 1024) % geo.stages);
+  int mt = (int)(t / (1024 * (int64_t)geo.stages));
+  int b = 2 * s + i;
+  int tap = b % geo.taps;
+  int co = mt * kTileM + L;
+  uint32_t word = 0;
+#pragma unroll
+  for (int n = 0; n < 8; ++n) {
+    int c = (b / geo.taps) * 128 + 4 * (8 * j + n);
+    uint32_t code = 0x4u;
+    if (co < d.C_out && b < geo.kblocks && c < d.C_in) {
+      int64_t g = ((int64_t)co * geo.taps + tap) * (d.C_in / 4) + c / 4;
+      code = pattern_code(pattern[g]);
+    }
+    word |= code << (4 * n);
+  }
+  meta[t] = word;
+}
+
+__global__ void decompress_e4m3_kernel(ssconv_desc_t d, Geometry geo, const uint16_t* __restrict__ w_comp,
+                                       const uint32_t* __restrict__ meta, uint32_t* __restrict__ w_out,
+                                       uint8_t* __restrict__ pattern_out) {
+  int64_t g = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  int groups_per_tap = d.C_in / 4;
+  int64_t G = (int64_t)d.C_out * geo.taps * groups_per_tap;
+  if (g >= G) return;
+  int c = (int)(g % groups_per_tap) * 4;
+  int tap = (int)((g / groups_per_tap) % geo.taps);
+  int co = (int)(g / ((int64_t)groups_per_tap * geo.taps));
+  int b = (c / 128) * geo.taps + tap;
+  int q = (c % 128) / 4;
+  int mt = co / kTileM, L = co % kTileM;
+  uint32_t word = meta[((((int64_t)mt * geo.stages + (b >> 1)) * 2 + (b & 1)) * 128 + L) * 4 + q / 8];
+  uint32_t code = (word >> (4 * (q % 8))) & 0xFu;
+  uint32_t pair = w_comp[(int64_t)co * (32 * geo.kblocks_pad) + 32 * b + q];
+  uint32_t out = ((pair & 0xFFu) << (8 * (code & 3u))) | ((pair >> 8) << (8 * ((code >> 2) & 3u)));
+  w_out[g] = out;
+  if (pattern_out) pattern_out[g] = (uint8_t)code_pattern(code);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -168,8 +273,44 @@ cudaError_t launch_select(int mode, const void* scores, int64_t G, uint8_t* patt
   count_launch();
   if (mode == SSCONV_MASK_LOGITS_F32)
     select_logits_kernel<<<blocks_for(G, T), T, 0, st>>>((const float2*)scores, G, pattern);
+  else if (mode == SSCONV_MASK_MAGNITUDE_E4M3)
+    select_magnitude_e4m3_kernel<<<blocks_for(G, T), T, 0, st>>>((const uint32_t*)scores, G, pattern);
   else
     select_magnitude_kernel<<<blocks_for(G, T), T, 0, st>>>((const uint2*)scores, G, pattern);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_e4m3(const void* x, void* y, int64_t n, float scale, cudaStream_t st) {
+  const int T = 256;
+  if (n == 0) return cudaSuccess;
+  count_launch();
+  quantize_e4m3_kernel<<<blocks_for(n / 2, T), T, 0, st>>>((const uint32_t*)x, (uint16_t*)y, n / 2, scale);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_compress_e4m3(const ssconv_desc_t& d, const void* w, const uint8_t* pattern, void* w_comp, void* meta,
+                                 cudaStream_t st) {
+  Geometry geo = make_geometry(d, 128);
+  const int T = 256;
+  int64_t nv = (int64_t)geo.Mp * geo.kblocks_pad * 32;
+  count_launch();
+  compress_values_e4m3_kernel<<<blocks_for(nv, T), T, 0, st>>>(d, geo, (const uint32_t*)w, pattern, (uint16_t*)w_comp);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  int64_t nm = (int64_t)geo.m_tiles * geo.stages * 1024;
+  count_launch();
+  compress_meta_e4m3_kernel<<<blocks_for(nm, T), T, 0, st>>>(d, geo, pattern, (uint32_t*)meta);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decompress_e4m3(const ssconv_desc_t& d, const void* w_comp, const void* meta, void* w_out,
+                                   uint8_t* pattern_out, cudaStream_t st) {
+  Geometry geo = make_geometry(d, 128);
+  const int T = 256;
+  int64_t G = (int64_t)d.C_out * geo.taps * (d.C_in / 4);
+  count_launch();
+  decompress_e4m3_kernel<<<blocks_for(G, T), T, 0, st>>>(d, geo, (const uint16_t*)w_comp, (const uint32_t*)meta,
+                                                         (uint32_t*)w_out, pattern_out);
   return cudaGetLastError();
 }
 

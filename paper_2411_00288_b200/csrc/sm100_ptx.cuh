@@ -176,6 +176,12 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(uint32_t M, uint32_t N, b
   return (sparse ? (1u << 2) : 0u) | (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
+// Instruction descriptor of tcgen05.mma kind::f8f6f4 with e4m3 A and B (format code 0 in bits 7-9 and
+// 10-12; both K-major) and an fp32 accumulator; the other fields as above.
+__host__ __device__ constexpr uint32_t make_idesc_e4m3(uint32_t M, uint32_t N, bool sparse) {
+  return (sparse ? (1u << 2) : 0u) | (1u << 4) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
 // ---------------------------------------------------------------- tcgen05: mma / cp / ld
 
 // 16 lanes x 8N consecutive 32-bit columns in the layout of an MMA accumulator fragment: per
@@ -372,6 +378,33 @@ __device__ __forceinline__ void bulk_load_w(uint32_t dst, const void* gsrc, uint
       "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
       "@e cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n\t}"
       ::"r"(dst), "l"(gsrc), "r"(bytes), "r"(bar)
+      : "memory");
+}
+
+// 8-bit operands (kind::f8f6f4, here e4m3): a dense MMA covers K = 32 elements, a 2:4 sparse one K = 64
+// (A holds the 32 kept bytes per row); in bytes per row the operand steps are those of the 16-bit forms.
+__device__ __forceinline__ void tc_mma_f8_dense_w(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                                  uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, e;\n\t.reg .b64 da, db;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
+      "mov.b64 da, {%1, %5};\n\t"
+      "mov.b64 db, {%2, %5};\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHiSw128)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_f8_sparse_w(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t meta_tmem,
+                                                   uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, e;\n\t.reg .b64 da, db;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
+      "mov.b64 da, {%1, %6};\n\t"
+      "mov.b64 db, {%2, %6};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "@e tcgen05.mma.sp.cta_group::1.kind::f8f6f4 [%0], da, db, [%3], %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(meta_tmem), "r"(idesc), "r"(accumulate), "r"(kDescHiSw128)
       : "memory");
 }
 
