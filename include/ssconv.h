@@ -140,6 +140,21 @@ int32_t ssconv_selftest_wait_timeout(int64_t limit_cycles, int32_t* dev_status, 
 int32_t ssconv_select_mask(int32_t mode, const void* scores, int64_t G, uint8_t* pattern,
                            void* stream);
 
+/* General N:M masks (Sec. 3.1: blocks of M consecutive entries of a row of W of which N are kept;
+ * the n = C(M, N) possible blocks are the columns of D in Eq. 2), 1 <= N <= M <= 8.  Patterns are
+ * numbered lexicographically in the kept positions (for 2:4 the numbering of ssconv_select_mask).
+ * ssconv_nm_patterns returns n (0 for an N, M out of range).  ssconv_select_mask_nm: mode LOGITS takes
+ * float scores [G, n] (Eq. 1: first maximum), mode MAGNITUDE_BF16 takes bf16 weights [G, M] and keeps
+ * the N largest |w| of each block (equal magnitudes: the lower position).  ssconv_apply_mask_nm writes
+ * M .* W (Eq. 6): kept values bit for bit, +0 elsewhere; a pattern index >= n counts as pattern 0.  The
+ * sparse tensor-core operation exists for 2:4 only: weights masked with another N:M go through
+ * ssconv_forward_dense.  scores / w: device, 4- / 2-byte aligned; pattern: device uint8 [G]. */
+int32_t ssconv_nm_patterns(int32_t N, int32_t M);
+int32_t ssconv_select_mask_nm(int32_t mode, const void* scores, int64_t G, int32_t N, int32_t M, uint8_t* pattern,
+                              void* stream);
+int32_t ssconv_apply_mask_nm(const void* w_bf16, const uint8_t* pattern, int64_t G, int32_t N, int32_t M,
+                             void* w_masked_bf16, void* stream);
+
 /* Apply the mask (M .* W of Eq. 6) and pack the result in the structured form of Fig. 1:
  * the two kept bf16 values of each group, in ascending position order, bit-exact, plus
  * two 2-bit position indices per group, laid out in the tile order the sparse tensor-core
@@ -350,6 +365,41 @@ int32_t ssconv_absmax(const void* x_bf16, int64_t n, float* out, void* stream);
 enum { SSCONV_LEMMA_PERTURBATION = 34, SSCONV_LEMMA_ANY_MASK = 35, SSCONV_LEMMA_MASKED_UPDATE = 36 };
 double ssconv_stability_threshold(int32_t lemma, double L, const double* layer_norms, int32_t depth,
                                   int32_t j, double extra_norm, double x_norm);
+
+/* ---- Grouped convolutions (Sec. 4: the paper leaves grouped convolutions dense; here both forms
+ * exist).  The layer is `groups` independent convolutions on channel slices: group g reads input
+ * channels [g C_in/groups, (g+1) C_in/groups) and writes output channels [g C_out/groups, ...).  desc
+ * names the whole layer; weights are [C_out, KH, KW, C_in/groups] (each output channel sees its group's
+ * inputs); the 2:4 groups of four are four consecutive input channels *of the group's slice*, the
+ * pattern array follows the weight order, and the compressed operand is the concatenation of the
+ * per-group blobs (ssconv_sizes_grouped gives the totals; each part is what ssconv_sizes reports for the
+ * per-group layer and can be read back with ssconv_decompress).  Needs (C_in/groups) % 8 == 0 and
+ * (C_out/groups) % 8 == 0; one launch per group on strided views of x and y.  ws as for
+ * ssconv_forward (NULL allowed). */
+int32_t ssconv_sizes_grouped(const ssconv_desc_t* desc, int32_t groups, int64_t* G, size_t* w_comp_bytes,
+                             size_t* meta_bytes);
+int32_t ssconv_compress_grouped(const ssconv_desc_t* desc, int32_t groups, const void* w_bf16, const uint8_t* pattern,
+                                void* w_comp, void* meta, void* stream);
+int32_t ssconv_forward_grouped(const ssconv_desc_t* desc, int32_t groups, const void* x, const void* w_comp,
+                               const void* meta, const float* bias, void* y, void* ws, size_t ws_bytes,
+                               int32_t* dev_status, void* stream);
+int32_t ssconv_forward_dense_grouped(const ssconv_desc_t* desc, int32_t groups, const void* x, const void* w_bf16,
+                                     const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
+                                     void* stream);
+
+/* Depthwise convolution (groups = C_in = C_out), dense, as the paper leaves it (Sec. 4):
+ *   y[n,ho,wo,c] = act( bias[c] + sum_{kh,kw} x[n, ho*s-p+kh*d, wo*s-p+kw*d, c] * w[kh,kw,c] ),
+ * weights tap-major [KH, KW, C] bf16, fp32 accumulation, one rounding to bf16; act = ReLU or none.
+ * Equal strides, paddings and dilations in both directions; C % 8 == 0; 16-byte aligned pointers. */
+int32_t ssconv_depthwise(const ssconv_desc_t* desc, const void* x, const void* w_bf16, const float* bias, void* y,
+                         void* stream);
+
+/* Layer normalisation over the channels of each pixel, y = (x - mean) / sqrt(var + eps) * gamma + beta
+ * (biased variance; fp32 arithmetic, one rounding to bf16): the normalisation between the depthwise and
+ * the point-wise convolutions of a ConvNeXt block (Sec. 4 evaluates on ConvNeXt); no counterpart in the
+ * paper's method.  x, y: bf16 [pixels, C]; gamma, beta: float [C]. */
+int32_t ssconv_layernorm(const void* x_bf16, const float* gamma, const float* beta, float eps, void* y_bf16,
+                         int64_t pixels, int32_t C, void* stream);
 
 /* ---- 8-bit (e4m3) operands.  The paper's method is stated for any operand type the 2:4 hardware
  * operation supports (Sec. 2: the sparse operation halves storage and time; Sec. 3.1 defines the

@@ -25,11 +25,13 @@ ERR_TIMEOUT = 8
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.so")
 EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes",
            "ssconv_plan", "ssconv_plan_for_sms", "ssconv_tune", "ssconv_window_extent", "ssconv_selftest_wait_timeout",
-           "ssconv_select_mask",
+           "ssconv_select_mask", "ssconv_nm_patterns", "ssconv_select_mask_nm", "ssconv_apply_mask_nm",
            "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_pad_channels", "ssconv_space_to_depth", "ssconv_unfold_w", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense", "ssconv_forward_dense_strided",
            "ssconv_mask_norms", "ssconv_absmax", "ssconv_stability_threshold", "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_dgrad_prepare", "ssconv_dgrad_spread", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
            "ssconv_forward_static_ws",
+           "ssconv_sizes_grouped", "ssconv_compress_grouped", "ssconv_forward_grouped", "ssconv_forward_dense_grouped",
+           "ssconv_depthwise", "ssconv_layernorm",
            "ssconv_quantize_e4m3", "ssconv_sizes_fp8", "ssconv_compress_fp8", "ssconv_decompress_fp8",
            "ssconv_forward_fp8", "ssconv_forward_dense_fp8")
 
@@ -165,6 +167,38 @@ def ssconv_select_mask(mode: int, scores: torch.Tensor, G: int, pattern: Optiona
         pattern = torch.empty((G,), dtype=torch.uint8, device=scores.device)
     _check("ssconv_select_mask", lib().ssconv_select_mask(mode, _ptr(scores), G, _ptr(pattern), _stream(stream)))
     return pattern
+
+
+def ssconv_nm_patterns(N: int, M: int) -> int:
+    """n = C(M, N), the number of N:M patterns (0 if N, M are out of the supported range)."""
+    f = lib().ssconv_nm_patterns
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_int32, ctypes.c_int32]
+    return int(f(int(N), int(M)))
+
+
+def ssconv_select_mask_nm(mode: int, scores: torch.Tensor, G: int, N: int, M: int, stream=None) -> torch.Tensor:
+    """pattern uint8 [G] for N:M blocks from fp32 scores [G, n] (mode LOGITS) or bf16 weights [G, M] (MAGNITUDE)."""
+    _need_cuda(scores)
+    pattern = torch.empty((G,), dtype=torch.uint8, device=scores.device)
+    f = lib().ssconv_select_mask_nm
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_int32, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                  ctypes.c_void_p]
+    _check("ssconv_select_mask_nm", f(mode, _ptr(scores), G, N, M, _ptr(pattern), _stream(stream)))
+    return pattern
+
+
+def ssconv_apply_mask_nm(w: torch.Tensor, pattern: torch.Tensor, N: int, M: int, stream=None) -> torch.Tensor:
+    """M .* W for an N:M mask: bf16 weights of w's shape with the dropped positions zeroed."""
+    _need_cuda(w, pattern)
+    out = torch.empty_like(w)
+    f = lib().ssconv_apply_mask_nm
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                  ctypes.c_void_p]
+    _check("ssconv_apply_mask_nm", f(_ptr(w), _ptr(pattern), pattern.numel(), N, M, _ptr(out), _stream(stream)))
+    return out
 
 
 def ssconv_compress(desc: Desc, w: torch.Tensor, pattern: torch.Tensor, stream=None):
@@ -393,6 +427,94 @@ def ssconv_forward_static_ws(desc: Desc, x: torch.Tensor, w_comp: torch.Tensor, 
     _check("ssconv_forward_static_ws", lib().ssconv_forward_static_ws(
         ctypes.byref(desc), _ptr(x), _ptr(w_comp), _ptr(meta), _ptr(bias), _ptr(y), _ptr(dev_status),
         _stream(stream)))
+    return y
+
+
+# ----------------------------------------------------------------------------- grouped / depthwise / layer norm
+def ssconv_sizes_grouped(desc: Desc, groups: int):
+    G = ctypes.c_int64()
+    a, b = ctypes.c_size_t(), ctypes.c_size_t()
+    f = lib().ssconv_sizes_grouped
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_int32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_size_t),
+                  ctypes.POINTER(ctypes.c_size_t)]
+    _check("ssconv_sizes_grouped", f(ctypes.byref(desc), groups, ctypes.byref(G), ctypes.byref(a), ctypes.byref(b)))
+    return int(G.value), int(a.value), int(b.value)
+
+
+def ssconv_compress_grouped(desc: Desc, groups: int, w: torch.Tensor, pattern: torch.Tensor, stream=None):
+    """(w_comp, meta) of a grouped layer: the per-group blobs one after another."""
+    _need_cuda(w, pattern)
+    _, nv, nm = ssconv_sizes_grouped(desc, groups)
+    w_comp = torch.empty((nv,), dtype=torch.uint8, device=w.device)
+    meta = torch.empty((nm,), dtype=torch.uint8, device=w.device)
+    f = lib().ssconv_compress_grouped
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_int32] + [ctypes.c_void_p] * 5
+    _check("ssconv_compress_grouped", f(ctypes.byref(desc), groups, _ptr(w), _ptr(pattern), _ptr(w_comp), _ptr(meta),
+                                        _stream(stream)))
+    return w_comp, meta
+
+
+def ssconv_forward_grouped(desc: Desc, groups: int, x: torch.Tensor, w_comp: torch.Tensor, meta: torch.Tensor,
+                           bias: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None,
+                           dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """2:4 masked grouped convolution (one launch per group on channel slices)."""
+    _need_cuda(x, w_comp, meta, bias, y, dev_status)
+    if y is None:
+        y = _alloc_y(desc, x)
+    ws = default_workspace(x.device)
+    f = lib().ssconv_forward_grouped
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_int32] + [ctypes.c_void_p] * 6 + [ctypes.c_size_t, ctypes.c_void_p,
+                                                                                  ctypes.c_void_p]
+    _check("ssconv_forward_grouped", f(ctypes.byref(desc), groups, _ptr(x), _ptr(w_comp), _ptr(meta), _ptr(bias), _ptr(y),
+                                       _ptr(ws), ws.numel(), _ptr(dev_status), _stream(stream)))
+    return y
+
+
+def ssconv_forward_dense_grouped(desc: Desc, groups: int, x: torch.Tensor, w: torch.Tensor,
+                                 bias: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None,
+                                 dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Dense grouped convolution; w bf16 [C_out, KH, KW, C_in/groups]."""
+    _need_cuda(x, w, bias, y, dev_status)
+    if y is None:
+        y = _alloc_y(desc, x)
+    ws = default_workspace(x.device)
+    f = lib().ssconv_forward_dense_grouped
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_int32] + [ctypes.c_void_p] * 5 + [ctypes.c_size_t, ctypes.c_void_p,
+                                                                                  ctypes.c_void_p]
+    _check("ssconv_forward_dense_grouped", f(ctypes.byref(desc), groups, _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _ptr(ws),
+                                             ws.numel(), _ptr(dev_status), _stream(stream)))
+    return y
+
+
+def ssconv_depthwise(desc: Desc, x: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor] = None,
+                     y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Dense depthwise convolution; w bf16 tap-major [KH, KW, C]."""
+    _need_cuda(x, w, bias, y)
+    if y is None:
+        y = _alloc_y(desc, x)
+    f = lib().ssconv_depthwise
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc)] + [ctypes.c_void_p] * 5
+    _check("ssconv_depthwise", f(ctypes.byref(desc), _ptr(x), _ptr(w), _ptr(bias), _ptr(y), _stream(stream)))
+    return y
+
+
+def ssconv_layernorm(x: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor, eps: float = 1e-6,
+                     y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Layer normalisation over the last axis of x (bf16), gamma / beta fp32 [C]."""
+    _need_cuda(x, gamma, beta, y)
+    c = x.shape[-1]
+    if y is None:
+        y = torch.empty_like(x)
+    f = lib().ssconv_layernorm
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p, ctypes.c_int64,
+                  ctypes.c_int32, ctypes.c_void_p]
+    _check("ssconv_layernorm", f(_ptr(x), _ptr(gamma), _ptr(beta), float(eps), _ptr(y), x.numel() // c, c, _stream(stream)))
     return y
 
 

@@ -29,6 +29,17 @@ cudaError_t launch_compress_e4m3(const ssconv_desc_t& d, const void* w, const ui
                                  cudaStream_t st);
 cudaError_t launch_decompress_e4m3(const ssconv_desc_t& d, const void* w_comp, const void* meta, void* w_out,
                                    uint8_t* pattern_out, cudaStream_t st);
+int nm_pattern_count(int N, int M);
+cudaError_t launch_nm_select(int mode, const void* scores, int64_t G, int N, int M, uint8_t* pattern, cudaStream_t st);
+cudaError_t launch_nm_apply(const void* w, const uint8_t* pattern, int64_t G, int N, int M, void* w_masked,
+                            cudaStream_t st);
+int32_t launch_forward_grouped(const ssconv_desc_t& d, int groups, bool sparse, const void* x, const void* weights,
+                               const void* meta, const float* bias, void* y, void* ws, size_t ws_bytes,
+                               int32_t* dev_status, cudaStream_t stream);
+cudaError_t launch_depthwise(const void* x, const void* w, const float* bias, void* y, int N, int H, int W, int C, int Ho,
+                             int Wo, int KH, int KW, int stride, int pad, int dil, uint32_t flags, cudaStream_t st);
+cudaError_t launch_layernorm(const void* x, const float* gamma, const float* beta, void* y, long long pixels, int C,
+                             float eps, cudaStream_t st);
 size_t workspace_bytes();
 int32_t set_tuning(int32_t option, int32_t value);
 cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad,
@@ -187,6 +198,31 @@ int32_t ssconv_select_mask(int32_t mode, const void* scores, int64_t G, uint8_t*
                                                                                               : SSCONV_ERR_CUDA;
 }
 
+int32_t ssconv_nm_patterns(int32_t N, int32_t M) { return ssconv::nm_pattern_count(N, M); }
+
+int32_t ssconv_select_mask_nm(int32_t mode, const void* scores, int64_t G, int32_t N, int32_t M, uint8_t* pattern,
+                              void* stream) {
+  if (mode != SSCONV_MASK_LOGITS_F32 && mode != SSCONV_MASK_MAGNITUDE_BF16) return SSCONV_ERR_BAD_DESC;
+  if (G < 0 || ssconv::nm_pattern_count(N, M) == 0) return SSCONV_ERR_BAD_DESC;
+  if (G == 0) return SSCONV_OK;
+  if (!scores || !pattern) return SSCONV_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(scores) & (mode == SSCONV_MASK_LOGITS_F32 ? 3u : 1u)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_nm_select(mode, scores, G, N, M, pattern, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_apply_mask_nm(const void* w_bf16, const uint8_t* pattern, int64_t G, int32_t N, int32_t M,
+                             void* w_masked_bf16, void* stream) {
+  if (G < 0 || ssconv::nm_pattern_count(N, M) == 0) return SSCONV_ERR_BAD_DESC;
+  if (G == 0) return SSCONV_OK;
+  if (!w_bf16 || !pattern || !w_masked_bf16) return SSCONV_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(w_bf16) | reinterpret_cast<uintptr_t>(w_masked_bf16)) & 1u) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_nm_apply(w_bf16, pattern, G, N, M, w_masked_bf16, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
 int32_t ssconv_compress(const ssconv_desc_t* desc, const void* w_bf16, const uint8_t* pattern, void* w_comp,
                         void* meta, void* stream) {
   int32_t rc = check_desc(desc, false);
@@ -323,6 +359,111 @@ static int32_t check_fp8(const ssconv_desc_t* desc, float out_scale) {
   if (desc->C_in % 16 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
   if (!(out_scale > 0.0f) || !(out_scale < 3.0e38f)) return SSCONV_ERR_BAD_DESC;
   return SSCONV_OK;
+}
+
+// ---- grouped convolutions
+static int32_t check_groups(const ssconv_desc_t* desc, int32_t groups, ssconv_desc_t* sub) {
+  int32_t rc = check_desc(desc, true);
+  if (rc != SSCONV_OK) return rc;
+  if (groups < 1 || desc->C_in % groups != 0 || desc->C_out % groups != 0) return SSCONV_ERR_BAD_DESC;
+  *sub = *desc;
+  sub->C_in = desc->C_in / groups;
+  sub->C_out = desc->C_out / groups;
+  if (sub->C_in % 8 != 0 || sub->C_out % 8 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;  // (one channel per group: ssconv_depthwise)
+  return SSCONV_OK;
+}
+
+int32_t ssconv_sizes_grouped(const ssconv_desc_t* desc, int32_t groups, int64_t* G, size_t* w_comp_bytes,
+                             size_t* meta_bytes) {
+  ssconv_desc_t sub;
+  int32_t rc = check_groups(desc, groups, &sub);
+  if (rc != SSCONV_OK) return rc;
+  int64_t g1 = 0;
+  size_t a = 0, b = 0;
+  rc = ssconv_sizes(&sub, &g1, &a, &b, nullptr, nullptr);
+  if (rc != SSCONV_OK) return rc;
+  if (G) *G = g1 * groups;
+  if (w_comp_bytes) *w_comp_bytes = a * groups;
+  if (meta_bytes) *meta_bytes = b * groups;
+  return SSCONV_OK;
+}
+
+int32_t ssconv_compress_grouped(const ssconv_desc_t* desc, int32_t groups, const void* w_bf16, const uint8_t* pattern,
+                                void* w_comp, void* meta, void* stream) {
+  ssconv_desc_t sub;
+  int32_t rc = check_groups(desc, groups, &sub);
+  if (rc != SSCONV_OK) return rc;
+  int64_t g1 = 0;
+  size_t a = 0, b = 0;
+  rc = ssconv_sizes(&sub, &g1, &a, &b, nullptr, nullptr);
+  if (rc != SSCONV_OK) return rc;
+  if (!w_bf16 || !pattern || !w_comp || !meta) return SSCONV_ERR_NULL;
+  if (!aligned16(w_bf16) || !aligned16(w_comp) || !aligned16(meta)) return SSCONV_ERR_ALIGNMENT;
+  const size_t w_step = (size_t)sub.C_out * sub.KH * sub.KW * sub.C_in * 2;
+  for (int32_t i = 0; i < groups; ++i) {
+    rc = ssconv_compress(&sub, static_cast<const char*>(w_bf16) + i * w_step, pattern + (size_t)i * g1,
+                         static_cast<char*>(w_comp) + i * a, static_cast<char*>(meta) + i * b, stream);
+    if (rc != SSCONV_OK) return rc;
+  }
+  return SSCONV_OK;
+}
+
+int32_t ssconv_forward_grouped(const ssconv_desc_t* desc, int32_t groups, const void* x, const void* w_comp,
+                               const void* meta, const float* bias, void* y, void* ws, size_t ws_bytes,
+                               int32_t* dev_status, void* stream) {
+  ssconv_desc_t sub;
+  int32_t rc = check_groups(desc, groups, &sub);
+  if (rc != SSCONV_OK) return rc;
+  if (!x || !w_comp || !meta || !y) return SSCONV_ERR_NULL;
+  if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
+  if (!aligned16(x) || !aligned16(w_comp) || !aligned16(meta) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_forward_grouped(*desc, groups, true, x, w_comp, meta, bias, y, ws, ws_bytes, dev_status,
+                                        (cudaStream_t)stream);
+}
+
+int32_t ssconv_forward_dense_grouped(const ssconv_desc_t* desc, int32_t groups, const void* x, const void* w_bf16,
+                                     const float* bias, void* y, void* ws, size_t ws_bytes, int32_t* dev_status,
+                                     void* stream) {
+  ssconv_desc_t sub;
+  int32_t rc = check_groups(desc, groups, &sub);
+  if (rc != SSCONV_OK) return rc;
+  if (!x || !w_bf16 || !y) return SSCONV_ERR_NULL;
+  if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
+  if (!aligned16(x) || !aligned16(w_bf16) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  return ssconv::launch_forward_grouped(*desc, groups, false, x, w_bf16, nullptr, bias, y, ws, ws_bytes, dev_status,
+                                        (cudaStream_t)stream);
+}
+
+int32_t ssconv_depthwise(const ssconv_desc_t* desc, const void* x, const void* w_bf16, const float* bias, void* y,
+                         void* stream) {
+  int32_t rc = check_desc(desc, false);
+  if (rc != SSCONV_OK) return rc;
+  if (desc->C_in != desc->C_out) return SSCONV_ERR_BAD_DESC;
+  if (desc->C_in % 8 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if (desc->flags & SSCONV_FLAG_GELU) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if (!x || !w_bf16 || !y) return SSCONV_ERR_NULL;
+  if ((desc->flags & SSCONV_FLAG_BIAS) && !bias) return SSCONV_ERR_NULL;
+  if (!aligned16(x) || !aligned16(w_bf16) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  const int Ho = out_extent(desc->H, desc->KH, desc->stride_h, desc->pad_h, desc->dil_h);
+  const int Wo = out_extent(desc->W, desc->KW, desc->stride_w, desc->pad_w, desc->dil_w);
+  if (desc->stride_h != desc->stride_w || desc->pad_h != desc->pad_w || desc->dil_h != desc->dil_w)
+    return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  return ssconv::launch_depthwise(x, w_bf16, bias, y, desc->N, desc->H, desc->W, desc->C_in, Ho, Wo, desc->KH, desc->KW,
+                                  desc->stride_h, desc->pad_h, desc->dil_h, desc->flags, (cudaStream_t)stream) ==
+                 cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+int32_t ssconv_layernorm(const void* x_bf16, const float* gamma, const float* beta, float eps, void* y_bf16,
+                         int64_t pixels, int32_t C, void* stream) {
+  if (pixels < 0 || C <= 0 || !(eps >= 0.0f)) return SSCONV_ERR_BAD_DESC;
+  if (pixels == 0) return SSCONV_OK;
+  if (!x_bf16 || !gamma || !beta || !y_bf16) return SSCONV_ERR_NULL;
+  if (pixels > 0x3FFFFFFLL * 8) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  return ssconv::launch_layernorm(x_bf16, gamma, beta, y_bf16, pixels, C, eps, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
 }
 
 int32_t ssconv_quantize_e4m3(const void* x_bf16, void* y_e4m3, int64_t n, float scale, void* stream) {

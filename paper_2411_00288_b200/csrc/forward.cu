@@ -823,6 +823,7 @@ struct FinishParams {
   const float* bias;
   const __nv_bfloat16* residual;  // nullable
   __nv_bfloat16* y;
+  int y_pitch;  // elements between consecutive positions of y (and of the residual): C_out, or more for a channel slice
 };
 constexpr int kFinishThreads = 128;
 // work items per tile: epilogue groups x pieces per group x blocks of 8 positions per piece
@@ -888,7 +889,7 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
   if (f.residual != nullptr) {
     // residual block -> staging buffer (same layout), read back in fragment layout, added in fp32
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (in_range) v = *reinterpret_cast<const uint4*>(f.residual + (size_t)q_pos * f.C_out + co16);
+    if (in_range) v = *reinterpret_cast<const uint4*>(f.residual + (size_t)q_pos * f.y_pitch + co16);
     *reinterpret_cast<uint4*>(stage + pos * 256 + ((ch16 ^ pos) << 4)) = v;
     __syncthreads();
     uint32_t res[4];
@@ -909,7 +910,7 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
   __syncthreads();
   if (in_range) {
     const uint4 v = *reinterpret_cast<const uint4*>(stage + pos * 256 + ((ch16 ^ pos) << 4));
-    *reinterpret_cast<uint4*>(f.y + (size_t)q_pos * f.C_out + co16) = v;
+    *reinterpret_cast<uint4*>(f.y + (size_t)q_pos * f.y_pitch + co16) = v;
   }
 }
 
@@ -1527,12 +1528,13 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
                                    const float* bias, const void* residual, void* y, void* ws, size_t ws_bytes,
                                    int32_t* dev_status, cudaStream_t stream, int worker_cap = kMaxWorkers,
                                    bool force_split = false, const int64_t* x_strides = nullptr,
-                                   float out_scale = 1.0f) {
+                                   float out_scale = 1.0f, int64_t y_pitch = 0) {
   using C = Cfg<SPARSE, FP8>;
   constexpr int kKb = C::kKbChannels;
   constexpr size_t kElem = FP8 ? 1 : 2;  // bytes per operand element
   constexpr CUtensorMapDataType kOperandType = FP8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
   if (FP8 && residual != nullptr) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  const int64_t y_pitch_el = y_pitch > 0 ? y_pitch : d.C_out;
   if (!load_driver_entry_points()) return SSCONV_ERR_CUDA;
   int dev = 0;
   {
@@ -1659,7 +1661,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   // output: NHWC seen as (c, position); a box is one staging half piece, 64 channels x 40 positions
   {
     cuuint64_t dims[2] = {(cuuint64_t)d.C_out, (cuuint64_t)Q};
-    cuuint64_t strides[1] = {(cuuint64_t)d.C_out * 2};
+    cuuint64_t strides[1] = {(cuuint64_t)y_pitch_el * 2};  // (channels beyond C_out are clipped: a slice stays a slice)
     cuuint32_t box[2] = {64, (cuuint32_t)kPiece};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode_tiled(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, dims, strides, box, estr,
@@ -1786,6 +1788,7 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
     f.bias = bias;
     f.residual = static_cast<const __nv_bfloat16*>(residual);
     f.y = p.y;
+    f.y_pitch = (int)y_pitch_el;
     cfg.gridDim = dim3((unsigned)p.num_tiles * finish_items_per_tile(pieces));
     cfg.blockDim = dim3((unsigned)kFinishThreads);
     cfg.dynamicSmemBytes = 0;
@@ -1805,6 +1808,35 @@ int32_t launch_forward_dense(const ssconv_desc_t& d, const void* x, const void* 
                              cudaStream_t stream, const int64_t* x_strides) {
   return launch_forward_impl<false>(d, x, w, nullptr, bias, residual, y, ws, ws_bytes, dev_status, stream, kMaxWorkers,
                                     false, x_strides);
+}
+
+// Grouped convolution: `groups` independent convolutions on channel slices, group g reading input
+// channels [g C_in/groups, ...) and writing output channels [g C_out/groups, ...); one launch per group
+// on strided views of x and y.  The compressed operand of a grouped layer is the concatenation of the
+// groups' blobs (each of the size ssconv_sizes reports for the per-group layer).
+int32_t launch_forward_grouped(const ssconv_desc_t& d, int groups, bool sparse, const void* x, const void* weights,
+                               const void* meta, const float* bias, void* y, void* ws, size_t ws_bytes,
+                               int32_t* dev_status, cudaStream_t stream) {
+  ssconv_desc_t g = d;
+  g.C_in = d.C_in / groups;
+  g.C_out = d.C_out / groups;
+  const Geometry geo = make_geometry(g);
+  const size_t w_step = sparse ? (size_t)geo.Mp * geo.KC * 2 : (size_t)g.C_out * geo.taps * g.C_in * 2;
+  const size_t m_step = (size_t)geo.m_tiles * geo.stages * kMetaImageBytes;
+  const int64_t xs[3] = {d.C_in, (int64_t)d.W * d.C_in, (int64_t)d.H * d.W * d.C_in};
+  for (int i = 0; i < groups; ++i) {
+    const char* xg = static_cast<const char*>(x) + (size_t)i * g.C_in * 2;
+    char* yg = static_cast<char*>(y) + (size_t)i * g.C_out * 2;
+    const float* bg = bias ? bias + (size_t)i * g.C_out : nullptr;
+    const char* wg = static_cast<const char*>(weights) + (size_t)i * w_step;
+    const int32_t rc =
+        sparse ? launch_forward_impl<true>(g, xg, wg, static_cast<const char*>(meta) + (size_t)i * m_step, bg, nullptr, yg,
+                                           ws, ws_bytes, dev_status, stream, kMaxWorkers, false, xs, 1.0f, d.C_out)
+               : launch_forward_impl<false>(g, xg, wg, nullptr, bg, nullptr, yg, ws, ws_bytes, dev_status, stream,
+                                            kMaxWorkers, false, xs, 1.0f, d.C_out);
+    if (rc != SSCONV_OK) return rc;
+  }
+  return SSCONV_OK;
 }
 
 int32_t launch_forward_fp8(const ssconv_desc_t& d, bool sparse, const void* x, const void* weights, const void* meta,

@@ -86,6 +86,65 @@ __global__ void quantize_e4m3_kernel(const uint32_t* __restrict__ x, uint16_t* _
 }
 
 // ---------------------------------------------------------------------------------------
+// General N:M bookkeeping (Sec. 3.1): blocks of M consecutive weights of which N are kept, one of
+// n = C(M, N) patterns per block, numbered lexicographically in the kept positions.  The hardware
+// operation exists for 2:4 only; other N:M masks are selected and applied here and the masked weights
+// run through the dense kernel (Eq. 6 with a dense product).  M <= 8, so a pattern is a byte and its
+// kept positions a bitmask; the table of all patterns (at most C(8,4) = 70) travels as a kernel argument.
+// ---------------------------------------------------------------------------------------
+struct NmTable {
+  int N, M, n;
+  uint8_t kept_mask[70];  // bit i set: position i of the block is kept
+};
+
+__global__ void nm_select_logits_kernel(const float* __restrict__ scores, int64_t G, int n, uint8_t* __restrict__ pattern) {
+  int64_t g = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (g >= G) return;
+  const float* s = scores + g * n;
+  int best = 0;
+  float bv = s[0];
+  for (int i = 1; i < n; ++i) {
+    const float v = s[i];
+    if (v > bv) {
+      bv = v;
+      best = i;
+    }
+  }
+  pattern[g] = (uint8_t)best;
+}
+
+// Keep the N largest magnitudes of the block (15-bit integers below the bf16 sign bit); a position
+// beats another when it is larger, or equal and earlier; the kept ones are beaten by fewer than N.
+__global__ void nm_select_magnitude_kernel(const uint16_t* __restrict__ w, int64_t G, NmTable t,
+                                           uint8_t* __restrict__ pattern) {
+  int64_t g = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (g >= G) return;
+  uint32_t a[8];
+  for (int i = 0; i < t.M; ++i) a[i] = w[g * t.M + i] & 0x7FFFu;
+  uint32_t mask = 0;
+  for (int i = 0; i < t.M; ++i) {
+    int beaten = 0;
+    for (int j = 0; j < t.M; ++j)
+      if (j != i) beaten += (a[j] > a[i]) || (a[j] == a[i] && j < i);
+    if (beaten < t.N) mask |= 1u << i;
+  }
+  int p = 0;
+  for (int i = 0; i < t.n; ++i)
+    if (t.kept_mask[i] == mask) p = i;
+  pattern[g] = (uint8_t)p;
+}
+
+// Eq. 6 for an N:M mask: dropped positions become +0, kept values are copied bit for bit.
+__global__ void nm_apply_mask_kernel(const uint16_t* __restrict__ w, const uint8_t* __restrict__ pattern, int64_t G,
+                                     NmTable t, uint16_t* __restrict__ w_masked) {
+  int64_t g = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (g >= G) return;
+  const uint32_t p = pattern[g];
+  const uint32_t mask = p < (uint32_t)t.n ? t.kept_mask[p] : t.kept_mask[0];  // (an index out of range: pattern 0)
+  for (int i = 0; i < t.M; ++i) w_masked[g * t.M + i] = ((mask >> i) & 1u) ? w[g * t.M + i] : (uint16_t)0;
+}
+
+// ---------------------------------------------------------------------------------------
 // 8-bit (e4m3) weights: compress / decompress
 // ---------------------------------------------------------------------------------------
 // Geometry with k-blocks of 128 channels (make_geometry(d, 128)).  Value blob: bytes [Mp][64 * kblocks_pad]:
@@ -277,6 +336,53 @@ cudaError_t launch_select(int mode, const void* scores, int64_t G, uint8_t* patt
     select_magnitude_e4m3_kernel<<<blocks_for(G, T), T, 0, st>>>((const uint32_t*)scores, G, pattern);
   else
     select_magnitude_kernel<<<blocks_for(G, T), T, 0, st>>>((const uint2*)scores, G, pattern);
+  return cudaGetLastError();
+}
+
+// All N-subsets of {0..M-1} in lexicographic order of the kept positions, as bitmasks.
+static bool make_nm_table(int N, int M, NmTable* t) {
+  if (M < 1 || M > 8 || N < 1 || N > M) return false;
+  t->N = N;
+  t->M = M;
+  t->n = 0;
+  int idx[8];
+  for (int i = 0; i < N; ++i) idx[i] = i;
+  while (true) {
+    uint32_t mask = 0;
+    for (int i = 0; i < N; ++i) mask |= 1u << idx[i];
+    t->kept_mask[t->n++] = (uint8_t)mask;
+    int i = N - 1;
+    while (i >= 0 && idx[i] == M - N + i) --i;
+    if (i < 0) break;
+    ++idx[i];
+    for (int j = i + 1; j < N; ++j) idx[j] = idx[j - 1] + 1;
+  }
+  return true;
+}
+int nm_pattern_count(int N, int M) {
+  NmTable t;
+  return make_nm_table(N, M, &t) ? t.n : 0;
+}
+cudaError_t launch_nm_select(int mode, const void* scores, int64_t G, int N, int M, uint8_t* pattern, cudaStream_t st) {
+  NmTable t;
+  if (!make_nm_table(N, M, &t)) return cudaErrorInvalidValue;
+  if (G == 0) return cudaSuccess;
+  const int T = 256;
+  count_launch();
+  if (mode == SSCONV_MASK_LOGITS_F32)
+    nm_select_logits_kernel<<<blocks_for(G, T), T, 0, st>>>((const float*)scores, G, t.n, pattern);
+  else
+    nm_select_magnitude_kernel<<<blocks_for(G, T), T, 0, st>>>((const uint16_t*)scores, G, t, pattern);
+  return cudaGetLastError();
+}
+cudaError_t launch_nm_apply(const void* w, const uint8_t* pattern, int64_t G, int N, int M, void* w_masked,
+                            cudaStream_t st) {
+  NmTable t;
+  if (!make_nm_table(N, M, &t)) return cudaErrorInvalidValue;
+  if (G == 0) return cudaSuccess;
+  const int T = 256;
+  count_launch();
+  nm_apply_mask_kernel<<<blocks_for(G, T), T, 0, st>>>((const uint16_t*)w, pattern, G, t, (uint16_t*)w_masked);
   return cudaGetLastError();
 }
 

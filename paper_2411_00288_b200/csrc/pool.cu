@@ -148,6 +148,110 @@ cudaError_t launch_space_to_depth(const void* x, void* y, int N, int H, int W, i
   return cudaGetLastError();
 }
 
+// Depthwise convolution (groups = C_in = C_out), dense, direct: every output element is its own sum over
+// the KH x KW window of one channel (Eq. 4 with a single input channel per output channel).  The paper
+// leaves such layers untouched by the mask (Sec. 4); they are here so that a ConvNeXt-shaped block
+// chains through the library.  One thread per 8 channels of an output pixel: 16-byte loads of pixels
+// and of the tap-major weights [KH, KW, C], fp32 accumulation, bias, one rounding to bf16.
+__global__ void __launch_bounds__(256) depthwise_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w,
+                                                        const float* __restrict__ bias, uint4* __restrict__ y, int N,
+                                                        int H, int W, int C8, int Ho, int Wo, int KH, int KW, int stride,
+                                                        int pad, int dil, uint32_t flags) {
+  const long long total = (long long)N * Ho * Wo * C8;
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int c = (int)(i % C8);
+  long long pix = i / C8;
+  const int wo = (int)(pix % Wo);
+  pix /= Wo;
+  const int ho = (int)(pix % Ho);
+  const int n = (int)(pix / Ho);
+  float acc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
+  for (int kh = 0; kh < KH; ++kh) {
+    const int h = ho * stride - pad + kh * dil;
+    if (h < 0 || h >= H) continue;
+    for (int kw = 0; kw < KW; ++kw) {
+      const int ww = wo * stride - pad + kw * dil;
+      if (ww < 0 || ww >= W) continue;
+      const uint4 xv = __ldg(x + ((long long)(n * H + h) * W + ww) * C8 + c);
+      const uint4 wv = __ldg(w + (long long)(kh * KW + kw) * C8 + c);
+      const uint32_t xa[4] = {xv.x, xv.y, xv.z, xv.w}, wa[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        acc[2 * j] = fmaf(__uint_as_float(xa[j] << 16), __uint_as_float(wa[j] << 16), acc[2 * j]);
+        acc[2 * j + 1] = fmaf(__uint_as_float(xa[j] & 0xFFFF0000u), __uint_as_float(wa[j] & 0xFFFF0000u), acc[2 * j + 1]);
+      }
+    }
+  }
+  uint32_t out[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    float lo = acc[2 * j], hi = acc[2 * j + 1];
+    if (flags & SSCONV_FLAG_BIAS) {
+      lo += bias[8 * c + 2 * j];
+      hi += bias[8 * c + 2 * j + 1];
+    }
+    if (flags & SSCONV_FLAG_RELU) {
+      lo = fmaxf(lo, 0.0f);
+      hi = fmaxf(hi, 0.0f);
+    }
+    __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    out[j] = *reinterpret_cast<uint32_t*>(&b);
+  }
+  y[i] = make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+cudaError_t launch_depthwise(const void* x, const void* w, const float* bias, void* y, int N, int H, int W, int C, int Ho,
+                             int Wo, int KH, int KW, int stride, int pad, int dil, uint32_t flags, cudaStream_t st) {
+  const long long total = (long long)N * Ho * Wo * (C / 8);
+  if (total == 0) return cudaSuccess;
+  const int T = 256;
+  count_launch();
+  depthwise_kernel<<<(unsigned)((total + T - 1) / T), T, 0, st>>>(static_cast<const uint4*>(x), static_cast<const uint4*>(w),
+                                                                  bias, static_cast<uint4*>(y), N, H, W, C / 8, Ho, Wo, KH,
+                                                                  KW, stride, pad, dil, flags);
+  return cudaGetLastError();
+}
+
+// Layer normalisation over the channels of each pixel (the normalisation of a ConvNeXt block; not part
+// of the paper's method): y = (x - mean) / sqrt(var + eps) * gamma + beta with the biased variance, in
+// fp32, one rounding to bf16.  One warp per pixel; a lane holds C / 32 rounded up channels in registers.
+__global__ void __launch_bounds__(256) layernorm_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ gamma,
+                                                        const float* __restrict__ beta, __nv_bfloat16* __restrict__ y,
+                                                        long long pixels, int C, float eps) {
+  const long long pix = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (pix >= pixels) return;
+  const __nv_bfloat16* xp = x + pix * C;
+  float sum = 0.0f;
+  for (int c = lane; c < C; c += 32) sum += __bfloat162float(xp[c]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  const float mean = sum / (float)C;
+  float sq = 0.0f;
+  for (int c = lane; c < C; c += 32) {
+    const float d = __bfloat162float(xp[c]) - mean;
+    sq += d * d;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+  const float rstd = rsqrtf(sq / (float)C + eps);
+  for (int c = lane; c < C; c += 32)
+    y[pix * C + c] = __float2bfloat16_rn((__bfloat162float(xp[c]) - mean) * rstd * gamma[c] + beta[c]);
+}
+
+cudaError_t launch_layernorm(const void* x, const float* gamma, const float* beta, void* y, long long pixels, int C,
+                             float eps, cudaStream_t st) {
+  if (pixels == 0) return cudaSuccess;
+  const int T = 256;
+  count_launch();
+  layernorm_kernel<<<(unsigned)((pixels * 32 + T - 1) / T), T, 0, st>>>(static_cast<const __nv_bfloat16*>(x), gamma, beta,
+                                                                        static_cast<__nv_bfloat16*>(y), pixels, C, eps);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_pad_channels(const void* x, void* y, long long pixels, int C, int C_pad, cudaStream_t st) {
   const long long total = pixels * (C_pad / 8);
   if (total == 0) return cudaSuccess;
