@@ -198,7 +198,8 @@ int32_t ssconv_pad_channels(const void* x, void* y, int64_t pixels, int32_t C, i
  * over y, and, reading T neighbouring pixels of y as one pixel of T*C_pad channels through
  * ssconv_forward_dense_strided, a T x 1 convolution.  The weights are rearranged by the same call:
  * [C_out, K, K, C] as C_out "images" with pad 0 and Hb = Wb = T gives [C_out, T, T, C_pad].
- * x: device, 2-byte aligned; y: device, 16-byte aligned; C_pad % 8 == 0, C_pad >= block*block*C. */
+ * x: device, 2-byte aligned; y: device, 16-byte aligned (8-byte when C_pad % 8 != 0); C_pad % 4 == 0,
+ * C_pad >= block*block*C. */
 int32_t ssconv_space_to_depth(const void* x, void* y, int32_t N, int32_t H, int32_t W, int32_t C, int32_t block,
                               int32_t pad, int32_t Hb, int32_t Wb, int32_t C_pad, void* stream);
 
@@ -430,6 +431,28 @@ int32_t ssconv_forward_fp8(const ssconv_desc_t* desc, const void* x_e4m3, const 
                            const float* bias, float out_scale, void* y, int32_t* dev_status, void* stream);
 int32_t ssconv_forward_dense_fp8(const ssconv_desc_t* desc, const void* x_e4m3, const void* w_e4m3, const float* bias,
                                  float out_scale, void* y, int32_t* dev_status, void* stream);
+
+/* Folding of f neighbouring output pixels of a row into the output channels.  A tile of the forward
+ * kernels always spends 128 accumulator rows on output channels, so a layer with C_out <= 64 wastes
+ * half of every multiply-add it issues.  The convolution of Eq. 4 with KW taps of stride s and
+ * dilation d along the width equals, output pixel (h, f i + j) <-> channel block j of pixel (h, i), a
+ * convolution with f C_out output channels, KW' = (f-1) s + (KW-1) d + 1 undilated taps and stride f s,
+ *   W'[j C_out + c, kh, kw', :] = W[c, kh, kw, :]  where kw' = j s + kw d, and 0 elsewhere,
+ * whose NHWC output [N, H_out, W_out / f, f C_out] is byte for byte the output [N, H_out, W_out, C_out]
+ * of the original.  Groups of four input channels stay together, so a 2:4 pattern folds with its
+ * weights (all-zero groups take pattern 0) and the folded layer goes through ssconv_compress /
+ * ssconv_forward, or ssconv_forward_dense, like any other; bias and residual keep their meaning (the
+ * bias is repeated f times, the residual tensor is read through the same byte identity).
+ *   ssconv_fold_factor: the factor (1 or 2) the planner suggests for a layer: 2 when C_out <= 64,
+ *     W_out is even and the folded layer issues at least 15 % fewer multiply-adds per output.
+ *   ssconv_fold_desc: the folded descriptor; W_out % f != 0 -> SSCONV_ERR_UNSUPPORTED_SHAPE.
+ *   ssconv_fold_weights: w (nullable) is [C_out, KH, KW] vectors of tap_bytes bytes each (bf16 weights:
+ *     2 C_in; e4m3 weights: C_in; patterns: C_in / 4), w_folded [f C_out, KH, KW'] such vectors;
+ *     bias (nullable) [C_out] floats, bias_folded [f C_out].  Device pointers, no alignment rule. */
+int32_t ssconv_fold_factor(const ssconv_desc_t* desc);
+int32_t ssconv_fold_desc(const ssconv_desc_t* desc, int32_t f, ssconv_desc_t* folded);
+int32_t ssconv_fold_weights(const ssconv_desc_t* desc, int32_t f, const void* w, void* w_folded, int64_t tap_bytes,
+                            const float* bias, float* bias_folded, void* stream);
 
 /* ssconv_forward_dense on a strided view of the input: pixel (n, h, w) of the H x W x C_in input the
  * descriptor names starts stride_n*n + stride_h*h + stride_w*w elements into x.  The strides are

@@ -26,7 +26,8 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libssconv.
 EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssconv_out_shape", "ssconv_sizes",
            "ssconv_plan", "ssconv_plan_for_sms", "ssconv_tune", "ssconv_window_extent", "ssconv_selftest_wait_timeout",
            "ssconv_select_mask", "ssconv_nm_patterns", "ssconv_select_mask_nm", "ssconv_apply_mask_nm",
-           "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_pad_channels", "ssconv_space_to_depth", "ssconv_unfold_w", "ssconv_forward", "ssconv_forward_res",
+           "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_pad_channels", "ssconv_space_to_depth", "ssconv_unfold_w",
+           "ssconv_fold_factor", "ssconv_fold_desc", "ssconv_fold_weights", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense", "ssconv_forward_dense_strided",
            "ssconv_mask_norms", "ssconv_absmax", "ssconv_stability_threshold", "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_dgrad_prepare", "ssconv_dgrad_spread", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
            "ssconv_forward_static_ws",
@@ -376,6 +377,52 @@ def ssconv_space_to_depth(x: torch.Tensor, block: int, pad: int, Hb: int, Wb: in
     f.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int32] * 9 + [ctypes.c_void_p]
     _check("ssconv_space_to_depth", f(_ptr(x), _ptr(y), n, h, w, c, block, pad, Hb, Wb, C_pad, _stream(stream)))
     return y
+
+
+def ssconv_fold_factor(desc: Desc) -> int:
+    """The number of neighbouring output pixels (1 or 2) the planner suggests folding into the output channels."""
+    f = lib().ssconv_fold_factor
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc)]
+    return int(f(ctypes.byref(desc)))
+
+
+def ssconv_fold_desc(desc: Desc, f: int) -> Desc:
+    """Descriptor of the layer with f output pixels of a row folded into f * C_out output channels."""
+    out = Desc()
+    fn = lib().ssconv_fold_desc
+    fn.restype = ctypes.c_int32
+    fn.argtypes = [ctypes.POINTER(Desc), ctypes.c_int32, ctypes.POINTER(Desc)]
+    _check("ssconv_fold_desc", fn(ctypes.byref(desc), int(f), ctypes.byref(out)))
+    return out
+
+
+def ssconv_fold_weights(desc: Desc, f: int, w: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                        stream=None):
+    """(w_folded, bias_folded) for ssconv_fold_desc(desc, f).  w: any tensor of C_out*KH*KW equal vectors (bf16 or
+    e4m3 weights [C_out,KH,KW,C_in], patterns [G]); w_folded has the same dtype and f*C_out*KH*KW' vectors."""
+    _need_cuda(w, bias)
+    folded = ssconv_fold_desc(desc, f)
+    w2 = b2 = None
+    tap = 0
+    if w is not None:
+        vecs = desc.C_out * desc.KH * desc.KW
+        assert w.is_contiguous() and w.numel() % vecs == 0
+        per = w.numel() // vecs
+        tap = per * w.element_size()
+        w2 = torch.empty((folded.C_out, folded.KH, folded.KW, per), dtype=w.dtype, device=w.device)
+        if w.dim() == 1:
+            w2 = w2.view(-1)
+    if bias is not None:
+        assert bias.dtype == torch.float32
+        b2 = torch.empty((folded.C_out,), dtype=torch.float32, device=bias.device)
+    fn = lib().ssconv_fold_weights
+    fn.restype = ctypes.c_int32
+    fn.argtypes = [ctypes.POINTER(Desc), ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    _check("ssconv_fold_weights", fn(ctypes.byref(desc), int(f), _ptr(w), _ptr(w2), tap, _ptr(bias), _ptr(b2),
+                                     _stream(stream)))
+    return w2, b2
 
 
 def ssconv_forward_dense_strided(desc: Desc, x: torch.Tensor, strides, w: torch.Tensor,

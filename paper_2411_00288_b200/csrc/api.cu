@@ -45,6 +45,8 @@ int32_t set_tuning(int32_t option, int32_t value);
 cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad,
                            cudaStream_t st);
 cudaError_t launch_pad_channels(const void* x, void* y, long long pixels, int C, int C_pad, cudaStream_t st);
+cudaError_t launch_fold_weights(const void* w, void* out, int C_out, int KH, int KW, int KWf, int s, int d, int f,
+                                long long tap_bytes, const float* bias, float* bias_out, cudaStream_t st);
 cudaError_t launch_unfold_w(const void* x, void* y, long long rows, int W, int C, int KW, int stride, int pad, int dil,
                             int C_pad, cudaStream_t st);
 int32_t plan_query(const ssconv_desc_t& d, bool sparse, int32_t* bn, int32_t* split, int32_t* ctas,
@@ -343,11 +345,67 @@ int32_t ssconv_space_to_depth(const void* x, void* y, int32_t N, int32_t H, int3
                               int32_t pad, int32_t Hb, int32_t Wb, int32_t C_pad, void* stream) {
   if (!x || !y) return SSCONV_ERR_NULL;
   if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || block <= 0 || pad < 0 || Hb <= 0 || Wb <= 0) return SSCONV_ERR_BAD_DESC;
-  if (C_pad % 8 != 0 || (long long)block * block * C > C_pad) return SSCONV_ERR_UNSUPPORTED_SHAPE;
-  if ((reinterpret_cast<uintptr_t>(x) & 1u) || !aligned16(y)) return SSCONV_ERR_ALIGNMENT;
+  if (C_pad % 4 != 0 || (long long)block * block * C > C_pad) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(x) & 1u) || (reinterpret_cast<uintptr_t>(y) & (C_pad % 8 == 0 ? 15u : 7u)))
+    return SSCONV_ERR_ALIGNMENT;
   if ((long long)N * Hb > 0x7FFFFFFFLL || (long long)Wb * C_pad > 0x7FFFFFFFLL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
-  if ((long long)Wb * (C_pad / 8) > 65535LL * 256) return SSCONV_ERR_UNSUPPORTED_SHAPE;  // grid limit along a row
+  if ((long long)Wb * (C_pad / 4) > 65535LL * 256) return SSCONV_ERR_UNSUPPORTED_SHAPE;  // grid limit along a row
   return ssconv::launch_space_to_depth(x, y, N, H, W, C, block, pad, Hb, Wb, C_pad, (cudaStream_t)stream) == cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+// ---- folding of neighbouring output pixels into the output channels
+static int32_t fold_geometry(const ssconv_desc_t* d, int32_t f, int* KWf, int* Wo) {
+  if (!d) return SSCONV_ERR_NULL;
+  if (d->N <= 0 || d->H <= 0 || d->W <= 0 || d->C_in <= 0 || d->C_out <= 0 || d->KH <= 0 || d->KW <= 0 ||
+      d->stride_w <= 0 || d->stride_h <= 0 || d->dil_w <= 0 || d->dil_h <= 0 || d->pad_w < 0 || d->pad_h < 0)
+    return SSCONV_ERR_BAD_DESC;
+  if (f < 1 || f > 16) return SSCONV_ERR_BAD_DESC;
+  const long long span = (long long)d->W + 2LL * d->pad_w - (long long)d->dil_w * (d->KW - 1) - 1;
+  if (span < 0) return SSCONV_ERR_BAD_DESC;
+  *Wo = (int)(span / d->stride_w) + 1;
+  if (*Wo % f != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  const long long kwf = (long long)(f - 1) * d->stride_w + (long long)(d->KW - 1) * d->dil_w + 1;
+  if (kwf > 0x7FFF || (long long)f * d->C_out > 0x7FFFFFFFLL || (long long)f * d->stride_w > 0x7FFF)
+    return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  *KWf = (int)kwf;
+  return SSCONV_OK;
+}
+
+int32_t ssconv_fold_desc(const ssconv_desc_t* desc, int32_t f, ssconv_desc_t* folded) {
+  if (!folded) return SSCONV_ERR_NULL;
+  int KWf = 0, Wo = 0;
+  const int32_t rc = fold_geometry(desc, f, &KWf, &Wo);
+  if (rc != SSCONV_OK) return rc;
+  *folded = *desc;
+  folded->C_out = desc->C_out * f;
+  folded->KW = KWf;
+  folded->stride_w = desc->stride_w * f;
+  folded->dil_w = 1;
+  return SSCONV_OK;
+}
+
+int32_t ssconv_fold_factor(const ssconv_desc_t* desc) {
+  int KWf = 0, Wo = 0;
+  if (fold_geometry(desc, 2, &KWf, &Wo) != SSCONV_OK) return 1;
+  // Tiles have 128 accumulator rows whatever C_out is: with two pixels per row block the multiply-adds
+  // issued per output change by KW' / (2 KW); worth it from 15 % on.
+  if (desc->C_out > 64 || desc->C_out % 8 != 0) return 1;
+  return (20LL * KWf <= 17LL * 2 * desc->KW) ? 2 : 1;
+}
+
+int32_t ssconv_fold_weights(const ssconv_desc_t* desc, int32_t f, const void* w, void* w_folded, int64_t tap_bytes,
+                            const float* bias, float* bias_folded, void* stream) {
+  int KWf = 0, Wo = 0;
+  const int32_t rc = fold_geometry(desc, f, &KWf, &Wo);
+  if (rc != SSCONV_OK) return rc;
+  if ((w == nullptr) != (w_folded == nullptr) || (bias == nullptr) != (bias_folded == nullptr)) return SSCONV_ERR_NULL;
+  if (w != nullptr && (tap_bytes <= 0 || tap_bytes > 0x7FFFFFFFLL)) return SSCONV_ERR_BAD_DESC;
+  if ((long long)f * desc->C_out * desc->KH * KWf > (0x7FFFFFFFLL * 256) / (tap_bytes > 0 ? tap_bytes : 1))
+    return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  return ssconv::launch_fold_weights(w, w_folded, desc->C_out, desc->KH, desc->KW, KWf, desc->stride_w, desc->dil_w, f,
+                                     tap_bytes, bias, bias_folded, (cudaStream_t)stream) == cudaSuccess
              ? SSCONV_OK
              : SSCONV_ERR_CUDA;
 }

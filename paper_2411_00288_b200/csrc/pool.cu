@@ -103,23 +103,24 @@ __global__ void __launch_bounds__(256) pad_channels_kernel(const __nv_bfloat16* 
 // pad over x is then a ceil(K/s) x ceil(K/s) convolution of unit stride and no padding over y (with
 // weights rearranged by the same call, as K x K "images" with pad 0), when Hb = H_out + ceil(K/s) - 1
 // rows are produced: few-channel images turn into pixels wide enough for the tensor-core path without
-// the (K-fold) duplication of an unfold.  One thread per 16 bytes of y; scalar reads.
-__global__ void __launch_bounds__(256) space_to_depth_kernel(const unsigned short* __restrict__ x, uint4* __restrict__ y,
+// the (K-fold) duplication of an unfold.  One thread per V channels (16 or 8 bytes) of y; scalar reads.
+template <int V>
+__global__ void __launch_bounds__(256) space_to_depth_kernel(const unsigned short* __restrict__ x, uint32_t* __restrict__ y,
                                                              int H, int W, int C, int s, int pad, int Hb, int Wb,
-                                                             int Cp8) {
-  // one grid row per row of y (n, r); threads along the row's 16-byte chunks (q, k)
+                                                             int CpV) {
+  // one grid row per row of y (n, r); threads along the row's chunks of V channels (q, k)
   const int col = blockIdx.y * blockDim.x + threadIdx.x;
-  if (col >= Wb * Cp8) return;
+  if (col >= Wb * CpV) return;
   const int row = blockIdx.x;
   const int n = row / Hb, r = row - n * Hb;
-  const int q = col / Cp8, k = col - q * Cp8;
-  // channel 8 k of the pixel = (block pixel blk = bh s + bw, channel c); the next seven follow incrementally
-  int blk = (8 * k) / C, c = 8 * k - blk * C;
+  const int q = col / CpV, k = col - q * CpV;
+  // channel V k of the pixel = (block pixel blk = bh s + bw, channel c); the next V - 1 follow incrementally
+  int blk = (V * k) / C, c = V * k - blk * C;
   int bh = blk / s, bw = blk - bh * s;
   const unsigned short* img = x + (size_t)n * H * W * C;
-  unsigned short v[8];
+  unsigned short v[V];
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
+  for (int j = 0; j < V; ++j) {
     const int h = s * r - pad + bh, w = s * q - pad + bw;
     v[j] = (bh < s && h >= 0 && h < H && w >= 0 && w < W) ? __ldg(img + ((size_t)h * W + w) * C + c) : (unsigned short)0;
     if (++c == C) {
@@ -130,21 +131,129 @@ __global__ void __launch_bounds__(256) space_to_depth_kernel(const unsigned shor
       }
     }
   }
-  uint4 o;
-  o.x = v[0] | ((uint32_t)v[1] << 16);
-  o.y = v[2] | ((uint32_t)v[3] << 16);
-  o.z = v[4] | ((uint32_t)v[5] << 16);
-  o.w = v[6] | ((uint32_t)v[7] << 16);
-  y[(size_t)row * Wb * Cp8 + col] = o;
+  uint32_t* dst = y + ((size_t)row * Wb * CpV + col) * (V / 2);
+  if (V == 8) {
+    *reinterpret_cast<uint4*>(dst) = make_uint4(v[0] | ((uint32_t)v[1] << 16), v[2] | ((uint32_t)v[3] << 16),
+                                                v[4 % V] | ((uint32_t)v[5 % V] << 16), v[6 % V] | ((uint32_t)v[7 % V] << 16));
+  } else {
+    *reinterpret_cast<uint2*>(dst) = make_uint2(v[0] | ((uint32_t)v[1] << 16), v[2] | ((uint32_t)v[3] << 16));
+  }
+}
+
+// The same for RGB images, blocks of 2 x 2 pixels and unpadded pixels of 12 channels (24 bytes): a row
+// of y interleaves 12-byte pieces of two image rows, so a block stages the two rows in shared memory
+// (16-byte loads; element (w + pad) 3 + c of a staged row is channel c of column w, zeros outside the
+// image) and writes the row of y as 8-byte words: pixel q is elements 6 q .. 6 q + 5 of the first row,
+// then of the second.  Every image byte is read once and every byte of y written once.
+__global__ void __launch_bounds__(128) space_to_depth_rgb2_kernel(const uint4* __restrict__ x, uint2* __restrict__ y, int H,
+                                                                  int W, int pad, int Hb, int Wb) {
+  extern __shared__ uint32_t s2d_rows[];  // two rows of 3 Wb words (6 Wb elements)
+  const int row = blockIdx.x;
+  const int n = row / Hb, r = row - n * Hb;
+  const int words = 3 * Wb;
+  unsigned short* el = reinterpret_cast<unsigned short*>(s2d_rows);
+  const int lead = pad * 3, body = W * 3, len = 6 * Wb;
+#pragma unroll
+  for (int dy = 0; dy < 2; ++dy) {
+    const int h = 2 * r - pad + dy;
+    unsigned short* dst = el + dy * len;
+    if (h < 0 || h >= H) {
+      for (int i = threadIdx.x; i < words; i += blockDim.x) s2d_rows[dy * words + i] = 0u;
+      continue;
+    }
+    for (int i = threadIdx.x; i < lead; i += blockDim.x) dst[i] = 0;
+    for (int i = lead + body + threadIdx.x; i < len; i += blockDim.x) dst[i] = 0;
+    const uint4* src = x + ((size_t)n * H + h) * (size_t)(body / 8);
+    for (int i = threadIdx.x; i < body / 8; i += blockDim.x) {
+      const uint4 v = __ldg(src + i);
+      const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int e = lead + 8 * i + 2 * j;
+        if (e < len) dst[e] = (unsigned short)(wv[j] & 0xFFFFu);
+        if (e + 1 < len) dst[e + 1] = (unsigned short)(wv[j] >> 16);
+      }
+    }
+  }
+  __syncthreads();
+  uint2* out = y + (size_t)row * words;
+  const uint32_t* r0 = s2d_rows;
+  const uint32_t* r1 = s2d_rows + words;
+  for (int u = threadIdx.x; u < words; u += blockDim.x) {
+    const int q = u / 3, part = u - 3 * q;
+    uint2 o;
+    if (part == 0) o = make_uint2(r0[3 * q], r0[3 * q + 1]);
+    else if (part == 1) o = make_uint2(r0[3 * q + 2], r1[3 * q]);
+    else o = make_uint2(r1[3 * q + 1], r1[3 * q + 2]);
+    out[u] = o;
+  }
 }
 
 cudaError_t launch_space_to_depth(const void* x, void* y, int N, int H, int W, int C, int s, int pad, int Hb, int Wb,
                                   int C_pad, cudaStream_t st) {
-  const int T = 256;
-  const int per_row = Wb * (C_pad / 8);
   count_launch();
-  space_to_depth_kernel<<<dim3((unsigned)(N * Hb), (unsigned)((per_row + T - 1) / T)), T, 0, st>>>(
-      static_cast<const unsigned short*>(x), static_cast<uint4*>(y), H, W, C, s, pad, Hb, Wb, C_pad / 8);
+  if (s == 2 && C == 3 && C_pad == 12 && W % 8 == 0 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && Wb <= 1024) {
+    space_to_depth_rgb2_kernel<<<(unsigned)(N * Hb), 128, (size_t)Wb * 24, st>>>(
+        static_cast<const uint4*>(x), static_cast<uint2*>(y), H, W, pad, Hb, Wb);
+    return cudaGetLastError();
+  }
+  const int T = 256;
+  if (C_pad % 8 == 0) {
+    const int per_row = Wb * (C_pad / 8);
+    space_to_depth_kernel<8><<<dim3((unsigned)(N * Hb), (unsigned)((per_row + T - 1) / T)), T, 0, st>>>(
+        static_cast<const unsigned short*>(x), static_cast<uint32_t*>(y), H, W, C, s, pad, Hb, Wb, C_pad / 8);
+  } else {
+    const int per_row = Wb * (C_pad / 4);
+    space_to_depth_kernel<4><<<dim3((unsigned)(N * Hb), (unsigned)((per_row + T - 1) / T)), T, 0, st>>>(
+        static_cast<const unsigned short*>(x), static_cast<uint32_t*>(y), H, W, C, s, pad, Hb, Wb, C_pad / 4);
+  }
+  return cudaGetLastError();
+}
+
+// Folding of f neighbouring output pixels of a row into the output channels (a rearrangement of the
+// weights of Eq. 4, no arithmetic): output pixel f i + j of a convolution with KW taps of stride s and
+// dilation d along the width is channel block j of pixel i of a convolution with
+// KW' = (f - 1) s + (KW - 1) d + 1 undilated taps of stride f s,
+//   W'[j C_out + c, kh, kw', :] = W[c, kh, kw, :]  where kw' = j s + kw d,   0 elsewhere.
+// A layer of C_out <= 64 fills the 128 accumulator rows of a tile this way instead of half of them.
+// Bytes, not elements: `tap` is the size of one (row, tap) vector, so the same kernel moves bf16 or
+// 8-bit weights and the 2:4 patterns of their groups (whose groups of four lie inside one tap vector).
+__global__ void __launch_bounds__(256) fold_weights_kernel(const uint8_t* __restrict__ w, uint8_t* __restrict__ out,
+                                                           long long total, int C_out, int KH, int KW, int KWf, int s, int d,
+                                                           int tap) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int b = (int)(i % tap);
+  long long t = i / tap;
+  const int kwf = (int)(t % KWf);
+  t /= KWf;
+  const int kh = (int)(t % KH);
+  const int row = (int)(t / KH);
+  const int j = row / C_out, c = row - j * C_out;
+  const int off = kwf - j * s;
+  uint8_t v = 0;
+  if (off >= 0 && off % d == 0 && off / d < KW) v = w[(((long long)c * KH + kh) * KW + off / d) * tap + b];
+  out[i] = v;
+}
+__global__ void fold_bias_kernel(const float* __restrict__ bias, float* __restrict__ out, int C_out, int total) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < total) out[i] = bias[i % C_out];
+}
+
+cudaError_t launch_fold_weights(const void* w, void* out, int C_out, int KH, int KW, int KWf, int s, int d, int f,
+                                long long tap_bytes, const float* bias, float* bias_out, cudaStream_t st) {
+  const long long total = (long long)f * C_out * KH * KWf * tap_bytes;
+  if (w != nullptr && total > 0) {
+    count_launch();
+    fold_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(static_cast<const uint8_t*>(w),
+                                                                       static_cast<uint8_t*>(out), total, C_out, KH, KW,
+                                                                       KWf, s, d, (int)tap_bytes);
+    if (cudaGetLastError() != cudaSuccess) return cudaErrorUnknown;
+  }
+  if (bias != nullptr) {
+    count_launch();
+    fold_bias_kernel<<<(unsigned)((f * C_out + 255) / 256), 256, 0, st>>>(bias, bias_out, C_out, f * C_out);
+  }
   return cudaGetLastError();
 }
 

@@ -39,10 +39,21 @@ class ConvStack:
                 w = inp.w.to(self.device)
                 bias = inp.bias.to(self.device) if inp.bias is not None else None
                 entry = dict(desc=desc, w=None, bias=bias, w_comp=None, meta=None, w_host=inp.w, bias_host=inp.bias)
+                fold = api.ssconv_fold_factor(desc) if st.kind == "conv" else 1
+                entry["fold"] = fold
                 if st.kind == "conv":
                     pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
-                    entry["w_comp"], entry["meta"] = api.ssconv_compress(desc, w, pat)
                     entry["pattern"] = pat
+                    if fold > 1:
+                        # neighbouring output pixels as extra output channels: weights, patterns and bias are
+                        # rearranged once, the layer then runs under the folded descriptor on the same bytes
+                        entry["desc"] = api.ssconv_fold_desc(desc, fold)
+                        w_f, entry["bias"] = api.ssconv_fold_weights(desc, fold, w, bias)
+                        pat_f, _ = api.ssconv_fold_weights(desc, fold, pat)
+                        entry["w_comp"], entry["meta"] = api.ssconv_compress(entry["desc"], w_f, pat_f)
+                        w = w_f
+                    else:
+                        entry["w_comp"], entry["meta"] = api.ssconv_compress(desc, w, pat)
                 if st.kind == "dense" or with_dense:
                     entry["w"] = w
                 if st.kind == "dense" and spec.C_in == 8 and spec.KW > 1:
@@ -55,29 +66,42 @@ class ConvStack:
                                            stride=(spec.stride, 1), pad=(spec.pad, 0), dil=(spec.dil, 1),
                                            bias=spec.has_bias, relu=spec.relu and not spec.gelu, gelu=spec.gelu))
                 if st.kind == "dense" and spec.C_in == 8 and spec.KH == spec.KW and spec.stride > 1 and st.src < 0:
-                    entry["s2d"] = self._prepare_s2d(spec, w, real_c=3)
+                    entry["s2d"] = self._prepare_s2d(spec, w, real_c=3, bias=bias)
                 self.layers.append(entry)
                 shape = (spec.N, spec.H_out, spec.W_out, spec.C_out)
             shapes.append(shape)
             self.outputs.append(torch.empty(shape, dtype=torch.bfloat16, device=self.device))
         torch.cuda.synchronize(self.device)
 
-    def _prepare_s2d(self, spec, w: torch.Tensor, real_c: int):
+    def _prepare_s2d(self, spec, w: torch.Tensor, real_c: int, bias: Optional[torch.Tensor]):
         """Buffers, weights and descriptor of the space-to-depth form of a K x K stride-s layer on images
-        of `real_c` channels: blocks of s x s pixels become one pixel of C_pad channels, T = ceil(K/s)
-        neighbouring block pixels are read as one pixel of T*C_pad channels, and the layer is a T x 1
-        convolution of unit stride without padding over that view."""
+        of `real_c` channels: blocks of s x s pixels become one pixel of C_pad channels, and the layer is a
+        T x T convolution of unit stride without padding over them, T = ceil(K/s).  With few output
+        channels two output pixels of a row are folded into the output channels (T + 1 taps of stride 2
+        along the width); the taps of a row are then read as one pixel of 64 channels through a sliding
+        window over neighbouring block pixels, which leaves a T x 1 convolution for the tensor cores."""
         s, K = spec.stride, spec.KH
         T = -(-K // s)
-        c_pad = -(-s * s * real_c // 8) * 8
-        hb, wb = spec.H_out + T - 1, spec.W_out + T - 1
+        c_blk = s * s * real_c
+        c_pad = -(-c_blk // 4) * 4
         w_real = w[..., :real_c].contiguous()
         w_s2d = api.ssconv_space_to_depth(w_real, s, 0, T, T, c_pad)          # [C_out, T, T, c_pad]
-        desc = api.make_desc(spec.N, hb, spec.W_out, T * c_pad, spec.C_out, T, 1, stride=1, pad=0, dil=1,
+        hb, wb = spec.H_out + T - 1, spec.W_out + T - 1
+        conv = api.make_desc(spec.N, hb, wb, c_pad, spec.C_out, T, T, stride=1, pad=0, dil=1)
+        f = 2 if (2 * spec.C_out <= 128 and spec.W_out % 2 == 0 and (T + 1) * c_pad <= 64 and (2 * c_pad) % 8 == 0) else 1
+        taps = T + f - 1
+        c_view = -(-taps * c_pad // 64) * 64
+        wb += wb % 2                                                            # row pitch a multiple of 16 bytes
+        w_f, bias_f = api.ssconv_fold_weights(conv, f, w_s2d, bias)            # [f C_out, T, taps, c_pad]
+        w_view = api.ssconv_pad_channels(w_f.view(-1, taps * c_pad), C_pad=c_view).view(f * spec.C_out, T, 1, c_view)
+        desc = api.make_desc(spec.N, hb, spec.W_out // f, c_view, f * spec.C_out, T, 1, stride=1, pad=0, dil=1,
                              bias=spec.has_bias, relu=spec.relu and not spec.gelu, gelu=spec.gelu)
-        return dict(block=s, pad=spec.pad, hb=hb, wb=wb, c_pad=c_pad, real_c=real_c, w=w_s2d, desc=desc,
-                    strides=(c_pad, wb * c_pad, hb * wb * c_pad),
-                    x=torch.empty((spec.N, hb, wb, c_pad), dtype=torch.bfloat16, device=self.device))
+        # the window of the last pixel of the last row ends c_view - taps*c_pad channels past the buffer's rows
+        slack = c_view
+        buf = torch.zeros((spec.N * hb * wb * c_pad + slack,), dtype=torch.bfloat16, device=self.device)
+        return dict(block=s, pad=spec.pad, hb=hb, wb=wb, c_pad=c_pad, real_c=real_c, w=w_view, bias=bias_f, desc=desc,
+                    fold=f, strides=(f * c_pad, wb * c_pad, hb * wb * c_pad),
+                    x=buf[:spec.N * hb * wb * c_pad].view(spec.N, hb, wb, c_pad))
 
     def run_step(self, i: int, x: torch.Tensor, sparse: bool = True) -> torch.Tensor:
         """Enqueue step i alone (its input must already be in place); returns its output tensor."""
@@ -95,7 +119,7 @@ class ConvStack:
         elif "s2d" in L and src.shape[-1] == L["s2d"]["real_c"]:
             S = L["s2d"]
             api.ssconv_space_to_depth(src, S["block"], S["pad"], S["hb"], S["wb"], S["c_pad"], y=S["x"])
-            api.ssconv_forward_dense_strided(S["desc"], S["x"], S["strides"], S["w"], L["bias"], y=y,
+            api.ssconv_forward_dense_strided(S["desc"], S["x"], S["strides"], S["w"], S["bias"], y=y,
                                              dev_status=self.status)
         elif "unfold" in L:
             U = L["unfold"]
