@@ -320,13 +320,18 @@ def sweep_measure(cfg, api, synth, torch, tm, dev, peaks, l2_bytes, steps, regio
             pat = api.ssconv_select_mask(api.MASK_LOGITS_F32, inp.scores.to(dev), spec.G)
         else:
             pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
+        fold = api.ssconv_fold_factor(desc)
+        if fold > 1:   # few output channels: neighbouring output pixels as extra output channels, same bytes out
+            w, bias_f = api.ssconv_fold_weights(desc, fold, w, bias)
+            pat, _ = api.ssconv_fold_weights(desc, fold, pat)
+            desc, bias = api.ssconv_fold_desc(desc, fold), bias_f
         w_comp, meta = api.ssconv_compress(desc, w, pat)
         xs = [inp.x.to(dev)]
         for _ in range(1, n_sets):   # further buffer sets only rotate the traffic: drawn on the device
             xs.append(torch.randn(inp.x.shape, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16))
         ys = [torch.empty((spec.N, spec.H_out, spec.W_out, spec.C_out), dtype=torch.bfloat16, device=dev)
               for _ in range(n_sets)]
-        entry = dict(spec=spec, desc=desc, w=w, bias=bias, w_comp=w_comp, meta=meta, xs=xs, ys=ys)
+        entry = dict(spec=spec, desc=desc, w=w, bias=bias, w_comp=w_comp, meta=meta, xs=xs, ys=ys, fold=fold)
         if want_e2e:
             entry["x_host"] = inp.x.pin_memory()
             entry["y_host"] = torch.empty(ys[0].shape, dtype=torch.bfloat16).pin_memory()
@@ -377,7 +382,7 @@ def sweep_measure(cfg, api, synth, torch, tm, dev, peaks, l2_bytes, steps, regio
                           "tflops": round(flops / res[True] / 1e9, 1), "gbs": round(bytes_alg / res[True] / 1e6, 1),
                           "bound": "tensor" if t_c >= t_m else "hbm", "us_roofline": round(roof * 1e3, 2),
                           "roofline_frac": round(roof / res[True], 4), "x_dense": round(res[False] / res[True], 3),
-                          "plan": api.ssconv_plan(L["desc"], True)})
+                          "plan": dict(api.ssconv_plan(L["desc"], True), fold=L["fold"])})
     total_flops = sum(s.dense_equiv_flops for s in layers)
     out = dict(layers=layers, prep=prep, n_sets=n_sets, set_bytes=set_bytes, prep_seconds=prep_seconds,
                launches_per_step=launches_per_step, ms_sparse=ms_sparse, ms_dense=ms_dense, per_layer=per_layer,
@@ -653,7 +658,7 @@ def stack_arm(args):
             if masked:
                 row["us_dense"] = round(res[False] * 1e3, 2)
                 row["x_dense"] = round(res[False] / t, 3)
-                row["plan"] = api.ssconv_plan(net.layers[i]["desc"], True)
+                row["plan"] = dict(api.ssconv_plan(net.layers[i]["desc"], True), fold=net.layers[i]["fold"])
                 sums["t_masked"] += t
                 sums["t_dense_masked"] += res[False]
                 sums["roof_masked"] += max(t_c, t_m)

@@ -1307,6 +1307,7 @@ static double kblock_cycles(int BN, int stage_bufs, bool steady_ring = true) {
 
 // Process-wide overrides of the planner (ssconv_tune): tile width (0 lets the model choose) and the
 // use of the pair kernel.
+int32_t wgrad_set_tuning(int32_t option, int32_t value);  // (wgrad.cu)
 static int g_tune_bn = 0;
 static int g_tune_pair = -1;  // -1: the model chooses; 0: never the pair kernel; 1: wherever it applies
 int32_t set_tuning(int32_t option, int32_t value) {
@@ -1320,7 +1321,7 @@ int32_t set_tuning(int32_t option, int32_t value) {
     g_tune_bn = value;
     return SSCONV_OK;
   }
-  return SSCONV_ERR_BAD_DESC;
+  return wgrad_set_tuning(option, value);
 }
 
 // Tile width and partition of a layer.

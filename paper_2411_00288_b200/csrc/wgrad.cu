@@ -253,6 +253,255 @@ ssconv_wgrad_kernel(const __grid_constant__ CUtensorMap tm_dy, const __grid_cons
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// The same product on CTA pairs (tcgen05.mma cta_group::2), transposed:
+//
+//   dW^T[K x C_out] = U(X)[K x Q] * dY[Q x C_out]
+//
+// A pair owns four k-blocks (M = 256 rows of dW^T: each CTA loads the activation tiles of its two
+// k-blocks, 128 rows) x one tile of NT = 128 or 256 output channels (each CTA loads the gradient
+// tiles of its half of them) x one range of positions, walked 128 positions at a time through a
+// three-stage ring.  Against the one-CTA kernel above, every byte staged in shared memory serves
+// twice the multiply-adds (the other CTA's tensor core reads it too), which is what that kernel is
+// bound by; and since the accumulator's lanes now run along K, a warp's 32 lanes write 128 contiguous
+// bytes of dW [C_out][K] itself: the slices of the position ranges have the layout of the result (a
+// CTA's part of the tile is staged in shared memory and leaves as two-dimensional bulk copies) and the
+// second kernel only adds them, in slice order.
+// Layout of a stage in each CTA: two activation tiles, then two gradient tiles, 128 positions x 64
+// channels (16 KB) each, position-major in the 128-byte swizzle as above.  Barriers as in the forward
+// pair kernel: "full" lives in the even CTA (the leader) and collects the bytes of both CTAs' loads,
+// "empty" and "accumulator complete" exist in both and the leader commits to both.  No load is
+// multicast.  Tiles that lie outside the tensors (k-blocks past the last one, channels past C_out,
+// positions past Q) are loaded all the same and arrive as zeros.
+constexpr int kWpThreads = 256;        // warp 0: activation loads, warp 1: MMA (leader), warp 2: gradient loads, 4-7: epilogue
+constexpr int kWpPos = 128;            // positions per ring stage
+constexpr int kWpStages = 3;
+constexpr uint32_t kWpTileBytes = kWpPos * 128;
+constexpr uint32_t kWpStageBytes = 4 * kWpTileBytes;
+constexpr uint32_t kWpTmemCols = 256;
+constexpr uint32_t kWpSmemBytes = 1024 + kWpStages * kWpStageBytes + 256;
+
+struct WpParams {
+  int C_in, C_out, Ho, Wo;
+  int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
+  int taps, kblocks, cblocks;
+  int kgroups, n_tiles, NT;
+  int ksteps, ksteps_per_split;
+  int32_t* dev_status;
+};
+
+__device__ __forceinline__ uint32_t wp_desc_lo(uint32_t smem_addr) {
+  return ((smem_addr & 0x3FFFFu) >> 4) | ((kWpTileBytes >> 4) << 16);
+}
+
+__global__ void __launch_bounds__(kWpThreads, 1)
+ssconv_wgrad_pair_kernel(const __grid_constant__ CUtensorMap tm_dy, const __grid_constant__ CUtensorMap tm_x,
+                         const __grid_constant__ CUtensorMap tm_dw, const WpParams p) {
+  extern __shared__ uint8_t wp_smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(wp_smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kWpStages * kWpStageBytes);
+  uint64_t* bar_full = bars;                  // [kWpStages], used in the leader
+  uint64_t* bar_empty = bars + kWpStages;     // [kWpStages]
+  uint64_t* bar_acc = bars + 2 * kWpStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kWpStages + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  // item of this pair: (range of positions, tile of output channels, group of four k-blocks)
+  int i = (int)(blockIdx.x >> 1);
+  const int kg = i % p.kgroups;
+  i /= p.kgroups;
+  const int nt = i % p.n_tiles;
+  const int split = i / p.n_tiles;
+  const int ks0 = split * p.ksteps_per_split;
+  const int ks1 = min(p.ksteps, ks0 + p.ksteps_per_split);
+  const int b_first = 4 * kg + 2 * (int)rank;   // this CTA's two k-blocks
+  const int n_half = p.NT >> 1;                 // this CTA's gradient channels: n_first .. n_first + n_half
+  const int n_first = nt * p.NT + (int)rank * n_half;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int s = 0; s < kWpStages; ++s) {
+        mbar_init(&bar_full[s], 2u);   // the leader's two producer warps
+        mbar_init(&bar_empty[s], 1u);
+      }
+      mbar_init(bar_acc, 1u);
+      *abort_flag = 0;
+      mbar_fence_init();
+      fence_proxy_async_smem();
+      prefetch_tensormap(&tm_dy);
+      prefetch_tensormap(&tm_x);
+      prefetch_tensormap(&tm_dw);
+      grid_launch_dependents();   // (the adding kernel waits for this grid's completion itself)
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    tmem_alloc2(tmem_slot, kWpTmemCols);
+    tmem_relinquish2();
+  }
+  // both CTAs' barriers and TMEM exist before either touches the other's
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t full0_local = smem_u32(bar_full), empty0 = smem_u32(bar_empty), ring0 = smem_u32(smem);
+  const uint32_t full0_leader = map_to_cta(full0_local, 0);
+
+  if (warp == 0 || warp == 2) {
+    // ------------------------------------------------------------------ TMA producers (whole warps)
+    uint32_t s = 0, ph = 0;
+    int cc[2], kh[2], kw[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const int b = b_first + t;
+      // (a k-block past the last one reads the channel chunk after the last: zeros)
+      cc[t] = b < p.kblocks ? b / p.taps : p.cblocks;
+      const int tap = b < p.kblocks ? b - cc[t] * p.taps : 0;
+      kh[t] = tap / p.KW;
+      kw[t] = tap - kh[t] * p.KW;
+    }
+    grid_dependency_wait();   // everything above may overlap the tail of the kernel before this one
+    for (int ks = ks0; ks < ks1; ++ks) {
+      if (!mbar_wait_a(empty0 + 8u * s, ph ^ 1u, abort_flag, kWgWaitLimitCycles)) break;
+      const uint32_t full = full0_leader + 8u * s;
+      const uint32_t dst = ring0 + s * kWpStageBytes;
+      const int q0 = ks * kWpPos;
+      if (warp == 0) {
+        if (rank == 0) mbar_expect_tx_w(full0_local + 8u * s, 4u * kWpTileBytes);   // both CTAs' activation tiles
+        const int rho = q0 / p.Wo;
+        const int wo = q0 - rho * p.Wo;
+        const int n = rho / p.Ho;
+        const int ho = rho - n * p.Ho;
+        const int base_w = wo * p.stride_w - p.pad_w;
+        const int base_h = ho * p.stride_h - p.pad_h;
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+          tma2_load_im2col_4d_w(dst + (uint32_t)t * kWpTileBytes, &tm_x, full, cc[t] * kBlockK, base_w, base_h, n,
+                                (uint16_t)(kw[t] * p.dil_w), (uint16_t)(kh[t] * p.dil_h));
+      } else {
+        const uint32_t tiles = (uint32_t)(n_half >> 6);
+        if (rank == 0) mbar_expect_tx_w(full0_local + 8u * s, 2u * tiles * kWpTileBytes);
+        for (uint32_t t = 0; t < tiles; ++t)
+          tma2_load_2d_w(dst + (2u + t) * kWpTileBytes, &tm_dy, full, n_first + 64 * (int)t, q0);
+      }
+      if (++s == kWpStages) {
+        s = 0;
+        ph ^= 1u;
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only, whole warp)
+    if (rank == 0) {
+      const uint32_t idesc = make_idesc_bf16(2 * kTileM, (uint32_t)p.NT, false) | (1u << 15) | (1u << 16);
+      uint32_t s = 0, ph = 0, accumulate = 0;
+      bool ok = true;
+      for (int ks = ks0; ks < ks1; ++ks) {
+        if (!mbar_wait_a(full0_local + 8u * s, ph, abort_flag, kWgWaitLimitCycles)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t a_lo = wp_desc_lo(ring0 + s * kWpStageBytes);
+        const uint32_t b_lo = a_lo + ((2u * kWpTileBytes) >> 4);
+        // 16 positions per MMA = two groups of 8 rows = 2048 B
+#pragma unroll
+        for (int k = 0; k < kWpPos / 16; ++k) {
+          tc2_mma_dense_w(tmem_base, a_lo + (uint32_t)k * 128u, b_lo + (uint32_t)k * 128u, idesc, accumulate);
+          accumulate = 1;
+        }
+        tc2_commit_both_w(empty0 + 8u * s);
+        if (++s == kWpStages) {
+          s = 0;
+          ph ^= 1u;
+        }
+      }
+      if (ok) tc2_commit_both_w(smem_u32(bar_acc));
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ epilogue
+    const int qd = warp & 3;  // TMEM lane quadrant of this warp
+    const bool got =
+        __all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar_acc, 0u, abort_flag, kWgWaitLimitCycles, 64) ? 1 : 0) != 0;
+    if (got) {
+      tc_fence_after();
+      // Lane row 32 qd + lane of this CTA = channel (32 qd + lane) % 64 of its k-block (32 qd + lane) / 64.
+      // The tile goes through shared memory (the ring is idle by now: every load has been consumed), as
+      // [k-block][output channel][64 channels] fp32, and from there to dW [C_out][taps][C_in] as boxes of
+      // 128 output channels x 64 channels: per-lane stores of 4 bytes would take several times the
+      // main loop of a short position range.  Rows and columns outside the tensor are clipped by the copy.
+      const uint32_t stage = ring0 + (uint32_t)(qd >> 1) * (uint32_t)p.NT * 256u + (uint32_t)((qd & 1) * 32 + lane) * 4u;
+      const int n0 = nt * p.NT;
+#pragma unroll 1
+      for (int j0 = 0; j0 < p.NT; j0 += 128) {
+        if (n0 + j0 >= p.C_out) break;   // (uniform over the warp)
+        uint32_t r[4][32];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          tc_ld_32x32b_x32(tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(j0 + 32 * u), r[u]);
+        tc_wait_ld();
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(stage + (uint32_t)(j0 + 32 * u + j) * 256u), "r"(r[u][j]) : "memory");
+        }
+      }
+      fence_proxy_async_smem();
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps
+    if (got && warp == 4 && lane == 0 && *abort_flag == 0) {
+      const int n0 = nt * p.NT;
+      grid_dependency_wait();
+      for (int t = 0; t < 2; ++t) {
+        const int b = b_first + t;
+        if (b >= p.kblocks) break;
+        const int ccb = b / p.taps;
+        const int tap = b - ccb * p.taps;
+        for (int j0 = 0; j0 < p.NT && n0 + j0 < p.C_out; j0 += 128)
+          tma_store_4d(&tm_dw, ring0 + (uint32_t)t * (uint32_t)p.NT * 256u + (uint32_t)j0 * 256u, ccb * kBlockK, tap,
+                       n0 + j0, split);
+      }
+      bulk_commit_group();
+      bulk_wait_group_read0();   // shared memory is released below; the writes complete with the grid
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  // Neither CTA may leave while the other can still signal its barriers or read its shared memory.
+  tc_fence_before();
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  if (*abort_flag != 0) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    if (threadIdx.x == 0 && p.dev_status != nullptr) atomicExch(p.dev_status, (int)SSCONV_ERR_TIMEOUT);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc2(tmem_base, kWpTmemCols);
+  }
+}
+
+// dW = the sum, in slice order, of `splits` slices of the same layout (four elements per thread).
+__global__ void __launch_bounds__(256) wgrad_sum_kernel(const float4* __restrict__ slices, int splits, size_t slice_vec,
+                                                        float4* __restrict__ dw) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  grid_dependency_wait();   // launched while the kernel that writes the slices is still running
+  if (i >= slice_vec) return;
+  float4 acc = slices[i];
+  for (int s = 1; s < splits; ++s) {
+    const float4 v = slices[(size_t)s * slice_vec + i];
+    acc.x += v.x;
+    acc.y += v.y;
+    acc.z += v.z;
+    acc.w += v.w;
+  }
+  dw[i] = acc;
+}
+
 // dW [C_out][K] = transpose of the sum, in slice order, of the slices [m_tiles][K][128].  A block
 // of 32 x 8 threads handles 32 output channels x 8 columns of K, one element per thread: reads are
 // contiguous along the output channels, writes go out as 32-byte runs along K.  With many slices
@@ -317,28 +566,55 @@ int wg_out_extent(int in, int k, int stride, int pad, int dil) {
 }
 
 bool g_wg_attr_set[64] = {false};
+int g_tune_wg_ranges = 0;   // 0: the planner chooses; otherwise an upper limit on the position ranges
+int g_tune_wg_pair = -1;    // -1: the planner chooses; 0: one-CTA kernel only; 1: the pair kernel wherever it applies
 
 // How a layer's weight gradient is cut into work items.
 struct WgPlan {
   int taps, kblocks, T, items_b, m_tiles, ksteps, splits, ksteps_per_split;
   long long Q;
+  bool pair;                 // the CTA-pair kernel
+  int kgroups, n_tiles, NT;  // its items: groups of four k-blocks x tiles of NT output channels
 };
 WgPlan wg_plan(const ssconv_desc_t& d, int sms) {
   WgPlan w;
   w.taps = d.KH * d.KW;
   w.kblocks = w.taps * ((d.C_in + kBlockK - 1) / kBlockK);
+  w.Q = (long long)d.N * wg_out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h) *
+        wg_out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
+  // CTA pairs whenever at least three of a pair's four k-blocks exist (its 256 accumulator rows run
+  // along K); layers with one or two k-blocks (1 x 1 convolutions over at most 128 channels) keep
+  // the one-CTA kernel, whose 128 rows run along C_out.
+  w.pair = (g_tune_wg_pair < 0 ? w.kblocks >= 3 : g_tune_wg_pair == 1) && sms >= 2;
+  if (w.pair) {
+    w.kgroups = (w.kblocks + 3) / 4;
+    w.NT = d.C_out > 128 ? 256 : 128;
+    w.n_tiles = (d.C_out + w.NT - 1) / w.NT;
+    w.ksteps = (int)((w.Q + kWpPos - 1) / kWpPos);
+    w.T = 4;
+    w.items_b = w.kgroups;
+    w.m_tiles = w.n_tiles;
+    const int items = w.kgroups * w.n_tiles;
+    int splits = (sms / 2) / items;
+    if (splits > w.ksteps / 4) splits = w.ksteps / 4;   // at least four steps of 128 positions per range
+    if (g_tune_wg_ranges > 0 && splits > g_tune_wg_ranges) splits = g_tune_wg_ranges;
+    if (splits < 1) splits = 1;
+    w.ksteps_per_split = (w.ksteps + splits - 1) / splits;
+    w.splits = (w.ksteps + w.ksteps_per_split - 1) / w.ksteps_per_split;
+    return w;
+  }
+  w.kgroups = w.n_tiles = w.NT = 0;
   const int groups = (w.kblocks + kWgMaxT - 1) / kWgMaxT;
   w.T = (w.kblocks + groups - 1) / groups;
   w.items_b = (w.kblocks + w.T - 1) / w.T;
   w.m_tiles = (d.C_out + kTileM - 1) / kTileM;
-  w.Q = (long long)d.N * wg_out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h) *
-        wg_out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
   w.ksteps = (int)((w.Q + kWgPos - 1) / kWgPos);
   // Split the positions when the items alone would leave SMs idle, but keep at least 8 steps per
   // range so that the pipeline's ramp and the epilogue stay small against the loop.
   const int items = w.m_tiles * w.items_b;
   int splits = sms / items;
   if (splits > w.ksteps / 8) splits = w.ksteps / 8;
+  if (g_tune_wg_ranges > 0 && splits > g_tune_wg_ranges) splits = g_tune_wg_ranges;
   if (splits < 1) splits = 1;
   w.ksteps_per_split = (w.ksteps + splits - 1) / splits;
   w.splits = (w.ksteps + w.ksteps_per_split - 1) / w.ksteps_per_split;  // no empty range
@@ -358,15 +634,147 @@ int wg_sm_count(int* sms) {
 
 }  // namespace
 
+int32_t wgrad_set_tuning(int32_t option, int32_t value) {
+  if (option == SSCONV_TUNE_WGRAD_RANGES) {
+    if (value < 0 || value > 1024) return SSCONV_ERR_BAD_DESC;
+    g_tune_wg_ranges = value;
+    return SSCONV_OK;
+  }
+  if (option == SSCONV_TUNE_WGRAD_PAIR) {
+    if (value < -1 || value > 1) return SSCONV_ERR_BAD_DESC;
+    g_tune_wg_pair = value;
+    return SSCONV_OK;
+  }
+  return SSCONV_ERR_BAD_DESC;
+}
+
 // Scratch the layer's weight gradient needs on the current device: one slice per position range.
 int32_t wgrad_workspace_bytes(const ssconv_desc_t& d, size_t* bytes) {
   int sms = 0;
   const int32_t st = wg_sm_count(&sms);
   if (st != SSCONV_OK) return st;
   const WgPlan w = wg_plan(d, sms);
-  *bytes = (size_t)w.splits * w.m_tiles * kTileM * w.taps * d.C_in * sizeof(float);
+  if (w.pair)
+    *bytes = w.splits > 1 ? (size_t)w.splits * d.C_out * w.taps * d.C_in * sizeof(float) : 0;
+  else
+    *bytes = (size_t)w.splits * w.m_tiles * kTileM * w.taps * d.C_in * sizeof(float);
   return SSCONV_OK;
 }
+
+namespace {
+bool g_wp_attr_set[64] = {false};
+
+int32_t launch_wgrad_pair(const ssconv_desc_t& d, const WgPlan& w, int Ho, int Wo, const void* x, const void* dy,
+                          float* dw, void* ws, size_t ws_bytes, int32_t* dev_status, cudaStream_t stream) {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!g_wp_attr_set[dev]) {
+    if (cudaFuncSetAttribute(ssconv_wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kWpSmemBytes) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
+    g_wp_attr_set[dev] = true;
+  }
+  const size_t slice_elems = (size_t)d.C_out * w.taps * d.C_in;
+  if (w.splits > 1 && (ws == nullptr || ws_bytes < (size_t)w.splits * slice_elems * sizeof(float)))
+    return SSCONV_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(dw) & 15u) || (w.splits > 1 && (reinterpret_cast<uintptr_t>(ws) & 15u)))
+    return SSCONV_ERR_ALIGNMENT;
+  CUtensorMap tm_dy, tm_x;
+  {
+    // gradient of the output, NHWC seen as (c, position); a box is 64 channels x 128 positions
+    cuuint64_t dims[2] = {(cuuint64_t)d.C_out, (cuuint64_t)w.Q};
+    cuuint64_t strides[1] = {(cuuint64_t)d.C_out * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kWpPos};
+    cuuint32_t estr[2] = {1, 1};
+    if (wg_encode_tiled(&tm_dy, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(dy), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return SSCONV_ERR_CUDA;
+  }
+  {
+    // activations in im2col mode as in the one-CTA kernel, 128 positions per load
+    cuuint64_t dims[4] = {(cuuint64_t)d.C_in, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
+    cuuint64_t strides[3] = {(cuuint64_t)d.C_in * 2, (cuuint64_t)d.W * d.C_in * 2,
+                             (cuuint64_t)d.H * d.W * d.C_in * 2};
+    int lower[2] = {-d.pad_w, -d.pad_h};
+    int upper[2] = {d.pad_w - (d.KW - 1) * d.dil_w, d.pad_h - (d.KH - 1) * d.dil_h};
+    cuuint32_t estr[4] = {1, (cuuint32_t)d.stride_w, (cuuint32_t)d.stride_h, 1};
+    if (wg_encode_im2col(&tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), dims, strides, lower,
+                         upper, (cuuint32_t)kBlockK, (cuuint32_t)kWpPos, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return SSCONV_ERR_CUDA;
+  }
+  CUtensorMap tm_dw;
+  {
+    // the result (or its slices, one per position range) as (c_in, tap, c_out, range) fp32; a box is 64
+    // channels of one tap x 128 output channels, unswizzled
+    float* out = w.splits > 1 ? static_cast<float*>(ws) : dw;
+    cuuint64_t dims[4] = {(cuuint64_t)d.C_in, (cuuint64_t)w.taps, (cuuint64_t)d.C_out, (cuuint64_t)w.splits};
+    cuuint64_t strides[3] = {(cuuint64_t)d.C_in * 4, (cuuint64_t)w.taps * d.C_in * 4, (cuuint64_t)slice_elems * 4};
+    cuuint32_t box[4] = {64, 1, 128, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (wg_encode_tiled(&tm_dw, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, out, dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return SSCONV_ERR_CUDA;
+  }
+  WpParams p;
+  p.C_in = d.C_in;
+  p.C_out = d.C_out;
+  p.Ho = Ho;
+  p.Wo = Wo;
+  p.stride_h = d.stride_h;
+  p.stride_w = d.stride_w;
+  p.pad_h = d.pad_h;
+  p.pad_w = d.pad_w;
+  p.dil_h = d.dil_h;
+  p.dil_w = d.dil_w;
+  p.KW = d.KW;
+  p.taps = w.taps;
+  p.kblocks = w.kblocks;
+  p.cblocks = (d.C_in + kBlockK - 1) / kBlockK;
+  p.kgroups = w.kgroups;
+  p.n_tiles = w.n_tiles;
+  p.NT = w.NT;
+  p.ksteps = w.ksteps;
+  p.ksteps_per_split = w.ksteps_per_split;
+  p.dev_status = dev_status;
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * w.splits * w.n_tiles * w.kgroups));
+  cfg.blockDim = dim3(kWpThreads);
+  cfg.dynamicSmemBytes = kWpSmemBytes;
+  cfg.stream = stream;
+  // Programmatic stream serialisation on both kernels: a grid's set-up overlaps the tail of the grid
+  // before it; each waits for that grid's completion before it touches global memory.
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  count_launch();
+  if (cudaLaunchKernelEx(&cfg, ssconv_wgrad_pair_kernel, tm_dy, tm_x, tm_dw, p) != cudaSuccess) return SSCONV_ERR_CUDA;
+  if (w.splits > 1) {
+    const size_t vec = slice_elems / 4;
+    cudaLaunchConfig_t cs = {};
+    cs.gridDim = dim3((unsigned)((vec + 255) / 256));
+    cs.blockDim = dim3(256);
+    cs.stream = stream;
+    cs.attrs = attr;
+    cs.numAttrs = 1;
+    count_launch();
+    if (cudaLaunchKernelEx(&cs, wgrad_sum_kernel, static_cast<const float4*>(ws), (int)w.splits, vec,
+                           reinterpret_cast<float4*>(dw)) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
+  }
+  return SSCONV_OK;
+}
+}  // namespace
 
 int32_t launch_wgrad(const ssconv_desc_t& d, const void* x, const void* dy, float* dw, void* ws, size_t ws_bytes,
                      int32_t* dev_status, cudaStream_t stream) {
@@ -386,10 +794,11 @@ int32_t launch_wgrad(const ssconv_desc_t& d, const void* x, const void* dy, floa
   }
   const WgPlan w = wg_plan(d, sms);
   if (w.Q > 0x7FFFFF00LL) return SSCONV_ERR_UNSUPPORTED_SHAPE;
-  const size_t slice_bytes = (size_t)w.m_tiles * kTileM * w.taps * d.C_in * sizeof(float);
-  if (ws == nullptr || ws_bytes < (size_t)w.splits * slice_bytes) return SSCONV_ERR_WORKSPACE;
   const int Ho = wg_out_extent(d.H, d.KH, d.stride_h, d.pad_h, d.dil_h);
   const int Wo = wg_out_extent(d.W, d.KW, d.stride_w, d.pad_w, d.dil_w);
+  if (w.pair) return launch_wgrad_pair(d, w, Ho, Wo, x, dy, dw, ws, ws_bytes, dev_status, stream);
+  const size_t slice_bytes = (size_t)w.m_tiles * kTileM * w.taps * d.C_in * sizeof(float);
+  if (ws == nullptr || ws_bytes < (size_t)w.splits * slice_bytes) return SSCONV_ERR_WORKSPACE;
 
   CUtensorMap tm_dy, tm_x;
   {

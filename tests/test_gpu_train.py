@@ -88,6 +88,15 @@ WG_SWEEP = [
     ("one_pixel",             1, 1,  1,  8,   8,  1, 1, 1, 0, 1),
     ("many_positions_split",  4, 40, 40, 64,  64, 3, 3, 1, 1, 1),
     ("pw_many_positions",     2, 64, 50, 64,  128, 1, 1, 1, 0, 1),
+    # CTA-pair kernel: two tiles of 256 output channels (the second partly filled), a last group of k-blocks
+    # with one, two and three members, a partial channel chunk, position ranges, one range only
+    ("pair_two_n_tiles",      2, 9,  9,  64,  328, 3, 3, 1, 1, 1),
+    ("pair_pw_5_kblocks",     2, 12, 10, 320, 200, 1, 1, 1, 0, 1),
+    ("pair_pw_6_kblocks",     3, 9,  9,  384, 96,  1, 1, 1, 0, 1),
+    ("pair_pw_3_kblocks",     2, 14, 14, 192, 768, 1, 1, 1, 0, 1),
+    ("pair_c3_chunk_of_40",   2, 10, 11, 104, 72,  3, 3, 2, 1, 1),
+    ("pair_split_ranges",     8, 28, 28, 256, 256, 3, 3, 1, 1, 1),
+    ("pair_one_step",         1, 5,  5,  256, 256, 1, 1, 1, 0, 1),
 ]
 
 
