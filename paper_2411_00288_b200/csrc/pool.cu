@@ -52,6 +52,52 @@ __global__ void __launch_bounds__(256) maxpool_nhwc_kernel(const uint4* __restri
   y[i] = m;
 }
 
+// The 3 x 3 window of stride 2 and padding 1 (the pooling of the ResNets): a thread walks kPoolRows
+// output rows of one (column, 8 channels) and keeps the maximum over the three columns of the odd image
+// row that two neighbouring windows share, so every image row is loaded once per thread (six 16-byte
+// loads per output instead of nine, all independent).
+constexpr int kPoolRows = 8;
+__device__ __forceinline__ uint4 max4(uint4 a, uint4 b) {
+  return make_uint4(max_bf16x2(a.x, b.x), max_bf16x2(a.y, b.y), max_bf16x2(a.z, b.z), max_bf16x2(a.w, b.w));
+}
+__global__ void __launch_bounds__(256) maxpool3s2_nhwc_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int N,
+                                                              int H, int W, int C8, int Ho, int Wo, int strips) {
+  const long long total = (long long)N * strips * Wo * C8;
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int c = (int)(i % C8);
+  i /= C8;
+  const int wo = (int)(i % Wo);
+  i /= Wo;
+  const int strip = (int)(i % strips);
+  const int n = (int)(i / strips);
+  const uint32_t neg_inf2 = 0xFF80FF80u;  // bf16 -inf twice: padding never wins
+  const uint4 lowest = make_uint4(neg_inf2, neg_inf2, neg_inf2, neg_inf2);
+  const int w0 = 2 * wo - 1;
+  const bool left = w0 >= 0, right = w0 + 2 < W;
+  const uint4* img = x + (long long)n * H * W * C8 + c;
+  // maximum over the window's three columns of image row h
+  auto row_max = [&](int h) -> uint4 {
+    if (h < 0 || h >= H) return lowest;
+    const uint4* centre = img + ((long long)h * W + w0 + 1) * C8;
+    uint4 m = __ldg(centre);
+    if (left) m = max4(m, __ldg(centre - C8));
+    if (right) m = max4(m, __ldg(centre + C8));
+    return m;
+  };
+  const int ho0 = strip * kPoolRows;
+  uint4 prev = row_max(2 * ho0 - 1);
+  uint4* out = y + (((long long)n * Ho + ho0) * Wo + wo) * C8 + c;
+#pragma unroll 2
+  for (int r = 0; r < kPoolRows; ++r) {
+    const int ho = ho0 + r;
+    if (ho >= Ho) break;
+    const uint4 m1 = row_max(2 * ho), m2 = row_max(2 * ho + 1);
+    out[(long long)r * Wo * C8] = max4(max4(prev, m1), m2);
+    prev = m2;
+  }
+}
+
 // Partial unfold along the width (the unfold U(X) of Eq. 5 restricted to one filter row): the KW
 // taps of a filter row become channels,
 //   y[n, h, wo, kw C + c] = x[n, h, wo s - p + kw d, c]   (0 outside the image and for channels >= KW C),
@@ -391,6 +437,13 @@ cudaError_t launch_maxpool(const void* x, void* y, int N, int H, int W, int C, i
   if (total == 0) return cudaSuccess;
   const int T = 256;
   count_launch();
+  if (k == 3 && stride == 2 && pad == 1 && W >= 2) {
+    const int strips = (Ho + kPoolRows - 1) / kPoolRows;
+    const long long threads = (long long)N * strips * Wo * (C / 8);
+    maxpool3s2_nhwc_kernel<<<(unsigned)((threads + T - 1) / T), T, 0, st>>>(
+        static_cast<const uint4*>(x), static_cast<uint4*>(y), N, H, W, C / 8, Ho, Wo, strips);
+    return cudaGetLastError();
+  }
   maxpool_nhwc_kernel<<<(unsigned)((total + T - 1) / T), T, 0, st>>>(static_cast<const uint4*>(x),
                                                                      static_cast<uint4*>(y), N, H, W, C / 8, Ho, Wo,
                                                                      k, stride, pad);
