@@ -107,10 +107,18 @@ int32_t ssconv_plan(const ssconv_desc_t* desc, int32_t sparse, int32_t* tile_pos
  * the pair kernel takes 64 and up).  SSCONV_TUNE_PAIR: -1 lets the planner choose (default), 0 never
  * uses pairs of thread blocks, 1 uses them wherever they apply.  SSCONV_TUNE_WGRAD_RANGES: 0 lets
  * ssconv_wgrad choose into how many position ranges it cuts a layer (default), otherwise an upper limit
- * (ssconv_wgrad_ws_bytes follows).  SSCONV_TUNE_WGRAD_PAIR: as SSCONV_TUNE_PAIR, for ssconv_wgrad.  Not
+ * (ssconv_wgrad_ws_bytes follows).  SSCONV_TUNE_WGRAD_PAIR: as SSCONV_TUNE_PAIR, for ssconv_wgrad.
+ * SSCONV_TUNE_RESIDENT_WEIGHTS: 1 (default) keeps the weights of dense layers with one channel tile and
+ * at most four k-blocks in shared memory, 0 sends them through the ring like every other layer's.  Not
  * thread-safe against concurrent calls.  Returns SSCONV_ERR_BAD_DESC for an unknown option or a value
  * out of range. */
-enum { SSCONV_TUNE_TILE_POSITIONS = 1, SSCONV_TUNE_PAIR = 2, SSCONV_TUNE_WGRAD_RANGES = 3, SSCONV_TUNE_WGRAD_PAIR = 4 };
+enum {
+  SSCONV_TUNE_TILE_POSITIONS = 1,
+  SSCONV_TUNE_PAIR = 2,
+  SSCONV_TUNE_WGRAD_RANGES = 3,
+  SSCONV_TUNE_WGRAD_PAIR = 4,
+  SSCONV_TUNE_RESIDENT_WEIGHTS = 5
+};
 int32_t ssconv_tune(int32_t option, int32_t value);
 
 /* ssconv_plan for a device with `sm_count` SMs, without looking at any device (host arithmetic

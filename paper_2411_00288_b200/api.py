@@ -266,7 +266,7 @@ def ssconv_plan(desc: Desc, sparse: bool = True) -> dict:
                 pair=bool(out[4].value))
 
 
-TUNE_TILE_POSITIONS, TUNE_PAIR, TUNE_WGRAD_RANGES, TUNE_WGRAD_PAIR = 1, 2, 3, 4
+TUNE_TILE_POSITIONS, TUNE_PAIR, TUNE_WGRAD_RANGES, TUNE_WGRAD_PAIR, TUNE_RESIDENT_WEIGHTS = 1, 2, 3, 4, 5
 
 
 def ssconv_tune(option: int, value: int) -> None:

@@ -102,6 +102,10 @@ struct FwdParams {
   int ring_groups;          // groups in the shared-memory ring
   int stage_bufs;           // staging buffers per epilogue group: 2, or 4 when residual pieces are prefetched
   int small_c;              // dense layers with C_in == 8: a k-block is 8 filter taps (see producer_role)
+  uint32_t a_grp_bytes;     // bytes of weights (and metadata) at the head of a ring group; 0: weights resident
+  uint32_t a_res_bytes;     // dense layers of one channel tile and at most four k-blocks: the whole weight
+                            // tile stays in shared memory after the ring (loaded once per CTA), groups hold
+                            // activations only
   int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, KW;
   int taps, cblocks, kblocks;
   int m_tiles, num_tiles;   // (pair kernel: m_tiles counts pairs of 128-channel tiles, m_real the tiles themselves)
@@ -303,12 +307,13 @@ struct TapIter {
 constexpr int kRoleActFirst = 0, kRoleActSecond = 1, kRoleWeights = 2;
 template <bool SPARSE, int ROLE, bool FP8 = false>
 __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUtensorMap* tm_b, const FwdParams& p,
-                                              uint32_t full0, uint32_t empty0, uint32_t ring0,
+                                              uint32_t full0, uint32_t empty0, uint32_t ring0, uint32_t res_bar,
                                               volatile int* abort_flag) {
   using C = Cfg<SPARSE, FP8>;
   constexpr int kKb = C::kKbChannels;
   const uint32_t b_bytes = (uint32_t)p.BN * 128u;  // one activation tile: BN positions x 64 channels
-  const uint32_t grp_bytes = group_bytes(C::kAGroupBytes, p.BN);
+  const uint32_t grp_bytes = p.a_grp_bytes + 2u * b_bytes;
+  const bool resident = !SPARSE && !FP8 && p.a_res_bytes != 0;
   uint32_t g = 0, ph = 0;  // group slot and its phase parity
   bool ok = true;
   bool first_segment = true;
@@ -328,6 +333,17 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
       // results (our inputs) are complete from here on
       grid_dependency_wait();
       first_segment = false;
+      if (ROLE == kRoleWeights && resident) {
+        // the layer's whole weight tile, once: k-block b at b * kATileBytes after the ring
+        const uint32_t res0 = ring0 + (uint32_t)p.ring_groups * grp_bytes;
+        mbar_expect_tx_w(res_bar, (uint32_t)p.kblocks * kATileBytes);
+        TapIter rit;
+        rit.init(0, p);
+        for (int b = 0; b < p.kblocks; ++b) {
+          tma_load_3d_w(res0 + (uint32_t)b * kATileBytes, tm_a, res_bar, rit.cc * kKb, rit.tap, m * kTileM);
+          rit.advance(p);
+        }
+      }
     }
     for (int a = seg.a0; a < seg.a1; ++a) {
       if (!mbar_wait_a(empty0 + 8u * g, ph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
@@ -358,13 +374,15 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
         } else {
           const uint32_t chunk_bytes = (uint32_t)p.BN * 16u;
           mbar_expect_tx_w(full, (uint32_t)chunks * chunk_bytes);
-          const uint32_t b_dst = dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? b_bytes : 0u);
+          const uint32_t b_dst = dst + p.a_grp_bytes + (ROLE == kRoleActSecond ? b_bytes : 0u);
           for (int j = 0; j < chunks; ++j) {
             tma_load_im2col_4d_w(b_dst + (uint32_t)j * chunk_bytes, tm_b, full, it.cc * kKb, base_w, base_h,
                                  q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
             it.advance(p);
           }
         }
+      } else if (ROLE == kRoleWeights && resident) {
+        mbar_arrive_w(full);  // nothing to load per group: only keep the barrier's count
       } else if (ROLE == kRoleWeights) {
         if (SPARSE) {
           mbar_expect_tx_w(full, C::kAGroupBytes);
@@ -380,7 +398,7 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tm_a, const CUt
         }
       } else if (ROLE == kRoleActFirst || has_second) {
         mbar_expect_tx_w(full, b_bytes);
-        tma_load_im2col_4d_w(dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? b_bytes : 0u), tm_b, full,
+        tma_load_im2col_4d_w(dst + p.a_grp_bytes + (ROLE == kRoleActSecond ? b_bytes : 0u), tm_b, full,
                              it.cc * kKb, base_w, base_h, q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
         it.advance(p);
         it.advance(p);
@@ -409,7 +427,8 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* ring = smem;                                                    // ring_groups groups
-  uint8_t* out_stage = ring + p.ring_groups * group_bytes(C::kAGroupBytes, p.BN);  // per epilogue group two buffers
+  // (then the resident weight tile, if any), then per epilogue group two buffers
+  uint8_t* out_stage = ring + p.ring_groups * (p.a_grp_bytes + 2u * (uint32_t)p.BN * 128u) + p.a_res_bytes;
   // barrier slots: [0,4) group full, [4,8) group empty, [8,10) accumulator full, [10,12) accumulator empty,
   // [12,20) residual piece landed (per epilogue group and staging buffer), [20,24) first k-block of a
   // group consumed (two-slot rings only: its activation tile may be refilled ahead of the rest)
@@ -479,11 +498,12 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty), ring0 = smem_u32(ring);
       if (warp == 0)
         producer_role<SPARSE, kRoleActFirst, FP8>(&tm_a, &tm_b, p, full0,
-                                             p.ring_groups == 2 ? smem_u32(bar_empty_first) : empty0, ring0, abort_flag);
+                                             p.ring_groups == 2 ? smem_u32(bar_empty_first) : empty0, ring0,
+                                             smem_u32(bar_res), abort_flag);
       else if (warp == kFirstExtraProducerWarp)
-        producer_role<SPARSE, kRoleActSecond, FP8>(&tm_a, &tm_b, p, full0, empty0, ring0, abort_flag);
+        producer_role<SPARSE, kRoleActSecond, FP8>(&tm_a, &tm_b, p, full0, empty0, ring0, smem_u32(bar_res), abort_flag);
       else
-        producer_role<SPARSE, kRoleWeights, FP8>(&tm_a, &tm_b, p, full0, empty0, ring0, abort_flag);
+        producer_role<SPARSE, kRoleWeights, FP8>(&tm_a, &tm_b, p, full0, empty0, ring0, smem_u32(bar_res), abort_flag);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -494,9 +514,15 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
                                  : make_idesc_bf16(kTileM, (uint32_t)p.BN, SPARSE);
       constexpr int kKb = C::kKbChannels;
       // descriptor address units are 16 B
-      const uint32_t grp_desc = group_bytes(C::kAGroupBytes, p.BN) >> 4;
+      const uint32_t grp_desc = (p.a_grp_bytes + 2u * (uint32_t)p.BN * 128u) >> 4;
       const uint32_t b_desc = ((uint32_t)p.BN * 128u) >> 4;
       const uint32_t ring_lo0 = desc_lo(smem_u32(ring));
+      const uint32_t a_off_desc = p.a_grp_bytes >> 4;
+      // resident weights (dense, bf16 only): the tile's k-blocks lie after the ring and arrive once
+      const bool resident = !SPARSE && !FP8 && p.a_res_bytes != 0;
+      const uint32_t res_lo0 = ring_lo0 + (uint32_t)p.ring_groups * grp_desc;
+      bool ok = true;
+      if (resident && !mbar_wait_bounded(&bar_res[0], 0u, abort_flag, kWaitLimitCycles)) ok = false;
       const uint32_t full0 = smem_u32(bar_full), empty0 = smem_u32(bar_empty);
       // With two ring slots the ring's depth bounds the main loop: the first k-block's activation
       // tile is then released on its own, so that its reload starts one k-block earlier.
@@ -513,7 +539,6 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
       uint32_t g = 0, ph = 0;  // group slot and its phase parity
       uint32_t tcount = 0;
       uint32_t mslot = 0;
-      bool ok = true;
       WorkIter work(p);
       Segment seg;
       for (; ok && work.next(seg); ++tcount) {
@@ -531,8 +556,9 @@ ssconv_fwd_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
           constexpr bool kEarly = decltype(early_tag)::value;
           for (int a = seg.a0; a < seg.a1; ++a) {
             if (!mbar_wait_a(full0 + 8u * g, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
-            const uint32_t a_lo = ring_lo0 + g * grp_desc;
-            const uint32_t b0_lo = a_lo + (C::kAGroupBytes >> 4);
+            const uint32_t grp_lo = ring_lo0 + g * grp_desc;
+            const uint32_t a_lo = resident ? res_lo0 + (uint32_t)a * ((2u * kATileBytes) >> 4) : grp_lo;
+            const uint32_t b0_lo = grp_lo + a_off_desc;
             const uint32_t b1_lo = b0_lo + b_desc;
             if (SPARSE && FP8) {
               // two metadata images -> 8 TMEM columns: 2 per MMA of 64 dense columns; operand steps in
@@ -1309,11 +1335,17 @@ static double kblock_cycles(int BN, int stage_bufs, bool steady_ring = true) {
 // use of the pair kernel.
 int32_t wgrad_set_tuning(int32_t option, int32_t value);  // (wgrad.cu)
 static int g_tune_bn = 0;
+static int g_tune_resident = 1;  // 0: weights always travel through the ring
 static int g_tune_pair = -1;  // -1: the model chooses; 0: never the pair kernel; 1: wherever it applies
 int32_t set_tuning(int32_t option, int32_t value) {
   if (option == SSCONV_TUNE_PAIR) {
     if (value < -1 || value > 1) return SSCONV_ERR_BAD_DESC;
     g_tune_pair = value;
+    return SSCONV_OK;
+  }
+  if (option == SSCONV_TUNE_RESIDENT_WEIGHTS) {
+    if (value < 0 || value > 1) return SSCONV_ERR_BAD_DESC;
+    g_tune_resident = value;
     return SSCONV_OK;
   }
   if (option == SSCONV_TUNE_TILE_POSITIONS) {
@@ -1588,9 +1620,22 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   const int pieces = (BN / 2 + kPiece - 1) / kPiece;
   const int tail_cols = BN / 2 - (pieces - 1) * kPiece;
   const bool pair = plan.pair;  // a CTA of a pair holds half of each activation tile
-  const uint32_t grp_bytes = pair ? C::kAGroupBytes + (uint32_t)BN * 128u : group_bytes(C::kAGroupBytes, BN);
-  const int ring_groups = pair ? pair_ring_groups(C::kAGroupBytes, BN) : ring_groups_for(C::kAGroupBytes, BN, stage_bufs);
-  const uint32_t smem_bytes = 1024 + (uint32_t)ring_groups * grp_bytes + staging_bytes(stage_bufs) + kBarrierBytes;
+  // Dense layers of one channel tile and at most four k-blocks (a stem run as a T x 1 convolution over 64
+  // channels): every tile needs the same 16-64 KB of weights, which then stay in shared memory for the
+  // life of the CTA instead of travelling through the ring with every tile; the groups hold activations
+  // only, and more of them fit.
+  const bool resident = !SPARSE && !FP8 && !small_c && !pair && !plan.split && residual == nullptr && geo.m_tiles == 1 &&
+                        geo.kblocks <= 4 && g_tune_resident != 0;
+  const uint32_t a_grp_bytes = resident ? 0u : C::kAGroupBytes;
+  const uint32_t a_res_bytes = resident ? (uint32_t)geo.stages * 2u * kATileBytes : 0u;
+  const uint32_t grp_bytes = pair ? C::kAGroupBytes + (uint32_t)BN * 128u : group_bytes(a_grp_bytes, BN);
+  int ring_groups = pair ? pair_ring_groups(C::kAGroupBytes, BN) : ring_groups_for(C::kAGroupBytes, BN, stage_bufs);
+  if (resident) {
+    ring_groups = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(stage_bufs) - a_res_bytes) / grp_bytes);
+    if (ring_groups > kMaxGroups) ring_groups = kMaxGroups;
+  }
+  const uint32_t smem_bytes =
+      1024 + (uint32_t)ring_groups * grp_bytes + a_res_bytes + staging_bytes(stage_bufs) + kBarrierBytes;
   if (pair && !g_pair_attr_set[dev][SPARSE ? 1 : 0]) {
     if (cudaFuncSetAttribute(ssconv_fwd_pair_kernel<SPARSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)kMaxSmemBytes) != cudaSuccess)
@@ -1704,6 +1749,8 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.tail_cols = tail_cols;
   p.ring_groups = ring_groups;
   p.small_c = small_c ? 1 : 0;
+  p.a_grp_bytes = a_grp_bytes;
+  p.a_res_bytes = a_res_bytes;
   p.stage_bufs = stage_bufs;
   p.stride_h = d.stride_h;
   p.stride_w = d.stride_w;
