@@ -403,6 +403,66 @@ def sweep_summary(cfg, m, world, ranks):
                           for r in m["per_layer"]]}
 
 
+def fp8_summary(api, synth, torch, tm, dev, l2_bytes, batch, status):
+    """The masked convolutions of the stack on e4m3 operands (ssconv_forward_fp8), layer by layer on seeded
+    inputs of each distinct shape, beside the bf16 kernels on the same shapes: device times weighted by how
+    often a shape occurs in the stack.  Context for the 8-bit path, not part of the step."""
+    shapes = {}
+    for spec in synth.config_layers(5, batch):
+        if spec.C_in % 16 or spec.extra:
+            continue
+        key = (spec.H, spec.C_in, spec.C_out, spec.KH, spec.stride)
+        shapes.setdefault(key, [spec, 0])[1] += 1
+    rows, t_bf16, t_fp8, flops = [], 0.0, 0.0, 0.0
+    iters = 10
+    for spec, count in shapes.values():
+        desc = api.desc_from_spec(spec)
+        inp = synth.make_inputs(spec)
+        w, bias = inp.w.to(dev), inp.bias.to(dev)
+        pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
+        fold = api.ssconv_fold_factor(desc)
+        d16, w16, b16 = desc, w, bias
+        if fold > 1:
+            w16, b16 = api.ssconv_fold_weights(desc, fold, w, bias)
+            pat, _ = api.ssconv_fold_weights(desc, fold, pat)
+            d16 = api.ssconv_fold_desc(desc, fold)
+        w_comp, meta = api.ssconv_compress(d16, w16, pat)
+        wq = api.ssconv_quantize_e4m3(w16, 16.0)
+        pq = api.ssconv_select_mask(api.MASK_MAGNITUDE_E4M3, wq, wq.numel() // 4)
+        wq_comp, metaq = api.ssconv_compress_fp8(d16, wq, pq)
+        set_bytes = spec.N * spec.H * spec.W * spec.C_in * 2 + 2 * spec.P * spec.C_out
+        n_sets = min(16, max(2, -(-int(1.5 * l2_bytes) // set_bytes) + 1))
+        xs = [inp.x.to(dev)] + [torch.randn(inp.x.shape, device=dev).to(torch.bfloat16) for _ in range(n_sets - 1)]
+        xq = [api.ssconv_quantize_e4m3(x, 1.0) for x in xs]
+        ys = [torch.empty((spec.N, spec.H_out, spec.W_out, spec.C_out), dtype=torch.bfloat16, device=dev)
+              for _ in range(n_sets)]
+        res = {}
+        for name, call in (
+                ("bf16", lambda r: api.ssconv_forward(d16, xs[r], w_comp, meta, b16, y=ys[r], dev_status=status)),
+                ("e4m3", lambda r: api.ssconv_forward_fp8(d16, xq[r], wq_comp, metaq, b16, 1.0 / 16.0, y=ys[r],
+                                                          dev_status=status))):
+            for r in range(min(3, n_sets)):
+                call(r)
+            torch.cuda.synchronize()
+            g = tm.capture(lambda call=call: [call(i % n_sets) for i in range(iters)])
+            tm.region(g, 1)
+            res[name] = min(tm.region(g, 2) / 2 for _ in range(3)) / iters
+            del g
+        t_bf16 += count * res["bf16"]
+        t_fp8 += count * res["e4m3"]
+        flops += count * spec.dense_equiv_flops
+        rows.append({"layer": spec.name, "count": count, "us_bf16": round(res["bf16"] * 1e3, 2),
+                     "us_e4m3": round(res["e4m3"] * 1e3, 2),
+                     "tflops_e4m3": round(spec.dense_equiv_flops / (res["e4m3"] * 1e-3) / 1e12, 1)})
+        del xs, xq, ys
+        torch.cuda.empty_cache()
+    return {"what": "the stack's masked convolutions on e4m3 activations and weights (fp32 accumulation, bf16 outputs) "
+                    "against the bf16 kernels on the same shapes; sums weighted by the shapes' multiplicity",
+            "layers": int(sum(c for _, c in shapes.values())), "sum_ms_bf16": round(t_bf16, 4),
+            "sum_ms_e4m3": round(t_fp8, 4), "x_bf16": round(t_bf16 / t_fp8, 3),
+            "tflops_e4m3": round(flops / (t_fp8 * 1e-3) / 1e12, 1), "per_layer": rows}
+
+
 # ----------------------------------------------------------------------------- mask-learning step
 def train_arm(args):
     """One mask-learning step per layer of the chosen layer set (Sec. 3.1): soft mask -> dense forward
@@ -560,7 +620,8 @@ def train_arm(args):
                        "batch_per_gpu": prep[0]["spec"].N,
                        "launch": "the step's C-ABI calls recorded into one CUDA graph and replayed",
                        "l2": "one buffer set (the step's tensors total more than L2 only for the larger layer sets)"},
-            "roofline": {"bound": "tensor", "kernel": "ssconv_wgrad_kernel", "achieved": wg_tflops,
+            "roofline": {"bound": "tensor", "kernel": "ssconv_wgrad_pair_kernel (ssconv_wgrad_kernel on layers of one or two "
+                                                        "k-blocks) + the adding kernel", "achieved": wg_tflops,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": wg_tflops / peaks["bf16_tflops"],
                          "peak_source": f"dense bf16 burst of {peaks['source']} peaks", "traffic": None},
             "per_layer": per_layer, "elementwise_at_resnet50_size": elementwise,
@@ -743,6 +804,8 @@ def stack_arm(args):
             summaries[f"summary_cfg{cfg}"] = sweep_summary(cfg, m, world, ranks)
             del m
             torch.cuda.empty_cache()
+        sampler.mark("summary_e4m3")
+        summaries["summary_e4m3"] = fp8_summary(api, synth, torch, tm, dev, l2_bytes, batch, status)
         dev_status |= int(status.item())
     clocks = sampler.stop() if rank == 0 else None
 
@@ -802,7 +865,9 @@ def stack_arm(args):
                     "peak_tflops": 2.0 * peaks["bf16_tflops"],
                     "frac": sums["roof_tensor"] / max(sums["t_tensor"], 1e-9)},
                 "traffic": None,
-                "traffic_note": "no ncu DRAM counters are committed for the current kernels at this batch"},
+                "traffic_note": "no per-step figure: outputs still in L2 when a kernel ends are never counted as written; the "
+                                "DRAM counters of single layers at this batch are in profiles/ (reads = algorithmic "
+                                "input bytes to 0.1-2 %)"},
             "per_layer": per_layer,
             "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
@@ -854,6 +919,11 @@ def sweep_arm(args):
         desc = api.desc_from_spec(spec)
         w, bias = inp.w.to(dev), inp.bias.to(dev)
         pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
+        fold = api.ssconv_fold_factor(desc)
+        if fold > 1:
+            w, bias_f = api.ssconv_fold_weights(desc, fold, w, bias)
+            pat, _ = api.ssconv_fold_weights(desc, fold, pat)
+            desc, bias = api.ssconv_fold_desc(desc, fold), bias_f
         w_comp, meta = api.ssconv_compress(desc, w, pat)
         n_sets = max(2, -(-int(1.5 * l2_bytes) // (2 * (spec.N * spec.H * spec.W * spec.C_in + spec.P * spec.C_out))) + 1)
         xs = [inp.x.to(dev)] + [torch.randn(inp.x.shape, device=dev).to(torch.bfloat16) for _ in range(n_sets - 1)]
@@ -869,7 +939,8 @@ def sweep_arm(args):
         if rank == 0:
             sampler.stop()
         print(json.dumps({"only_layer": spec.name, "launches": args.layer_iters, "dense": args.dense,
-                          "plan": api.ssconv_plan(desc, not args.dense), "dev_status": int(status.item())}))
+                          "plan": dict(api.ssconv_plan(desc, not args.dense), fold=fold),
+                          "dev_status": int(status.item())}))
         return
 
     m = sweep_measure(CONFIG_ID, api, synth, torch, tm, dev, peaks, l2_bytes, steps=steps,
