@@ -1032,7 +1032,7 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
   uint8_t* out_stage = ring + p.ring_groups * grp_bytes;
   // barrier slots: [0,4) group full (used in the leader), [4,8) group empty, [8,10) accumulator full,
   // [10,12) accumulator empty (used in the leader)
-  uint64_t* bars = reinterpret_cast<uint64_t*>(out_stage + staging_bytes(2));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_stage + staging_bytes(p.stage_bufs));
   uint64_t* bar_full = bars;
   uint64_t* bar_empty = bars + 4;
   uint64_t* bar_acc_full = bars + 8;
@@ -1169,7 +1169,10 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     const bool leader = (q == 2 && lane == 0);
     const int act = activation_of(p.flags);
     const int col_base = grp * (p.BN >> 1);
-    uint8_t* my_stage = out_stage + grp * 2 * kPieceBytes;
+    // one or two staging buffers per group (one where the K loop is long enough to hide the wait for the
+    // previous piece's store, which then leaves room for another ring group)
+    const bool one_buffer = p.stage_bufs == 1;
+    uint8_t* my_stage = out_stage + grp * p.stage_bufs * kPieceBytes;
     volatile int* my_go = epi_go + 2 * grp;
     const uint32_t acc_empty0_leader = map_to_cta(smem_u32(bar_acc_empty), 0);
     const uint32_t st_offset = (uint32_t)(q >> 1) * kHalfPieceBytes + (uint32_t)(lane & 7) * 128u +
@@ -1198,7 +1201,7 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
       }
 #pragma unroll 1
       for (int piece = 0; piece < p.pieces; ++piece, ++piece_count) {
-        uint8_t* stage = my_stage + (piece_count & 1u) * kPieceBytes;
+        uint8_t* stage = my_stage + (one_buffer ? 0u : (piece_count & 1u)) * kPieceBytes;
         uint32_t r[kPiece];
         tc_ld_piece(t_row + piece * kPiece, r);
         tc_wait_ld();
@@ -1206,6 +1209,10 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(acc_empty0_leader + 8u * buf);
+        }
+        if (one_buffer) {  // the previous piece's store has read the buffer before anyone overwrites it
+          if (leader) bulk_wait_group_read0();
+          epilogue_bar_sync(grp);
         }
         const uint32_t st_addr = smem_u32(stage) + st_offset;
         if (act == kActRelu)
@@ -1410,8 +1417,13 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
 }
 
 // Pair kernel: a CTA holds the group's weights and half of each activation tile.
-static int pair_ring_groups(uint32_t a_group_bytes, int BN) {
-  const int n = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(2)) / (a_group_bytes + (uint32_t)BN * 128u));
+// Staging buffers per epilogue group in the pair kernel: with a deep K (its loop hides the epilogue)
+// one buffer, which leaves room for one more ring group at the widest tiles; two otherwise.
+constexpr int kPairOneBufferKBlocks = 24;
+static int pair_stage_bufs(int kblocks) { return kblocks >= kPairOneBufferKBlocks ? 1 : 2; }
+static int pair_ring_groups(uint32_t a_group_bytes, int BN, int kblocks) {
+  const int n = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(pair_stage_bufs(kblocks))) /
+                      (a_group_bytes + (uint32_t)BN * 128u));
   return n > kMaxGroups ? kMaxGroups : n;
 }
 // Plan for the pair kernel (whole tiles of 256 channels x BN positions dealt out to workers / 2
@@ -1439,7 +1451,7 @@ static Plan plan_pair(long long Q, const Geometry& geo, int workers, bool forced
   const double a_bytes = Cfg<SPARSE>::kAGroupBytes / 2.0;
   const double issue = SPARSE ? kIssueSparse : kIssueDense;
   for (int BN = max_bn; BN >= min_bn; BN -= 16) {
-    const int groups = pair_ring_groups(Cfg<SPARSE>::kAGroupBytes, BN);
+    const int groups = pair_ring_groups(Cfg<SPARSE>::kAGroupBytes, BN, geo.kblocks);
     if (groups < 2) continue;
     const long long tiles = ((Q + BN - 1) / BN) * mp_tiles;
     const long long per_pair = (tiles + pairs - 1) / pairs;
@@ -1544,7 +1556,7 @@ int32_t plan_query_sms(const ssconv_desc_t& d, bool sparse, int sm_count, int32_
     const long long pairs = workers / 2;
     if (split) *split = 0;
     if (ctas) *ctas = (int32_t)(2 * (tiles < pairs ? tiles : pairs));
-    if (ring_groups) *ring_groups = pair_ring_groups(a_group_bytes, plan.BN);
+    if (ring_groups) *ring_groups = pair_ring_groups(a_group_bytes, plan.BN, geo.kblocks);
     return SSCONV_OK;
   }
   const long long tiles = q_tiles * geo.m_tiles;
@@ -1629,7 +1641,8 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   const uint32_t a_grp_bytes = resident ? 0u : C::kAGroupBytes;
   const uint32_t a_res_bytes = resident ? (uint32_t)geo.stages * 2u * kATileBytes : 0u;
   const uint32_t grp_bytes = pair ? C::kAGroupBytes + (uint32_t)BN * 128u : group_bytes(a_grp_bytes, BN);
-  int ring_groups = pair ? pair_ring_groups(C::kAGroupBytes, BN) : ring_groups_for(C::kAGroupBytes, BN, stage_bufs);
+  if (pair) stage_bufs = pair_stage_bufs(geo.kblocks);
+  int ring_groups = pair ? pair_ring_groups(C::kAGroupBytes, BN, geo.kblocks) : ring_groups_for(C::kAGroupBytes, BN, stage_bufs);
   if (resident) {
     ring_groups = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(stage_bufs) - a_res_bytes) / grp_bytes);
     if (ring_groups > kMaxGroups) ring_groups = kMaxGroups;
