@@ -565,6 +565,18 @@ def train_arm(args):
         row = {"layer": spec.name}
         for name, k in kernels.items():
             row["us_" + name] = round(replay_ms(lambda: [k(L) for _ in range(iters)], 5) / iters * 1e3, 2)
+        # the gradient with respect to the layer's input (what chains layers; not part of the step timed above),
+        # from the output gradient and the effective weights
+        try:
+            dws = torch.empty((max(api.ssconv_dgrad_ws_bytes(L["desc"]), 16),), dtype=torch.uint8, device=dev)
+            dxb = torch.empty(L["x"].shape, dtype=torch.bfloat16, device=dev)
+            row["us_dgrad"] = round(replay_ms(lambda: [api.ssconv_dgrad(L["desc"], L["dy"], L["w_eff"], dx=dxb, ws=dws,
+                                                                        dev_status=status) for _ in range(iters)], 5)
+                                    / iters * 1e3, 2)
+            row["dgrad_tflops"] = round(spec.dense_equiv_flops / row["us_dgrad"] / 1e6, 1)
+            del dws, dxb
+        except api.SsconvError:
+            row["us_dgrad"] = None
         row["wgrad_tflops"] = round(spec.dense_equiv_flops / row["us_wgrad"] / 1e6, 1)
         row["wgrad_frac_of_dense_peak"] = round(row["wgrad_tflops"] / peaks["bf16_tflops"], 4)
         # soft_mask moves 88 bytes per group (logits, noise, weights in; z, effective weights out),

@@ -349,6 +349,24 @@ int32_t ssconv_adamw(float* theta, const float* g, float* m, float* v, int64_t n
  * and writes dw.  Needs no initialisation.  dev_status: as in ssconv_forward. */
 int32_t ssconv_wgrad(const ssconv_desc_t* desc, const void* x, const void* dy, float* dw, void* ws,
                      size_t ws_bytes, int32_t* dev_status, void* stream);
+/* The gradient with respect to the layer's input in one call (Eq. 4 differentiated in x; the paper prints
+ * no gradient):  dx[n,h,w,ci] = sum over (kh,kw,co) of dy[n,ho,wo,co] * w[co,kh,kw,ci]  for the outputs
+ * (ho,wo) whose tap (kh,kw) read pixel (h,w).  dy: bf16 [N,H_out,W_out,C_out], w: bf16 [C_out,KH,KW,C_in],
+ * dx: bf16 [N,H,W,C_in] (every element is written), all device, 16-byte aligned; one rounding to bf16.
+ * With unit stride it is one convolution of dy with the reversed, channel-exchanged filter (as
+ * ssconv_dgrad_prepare + ssconv_forward_dense).  With a stride s > 1 the input pixels are split into the
+ * s_h x s_w residue classes of their padded position: a pixel with (h + pad) mod s = a only met the taps
+ * kh = a, a + s, ..., so each class is a unit-stride convolution of dy with its own few taps (all classes
+ * together carry the layer's KH x KW taps, where ssconv_dgrad_spread makes every input pixel meet all of
+ * them, s_h s_w - 1 of every s_h s_w products being zeros), written to scratch and interleaved into dx
+ * by a gather kernel.  The flags of desc are ignored (no bias, no activation).
+ * ws: device scratch of ssconv_dgrad_ws_bytes(desc) bytes (reversed weights; per class its weights and
+ * tensor), too small -> SSCONV_ERR_WORKSPACE.  SSCONV_ERR_UNSUPPORTED_SHAPE: padding beyond the filter's
+ * reach, C_out % 8 != 0, and for strided layers a dilation other than 1 or a stride above 4. */
+int32_t ssconv_dgrad_ws_bytes(const ssconv_desc_t* desc, size_t* bytes);
+int32_t ssconv_dgrad(const ssconv_desc_t* desc, const void* dy, const void* w_bf16, void* dx, void* ws, size_t ws_bytes,
+                     int32_t* dev_status, void* stream);
+
 /* Scratch bytes ssconv_wgrad needs for this layer on the current device. */
 int32_t ssconv_wgrad_ws_bytes(const ssconv_desc_t* desc, size_t* bytes);
 

@@ -29,7 +29,7 @@ EXPORTS = ("ssconv_version", "ssconv_launch_count", "ssconv_status_string", "ssc
            "ssconv_compress", "ssconv_decompress", "ssconv_maxpool", "ssconv_pad_channels", "ssconv_space_to_depth", "ssconv_unfold_w",
            "ssconv_fold_factor", "ssconv_fold_desc", "ssconv_fold_weights", "ssconv_forward", "ssconv_forward_res",
            "ssconv_forward_dense_res", "ssconv_forward_dense", "ssconv_forward_dense_strided",
-           "ssconv_mask_norms", "ssconv_absmax", "ssconv_stability_threshold", "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_dgrad_prepare", "ssconv_dgrad_spread", "ssconv_wgrad", "ssconv_wgrad_ws_bytes",
+           "ssconv_mask_norms", "ssconv_absmax", "ssconv_stability_threshold", "ssconv_soft_mask", "ssconv_mask_grad", "ssconv_adamw", "ssconv_dgrad_prepare", "ssconv_dgrad_spread", "ssconv_wgrad", "ssconv_wgrad_ws_bytes", "ssconv_dgrad", "ssconv_dgrad_ws_bytes",
            "ssconv_forward_static_ws",
            "ssconv_sizes_grouped", "ssconv_compress_grouped", "ssconv_forward_grouped", "ssconv_forward_dense_grouped",
            "ssconv_depthwise", "ssconv_layernorm",
@@ -709,6 +709,33 @@ def ssconv_wgrad(desc: Desc, x: torch.Tensor, dy: torch.Tensor, dw: Optional[tor
     _check("ssconv_wgrad", f(ctypes.byref(desc), _ptr(x), _ptr(dy), _ptr(dw), _ptr(ws), ws_bytes, _ptr(dev_status),
                              _stream(stream)))
     return dw
+
+
+def ssconv_dgrad_ws_bytes(desc: Desc) -> int:
+    n = ctypes.c_size_t()
+    f = lib().ssconv_dgrad_ws_bytes
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.POINTER(ctypes.c_size_t)]
+    _check("ssconv_dgrad_ws_bytes", f(ctypes.byref(desc), ctypes.byref(n)))
+    return int(n.value)
+
+
+def ssconv_dgrad(desc: Desc, dy: torch.Tensor, w: torch.Tensor, dx: Optional[torch.Tensor] = None,
+                 ws: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                 stream=None) -> torch.Tensor:
+    """Input gradient bf16 [N,H,W,C_in] of the layer from its output gradient dy and bf16 weights, any stride."""
+    _need_cuda(dy, w, dx, ws, dev_status)
+    if dx is None:
+        dx = torch.empty((desc.N, desc.H, desc.W, desc.C_in), dtype=torch.bfloat16, device=dy.device)
+    if ws is None:
+        ws = torch.empty((max(ssconv_dgrad_ws_bytes(desc), 16),), dtype=torch.uint8, device=dy.device)
+    f = lib().ssconv_dgrad
+    f.restype = ctypes.c_int32
+    f.argtypes = [ctypes.POINTER(Desc), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                  ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p]
+    _check("ssconv_dgrad", f(ctypes.byref(desc), _ptr(dy), _ptr(w), _ptr(dx), _ptr(ws), ws.numel() * ws.element_size(),
+                             _ptr(dev_status), _stream(stream)))
+    return dx
 
 
 def ssconv_adamw(theta: torch.Tensor, g: torch.Tensor, m: torch.Tensor, v: torch.Tensor, step: int, lr: float = 1.0,

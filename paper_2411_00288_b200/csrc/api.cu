@@ -55,6 +55,13 @@ int32_t launch_forward_static_ws(const ssconv_desc_t& d, const void* x, const vo
                                  const float* bias, void* y, int32_t* dev_status, cudaStream_t stream);
 cudaError_t launch_soft_mask(const float* logits, const float* noise, float tau, const void* w, int64_t G, float* z,
                              void* w_eff, cudaStream_t st);
+cudaError_t launch_dgrad_weights(const void* w, void* w_t, int C_out, int KH, int KW, int C_in, cudaStream_t st);
+cudaError_t launch_dgrad_class_weights(const void* w, void* w_c, int C_out, int KH, int KW, int C_in, int a, int b,
+                                       int Ja, int Jb, int sh, int sw, cudaStream_t st);
+cudaError_t launch_dgrad_gather(const DgradClasses& cls, void* dx, int N, int H, int W, int C, int pitch, int sh, int sw,
+                                int ph, int pw, cudaStream_t st);
+cudaError_t launch_dgrad_fused_weights(const void* w, void* w_all, int C_out, int KH, int KW, int C_in, int Jh, int Jw,
+                                       int sh, int sw, cudaStream_t st);
 cudaError_t launch_mask_grad(const float* z, float tau, const void* w, const float* g_w_eff, int64_t G,
                              float* g_logits, cudaStream_t st);
 cudaError_t launch_adamw(float* theta, const float* g, float* m, float* v, int64_t n, float lr, float beta1,
@@ -730,6 +737,176 @@ int32_t ssconv_dgrad_prepare(const ssconv_desc_t* desc, const void* w_bf16, void
   if (!aligned16(w_bf16) || !aligned16(w_t_bf16)) return SSCONV_ERR_ALIGNMENT;
   return ssconv::launch_dgrad_weights(w_bf16, w_t_bf16, d.C_out, d.KH, d.KW, d.C_in, (cudaStream_t)stream) ==
                  cudaSuccess
+             ? SSCONV_OK
+             : SSCONV_ERR_CUDA;
+}
+
+// ---- input gradient in one call
+namespace {
+struct DgradPlan {
+  bool strided;
+  int classes;                      // stride_h * stride_w
+  int Ja[4], Jb[4];                 // taps per residue of the padded row / column
+  int Ho, Wo;
+  bool fused;                       // all classes in one convolution (three or more of them have taps)
+  int Jh, Jw;                       // its window: ceil(KH / s_h) x ceil(KW / s_w)
+  size_t w_off[ssconv::kMaxDgradClasses], t_off[ssconv::kMaxDgradClasses];
+  size_t fwd_off, fwd_bytes;        // scratch of the convolution(s) themselves (K split)
+  size_t bytes;
+};
+size_t round256(size_t v) { return (v + 255) & ~size_t(255); }
+
+// Shape rules and workspace layout: per class its weights [C_in, Ja, Jb, C_out] and its tensor
+// [N, Ho + Ja - 1, Wo + Jb - 1, C_in]; with unit stride only the reversed weights.
+int32_t dgrad_plan(const ssconv_desc_t& d, DgradPlan* p) {
+  if (d.C_out % 8 != 0) return SSCONV_ERR_UNSUPPORTED_SHAPE;  // dy's channels are the convolutions' input channels
+  if (d.dil_h * (d.KH - 1) < d.pad_h || d.dil_w * (d.KW - 1) < d.pad_w) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  p->strided = d.stride_h > 1 || d.stride_w > 1;
+  p->Ho = (d.H + 2 * d.pad_h - d.dil_h * (d.KH - 1) - 1) / d.stride_h + 1;
+  p->Wo = (d.W + 2 * d.pad_w - d.dil_w * (d.KW - 1) - 1) / d.stride_w + 1;
+  const size_t w_bytes = (size_t)d.C_in * d.KH * d.KW * d.C_out * 2;
+  p->fwd_bytes = ssconv::workspace_bytes();
+  if (!p->strided) {
+    p->classes = 1;
+    p->fwd_off = round256(w_bytes);
+    p->bytes = p->fwd_off + p->fwd_bytes;
+    return SSCONV_OK;
+  }
+  if (d.dil_h != 1 || d.dil_w != 1 || d.stride_h > 4 || d.stride_w > 4) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  p->classes = d.stride_h * d.stride_w;
+  for (int a = 0; a < d.stride_h; ++a) p->Ja[a] = a < d.KH ? (d.KH - 1 - a) / d.stride_h + 1 : 0;
+  for (int b = 0; b < d.stride_w; ++b) p->Jb[b] = b < d.KW ? (d.KW - 1 - b) / d.stride_w + 1 : 0;
+  int with_taps = 0;
+  for (int a = 0; a < d.stride_h; ++a)
+    for (int b = 0; b < d.stride_w; ++b) with_taps += (p->Ja[a] > 0 && p->Jb[b] > 0) ? 1 : 0;
+  p->Jh = (d.KH + d.stride_h - 1) / d.stride_h;
+  p->Jw = (d.KW + d.stride_w - 1) / d.stride_w;
+  p->fused = with_taps >= 3;
+  if (p->fused) {  // weights [classes C_in, Jh, Jw, C_out], tensor [N, Ho + Jh - 1, Wo + Jw - 1, classes C_in]
+    p->w_off[0] = 0;
+    p->t_off[0] = round256((size_t)p->classes * d.C_in * p->Jh * p->Jw * d.C_out * 2);
+    p->fwd_off = p->t_off[0] + round256((size_t)d.N * (p->Ho + p->Jh - 1) * (p->Wo + p->Jw - 1) * p->classes * d.C_in * 2);
+    p->bytes = p->fwd_off + p->fwd_bytes;
+    return SSCONV_OK;
+  }
+  size_t off = 0;
+  for (int a = 0; a < d.stride_h; ++a)
+    for (int b = 0; b < d.stride_w; ++b) {
+      const int k = a * d.stride_w + b;
+      const int Ja = p->Ja[a], Jb = p->Jb[b];
+      p->w_off[k] = off;
+      off += round256((size_t)d.C_in * Ja * Jb * d.C_out * 2);
+      p->t_off[k] = off;
+      if (Ja > 0 && Jb > 0) off += round256((size_t)d.N * (p->Ho + Ja - 1) * (p->Wo + Jb - 1) * d.C_in * 2);
+    }
+  p->fwd_off = off;
+  p->bytes = off + p->fwd_bytes;
+  return SSCONV_OK;
+}
+}  // namespace
+
+int32_t ssconv_dgrad_ws_bytes(const ssconv_desc_t* desc, size_t* bytes) {
+  if (!bytes) return SSCONV_ERR_NULL;
+  ssconv_desc_t d;
+  if (desc) {
+    d = *desc;
+    d.flags = 0;
+  }
+  int32_t rc = check_desc(desc ? &d : nullptr, true);
+  if (rc != SSCONV_OK) return rc;
+  DgradPlan p;
+  rc = dgrad_plan(d, &p);
+  if (rc != SSCONV_OK) return rc;
+  *bytes = p.bytes;
+  return SSCONV_OK;
+}
+
+int32_t ssconv_dgrad(const ssconv_desc_t* desc, const void* dy, const void* w_bf16, void* dx, void* ws, size_t ws_bytes,
+                     int32_t* dev_status, void* stream) {
+  ssconv_desc_t d;
+  if (desc) {
+    d = *desc;
+    d.flags = 0;
+  }
+  int32_t rc = check_desc(desc ? &d : nullptr, true);
+  if (rc != SSCONV_OK) return rc;
+  if (!dy || !w_bf16 || !dx) return SSCONV_ERR_NULL;
+  if (!aligned16(dy) || !aligned16(w_bf16) || !aligned16(dx) || !aligned16(ws)) return SSCONV_ERR_ALIGNMENT;
+  DgradPlan p;
+  rc = dgrad_plan(d, &p);
+  if (rc != SSCONV_OK) return rc;
+  if (ws == nullptr || ws_bytes < p.bytes) return SSCONV_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  ssconv_desc_t c = d;  // the convolution(s) of dy: channels exchanged, unit stride
+  c.H = p.Ho;
+  c.W = p.Wo;
+  c.C_in = d.C_out;
+  c.C_out = d.C_in;
+  c.stride_h = c.stride_w = 1;
+  c.dil_h = d.dil_h;
+  c.dil_w = d.dil_w;
+  c.flags = 0;
+  if (!p.strided) {
+    c.pad_h = d.dil_h * (d.KH - 1) - d.pad_h;
+    c.pad_w = d.dil_w * (d.KW - 1) - d.pad_w;
+    rc = check_desc(&c, true);
+    if (rc != SSCONV_OK) return rc;
+    if (ssconv::launch_dgrad_weights(w_bf16, base, d.C_out, d.KH, d.KW, d.C_in, st) != cudaSuccess) return SSCONV_ERR_CUDA;
+    return ssconv::launch_forward_dense(c, dy, base, nullptr, nullptr, dx, base + p.fwd_off, p.fwd_bytes, dev_status, st);
+  }
+  ssconv::DgradClasses cls;
+  for (int k = 0; k < ssconv::kMaxDgradClasses; ++k) {
+    cls.t[k] = nullptr;
+    cls.rows[k] = cls.cols[k] = 0;
+  }
+  if (p.fused) {
+    c.KH = p.Jh;
+    c.KW = p.Jw;
+    c.pad_h = p.Jh - 1;
+    c.pad_w = p.Jw - 1;
+    c.C_out = p.classes * d.C_in;
+    rc = check_desc(&c, true);
+    if (rc != SSCONV_OK) return rc;
+    if (ssconv::launch_dgrad_fused_weights(w_bf16, base, d.C_out, d.KH, d.KW, d.C_in, p.Jh, p.Jw, d.stride_h, d.stride_w,
+                                           st) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
+    rc = ssconv::launch_forward_dense(c, dy, base, nullptr, nullptr, base + p.t_off[0], base + p.fwd_off, p.fwd_bytes,
+                                      dev_status, st);
+    if (rc != SSCONV_OK) return rc;
+    for (int k = 0; k < p.classes; ++k) {
+      cls.t[k] = base + p.t_off[0] + (size_t)k * d.C_in * 2;
+      cls.rows[k] = p.Ho + p.Jh - 1;
+      cls.cols[k] = p.Wo + p.Jw - 1;
+    }
+    return ssconv::launch_dgrad_gather(cls, dx, d.N, d.H, d.W, d.C_in, p.classes * d.C_in, d.stride_h, d.stride_w,
+                                       d.pad_h, d.pad_w, st) == cudaSuccess
+               ? SSCONV_OK
+               : SSCONV_ERR_CUDA;
+  }
+  for (int a = 0; a < d.stride_h; ++a)
+    for (int b = 0; b < d.stride_w; ++b) {
+      const int k = a * d.stride_w + b;
+      const int Ja = p.Ja[a], Jb = p.Jb[b];
+      if (Ja == 0 || Jb == 0) continue;
+      c.KH = Ja;
+      c.KW = Jb;
+      c.pad_h = Ja - 1;
+      c.pad_w = Jb - 1;
+      rc = check_desc(&c, true);
+      if (rc != SSCONV_OK) return rc;
+      if (ssconv::launch_dgrad_class_weights(w_bf16, base + p.w_off[k], d.C_out, d.KH, d.KW, d.C_in, a, b, Ja, Jb,
+                                             d.stride_h, d.stride_w, st) != cudaSuccess)
+        return SSCONV_ERR_CUDA;
+      rc = ssconv::launch_forward_dense(c, dy, base + p.w_off[k], nullptr, nullptr, base + p.t_off[k], base + p.fwd_off,
+                                        p.fwd_bytes, dev_status, st);
+      if (rc != SSCONV_OK) return rc;
+      cls.t[k] = base + p.t_off[k];
+      cls.rows[k] = p.Ho + Ja - 1;
+      cls.cols[k] = p.Wo + Jb - 1;
+    }
+  return ssconv::launch_dgrad_gather(cls, dx, d.N, d.H, d.W, d.C_in, d.C_in, d.stride_h, d.stride_w, d.pad_h, d.pad_w,
+                                     st) == cudaSuccess
              ? SSCONV_OK
              : SSCONV_ERR_CUDA;
 }

@@ -82,4 +82,13 @@ __host__ __device__ inline uint32_t code_pattern(uint32_t code) {
 // Kernels launched by this library in this process (all devices, all threads); see ssconv_launch_count.
 void count_launch();
 
+// The residue classes of a strided layer's input gradient (at most 4 x 4): per class the tensor its
+// convolution wrote, [N, rows, cols, C_in] bf16, or null for a class that meets no filter tap.
+constexpr int kMaxDgradClasses = 16;
+struct DgradClasses {
+  const void* t[kMaxDgradClasses];
+  int rows[kMaxDgradClasses];
+  int cols[kMaxDgradClasses];
+};
+
 }  // namespace ssconv

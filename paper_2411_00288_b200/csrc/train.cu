@@ -288,6 +288,119 @@ cudaError_t launch_dgrad_spread(const void* dy, void* dyz, int N, int Ho, int Wo
   return cudaGetLastError();
 }
 
+// Strided layers without the zeros: the input pixels fall into stride_h x stride_w residue classes of
+// their padded position, (h + pad) mod s = a.  A pixel of class a only ever met the filter taps
+// kh = a, a + s, a + 2 s, ... (J_a of them), at the outputs ho = i - j for kh = a + j s, i = (h + pad) / s:
+//   dx[h] = sum_j dy[i - j] w[a + j s],
+// a unit-stride convolution of dy with J_a x J_b taps per class (all classes together have the layer's
+// KH x KW taps, where the zero-spread form multiplies KH x KW taps at every input pixel).  As a
+// cross-correlation with padding J - 1 its output row t is i = t.  This kernel writes the weights of one
+// class, w_c[ci][u_h][u_w][co] = w[co][a + (J_a - 1 - u_h) s_h][b + (J_b - 1 - u_w) s_w][ci].
+__global__ void __launch_bounds__(256) dgrad_class_weights_kernel(const uint16_t* __restrict__ w, uint16_t* __restrict__ w_c,
+                                                                  int C_out, int KH, int KW, int C_in, int a, int b,
+                                                                  int Ja, int Jb, int sh, int sw) {
+  const int64_t total = (int64_t)C_in * Ja * Jb * C_out;
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int co = (int)(i % C_out);
+  int64_t r = i / C_out;
+  const int uw = (int)(r % Jb);
+  r /= Jb;
+  const int uh = (int)(r % Ja);
+  const int ci = (int)(r / Ja);
+  const int kh = a + (Ja - 1 - uh) * sh, kw = b + (Jb - 1 - uw) * sw;
+  w_c[i] = w[(((int64_t)co * KH + kh) * KW + kw) * C_in + ci];
+}
+
+// All classes in one convolution: the classes' output channels side by side (class k = a s_w + b holds
+// channels [k C_in, (k + 1) C_in)), every class on the common window of Jh x Jw = ceil(KH / s_h) x
+// ceil(KW / s_w) taps with zeros where its own taps end:
+//   w_all[k C_in + ci][u_h][u_w][co] = w[co][a + (Jh - 1 - u_h) s_h][b + (Jw - 1 - u_w) s_w][ci]  (0 past KH, KW).
+// One launch instead of s_h s_w small ones; the zero taps cost multiply-adds (16 tap-classes for the 9
+// taps of a 3x3 stride-2 layer, against 36 for the zero-spread form).
+__global__ void __launch_bounds__(256) dgrad_fused_weights_kernel(const uint16_t* __restrict__ w, uint16_t* __restrict__ w_all,
+                                                                  int C_out, int KH, int KW, int C_in, int Jh, int Jw,
+                                                                  int sh, int sw) {
+  // A block transposes one 32 (ci) x 32 (co) tile of one (class, tap): reads run along ci, writes along co.
+  __shared__ uint16_t tile[32][33];
+  int z = blockIdx.z;
+  const int uw = z % Jw;
+  z /= Jw;
+  const int uh = z % Jh;
+  const int k = z / Jh;
+  const int a = k / sw, b = k - a * sw;
+  const int kh = a + (Jh - 1 - uh) * sh, kw = b + (Jw - 1 - uw) * sw;
+  const bool tap = kh < KH && kw < KW;
+  const int ci0 = blockIdx.x * 32, co0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
+#pragma unroll
+  for (int r = ty; r < 32; r += 8) {
+    const int co = co0 + r, ci = ci0 + tx;
+    tile[r][tx] = (tap && co < C_out && ci < C_in) ? w[(((int64_t)co * KH + kh) * KW + kw) * C_in + ci] : (uint16_t)0;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = ty; r < 32; r += 8) {
+    const int ci = ci0 + r, co = co0 + tx;
+    if (ci < C_in && co < C_out)
+      w_all[((((int64_t)k * C_in + ci) * Jh + uh) * Jw + uw) * C_out + co] = tile[tx][r];
+  }
+}
+
+cudaError_t launch_dgrad_fused_weights(const void* w, void* w_all, int C_out, int KH, int KW, int C_in, int Jh, int Jw,
+                                       int sh, int sw, cudaStream_t st) {
+  if (C_in == 0 || C_out == 0) return cudaSuccess;
+  const dim3 grid((unsigned)((C_in + 31) / 32), (unsigned)((C_out + 31) / 32), (unsigned)(sh * sw * Jh * Jw));
+  dgrad_fused_weights_kernel<<<grid, 256, 0, st>>>((const uint16_t*)w, (uint16_t*)w_all, C_out, KH, KW, C_in, Jh, Jw, sh,
+                                                   sw);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_dgrad_class_weights(const void* w, void* w_c, int C_out, int KH, int KW, int C_in, int a, int b,
+                                       int Ja, int Jb, int sh, int sw, cudaStream_t st) {
+  const int64_t total = (int64_t)C_in * Ja * Jb * C_out;
+  if (total == 0) return cudaSuccess;
+  dgrad_class_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>((const uint16_t*)w, (uint16_t*)w_c, C_out,
+                                                                              KH, KW, C_in, a, b, Ja, Jb, sh, sw);
+  count_launch();
+  return cudaGetLastError();
+}
+
+// dx[n, h, w, :] = T_class[n, (h + pad_h) / s_h, (w + pad_w) / s_w, :] with class = the residues of the
+// padded position; zero for a class without taps and beyond a class tensor's extent (no filter placement
+// reaches those pixels).  `pitch8` = 16-byte units between pixels of a class tensor (C_in / 8, or the
+// channels of all classes when they share one tensor).  One thread per 16 bytes of dx.
+__global__ void __launch_bounds__(256) dgrad_gather_kernel(DgradClasses cls, uint4* __restrict__ dx, long long total, int H,
+                                                           int W, int C8, int pitch8, int sh, int sw, int ph, int pw) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int c = (int)(i % C8);
+  long long r = i / C8;
+  const int w = (int)(r % W);
+  r /= W;
+  const int h = (int)(r % H);
+  const long long n = r / H;
+  const int hp = h + ph, wp = w + pw;
+  const int ih = hp / sh, iw = wp / sw;
+  const int k = (hp - ih * sh) * sw + (wp - iw * sw);
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  const uint4* t = static_cast<const uint4*>(cls.t[k]);
+  if (t != nullptr && ih < cls.rows[k] && iw < cls.cols[k])
+    v = __ldg(t + ((n * cls.rows[k] + ih) * cls.cols[k] + iw) * pitch8 + c);
+  dx[i] = v;
+}
+
+cudaError_t launch_dgrad_gather(const DgradClasses& cls, void* dx, int N, int H, int W, int C, int pitch, int sh, int sw,
+                                int ph, int pw, cudaStream_t st) {
+  const long long total = (long long)N * H * W * (C / 8);
+  if (total == 0) return cudaSuccess;
+  dgrad_gather_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(cls, (uint4*)dx, total, H, W, C / 8, pitch / 8, sh,
+                                                                       sw, ph, pw);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_soft_mask(const float* logits, const float* noise, float tau, const void* w, int64_t G, float* z,
                              void* w_eff, cudaStream_t st) {
   const int threads = 256;

@@ -313,6 +313,76 @@ def test_input_gradient_of_strided_layers_matches_oracle(case):
     assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL * max(1.0, float(np.abs(ref).max()) / 4.0), (rel, mx)
 
 
+# The one-call input gradient: unit stride through the reversed filter, strided layers through the residue
+# classes of the input position (no zero-spread tensor).  Sentinel bands around dx.
+#               name              N  H   W   Ci   Co   KH KW  s       p  d
+DG_ONE_CALL = [
+    ("s1_3x3",          2, 12, 9,  64,  128, 3, 3, (1, 1), 1, 1),
+    ("s1_3x3_dil2",     1, 12, 12, 64,  64,  3, 3, (1, 1), 2, 2),
+    ("s2_3x3",          2, 16, 16, 64,  64,  3, 3, (2, 2), 1, 1),
+    ("s2_3x3_odd",      2, 15, 18, 64,  96,  3, 3, (2, 2), 1, 1),
+    ("s2_1x1",          2, 14, 14, 128, 64,  1, 1, (2, 2), 0, 1),
+    ("s2_1x1_odd",      1, 13, 11, 64,  128, 1, 1, (2, 2), 0, 1),
+    ("s3_5x5",          1, 20, 17, 32,  40,  5, 5, (3, 3), 2, 1),
+    ("s2_3x3_p0",       1, 12, 13, 32,  64,  3, 3, (2, 2), 0, 1),
+    ("s2_3x3_p2",       1, 11, 12, 32,  32,  3, 3, (2, 2), 2, 1),
+    ("s2_7x7_stem",     2, 30, 34, 8,   64,  7, 7, (2, 2), 3, 1),
+    ("s4_4x4_patchify", 2, 16, 16, 8,   96,  4, 4, (4, 4), 0, 1),
+    ("s2x1_3x3",        1, 14, 10, 64,  64,  3, 3, (2, 1), 1, 1),
+    ("r18_s2_64to128",  4, 56, 56, 64,  128, 3, 3, (2, 2), 1, 1),
+]
+
+
+@pytest.mark.parametrize("case", DG_ONE_CALL, ids=[c[0] for c in DG_ONE_CALL])
+def test_input_gradient_in_one_call_matches_oracle(case):
+    name, N, H, W, Ci, Co, KH, KW, (sh, sw), p, d = case
+    g = torch.Generator().manual_seed(synth.SEED_BASE + 4100 + DG_ONE_CALL.index(case))
+    w = (torch.randn((Co, KH, KW, Ci), generator=g) * (2.0 / (KH * KW * Ci)) ** 0.5).to(torch.bfloat16)
+    desc = api.make_desc(N, H, W, Ci, Co, KH, KW, stride=(sh, sw), pad=p, dil=d)
+    Ho, Wo = api.ssconv_out_shape(desc)
+    dy = torch.randn((N, Ho, Wo, Co), generator=g).to(torch.bfloat16)
+    band = 4096
+    buf = torch.full((N * H * W * Ci + 2 * band,), -7.0, dtype=torch.bfloat16, device=DEV)
+    dx = buf[band:band + N * H * W * Ci].view(N, H, W, Ci)
+    need = api.ssconv_dgrad_ws_bytes(desc)
+    wsbuf = torch.full((need + 2 * band,), 0x5A, dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.ssconv_dgrad(desc, dy.to(DEV), w.to(DEV), dx=dx, ws=wsbuf[band:band + need], dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert bool((buf[:band] == -7.0).all()) and bool((buf[-band:] == -7.0).all())
+    assert bool((wsbuf[:band] == 0x5A).all()) and bool((wsbuf[-band:] == 0x5A).all())
+    if sh == sw:
+        ref = otrain.dgrad_f64(synth.bf16_bits(dy), parity.bf16_tensor_to_f64(w), H, W, sh, p, d)
+    else:   # the oracle takes one stride: differentiate Eq. 4 term by term for the mixed case
+        ref = np.zeros((N, H, W, Ci))
+        dyf, wf = parity.bf16_tensor_to_f64(dy), parity.bf16_tensor_to_f64(w)
+        for ho in range(Ho):
+            for wo in range(Wo):
+                for kh in range(KH):
+                    for kw in range(KW):
+                        h, ww = ho * sh - p + kh * d, wo * sw - p + kw * d
+                        if 0 <= h < H and 0 <= ww < W:
+                            ref[:, h, ww, :] += dyf[:, ho, wo, :] @ wf[:, kh, kw, :]
+    rel, mx = parity.errors(parity.bf16_tensor_to_f64(dx), ref)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL * max(1.0, float(np.abs(ref).max()) / 4.0), (rel, mx)
+
+
+def test_one_call_input_gradient_argument_rules():
+    d = api.make_desc(1, 8, 8, 64, 64, 3, 3, stride=2, pad=1)
+    dy = torch.zeros((1, 4, 4, 64), dtype=torch.bfloat16, device=DEV)
+    w = torch.zeros((64, 3, 3, 64), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(api.SsconvError) as e:
+        api.ssconv_dgrad(d, dy, w, ws=torch.empty((16,), dtype=torch.uint8, device=DEV))
+    assert e.value.status == 5          # workspace too small
+    with pytest.raises(api.SsconvError) as e:
+        api.ssconv_dgrad_ws_bytes(api.make_desc(1, 9, 9, 64, 64, 3, 3, stride=2, pad=2, dil=2))
+    assert e.value.status == 3          # strided and dilated
+    with pytest.raises(api.SsconvError) as e:
+        api.ssconv_dgrad_ws_bytes(api.make_desc(1, 8, 8, 64, 64, 1, 1, stride=1, pad=1))
+    assert e.value.status == 3          # padding beyond the filter's reach
+
+
 @pytest.mark.parametrize("second", [(1, 1, 1, 0), (3, 3, 2, 1)], ids=["1x1", "3x3_stride2"])
 def test_learning_the_masks_of_two_chained_layers(second):
     """Two layers trained together: the loss gradient reaches the first layer's choice weights through
