@@ -463,6 +463,40 @@ def fp8_summary(api, synth, torch, tm, dev, l2_bytes, batch, status):
             "tflops_e4m3": round(flops / (t_fp8 * 1e-3) / 1e12, 1), "per_layer": rows}
 
 
+def convnext_summary(api, torch, tm, dev, batch=128):
+    """A ConvNeXt-T-shaped network chained through the library (convnext.py: patchify stem, 18 blocks of depthwise 7x7
+    -> layer norm -> 1x1 2:4 with GELU -> 1x1 2:4 with the skip connection fused, three downsample convolutions), the
+    whole forward pass recorded into one CUDA graph.  Context for the other network family of Sec. 4."""
+    from paper_2411_00288_b200 import convnext
+    net = convnext.ConvNeXtStack(batch, dev)
+    x = torch.randn((batch, 224, 224, 3), device=dev).to(torch.bfloat16)
+    for sparse in (True, False):
+        net.forward(x, sparse)
+    torch.cuda.synchronize()
+    res = {}
+    for sparse in (True, False):
+        g = tm.capture(lambda sparse=sparse: net.forward(x, sparse))
+        tm.region(g, 2)
+        res[sparse] = min(tm.region(g, 5) / 5 for _ in range(3))
+        del g
+    kinds = {}
+    for i, st in enumerate(net.steps):
+        g = tm.capture(lambda i=i: [net.run_step(i, x) for _ in range(3)])
+        tm.region(g, 1)
+        kinds[st.kind] = kinds.get(st.kind, 0.0) + tm.region(g, 2) / 6
+        del g
+    out = {"what": "ConvNeXt-T-shaped forward pass, 224 x 224 images, all convolutions but the stem and the depthwise ones "
+                   "2:4 masked; seeded synthetic weights", "batch": batch, "calls_per_step": len(net.steps),
+           "ms_per_step": round(res[True], 4), "images_per_s": round(batch / res[True] * 1e3, 1),
+           "x_dense": round(res[False] / res[True], 3),
+           "masked_conv_tflops": round(net.masked_conv_flops() / (kinds["conv"] * 1e-3) / 1e12, 1),
+           "ms_by_kind": {("masked_conv" if k == "conv" else k): round(v, 4) for k, v in kinds.items()},
+           "dev_status": int(net.status.item())}
+    del net
+    torch.cuda.empty_cache()
+    return out
+
+
 # ----------------------------------------------------------------------------- mask-learning step
 def train_arm(args):
     """One mask-learning step per layer of the chosen layer set (Sec. 3.1): soft mask -> dense forward
@@ -818,6 +852,9 @@ def stack_arm(args):
             torch.cuda.empty_cache()
         sampler.mark("summary_e4m3")
         summaries["summary_e4m3"] = fp8_summary(api, synth, torch, tm, dev, l2_bytes, batch, status)
+        sampler.mark("summary_convnext_t")
+        summaries["summary_convnext_t"] = convnext_summary(api, torch, tm, dev)
+        dev_status |= summaries["summary_convnext_t"]["dev_status"]
         dev_status |= int(status.item())
     clocks = sampler.stop() if rank == 0 else None
 

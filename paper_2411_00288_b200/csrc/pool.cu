@@ -358,12 +358,116 @@ __global__ void __launch_bounds__(256) depthwise_kernel(const uint4* __restrict_
   y[i] = make_uint4(out[0], out[1], out[2], out[3]);
 }
 
+// Unit stride, no dilation, KW = 3, 5 or 7: a thread computes kDwRun consecutive output pixels of a row for
+// its 8 channels, so an image pixel is loaded once per filter row for all the outputs of the run it
+// touches (10 loads per row for 4 outputs of a 7-wide filter instead of 28) and the row's weights are
+// unpacked to fp32 once; what remains is the 8 KH KW multiply-adds per output, in fp32, two per instruction.
+constexpr int kDwRun = 8;
+// Two fp32 multiply-adds in one instruction (sm_100: fma.rn.f32x2 on register pairs): d = a * b + d per half.
+__device__ __forceinline__ void fma2(unsigned long long& d, unsigned long long a, unsigned long long b) {
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
+}
+// A bf16 pair widened to an fp32 pair (low element in the low half).
+__device__ __forceinline__ unsigned long long widen2(uint32_t v) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(v << 16), "r"(v & 0xFFFF0000u));
+  return r;
+}
+template <int KW>
+__global__ void __launch_bounds__(128, 4) depthwise_run_kernel(const uint2* __restrict__ x, const uint2* __restrict__ w,
+                                                               const float* __restrict__ bias, uint2* __restrict__ y, int N,
+                                                               int H, int W, int C4, int Ho, int Wo, int KH, int pad,
+                                                               int runs, uint32_t flags) {
+  // (4 channels = 8 bytes per thread: half the registers of a 16-byte version, twice the resident warps)
+  const long long total = (long long)N * Ho * runs * C4;
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int c = (int)(i % C4);
+  i /= C4;
+  const int run = (int)(i % runs);
+  i /= runs;
+  const int ho = (int)(i % Ho);
+  const int n = (int)(i / Ho);
+  const int wo0 = run * kDwRun;
+  unsigned long long acc[kDwRun][2];  // fp32 pairs
+#pragma unroll
+  for (int t = 0; t < kDwRun; ++t) acc[t][0] = acc[t][1] = 0ull;
+  for (int kh = 0; kh < KH; ++kh) {
+    const int h = ho - pad + kh;
+    if (h < 0 || h >= H) continue;
+    unsigned long long wf[KW][2];
+#pragma unroll
+    for (int kw = 0; kw < KW; ++kw) {
+      const uint2 wv = __ldg(w + (long long)(kh * KW + kw) * C4 + c);
+      wf[kw][0] = widen2(wv.x);
+      wf[kw][1] = widen2(wv.y);
+    }
+    // all pixels of the row first (independent loads in flight together), then the arithmetic
+    const uint2* row = x + ((long long)(n * H + h) * W) * C4 + c;
+    uint2 xv[kDwRun + KW - 1];
+#pragma unroll
+    for (int col = 0; col < kDwRun + KW - 1; ++col) {
+      const int ww = wo0 - pad + col;
+      const bool in = ww >= 0 && ww < W;
+      xv[col] = in ? __ldg(row + (long long)(in ? ww : 0) * C4) : make_uint2(0u, 0u);
+    }
+#pragma unroll
+    for (int col = 0; col < kDwRun + KW - 1; ++col) {
+      const unsigned long long x0 = widen2(xv[col].x), x1 = widen2(xv[col].y);
+#pragma unroll
+      for (int kw = 0; kw < KW; ++kw) {
+        const int t = col - kw;  // the output of the run that meets this pixel at tap kw
+        if (t >= 0 && t < kDwRun) {
+          fma2(acc[t][0], x0, wf[kw][0]);
+          fma2(acc[t][1], x1, wf[kw][1]);
+        }
+      }
+    }
+  }
+  float bv[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) bv[j] = (flags & SSCONV_FLAG_BIAS) ? bias[4 * c + j] : 0.0f;
+  uint2* out = y + ((long long)(n * Ho + ho) * Wo + wo0) * C4 + c;
+#pragma unroll
+  for (int t = 0; t < kDwRun; ++t) {
+    if (wo0 + t >= Wo) break;
+    uint32_t o[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      float lo = __uint_as_float((uint32_t)acc[t][j]) + bv[2 * j];
+      float hi = __uint_as_float((uint32_t)(acc[t][j] >> 32)) + bv[2 * j + 1];
+      if (flags & SSCONV_FLAG_RELU) {
+        lo = fmaxf(lo, 0.0f);
+        hi = fmaxf(hi, 0.0f);
+      }
+      __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+      o[j] = *reinterpret_cast<uint32_t*>(&b2);
+    }
+    out[(long long)t * C4] = make_uint2(o[0], o[1]);
+  }
+}
+
 cudaError_t launch_depthwise(const void* x, const void* w, const float* bias, void* y, int N, int H, int W, int C, int Ho,
                              int Wo, int KH, int KW, int stride, int pad, int dil, uint32_t flags, cudaStream_t st) {
   const long long total = (long long)N * Ho * Wo * (C / 8);
   if (total == 0) return cudaSuccess;
   const int T = 256;
   count_launch();
+  if (stride == 1 && dil == 1 && (KW == 3 || KW == 5 || KW == 7)) {
+    const int runs = (Wo + kDwRun - 1) / kDwRun;
+    const long long threads = (long long)N * Ho * runs * (C / 4);
+    const unsigned grid = (unsigned)((threads + 127) / 128);
+    const uint2* xp = static_cast<const uint2*>(x);
+    const uint2* wp = static_cast<const uint2*>(w);
+    uint2* yp = static_cast<uint2*>(y);
+    if (KW == 3)
+      depthwise_run_kernel<3><<<grid, 128, 0, st>>>(xp, wp, bias, yp, N, H, W, C / 4, Ho, Wo, KH, pad, runs, flags);
+    else if (KW == 5)
+      depthwise_run_kernel<5><<<grid, 128, 0, st>>>(xp, wp, bias, yp, N, H, W, C / 4, Ho, Wo, KH, pad, runs, flags);
+    else
+      depthwise_run_kernel<7><<<grid, 128, 0, st>>>(xp, wp, bias, yp, N, H, W, C / 4, Ho, Wo, KH, pad, runs, flags);
+    return cudaGetLastError();
+  }
   depthwise_kernel<<<(unsigned)((total + T - 1) / T), T, 0, st>>>(static_cast<const uint4*>(x), static_cast<const uint4*>(w),
                                                                   bias, static_cast<uint4*>(y), N, H, W, C / 8, Ho, Wo, KH,
                                                                   KW, stride, pad, dil, flags);
@@ -397,11 +501,96 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const __nv_bfloat16* __r
     y[pix * C + c] = __float2bfloat16_rn((__bfloat162float(xp[c]) - mean) * rstd * gamma[c] + beta[c]);
 }
 
+// C a multiple of 8 and at most 1024: a group of G lanes (a power of two, G >= C / 8 up to 32) per pixel,
+// a lane holding V 16-byte pieces of it in registers: one read and one write of the tensor, 16 bytes at
+// a time, statistics by shuffles within the group.
+template <int V>
+__global__ void __launch_bounds__(256) layernorm_vec_kernel(const uint4* __restrict__ x, const float* __restrict__ gamma,
+                                                            const float* __restrict__ beta, uint4* __restrict__ y,
+                                                            long long pixels, int C8, int G, float eps) {
+  const int lane = threadIdx.x & 31;
+  const int sub = lane & (G - 1);
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long pix = warp * (32 / G) + lane / G;
+  const bool live = pix < pixels;
+  float f[V][8];
+  float sum = 0.0f;
+#pragma unroll
+  for (int k = 0; k < V; ++k) {
+    const int idx = sub + k * G;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (live && idx < C8) v = __ldg(x + pix * C8 + idx);
+    const uint32_t a[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      f[k][2 * j] = __uint_as_float(a[j] << 16);
+      f[k][2 * j + 1] = __uint_as_float(a[j] & 0xFFFF0000u);
+      sum += f[k][2 * j] + f[k][2 * j + 1];
+    }
+  }
+  for (int o = G >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  const float inv_c = 1.0f / (float)(8 * C8);
+  const float mean = sum * inv_c;
+  float sq = 0.0f;
+#pragma unroll
+  for (int k = 0; k < V; ++k) {
+    if (sub + k * G < C8) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float d = f[k][j] - mean;
+        sq += d * d;
+      }
+    }
+  }
+  for (int o = G >> 1; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+  const float rstd = rsqrtf(sq * inv_c + eps);
+#pragma unroll
+  for (int k = 0; k < V; ++k) {
+    const int idx = sub + k * G;
+    if (!live || idx >= C8) continue;
+    const float4 g0 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * idx);
+    const float4 g1 = __ldg(reinterpret_cast<const float4*>(gamma) + 2 * idx + 1);
+    const float4 b0 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * idx);
+    const float4 b1 = __ldg(reinterpret_cast<const float4*>(beta) + 2 * idx + 1);
+    const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+    const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      __nv_bfloat162 p = __floats2bfloat162_rn((f[k][2 * j] - mean) * rstd * gg[2 * j] + bb[2 * j],
+                                               (f[k][2 * j + 1] - mean) * rstd * gg[2 * j + 1] + bb[2 * j + 1]);
+      o[j] = *reinterpret_cast<uint32_t*>(&p);
+    }
+    y[pix * C8 + idx] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 cudaError_t launch_layernorm(const void* x, const float* gamma, const float* beta, void* y, long long pixels, int C,
                              float eps, cudaStream_t st) {
   if (pixels == 0) return cudaSuccess;
   const int T = 256;
   count_launch();
+  const bool aligned = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(gamma) |
+                         reinterpret_cast<uintptr_t>(beta)) & 15u) == 0;
+  if (C % 8 == 0 && C <= 1024 && aligned) {
+    const int C8 = C / 8;
+    int G = 1;
+    while (G < C8 && G < 32) G <<= 1;
+    const int V = (C8 + G - 1) / G;
+    const long long warps = (pixels + (32 / G) - 1) / (32 / G);
+    const unsigned grid = (unsigned)((warps * 32 + T - 1) / T);
+    const uint4* xp = static_cast<const uint4*>(x);
+    uint4* yp = static_cast<uint4*>(y);
+    if (V == 1)
+      layernorm_vec_kernel<1><<<grid, T, 0, st>>>(xp, gamma, beta, yp, pixels, C8, G, eps);
+    else if (V == 2)
+      layernorm_vec_kernel<2><<<grid, T, 0, st>>>(xp, gamma, beta, yp, pixels, C8, G, eps);
+    else if (V == 3)
+      layernorm_vec_kernel<3><<<grid, T, 0, st>>>(xp, gamma, beta, yp, pixels, C8, G, eps);
+    else
+      layernorm_vec_kernel<4><<<grid, T, 0, st>>>(xp, gamma, beta, yp, pixels, C8, G, eps);
+    return cudaGetLastError();
+  }
   layernorm_kernel<<<(unsigned)((pixels * 32 + T - 1) / T), T, 0, st>>>(static_cast<const __nv_bfloat16*>(x), gamma, beta,
                                                                         static_cast<__nv_bfloat16*>(y), pixels, C, eps);
   return cudaGetLastError();

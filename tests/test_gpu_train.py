@@ -386,7 +386,8 @@ def test_one_call_input_gradient_argument_rules():
 @pytest.mark.parametrize("second", [(1, 1, 1, 0), (3, 3, 2, 1)], ids=["1x1", "3x3_stride2"])
 def test_learning_the_masks_of_two_chained_layers(second):
     """Two layers trained together: the loss gradient reaches the first layer's choice weights through
-    the second layer's input gradient (spread out first when that layer is strided).  Twenty-five steps
+    the second layer's input gradient (the one-call form and, on alternate steps, its parts with the
+    gradient spread out first when that layer is strided).  Twenty-five steps
     must lower the loss."""
     KH2, KW2, st2, p2 = second
     s1 = synth.LayerSpec("chain1", 2, 12, 12, 64, 64, 3, 3, 1, 1, 1, relu=False, has_bias=False, w_std="he",
@@ -411,8 +412,11 @@ def test_learning_the_masks_of_two_chained_layers(second):
         losses.append(float((diff ** 2).mean()))
         dy = (diff * (2.0 / diff.numel()) * 1e4).to(torch.bfloat16)  # scaled so that bf16 keeps it; Adam is scale-free
         g2 = api.ssconv_mask_grad(z2, tau, w2, api.ssconv_wgrad(d2, h, dy))
-        dd, wt = api.ssconv_dgrad_prepare(d2, e2)
-        dh = api.ssconv_forward_dense(dd, api.ssconv_dgrad_spread(d2, dy) if st2 > 1 else dy, wt, None)
+        if step % 2:   # both routes to the second layer's input gradient take turns
+            dh = api.ssconv_dgrad(d2, dy, e2)
+        else:
+            dd, wt = api.ssconv_dgrad_prepare(d2, e2)
+            dh = api.ssconv_forward_dense(dd, api.ssconv_dgrad_spread(d2, dy) if st2 > 1 else dy, wt, None)
         g1 = api.ssconv_mask_grad(z1, tau, w1, api.ssconv_wgrad(d1, x, dh))
         api.ssconv_adamw(l1, g1, m1, v1, step, lr=0.3)
         api.ssconv_adamw(l2, g2, m2, v2, step, lr=0.3)
