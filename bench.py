@@ -497,6 +497,18 @@ def convnext_summary(api, torch, tm, dev, batch=128):
     return out
 
 
+def convnext_arm(args):
+    """The ConvNeXt-T-shaped pass on its own (one GPU): prints convnext_summary as one JSON line."""
+    import torch
+    from paper_2411_00288_b200 import api, ranks, build as libbuild
+    libbuild.build()
+    api.lib()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    tm = Timer(torch, None, ranks, dev, False)
+    print(json.dumps(convnext_summary(api, torch, tm, dev, batch=args.batch or 128)))
+
+
 # ----------------------------------------------------------------------------- mask-learning step
 def train_arm(args):
     """One mask-learning step per layer of the chosen layer set (Sec. 3.1): soft mask -> dense forward
@@ -1122,6 +1134,8 @@ def main():
     ap.add_argument("--train", action="store_true",
                     help="time one mask-learning step per layer (soft mask, dense forward, weight gradient, "
                          "choice-weight gradient) on one of the per-layer sweeps (default: the ResNet-18 sweep)")
+    ap.add_argument("--convnext", action="store_true",
+                    help="only the ConvNeXt-T-shaped forward pass (the default line's summary_convnext_t), one GPU")
     ap.add_argument("--batch", type=int, default=None, help="images per GPU of the stack (default 256)")
     ap.add_argument("--workload-config", type=int, default=None, choices=sorted(WORKLOADS),
                     help="5 (default): the ResNet-50 stack; 2, 3, 4: one of the per-layer sweeps")
@@ -1134,6 +1148,8 @@ def main():
         args.layer_iters = 10 if CONFIG_ID == 5 else 100
     if args.impl == "reference":
         reference_arm(args)
+    elif args.convnext:
+        convnext_arm(args)
     elif args.train:
         if CONFIG_ID == 5:
             CONFIG_ID, WORKLOAD = 2, WORKLOADS[2]
