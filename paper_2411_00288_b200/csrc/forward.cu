@@ -957,12 +957,13 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
 // and "accumulator full" exist in each CTA and the leader commits to both; "accumulator empty" lives
 // in the leader and counts the epilogue warps of both CTAs.  No load is multicast: each CTA fetches
 // what it needs itself.  Whole tiles only (no K split), no residual, no 8-channel mode.
-template <bool SPARSE, int ROLE>
+template <bool SPARSE, int ROLE, bool FP8 = false>
 __device__ __forceinline__ void pair_producer_role(const CUtensorMap* tm_a, const CUtensorMap* tm_b,
                                                    const CUtensorMap* tm_meta, const FwdParams& p, uint32_t rank,
                                                    uint32_t pair, uint32_t full0_leader, uint32_t full0_local,
                                                    uint32_t empty0, uint32_t ring0, volatile int* abort_flag) {
-  using C = Cfg<SPARSE>;
+  using C = Cfg<SPARSE, FP8>;
+  constexpr int kKb = C::kKbChannels;
   const uint32_t half_bytes = (uint32_t)(p.BN >> 1) * 128u;  // this CTA's half of an activation tile
   const uint32_t grp_bytes = C::kAGroupBytes + 2u * half_bytes;
   const bool leader = rank == 0;
@@ -992,19 +993,19 @@ __device__ __forceinline__ void pair_producer_role(const CUtensorMap* tm_a, cons
       if (ROLE == kRoleWeights) {
         if (SPARSE) {
           if (leader) mbar_expect_tx_w(full0_local + 8u * g, 2u * C::kAGroupBytes);
-          tma2_load_2d_w(dst, tm_a, full, a * 64, m * kTileM);
-          tma2_load_2d_w(dst + kATileBytes, tm_meta, full, 0, (m_meta * p.a_tiles + a) * kTileM);
+          tma2_load_2d_w(dst, tm_a, full, a * (FP8 ? 128 : 64), m * kTileM);  // 128 bytes of kept values per group
+          tma2_load_2d_w(dst + kATileBytes, tm_meta, full, 0, (m_meta * p.a_tiles + a) * (int)(C::kMetaBytes / 16));
         } else {
           if (leader) mbar_expect_tx_w(full0_local + 8u * g, (has_second ? 4u : 2u) * kATileBytes);
-          tma2_load_3d_w(dst, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+          tma2_load_3d_w(dst, tm_a, full, it.cc * kKb, it.tap, m * kTileM);
           it.advance(p);
-          if (has_second) tma2_load_3d_w(dst + kATileBytes, tm_a, full, it.cc * kBlockK, it.tap, m * kTileM);
+          if (has_second) tma2_load_3d_w(dst + kATileBytes, tm_a, full, it.cc * kKb, it.tap, m * kTileM);
           it.advance(p);
         }
       } else if (ROLE == kRoleActFirst || has_second) {
         if (leader) mbar_expect_tx_w(full0_local + 8u * g, 2u * half_bytes);
         tma2_load_im2col_4d_w(dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? half_bytes : 0u), tm_b, full,
-                              it.cc * kBlockK, base_w, base_h, q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
+                              it.cc * kKb, base_w, base_h, q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
         it.advance(p);
         it.advance(p);
       } else if (leader) {
@@ -1018,12 +1019,13 @@ __device__ __forceinline__ void pair_producer_role(const CUtensorMap* tm_a, cons
   }
 }
 
-template <bool SPARSE>
+template <bool SPARSE, bool FP8 = false>
 __global__ void __launch_bounds__(kThreads, 1)
 ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                        const __grid_constant__ CUtensorMap tm_meta, const __grid_constant__ CUtensorMap tm_y,
                        const __grid_constant__ CUtensorMap tm_y_tail, const FwdParams p) {
-  using C = Cfg<SPARSE>;
+  using C = Cfg<SPARSE, FP8>;
+  static_assert(!FP8 || SPARSE, "the pair kernel takes 8-bit operands only in the 2:4 form");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t half_bytes = (uint32_t)(p.BN >> 1) * 128u;
@@ -1091,28 +1093,31 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     const uint32_t full0_leader = map_to_cta(full0_local, 0);
     const uint32_t empty0 = smem_u32(bar_empty), ring0 = smem_u32(ring);
     if (warp == 0)
-      pair_producer_role<SPARSE, kRoleActFirst>(&tm_a, &tm_b, &tm_meta, p, rank, pair, full0_leader, full0_local, empty0,
+      pair_producer_role<SPARSE, kRoleActFirst, FP8>(&tm_a, &tm_b, &tm_meta, p, rank, pair, full0_leader, full0_local, empty0,
                                                 ring0, abort_flag);
     else if (warp == kFirstExtraProducerWarp)
-      pair_producer_role<SPARSE, kRoleActSecond>(&tm_a, &tm_b, &tm_meta, p, rank, pair, full0_leader, full0_local,
+      pair_producer_role<SPARSE, kRoleActSecond, FP8>(&tm_a, &tm_b, &tm_meta, p, rank, pair, full0_leader, full0_local,
                                                  empty0, ring0, abort_flag);
     else
-      pair_producer_role<SPARSE, kRoleWeights>(&tm_a, &tm_b, &tm_meta, p, rank, pair, full0_leader, full0_local, empty0,
+      pair_producer_role<SPARSE, kRoleWeights, FP8>(&tm_a, &tm_b, &tm_meta, p, rank, pair, full0_leader, full0_local, empty0,
                                                ring0, abort_flag);
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (leader_cta) {
-      const uint32_t idesc = make_idesc_bf16(2 * kTileM, (uint32_t)p.BN, SPARSE);
+      const uint32_t idesc = FP8 ? make_idesc_e4m3(2 * kTileM, (uint32_t)p.BN, SPARSE)
+                                 : make_idesc_bf16(2 * kTileM, (uint32_t)p.BN, SPARSE);
+      constexpr int kKb = C::kKbChannels;
       const uint32_t grp_desc = grp_bytes >> 4;
       const uint32_t half_desc = half_bytes >> 4;
       const uint32_t ring_lo0 = desc_lo(smem_u32(ring));
       const uint32_t full0 = smem_u32(bar_full);
       const uint32_t empty0 = smem_u32(bar_empty), accf0 = smem_u32(bar_acc_full);
       const uint32_t meta_tmem0 = tmem_base + kMetaCol;
-      const int tail_c = p.C_in - (p.cblocks - 1) * kBlockK;
+      const int tail_c = p.C_in - (p.cblocks - 1) * kKb;
       const int mma_full = SPARSE ? 2 : 4;
-      const int mma_tail = SPARSE ? ((tail_c + 31) >> 5) : ((tail_c + 15) >> 4);
-      const int tail_start = (tail_c == kBlockK) ? p.kblocks : (p.cblocks - 1) * p.taps;  // first k-block of the tail
+      // channels per MMA: bf16 32 sparse / 16 dense, e4m3 64 sparse
+      const int mma_tail = SPARSE ? ((tail_c + kKb / 2 - 1) / (kKb / 2)) : ((tail_c + 15) >> 4);
+      const int tail_start = (tail_c == kKb) ? p.kblocks : (p.cblocks - 1) * p.taps;  // first k-block of the tail
       uint32_t g = 0, ph = 0, tcount = 0, mslot = 0;
       uint32_t ready = 0;  // the look-ahead saw the group in hand complete
       bool ok = true;
@@ -1138,7 +1143,17 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
           const uint32_t b1_lo = b0_lo + half_desc;
           const int n0 = (2 * a >= tail_start) ? mma_tail : mma_full;
           const int n1 = (2 * a + 1 >= p.kblocks) ? 0 : ((2 * a + 1 >= tail_start) ? mma_tail : mma_full);
-          if (SPARSE) {
+          if (SPARSE && FP8) {
+            // two metadata images -> 8 TMEM columns, 2 per MMA of 64 dense columns (as in the one-block kernel)
+            const uint32_t meta_tmem = meta_tmem0 + 8u * mslot;
+            mslot ^= 1u;
+            tc2_cp_128x128b_w(meta_tmem, a_lo + (kATileBytes >> 4));
+            tc2_cp_128x128b_w(meta_tmem + 4u, a_lo + ((kATileBytes + (uint32_t)kMetaImageBytes) >> 4));
+            tc2_mma_f8_sparse_w(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
+            if (n0 > 1) tc2_mma_f8_sparse_w(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem + 2u, idesc, 1u);
+            if (n1 > 0) tc2_mma_f8_sparse_w(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 4u, idesc, 1u);
+            if (n1 > 1) tc2_mma_f8_sparse_w(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 6u, idesc, 1u);
+          } else if (SPARSE) {
             const uint32_t meta_tmem = meta_tmem0 + 4u * mslot;
             mslot ^= 1u;
             tc2_cp_128x128b_w(meta_tmem, a_lo + (kATileBytes >> 4));
@@ -1209,6 +1224,10 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(acc_empty0_leader + 8u * buf);
+        }
+        if (FP8) {
+#pragma unroll
+          for (int i = 0; i < kPiece; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * p.out_scale);
         }
         if (one_buffer) {  // the previous piece's store has read the buffer before anyone overwrites it
           if (leader) bulk_wait_group_read0();
@@ -1481,6 +1500,7 @@ static int g_sm_count[64] = {0};
 static bool g_attr_set[64][2][2] = {{{false}}};
 static bool g_pair_attr_set[64][2] = {{false}};
 static bool g_fp8_attr_set[64][2] = {{false}};
+static bool g_pair_fp8_attr_set[64] = {false};
 
 // Dense layers with 8 input channels (a channel-padded RGB stem): a k-block of 64 K-elements is 8
 // filter taps instead of 64 channels of one tap, which would be 7/8 padding.
@@ -1617,8 +1637,9 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   const bool have_ws = !FP8 && ws != nullptr && ws_bytes >= scratch_bytes(worker_cap);  // (8-bit: whole tiles only)
   if (have_ws && (reinterpret_cast<uintptr_t>(ws) & 15u)) return SSCONV_ERR_ALIGNMENT;
   if (force_split && !have_ws) return SSCONV_ERR_WORKSPACE;
-  Plan plan = (residual != nullptr || FP8) ? plan_layer<SPARSE>(Q, geo, workers, force_split, kBN, 2, have_ws)
-                                           : choose_plan<SPARSE>(d, Q, geo, workers, force_split, have_ws);
+  // (8-bit operands: the pair kernel exists for the 2:4 form only; the dense counterpart stays on one-block tiles)
+  Plan plan = (residual != nullptr || (FP8 && !SPARSE)) ? plan_layer<SPARSE>(Q, geo, workers, force_split, kBN, 2, have_ws)
+                                                        : choose_plan<SPARSE>(d, Q, geo, workers, force_split, have_ws);
   int stage_bufs = 2;
   if (residual != nullptr && !plan.split) {
     stage_bufs = 4;
@@ -1649,11 +1670,17 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   }
   const uint32_t smem_bytes =
       1024 + (uint32_t)ring_groups * grp_bytes + a_res_bytes + staging_bytes(stage_bufs) + kBarrierBytes;
-  if (pair && !g_pair_attr_set[dev][SPARSE ? 1 : 0]) {
+  if (pair && !FP8 && !g_pair_attr_set[dev][SPARSE ? 1 : 0]) {
     if (cudaFuncSetAttribute(ssconv_fwd_pair_kernel<SPARSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)kMaxSmemBytes) != cudaSuccess)
       return SSCONV_ERR_CUDA;
     g_pair_attr_set[dev][SPARSE ? 1 : 0] = true;
+  }
+  if (pair && FP8 && !g_pair_fp8_attr_set[dev]) {
+    if (cudaFuncSetAttribute(ssconv_fwd_pair_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kMaxSmemBytes) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
+    g_pair_fp8_attr_set[dev] = true;
   }
 
   CUtensorMap tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail;
@@ -1708,9 +1735,11 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   // come in by a tensor copy, which unlike the plain bulk copy can signal a barrier in the peer CTA
   CUtensorMap tm_meta = tm_a;
   if (pair && SPARSE) {
-    cuuint64_t dims[2] = {16, (cuuint64_t)geo.m_tiles * geo.stages * kTileM};
+    // (8-bit operands: two images per group = 256 rows)
+    const cuuint32_t rows = C::kMetaBytes / 16;
+    cuuint64_t dims[2] = {16, (cuuint64_t)geo.m_tiles * geo.stages * rows};
     cuuint64_t strides[1] = {16};
-    cuuint32_t box[2] = {16, (cuuint32_t)kTileM};
+    cuuint32_t box[2] = {16, rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode_tiled(&tm_meta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(meta), dims, strides, box,
                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
@@ -1826,7 +1855,8 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   cfg.attrs = attr;
   cfg.numAttrs = pair ? 2 : 1;
   const cudaError_t launched =
-      FP8 ? cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, false, FP8>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p)
+      (FP8 && pair) ? cudaLaunchKernelEx(&cfg, ssconv_fwd_pair_kernel<true, true>, tm_a, tm_b, tm_meta, tm_y, tm_y_tail, p)
+      : FP8 ? cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, false, FP8>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p)
       : pair ? cudaLaunchKernelEx(&cfg, ssconv_fwd_pair_kernel<SPARSE>, tm_a, tm_b, tm_meta, tm_y, tm_y_tail, p)
       : residual != nullptr
           ? cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, true>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p)

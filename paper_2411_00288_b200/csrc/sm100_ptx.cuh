@@ -473,6 +473,18 @@ __device__ __forceinline__ void tc2_mma_sparse_w(uint32_t d_tmem, uint32_t a_lo,
       ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(meta_tmem), "r"(idesc), "r"(accumulate), "r"(kDescHiSw128)
       : "memory");
 }
+__device__ __forceinline__ void tc2_mma_f8_sparse_w(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t meta_tmem,
+                                                    uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, e;\n\t.reg .b64 da, db;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
+      "mov.b64 da, {%1, %6};\n\t"
+      "mov.b64 db, {%2, %6};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "@e tcgen05.mma.sp.cta_group::2.kind::f8f6f4 [%0], da, db, [%3], %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(meta_tmem), "r"(idesc), "r"(accumulate), "r"(kDescHiSw128)
+      : "memory");
+}
 // In both CTAs: 128 rows x 128 bits from the CTA's own shared memory into its own TMEM.
 __device__ __forceinline__ void tc2_cp_128x128b_w(uint32_t dst_tmem, uint32_t src_lo) {
   asm volatile(

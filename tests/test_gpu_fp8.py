@@ -129,6 +129,43 @@ def test_forward_fp8_matches_oracle(case, sparse):
     assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"{case[0]} sparse={sparse}: rel={rel:.3e} max={mx:.3e}"
 
 
+FP8_PAIR_LAYERS = [  # run with the pair kernel forced (tiles of 256 channels on two thread blocks)
+    ("f8p_3x3_256", 2, 14, 14, 256, 256, 3, 1, 1, 1),
+    ("f8p_1x1_384to320", 3, 12, 12, 384, 320, 1, 1, 0, 1),       # three channel tiles: the last pair's second block idles
+    ("f8p_3x3_s2_c192to264", 2, 15, 17, 192, 264, 3, 2, 1, 1),   # channel tail 128 + 64, ragged channels, stride 2
+    ("f8p_1x1_c144_odd", 2, 20, 20, 144, 512, 1, 1, 0, 1),       # an odd number of k-blocks (2), tail of 16 channels
+    ("f8p_3x3_tiles", 4, 28, 28, 128, 256, 3, 1, 1, 1),          # several tiles per pair
+]
+
+
+@pytest.mark.parametrize("case", FP8_PAIR_LAYERS, ids=[c[0] for c in FP8_PAIR_LAYERS])
+def test_forward_fp8_on_thread_block_pairs_matches_oracle(case):
+    desc, shape, x, w, bias, out_scale = _fp8_case(case)
+    xd, wd, bd = torch.from_numpy(x).to(DEV), torch.from_numpy(w).to(DEV), torch.from_numpy(bias).to(DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_E4M3, wd, w.size // 4)
+    pat_ref = masks.select_from_magnitude(None, magnitudes=fp8.abs_code(w))
+    mask = masks.mask_from_pattern(pat_ref, w.shape)
+    w_comp, meta = api.ssconv_compress_fp8(desc, wd, pat)
+    band = 4096
+    ho, wo = api.ssconv_out_shape(desc)
+    n_out = desc.N * ho * wo * desc.C_out
+    buf = torch.full((n_out + 2 * band,), -7.0, dtype=torch.bfloat16, device=DEV)
+    y = buf[band:band + n_out].view(desc.N, ho, wo, desc.C_out)
+    api.ssconv_tune(api.TUNE_PAIR, 1)
+    try:
+        api.ssconv_forward_fp8(desc, xd, w_comp, meta, bd, out_scale, y=y, dev_status=status)
+        torch.cuda.synchronize()
+    finally:
+        api.ssconv_tune(api.TUNE_PAIR, -1)
+    assert int(status.item()) == 0
+    assert bool((buf[:band] == -7.0).all()) and bool((buf[-band:] == -7.0).all()) and bool((y >= 0).all())
+    acc = conv2d_f64(shape, fp8.e4m3_to_bf16_bits(x), fp8.e4m3_to_bf16_bits(w), mask=mask, bias=None)
+    ref = np.maximum(acc * np.float64(np.float32(out_scale)) + bias.astype(np.float64), 0.0)
+    rel, mx = parity.errors(parity.bf16_tensor_to_f64(y), ref)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"{case[0]}: rel={rel:.3e} max={mx:.3e}"
+
+
 def test_forward_fp8_argument_rules():
     desc, shape, x, w, bias, out_scale = _fp8_case(FP8_LAYERS[0])
     xd, wd = torch.from_numpy(x).to(DEV), torch.from_numpy(w).to(DEV)
