@@ -149,6 +149,29 @@ def test_gelu_epilogue(case, sparse, residual):
     _assert_ok(*parity.check_layer(spec, DEV, sparse=sparse, residual=residual), name)
 
 
+def test_gelu_over_every_bf16_input_up_to_8():
+    """Every finite bf16 value of magnitude up to 8 goes through a 1x1 convolution with identity weights:
+    the output must be GELU(x) = x Phi(x) from erf in fp64, to one bf16 rounding (2^-9 relative; 2^-8 is
+    allowed) plus 2e-6 absolute for the kernel's fp32 evaluation of erf."""
+    from scipy.special import erf
+    bits = np.arange(0, 0x4100 + 1, dtype=np.uint16)                       # +0 .. 8.0
+    bits = np.concatenate([bits, bits | 0x8000]).astype(np.uint16)         # and the negatives
+    n = (bits.size + 7) // 8 * 8
+    allb = np.zeros(n, dtype=np.uint16)
+    allb[:bits.size] = bits
+    x = torch.from_numpy(allb.view(np.int16)).view(torch.bfloat16).reshape(1, 1, n // 8, 8)
+    w = torch.zeros((8, 1, 1, 8), dtype=torch.bfloat16)
+    for c in range(8):
+        w[c, 0, 0, c] = 1.0
+    desc = api.make_desc(1, 1, n // 8, 8, 8, 1, 1, bias=False, gelu=True)
+    y = api.ssconv_forward_dense(desc, x.to(DEV), w.to(DEV), None).float().cpu().numpy().reshape(-1)[:bits.size]
+    xv = x.float().numpy().reshape(-1)[:bits.size].astype(np.float64)
+    ref = 0.5 * xv * (1.0 + erf(xv / np.sqrt(2.0)))
+    err = np.abs(y - ref)
+    bad = err > 2.0 ** -8 * np.abs(ref) + 2e-6
+    assert not bad.any(), (xv[bad][:5], y[bad][:5], ref[bad][:5])
+
+
 def test_gelu_matches_closed_values_and_flag_rules():
     """x == 1, one kept weight w per output channel and zero bias give y = GELU(w) exactly enough to tell
     GELU from ReLU and identity; RELU and GELU together are refused."""
