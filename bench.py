@@ -41,6 +41,27 @@ WORKLOAD = WORKLOADS[CONFIG_ID]
 MIN_REGIONS = 30       # timed regions of --steps steps each; the median is reported
 
 
+# DRAM bytes of one step of the stack at batch 256, from the ncu counters summarised in
+# profiles/bench_resnet50_stack_dram_traffic.md; valid for the kernels whose sources hash to `sources`
+# (anything else reports null: the counters would have to be taken again).
+STACK_TRAFFIC = {"batch": 256, "read": 4_511_588_480, "write": 5_833_819_136, "sources": "fae92280f2aced63"}
+TRAFFIC_SOURCES = ("paper_2411_00288_b200/csrc/forward.cu", "paper_2411_00288_b200/csrc/pool.cu",
+                   "paper_2411_00288_b200/csrc/sm100_ptx.cuh", "paper_2411_00288_b200/csrc/layout.cuh",
+                   "paper_2411_00288_b200/stack.py")
+
+
+def stack_traffic(batch, residual):
+    """Measured DRAM bytes per step, or None when the measured kernels are not the ones in the tree."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in TRAFFIC_SOURCES:
+        with open(os.path.join(ROOT, f), "rb") as fh:
+            h.update(fh.read())
+    if batch != STACK_TRAFFIC["batch"] or residual or h.hexdigest()[:16] != STACK_TRAFFIC["sources"]:
+        return None
+    return STACK_TRAFFIC["read"] + STACK_TRAFFIC["write"]
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -925,10 +946,11 @@ def stack_arm(args):
                     "sum_layer_ms": sums["t_tensor"], "tflops": sums["flops_tensor"] / max(sums["t_tensor"], 1e-9) / 1e9,
                     "peak_tflops": 2.0 * peaks["bf16_tflops"],
                     "frac": sums["roof_tensor"] / max(sums["t_tensor"], 1e-9)},
-                "traffic": None,
-                "traffic_note": "no per-step figure: outputs still in L2 when a kernel ends are never counted as written; the "
-                                "DRAM counters of single layers at this batch are in profiles/ (reads = algorithmic "
-                                "input bytes to 0.1-2 %)"},
+                "traffic": stack_traffic(batch, args.residual),
+                "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum over the 55 launches of one step (single-pass "
+                                "ncu capture at this batch, caches left alone between launches so that write-backs are "
+                                "counted in the step; profiles/bench_resnet50_stack_dram_traffic.md); null when the kernel "
+                                "sources differ from the ones measured"},
             "per_layer": per_layer,
             "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
