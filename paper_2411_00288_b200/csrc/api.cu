@@ -852,7 +852,9 @@ int32_t ssconv_dgrad(const ssconv_desc_t* desc, const void* dy, const void* w_bf
     c.pad_w = d.dil_w * (d.KW - 1) - d.pad_w;
     rc = check_desc(&c, true);
     if (rc != SSCONV_OK) return rc;
-    if (ssconv::launch_dgrad_weights(w_bf16, base, d.C_out, d.KH, d.KW, d.C_in, st) != cudaSuccess) return SSCONV_ERR_CUDA;
+    // (the reversed, channel-exchanged filter = the one class of a unit stride, written by the tiled transpose)
+    if (ssconv::launch_dgrad_fused_weights(w_bf16, base, d.C_out, d.KH, d.KW, d.C_in, d.KH, d.KW, 1, 1, st) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
     return ssconv::launch_forward_dense(c, dy, base, nullptr, nullptr, dx, base + p.fwd_off, p.fwd_bytes, dev_status, st);
   }
   ssconv::DgradClasses cls;
