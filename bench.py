@@ -1012,9 +1012,16 @@ def sweep_arm(args):
         xs = [inp.x.to(dev)] + [torch.randn(inp.x.shape, device=dev).to(torch.bfloat16) for _ in range(n_sets - 1)]
         ys = [torch.empty((spec.N, spec.H_out, spec.W_out, spec.C_out), dtype=torch.bfloat16, device=dev)
               for _ in range(n_sets)]
+        if args.e4m3:   # the same layer on 8-bit operands (2:4 form)
+            wq = api.ssconv_quantize_e4m3(w, 16.0)
+            pq = api.ssconv_select_mask(api.MASK_MAGNITUDE_E4M3, wq, wq.numel() // 4)
+            wq_comp, metaq = api.ssconv_compress_fp8(desc, wq, pq)
+            xq = [api.ssconv_quantize_e4m3(x, 1.0) for x in xs]
         for i in range(args.layer_iters):
             r = i % n_sets
-            if args.dense:
+            if args.e4m3:
+                api.ssconv_forward_fp8(desc, xq[r], wq_comp, metaq, bias, 1.0 / 16.0, y=ys[r], dev_status=status)
+            elif args.dense:
                 api.ssconv_forward_dense(desc, xs[r], w, bias, y=ys[r], dev_status=status)
             else:
                 api.ssconv_forward(desc, xs[r], w_comp, meta, bias, y=ys[r], dev_status=status)
@@ -1156,6 +1163,7 @@ def main():
     ap.add_argument("--train", action="store_true",
                     help="time one mask-learning step per layer (soft mask, dense forward, weight gradient, "
                          "choice-weight gradient) on one of the per-layer sweeps (default: the ResNet-18 sweep)")
+    ap.add_argument("--e4m3", action="store_true", help="with --only-layer: launch the layer's 2:4 e4m3 form")
     ap.add_argument("--convnext", action="store_true",
                     help="only the ConvNeXt-T-shaped forward pass (the default line's summary_convnext_t), one GPU")
     ap.add_argument("--batch", type=int, default=None, help="images per GPU of the stack (default 256)")
