@@ -447,12 +447,146 @@ __global__ void __launch_bounds__(128, 4) depthwise_run_kernel(const uint2* __re
   }
 }
 
+// Unit stride, no dilation, square K x K filter, C a multiple of 32: a thread computes a tile of
+// kDwTileH x kDwTileW output pixels for one pair of channels, so that an image pixel is loaded and widened
+// once for all the (up to K per direction) outputs of the tile it meets: (kDwTileH + K - 1)(kDwTileW + K - 1)
+// four-byte loads for kDwTileH kDwTileW K^2 paired multiply-adds (140 for 1568 with K = 7), against one load
+// per K paired multiply-adds in the row-run kernel above.  Sixteen lanes hold sixteen neighbouring channel
+// pairs of one tile (64 contiguous bytes per pixel); a block's eight tiles share the same 32 channels,
+// whose filter it keeps in shared memory as fp32 pairs.  The loop over image rows stays rolled (the filter
+// row under which image row r meets output row o is r - o, looked up at run time): unrolled, the kernel
+// waited on instruction fetch.  Addresses are a per-row pointer plus 32-bit offsets, constants when the
+// channel count is one of the instantiated ones (C2T, in channel pairs; 0 = taken from the argument).
+// The tile is TW = 8 pixels wide, or 7 where that divides the output width and 8 does not (feature maps
+// of 7, 14, 28 and 56 pixels: no multiply-adds spent beyond the row's end); output rows beyond the
+// map's last are skipped.
+constexpr int kDwTileH = 4;
+__device__ __forceinline__ float2 widen_f2(uint32_t v) {
+  return make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xFFFF0000u));
+}
+template <int K, int C2T, int TW>
+__global__ void __launch_bounds__(128, 4) depthwise_tile_kernel(const uint32_t* __restrict__ x, const uint32_t* __restrict__ w,
+                                                                const float* __restrict__ bias, uint32_t* __restrict__ y,
+                                                                int H, int W, int C2r, int Ho, int Wo, int pad, int tiles_h,
+                                                                int tiles_w, long long tiles, uint32_t flags) {
+  const int C2 = C2T ? C2T : C2r;
+  __shared__ float2 w_s[K * K][16];
+  const int sub = threadIdx.x & 15;
+  const int c2 = blockIdx.y * 16 + sub;
+  for (int i = threadIdx.x; i < K * K * 16; i += 128)
+    w_s[i >> 4][i & 15] = widen_f2(__ldg(w + (long long)(i >> 4) * C2 + blockIdx.y * 16 + (i & 15)));
+  __syncthreads();
+  long long tile = (long long)blockIdx.x * 8 + (threadIdx.x >> 4);
+  if (tile >= tiles) return;
+  const int tw = (int)(tile % tiles_w);
+  tile /= tiles_w;
+  const int th = (int)(tile % tiles_h);
+  const int n = (int)(tile / tiles_h);
+  const int h0 = th * kDwTileH, w0 = tw * TW;
+  constexpr int kCols = TW + K - 1, kRows = kDwTileH + K - 1;
+  float2 acc[kDwTileH][TW];
+  {
+    float2 b = make_float2(0.0f, 0.0f);
+    if (flags & SSCONV_FLAG_BIAS) b = __ldg(reinterpret_cast<const float2*>(bias) + c2);
+#pragma unroll
+    for (int o = 0; o < kDwTileH; ++o)
+#pragma unroll
+      for (int t = 0; t < TW; ++t) acc[o][t] = b;
+  }
+  const int wi0 = w0 - pad;  // image column under the tile's first output at tap 0
+  const bool cols_in = wi0 >= 0 && wi0 + kCols <= W;
+  // image column wi0 of image row h0 - pad (possibly outside the image: dereferenced only where it is inside)
+  const uint32_t* rowp = x + (((long long)n * H + (h0 - pad)) * W + wi0) * C2 + c2;
+  const int row_step = W * C2;
+  const float2* wp = &w_s[0][sub];
+#pragma unroll 1
+  for (int r = 0; r < kRows; ++r, rowp += row_step) {
+    const int h = h0 - pad + r;
+    if (h < 0 || h >= H) continue;
+    float2 xv[kCols];
+    if (cols_in) {
+#pragma unroll
+      for (int col = 0; col < kCols; ++col) xv[col] = widen_f2(__ldg(rowp + col * C2));
+    } else {
+#pragma unroll
+      for (int col = 0; col < kCols; ++col) {
+        uint32_t v = 0u;
+        if (wi0 + col >= 0 && wi0 + col < W) v = __ldg(rowp + col * C2);
+        xv[col] = widen_f2(v);
+      }
+    }
+#pragma unroll
+    for (int o = 0; o < kDwTileH; ++o) {
+      const int ky = r - o;  // filter row under which image row r meets output row o of the tile
+      if (ky < 0 || ky >= K || h0 + o >= Ho) continue;
+      const float2* wr = wp + ky * (K * 16);
+#pragma unroll
+      for (int kx = 0; kx < K; ++kx) {
+        const float2 wk = wr[kx * 16];
+#pragma unroll
+        for (int t = 0; t < TW; ++t) acc[o][t] = __ffma2_rn(xv[t + kx], wk, acc[o][t]);
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 0; o < kDwTileH; ++o) {
+    if (h0 + o >= Ho) break;
+    uint32_t* out = y + (((long long)n * Ho + h0 + o) * Wo + w0) * C2 + c2;
+#pragma unroll
+    for (int t = 0; t < TW; ++t) {
+      if (w0 + t >= Wo) break;
+      float lo = acc[o][t].x, hi = acc[o][t].y;
+      if (flags & SSCONV_FLAG_RELU) {
+        lo = fmaxf(lo, 0.0f);
+        hi = fmaxf(hi, 0.0f);
+      }
+      __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+      out[t * C2] = *reinterpret_cast<uint32_t*>(&b2);
+    }
+  }
+}
+
 cudaError_t launch_depthwise(const void* x, const void* w, const float* bias, void* y, int N, int H, int W, int C, int Ho,
                              int Wo, int KH, int KW, int stride, int pad, int dil, uint32_t flags, cudaStream_t st) {
   const long long total = (long long)N * Ho * Wo * (C / 8);
   if (total == 0) return cudaSuccess;
   const int T = 256;
   count_launch();
+  if (stride == 1 && dil == 1 && KH == KW && (KW == 3 || KW == 5 || KW == 7) && C % 32 == 0) {
+    const int tw = (KW == 7 && Wo % 7 == 0 && Wo % 8 != 0) ? 7 : 8;
+    const int tiles_h = (Ho + kDwTileH - 1) / kDwTileH, tiles_w = (Wo + tw - 1) / tw;
+    const long long tiles = (long long)N * tiles_h * tiles_w;
+    const dim3 grid((unsigned)((tiles + 7) / 8), (unsigned)(C / 32));
+    const uint32_t* xp = static_cast<const uint32_t*>(x);
+    const uint32_t* wp = static_cast<const uint32_t*>(w);
+    uint32_t* yp = static_cast<uint32_t*>(y);
+#define SSCONV_DW_TILE(KK, CC, TT) \
+  depthwise_tile_kernel<KK, CC, TT><<<grid, 128, 0, st>>>(xp, wp, bias, yp, H, W, C / 2, Ho, Wo, pad, tiles_h, tiles_w, tiles, flags)
+#define SSCONV_DW_TILE7(CC)  \
+  do {                       \
+    if (tw == 7)             \
+      SSCONV_DW_TILE(7, CC, 7); \
+    else                     \
+      SSCONV_DW_TILE(7, CC, 8); \
+  } while (0)
+    if (KW == 3)
+      SSCONV_DW_TILE(3, 0, 8);
+    else if (KW == 5)
+      SSCONV_DW_TILE(5, 0, 8);
+    else if (C == 96)
+      SSCONV_DW_TILE7(48);
+    else if (C == 192)
+      SSCONV_DW_TILE7(96);
+    else if (C == 384)
+      SSCONV_DW_TILE7(192);
+    else if (C == 768)
+      SSCONV_DW_TILE7(384);
+    else
+      SSCONV_DW_TILE7(0);
+#undef SSCONV_DW_TILE7
+#undef SSCONV_DW_TILE
+    return cudaGetLastError();
+  }
   if (stride == 1 && dil == 1 && (KW == 3 || KW == 5 || KW == 7)) {
     const int runs = (Wo + kDwRun - 1) / kDwRun;
     const long long threads = (long long)N * Ho * runs * (C / 4);
@@ -574,8 +708,14 @@ cudaError_t launch_layernorm(const void* x, const float* gamma, const float* bet
                          reinterpret_cast<uintptr_t>(beta)) & 15u) == 0;
   if (C % 8 == 0 && C <= 1024 && aligned) {
     const int C8 = C / 8;
+    // lanes per pixel: the largest power of two dividing C8 if that leaves at most four pieces per lane
+    // (every lane busy: 96 channels = 4 lanes x 3 pieces), else the smallest power of two covering C8
     int G = 1;
-    while (G < C8 && G < 32) G <<= 1;
+    while (G < 32 && C8 % (2 * G) == 0) G <<= 1;
+    if (C8 / G > 4) {
+      G = 1;
+      while (G < C8 && G < 32) G <<= 1;
+    }
     const int V = (C8 + G - 1) / G;
     const long long warps = (pixels + (32 / G) - 1) / (32 / G);
     const unsigned grid = (unsigned)((warps * 32 + T - 1) / T);

@@ -72,9 +72,14 @@ def test_grouped_convolution_matches_oracle(case, sparse):
     assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"rel={rel:.3e} max={mx:.3e}"
 
 
-@pytest.mark.parametrize("case", [(2, 14, 14, 96, 7, 1, 3, 1), (2, 15, 13, 64, 3, 2, 1, 1), (1, 12, 12, 8, 3, 1, 2, 2)],
-                         ids=["7x7", "3x3s2", "3x3d2"])
+@pytest.mark.parametrize("case", [(2, 14, 14, 96, 7, 1, 3, 1), (2, 15, 13, 64, 3, 2, 1, 1), (1, 12, 12, 8, 3, 1, 2, 2),
+                                  (3, 7, 7, 64, 7, 1, 3, 1), (1, 19, 21, 32, 5, 1, 2, 1), (2, 9, 11, 32, 3, 1, 0, 1),
+                                  (1, 10, 13, 160, 7, 1, 1, 1), (1, 17, 9, 40, 7, 1, 3, 1), (2, 33, 18, 32, 7, 1, 5, 1)],
+                         ids=["7x7", "3x3s2", "3x3d2", "7x7_map7_tile_tails", "5x5_c32", "3x3_pad0", "7x7_pad1", "7x7_c40_row_runs",
+                              "7x7_pad5"])
 def test_depthwise_matches_oracle(case):
+    # unit-stride square filters on channel counts that are multiples of 32 run on the tile kernel (4 x 8 outputs
+    # per thread), other unit-stride ones on the row-run kernel, the rest on the generic one
     N, H, W, C, K, s, p, d = case
     g = torch.Generator().manual_seed(synth.SEED_BASE + 3100 + C + K)
     x = torch.randn((N, H, W, C), generator=g).to(torch.bfloat16)
