@@ -186,22 +186,25 @@ __global__ void __launch_bounds__(256) space_to_depth_kernel(const unsigned shor
   }
 }
 
-// The same for RGB images, blocks of 2 x 2 pixels and unpadded pixels of 12 channels (24 bytes): a row
-// of y interleaves 12-byte pieces of two image rows, so a block stages the two rows in shared memory
-// (16-byte loads; element (w + pad) 3 + c of a staged row is channel c of column w, zeros outside the
-// image) and writes the row of y as 8-byte words: pixel q is elements 6 q .. 6 q + 5 of the first row,
-// then of the second.  Every image byte is read once and every byte of y written once.
-__global__ void __launch_bounds__(128) space_to_depth_rgb2_kernel(const uint4* __restrict__ x, uint2* __restrict__ y, int H,
-                                                                  int W, int pad, int Hb, int Wb) {
-  extern __shared__ uint32_t s2d_rows[];  // two rows of 3 Wb words (6 Wb elements)
+// The same for RGB images and blocks of S x S pixels, S = 2 or 4, with unpadded pixels of 3 S S channels
+// (24 or 96 bytes): a row of y interleaves pieces of 3 S elements of S image rows, so a block stages the S
+// rows in shared memory (16-byte loads; element (w + pad) 3 + c of a staged row is channel c of column w,
+// zeros outside the image) and writes the row of y as 8-byte words: pixel q is elements 3 S q .. 3 S q + 3 S - 1
+// of the first row, then of the second, and so on.  Every image byte is read once and every byte of y
+// written once.
+template <int S>
+__global__ void __launch_bounds__(128) space_to_depth_rgb_kernel(const uint4* __restrict__ x, uint2* __restrict__ y, int H,
+                                                                 int W, int pad, int Hb, int Wb) {
+  extern __shared__ uint32_t s2d_rows[];  // S rows of 3 S Wb / 2 words (3 S Wb elements)
   const int row = blockIdx.x;
   const int n = row / Hb, r = row - n * Hb;
-  const int words = 3 * Wb;
+  constexpr int kPieceWords = 3 * S / 2;       // words of one image row in one pixel of y
+  const int words = kPieceWords * Wb;          // words of a staged row
   unsigned short* el = reinterpret_cast<unsigned short*>(s2d_rows);
-  const int lead = pad * 3, body = W * 3, len = 6 * Wb;
+  const int lead = pad * 3, body = W * 3, len = 2 * words;
 #pragma unroll
-  for (int dy = 0; dy < 2; ++dy) {
-    const int h = 2 * r - pad + dy;
+  for (int dy = 0; dy < S; ++dy) {
+    const int h = S * r - pad + dy;
     unsigned short* dst = el + dy * len;
     if (h < 0 || h >= H) {
       for (int i = threadIdx.x; i < words; i += blockDim.x) s2d_rows[dy * words + i] = 0u;
@@ -222,25 +225,43 @@ __global__ void __launch_bounds__(128) space_to_depth_rgb2_kernel(const uint4* _
     }
   }
   __syncthreads();
-  uint2* out = y + (size_t)row * words;
-  const uint32_t* r0 = s2d_rows;
-  const uint32_t* r1 = s2d_rows + words;
-  for (int u = threadIdx.x; u < words; u += blockDim.x) {
-    const int q = u / 3, part = u - 3 * q;
-    uint2 o;
-    if (part == 0) o = make_uint2(r0[3 * q], r0[3 * q + 1]);
-    else if (part == 1) o = make_uint2(r0[3 * q + 2], r1[3 * q]);
-    else o = make_uint2(r1[3 * q + 1], r1[3 * q + 2]);
-    out[u] = o;
+  const int out_words = S * words / 2;  // 8-byte words of the row of y
+  uint2* out = y + (size_t)row * out_words;
+  if (S == 2) {
+    const uint32_t* r0 = s2d_rows;
+    const uint32_t* r1 = s2d_rows + words;
+    for (int u = threadIdx.x; u < out_words; u += blockDim.x) {
+      const int q = u / 3, part = u - 3 * q;
+      uint2 o;
+      if (part == 0) o = make_uint2(r0[3 * q], r0[3 * q + 1]);
+      else if (part == 1) o = make_uint2(r0[3 * q + 2], r1[3 * q]);
+      else o = make_uint2(r1[3 * q + 1], r1[3 * q + 2]);
+      out[u] = o;
+    }
+  } else {
+    // a pixel of y is S pieces of kPieceWords (an even number of) words: 8-byte word p of pixel q comes from
+    // row p / (kPieceWords / 2), words kPieceWords q + 2 (p % (kPieceWords / 2)) and the next
+    constexpr int kHalf = kPieceWords / 2;
+    for (int u = threadIdx.x; u < out_words; u += blockDim.x) {
+      const int q = u / (S * kHalf), p = u - q * (S * kHalf);
+      const int dy = p / kHalf, part = p - dy * kHalf;
+      out[u] = *reinterpret_cast<const uint2*>(s2d_rows + dy * words + kPieceWords * q + 2 * part);
+    }
   }
 }
 
 cudaError_t launch_space_to_depth(const void* x, void* y, int N, int H, int W, int C, int s, int pad, int Hb, int Wb,
                                   int C_pad, cudaStream_t st) {
   count_launch();
-  if (s == 2 && C == 3 && C_pad == 12 && W % 8 == 0 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && Wb <= 1024) {
-    space_to_depth_rgb2_kernel<<<(unsigned)(N * Hb), 128, (size_t)Wb * 24, st>>>(
-        static_cast<const uint4*>(x), static_cast<uint2*>(y), H, W, pad, Hb, Wb);
+  if ((s == 2 || s == 4) && C == 3 && C_pad == 3 * s * s && W % 8 == 0 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 &&
+      Wb <= 1024 / s) {
+    // (an image row ends at a 16-byte boundary when W is a multiple of 8; the staged rows take 6 s s Wb bytes)
+    if (s == 2)
+      space_to_depth_rgb_kernel<2><<<(unsigned)(N * Hb), 128, (size_t)Wb * 24, st>>>(
+          static_cast<const uint4*>(x), static_cast<uint2*>(y), H, W, pad, Hb, Wb);
+    else
+      space_to_depth_rgb_kernel<4><<<(unsigned)(N * Hb), 128, (size_t)Wb * 96, st>>>(
+          static_cast<const uint4*>(x), static_cast<uint2*>(y), H, W, pad, Hb, Wb);
     return cudaGetLastError();
   }
   const int T = 256;

@@ -121,8 +121,12 @@ def _s2d_numpy(x_bits, s, pad, Hb, Wb, c_pad):
     ((2, 10, 11, 3), 2, 3, 8, 9, 12),      # odd width: the generic kernel at 8-byte granularity
     ((1, 7, 9, 1), 3, 2, 4, 5, 12),        # one channel, blocks of 3 x 3
     ((64, 7, 7, 3), 2, 0, 4, 4, 12),       # a weight tensor
+    ((2, 32, 24, 3), 4, 0, 8, 6, 48),      # RGB, blocks of 4 x 4 (a patchify stem): the staged four-row kernel
+    ((3, 18, 16, 3), 4, 3, 7, 6, 48),      # the same with padding on every side and rows past the bottom edge
+    ((1, 16, 40, 3), 4, 2, 4, 7, 48),      # fewer block columns than the image has: the row's tail is dropped
+    ((2, 12, 10, 3), 4, 1, 4, 4, 48),      # width not a multiple of 8: the generic kernel
 ])
-def test_space_to_depth_with_12_channel_pixels_is_bit_exact(shape, s, pad, Hb, Wb, c_pad):
+def test_space_to_depth_of_few_channel_images_is_bit_exact(shape, s, pad, Hb, Wb, c_pad):
     g = torch.Generator().manual_seed(synth.SEED_BASE + 3500 + shape[1] + shape[2])
     x = torch.randn(shape, generator=g).to(torch.bfloat16)
     band = 64
