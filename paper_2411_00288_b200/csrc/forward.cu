@@ -228,27 +228,20 @@ __device__ __forceinline__ void tc_ld_piece(uint32_t taddr, uint32_t (&r)[kPiece
 // 0.5 x (1 + erf(x / sqrt 2)), evaluated in fp32 before the rounding.
 // erf without branches: erf(z) = 1 - 2^R(z) for z >= 0 with R a degree-6 polynomial (no constant term)
 // fitted to log2(erfc(z)) on [0, 4] (beyond 4, erfc < 2e-8 and z is clamped), odd extension by the sign of
-// x.  The difference 1 - 2^R loses relative accuracy near 0, which x Phi(x) does not need: against fp64
-// over every bf16 input up to 8 the result is within 5.1e-6 absolute and 3.3e-5 relative of x Phi(x)
-// (|R - log2 erfc| <= 4.8e-5), a sixtieth of the rounding to bf16 that follows (2^-9); a degree-8 fit
-// (3e-6 relative) bought nothing after that rounding and cost two more multiply-adds per value, which
-// matters because shallow layers with this activation are bound by the epilogue's arithmetic.
+// x; the factor 1 / sqrt 2 of z = |x| / sqrt 2 is folded into the coefficients, so the polynomial takes
+// |x| clamped at 4 sqrt 2.  The difference 1 - 2^R loses relative accuracy near 0, which x Phi(x) does not
+// need.  Against fp64 over every bf16 input up to 8: |R - log2 erfc| <= 4.8e-5, i.e. 3.3e-5 relative in
+// exact arithmetic; evaluated in fp32 the result is within 5.1e-6 absolute, and within 3e-4 relative
+// wherever |x Phi(x)| > 1e-4 (the largest ratio sits in the far negative tail, where 0.5 x and |x| t
+// cancel), a seventh of the rounding to bf16 that follows (2^-9).  A degree-8 fit bought nothing after that
+// rounding and cost two more multiply-adds per value, which matters because shallow layers with this
+// activation are bound by the epilogue's arithmetic.
 constexpr int kActNone = 0, kActRelu = 1, kActGelu = 2;
-__device__ __forceinline__ float gelu_f32(float x) {
-  const float z = fminf(fabsf(x) * 0.70710678118654752f, 4.0f);
-  float r = 0.00020432738529052585f;
-  r = fmaf(r, z, -0.003693065606057644f);
-  r = fmaf(r, z, 0.02980932965874672f);
-  r = fmaf(r, z, -0.14685025811195374f);
-  r = fmaf(r, z, -0.9205983281135559f);
-  r = fmaf(r, z, -1.6273139715194702f);
-  r *= z;
-  float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(r));
-  // x (0.5 + sign(x) (0.5 - 0.5 e)) = 0.5 x + |x| (0.5 - 0.5 e)
-  return fmaf(fmaf(-0.5f, e, 0.5f), fabsf(x), 0.5f * x);
-}
-// The same for two values at once, the polynomial on fp32 pairs (fma.rn.f32x2).
+constexpr float kGeluClamp = 5.656854152679443f;  // 4 sqrt 2
+constexpr float kGeluC1 = -1.1506847143173218f, kGeluC2 = -0.46029916405677795f, kGeluC3 = -0.05191940814256668f,
+                kGeluC4 = 0.00745233241468668f, kGeluC5 = -0.0006528479279950261f, kGeluC6 = 2.5540923161315732e-05f;
+// Two values at once, the polynomial on fp32 pairs (fma.rn.f32x2); the result is formed as
+// x (0.5 + sign(x) (0.5 - 0.5 e)) = 0.5 x + |x| (0.5 - 0.5 e) with e = 2^R.
 __device__ __forceinline__ unsigned long long f32x2(float lo, float hi) {
   unsigned long long r;
   asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
@@ -259,15 +252,14 @@ __device__ __forceinline__ unsigned long long horner2(unsigned long long r, unsi
   return r;
 }
 __device__ __forceinline__ void gelu_f32x2(float& lo, float& hi) {
-  const unsigned long long z = f32x2(fminf(fabsf(lo) * 0.70710678118654752f, 4.0f),
-                                     fminf(fabsf(hi) * 0.70710678118654752f, 4.0f));
-  unsigned long long r = f32x2(0.00020432738529052585f, 0.00020432738529052585f);
-  r = horner2(r, z, -0.003693065606057644f);
-  r = horner2(r, z, 0.02980932965874672f);
-  r = horner2(r, z, -0.14685025811195374f);
-  r = horner2(r, z, -0.9205983281135559f);
-  r = horner2(r, z, -1.6273139715194702f);
-  asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(r) : "l"(z));
+  const unsigned long long a = f32x2(fminf(fabsf(lo), kGeluClamp), fminf(fabsf(hi), kGeluClamp));
+  unsigned long long r = f32x2(kGeluC6, kGeluC6);
+  r = horner2(r, a, kGeluC5);
+  r = horner2(r, a, kGeluC4);
+  r = horner2(r, a, kGeluC3);
+  r = horner2(r, a, kGeluC2);
+  r = horner2(r, a, kGeluC1);
+  asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(r) : "l"(a));
   float r0, r1, e0, e1;
   asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(r));
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(r0));
