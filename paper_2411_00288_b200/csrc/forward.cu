@@ -251,7 +251,15 @@ __device__ __forceinline__ unsigned long long horner2(unsigned long long r, unsi
   asm("fma.rn.f32x2 %0, %0, %1, %2;" : "+l"(r) : "l"(z), "l"(f32x2(c, c)));
   return r;
 }
-__device__ __forceinline__ void gelu_f32x2(float& lo, float& hi) {
+__device__ __forceinline__ void split2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// GELU of the pair x, returned as a pair; everything that has a paired form is done on pairs (the polynomial,
+// 0.5 - 0.5 e, 0.5 x and the final multiply-add), so that the eight epilogue warps issue as few instructions as
+// possible: the result is x s + 0.5 x with s = sign(x) (0.5 - 0.5 e).
+__device__ __forceinline__ unsigned long long gelu_f32x2(unsigned long long x) {
+  float lo, hi;
+  split2(x, lo, hi);
   const unsigned long long a = f32x2(fminf(fabsf(lo), kGeluClamp), fminf(fabsf(hi), kGeluClamp));
   unsigned long long r = f32x2(kGeluC6, kGeluC6);
   r = horner2(r, a, kGeluC5);
@@ -261,15 +269,22 @@ __device__ __forceinline__ void gelu_f32x2(float& lo, float& hi) {
   r = horner2(r, a, kGeluC1);
   asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(r) : "l"(a));
   float r0, r1, e0, e1;
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(r));
+  split2(r, r0, r1);
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(r0));
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(r1));
-  lo = fmaf(fmaf(-0.5f, e0, 0.5f), fabsf(lo), 0.5f * lo);
-  hi = fmaf(fmaf(-0.5f, e1, 0.5f), fabsf(hi), 0.5f * hi);
+  unsigned long long t = f32x2(e0, e1);
+  asm("fma.rn.f32x2 %0, %0, %1, %2;" : "+l"(t) : "l"(f32x2(-0.5f, -0.5f)), "l"(f32x2(0.5f, 0.5f)));
+  float t0, t1;
+  split2(t, t0, t1);
+  const unsigned long long sgn = f32x2(copysignf(t0, lo), copysignf(t1, hi));
+  unsigned long long y;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(y) : "l"(x), "l"(f32x2(0.5f, 0.5f)));
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(y) : "l"(x), "l"(sgn));
+  return y;
 }
 template <int ACT>
 __device__ __forceinline__ uint32_t activate_pack(float lo, float hi) {
-  if (ACT == kActGelu) gelu_f32x2(lo, hi);
+  if (ACT == kActGelu) split2(gelu_f32x2(f32x2(lo, hi)), lo, hi);
   return pack_bf16x2<ACT == kActRelu>(lo, hi);
 }
 __host__ __device__ inline int activation_of(uint32_t flags) {
@@ -285,6 +300,15 @@ __device__ __forceinline__ void stage_piece(const uint32_t (&r)[kPiece], const f
 #pragma unroll
     for (int i = 0; i < 4; ++i) {  // channel block i = 2 h + s of the warp's 32 channels
       const int at = 20 * (i >> 1) + 4 * k + 2 * (i & 1);
+      if (ACT == kActGelu && !RES) {
+        // (the bias goes in as a pair too)
+        unsigned long long x = f32x2(__uint_as_float(r[at]), __uint_as_float(r[at + 1]));
+        asm("add.rn.f32x2 %0, %0, %1;" : "+l"(x) : "l"(f32x2(bias[i], bias[i])));
+        float lo, hi;
+        split2(gelu_f32x2(x), lo, hi);
+        w[i] = pack_bf16x2<false>(lo, hi);
+        continue;
+      }
       float lo = __uint_as_float(r[at]) + bias[i], hi = __uint_as_float(r[at + 1]) + bias[i];
       if (RES) {
         lo += bf16_lo(res[i]);
