@@ -359,10 +359,12 @@ int32_t ssconv_wgrad(const ssconv_desc_t* desc, const void* x, const void* dy, f
  * kh = a, a + s, ..., so each class is a unit-stride convolution of dy with its own few taps (all classes
  * together carry the layer's KH x KW taps, where ssconv_dgrad_spread makes every input pixel meet all of
  * them, s_h s_w - 1 of every s_h s_w products being zeros), written to scratch and interleaved into dx
- * by a gather kernel.  The flags of desc are ignored (no bias, no activation).
+ * by a gather kernel.  Strided layers with a dilation other than 1 or a stride above 4 take the plain route
+ * instead (dy spread out with zeros as by ssconv_dgrad_spread, into scratch, then one convolution).
+ * The flags of desc are ignored (no bias, no activation).
  * ws: device scratch of ssconv_dgrad_ws_bytes(desc) bytes (reversed weights; per class its weights and
- * tensor), too small -> SSCONV_ERR_WORKSPACE.  SSCONV_ERR_UNSUPPORTED_SHAPE: padding beyond the filter's
- * reach, C_out % 8 != 0, and for strided layers a dilation other than 1 or a stride above 4. */
+ * tensor, or the spread gradient), too small -> SSCONV_ERR_WORKSPACE.  SSCONV_ERR_UNSUPPORTED_SHAPE: padding
+ * beyond the filter's reach, C_out % 8 != 0. */
 int32_t ssconv_dgrad_ws_bytes(const ssconv_desc_t* desc, size_t* bytes);
 int32_t ssconv_dgrad(const ssconv_desc_t* desc, const void* dy, const void* w_bf16, void* dx, void* ws, size_t ws_bytes,
                      int32_t* dev_status, void* stream);

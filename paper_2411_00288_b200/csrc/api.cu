@@ -745,6 +745,9 @@ int32_t ssconv_dgrad_prepare(const ssconv_desc_t* desc, const void* w_bf16, void
 namespace {
 struct DgradPlan {
   bool strided;
+  bool spread;                      // strided with a dilation, or a stride above 4: zero-spread dy, one convolution
+  int Hz, Wz;                       // extents of the spread gradient
+  size_t spread_off;
   int classes;                      // stride_h * stride_w
   int Ja[4], Jb[4];                 // taps per residue of the padded row / column
   int Ho, Wo;
@@ -766,13 +769,26 @@ int32_t dgrad_plan(const ssconv_desc_t& d, DgradPlan* p) {
   p->Wo = (d.W + 2 * d.pad_w - d.dil_w * (d.KW - 1) - 1) / d.stride_w + 1;
   const size_t w_bytes = (size_t)d.C_in * d.KH * d.KW * d.C_out * 2;
   p->fwd_bytes = ssconv::workspace_bytes();
+  p->spread = false;
   if (!p->strided) {
     p->classes = 1;
     p->fwd_off = round256(w_bytes);
     p->bytes = p->fwd_off + p->fwd_bytes;
     return SSCONV_OK;
   }
-  if (d.dil_h != 1 || d.dil_w != 1 || d.stride_h > 4 || d.stride_w > 4) return SSCONV_ERR_UNSUPPORTED_SHAPE;
+  p->spread = d.dil_h != 1 || d.dil_w != 1 || d.stride_h > 4 || d.stride_w > 4;
+  if (p->spread) {
+    // The residue classes are built for undilated filters and strides up to 4.  The rest (rare shapes) take
+    // the plain route: dy spread out by the stride with zeros in between, then the unit-stride convolution
+    // with the reversed filter; its multiplications by the zeros are the price.
+    p->classes = 1;
+    p->Hz = d.H + 2 * d.pad_h - d.dil_h * (d.KH - 1);
+    p->Wz = d.W + 2 * d.pad_w - d.dil_w * (d.KW - 1);
+    p->spread_off = round256(w_bytes);
+    p->fwd_off = p->spread_off + round256((size_t)d.N * p->Hz * p->Wz * d.C_out * 2);
+    p->bytes = p->fwd_off + p->fwd_bytes;
+    return SSCONV_OK;
+  }
   p->classes = d.stride_h * d.stride_w;
   for (int a = 0; a < d.stride_h; ++a) p->Ja[a] = a < d.KH ? (d.KH - 1 - a) / d.stride_h + 1 : 0;
   for (int b = 0; b < d.stride_w; ++b) p->Jb[b] = b < d.KW ? (d.KW - 1 - b) / d.stride_w + 1 : 0;
@@ -856,6 +872,21 @@ int32_t ssconv_dgrad(const ssconv_desc_t* desc, const void* dy, const void* w_bf
     if (ssconv::launch_dgrad_fused_weights(w_bf16, base, d.C_out, d.KH, d.KW, d.C_in, d.KH, d.KW, 1, 1, st) != cudaSuccess)
       return SSCONV_ERR_CUDA;
     return ssconv::launch_forward_dense(c, dy, base, nullptr, nullptr, dx, base + p.fwd_off, p.fwd_bytes, dev_status, st);
+  }
+  if (p.spread) {
+    c.H = p.Hz;
+    c.W = p.Wz;
+    c.pad_h = d.dil_h * (d.KH - 1) - d.pad_h;
+    c.pad_w = d.dil_w * (d.KW - 1) - d.pad_w;
+    rc = check_desc(&c, true);
+    if (rc != SSCONV_OK) return rc;
+    if (ssconv::launch_dgrad_fused_weights(w_bf16, base, d.C_out, d.KH, d.KW, d.C_in, d.KH, d.KW, 1, 1, st) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
+    if (ssconv::launch_dgrad_spread(dy, base + p.spread_off, d.N, p.Ho, p.Wo, d.C_out, p.Hz, p.Wz, d.stride_h, d.stride_w,
+                                    st) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
+    return ssconv::launch_forward_dense(c, base + p.spread_off, base, nullptr, nullptr, dx, base + p.fwd_off, p.fwd_bytes,
+                                        dev_status, st);
   }
   ssconv::DgradClasses cls;
   for (int k = 0; k < ssconv::kMaxDgradClasses; ++k) {

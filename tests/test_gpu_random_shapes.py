@@ -60,3 +60,78 @@ def test_the_draw_is_varied():
     assert any(s.C_out > 128 for s in specs) and any(s.C_out < 64 for s in specs) and any(s.C_in % 64 for s in specs)
     assert any(c[1] for c in CASES) and any(s.gelu for s in specs) and any(not s.has_bias for s in specs)
     assert any(s.KH != s.KW for s in specs)
+
+
+# ---------------------------------------------------------------- the training kernels on drawn shapes
+def _draw_train_cases(count, seed, max_macs):
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < count:
+        KH, KW = (int(rng.choice([1, 1, 2, 3, 3, 5, 7])) for _ in range(2))
+        d = int(rng.choice([1, 1, 1, 2]))
+        s = int(rng.choice([1, 1, 2, 2, 3]))
+        p = int(rng.integers(0, min(d * (KH - 1), d * (KW - 1)) + 1)) if min(KH, KW) > 1 else 0
+        N, H, W = int(rng.integers(1, 5)), int(rng.integers(1, 33)), int(rng.integers(1, 33))
+        Ci = int(rng.choice([8, 16, 40, 64, 72, 104, 128, 192, 256, 320]))
+        Co = int(rng.choice([8, 24, 40, 64, 96, 128, 136, 200, 256, 328]))
+        spec = synth.LayerSpec(f"trn{len(cases)}", N, H, W, Ci, Co, KH, KW, s, p, d, config=13, index=len(cases))
+        if spec.H_out < 1 or spec.W_out < 1 or spec.P * Co * spec.K > max_macs:
+            continue
+        cases.append(spec)
+    return cases
+
+
+def _tid(s):
+    return f"{s.name}_{s.N}x{s.H}x{s.W}x{s.C_in}to{s.C_out}_k{s.KH}x{s.KW}s{s.stride}p{s.pad}d{s.dil}"
+
+
+WG_CASES = _draw_train_cases(24, 2411_00289, 4e8)
+DG_CASES = _draw_train_cases(24, 2411_00290, 2e8)
+
+
+@pytest.mark.parametrize("spec", WG_CASES, ids=[_tid(s) for s in WG_CASES])
+def test_random_shape_weight_gradient_matches_oracle(spec):
+    """dL/dW of Eq. 4 (Sec. 3.1's training step differentiates it): fp32 accumulation of exact products."""
+    from oracle import train as otrain
+    from paper_2411_00288_b200 import api
+    inp = synth.make_inputs(spec, x_only=True)
+    tr = synth.make_train_inputs(spec)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    dw = api.ssconv_wgrad(api.desc_from_spec(spec), inp.x.to(DEV), tr.dy.to(DEV), dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = otrain.wgrad_f64(synth.bf16_bits(inp.x), synth.bf16_bits(tr.dy), spec.KH, spec.KW, spec.stride, spec.pad,
+                           spec.dil)
+    got = dw.cpu().numpy().astype(np.float64)
+    assert got.shape == ref.shape
+    scale = max(float(np.abs(ref).max()), 1e-30)
+    rel = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30))
+    assert rel <= 1e-4 and float(np.abs(got - ref).max()) <= 2e-4 * scale, (_tid(spec), rel)
+
+
+@pytest.mark.parametrize("spec", DG_CASES, ids=[_tid(s) for s in DG_CASES])
+def test_random_shape_input_gradient_matches_oracle(spec):
+    """dL/dx of Eq. 4 in one call (residue classes of the input position for strided layers), with sentinel
+    bands around the gradient and the workspace."""
+    from oracle import train as otrain
+    from paper_2411_00288_b200 import api
+    g = torch.Generator().manual_seed(synth.SEED_BASE + 5200 + spec.index)
+    w = (torch.randn((spec.C_out, spec.KH, spec.KW, spec.C_in), generator=g) * (2.0 / spec.K) ** 0.5).to(torch.bfloat16)
+    dy = torch.randn((spec.N, spec.H_out, spec.W_out, spec.C_out), generator=g).to(torch.bfloat16)
+    desc = api.make_desc(spec.N, spec.H, spec.W, spec.C_in, spec.C_out, spec.KH, spec.KW, stride=spec.stride, pad=spec.pad,
+                         dil=spec.dil)
+    band = 2048
+    n_dx = spec.N * spec.H * spec.W * spec.C_in
+    buf = torch.full((n_dx + 2 * band,), -7.0, dtype=torch.bfloat16, device=DEV)
+    dx = buf[band:band + n_dx].view(spec.N, spec.H, spec.W, spec.C_in)
+    need = api.ssconv_dgrad_ws_bytes(desc)
+    wsbuf = torch.full((need + 2 * band,), 0x5A, dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    api.ssconv_dgrad(desc, dy.to(DEV), w.to(DEV), dx=dx, ws=wsbuf[band:band + need], dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert bool((buf[:band] == -7.0).all()) and bool((buf[-band:] == -7.0).all())
+    assert bool((wsbuf[:band] == 0x5A).all()) and bool((wsbuf[-band:] == 0x5A).all())
+    ref = otrain.dgrad_f64(synth.bf16_bits(dy), parity.bf16_tensor_to_f64(w), spec.H, spec.W, spec.stride, spec.pad, spec.dil)
+    rel, mx = parity.errors(parity.bf16_tensor_to_f64(dx), ref)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL * max(1.0, float(np.abs(ref).max()) / 4.0), (_tid(spec), rel, mx)

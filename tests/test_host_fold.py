@@ -61,5 +61,9 @@ def test_input_gradient_scratch_size():
     # 1x1 stride 2: one class with a tap, its own convolution: weights [64, 1, 1, 128], tensor [2, 7, 7, 64]
     d = api.make_desc(2, 14, 14, 64, 128, 1, 1, 2, 0)
     assert api.ssconv_dgrad_ws_bytes(d) == r256(64 * 128 * 2) + r256(2 * 7 * 7 * 64 * 2) + fwd
+    # strided and dilated: the plain route: reversed weights [64, 3, 3, 64] + dy spread over all 9 x 9 filter
+    # placements of unit stride (H + 2 pad - dil (K - 1) = 9) + the convolution's scratch
+    d = api.make_desc(1, 9, 9, 64, 64, 3, 3, 2, 2, 2)
+    assert api.ssconv_dgrad_ws_bytes(d) == r256(64 * 9 * 64 * 2) + r256(9 * 9 * 64 * 2) + fwd
     with pytest.raises(api.SsconvError):
-        api.ssconv_dgrad_ws_bytes(api.make_desc(1, 9, 9, 64, 64, 3, 3, 2, 2, 2))   # strided and dilated
+        api.ssconv_dgrad_ws_bytes(api.make_desc(1, 8, 8, 64, 64, 1, 1, 1, 1))      # padding beyond the filter's reach
