@@ -178,3 +178,52 @@ def test_forward_fp8_argument_rules():
     with pytest.raises(api.SsconvError) as e:
         api.ssconv_sizes_fp8(odd)
     assert e.value.status == 3
+
+
+def _draw_fp8_cases(count=20, seed=2411_00291):
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < count:
+        K = int(rng.choice([1, 1, 2, 3, 3, 5]))
+        d = int(rng.choice([1, 1, 2]))
+        s = int(rng.choice([1, 1, 2, 3]))
+        p = int(rng.integers(0, d * (K - 1) + 1))
+        N, H, W = int(rng.integers(1, 4)), int(rng.integers(1, 33)), int(rng.integers(1, 33))
+        Ci = int(rng.choice([16, 32, 48, 64, 80, 128, 144, 192, 256, 320]))
+        Co = int(rng.choice([8, 24, 64, 72, 128, 136, 200, 256, 264]))
+        if H + 2 * p < d * (K - 1) + 1 or W + 2 * p < d * (K - 1) + 1:
+            continue
+        Ho, Wo = (H + 2 * p - d * (K - 1) - 1) // s + 1, (W + 2 * p - d * (K - 1) - 1) // s + 1
+        if N * Ho * Wo * Co * K * K * Ci > 3e8:
+            continue
+        cases.append((f"f8r{len(cases)}_{N}x{H}x{W}x{Ci}to{Co}_k{K}s{s}p{p}d{d}", N, H, W, Ci, Co, K, s, p, d))
+    return cases
+
+
+FP8_RANDOM = _draw_fp8_cases()
+
+
+@pytest.mark.parametrize("case", FP8_RANDOM, ids=[c[0] for c in FP8_RANDOM])
+@pytest.mark.parametrize("sparse", [True, False], ids=["sparse", "dense"])
+def test_forward_fp8_on_drawn_shapes_matches_oracle(case, sparse):
+    """The same check on a seeded draw of shapes (channel tails of 16 to 112, ragged output channels, strides,
+    dilations, paddings) nobody picked by hand."""
+    desc, shape, x, w, bias, out_scale = _fp8_case(case)
+    xd, wd, bd = torch.from_numpy(x).to(DEV), torch.from_numpy(w).to(DEV), torch.from_numpy(bias).to(DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    mask = None
+    if sparse:
+        pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_E4M3, wd, w.size // 4)
+        pat_ref = masks.select_from_magnitude(None, magnitudes=fp8.abs_code(w))
+        assert np.array_equal(pat.cpu().numpy(), pat_ref)
+        mask = masks.mask_from_pattern(pat_ref, w.shape)
+        w_comp, meta = api.ssconv_compress_fp8(desc, wd, pat)
+        y = api.ssconv_forward_fp8(desc, xd, w_comp, meta, bd, out_scale, dev_status=status)
+    else:
+        y = api.ssconv_forward_dense_fp8(desc, xd, wd, bd, out_scale, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    acc = conv2d_f64(shape, fp8.e4m3_to_bf16_bits(x), fp8.e4m3_to_bf16_bits(w), mask=mask, bias=None)
+    ref = np.maximum(acc * np.float64(np.float32(out_scale)) + bias.astype(np.float64), 0.0)
+    rel, mx = parity.errors(parity.bf16_tensor_to_f64(y), ref)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"{case[0]} sparse={sparse}: rel={rel:.3e} max={mx:.3e}"

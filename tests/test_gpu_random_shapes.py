@@ -135,3 +135,75 @@ def test_random_shape_input_gradient_matches_oracle(spec):
     ref = otrain.dgrad_f64(synth.bf16_bits(dy), parity.bf16_tensor_to_f64(w), spec.H, spec.W, spec.stride, spec.pad, spec.dil)
     rel, mx = parity.errors(parity.bf16_tensor_to_f64(dx), ref)
     assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL * max(1.0, float(np.abs(ref).max()) / 4.0), (_tid(spec), rel, mx)
+
+
+# ---------------------------------------------------------------- pooling, depthwise convolution, layer norm
+def _draw_block_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        K = int(rng.choice([2, 3, 3, 5, 7, 7]))
+        s = int(rng.choice([1, 1, 1, 2, 3]))
+        d = int(rng.choice([1, 1, 1, 2]))
+        p = int(rng.integers(0, (K - 1) * d + 1))
+        N, H, W = int(rng.integers(1, 4)), int(rng.integers(1, 30)), int(rng.integers(1, 30))
+        C = int(rng.choice([8, 24, 32, 40, 64, 96, 160, 192, 200, 384]))
+        if H + 2 * p < d * (K - 1) + 1 or W + 2 * p < d * (K - 1) + 1:
+            continue
+        out.append((N, H, W, C, K, s, p, d))
+    return out
+
+
+DW_CASES = _draw_block_cases(30, 2411_00292)
+
+
+@pytest.mark.parametrize("case", DW_CASES, ids=[f"dw{i}_" + "x".join(map(str, c[:4])) + f"_k{c[4]}s{c[5]}p{c[6]}d{c[7]}"
+                                                 for i, c in enumerate(DW_CASES)])
+def test_random_shape_depthwise_matches_oracle(case):
+    """Channel counts on both sides of the tile kernel's rule (multiples of 32), filters with and without a
+    specialised kernel, strides and dilations (the generic kernel), maps smaller than one tile."""
+    from oracle import blocks
+    from oracle.conv import ConvShape
+    from paper_2411_00288_b200 import api
+    N, H, W, C, K, s, p, d = case
+    g = torch.Generator().manual_seed(synth.SEED_BASE + 5300 + DW_CASES.index(case))
+    x = torch.randn((N, H, W, C), generator=g).to(torch.bfloat16)
+    w = (torch.randn((K, K, C), generator=g) / K).to(torch.bfloat16)
+    bias = torch.randn((C,), generator=g) * 0.1
+    relu = bool(DW_CASES.index(case) % 3 == 0)
+    desc = api.make_desc(N, H, W, C, C, K, K, s, p, d, bias=True, relu=relu)
+    Ho, Wo = api.ssconv_out_shape(desc)
+    band = 256
+    buf = torch.full((N * Ho * Wo * C + 2 * band,), -5.0, dtype=torch.bfloat16, device=DEV)
+    y = buf[band:band + N * Ho * Wo * C].view(N, Ho, Wo, C)
+    api.ssconv_depthwise(desc, x.to(DEV), w.to(DEV), bias.to(DEV), y=y)
+    torch.cuda.synchronize()
+    assert bool((buf[:band] == -5.0).all()) and bool((buf[-band:] == -5.0).all())
+    shape = ConvShape(N, H, W, C, C, K, K, (s, s), (p, p), (d, d), relu=False)
+    ref = blocks.depthwise_conv2d_f64(shape, synth.bf16_bits(x), synth.bf16_bits(w), bias=bias.numpy())
+    if relu:
+        ref = np.maximum(ref, 0.0)
+    rel, mx = parity.errors(parity.bf16_tensor_to_f64(y), ref)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, (case, rel, mx)
+
+
+@pytest.mark.parametrize("pixels,C", [(1, 8), (37, 24), (301, 40), (77, 96), (64, 104), (129, 192), (50, 264), (33, 384),
+                                      (19, 768), (7, 1024), (11, 1032), (23, 20), (5, 1048)])
+def test_layernorm_over_channel_counts_matches_oracle(pixels, C):
+    """Every lane grouping of the vector kernel (1 to 32 lanes per pixel, one to four pieces per lane, idle lanes
+    and none), a pixel count that leaves a warp partly filled, and channel counts only the scalar kernel takes."""
+    from oracle import blocks
+    from paper_2411_00288_b200 import api
+    g = torch.Generator().manual_seed(synth.SEED_BASE + 5400 + C)
+    x = (torch.randn((pixels, C), generator=g) * 2 + 0.5).to(torch.bfloat16)
+    gamma, beta = torch.randn((C,), generator=g) * 0.5 + 1.0, torch.randn((C,), generator=g) * 0.2
+    band = 128
+    buf = torch.full((pixels * C + 2 * band,), -5.0, dtype=torch.bfloat16, device=DEV)
+    y = buf[band:band + pixels * C].view(pixels, C)
+    api.ssconv_layernorm(x.to(DEV), gamma.to(DEV), beta.to(DEV), 1e-6, y=y)
+    torch.cuda.synchronize()
+    assert bool((buf[:band] == -5.0).all()) and bool((buf[-band:] == -5.0).all())
+    ref = blocks.layernorm_f64(parity.bf16_tensor_to_f64(x), gamma.numpy(), beta.numpy(), 1e-6)
+    got = parity.bf16_tensor_to_f64(y)
+    # fp32 statistics and one rounding to bf16
+    assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-3), float(np.abs(got - ref).max())
