@@ -41,12 +41,20 @@ def test_select_empty_input_is_a_noop():
     assert out.numel() == 0
 
 
+def _drawn_weight_shapes(count=12, seed=2411_00293):
+    """A seeded draw of weight shapes nobody picked by hand: non-square filters, channel counts with tails of 8
+    to 56 in the last 64-channel chunk, output channels on both sides of one tile of 128."""
+    rng = np.random.default_rng(seed)
+    return [(int(rng.choice([8, 24, 72, 128, 136, 200, 264])), int(rng.integers(1, 6)), int(rng.integers(1, 6)),
+             int(rng.choice([8, 16, 40, 64, 72, 104, 120, 192, 200, 328]))) for _ in range(count)]
+
+
 @pytest.mark.parametrize("shape", [
     (64, 3, 3, 64),     # config-1 layer: padded rows (64 -> 128) and an odd number of k-blocks
     (136, 1, 1, 96),    # ragged C_out, C_in not a multiple of 64
     (256, 3, 3, 128),
     (8, 2, 3, 8),       # smallest legal channel counts
-])
+] + _drawn_weight_shapes())
 def test_compress_roundtrip_bit_exact(shape):
     Co, KH, KW, Ci = shape
     rng = np.random.default_rng(Co * 1000 + Ci)
