@@ -100,3 +100,43 @@ def test_bounded_wait_runs_out_returns_a_status_and_leaves_the_context_usable():
     assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL
     with pytest.raises(api.SsconvError):
         api.ssconv_selftest_wait_timeout(10, status)       # limit below the accepted range
+
+
+def test_calls_on_two_streams_with_their_own_scratch_do_not_disturb_each_other():
+    """The library keeps no hidden device state between calls (the one entry point that does says so in the
+    header): two layers launched again and again on two streams that overlap on the GPU, each with its own
+    scratch and status word, give bit for bit what they give alone.  A K-split layer (scratch + finishing
+    kernel) on one stream, a layer for the thread-block-pair kernel on the other."""
+    specs = [synth.LayerSpec("deep_k_split", 2, 7, 7, 512, 128, 3, 3, 1, 1, 1, config=14, index=0),
+             synth.LayerSpec("pair_3x3", 8, 14, 14, 256, 256, 3, 3, 1, 1, 1, config=14, index=1)]
+    ctx = []
+    for spec in specs:
+        inp = synth.make_inputs(spec)
+        desc = api.desc_from_spec(spec)
+        w = inp.w.to(DEV)
+        pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
+        w_comp, meta = api.ssconv_compress(desc, w, pat)
+        ws = torch.empty((api.ssconv_sizes(desc).ws_bytes_sparse,), dtype=torch.uint8, device=DEV)
+        ctx.append(dict(desc=desc, x=inp.x.to(DEV), w_comp=w_comp, meta=meta, bias=inp.bias.to(DEV), ws=ws,
+                        status=torch.zeros(1, dtype=torch.int32, device=DEV), stream=torch.cuda.Stream(device=DEV)))
+    torch.cuda.synchronize()
+
+    def run(c, y):
+        api.ssconv_forward(c["desc"], c["x"], c["w_comp"], c["meta"], c["bias"], y=y, ws=c["ws"], dev_status=c["status"],
+                           stream=c["stream"])
+
+    alone = []
+    for c in ctx:
+        y = torch.empty((c["desc"].N, *api.ssconv_out_shape(c["desc"]), c["desc"].C_out), dtype=torch.bfloat16, device=DEV)
+        run(c, y)
+        torch.cuda.synchronize()
+        alone.append(y.clone())
+    outs = [[torch.empty_like(a) for _ in range(12)] for a in alone]
+    for it in range(12):
+        for c, o in zip(ctx, outs):
+            run(c, o[it])
+    torch.cuda.synchronize()
+    for c, a, o in zip(ctx, alone, outs):
+        assert int(c["status"].item()) == 0
+        for y in o:
+            assert torch.equal(y, a)
