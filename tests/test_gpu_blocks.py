@@ -31,7 +31,25 @@ GROUPED = [  # N, H, W, C_in, C_out, K, stride, pad, groups
 ]
 
 
-@pytest.mark.parametrize("case", GROUPED, ids=[f"g{c[8]}_{c[3]}to{c[4]}_k{c[5]}" for c in GROUPED])
+def _drawn_grouped(count=10, seed=2411_00294):
+    """A seeded draw on top of the list above: 2 to 6 groups, 8 to 72 input and 8 to 136 output channels per group."""
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        groups = int(rng.choice([2, 3, 4, 6]))
+        ci, co = int(rng.choice([8, 16, 24, 40, 64, 72])), int(rng.choice([8, 16, 40, 64, 72, 136]))
+        K = int(rng.choice([1, 3, 3, 5]))
+        s = int(rng.choice([1, 1, 2]))
+        p = int(rng.integers(0, K))
+        N, H, W = int(rng.integers(1, 4)), int(rng.integers(5, 20)), int(rng.integers(5, 20))
+        out.append((N, H, W, groups * ci, groups * co, K, s, p, groups))
+    return out
+
+
+GROUPED = GROUPED + _drawn_grouped()
+
+
+@pytest.mark.parametrize("case", GROUPED, ids=[f"g{c[8]}_{c[3]}to{c[4]}_k{c[5]}s{c[6]}p{c[7]}_{c[1]}x{c[2]}" for c in GROUPED])
 @pytest.mark.parametrize("sparse", [True, False], ids=["sparse", "dense"])
 def test_grouped_convolution_matches_oracle(case, sparse):
     N, H, W, Ci, Co, K, s, p, groups = case
