@@ -109,7 +109,10 @@ int32_t ssconv_plan(const ssconv_desc_t* desc, int32_t sparse, int32_t* tile_pos
  * ssconv_wgrad choose into how many position ranges it cuts a layer (default), otherwise an upper limit
  * (ssconv_wgrad_ws_bytes follows).  SSCONV_TUNE_WGRAD_PAIR: as SSCONV_TUNE_PAIR, for ssconv_wgrad.
  * SSCONV_TUNE_RESIDENT_WEIGHTS: 1 (default) keeps the weights of dense layers with one channel tile and
- * at most four k-blocks in shared memory, 0 sends them through the ring like every other layer's.  Not
+ * at most four k-blocks in shared memory, 0 sends them through the ring like every other layer's.
+ * SSCONV_TUNE_PAIR_TILES: -1 lets the planner choose (default) whether a work item of the pair kernel is two
+ * neighbouring position tiles that share every group's weights, 0 never, 1 wherever the ring still holds two
+ * groups (tiles of at most 192 positions keep three).  Not
  * thread-safe against concurrent calls.  Returns SSCONV_ERR_BAD_DESC for an unknown option or a value
  * out of range. */
 enum {
@@ -117,7 +120,8 @@ enum {
   SSCONV_TUNE_PAIR = 2,
   SSCONV_TUNE_WGRAD_RANGES = 3,
   SSCONV_TUNE_WGRAD_PAIR = 4,
-  SSCONV_TUNE_RESIDENT_WEIGHTS = 5
+  SSCONV_TUNE_RESIDENT_WEIGHTS = 5,
+  SSCONV_TUNE_PAIR_TILES = 6
 };
 int32_t ssconv_tune(int32_t option, int32_t value);
 

@@ -266,12 +266,13 @@ def ssconv_plan(desc: Desc, sparse: bool = True) -> dict:
                 pair=bool(out[4].value))
 
 
-TUNE_TILE_POSITIONS, TUNE_PAIR, TUNE_WGRAD_RANGES, TUNE_WGRAD_PAIR, TUNE_RESIDENT_WEIGHTS = 1, 2, 3, 4, 5
+TUNE_TILE_POSITIONS, TUNE_PAIR, TUNE_WGRAD_RANGES, TUNE_WGRAD_PAIR, TUNE_RESIDENT_WEIGHTS, TUNE_PAIR_TILES = 1, 2, 3, 4, 5, 6
 
 
 def ssconv_tune(option: int, value: int) -> None:
     """Process-wide planner override: TUNE_TILE_POSITIONS (0 = automatic, or a multiple of 16 in [48, 240]),
-    TUNE_PAIR (-1 automatic, 0 never, 1 wherever thread-block pairs apply)."""
+    TUNE_PAIR (-1 automatic, 0 never, 1 wherever thread-block pairs apply), TUNE_PAIR_TILES (-1 automatic, 0 one
+    position tile per work item of the pair kernel, 1 two wherever they fit), the others as the header says."""
     f = lib().ssconv_tune
     f.restype = ctypes.c_int32
     f.argtypes = [ctypes.c_int32, ctypes.c_int32]

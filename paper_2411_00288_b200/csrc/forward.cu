@@ -111,6 +111,7 @@ struct FwdParams {
   int m_tiles, num_tiles;   // (pair kernel: m_tiles counts pairs of 128-channel tiles, m_real the tiles themselves)
   int m_real;
   int a_tiles;              // pairs of k-blocks (groups) per output tile
+  int dual;                 // pair kernel: a work item is two neighbouring position tiles sharing the group's weights
   int split;                // 1: units dealt out evenly across CTAs (stream-K); 0: whole tiles per CTA
   int work_quot, work_rem;  // work items per CTA: quotient and remainder of (tiles or units) / grid
   float out_scale;          // 8-bit operands: factor applied to the accumulators before the bias
@@ -1025,7 +1026,8 @@ __device__ __forceinline__ void pair_producer_role(const CUtensorMap* tm_a, cons
   using C = Cfg<SPARSE, FP8>;
   constexpr int kKb = C::kKbChannels;
   const uint32_t half_bytes = (uint32_t)(p.BN >> 1) * 128u;  // this CTA's half of an activation tile
-  const uint32_t grp_bytes = C::kAGroupBytes + 2u * half_bytes;
+  const uint32_t tiles_per = p.dual ? 2u : 1u;                // position tiles per work item
+  const uint32_t grp_bytes = C::kAGroupBytes + 2u * tiles_per * half_bytes;
   const bool leader = rank == 0;
   uint32_t g = 0, ph = 0;
   bool ok = true;
@@ -1033,12 +1035,17 @@ __device__ __forceinline__ void pair_producer_role(const CUtensorMap* tm_a, cons
   WorkIter work(p, pair);
   Segment seg;
   while (ok && work.next(seg)) {
-    const int pt = seg.tile / p.m_tiles;  // (m_tiles counts pairs of 128-channel tiles here)
-    const int m = 2 * (seg.tile - pt * p.m_tiles) + (int)rank;
+    const int pu = seg.tile / p.m_tiles;  // (m_tiles counts pairs of 128-channel tiles here)
+    const int pt = pu * (int)tiles_per;   // the item's first position tile
+    const int m = 2 * (seg.tile - pu * p.m_tiles) + (int)rank;
     const int m_meta = m < p.m_real ? m : p.m_real - 1;  // a CTA beyond the last channel tile multiplies zeros
     const Pos q0 = decode_pos(pt * p.BN + (int)rank * (p.BN >> 1), p.Wo, p.Ho);
     const int base_w = q0.c * p.stride_w - p.pad_w;
     const int base_h = q0.r * p.stride_h - p.pad_h;
+    // second tile of the item (a tile past the last position reads zeros: its pixels lie outside the tensor)
+    const Pos q1 = decode_pos((pt + 1) * p.BN + (int)rank * (p.BN >> 1), p.Wo, p.Ho);
+    const int base_w1 = q1.c * p.stride_w - p.pad_w;
+    const int base_h1 = q1.r * p.stride_h - p.pad_h;
     TapIter it;
     it.init(ROLE == kRoleActSecond ? 1 : 0, p);
     if (first_segment) {
@@ -1063,9 +1070,12 @@ __device__ __forceinline__ void pair_producer_role(const CUtensorMap* tm_a, cons
           it.advance(p);
         }
       } else if (ROLE == kRoleActFirst || has_second) {
-        if (leader) mbar_expect_tx_w(full0_local + 8u * g, 2u * half_bytes);
-        tma2_load_im2col_4d_w(dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? half_bytes : 0u), tm_b, full,
-                              it.cc * kKb, base_w, base_h, q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
+        if (leader) mbar_expect_tx_w(full0_local + 8u * g, 2u * tiles_per * half_bytes);
+        const uint32_t b_dst = dst + C::kAGroupBytes + (ROLE == kRoleActSecond ? half_bytes : 0u);
+        tma2_load_im2col_4d_w(b_dst, tm_b, full, it.cc * kKb, base_w, base_h, q0.n, (uint16_t)it.off_w, (uint16_t)it.off_h);
+        if (p.dual)
+          tma2_load_im2col_4d_w(b_dst + 2u * half_bytes, tm_b, full, it.cc * kKb, base_w1, base_h1, q1.n,
+                                (uint16_t)it.off_w, (uint16_t)it.off_h);
         it.advance(p);
         it.advance(p);
       } else if (leader) {
@@ -1089,7 +1099,7 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t half_bytes = (uint32_t)(p.BN >> 1) * 128u;
-  const uint32_t grp_bytes = C::kAGroupBytes + 2u * half_bytes;
+  const uint32_t grp_bytes = C::kAGroupBytes + (p.dual ? 4u : 2u) * half_bytes;
   uint8_t* ring = smem;
   uint8_t* out_stage = ring + p.ring_groups * grp_bytes;
   // barrier slots: [0,4) group full (used in the leader), [4,8) group empty, [8,10) accumulator full,
@@ -1183,12 +1193,17 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
       bool ok = true;
       WorkIter work(p, pair);
       Segment seg;
+      const bool dual = p.dual != 0;
+      const uint32_t tile1_desc = 2u * half_desc;  // the item's second tile lies behind the first one's two k-blocks
       for (; ok && work.next(seg); ++tcount) {
-        const uint32_t buf = tcount & 1u;
-        const uint32_t aph = (tcount >> 1) & 1u;
+        // one accumulator per tile: alternating between the two buffers, or (two tiles per item) both at once
+        const uint32_t buf = dual ? 0u : (tcount & 1u);
+        const uint32_t aph = dual ? (tcount & 1u) : ((tcount >> 1) & 1u);
         if (!mbar_wait_bounded(&bar_acc_empty[buf], aph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
+        if (dual && !mbar_wait_bounded(&bar_acc_empty[1], aph ^ 1u, abort_flag, kWaitLimitCycles)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kAccCol1;
+        const uint32_t d_tmem1 = tmem_base + kAccCol1;
         uint32_t accumulate = 0;
         for (int a = 0; a < p.a_tiles; ++a) {
           if (!ready && !mbar_wait_a(full0 + 8u * g, ph, abort_flag, kWaitLimitCycles)) { ok = false; break; }
@@ -1209,10 +1224,13 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
             mslot ^= 1u;
             tc2_cp_128x128b_w(meta_tmem, a_lo + (kATileBytes >> 4));
             tc2_cp_128x128b_w(meta_tmem + 4u, a_lo + ((kATileBytes + (uint32_t)kMetaImageBytes) >> 4));
-            tc2_mma_f8_sparse_w(d_tmem, a_lo, b0_lo, meta_tmem, idesc, accumulate);
-            if (n0 > 1) tc2_mma_f8_sparse_w(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem + 2u, idesc, 1u);
-            if (n1 > 0) tc2_mma_f8_sparse_w(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 4u, idesc, 1u);
-            if (n1 > 1) tc2_mma_f8_sparse_w(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 6u, idesc, 1u);
+            for (uint32_t t = 0; t < (dual ? 2u : 1u); ++t) {  // (the second tile: same weights and metadata)
+              const uint32_t d = t ? d_tmem1 : d_tmem, tb = t * tile1_desc;
+              tc2_mma_f8_sparse_w(d, a_lo, b0_lo + tb, meta_tmem, idesc, accumulate);
+              if (n0 > 1) tc2_mma_f8_sparse_w(d, a_lo + 2u, b0_lo + tb + 4u, meta_tmem + 2u, idesc, 1u);
+              if (n1 > 0) tc2_mma_f8_sparse_w(d, a_lo + 4u, b1_lo + tb, meta_tmem + 4u, idesc, 1u);
+              if (n1 > 1) tc2_mma_f8_sparse_w(d, a_lo + 6u, b1_lo + tb + 4u, meta_tmem + 6u, idesc, 1u);
+            }
           } else if (SPARSE) {
             const uint32_t meta_tmem = meta_tmem0 + 4u * mslot;
             mslot ^= 1u;
@@ -1221,11 +1239,21 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
             if (n0 > 1) tc2_mma_sparse_w(d_tmem, a_lo + 2u, b0_lo + 4u, meta_tmem, idesc | 1u, 1u);
             if (n1 > 0) tc2_mma_sparse_w(d_tmem, a_lo + 4u, b1_lo, meta_tmem + 2u, idesc, 1u);
             if (n1 > 1) tc2_mma_sparse_w(d_tmem, a_lo + 6u, b1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
+            if (dual) {  // the second tile: same weights and metadata
+              const uint32_t c0_lo = b0_lo + tile1_desc, c1_lo = b1_lo + tile1_desc;
+              tc2_mma_sparse_w(d_tmem1, a_lo, c0_lo, meta_tmem, idesc, accumulate);
+              if (n0 > 1) tc2_mma_sparse_w(d_tmem1, a_lo + 2u, c0_lo + 4u, meta_tmem, idesc | 1u, 1u);
+              if (n1 > 0) tc2_mma_sparse_w(d_tmem1, a_lo + 4u, c1_lo, meta_tmem + 2u, idesc, 1u);
+              if (n1 > 1) tc2_mma_sparse_w(d_tmem1, a_lo + 6u, c1_lo + 4u, meta_tmem + 2u, idesc | 1u, 1u);
+            }
           } else {
             const uint32_t a1_lo = a_lo + (kATileBytes >> 4);
-            for (int kk = 0; kk < n0; ++kk)
-              tc2_mma_dense_w(d_tmem, a_lo + 2u * kk, b0_lo + 2u * kk, idesc, (kk > 0) ? 1u : accumulate);
-            for (int kk = 0; kk < n1; ++kk) tc2_mma_dense_w(d_tmem, a1_lo + 2u * kk, b1_lo + 2u * kk, idesc, 1u);
+            for (uint32_t t = 0; t < (dual ? 2u : 1u); ++t) {
+              const uint32_t d = t ? d_tmem1 : d_tmem, tb = t * tile1_desc;
+              for (int kk = 0; kk < n0; ++kk)
+                tc2_mma_dense_w(d, a_lo + 2u * kk, b0_lo + tb + 2u * kk, idesc, (kk > 0) ? 1u : accumulate);
+              for (int kk = 0; kk < n1; ++kk) tc2_mma_dense_w(d, a1_lo + 2u * kk, b1_lo + tb + 2u * kk, idesc, 1u);
+            }
           }
           accumulate = 1;
           tc2_commit_both_w(empty0 + 8u * g);
@@ -1235,6 +1263,7 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
           }
         }
         if (ok) tc2_commit_both_w(accf0 + 8u * buf);
+        if (ok && dual) tc2_commit_both_w(accf0 + 8u);
       }
     }
   } else {
@@ -1252,19 +1281,26 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     const uint32_t acc_empty0_leader = map_to_cta(smem_u32(bar_acc_empty), 0);
     const uint32_t st_offset = (uint32_t)(q >> 1) * kHalfPieceBytes + (uint32_t)(lane & 7) * 128u +
                                ((((uint32_t)(q & 1) * 4u + (uint32_t)(lane >> 3)) ^ (uint32_t)(lane & 7)) << 4);
-    uint32_t tcount = 0, piece_count = 0;
+    uint32_t tcount = 0, piece_count = 0, icount = 0;
+    const uint32_t tiles_per = p.dual ? 2u : 1u;
+    bool go_on = true;
     grid_dependency_wait();
     WorkIter work(p, pair);
     Segment seg;
-    for (; work.next(seg); ++tcount) {
-      const int pt = seg.tile / p.m_tiles;
-      const int m = 2 * (seg.tile - pt * p.m_tiles) + (int)rank;
-      const uint32_t buf = tcount & 1u;
-      const uint32_t aph = (tcount >> 1) & 1u;
+    for (; go_on && work.next(seg); ++icount)
+    for (uint32_t t = 0; t < tiles_per; ++t, ++tcount) {  // the item's tiles, one accumulator each
+      const int pu = seg.tile / p.m_tiles;
+      const int pt = pu * (int)tiles_per + (int)t;
+      const int m = 2 * (seg.tile - pu * p.m_tiles) + (int)rank;
+      const uint32_t buf = p.dual ? t : (icount & 1u);
+      const uint32_t aph = p.dual ? (icount & 1u) : ((icount >> 1) & 1u);
       const bool got = mbar_wait_bounded(&bar_acc_full[buf], aph, abort_flag, kWaitLimitCycles, 64);
       if (leader) my_go[tcount & 1u] = (got && *abort_flag == 0) ? 1 : 0;
       epilogue_bar_sync(grp);
-      if (my_go[tcount & 1u] == 0) break;
+      if (my_go[tcount & 1u] == 0) {
+        go_on = false;
+        break;
+      }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kAccCol1 + col_base;
       const bool real = m < p.m_real;  // (the odd CTA of the last pair may have no channels at all)
@@ -1423,10 +1459,16 @@ int32_t wgrad_set_tuning(int32_t option, int32_t value);  // (wgrad.cu)
 static int g_tune_bn = 0;
 static int g_tune_resident = 1;  // 0: weights always travel through the ring
 static int g_tune_pair = -1;  // -1: the model chooses; 0: never the pair kernel; 1: wherever it applies
+static int g_tune_pair_dual = -1;  // pair kernel, two position tiles per work item: -1 the model, 0 never, 1 always
 int32_t set_tuning(int32_t option, int32_t value) {
   if (option == SSCONV_TUNE_PAIR) {
     if (value < -1 || value > 1) return SSCONV_ERR_BAD_DESC;
     g_tune_pair = value;
+    return SSCONV_OK;
+  }
+  if (option == SSCONV_TUNE_PAIR_TILES) {
+    if (value < -1 || value > 1) return SSCONV_ERR_BAD_DESC;
+    g_tune_pair_dual = value;
     return SSCONV_OK;
   }
   if (option == SSCONV_TUNE_RESIDENT_WEIGHTS) {
@@ -1448,6 +1490,7 @@ struct Plan {
   bool split;
   double cost = 0.0;  // the model's cycles for the layer
   bool pair = false;  // 256-channel tiles on CTA pairs (ssconv_fwd_pair_kernel)
+  bool dual = false;  // ... with two position tiles per work item
 };
 template <bool SPARSE>
 static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force_split, int max_bn = kBN,
@@ -1516,6 +1559,9 @@ static int pair_ring_groups(uint32_t a_group_bytes, int BN, int kblocks) {
 constexpr double kFillBytesPerCyclePair = 48.0;
 constexpr int kPairMinKBlocks = 12;
 constexpr double kPairMinTilesPerPair = 1.25;  // counted at the widest tile
+constexpr int kPairDualMinKBlocks = 32;
+constexpr int kPairDualMaxBN = 192;
+constexpr double kPairDualGain = 0.92;         // measured 0.88-0.95 where it applies
 template <bool SPARSE>
 static Plan plan_pair(long long Q, const Geometry& geo, int workers, bool forced) {
   Plan best{0, false};
@@ -1545,6 +1591,21 @@ static Plan plan_pair(long long Q, const Geometry& geo, int workers, bool forced
     if (best.BN == 0 || cost < 0.97 * best.cost) {
       best.BN = BN;
       best.cost = cost;
+    }
+  }
+  // Two position tiles per work item (the pair's ring group then holds the weights once and both tiles'
+  // halves, one accumulator each): measured at batch 256 / 128 on the layer sets, it pays where K is deep,
+  // the layer has at least two pairs of channel tiles and about one item per pair or more (3x3 512 channels
+  // at 7x7: 37 -> 33 us; 2048 -> 512 at 7x7: 22.3 -> 21.2; 3072 -> 768 at 7x7: 24.5 -> 22.7) and costs
+  // elsewhere (one pair of channel tiles, K under 32 k-blocks, few items: 1.1-1.5x slower; the dense form
+  // never gains).  Tiles of at most 192 positions, so that the ring keeps three groups.
+  best.dual = false;
+  if (best.BN != 0 && g_tune_pair_dual != 0 && best.BN <= kPairDualMaxBN) {
+    const long long items = (((Q + best.BN - 1) / best.BN + 1) / 2) * mp_tiles;
+    const bool pays = SPARSE && geo.kblocks >= kPairDualMinKBlocks && mp_tiles >= 2 && 4 * items >= 3 * (long long)pairs;
+    if ((pays || g_tune_pair_dual == 1) && pair_ring_groups(Cfg<SPARSE>::kAGroupBytes, 2 * best.BN, geo.kblocks) >= 2) {
+      best.dual = true;
+      best.cost *= kPairDualGain;
     }
   }
   return best;
@@ -1632,11 +1693,11 @@ int32_t plan_query_sms(const ssconv_desc_t& d, bool sparse, int sm_count, int32_
   if (bn) *bn = plan.BN;
   if (pair) *pair = plan.pair ? 1 : 0;
   if (plan.pair) {
-    const long long tiles = q_tiles * ((geo.m_tiles + 1) / 2);
+    const long long tiles = (plan.dual ? (q_tiles + 1) / 2 : q_tiles) * ((geo.m_tiles + 1) / 2);  // work items
     const long long pairs = workers / 2;
     if (split) *split = 0;
     if (ctas) *ctas = (int32_t)(2 * (tiles < pairs ? tiles : pairs));
-    if (ring_groups) *ring_groups = pair_ring_groups(a_group_bytes, plan.BN, geo.kblocks);
+    if (ring_groups) *ring_groups = pair_ring_groups(a_group_bytes, plan.dual ? 2 * plan.BN : plan.BN, geo.kblocks);
     return SSCONV_OK;
   }
   const long long tiles = q_tiles * geo.m_tiles;
@@ -1721,9 +1782,13 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
                         geo.kblocks <= 4 && g_tune_resident != 0;
   const uint32_t a_grp_bytes = resident ? 0u : C::kAGroupBytes;
   const uint32_t a_res_bytes = resident ? (uint32_t)geo.stages * 2u * kATileBytes : 0u;
-  const uint32_t grp_bytes = pair ? C::kAGroupBytes + (uint32_t)BN * 128u : group_bytes(a_grp_bytes, BN);
   if (pair) stage_bufs = pair_stage_bufs(geo.kblocks);
-  int ring_groups = pair ? pair_ring_groups(C::kAGroupBytes, BN, geo.kblocks) : ring_groups_for(C::kAGroupBytes, BN, stage_bufs);
+  // pair kernel: two neighbouring position tiles per work item share every group's weights (its ring group
+  // then holds both tiles' halves) where that still leaves a ring of two groups
+  const bool dual = pair && plan.dual && pair_ring_groups(C::kAGroupBytes, 2 * BN, geo.kblocks) >= 2;
+  const uint32_t grp_bytes = pair ? C::kAGroupBytes + (dual ? 2u : 1u) * (uint32_t)BN * 128u : group_bytes(a_grp_bytes, BN);
+  int ring_groups = pair ? pair_ring_groups(C::kAGroupBytes, dual ? 2 * BN : BN, geo.kblocks)
+                         : ring_groups_for(C::kAGroupBytes, BN, stage_bufs);
   if (resident) {
     ring_groups = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(stage_bufs) - a_res_bytes) / grp_bytes);
     if (ring_groups > kMaxGroups) ring_groups = kMaxGroups;
@@ -1867,7 +1932,8 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   p.m_real = geo.m_tiles;
   p.m_tiles = pair ? (geo.m_tiles + 1) / 2 : geo.m_tiles;
   const long long q_tiles = (Q + BN - 1) / BN;
-  p.num_tiles = (int)(q_tiles * p.m_tiles);
+  p.dual = dual ? 1 : 0;
+  p.num_tiles = (int)((dual ? (q_tiles + 1) / 2 : q_tiles) * p.m_tiles);  // (work items, where they hold two tiles)
   p.a_tiles = geo.stages;
   p.flags = d.flags;
   p.bias = bias;

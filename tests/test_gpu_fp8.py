@@ -139,7 +139,8 @@ FP8_PAIR_LAYERS = [  # run with the pair kernel forced (tiles of 256 channels on
 
 
 @pytest.mark.parametrize("case", FP8_PAIR_LAYERS, ids=[c[0] for c in FP8_PAIR_LAYERS])
-def test_forward_fp8_on_thread_block_pairs_matches_oracle(case):
+@pytest.mark.parametrize("tiles_per_item", [1, 2])
+def test_forward_fp8_on_thread_block_pairs_matches_oracle(case, tiles_per_item):
     desc, shape, x, w, bias, out_scale = _fp8_case(case)
     xd, wd, bd = torch.from_numpy(x).to(DEV), torch.from_numpy(w).to(DEV), torch.from_numpy(bias).to(DEV)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
@@ -153,11 +154,16 @@ def test_forward_fp8_on_thread_block_pairs_matches_oracle(case):
     buf = torch.full((n_out + 2 * band,), -7.0, dtype=torch.bfloat16, device=DEV)
     y = buf[band:band + n_out].view(desc.N, ho, wo, desc.C_out)
     api.ssconv_tune(api.TUNE_PAIR, 1)
+    api.ssconv_tune(api.TUNE_PAIR_TILES, tiles_per_item - 1)        # 2: two position tiles share a group's weights
+    if tiles_per_item == 2:
+        api.ssconv_tune(api.TUNE_TILE_POSITIONS, 112)
     try:
         api.ssconv_forward_fp8(desc, xd, w_comp, meta, bd, out_scale, y=y, dev_status=status)
         torch.cuda.synchronize()
     finally:
         api.ssconv_tune(api.TUNE_PAIR, -1)
+        api.ssconv_tune(api.TUNE_PAIR_TILES, -1)
+        api.ssconv_tune(api.TUNE_TILE_POSITIONS, 0)
     assert int(status.item()) == 0
     assert bool((buf[:band] == -7.0).all()) and bool((buf[-band:] == -7.0).all()) and bool((y >= 0).all())
     acc = conv2d_f64(shape, fp8.e4m3_to_bf16_bits(x), fp8.e4m3_to_bf16_bits(w), mask=mask, bias=None)

@@ -22,6 +22,7 @@ def _reset_tuning():
     yield
     api.ssconv_tune(api.TUNE_PAIR, -1)
     api.ssconv_tune(api.TUNE_TILE_POSITIONS, 0)
+    api.ssconv_tune(api.TUNE_PAIR_TILES, -1)
 
 
 def _spec(name, n, h, w, cin, cout, k, stride, pad, dil=1, relu=True, gelu=False, idx=0):
@@ -108,3 +109,71 @@ def test_pair_output_guard_bands_and_determinism():
         assert bool((y >= 0).all())  # ReLU output: every element was written
         outs.append(y.clone())
     assert torch.equal(outs[0], outs[1])
+
+
+# ---- two position tiles per work item (the pair's ring group holds the weights once for both)
+@pytest.mark.parametrize("spec", SHAPES, ids=[s.name for s in SHAPES])
+@pytest.mark.parametrize("sparse", [True, False], ids=["sparse", "dense"])
+def test_pair_with_two_tiles_per_item_forced_matches_oracle(spec, sparse):
+    """The same corner shapes with two tiles per work item forced on: odd numbers of position tiles (the last
+    item's second tile lies past the last position: it reads zeros and stores nothing), items whose tiles wrap
+    images, ragged channels, every activation, both weight forms."""
+    if not sparse and spec.C_in == 8:
+        pytest.skip("dense layers with 8 input channels run in the 8-channel mode of the one-block kernel")
+    api.ssconv_tune(api.TUNE_PAIR, 1)
+    api.ssconv_tune(api.TUNE_PAIR_TILES, 1)
+    api.ssconv_tune(api.TUNE_TILE_POSITIONS, 112 if spec.index % 2 else 176)
+    plan = api.ssconv_plan(api.desc_from_spec(spec), sparse)
+    assert plan["pair"], plan
+    rel, mx = parity.check_layer(spec, DEV, sparse=sparse)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"{spec.name} {plan}: rel={rel:.3e} max={mx:.3e}"
+
+
+@pytest.mark.parametrize("bn", [64, 96, 144, 192])
+def test_pair_with_two_tiles_per_item_over_many_items(bn):
+    """Every pair works through several items (ring and accumulator phases wrap), at tile widths whose last
+    epilogue piece is short, with an odd and an even number of position tiles; bit for bit what the
+    one-tile-per-item form gives (same products, same order per tile)."""
+    for n in (40, 41):
+        spec = _spec(f"dual_bn{bn}_{n}", n, 28, 28, 128, 256, 3, 1, 1, idx=30 + n)
+        inp = synth.make_inputs(spec)
+        desc = api.desc_from_spec(spec)
+        x, w, bias = inp.x.to(DEV), inp.w.to(DEV), inp.bias.to(DEV)
+        pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
+        w_comp, meta = api.ssconv_compress(desc, w, pat)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        api.ssconv_tune(api.TUNE_PAIR, 1)
+        api.ssconv_tune(api.TUNE_TILE_POSITIONS, bn)
+        outs = []
+        for tiles in (0, 1):
+            api.ssconv_tune(api.TUNE_PAIR_TILES, tiles)
+            outs.append(api.ssconv_forward(desc, x, w_comp, meta, bias, dev_status=status))
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(outs[0], outs[1])
+        rel, mx = parity.check_layer(spec, DEV, sparse=True, sample=30000)
+        assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"bn {bn} n {n}: rel={rel:.3e} max={mx:.3e}"
+
+
+def test_two_tiles_per_item_is_the_planners_choice_only_where_it_was_measured_to_pay():
+    """Deep K, two or more pairs of channel tiles, about one item per pair: yes (ResNet-50's last stage at batch
+    256); one pair of channel tiles, a shallow K, few items or the dense form: no.  The call must then agree with
+    the same layer run one tile per item."""
+    yes = synth.LayerSpec("s4_3x3", 256, 7, 7, 512, 512, 3, 3, 1, 1, 1, config=10, index=50)
+    d = api.desc_from_spec(yes)
+    auto = api.ssconv_plan(d, True)
+    api.ssconv_tune(api.TUNE_PAIR_TILES, 0)
+    single = api.ssconv_plan(d, True)
+    api.ssconv_tune(api.TUNE_PAIR_TILES, -1)
+    assert auto["pair"] and single["pair"] and auto["tile_positions"] == single["tile_positions"]
+    assert auto["ctas"] == 144 and single["ctas"] == 148, (auto, single)     # 72 items of two tiles against 144 tiles
+    assert api.ssconv_plan(d, False)["ctas"] == 148                           # the dense form: one tile per item
+    for n, h, ci, co, k in ((256, 14, 256, 256, 3), (256, 14, 1024, 512, 1), (64, 7, 512, 512, 3)):
+        dn = api.make_desc(n, h, h, ci, co, k, k, 1, k // 2)
+        a = api.ssconv_plan(dn, True)
+        api.ssconv_tune(api.TUNE_PAIR_TILES, 0)
+        b = api.ssconv_plan(dn, True)
+        api.ssconv_tune(api.TUNE_PAIR_TILES, -1)
+        assert a == b, (a, b)
+    rel, mx = parity.check_layer(yes, DEV, sparse=True, sample=30000)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL
