@@ -1559,7 +1559,7 @@ static int pair_ring_groups(uint32_t a_group_bytes, int BN, int kblocks) {
 constexpr double kFillBytesPerCyclePair = 48.0;
 constexpr int kPairMinKBlocks = 12;
 constexpr double kPairMinTilesPerPair = 1.25;  // counted at the widest tile
-constexpr int kPairDualMinKBlocks = 32;
+constexpr int kPairDualMinKBlocks = 48;
 constexpr int kPairDualMaxBN = 192;
 constexpr double kPairDualGain = 0.92;         // measured 0.88-0.95 where it applies
 template <bool SPARSE>
@@ -1596,9 +1596,9 @@ static Plan plan_pair(long long Q, const Geometry& geo, int workers, bool forced
   // Two position tiles per work item (the pair's ring group then holds the weights once and both tiles'
   // halves, one accumulator each): measured at batch 256 / 128 on the layer sets, it pays where K is deep,
   // the layer has at least two pairs of channel tiles and about one item per pair or more (3x3 512 channels
-  // at 7x7: 37 -> 33 us; 2048 -> 512 at 7x7: 22.3 -> 21.2; 3072 -> 768 at 7x7: 24.5 -> 22.7) and costs
-  // elsewhere (one pair of channel tiles, K under 32 k-blocks, few items: 1.1-1.5x slower; the dense form
-  // never gains).  Tiles of at most 192 positions, so that the ring keeps three groups.
+  // at 7x7: 37 -> 33 us; 3072 -> 768 at 7x7: 24.5 -> 22.7; 2048 -> 512 at 7x7, 32 k-blocks: no difference in
+  // the stack) and costs elsewhere (one pair of channel tiles, 16 k-blocks, few items: 1.1-1.5x slower; the
+  // dense form never gains).  Tiles of at most 192 positions, so that the ring keeps three groups.
   best.dual = false;
   if (best.BN != 0 && g_tune_pair_dual != 0 && best.BN <= kPairDualMaxBN) {
     const long long items = (((Q + best.BN - 1) / best.BN + 1) / 2) * mp_tiles;

@@ -168,7 +168,7 @@ def test_two_tiles_per_item_is_the_planners_choice_only_where_it_was_measured_to
     assert auto["pair"] and single["pair"] and auto["tile_positions"] == single["tile_positions"]
     assert auto["ctas"] == 144 and single["ctas"] == 148, (auto, single)     # 72 items of two tiles against 144 tiles
     assert api.ssconv_plan(d, False)["ctas"] == 148                           # the dense form: one tile per item
-    for n, h, ci, co, k in ((256, 14, 256, 256, 3), (256, 14, 1024, 512, 1), (64, 7, 512, 512, 3)):
+    for n, h, ci, co, k in ((256, 14, 256, 256, 3), (256, 14, 1024, 512, 1), (64, 7, 512, 512, 3), (256, 7, 2048, 512, 1)):
         dn = api.make_desc(n, h, h, ci, co, k, k, 1, k // 2)
         a = api.ssconv_plan(dn, True)
         api.ssconv_tune(api.TUNE_PAIR_TILES, 0)
