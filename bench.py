@@ -1017,6 +1017,8 @@ def sweep_arm(args):
             pq = api.ssconv_select_mask(api.MASK_MAGNITUDE_E4M3, wq, wq.numel() // 4)
             wq_comp, metaq = api.ssconv_compress_fp8(desc, wq, pq)
             xq = [api.ssconv_quantize_e4m3(x, 1.0) for x in xs]
+        if args.pair_tiles is not None:   # the pair kernel with one (0) or two (1) position tiles per work item
+            api.ssconv_tune(api.TUNE_PAIR_TILES, args.pair_tiles)
         for i in range(args.layer_iters):
             r = i % n_sets
             if args.e4m3:
@@ -1164,6 +1166,8 @@ def main():
                     help="time one mask-learning step per layer (soft mask, dense forward, weight gradient, "
                          "choice-weight gradient) on one of the per-layer sweeps (default: the ResNet-18 sweep)")
     ap.add_argument("--e4m3", action="store_true", help="with --only-layer: launch the layer's 2:4 e4m3 form")
+    ap.add_argument("--pair-tiles", type=int, default=None, choices=[0, 1],
+                    help="with --only-layer: force one (0) or two (1) position tiles per work item of the pair kernel")
     ap.add_argument("--convnext", action="store_true",
                     help="only the ConvNeXt-T-shaped forward pass (the default line's summary_convnext_t), one GPU")
     ap.add_argument("--batch", type=int, default=None, help="images per GPU of the stack (default 256)")
