@@ -169,6 +169,8 @@ struct PieceAhead {
   int piece, pieces, a_tiles;
   bool have;
   __device__ PieceAhead(const FwdParams& p) : it(p), piece(0), pieces(p.pieces), a_tiles(p.a_tiles), have(false) {}
+  __device__ PieceAhead(const FwdParams& p, uint32_t worker)
+      : it(p, worker), piece(0), pieces(p.pieces), a_tiles(p.a_tiles), have(false) {}
   __device__ bool next(int& tile, int& piece_out) {
     while (!have || piece == pieces) {
       if (!it.next(seg)) return false;
@@ -1017,7 +1019,9 @@ __global__ void __launch_bounds__(kFinishThreads) ssconv_split_finish_kernel(con
 // of both CTAs' loads (the peer's copies signal it directly, the leader announces the sum); "empty"
 // and "accumulator full" exist in each CTA and the leader commits to both; "accumulator empty" lives
 // in the leader and counts the epilogue warps of both CTAs.  No load is multicast: each CTA fetches
-// what it needs itself.  Whole tiles only (no K split), no residual, no 8-channel mode.
+// what it needs itself.  Whole tiles only (no K split), no 8-channel mode.  RES: the fused residual, as in
+// the one-CTA kernel (each CTA prefetches the residual pieces of its own channels into four staging buffers
+// per epilogue group, on barriers of its own).
 template <bool SPARSE, int ROLE, bool FP8 = false>
 __device__ __forceinline__ void pair_producer_role(const CUtensorMap* tm_a, const CUtensorMap* tm_b,
                                                    const CUtensorMap* tm_meta, const FwdParams& p, uint32_t rank,
@@ -1089,13 +1093,15 @@ __device__ __forceinline__ void pair_producer_role(const CUtensorMap* tm_a, cons
   }
 }
 
-template <bool SPARSE, bool FP8 = false>
+template <bool SPARSE, bool FP8 = false, bool RES = false>
 __global__ void __launch_bounds__(kThreads, 1)
 ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                        const __grid_constant__ CUtensorMap tm_meta, const __grid_constant__ CUtensorMap tm_y,
-                       const __grid_constant__ CUtensorMap tm_y_tail, const FwdParams p) {
+                       const __grid_constant__ CUtensorMap tm_y_tail, const __grid_constant__ CUtensorMap tm_r,
+                       const __grid_constant__ CUtensorMap tm_r_tail, const FwdParams p) {
   using C = Cfg<SPARSE, FP8>;
   static_assert(!FP8 || SPARSE, "the pair kernel takes 8-bit operands only in the 2:4 form");
+  static_assert(!(FP8 && RES), "the residual epilogue is not built for 8-bit operands");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t half_bytes = (uint32_t)(p.BN >> 1) * 128u;
@@ -1103,13 +1109,15 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
   uint8_t* ring = smem;
   uint8_t* out_stage = ring + p.ring_groups * grp_bytes;
   // barrier slots: [0,4) group full (used in the leader), [4,8) group empty, [8,10) accumulator full,
-  // [10,12) accumulator empty (used in the leader)
+  // [10,12) accumulator empty (used in the leader), [12,20) residual piece landed (per epilogue group and
+  // staging buffer, each block its own)
   uint64_t* bars = reinterpret_cast<uint64_t*>(out_stage + staging_bytes(p.stage_bufs));
   uint64_t* bar_full = bars;
   uint64_t* bar_empty = bars + 4;
   uint64_t* bar_acc_full = bars + 8;
   uint64_t* bar_acc_empty = bars + 10;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
+  uint64_t* bar_res = bars + 12;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = abort_flag + 1;
 
@@ -1120,10 +1128,10 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
   const bool leader_cta = rank == 0;
 
   if (warp == 0) {
-    if (lane < 12) {
+    if (lane < 20) {
       // full: the leader's three producers; empty, accumulator full: one commit; accumulator empty: the
-      // epilogue warps of both CTAs
-      const uint32_t count = (lane < 4) ? 3u : (lane < 10) ? 1u : (uint32_t)(2 * 4 * kGroups);
+      // epilogue warps of both CTAs; residual: one arrival with bytes
+      const uint32_t count = (lane < 4) ? 3u : (lane < 10) ? 1u : (lane < 12) ? (uint32_t)(2 * 4 * kGroups) : 1u;
       mbar_init(&bars[lane], count);
     }
     if (lane == 0) {
@@ -1147,6 +1155,10 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     if (warp == 2) {
       prefetch_tensormap(&tm_y);
       prefetch_tensormap(&tm_y_tail);
+      if (RES) {
+        prefetch_tensormap(&tm_r);
+        prefetch_tensormap(&tm_r_tail);
+      }
     }
   }
   // both CTAs' barriers and TMEM exist before either touches the other's
@@ -1276,6 +1288,7 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     // one or two staging buffers per group (one where the K loop is long enough to hide the wait for the
     // previous piece's store, which then leaves room for another ring group)
     const bool one_buffer = p.stage_bufs == 1;
+    const uint32_t nbuf = (uint32_t)p.stage_bufs;  // 1 or 2; 4 with a residual (pieces prefetched three ahead)
     uint8_t* my_stage = out_stage + grp * p.stage_bufs * kPieceBytes;
     volatile int* my_go = epi_go + 2 * grp;
     const uint32_t acc_empty0_leader = map_to_cta(smem_u32(bar_acc_empty), 0);
@@ -1285,6 +1298,32 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
     const uint32_t tiles_per = p.dual ? 2u : 1u;
     bool go_on = true;
     grid_dependency_wait();
+    // Residual pieces come into the staging buffers by TMA, nbuf - 1 pieces ahead of the epilogue, as in the
+    // one-block kernel; each block loads its own channels' pieces on its own barriers.
+    PieceAhead ahead(p, pair);
+    auto load_residual = [&](uint32_t count) {  // leader only; count = running number of the piece to load
+      int tile_a, piece_a;
+      if (!ahead.next(tile_a, piece_a)) return;
+      const uint32_t b = count & (nbuf - 1u);
+      const uint32_t bar = smem_u32(&bar_res[4 * grp + b]);
+      const int pt_a = tile_a / p.m_tiles;
+      const int m_a = 2 * (tile_a - pt_a * p.m_tiles) + (int)rank;
+      const int q_piece = pt_a * p.BN + col_base + piece_a * kPiece;
+      if (q_piece >= p.Q || m_a >= p.m_real) {  // nothing of this piece is stored: only keep the barrier's phases in step
+        mbar_arrive_a(bar);
+        return;
+      }
+      const bool tail = (piece_a == p.pieces - 1 && p.tail_cols != kPiece);
+      const CUtensorMap* map = tail ? &tm_r_tail : &tm_r;
+      const uint32_t half_res = (uint32_t)(tail ? p.tail_cols : kPiece) * 128u;
+      const bool two = m_a * kTileM + 64 < p.C_out;
+      const uint32_t dst = smem_u32(my_stage + b * kPieceBytes);
+      mbar_expect_tx_a(bar, two ? 2u * half_res : half_res);
+      tma_load_2d_a(dst, map, bar, m_a * kTileM, q_piece);
+      if (two) tma_load_2d_a(dst + kHalfPieceBytes, map, bar, m_a * kTileM + 64, q_piece);
+    };
+    if (RES && leader)
+      for (uint32_t c = 0; c + 1 < nbuf; ++c) load_residual(c);
     WorkIter work(p, pair);
     Segment seg;
     for (; go_on && work.next(seg); ++icount)
@@ -1312,7 +1351,8 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
       }
 #pragma unroll 1
       for (int piece = 0; piece < p.pieces; ++piece, ++piece_count) {
-        uint8_t* stage = my_stage + (one_buffer ? 0u : (piece_count & 1u)) * kPieceBytes;
+        const uint32_t sbuf = RES ? (piece_count & (nbuf - 1u)) : (one_buffer ? 0u : (piece_count & 1u));
+        uint8_t* stage = my_stage + sbuf * kPieceBytes;
         uint32_t r[kPiece];
         tc_ld_piece(t_row + piece * kPiece, r);
         tc_wait_ld();
@@ -1325,19 +1365,30 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
 #pragma unroll
           for (int i = 0; i < kPiece; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * p.out_scale);
         }
-        if (one_buffer) {  // the previous piece's store has read the buffer before anyone overwrites it
+        if (!RES && one_buffer) {  // the previous piece's store has read the buffer before anyone overwrites it
           if (leader) bulk_wait_group_read0();
           epilogue_bar_sync(grp);
         }
         const uint32_t st_addr = smem_u32(stage) + st_offset;
-        if (act == kActRelu)
+        if (RES) {
+          // the residual piece has landed in this buffer (a wait that runs out raises the abort flag; the
+          // group still goes on to its barrier and stops at the next tile)
+          mbar_wait_bounded(&bar_res[4 * grp + sbuf], (piece_count >> 2) & 1u, abort_flag, kWaitLimitCycles);
+          if (act == kActRelu)
+            stage_piece<kActRelu, true>(r, bias_v, st_addr);
+          else if (act == kActGelu)
+            stage_piece<kActGelu, true>(r, bias_v, st_addr);
+          else
+            stage_piece<kActNone, true>(r, bias_v, st_addr);
+        } else if (act == kActRelu) {
           stage_piece<kActRelu, false>(r, bias_v, st_addr);
-        else if (act == kActGelu)
+        } else if (act == kActGelu) {
           stage_piece<kActGelu, false>(r, bias_v, st_addr);
-        else
+        } else {
           stage_piece<kActNone, false>(r, bias_v, st_addr);
+        }
         fence_proxy_async_smem();
-        if (leader) bulk_wait_group_read0();
+        if (leader && !RES) bulk_wait_group_read0();
         epilogue_bar_sync(grp);
         if (leader) {
           const int q_piece = pt * p.BN + col_base + piece * kPiece;
@@ -1347,6 +1398,11 @@ ssconv_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_co
             if (m * kTileM + 64 < p.C_out) tma_store_2d(map, stage + kHalfPieceBytes, m * kTileM + 64, q_piece);
           }
           bulk_commit_group();
+          if (RES) {
+            // refill the buffer the previous piece's store read: residual piece (count + nbuf - 1)
+            bulk_wait_group_read1();
+            load_residual(piece_count + nbuf - 1u);
+          }
         }
       }
     }
@@ -1543,10 +1599,13 @@ static Plan plan_layer(long long Q, const Geometry& geo, int workers, bool force
 // one buffer, which leaves room for one more ring group at the widest tiles; two otherwise.
 constexpr int kPairOneBufferKBlocks = 24;
 static int pair_stage_bufs(int kblocks) { return kblocks >= kPairOneBufferKBlocks ? 1 : 2; }
-static int pair_ring_groups(uint32_t a_group_bytes, int BN, int kblocks) {
-  const int n = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(pair_stage_bufs(kblocks))) /
+static int pair_ring_groups_with(uint32_t a_group_bytes, int BN, int stage_bufs) {
+  const int n = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(stage_bufs)) /
                       (a_group_bytes + (uint32_t)BN * 128u));
   return n > kMaxGroups ? kMaxGroups : n;
+}
+static int pair_ring_groups(uint32_t a_group_bytes, int BN, int kblocks) {
+  return pair_ring_groups_with(a_group_bytes, BN, pair_stage_bufs(kblocks));
 }
 // Plan for the pair kernel (whole tiles of 256 channels x BN positions dealt out to workers / 2
 // pairs), or BN = 0 where it does not apply.  Per k-block a CTA of a pair takes in its weights and
@@ -1620,6 +1679,7 @@ size_t workspace_bytes() { return scratch_bytes(kMaxWorkers); }
 static int g_sm_count[64] = {0};
 static bool g_attr_set[64][2][2] = {{{false}}};
 static bool g_pair_attr_set[64][2] = {{false}};
+static bool g_pair_res_attr_set[64][2] = {{false}};
 static bool g_fp8_attr_set[64][2] = {{false}};
 static bool g_pair_fp8_attr_set[64] = {false};
 
@@ -1769,6 +1829,16 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
       plan.split = false;
       plan.BN = widest_tile(C::kAGroupBytes, 4);
     }
+    // The pair kernel takes a residual too (four staging buffers per group there as well): where its model
+    // wins and the ring still holds two groups, one work item is one tile.
+    if (!FP8 && !force_split && !small_c && g_tune_pair != 0) {
+      Plan pp = plan_pair<SPARSE>(Q, geo, workers, g_tune_pair == 1);
+      if (pp.BN != 0 && pair_ring_groups_with(C::kAGroupBytes, pp.BN, 4) >= 2 &&
+          (g_tune_pair == 1 || plan.cost > kPairAdvantage * pp.cost)) {
+        pp.dual = false;
+        plan = pp;
+      }
+    }
   }
   const int BN = plan.BN;
   const int pieces = (BN / 2 + kPiece - 1) / kPiece;
@@ -1782,12 +1852,12 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
                         geo.kblocks <= 4 && g_tune_resident != 0;
   const uint32_t a_grp_bytes = resident ? 0u : C::kAGroupBytes;
   const uint32_t a_res_bytes = resident ? (uint32_t)geo.stages * 2u * kATileBytes : 0u;
-  if (pair) stage_bufs = pair_stage_bufs(geo.kblocks);
+  if (pair) stage_bufs = residual != nullptr ? 4 : pair_stage_bufs(geo.kblocks);
   // pair kernel: two neighbouring position tiles per work item share every group's weights (its ring group
   // then holds both tiles' halves) where that still leaves a ring of two groups
-  const bool dual = pair && plan.dual && pair_ring_groups(C::kAGroupBytes, 2 * BN, geo.kblocks) >= 2;
+  const bool dual = pair && plan.dual && residual == nullptr && pair_ring_groups(C::kAGroupBytes, 2 * BN, geo.kblocks) >= 2;
   const uint32_t grp_bytes = pair ? C::kAGroupBytes + (dual ? 2u : 1u) * (uint32_t)BN * 128u : group_bytes(a_grp_bytes, BN);
-  int ring_groups = pair ? pair_ring_groups(C::kAGroupBytes, dual ? 2 * BN : BN, geo.kblocks)
+  int ring_groups = pair ? pair_ring_groups_with(C::kAGroupBytes, dual ? 2 * BN : BN, stage_bufs)
                          : ring_groups_for(C::kAGroupBytes, BN, stage_bufs);
   if (resident) {
     ring_groups = (int)((kMaxSmemBytes - 1024 - kBarrierBytes - staging_bytes(stage_bufs) - a_res_bytes) / grp_bytes);
@@ -1800,6 +1870,12 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
                              (int)kMaxSmemBytes) != cudaSuccess)
       return SSCONV_ERR_CUDA;
     g_pair_attr_set[dev][SPARSE ? 1 : 0] = true;
+  }
+  if (pair && !FP8 && residual != nullptr && !g_pair_res_attr_set[dev][SPARSE ? 1 : 0]) {
+    if (cudaFuncSetAttribute(ssconv_fwd_pair_kernel<SPARSE, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kMaxSmemBytes) != cudaSuccess)
+      return SSCONV_ERR_CUDA;
+    g_pair_res_attr_set[dev][SPARSE ? 1 : 0] = true;
   }
   if (pair && FP8 && !g_pair_fp8_attr_set[dev]) {
     if (cudaFuncSetAttribute(ssconv_fwd_pair_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1981,9 +2057,13 @@ static int32_t launch_forward_impl(const ssconv_desc_t& d, const void* x, const 
   cfg.attrs = attr;
   cfg.numAttrs = pair ? 2 : 1;
   const cudaError_t launched =
-      (FP8 && pair) ? cudaLaunchKernelEx(&cfg, ssconv_fwd_pair_kernel<true, true>, tm_a, tm_b, tm_meta, tm_y, tm_y_tail, p)
+      (FP8 && pair) ? cudaLaunchKernelEx(&cfg, ssconv_fwd_pair_kernel<true, true>, tm_a, tm_b, tm_meta, tm_y, tm_y_tail, tm_r,
+                                         tm_r_tail, p)
       : FP8 ? cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, false, FP8>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p)
-      : pair ? cudaLaunchKernelEx(&cfg, ssconv_fwd_pair_kernel<SPARSE>, tm_a, tm_b, tm_meta, tm_y, tm_y_tail, p)
+      : (pair && residual != nullptr)
+          ? cudaLaunchKernelEx(&cfg, ssconv_fwd_pair_kernel<SPARSE, false, true>, tm_a, tm_b, tm_meta, tm_y, tm_y_tail, tm_r,
+                               tm_r_tail, p)
+      : pair ? cudaLaunchKernelEx(&cfg, ssconv_fwd_pair_kernel<SPARSE>, tm_a, tm_b, tm_meta, tm_y, tm_y_tail, tm_r, tm_r_tail, p)
       : residual != nullptr
           ? cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, true>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p)
           : cudaLaunchKernelEx(&cfg, ssconv_fwd_kernel<SPARSE, false>, tm_a, tm_b, tm_y, tm_y_tail, tm_r, tm_r_tail, p);

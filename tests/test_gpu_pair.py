@@ -177,3 +177,45 @@ def test_two_tiles_per_item_is_the_planners_choice_only_where_it_was_measured_to
         assert a == b, (a, b)
     rel, mx = parity.check_layer(yes, DEV, sparse=True, sample=30000)
     assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL
+
+
+# ---- the fused skip connection on pairs
+RES_SHAPES = [SHAPES[i] for i in (1, 2, 3, 5, 7, 9, 11, 12)]
+
+
+@pytest.mark.parametrize("spec", RES_SHAPES, ids=[s.name for s in RES_SHAPES])
+@pytest.mark.parametrize("sparse", [True, False], ids=["sparse", "dense"])
+def test_pair_forced_with_residual_matches_oracle(spec, sparse):
+    """y = act(bias + conv + residual) on thread-block pairs: residual pieces prefetched into four staging
+    buffers per group by each block for its own channels; odd numbers of channel tiles (a block without
+    channels only keeps its barriers in step), ragged channels, short last pieces, GELU."""
+    api.ssconv_tune(api.TUNE_PAIR, 1)
+    rel, mx = parity.check_layer(spec, DEV, sparse=sparse, residual=True)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"{spec.name}: rel={rel:.3e} max={mx:.3e}"
+
+
+@pytest.mark.parametrize("bn", [64, 112, 176, 208])
+def test_pair_with_residual_over_many_tiles_and_in_place(bn):
+    """Several tiles per pair (staging buffers and their barriers wrap many times), the residual read from the
+    output's own buffer, against the same call on one-block tiles bit for bit (same products, same order)."""
+    spec = _spec(f"pair_res_bn{bn}", 24, 28, 28, 256, 512, 1, 1, 0, idx=60)
+    inp = synth.make_inputs(spec)
+    desc = api.desc_from_spec(spec)
+    x, w, bias = inp.x.to(DEV), inp.w.to(DEV), inp.bias.to(DEV)
+    pat = api.ssconv_select_mask(api.MASK_MAGNITUDE_BF16, w, spec.G)
+    w_comp, meta = api.ssconv_compress(desc, w, pat)
+    res = parity.make_residual(spec, None).to(DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    outs = []
+    for pair in (0, 1):
+        api.ssconv_tune(api.TUNE_PAIR, pair)
+        api.ssconv_tune(api.TUNE_TILE_POSITIONS, bn)
+        y = res.clone()                       # in place: the residual is y's own buffer
+        api.ssconv_forward(desc, x, w_comp, meta, bias, y=y, dev_status=status, residual=y)
+        outs.append(y)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(outs[0], outs[1])
+    api.ssconv_tune(api.TUNE_PAIR, 1)
+    rel, mx = parity.check_layer(spec, DEV, sparse=True, sample=30000, residual=True)
+    assert rel <= parity.REL_FRO_TOL and mx <= parity.MAX_ABS_TOL, f"bn {bn}: rel={rel:.3e} max={mx:.3e}"
