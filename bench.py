@@ -44,7 +44,7 @@ MIN_REGIONS = 30       # timed regions of --steps steps each; the median is repo
 # DRAM bytes of one step of the stack at batch 256, from the ncu counters summarised in
 # profiles/bench_resnet50_stack_dram_traffic.md; valid for the kernels whose sources hash to `sources`
 # (anything else reports null: the counters would have to be taken again).
-STACK_TRAFFIC = {"batch": 256, "read": 4518215168, "write": 5833691904, "sources": "bb67cc6b3d80497a"}
+STACK_TRAFFIC = {"batch": 256, "read": 4516161792, "write": 5831267328, "sources": "97ecc4868de1270a"}
 TRAFFIC_SOURCES = ("paper_2411_00288_b200/csrc/forward.cu", "paper_2411_00288_b200/csrc/pool.cu",
                    "paper_2411_00288_b200/csrc/sm100_ptx.cuh", "paper_2411_00288_b200/csrc/layout.cuh",
                    "paper_2411_00288_b200/stack.py")
